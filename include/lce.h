@@ -1,0 +1,146 @@
+/*
+ * lce.h -- C ABI of the B200 (sm_100a) binarized 2-D convolution library.
+ *
+ * The operations are the ones the Larq Compute Engine paper defines in its
+ * Section 3.2 "Operator implementations": LceQuantize (sign + bit-pack),
+ * LceBConv2d (im2col over packed words, XOR+POPCOUNT binary GEMM, fused output
+ * transform), LceBMaxPool2d (bitwise AND) and LceDequantize.
+ *
+ * Common rules
+ *   - Unless a function says "host", every data pointer is a DEVICE pointer owned
+ *     by the caller; the library never frees or keeps it.  Buffers of one call
+ *     must not overlap.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Device-pointer entry points only enqueue work on it: they never synchronise,
+ *     never allocate and are safe to capture in a CUDA graph.
+ *   - Every function returns an lce_status.  Argument errors are detected on the
+ *     host before anything is launched; nothing is printed and nothing throws.
+ *   - Bit convention (Section 3.2, LceQuantize): a 0 bit stands for +1.0, a 1 bit
+ *     for -1.0.  Channel c of a pixel lives in word c/32, bit c%32 (least
+ *     significant bit = lowest channel).  The channel axis is padded up to a
+ *     multiple of 32 and pad bits are always 0, in activations, weights and
+ *     bit-packed outputs alike.
+ *   - Layouts are NHWC with the channel axis packed: activations
+ *     uint32 [batch][h][w][ceil(c/32)], weights uint32 [out_c][kh][kw][ceil(in_c/32)].
+ */
+#ifndef LCE_B200_H_
+#define LCE_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LCE_OK = 0,
+    LCE_ERR_INVALID_ARG = 1,    /* null pointer, non-positive extent, bad enum, empty output */
+    LCE_ERR_UNSUPPORTED = 2,    /* valid request that no kernel here implements */
+    LCE_ERR_ALIGNMENT = 3,      /* a pointer is not aligned to its element size (4 bytes) */
+    LCE_ERR_CUDA = 4,           /* the CUDA runtime reported an error at launch / copy */
+    LCE_ERR_DEVICE_TIMEOUT = 5, /* reserved: a bounded device-side wait gave up */
+    LCE_ERR_WORKSPACE = 6       /* caller's workspace is too small */
+} lce_status;
+
+/* Section 3.2, LceBConv2d: padded locations hold zero words (= +1.0, "one-padding");
+ * zero-padding is supported through a correction of the accumulator. */
+typedef enum { LCE_PAD_VALID = 0, LCE_PAD_SAME_ONE = 1, LCE_PAD_SAME_ZERO = 2 } lce_padding;
+
+/* Section 3.2, LceBConv2d: full-precision output or bit-packed output; INT32 exposes
+ * the raw accumulator (used by tests). */
+typedef enum { LCE_OUT_FLOAT32 = 0, LCE_OUT_BITPACKED = 1, LCE_OUT_INT32 = 2 } lce_out_type;
+
+/* Fused activation of the float output transform (Section 3.2; Section 5: ReLU before
+ * batch-norm in QuickNet).  Applied to the accumulator before multiplier and bias. */
+typedef enum { LCE_ACT_NONE = 0, LCE_ACT_RELU = 1 } lce_activation;
+
+/* Which kernel lce_bconv2d uses.  AUTO picks the tiled XOR/POPC kernel when it covers the
+ * shape and the direct kernel otherwise; the other values force one (tests, benchmarks). */
+typedef enum { LCE_KERNEL_AUTO = 0, LCE_KERNEL_DIRECT = 1, LCE_KERNEL_TILED = 2 } lce_kernel;
+
+const char *lce_version(void);
+const char *lce_status_string(lce_status status);
+
+/* LceQuantize (Section 3.2): out bit = (x < 0), so +0.0, -0.0 and NaN give a 0 bit.
+ *   x   fp32  [rows][channels]            (rows = batch*h*w of an NHWC tensor)
+ *   out uint32[rows][ceil(channels/32)]
+ * rows == 0 is a no-op.  Binary weights are packed with the same call on the
+ * [out_c*kh*kw][in_c] view of an OHWI float tensor (Section 3.1, weight compression). */
+lce_status lce_bitpack(const float *x, uint32_t *out, int64_t rows, int32_t channels, void *stream);
+
+/* LceDequantize (Section 3.2, footnote to LceQuantize): packed bits -> +1.0f / -1.0f.
+ *   in  uint32[rows][ceil(channels/32)]   out fp32 [rows][channels] */
+lce_status lce_unpack(const uint32_t *in, float *out, int64_t rows, int32_t channels, void *stream);
+
+/* LceBConv2d (Section 3.2).  in_c is the TRUE channel count: K = kernel_h*kernel_w*in_c. */
+typedef struct {
+    int32_t batch, in_h, in_w, in_c;
+    int32_t out_c, kernel_h, kernel_w, stride_h, stride_w;
+    int32_t padding;    /* lce_padding; SAME follows TensorFlow: out = ceil(in/stride),
+                           total pad max((out-1)*stride+k-in, 0), floor(half) before */
+    int32_t out_type;   /* lce_out_type */
+    int32_t activation; /* lce_activation; FLOAT32 output only */
+    int32_t kernel;     /* lce_kernel */
+} lce_bconv2d_desc;
+
+/* Output extent of the convolution; LCE_ERR_INVALID_ARG if the descriptor is malformed or
+ * the output would be empty. */
+lce_status lce_bconv2d_out_shape(const lce_bconv2d_desc *desc, int32_t *out_h, int32_t *out_w);
+
+/* acc[n][oh][ow][o] = sum over (ky,kx,c) of a(n, oh*s-pt+ky, ow*s-pl+kx, c) * w[o][ky][kx][c]
+ *                   = K - 2*popcount(a XOR w) over the packed words (Section 2; Section 3.2),
+ * with out-of-image taps +1 (SAME_ONE) or 0 (SAME_ZERO), then the output transform:
+ *   FLOAT32   out fp32  [batch][oh][ow][out_c]           = fmaf((float)act(acc), multiplier[o], bias[o])
+ *             (one rounding); multiplier, bias fp32[out_c] required, thresholds ignored.
+ *   BITPACKED out uint32[batch][oh][ow][ceil(out_c/32)]  bit o = (acc < thresholds[o]);
+ *             thresholds int32[out_c] required; activation must be LCE_ACT_NONE (the converter
+ *             folds it into the thresholds, Section 3.1); multiplier, bias ignored.
+ *   INT32     out int32 [batch][oh][ow][out_c]           = acc.
+ *   input   uint32[batch][in_h][in_w][ceil(in_c/32)]     weights uint32[out_c][kh][kw][ceil(in_c/32)]
+ * Pad bits of input and weights must be 0.  Errors: INVALID_ARG (null/extent/enum/missing
+ * per-channel array), ALIGNMENT, UNSUPPORTED (kernel forced to TILED on a shape it does not
+ * cover), CUDA. */
+lce_status lce_bconv2d(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
+                       const float *multiplier, const float *bias, const int32_t *thresholds,
+                       void *output, void *stream);
+
+/* Host-buffer form of lce_bconv2d, for callers whose tensors live in host memory: every data
+ * pointer is a HOST pointer (pinned memory makes the copies asynchronous); `workspace` is a
+ * DEVICE buffer of at least lce_bconv2d_host_workspace_bytes(desc) bytes that the call uses
+ * for the device copies of input, weights, per-channel arrays and output.  Copies in, runs
+ * the same kernel as lce_bconv2d, copies the output back, all on `stream`, and returns after
+ * synchronising that stream.  LCE_ERR_WORKSPACE if workspace_bytes is too small. */
+size_t lce_bconv2d_host_workspace_bytes(const lce_bconv2d_desc *desc);
+lce_status lce_bconv2d_host(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
+                            const float *multiplier, const float *bias, const int32_t *thresholds,
+                            void *output, void *workspace, size_t workspace_bytes, void *stream);
+
+/* LceBMaxPool2d (Section 3.2): max-pool of +-1 values on packed words = bitwise AND of the
+ * window's words.  padding is LCE_PAD_VALID or LCE_PAD_SAME_ONE (TensorFlow SAME; taps outside
+ * the image are skipped).
+ *   in uint32[batch][in_h][in_w][ceil(channels/32)] -> out uint32[batch][oh][ow][ceil(channels/32)] */
+lce_status lce_bmaxpool(const uint32_t *in, uint32_t *out, int32_t batch, int32_t in_h, int32_t in_w,
+                        int32_t channels, int32_t pool_h, int32_t pool_w, int32_t stride_h,
+                        int32_t stride_w, int32_t padding, void *stream);
+
+/* fp32 residual add out = a + b (one rounding), the shortcut pattern of Section 5.3
+ * (float output -> Add -> LceQuantize).  n == 0 is a no-op; out may equal a or b. */
+lce_status lce_add_f32(const float *a, const float *b, float *out, int64_t n, void *stream);
+
+/* Integer-pipe probe: runs a register/shared-memory resident loop of one instruction mix on
+ * every SM of the current device and reports how many 32-bit word operations (one XOR +
+ * POPCOUNT + accumulate of a packed word, i.e. 32 binary MACs) it retired per second.
+ * mix: 0 plain xor+popc+add, 1 3:2 carry-save, 2 9-word carry-save tree, 10 LOP3 only,
+ * 11 POPC only, 12 IADD3 only, 13 IMAD only (the last four count instructions, not word-ops),
+ * 20 mma.sync b1 xor.popc, 21 mma.sync b1 and.popc (count 32-bit word pairs).
+ * Synchronous (times itself with CUDA events on `stream`); allocates a few KB and frees them.
+ *   ops_per_second, ops_per_clock_per_sm: HOST pointers, written on success; the per-clock
+ *   figure uses the SM cycle counter read inside the kernel. */
+lce_status lce_probe_pipe(int32_t mix, int32_t iterations, double *ops_per_second,
+                          double *ops_per_clock_per_sm, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LCE_B200_H_ */

@@ -1,0 +1,14 @@
+"""B200 (sm_100a) binarized 2-D convolution: Python binding of the C-ABI CUDA library.
+
+The functions here only marshal arguments (device pointers of torch tensors, the current
+CUDA stream) into ``liblce_b200.so``; every step of the path runs in that library's
+kernels.  There is no CPU fallback: without the built library or without a CUDA device
+the calls raise.
+"""
+from .binding import (  # noqa: F401
+    ACT_NONE, ACT_RELU, KERNEL_AUTO, KERNEL_DIRECT, KERNEL_TILED, OUT_BITPACKED, OUT_FLOAT32, OUT_INT32,
+    PAD_SAME_ONE, PAD_SAME_ZERO, PAD_VALID, LceError, BConv2dDesc,
+    lce_add_f32, lce_bconv2d, lce_bconv2d_host, lce_bconv2d_host_workspace_bytes, lce_bconv2d_out_shape,
+    lce_bitpack, lce_bmaxpool, lce_probe_pipe, lce_status_string, lce_unpack, lce_version, library,
+    make_desc, pack_weights,
+)

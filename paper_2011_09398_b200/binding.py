@@ -1,0 +1,213 @@
+"""ctypes binding of include/lce.h.  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional, Tuple
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "liblce_b200.so"
+
+PAD_VALID, PAD_SAME_ONE, PAD_SAME_ZERO = 0, 1, 2
+OUT_FLOAT32, OUT_BITPACKED, OUT_INT32 = 0, 1, 2
+ACT_NONE, ACT_RELU = 0, 1
+KERNEL_AUTO, KERNEL_DIRECT, KERNEL_TILED = 0, 1, 2
+
+
+class LceError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lce_status_string(status)} (lce_status {status})")
+
+
+class BConv2dDesc(ctypes.Structure):
+    """Mirror of lce_bconv2d_desc."""
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "batch", "in_h", "in_w", "in_c", "out_c", "kernel_h", "kernel_w", "stride_h", "stride_w",
+        "padding", "out_type", "activation", "kernel")]
+
+
+_lib = None
+
+
+def library() -> ctypes.CDLL:
+    """Loads liblce_b200.so (built by paper_2011_09398_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_2011_09398_b200.build` "
+                              "(there is no fallback path)")
+        lib = ctypes.CDLL(str(_LIB_PATH))
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+        lib.lce_version.restype = ctypes.c_char_p
+        lib.lce_status_string.restype = ctypes.c_char_p
+        lib.lce_status_string.argtypes = [ctypes.c_int]
+        lib.lce_bitpack.argtypes = [vp, vp, i64, i32, vp]
+        lib.lce_unpack.argtypes = [vp, vp, i64, i32, vp]
+        lib.lce_bconv2d_out_shape.argtypes = [ctypes.POINTER(BConv2dDesc), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        lib.lce_bconv2d.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp]
+        lib.lce_bconv2d_host_workspace_bytes.restype = ctypes.c_size_t
+        lib.lce_bconv2d_host_workspace_bytes.argtypes = [ctypes.POINTER(BConv2dDesc)]
+        lib.lce_bconv2d_host.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        lib.lce_bmaxpool.argtypes = [vp, vp] + [i32] * 9 + [vp]
+        lib.lce_add_f32.argtypes = [vp, vp, vp, i64, vp]
+        lib.lce_probe_pipe.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), vp]
+        for name in ("lce_bitpack", "lce_unpack", "lce_bconv2d_out_shape", "lce_bconv2d", "lce_bconv2d_host",
+                     "lce_bmaxpool", "lce_add_f32", "lce_probe_pipe"):
+            getattr(lib, name).restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def lce_version() -> str:
+    return library().lce_version().decode()
+
+
+def lce_status_string(status: int) -> str:
+    return library().lce_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise LceError(status, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (there is no CPU path)")
+    if t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous {dtype}")
+    return t.data_ptr()
+
+
+def _words(c: int) -> int:
+    return (c + 31) // 32
+
+
+def make_desc(batch, in_h, in_w, in_c, out_c, kernel=(3, 3), stride=(1, 1), padding=PAD_SAME_ONE,
+              out_type=OUT_FLOAT32, activation=ACT_NONE, kernel_choice=KERNEL_AUTO) -> BConv2dDesc:
+    return BConv2dDesc(batch, in_h, in_w, in_c, out_c, kernel[0], kernel[1], stride[0], stride[1],
+                       padding, out_type, activation, kernel_choice)
+
+
+def lce_bconv2d_out_shape(desc: BConv2dDesc) -> Tuple[int, int]:
+    oh, ow = ctypes.c_int32(), ctypes.c_int32()
+    _check(library().lce_bconv2d_out_shape(ctypes.byref(desc), ctypes.byref(oh), ctypes.byref(ow)), "lce_bconv2d_out_shape")
+    return oh.value, ow.value
+
+
+def lce_bitpack(x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """LceQuantize: fp32 [..., C] -> int32-typed words [..., ceil(C/32)] (bit pattern of uint32)."""
+    C = x.shape[-1]
+    rows = x.numel() // C if C else 0
+    if out is None:
+        out = torch.empty(x.shape[:-1] + (_words(C),), dtype=torch.int32, device=x.device)
+    _check(library().lce_bitpack(_dev(x, torch.float32, "x"), _dev(out, torch.int32, "out"), rows, C, _stream()), "lce_bitpack")
+    return out
+
+
+def lce_unpack(words: torch.Tensor, channels: int, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """LceDequantize: words [..., ceil(C/32)] -> fp32 [..., C] of +-1.0."""
+    rows = words.numel() // _words(channels)
+    if out is None:
+        out = torch.empty(words.shape[:-1] + (channels,), dtype=torch.float32, device=words.device)
+    _check(library().lce_unpack(_dev(words, torch.int32, "words"), _dev(out, torch.float32, "out"), rows, channels, _stream()), "lce_unpack")
+    return out
+
+
+def pack_weights(w_ohwi: torch.Tensor) -> torch.Tensor:
+    """Binary weight compression: fp32/int8 +-1 weights [Cout,KH,KW,Cin] -> words [Cout,KH,KW,ceil(Cin/32)]
+    by the same LceQuantize kernel (a load-time step)."""
+    return lce_bitpack(w_ohwi.to(torch.float32).contiguous())
+
+
+def lce_bconv2d(desc: BConv2dDesc, input: torch.Tensor, weights: torch.Tensor,
+                multiplier: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+                thresholds: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """LceBConv2d on packed words; allocates `out` with torch when not given."""
+    oh, ow = lce_bconv2d_out_shape(desc)
+    if out is None:
+        if desc.out_type == OUT_FLOAT32:
+            out = torch.empty((desc.batch, oh, ow, desc.out_c), dtype=torch.float32, device=input.device)
+        elif desc.out_type == OUT_BITPACKED:
+            out = torch.empty((desc.batch, oh, ow, _words(desc.out_c)), dtype=torch.int32, device=input.device)
+        else:
+            out = torch.empty((desc.batch, oh, ow, desc.out_c), dtype=torch.int32, device=input.device)
+    expect_in = desc.batch * desc.in_h * desc.in_w * _words(desc.in_c)
+    expect_w = desc.out_c * desc.kernel_h * desc.kernel_w * _words(desc.in_c)
+    if input.numel() != expect_in or weights.numel() != expect_w:
+        raise ValueError("input / weights size does not match the descriptor")
+    out_dtype = torch.float32 if desc.out_type == OUT_FLOAT32 else torch.int32
+    _check(library().lce_bconv2d(
+        ctypes.byref(desc), _dev(input, torch.int32, "input"), _dev(weights, torch.int32, "weights"),
+        _dev(multiplier, torch.float32, "multiplier") if multiplier is not None else None,
+        _dev(bias, torch.float32, "bias") if bias is not None else None,
+        _dev(thresholds, torch.int32, "thresholds") if thresholds is not None else None,
+        _dev(out, out_dtype, "out"), _stream()), "lce_bconv2d")
+    return out
+
+
+def lce_bconv2d_host_workspace_bytes(desc: BConv2dDesc) -> int:
+    return int(library().lce_bconv2d_host_workspace_bytes(ctypes.byref(desc)))
+
+
+def _host(t: Optional[torch.Tensor], dtype, name: str):
+    if t is None:
+        return None
+    if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous host {dtype} tensor")
+    return t.data_ptr()
+
+
+def lce_bconv2d_host(desc: BConv2dDesc, input, weights, multiplier, bias, thresholds, out, workspace: torch.Tensor) -> None:
+    """Host-buffer form: all tensors on the host (pinned for asynchronous copies) except `workspace`
+    (a CUDA uint8 tensor of at least lce_bconv2d_host_workspace_bytes(desc))."""
+    out_dtype = torch.float32 if desc.out_type == OUT_FLOAT32 else torch.int32
+    _check(library().lce_bconv2d_host(
+        ctypes.byref(desc), _host(input, torch.int32, "input"), _host(weights, torch.int32, "weights"),
+        _host(multiplier, torch.float32, "multiplier"), _host(bias, torch.float32, "bias"),
+        _host(thresholds, torch.int32, "thresholds"), _host(out, out_dtype, "out"),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()), "lce_bconv2d_host")
+
+
+def lce_bmaxpool(words: torch.Tensor, channels: int, pool=(2, 2), stride=(2, 2), padding=PAD_VALID,
+                 out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """LceBMaxPool2d on packed words [N,H,W,ceil(C/32)]."""
+    N, H, W, Cw = words.shape
+    if Cw != _words(channels):
+        raise ValueError("last dimension does not match channels")
+
+    def osz(size, k, s):
+        if padding == PAD_VALID:
+            return (size - k) // s + 1 if size >= k else 0
+        return -(-size // s)
+
+    if out is None:
+        out = torch.empty((N, osz(H, pool[0], stride[0]), osz(W, pool[1], stride[1]), Cw), dtype=torch.int32, device=words.device)
+    _check(library().lce_bmaxpool(_dev(words, torch.int32, "words"), _dev(out, torch.int32, "out"), N, H, W, channels,
+                                  pool[0], pool[1], stride[0], stride[1], padding, _stream()), "lce_bmaxpool")
+    return out
+
+
+def lce_add_f32(a: torch.Tensor, b: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    if out is None:
+        out = torch.empty_like(a)
+    if a.numel() != b.numel() or a.numel() != out.numel():
+        raise ValueError("size mismatch")
+    _check(library().lce_add_f32(_dev(a, torch.float32, "a"), _dev(b, torch.float32, "b"), _dev(out, torch.float32, "out"),
+                                 a.numel(), _stream()), "lce_add_f32")
+    return out
+
+
+def lce_probe_pipe(mix: int, iterations: int = 2000) -> Tuple[float, float]:
+    """Returns (ops per second, ops per clock per SM) of one instruction mix; see lce.h."""
+    if not torch.cuda.is_available():
+        raise RuntimeError("lce_probe_pipe needs a CUDA device")
+    a, b = ctypes.c_double(), ctypes.c_double()
+    _check(library().lce_probe_pipe(mix, iterations, ctypes.byref(a), ctypes.byref(b), _stream()), "lce_probe_pipe")
+    return a.value, b.value

@@ -1,0 +1,139 @@
+// C ABI front: version/status strings, shape query and the LceBConv2d dispatch (device- and
+// host-buffer forms).  All argument checks happen here, before anything is launched.
+#include "common.cuh"
+
+namespace lce {
+namespace {
+
+lce_status check_conv_args(const lce_bconv2d_desc *desc, ConvGeom *g, const void *input, const void *weights,
+                           const void *multiplier, const void *bias, const void *thresholds, const void *output)
+{
+    lce_status st = make_geom(desc, g);
+    if (st != LCE_OK) return st;
+    if (!input || !weights || !output) return LCE_ERR_INVALID_ARG;
+    if (g->out_type == LCE_OUT_FLOAT32 && (!multiplier || !bias)) return LCE_ERR_INVALID_ARG;
+    if (g->out_type == LCE_OUT_BITPACKED) {
+        if (!thresholds) return LCE_ERR_INVALID_ARG;
+        if (g->activation != LCE_ACT_NONE) return LCE_ERR_INVALID_ARG;
+    }
+    return LCE_OK;
+}
+
+lce_status dispatch(const lce_bconv2d_desc *desc, const ConvGeom &g, const uint32_t *input, const uint32_t *weights,
+                    const float *multiplier, const float *bias, const int32_t *thresholds, void *output,
+                    cudaStream_t s)
+{
+    if (desc->kernel == LCE_KERNEL_DIRECT)
+        return launch_bconv_direct(g, input, weights, multiplier, bias, thresholds, output, s);
+    lce_status st = launch_bconv_tiled(g, input, weights, multiplier, bias, thresholds, output, s);
+    if (st == LCE_ERR_UNSUPPORTED && desc->kernel == LCE_KERNEL_AUTO)
+        st = launch_bconv_direct(g, input, weights, multiplier, bias, thresholds, output, s);
+    return st;
+}
+
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct HostLayout {
+    size_t in, w, mult, bias, thr, out, total;
+    size_t in_bytes, w_bytes, ch_bytes, out_bytes;
+};
+
+HostLayout host_layout(const ConvGeom &g)
+{
+    HostLayout L{};
+    L.in_bytes = (size_t)g.N * g.H * g.W * g.Cw * 4;
+    L.w_bytes = (size_t)g.Cout * g.KH * g.KW * g.Cw * 4;
+    L.ch_bytes = (size_t)g.Cout * 4;
+    L.out_bytes = (size_t)g.M * (g.out_type == LCE_OUT_BITPACKED ? g.Cow : g.Cout) * 4;
+    size_t off = 0;
+    L.in = off;   off += round_up(L.in_bytes, 256);
+    L.w = off;    off += round_up(L.w_bytes, 256);
+    L.mult = off; off += round_up(L.ch_bytes, 256);
+    L.bias = off; off += round_up(L.ch_bytes, 256);
+    L.thr = off;  off += round_up(L.ch_bytes, 256);
+    L.out = off;  off += round_up(L.out_bytes, 256);
+    L.total = off;
+    return L;
+}
+
+}  // namespace
+}  // namespace lce
+
+extern "C" const char *lce_version(void) { return "lce-b200 0.1 (sm_100a)"; }
+
+extern "C" const char *lce_status_string(lce_status status)
+{
+    switch (status) {
+        case LCE_OK: return "ok";
+        case LCE_ERR_INVALID_ARG: return "invalid argument";
+        case LCE_ERR_UNSUPPORTED: return "unsupported";
+        case LCE_ERR_ALIGNMENT: return "misaligned pointer";
+        case LCE_ERR_CUDA: return "CUDA error";
+        case LCE_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case LCE_ERR_WORKSPACE: return "workspace too small";
+    }
+    return "unknown status";
+}
+
+extern "C" lce_status lce_bconv2d_out_shape(const lce_bconv2d_desc *desc, int32_t *out_h, int32_t *out_w)
+{
+    lce::ConvGeom g;
+    lce_status st = lce::make_geom(desc, &g);
+    if (st != LCE_OK) return st;
+    if (!out_h || !out_w) return LCE_ERR_INVALID_ARG;
+    *out_h = g.OH;
+    *out_w = g.OW;
+    return LCE_OK;
+}
+
+extern "C" lce_status lce_bconv2d(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
+                                  const float *multiplier, const float *bias, const int32_t *thresholds,
+                                  void *output, void *stream)
+{
+    using namespace lce;
+    ConvGeom g;
+    lce_status st = check_conv_args(desc, &g, input, weights, multiplier, bias, thresholds, output);
+    if (st != LCE_OK) return st;
+    if (!aligned(input, 4) || !aligned(weights, 4) || !aligned(output, 4) ||
+        (multiplier && !aligned(multiplier, 4)) || (bias && !aligned(bias, 4)) ||
+        (thresholds && !aligned(thresholds, 4)))
+        return LCE_ERR_ALIGNMENT;
+    return dispatch(desc, g, input, weights, multiplier, bias, thresholds, output, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" size_t lce_bconv2d_host_workspace_bytes(const lce_bconv2d_desc *desc)
+{
+    lce::ConvGeom g;
+    if (lce::make_geom(desc, &g) != LCE_OK) return 0;
+    return lce::host_layout(g).total;
+}
+
+extern "C" lce_status lce_bconv2d_host(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
+                                       const float *multiplier, const float *bias, const int32_t *thresholds,
+                                       void *output, void *workspace, size_t workspace_bytes, void *stream)
+{
+    using namespace lce;
+    ConvGeom g;
+    lce_status st = check_conv_args(desc, &g, input, weights, multiplier, bias, thresholds, output);
+    if (st != LCE_OK) return st;
+    if (!workspace) return LCE_ERR_INVALID_ARG;
+    if (!aligned(workspace, 256)) return LCE_ERR_ALIGNMENT;
+    const HostLayout L = host_layout(g);
+    if (workspace_bytes < L.total) return LCE_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char *ws = static_cast<char *>(workspace);
+    bool ok = cudaMemcpyAsync(ws + L.in, input, L.in_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(ws + L.w, weights, L.w_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (multiplier) ok = ok && cudaMemcpyAsync(ws + L.mult, multiplier, L.ch_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (bias) ok = ok && cudaMemcpyAsync(ws + L.bias, bias, L.ch_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (thresholds) ok = ok && cudaMemcpyAsync(ws + L.thr, thresholds, L.ch_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (!ok) return LCE_ERR_CUDA;
+    st = dispatch(desc, g, reinterpret_cast<const uint32_t *>(ws + L.in), reinterpret_cast<const uint32_t *>(ws + L.w),
+                  multiplier ? reinterpret_cast<const float *>(ws + L.mult) : nullptr,
+                  bias ? reinterpret_cast<const float *>(ws + L.bias) : nullptr,
+                  thresholds ? reinterpret_cast<const int32_t *>(ws + L.thr) : nullptr, ws + L.out, s);
+    if (st != LCE_OK) return st;
+    if (cudaMemcpyAsync(output, ws + L.out, L.out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return LCE_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return LCE_ERR_CUDA;
+    return LCE_OK;
+}

@@ -1,0 +1,128 @@
+// LceQuantize / LceDequantize (paper Section 3.2): sign-binarize and pack 32 channels per
+// word, and the inverse.  Both are single-pass HBM streaming kernels.
+#include "common.cuh"
+
+namespace lce {
+namespace {
+
+constexpr int kPackThreads = 256;
+constexpr int kWordsPerWarpPass = 128;  // one warp turns 128x32 floats into 128 words per pass
+
+// channels % 32 == 0: the flat float array is a sequence of 32-float groups, each giving one
+// word.  A warp reads group g with one coalesced 128-byte load (lane = channel within the
+// group); __ballot_sync(x < 0) is the packed word (lane order = bit order, LSB = lowest
+// channel).  128 ballots per pass are handed out four per lane so that every lane ends up
+// with four consecutive words and writes them with one 128-bit store.
+__global__ void __launch_bounds__(kPackThreads)
+bitpack_aligned_kernel(const float *__restrict__ x, uint32_t *__restrict__ out, int64_t n_words)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * kPackThreads + threadIdx.x) >> 5;
+    const int64_t n_warps = ((int64_t)gridDim.x * kPackThreads) >> 5;
+    for (int64_t w0 = warp * kWordsPerWarpPass; w0 < n_words; w0 += n_warps * kWordsPerWarpPass) {
+        uint32_t mine[4] = {0u, 0u, 0u, 0u};
+        if (w0 + kWordsPerWarpPass <= n_words) {
+#pragma unroll
+            for (int b0 = 0; b0 < kWordsPerWarpPass; b0 += 16) {
+                float v[16];
+#pragma unroll
+                for (int u = 0; u < 16; ++u) v[u] = __ldcs(x + (w0 + b0 + u) * 32 + lane);
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    const uint32_t word = __ballot_sync(0xffffffffu, v[u] < 0.0f);
+                    const int b = b0 + u;
+                    if ((b >> 2) == lane) mine[b & 3] = word;
+                }
+            }
+            // out + w0 is 16-byte aligned: w0 is a multiple of 128 words and out is checked on the host
+            reinterpret_cast<uint4 *>(out + w0)[lane] = make_uint4(mine[0], mine[1], mine[2], mine[3]);
+        } else {  // ragged last pass of the tensor
+            for (int64_t w = w0; w < n_words; ++w) {
+                const uint32_t word = __ballot_sync(0xffffffffu, x[w * 32 + lane] < 0.0f);
+                if (lane == 0) out[w] = word;
+            }
+        }
+    }
+}
+
+// Any channel count: one thread builds one output word from its (up to 32) channels.  For a
+// small channel count (3-channel images: one word per pixel) neighbouring threads read
+// neighbouring pixels, so the loads of a warp still cover one contiguous span.
+__global__ void __launch_bounds__(kPackThreads)
+bitpack_generic_kernel(const float *__restrict__ x, uint32_t *__restrict__ out, int64_t rows, int32_t channels,
+                       int32_t words)
+{
+    const int64_t total = rows * words;
+    for (int64_t i = (int64_t)blockIdx.x * kPackThreads + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * kPackThreads) {
+        const int64_t r = i / words;
+        const int32_t j = (int32_t)(i - r * words);
+        const int32_t c0 = j * 32;
+        const int32_t nc = min(32, channels - c0);
+        const float *p = x + r * channels + c0;
+        uint32_t word = 0u;
+        for (int32_t c = 0; c < nc; ++c) word |= (p[c] < 0.0f ? 1u : 0u) << c;
+        out[i] = word;  // pad bits stay 0
+    }
+}
+
+// LceDequantize: one thread per output float.
+__global__ void __launch_bounds__(kPackThreads)
+unpack_kernel(const uint32_t *__restrict__ in, float *__restrict__ out, int64_t rows, int32_t channels,
+              int32_t words)
+{
+    const int64_t total = rows * channels;
+    for (int64_t i = (int64_t)blockIdx.x * kPackThreads + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * kPackThreads) {
+        const int64_t r = i / channels;
+        const int32_t c = (int32_t)(i - r * channels);
+        const uint32_t word = in[r * words + (c >> 5)];
+        out[i] = ((word >> (c & 31)) & 1u) ? -1.0f : 1.0f;
+    }
+}
+
+int grid_for(int64_t work_items, int per_block, int max_blocks)
+{
+    int64_t b = (work_items + per_block - 1) / per_block;
+    if (b < 1) b = 1;
+    if (b > max_blocks) b = max_blocks;
+    return (int)b;
+}
+
+}  // namespace
+}  // namespace lce
+
+extern "C" lce_status lce_bitpack(const float *x, uint32_t *out, int64_t rows, int32_t channels, void *stream)
+{
+    using namespace lce;
+    if (rows < 0 || channels <= 0) return LCE_ERR_INVALID_ARG;
+    if (rows == 0) return LCE_OK;
+    if (!x || !out) return LCE_ERR_INVALID_ARG;
+    if (!aligned(x, 4) || !aligned(out, 4)) return LCE_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int32_t words = (channels + 31) / 32;
+    const int64_t n_words = rows * words;
+    // 148 SMs x 8 resident blocks of 256 threads; grid-stride loops cover the rest
+    const int max_blocks = 148 * 8;
+    if (channels % 32 == 0 && aligned(out, 16)) {
+        const int64_t passes = (n_words + kWordsPerWarpPass - 1) / kWordsPerWarpPass;
+        bitpack_aligned_kernel<<<grid_for(passes, kPackThreads / 32, max_blocks), kPackThreads, 0, s>>>(x, out, n_words);
+    } else {
+        bitpack_generic_kernel<<<grid_for(n_words, kPackThreads, max_blocks * 4), kPackThreads, 0, s>>>(
+            x, out, rows, channels, words);
+    }
+    return launch_status();
+}
+
+extern "C" lce_status lce_unpack(const uint32_t *in, float *out, int64_t rows, int32_t channels, void *stream)
+{
+    using namespace lce;
+    if (rows < 0 || channels <= 0) return LCE_ERR_INVALID_ARG;
+    if (rows == 0) return LCE_OK;
+    if (!in || !out) return LCE_ERR_INVALID_ARG;
+    if (!aligned(in, 4) || !aligned(out, 4)) return LCE_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int32_t words = (channels + 31) / 32;
+    unpack_kernel<<<grid_for(rows * channels, kPackThreads, 148 * 32), kPackThreads, 0, s>>>(in, out, rows, channels, words);
+    return launch_status();
+}

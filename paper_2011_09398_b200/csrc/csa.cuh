@@ -1,0 +1,76 @@
+// Carry-save popcount accumulation for the binary GEMM inner loop.
+//
+// The paper's BGEMM multiplies with XOR and accumulates with POPCOUNT (Section 2, Section 3.2):
+// for one output, cnt = sum_k popc(a_k ^ w_k).  On this GPU POPC issues at a quarter of the
+// rate of the logic unit, so instead of one POPC per word the mismatch words x_k = a_k ^ w_k of
+// nine consecutive k are first compressed bitwise with full adders (3:2 carry-save counters,
+// one LOP3 per output bit-plane) into four words S, C, T, F with
+//     sum_{k<9} popc(x_k) = popc(S) + 2*popc(C) + 2*popc(T) + 4*popc(F)
+// which needs 4 POPC instead of 9.  The XORs with the weights are folded into the adders:
+// within a triple (x0,x1,x2)
+//     s = x0^x1^x2 = (a0^a1^a2) ^ (w0^w1^w2)         -- both factors are precomputed once per
+//     d = x0^x1    = (a0^a1)    ^ (w0^w1)               pixel resp. once per output channel
+//     c = maj(x0,x1,x2) = d ? ~s&... : x0  =  (d & ~s) | (~d & x0),   x0 = a0 ^ w0
+// so a triple costs 4 LOP3 per output instead of 5, and a nine-word group 16 LOP3 + 4 POPC.
+#pragma once
+#include <stdint.h>
+
+namespace lce {
+
+template <int LUT>
+__device__ __forceinline__ uint32_t lop3(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, %4;" : "=r"(r) : "r"(a), "r"(b), "r"(c), "n"(LUT));
+    return r;
+}
+__device__ __forceinline__ uint32_t xor3(uint32_t a, uint32_t b, uint32_t c) { return lop3<0x96>(a, b, c); }
+__device__ __forceinline__ uint32_t maj3(uint32_t a, uint32_t b, uint32_t c) { return lop3<0xE8>(a, b, c); }
+// carry of the triple from d = x0^x1, s = x0^x1^x2 and x0:  (d & ~s) | (~d & x0)
+__device__ __forceinline__ uint32_t carry_dsx(uint32_t d, uint32_t s, uint32_t x0) { return lop3<0x3A>(d, s, x0); }
+
+// Per-pixel (activation side) and per-channel (weight side) operands of one triple.
+struct Triple {
+    uint32_t all;    // v0 ^ v1 ^ v2
+    uint32_t pair;   // v0 ^ v1
+    uint32_t first;  // v0
+};
+
+__device__ __forceinline__ Triple make_triple(uint32_t v0, uint32_t v1, uint32_t v2)
+{
+    Triple t;
+    t.pair = v0 ^ v1;
+    t.all = t.pair ^ v2;
+    t.first = v0;
+    return t;
+}
+
+// popcount of the nine mismatch words of one (pixel, channel) pair, given the three triples of
+// each side: 16 LOP3 + 4 POPC + the weighted sum.
+__device__ __forceinline__ uint32_t popc9(const Triple (&a)[3], const Triple (&w)[3])
+{
+    uint32_t s[3], c[3];
+#pragma unroll
+    for (int g = 0; g < 3; ++g) {
+        s[g] = a[g].all ^ w[g].all;
+        const uint32_t d = a[g].pair ^ w[g].pair;
+        const uint32_t x0 = a[g].first ^ w[g].first;
+        c[g] = carry_dsx(d, s[g], x0);
+    }
+    const uint32_t S = xor3(s[0], s[1], s[2]);  // weight 1
+    const uint32_t C = maj3(s[0], s[1], s[2]);  // weight 2
+    const uint32_t T = xor3(c[0], c[1], c[2]);  // weight 2
+    const uint32_t F = maj3(c[0], c[1], c[2]);  // weight 4
+    return __popc(S) + 2u * (__popc(C) + __popc(T)) + 4u * __popc(F);
+}
+
+// popcount of one triple alone (used for K tails and by the 3:2 probe): 4 LOP3 + 2 POPC.
+__device__ __forceinline__ uint32_t popc3(const Triple &a, const Triple &w)
+{
+    const uint32_t s = a.all ^ w.all;
+    const uint32_t d = a.pair ^ w.pair;
+    const uint32_t x0 = a.first ^ w.first;
+    return __popc(s) + 2u * __popc(carry_dsx(d, s, x0));
+}
+
+}  // namespace lce

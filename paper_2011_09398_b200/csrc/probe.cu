@@ -1,0 +1,240 @@
+// Integer-pipe probes: register-resident loops of the candidate instruction mixes of the binary
+// GEMM inner loop (paper Section 3.2 and its Table 1 count instructions per binary MAC on a
+// Cortex-A76; this is the same exercise on an SM).  The rates measured here are the compute
+// ceilings the convolution kernel is judged against.
+#include "common.cuh"
+#include "csa.cuh"
+
+namespace lce {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int PX = 2;   // pixels per thread in the mix probes
+constexpr int CH = 8;   // output channels per thread
+
+// Makes the compiler treat a register as changed without emitting an instruction, so that the
+// loop body cannot be hoisted.
+__device__ __forceinline__ void touch(uint32_t &v) { asm volatile("" : "+r"(v)); }
+
+template <int MIX>
+__global__ void __launch_bounds__(kThreads)
+probe_mix_kernel(const uint32_t *__restrict__ seed, uint32_t *__restrict__ sink, long long *__restrict__ cycles,
+                 int iterations)
+{
+    uint32_t a[PX][9], w[CH][9];
+    uint32_t acc[PX][CH];
+#pragma unroll
+    for (int p = 0; p < PX; ++p)
+#pragma unroll
+        for (int t = 0; t < 9; ++t) a[p][t] = seed[(threadIdx.x * 31 + p * 9 + t) & 1023];
+#pragma unroll
+    for (int j = 0; j < CH; ++j)
+#pragma unroll
+        for (int t = 0; t < 9; ++t) w[j][t] = seed[(threadIdx.x * 17 + j * 9 + t + 512) & 1023];
+#pragma unroll
+    for (int p = 0; p < PX; ++p)
+#pragma unroll
+        for (int j = 0; j < CH; ++j) acc[p][j] = 0;
+
+    // weight-side triples are loop invariant in the real kernel too (they come from shared memory)
+    Triple wt[CH][3];
+#pragma unroll
+    for (int j = 0; j < CH; ++j)
+#pragma unroll
+        for (int g = 0; g < 3; ++g) wt[j][g] = make_triple(w[j][3 * g], w[j][3 * g + 1], w[j][3 * g + 2]);
+
+    __syncthreads();
+    const long long t0 = clock64();
+    for (int it = 0; it < iterations; ++it) {
+#pragma unroll
+        for (int p = 0; p < PX; ++p) {
+#pragma unroll
+            for (int t = 0; t < 9; ++t) touch(a[p][t]);
+            if (MIX == 0) {
+#pragma unroll
+                for (int j = 0; j < CH; ++j)
+#pragma unroll
+                    for (int t = 0; t < 9; ++t) acc[p][j] += __popc(a[p][t] ^ w[j][t]);
+            } else {
+                Triple at[3];
+#pragma unroll
+                for (int g = 0; g < 3; ++g) at[g] = make_triple(a[p][3 * g], a[p][3 * g + 1], a[p][3 * g + 2]);
+#pragma unroll
+                for (int j = 0; j < CH; ++j) {
+                    if (MIX == 1) {
+#pragma unroll
+                        for (int g = 0; g < 3; ++g) acc[p][j] += popc3(at[g], wt[j][g]);
+                    } else {
+                        acc[p][j] += popc9(at, wt[j]);
+                    }
+                }
+            }
+        }
+    }
+    const long long t1 = clock64();
+    uint32_t x = 0;
+#pragma unroll
+    for (int p = 0; p < PX; ++p)
+#pragma unroll
+        for (int j = 0; j < CH; ++j) x ^= acc[p][j];
+    sink[(size_t)blockIdx.x * kThreads + threadIdx.x] = x;
+    if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
+}
+
+// Single-instruction chains, 16 independent values per thread, each new value depending on
+// three different old ones so that consecutive operations cannot be merged.
+template <int KIND>
+__global__ void __launch_bounds__(kThreads)
+probe_unit_kernel(const uint32_t *__restrict__ seed, uint32_t *__restrict__ sink, long long *__restrict__ cycles,
+                  int iterations)
+{
+    uint32_t v[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = seed[(threadIdx.x + i * 37) & 1023];
+    __syncthreads();
+    const long long t0 = clock64();
+    for (int it = 0; it < iterations; ++it) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const uint32_t b = v[(i + 5) & 15], c = v[(i + 11) & 15];
+                if (KIND == 10) v[i] = lop3<0x3A>(v[i], b, c);
+                if (KIND == 11) v[i] = __popc(v[i]);
+                if (KIND == 12) asm volatile("add.u32 %0, %0, %1;\n\tadd.u32 %0, %0, %2;" : "+r"(v[i]) : "r"(b), "r"(c));
+                if (KIND == 13) asm volatile("mad.lo.u32 %0, %1, %2, %0;" : "+r"(v[i]) : "r"(b), "r"(c));
+            }
+        }
+    }
+    const long long t1 = clock64();
+    uint32_t x = 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) x ^= v[i];
+    sink[(size_t)blockIdx.x * kThreads + threadIdx.x] = x;
+    if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
+}
+
+// Legacy warp-level 1-bit MMA: m16n8k256, s32 accumulate, XOR+POPC or AND+POPC.
+template <bool USE_AND>
+__global__ void __launch_bounds__(kThreads)
+probe_mma_b1_kernel(const uint32_t *__restrict__ seed, uint32_t *__restrict__ sink, long long *__restrict__ cycles,
+                    int iterations)
+{
+    uint32_t a[4], b[2];
+    int32_t d[8][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) a[i] = seed[(threadIdx.x * 4 + i) & 1023];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) b[i] = seed[(threadIdx.x * 2 + i + 300) & 1023];
+#pragma unroll
+    for (int t = 0; t < 8; ++t)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) d[t][i] = 0;
+    __syncthreads();
+    const long long t0 = clock64();
+    for (int it = 0; it < iterations; ++it) {
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            if (USE_AND)
+                asm volatile(
+                    "mma.sync.aligned.m16n8k256.row.col.s32.b1.b1.s32.and.popc {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                    "{%0,%1,%2,%3};"
+                    : "+r"(d[t][0]), "+r"(d[t][1]), "+r"(d[t][2]), "+r"(d[t][3])
+                    : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+            else
+                asm volatile(
+                    "mma.sync.aligned.m16n8k256.row.col.s32.b1.b1.s32.xor.popc {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                    "{%0,%1,%2,%3};"
+                    : "+r"(d[t][0]), "+r"(d[t][1]), "+r"(d[t][2]), "+r"(d[t][3])
+                    : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+        }
+    }
+    const long long t1 = clock64();
+    uint32_t x = 0;
+#pragma unroll
+    for (int t = 0; t < 8; ++t)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) x ^= (uint32_t)d[t][i];
+    sink[(size_t)blockIdx.x * kThreads + threadIdx.x] = x;
+    if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
+}
+
+}  // namespace
+}  // namespace lce
+
+extern "C" lce_status lce_probe_pipe(int32_t mix, int32_t iterations, double *ops_per_second,
+                                     double *ops_per_clock_per_sm, void *stream)
+{
+    using namespace lce;
+    if (!ops_per_second || !ops_per_clock_per_sm || iterations <= 0) return LCE_ERR_INVALID_ARG;
+    double ops_per_thread_iter;
+    switch (mix) {
+        case 0: case 1: case 2: ops_per_thread_iter = PX * CH * 9; break;
+        case 10: case 11: case 13: ops_per_thread_iter = 64; break;
+        case 12: ops_per_thread_iter = 128; break;            // two adds per step
+        case 20: case 21: ops_per_thread_iter = 8 * 1024.0 / 32; break;  // 8 MMAs x 16*8*256/32 word pairs per warp
+        default: return LCE_ERR_INVALID_ARG;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LCE_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return LCE_ERR_CUDA;
+    typedef void (*probe_fn)(const uint32_t *, uint32_t *, long long *, int);
+    probe_fn fn = nullptr;
+    switch (mix) {
+        case 0: fn = probe_mix_kernel<0>; break;
+        case 1: fn = probe_mix_kernel<1>; break;
+        case 2: fn = probe_mix_kernel<2>; break;
+        case 10: fn = probe_unit_kernel<10>; break;
+        case 11: fn = probe_unit_kernel<11>; break;
+        case 12: fn = probe_unit_kernel<12>; break;
+        case 13: fn = probe_unit_kernel<13>; break;
+        case 20: fn = probe_mma_b1_kernel<false>; break;
+        default: fn = probe_mma_b1_kernel<true>; break;
+    }
+    // one wave exactly: as many blocks per SM as the kernel's registers let be resident
+    int blocks_per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, fn, kThreads, 0) != cudaSuccess ||
+        blocks_per_sm < 1)
+        return LCE_ERR_CUDA;
+    const int blocks = sms * blocks_per_sm;
+    uint32_t *seed = nullptr, *sink = nullptr;
+    long long *cycles = nullptr;
+    lce_status st = LCE_ERR_CUDA;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    uint32_t host_seed[1024];
+    uint32_t lcg = 2011093980u;
+    for (int i = 0; i < 1024; ++i) { lcg = lcg * 1664525u + 1013904223u; host_seed[i] = lcg ^ (lcg >> 13); }
+    long long *host_cycles = nullptr;
+    do {
+        if (cudaMalloc(&seed, sizeof(host_seed)) != cudaSuccess) break;
+        if (cudaMalloc(&sink, (size_t)blocks * kThreads * 4) != cudaSuccess) break;
+        if (cudaMalloc(&cycles, (size_t)blocks * 8) != cudaSuccess) break;
+        if (cudaMemcpyAsync(seed, host_seed, sizeof(host_seed), cudaMemcpyHostToDevice, s) != cudaSuccess) break;
+        if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) break;
+        for (int rep = 0; rep < 2; ++rep) {  // first repetition warms up
+            if (rep == 1) cudaEventRecord(e0, s);
+            fn<<<blocks, kThreads, 0, s>>>(seed, sink, cycles, iterations);
+        }
+        cudaEventRecord(e1, s);
+        if (cudaEventSynchronize(e1) != cudaSuccess) break;
+        if (cudaGetLastError() != cudaSuccess) break;
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess || ms <= 0.f) break;
+        host_cycles = new long long[blocks];
+        if (cudaMemcpy(host_cycles, cycles, (size_t)blocks * 8, cudaMemcpyDeviceToHost) != cudaSuccess) break;
+        double mean_cycles = 0;
+        for (int i = 0; i < blocks; ++i) mean_cycles += (double)host_cycles[i];
+        mean_cycles /= blocks;
+        const double per_thread = ops_per_thread_iter * (double)iterations;
+        const double total = per_thread * (double)blocks * kThreads;
+        *ops_per_second = total / (ms * 1e-3);
+        *ops_per_clock_per_sm = per_thread * kThreads * blocks_per_sm / mean_cycles;
+        st = LCE_OK;
+    } while (0);
+    delete[] host_cycles;
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    cudaFree(seed); cudaFree(sink); cudaFree(cycles);
+    return st;
+}

@@ -1,0 +1,188 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Integer and bit outputs must be identical; float outputs must agree within
+1e-6 * (|acc*multiplier| + |bias|) (the transform is a single fp32 multiply-add; the goal is 0 ulp)."""
+import numpy as np
+import pytest
+import torch
+
+import lce_workloads as wl
+import oracle
+import paper_2011_09398_b200 as lce
+from gpu_util import DEV, guarded, guards_intact, run_bconv, to_dev, to_dev_words, words_to_host
+
+pytestmark = pytest.mark.gpu
+
+KERNELS = [lce.KERNEL_DIRECT, lce.KERNEL_AUTO]
+
+
+def rand_pm1(rng, shape):
+    return (2 * rng.integers(0, 2, size=shape) - 1).astype(np.int8)
+
+
+def float_close(got, acc, mult, bias, act=0):
+    v = np.maximum(acc, 0) if act else acc
+    want = oracle.transform_float(acc, mult, bias, act)
+    tol = 1e-6 * (np.abs(v.astype(np.float64) * mult.astype(np.float64)) + np.abs(bias.astype(np.float64)))
+    err = np.abs(got.astype(np.float64) - want.astype(np.float64))
+    assert np.all(err <= tol), f"max err {err.max()}"
+    return int((got != want).sum())
+
+
+# ---- LceQuantize / LceDequantize ---------------------------------------------------------
+
+@pytest.mark.parametrize("rows,C", [(1, 1), (7, 3), (50, 31), (33, 32), (129, 33), (1000, 40), (4097, 64), (300, 96),
+                                    (513, 256), (2, 4096), (100003, 3)])
+def test_bitpack_matches_oracle(rows, C):
+    rng = np.random.default_rng(rows * 131 + C)
+    x = rng.standard_normal((rows, C)).astype(np.float32)
+    x.flat[:6] = [0.0, -0.0, np.nan, -np.nan, np.inf, -np.inf][: min(6, x.size)]
+    whole, out = guarded((rows, (C + 31) // 32), torch.int32, 0x5A5A5A5A)
+    lce.lce_bitpack(to_dev(x), out)
+    torch.cuda.synchronize()
+    assert guards_intact(whole, 0x5A5A5A5A)
+    np.testing.assert_array_equal(words_to_host(out), oracle.bitpack(x))
+
+
+def test_bitpack_one_hot_bit_order():
+    for C, c in ((64, 0), (64, 31), (64, 32), (70, 69)):
+        x = np.ones((3, C), np.float32)
+        x[1, c] = -1.0
+        got = words_to_host(lce.lce_bitpack(to_dev(x)))
+        np.testing.assert_array_equal(got, oracle.bitpack(x))
+        assert int(got[1, c // 32]) == 1 << (c % 32)
+
+
+@pytest.mark.parametrize("rows,C", [(5, 3), (64, 64), (77, 70), (1, 1)])
+def test_unpack_matches_oracle(rows, C):
+    rng = np.random.default_rng(C)
+    words = oracle.bitpack(rng.standard_normal((rows, C)).astype(np.float32))
+    got = lce.lce_unpack(to_dev_words(words), C).cpu().numpy()
+    np.testing.assert_array_equal(got, oracle.unpack_f32(words, C))
+
+
+def test_empty_bitpack_is_a_noop():
+    x = torch.empty((0, 64), dtype=torch.float32, device=DEV)
+    assert lce.lce_bitpack(x).shape == (0, 2)
+
+
+# ---- LceBConv2d: fuzz over small ragged shapes --------------------------------------------
+
+FUZZ = [
+    # N, H, W, Cin, Cout, k, s
+    (1, 1, 1, 1, 1, 1, 1), (2, 5, 7, 3, 4, 3, 1), (1, 6, 6, 31, 5, 3, 2), (2, 7, 5, 32, 33, 3, 1),
+    (1, 9, 8, 33, 31, 5, 1), (1, 8, 9, 64, 32, 5, 2), (3, 4, 4, 96, 64, 1, 1), (1, 7, 7, 40, 3, 1, 2),
+    (1, 2, 3, 64, 2, 3, 1), (2, 14, 14, 64, 64, 3, 1), (2, 14, 14, 64, 8, 3, 2), (1, 3, 3, 5, 7, 3, 1),
+    (3, 7, 7, 512, 64, 3, 1), (2, 9, 11, 160, 70, 3, 1), (1, 17, 13, 96, 96, 3, 2), (2, 8, 8, 128, 130, 3, 1),
+    (1, 29, 31, 64, 64, 3, 1), (2, 16, 16, 256, 32, 1, 1), (1, 57, 9, 32, 64, 3, 1), (5, 7, 7, 64, 64, 3, 1),
+]
+
+
+@pytest.mark.parametrize("kernel_choice", KERNELS)
+@pytest.mark.parametrize("padding", [lce.PAD_VALID, lce.PAD_SAME_ONE, lce.PAD_SAME_ZERO])
+@pytest.mark.parametrize("shape", FUZZ)
+def test_bconv_all_output_types_match_oracle(shape, padding, kernel_choice):
+    N, H, W, Cin, Cout, k, s = shape
+    if padding == lce.PAD_VALID and (H < k or W < k):
+        pytest.skip("empty VALID output")
+    rng = np.random.default_rng(abs(hash((shape, padding))) % 2**32)
+    a, w = rand_pm1(rng, (N, H, W, Cin)), rand_pm1(rng, (Cout, k, k, Cin))
+    aw, ww = oracle.bitpack_pm1(a), oracle.bitpack_pm1(w)
+    acc = oracle.bconv2d_acc(a, w, (s, s), padding)
+    kw = dict(in_c=Cin, stride=(s, s), padding=padding)
+    got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_INT32), kernel_choice=kernel_choice)
+    np.testing.assert_array_equal(got, acc)
+    K = k * k * Cin
+    thr = np.rint(np.sqrt(K) * rng.standard_normal(Cout)).astype(np.int32)
+    got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_BITPACKED), thr=thr, kernel_choice=kernel_choice)
+    np.testing.assert_array_equal(got, oracle.transform_bits(acc, thr))
+    mult = rng.uniform(0.5, 1.5, Cout).astype(np.float32)
+    bias = (0.1 * rng.standard_normal(Cout)).astype(np.float32)
+    for act in (lce.ACT_NONE, lce.ACT_RELU):
+        got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_FLOAT32, activation=act), mult=mult, bias=bias,
+                        kernel_choice=kernel_choice)
+        assert float_close(got, acc, mult, bias, act) == 0  # goal: bit-identical floats
+
+
+@pytest.mark.parametrize("kernel_choice", KERNELS)
+def test_saturated_thresholds_and_pad_bits(kernel_choice):
+    rng = np.random.default_rng(77)
+    a, w = rand_pm1(rng, (1, 6, 6, 64)), rand_pm1(rng, (40, 3, 3, 64))
+    aw, ww = oracle.bitpack_pm1(a), oracle.bitpack_pm1(w)
+    lo = np.full(40, np.iinfo(np.int32).min, np.int32)
+    hi = np.full(40, np.iinfo(np.int32).max, np.int32)
+    kw = dict(in_c=64, out_type=lce.OUT_BITPACKED)
+    assert not run_bconv(aw, ww, kw, thr=lo, kernel_choice=kernel_choice).any()
+    ones = run_bconv(aw, ww, kw, thr=hi, kernel_choice=kernel_choice)
+    assert np.all(ones[..., 0] == 0xFFFFFFFF) and np.all(ones[..., 1] == 0xFF)
+
+
+# ---- config 1 and batch-reduced versions of configs 2, 3 ------------------------------------
+
+def conv_case(config, first_index, spec, kernel_choice=lce.KERNEL_AUTO):
+    t = wl.conv_tensors(config, first_index, spec)
+    x = wl.activations(config, 0, (spec.batch, spec.in_h, spec.in_w, spec.in_c))
+    a_words_oracle = oracle.bitpack(x)
+    a_words_gpu = words_to_host(lce.lce_bitpack(to_dev(x)))
+    np.testing.assert_array_equal(a_words_gpu, a_words_oracle)
+    w_words = words_to_host(lce.pack_weights(to_dev(t.w_pm1)))
+    np.testing.assert_array_equal(w_words, oracle.bitpack_pm1(t.w_pm1))
+    acc = oracle.bconv2d_acc(oracle.sign(x), t.w_pm1, (spec.stride, spec.stride), spec.padding)
+    kw = dict(in_c=spec.in_c, stride=(spec.stride, spec.stride), padding=spec.padding, out_type=spec.out_type)
+    if spec.out_type == wl.OUT_FLOAT32:
+        got = run_bconv(a_words_gpu, w_words, kw, mult=t.multiplier, bias=t.bias, kernel_choice=kernel_choice)
+        assert float_close(got, acc, t.multiplier, t.bias) == 0
+    else:
+        got = run_bconv(a_words_gpu, w_words, kw, thr=t.thresholds, kernel_choice=kernel_choice)
+        np.testing.assert_array_equal(got, oracle.transform_bits(acc, t.thresholds))
+
+
+@pytest.mark.parametrize("kernel_choice", KERNELS)
+def test_config1_single_conv(kernel_choice):
+    conv_case(1, 1, wl.config1_spec(), kernel_choice)
+
+
+@pytest.mark.parametrize("spec", wl.config2_specs(batch=4) + wl.config3_specs(batch=4), ids=lambda s: s.name)
+def test_config2_config3_shapes_small_batch(spec):
+    conv_case(2, 1, spec)
+
+
+# ---- LceBMaxPool2d, add -------------------------------------------------------------------
+
+@pytest.mark.parametrize("shape,pool,stride,padding", [
+    ((2, 8, 8, 64), (2, 2), (2, 2), lce.PAD_VALID), ((1, 7, 9, 45), (3, 3), (2, 2), lce.PAD_SAME_ONE),
+    ((3, 5, 6, 130), (2, 3), (1, 2), lce.PAD_VALID), ((2, 56, 56, 64), (2, 2), (2, 2), lce.PAD_VALID),
+    ((1, 9, 9, 33), (3, 3), (1, 1), lce.PAD_SAME_ONE)])
+def test_bmaxpool_matches_oracle(shape, pool, stride, padding):
+    rng = np.random.default_rng(sum(shape))
+    C = shape[-1]
+    words = oracle.bitpack(rng.standard_normal(shape).astype(np.float32))
+    got = words_to_host(lce.lce_bmaxpool(to_dev_words(words), C, pool, stride, padding))
+    np.testing.assert_array_equal(got, oracle.bmaxpool(words, C, pool, stride, padding))
+
+
+@pytest.mark.parametrize("n", [1, 3, 4, 1023, 4096, 100001])
+def test_add_matches_oracle(n):
+    rng = np.random.default_rng(n)
+    a = (rng.standard_normal(n) * 100).astype(np.float32)
+    b = rng.standard_normal(n).astype(np.float32)
+    got = lce.lce_add_f32(to_dev(a), to_dev(b)).cpu().numpy()
+    np.testing.assert_array_equal(got, oracle.add_f32(a, b))
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    spec = wl.with_batch(wl.config2_specs()[1], 2)  # 56x56x64 bit-packed, batch 2
+    t = wl.conv_tensors(2, 1, spec)
+    x = wl.activations(2, 0, (spec.batch, spec.in_h, spec.in_w, spec.in_c))
+    aw, ww = oracle.bitpack(x), oracle.bitpack_pm1(t.w_pm1)
+    desc = lce.make_desc(spec.batch, spec.in_h, spec.in_w, spec.in_c, spec.out_c, out_type=lce.OUT_BITPACKED)
+    ws = torch.empty(lce.lce_bconv2d_host_workspace_bytes(desc), dtype=torch.uint8, device=DEV)
+    h_in = torch.from_numpy(aw.view(np.int32)).pin_memory()
+    h_w = torch.from_numpy(ww.view(np.int32)).pin_memory()
+    h_thr = torch.from_numpy(t.thresholds).pin_memory()
+    h_out = torch.empty((spec.batch, spec.out_h, spec.out_w, 2), dtype=torch.int32).pin_memory()
+    lce.lce_bconv2d_host(desc, h_in, h_w, None, None, h_thr, h_out, ws)
+    acc = oracle.bconv2d_acc(oracle.sign(x), t.w_pm1, (1, 1), spec.padding)
+    np.testing.assert_array_equal(h_out.numpy().view(np.uint32), oracle.transform_bits(acc, t.thresholds))
+    with pytest.raises(lce.LceError) as e:
+        lce.lce_bconv2d_host(desc, h_in, h_w, None, None, h_thr, h_out, ws[:1024])
+    assert e.value.status == 6

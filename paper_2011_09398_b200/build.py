@@ -38,7 +38,8 @@ def build(force: bool = False, verbose: bool = False) -> Path:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
-    cmd = [nvcc, *NVCC_FLAGS, f"-I{INCLUDE}", f"-I{CSRC}", "-o", str(tmp), *map(str, sources())]
+    extra = os.environ.get("LCE_NVCC_FLAGS", "").split()  # e.g. -DLCE_CTAS_PER_SM=3 for tuning runs
+    cmd = [nvcc, *NVCC_FLAGS, *extra, f"-I{INCLUDE}", f"-I{CSRC}", "-o", str(tmp), *map(str, sources())]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
         print(" ".join(cmd), file=sys.stderr)

@@ -1,8 +1,391 @@
+// LceBConv2d, tiled XOR/POPC kernels (paper Section 3.2: im2col -> BGEMM -> output transform,
+// here as one implicit-GEMM kernel: the im2col matrix is never materialised, the accumulators
+// never leave registers before the output transform).
+//
+// 3x3 kernel, stride 1 or 2, any channel counts and image sizes:
+//   * a CTA owns a run of consecutive output pixels (flat (n, oh, ow) order) times 64 output
+//     channels; a warp works on 4 pixels x 8 channel groups at a time, a thread on TP pixels
+//     (16 apart in the flat order) x 8 channels, i.e. TP x 8 accumulators in registers;
+//   * the CTA first copies the packed input rows its pixels need into shared memory, one plane
+//     per channel word, in "padded image" coordinates: rows/columns outside the image hold zero
+//     words, which is exactly the paper's one-padding (a zero bit is +1.0);
+//   * the weights of its 64 channels are turned into carry-save operands (csa.cuh) while they
+//     are copied to shared memory;
+//   * for every channel word the nine taps of a (pixel, channel) pair form one nine-word
+//     carry-save group: 16 LOP3 + 4 POPC + 4 IMAD instead of 9 XOR + 9 POPC + 9 adds.  The
+//     activation-side operands of the thread's TP pixels sit in registers for the whole channel
+//     word; the weight-side operands of one channel are read from shared memory once and used
+//     for all TP pixels (shared-memory bandwidth, not issue slots, is what this ordering saves);
+//   * epilogue: acc = K - 2*count, then float multiply-add, threshold + bit-pack, or raw int32.
 #include "common.cuh"
+#include "csa.cuh"
+
 namespace lce {
-lce_status launch_bconv_tiled(const ConvGeom &, const uint32_t *, const uint32_t *, const float *, const float *,
-                              const int32_t *, void *, cudaStream_t)
+namespace {
+
+constexpr int kThreads = 128;       // 4 warps; a warp = 4 pixels x 8 channel groups
+constexpr int kPixPerStep = 16;     // pixels the CTA works on at a time (4 warps x 4)
+constexpr int kChanPerCta = 64;
+constexpr int kChanPerThread = 8;
+constexpr int kWRow = 12;           // 9 carry-save operand words per (channel word, channel) + 3 pad
+constexpr int kWGroupStride = kChanPerThread * kWRow + 4;  // +4 words: the 8 channel groups hit distinct banks
+
+struct TiledParams {
+    const uint32_t *in;
+    const uint32_t *w;
+    const float *mult;
+    const float *bias;
+    const int32_t *thr;
+    void *out;
+    int32_t N, H, W, Cin, Cw, Cout, Cow, OH, OW, pt, pl;
+    int32_t tile_pixels;  // flat output pixels per CTA, a multiple of kPixPerStep * TP
+    int32_t M, Hp, Wp, pitch, plane;
+    int32_t padding, out_type, activation;
+};
+
+template <int BYTE_OFF>
+__device__ __forceinline__ uint4 lds128(uint32_t saddr)
 {
-    return LCE_ERR_UNSUPPORTED;
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(saddr), "n"(BYTE_OFF));
+    return v;
 }
+template <int BYTE_OFF>
+__device__ __forceinline__ uint32_t lds32(uint32_t saddr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(saddr), "n"(BYTE_OFF));
+    return v;
+}
+
+template <int J>
+__device__ __forceinline__ void load_w_triples(uint32_t saddr, Triple (&wt)[3])
+{
+    const uint4 q0 = lds128<J * 48>(saddr);
+    const uint4 q1 = lds128<J * 48 + 16>(saddr);
+    const uint32_t q2 = lds32<J * 48 + 32>(saddr);
+    wt[0].all = q0.x; wt[0].pair = q0.y; wt[0].first = q0.z;
+    wt[1].all = q0.w; wt[1].pair = q1.x; wt[1].first = q1.y;
+    wt[2].all = q1.z; wt[2].pair = q1.w; wt[2].first = q2;
+}
+
+__device__ __forceinline__ int32_t w_smem_offset(int cw, int ch)
+{
+    return cw * (kChanPerCta / kChanPerThread) * kWGroupStride + (ch >> 3) * kWGroupStride + (ch & 7) * kWRow;
+}
+
+template <int J, int TP>
+struct ChannelLoop {
+    // channel J of the thread: weight operands from shared memory once, then all TP pixels
+    __device__ __forceinline__ static void run(uint32_t w_saddr, const Triple (&at)[TP][3], const Weights124 &k,
+                                               uint32_t (&acc)[TP][kChanPerThread])
+    {
+        Triple wt[3];
+        load_w_triples<J>(w_saddr, wt);
+#pragma unroll
+        for (int i = 0; i < TP; ++i) popc9_mad(at[i], wt, k, acc[i][J]);
+        ChannelLoop<J + 1, TP>::run(w_saddr, at, k, acc);
+    }
+};
+template <int TP>
+struct ChannelLoop<kChanPerThread, TP> {
+    __device__ __forceinline__ static void run(uint32_t, const Triple (&)[TP][3], const Weights124 &,
+                                               uint32_t (&)[TP][kChanPerThread]) {}
+};
+
+template <int STRIDE, int TP>
+__global__ void __launch_bounds__(kThreads, (TP <= 4 ? 4 : (TP <= 7 ? 3 : 2)))
+bconv3x3_kernel(const TiledParams p)
+{
+    extern __shared__ __align__(16) uint32_t smem[];
+    uint32_t *sW = smem;                                                       // [Cw][8 groups][kWGroupStride]
+    uint32_t *sA = smem + p.Cw * (kChanPerCta / kChanPerThread) * kWGroupStride;  // [Cw][nv][pitch]
+    int32_t *sWsum = reinterpret_cast<int32_t *>(sA + p.Cw * p.plane);            // [64][9], zero-padding only
+
+    const int tid = threadIdx.x;
+    const int m0 = blockIdx.x * p.tile_pixels;
+    const int m_end = min(m0 + p.tile_pixels, p.M);
+    const int ch0 = blockIdx.y * kChanPerCta;
+
+    // virtual (padded-image) rows this CTA needs: v = n*Hp + oh*stride + ky
+    const int r_first = m0 / p.OW, r_last = (m_end - 1) / p.OW;
+    const int v_first = (r_first / p.OH) * p.Hp + (r_first % p.OH) * STRIDE;
+    const int v_last = (r_last / p.OH) * p.Hp + (r_last % p.OH) * STRIDE + 2;
+    const int nv = v_last - v_first + 1;
+
+    // ---- stage the input rows: global [n][iy][ix][cw] -> shared [cw][v][x] -------------------
+    {
+        const int row_words = p.Wp * p.Cw;
+        for (int v = tid >> 5; v < nv; v += kThreads / 32) {
+            const int va = v_first + v;
+            const int n = va / p.Hp;
+            const int iy = va - n * p.Hp - p.pt;
+            const bool row_ok = n < p.N && iy >= 0 && iy < p.H;
+            const uint32_t *src = p.in + ((int64_t)n * p.H + iy) * p.W * p.Cw;
+            for (int e = tid & 31; e < row_words; e += 32) {
+                const int x = e / p.Cw;
+                const int cw = e - x * p.Cw;
+                const int ix = x - p.pl;
+                uint32_t val = 0u;
+                if (row_ok && ix >= 0 && ix < p.W) val = __ldg(src + ix * p.Cw + cw);
+                sA[cw * p.plane + v * p.pitch + x] = val;
+            }
+        }
+    }
+    // ---- stage the weights as carry-save operands: [ch][ky][kx][cw] -> [cw][ch][9 (+3)] -------
+    for (int e = tid; e < kChanPerCta * p.Cw; e += kThreads) {
+        const int ch = e / p.Cw;
+        const int cw = e - ch * p.Cw;
+        uint32_t wv[9];
+#pragma unroll
+        for (int t = 0; t < 9; ++t)
+            wv[t] = (ch0 + ch < p.Cout) ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + t) * p.Cw + cw) : 0u;
+        uint32_t *dst = sW + w_smem_offset(cw, ch);
+#pragma unroll
+        for (int g = 0; g < 3; ++g) {
+            const Triple t = make_triple(wv[3 * g], wv[3 * g + 1], wv[3 * g + 2]);
+            dst[3 * g] = t.all;
+            dst[3 * g + 1] = t.pair;
+            dst[3 * g + 2] = t.first;
+        }
+        dst[9] = dst[10] = dst[11] = 0u;
+    }
+    if (p.padding == LCE_PAD_SAME_ZERO) {
+        // sum over the true channels of one tap's weights = Cin - 2*popcount (pad bits are 0)
+        for (int e = tid; e < kChanPerCta * 9; e += kThreads) {
+            const int ch = e / 9, t = e - ch * 9;
+            int32_t cnt = 0;
+            if (ch0 + ch < p.Cout)
+                for (int cw = 0; cw < p.Cw; ++cw) cnt += __popc(__ldg(p.w + ((int64_t)(ch0 + ch) * 9 + t) * p.Cw + cw));
+            sWsum[e] = p.Cin - 2 * cnt;
+        }
+    }
+
+    // ---- this thread's channels and pixels ---------------------------------------------------
+    const int lane = tid & 31, warp = tid >> 5;
+    const int px = lane >> 3, cg = lane & 7;
+    const int chan = ch0 + cg * kChanPerThread;
+    const int K = 9 * p.Cin;
+    Weights124 k124;
+    k124.one = p.N > 0 ? 1u : p.Cin;  // opaque to the compiler: keeps the weighted sum on multiply-adds
+    k124.two = p.N > 0 ? 2u : p.Cin;
+    k124.four = p.N > 0 ? 4u : p.Cin;
+    asm volatile("" : "+r"(k124.one), "+r"(k124.two), "+r"(k124.four));
+
+    // running (n, oh, ow) of this lane's next pixel; pixels of one lane are kPixPerStep apart
+    int m_next = m0 + warp * 4 + px;
+    int ow, voh;  // voh = n*Hp + oh*STRIDE: the pixel's first virtual row
+    {
+        const int r = m_next / p.OW;
+        ow = m_next - r * p.OW;
+        const int n = r / p.OH;
+        voh = n * p.Hp + (r - n * p.OH) * STRIDE;
+    }
+    int oh_left = p.OH - 1 - (m_next / p.OW) % p.OH;  // rows left in the image after this one
+    const int a_base_first = ((r_first / p.OH) * p.Hp + (r_first % p.OH) * STRIDE - v_first) * p.pitch +
+                             (m0 - r_first * p.OW) * STRIDE;
+    const uint32_t w_saddr0 = (uint32_t)__cvta_generic_to_shared(sW + cg * kWGroupStride);
+    __syncthreads();
+
+    for (int base = m0; base < m0 + p.tile_pixels; base += kPixPerStep * TP) {
+        int a_base[TP];
+#pragma unroll
+        for (int i = 0; i < TP; ++i) {
+            // pixels past the end of the tile redo the tile's first pixel and store nothing
+            a_base[i] = (m_next < m_end) ? (voh - v_first) * p.pitch + ow * STRIDE : a_base_first;
+            m_next += kPixPerStep;
+            ow += kPixPerStep;
+            while (ow >= p.OW) {
+                ow -= p.OW;
+                if (oh_left == 0) { oh_left = p.OH - 1; voh += 3; }   // next image: Hp - (OH-1)*STRIDE = 3
+                else { --oh_left; voh += STRIDE; }
+            }
+        }
+        uint32_t acc[TP][kChanPerThread];
+#pragma unroll
+        for (int i = 0; i < TP; ++i)
+#pragma unroll
+            for (int j = 0; j < kChanPerThread; ++j) acc[i][j] = 0u;
+
+        uint32_t w_saddr = w_saddr0;
+        const uint32_t *plane = sA;
+        for (int cw = 0; cw < p.Cw; ++cw) {
+            Triple at[TP][3];
+#pragma unroll
+            for (int i = 0; i < TP; ++i)
+#pragma unroll
+                for (int ky = 0; ky < 3; ++ky) {
+                    const uint32_t *row = plane + a_base[i] + ky * p.pitch;
+                    at[i][ky] = make_triple(row[0], row[1], row[2]);
+                }
+            ChannelLoop<0, TP>::run(w_saddr, at, k124, acc);
+            w_saddr += (kChanPerCta / kChanPerThread) * kWGroupStride * 4;
+            plane += p.plane;
+        }
+
+        // ---- output transform -------------------------------------------------------------
+        float mult[kChanPerThread], bias[kChanPerThread];
+        int32_t thr[kChanPerThread];
+#pragma unroll
+        for (int j = 0; j < kChanPerThread; ++j) {
+            const bool ok = chan + j < p.Cout;
+            mult[j] = (p.out_type == LCE_OUT_FLOAT32 && ok) ? __ldg(p.mult + chan + j) : 0.f;
+            bias[j] = (p.out_type == LCE_OUT_FLOAT32 && ok) ? __ldg(p.bias + chan + j) : 0.f;
+            thr[j] = (p.out_type == LCE_OUT_BITPACKED && ok) ? __ldg(p.thr + chan + j) : INT32_MIN;  // pad bits -> 0
+        }
+#pragma unroll
+        for (int i = 0; i < TP; ++i) {
+            const int m = base + i * kPixPerStep + warp * 4 + px;
+            const bool pix_ok = m < m_end;
+            int32_t v[kChanPerThread];
+#pragma unroll
+            for (int j = 0; j < kChanPerThread; ++j) v[j] = K - 2 * (int32_t)acc[i][j];
+            if (p.padding == LCE_PAD_SAME_ZERO) {
+                // zero-padding correction: taps outside the image contributed (+1)*w; take that out
+                const int mm = pix_ok ? m : m0;
+                const int r = mm / p.OW;
+                const int iy0 = (r % p.OH) * STRIDE - p.pt, ix0 = (mm - r * p.OW) * STRIDE - p.pl;
+#pragma unroll
+                for (int t = 0; t < 9; ++t) {
+                    const int iy = iy0 + t / 3, ix = ix0 + t % 3;
+                    if (iy < 0 || iy >= p.H || ix < 0 || ix >= p.W) {
+#pragma unroll
+                        for (int j = 0; j < kChanPerThread; ++j) v[j] -= sWsum[(cg * kChanPerThread + j) * 9 + t];
+                    }
+                }
+            }
+            if (p.out_type == LCE_OUT_BITPACKED) {
+                uint32_t bits = 0u;
+#pragma unroll
+                for (int j = 0; j < kChanPerThread; ++j) bits |= (v[j] < thr[j] ? 1u : 0u) << j;
+                // the 4 lanes cg&~3 .. cg|3 hold the 4 bytes of one output word
+                bits <<= 8 * (cg & 3);
+                bits |= __shfl_xor_sync(0xffffffffu, bits, 1);
+                bits |= __shfl_xor_sync(0xffffffffu, bits, 2);
+                const int word = (ch0 >> 5) + (cg >> 2);
+                if (pix_ok && (cg & 3) == 0 && word < p.Cow)
+                    static_cast<uint32_t *>(p.out)[(int64_t)m * p.Cow + word] = bits;
+            } else if (p.out_type == LCE_OUT_FLOAT32) {
+                float f[kChanPerThread];
+#pragma unroll
+                for (int j = 0; j < kChanPerThread; ++j) {
+                    const int32_t a = (p.activation == LCE_ACT_RELU && v[j] < 0) ? 0 : v[j];
+                    f[j] = __fmaf_rn((float)a, mult[j], bias[j]);
+                }
+                if (pix_ok) {
+                    float *dst = static_cast<float *>(p.out) + (int64_t)m * p.Cout + chan;
+                    if ((p.Cout & 3) == 0 && chan + kChanPerThread <= p.Cout) {
+                        reinterpret_cast<float4 *>(dst)[0] = make_float4(f[0], f[1], f[2], f[3]);
+                        reinterpret_cast<float4 *>(dst)[1] = make_float4(f[4], f[5], f[6], f[7]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < kChanPerThread; ++j)
+                            if (chan + j < p.Cout) dst[j] = f[j];
+                    }
+                }
+            } else {
+                if (pix_ok) {
+                    int32_t *dst = static_cast<int32_t *>(p.out) + (int64_t)m * p.Cout + chan;
+                    if ((p.Cout & 3) == 0 && chan + kChanPerThread <= p.Cout) {
+                        reinterpret_cast<int4 *>(dst)[0] = make_int4(v[0], v[1], v[2], v[3]);
+                        reinterpret_cast<int4 *>(dst)[1] = make_int4(v[4], v[5], v[6], v[7]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < kChanPerThread; ++j)
+                            if (chan + j < p.Cout) dst[j] = v[j];
+                    }
+                }
+            }
+        }
+    }
+}
+
+#ifndef LCE_TP
+#define LCE_TP 4
+#endif
+constexpr int kTP = LCE_TP;  // pixels per thread
+
+template <int STRIDE>
+lce_status launch3x3(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStream_t s)
+{
+    auto kernel = bconv3x3_kernel<STRIDE, kTP>;
+    if (smem_bytes > 48 * 1024) {
+        // opt in to the large dynamic shared memory carve-out
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
+            return LCE_ERR_CUDA;
+    }
+    kernel<<<grid, kThreads, smem_bytes, s>>>(p);
+    return launch_status();
+}
+
+size_t smem_bytes_for(const ConvGeom &g, const TiledParams &p)
+{
+    return ((size_t)g.Cw * (kChanPerCta / kChanPerThread) * kWGroupStride + (size_t)g.Cw * p.plane + kChanPerCta * 9) * 4;
+}
+
+void set_tile(const ConvGeom &g, TiledParams *p, int tile_pixels)
+{
+    p->tile_pixels = tile_pixels;
+    int rows_max = (tile_pixels - 1) / g.OW + 2;  // output rows a run of tile_pixels flat pixels can touch
+    if (rows_max > tile_pixels) rows_max = tile_pixels;
+    const int nv_max = (rows_max - 1) * 3 + 3;     // consecutive output rows are at most 3 virtual rows apart
+    p->plane = nv_max * p->pitch;
+}
+
+}  // namespace
+
+lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const float *mult,
+                              const float *bias, const int32_t *thr, void *out, cudaStream_t s)
+{
+    if (g.KH != 3 || g.KW != 3 || g.sh != g.sw || g.sh > 2) return LCE_ERR_UNSUPPORTED;
+    // 128-bit epilogue stores need a 16-byte aligned output when the channel count allows them
+    if ((g.Cout & 3) == 0 && g.out_type != LCE_OUT_BITPACKED && !aligned(out, 16)) return LCE_ERR_UNSUPPORTED;
+    if (g.M >= (1ll << 31) - 256) return LCE_ERR_UNSUPPORTED;
+    TiledParams p{};
+    p.in = in; p.w = w; p.mult = mult; p.bias = bias; p.thr = thr; p.out = out;
+    p.N = g.N; p.H = g.H; p.W = g.W; p.Cin = g.Cin; p.Cw = g.Cw; p.Cout = g.Cout; p.Cow = g.Cow;
+    p.OH = g.OH; p.OW = g.OW; p.pt = g.pt; p.pl = g.pl;
+    p.padding = g.padding; p.out_type = g.out_type; p.activation = g.activation;
+    p.M = (int32_t)g.M;
+    p.Hp = (g.OH - 1) * g.sh + 3;
+    p.Wp = (g.OW - 1) * g.sh + 3;
+    p.pitch = p.Wp | 1;  // odd pitch: the 4 pixels of a warp in 4 different rows hit 4 different banks
+    const int chan_blocks = (g.Cout + kChanPerCta - 1) / kChanPerCta;
+    if (chan_blocks > 65535) return LCE_ERR_UNSUPPORTED;
+
+    // Tile size: the largest of {128, 112, ..., 16} flat pixels whose shared memory lets at least
+    // three CTAs share an SM, then shrunk while that fills the machine's CTA slots more evenly.
+    int sms = 148;
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    int best_tile = 0;
+    double best_cost = 0;
+    const int unit = kPixPerStep * kTP;
+    for (int tile = (128 / unit > 0 ? 128 / unit : 1) * unit; tile >= unit; tile -= unit) {
+        set_tile(g, &p, tile);
+        const size_t smem = smem_bytes_for(g, p);
+        if (smem > 110 * 1024) continue;
+        int per_sm = (int)((220 * 1024) / (smem + 1024));
+        const int reg_limit = kTP <= 4 ? 4 : (kTP <= 7 ? 3 : 2);
+        if (per_sm > reg_limit) per_sm = reg_limit;
+        const int64_t ctas = ((g.M + tile - 1) / tile) * chan_blocks;
+        const int64_t slots = (int64_t)sms * per_sm;
+        const int64_t waves = (ctas + slots - 1) / slots;
+        // time ~ waves * (per-CTA work + fixed staging cost), per-CTA work ~ tile pixels
+        const double staging = 12.0 + 64.0 / (9.0 * g.Cw) ;  // in "pixels" of main-loop time; rough
+        const double cost = (double)waves * (tile + staging) / per_sm;
+        if (best_tile == 0 || cost < best_cost) { best_tile = tile; best_cost = cost; }
+    }
+    if (best_tile == 0) return LCE_ERR_UNSUPPORTED;
+    set_tile(g, &p, best_tile);
+    const size_t smem_bytes = smem_bytes_for(g, p);
+    const int64_t ctas = (g.M + best_tile - 1) / best_tile;
+    dim3 grid((unsigned)ctas, (unsigned)chan_blocks, 1);
+    return g.sh == 1 ? launch3x3<1>(p, smem_bytes, grid, s) : launch3x3<2>(p, smem_bytes, grid, s);
+}
+
 }  // namespace lce

@@ -64,6 +64,39 @@ __device__ __forceinline__ uint32_t popc9(const Triple (&a)[3], const Triple (&w
     return __popc(S) + 2u * (__popc(C) + __popc(T)) + 4u * __popc(F);
 }
 
+// The same nine-word count added onto an accumulator with four multiply-adds whose multipliers
+// (1, 2, 2, 4) arrive in registers: integer multiply-add issues on the FMA pipe, so the
+// weighted sum costs the logic pipe nothing.  `k` must hold {1, 2, 4}.
+struct Weights124 {
+    uint32_t one, two, four;
+};
+__device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t r;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+    return r;
+}
+__device__ __forceinline__ void popc9_mad(const Triple (&a)[3], const Triple (&w)[3], const Weights124 &k,
+                                          uint32_t &acc)
+{
+    uint32_t s[3], c[3];
+#pragma unroll
+    for (int g = 0; g < 3; ++g) {
+        s[g] = a[g].all ^ w[g].all;
+        const uint32_t d = a[g].pair ^ w[g].pair;
+        const uint32_t x0 = a[g].first ^ w[g].first;
+        c[g] = carry_dsx(d, s[g], x0);
+    }
+    const uint32_t S = xor3(s[0], s[1], s[2]);
+    const uint32_t C = maj3(s[0], s[1], s[2]);
+    const uint32_t T = xor3(c[0], c[1], c[2]);
+    const uint32_t F = maj3(c[0], c[1], c[2]);
+    acc = mad_u32(__popc(S), k.one, acc);
+    acc = mad_u32(__popc(C), k.two, acc);
+    acc = mad_u32(__popc(T), k.two, acc);
+    acc = mad_u32(__popc(F), k.four, acc);
+}
+
 // popcount of one triple alone (used for K tails and by the 3:2 probe): 4 LOP3 + 2 POPC.
 __device__ __forceinline__ uint32_t popc3(const Triple &a, const Triple &w)
 {

@@ -12,21 +12,23 @@ constexpr int kThreads = 256;
 constexpr int PX = 2;   // pixels per thread in the mix probes
 constexpr int CH = 8;   // output channels per thread
 
-// Makes the compiler treat a register as changed without emitting an instruction, so that the
-// loop body cannot be hoisted.
-__device__ __forceinline__ void touch(uint32_t &v) { asm volatile("" : "+r"(v)); }
-
 template <int MIX>
 __global__ void __launch_bounds__(kThreads)
 probe_mix_kernel(const uint32_t *__restrict__ seed, uint32_t *__restrict__ sink, long long *__restrict__ cycles,
                  int iterations)
 {
-    uint32_t a[PX][9], w[CH][9];
+    // multipliers of the weighted popcount sum, opaque to the compiler (iterations > 0 always)
+    Weights124 k124;
+    k124.one = iterations > 0 ? 1u : seed[0];
+    k124.two = iterations > 0 ? 2u : seed[1];
+    k124.four = iterations > 0 ? 4u : seed[2];
+    asm volatile("" : "+r"(k124.one), "+r"(k124.two), "+r"(k124.four));
+    // Activation words come from shared memory every iteration, as in the convolution kernel
+    // (per pixel nine LDS feed 8 x 9 word operations); weight-side operands stay in registers.
+    __shared__ uint32_t tile[1024 + 64];
+    for (int i = threadIdx.x; i < 1024 + 64; i += kThreads) tile[i] = seed[i & 1023];
+    uint32_t w[CH][9];
     uint32_t acc[PX][CH];
-#pragma unroll
-    for (int p = 0; p < PX; ++p)
-#pragma unroll
-        for (int t = 0; t < 9; ++t) a[p][t] = seed[(threadIdx.x * 31 + p * 9 + t) & 1023];
 #pragma unroll
     for (int j = 0; j < CH; ++j)
 #pragma unroll
@@ -35,8 +37,6 @@ probe_mix_kernel(const uint32_t *__restrict__ seed, uint32_t *__restrict__ sink,
     for (int p = 0; p < PX; ++p)
 #pragma unroll
         for (int j = 0; j < CH; ++j) acc[p][j] = 0;
-
-    // weight-side triples are loop invariant in the real kernel too (they come from shared memory)
     Triple wt[CH][3];
 #pragma unroll
     for (int j = 0; j < CH; ++j)
@@ -44,28 +44,33 @@ probe_mix_kernel(const uint32_t *__restrict__ seed, uint32_t *__restrict__ sink,
         for (int g = 0; g < 3; ++g) wt[j][g] = make_triple(w[j][3 * g], w[j][3 * g + 1], w[j][3 * g + 2]);
 
     __syncthreads();
+    const int base = (threadIdx.x >> 3) * 2;  // lanes that share a pixel read the same words (broadcast)
     const long long t0 = clock64();
     for (int it = 0; it < iterations; ++it) {
+        const uint32_t *row = tile + ((base + it * 11) & 1023);
 #pragma unroll
         for (int p = 0; p < PX; ++p) {
+            uint32_t a[9];
 #pragma unroll
-            for (int t = 0; t < 9; ++t) touch(a[p][t]);
+            for (int t = 0; t < 9; ++t) a[t] = row[p * 9 + t];
             if (MIX == 0) {
 #pragma unroll
                 for (int j = 0; j < CH; ++j)
 #pragma unroll
-                    for (int t = 0; t < 9; ++t) acc[p][j] += __popc(a[p][t] ^ w[j][t]);
+                    for (int t = 0; t < 9; ++t) acc[p][j] += __popc(a[t] ^ w[j][t]);
             } else {
                 Triple at[3];
 #pragma unroll
-                for (int g = 0; g < 3; ++g) at[g] = make_triple(a[p][3 * g], a[p][3 * g + 1], a[p][3 * g + 2]);
+                for (int g = 0; g < 3; ++g) at[g] = make_triple(a[3 * g], a[3 * g + 1], a[3 * g + 2]);
 #pragma unroll
                 for (int j = 0; j < CH; ++j) {
                     if (MIX == 1) {
 #pragma unroll
                         for (int g = 0; g < 3; ++g) acc[p][j] += popc3(at[g], wt[j][g]);
-                    } else {
+                    } else if (MIX == 2) {
                         acc[p][j] += popc9(at, wt[j]);
+                    } else {
+                        popc9_mad(at, wt[j], k124, acc[p][j]);
                     }
                 }
             }
@@ -103,6 +108,15 @@ probe_unit_kernel(const uint32_t *__restrict__ seed, uint32_t *__restrict__ sink
                 if (KIND == 11) v[i] = __popc(v[i]);
                 if (KIND == 12) asm volatile("add.u32 %0, %0, %1;\n\tadd.u32 %0, %0, %2;" : "+r"(v[i]) : "r"(b), "r"(c));
                 if (KIND == 13) asm volatile("mad.lo.u32 %0, %1, %2, %0;" : "+r"(v[i]) : "r"(b), "r"(c));
+                if (KIND == 14) {  // alternate logic and multiply-add: do the two pipes overlap?
+                    if (i & 1) asm volatile("mad.lo.u32 %0, %1, %2, %0;" : "+r"(v[i]) : "r"(b), "r"(c));
+                    else v[i] = lop3<0x3A>(v[i], b, c);
+                }
+                if (KIND == 15) {  // logic, multiply-add and popcount interleaved 4:1:1
+                    if ((i & 7) == 3) v[i] = __popc(v[i]) + b;
+                    else if ((i & 7) == 7) asm volatile("mad.lo.u32 %0, %1, %2, %0;" : "+r"(v[i]) : "r"(b), "r"(c));
+                    else v[i] = lop3<0x3A>(v[i], b, c);
+                }
             }
         }
     }
@@ -169,8 +183,8 @@ extern "C" lce_status lce_probe_pipe(int32_t mix, int32_t iterations, double *op
     if (!ops_per_second || !ops_per_clock_per_sm || iterations <= 0) return LCE_ERR_INVALID_ARG;
     double ops_per_thread_iter;
     switch (mix) {
-        case 0: case 1: case 2: ops_per_thread_iter = PX * CH * 9; break;
-        case 10: case 11: case 13: ops_per_thread_iter = 64; break;
+        case 0: case 1: case 2: case 3: ops_per_thread_iter = PX * CH * 9; break;
+        case 10: case 11: case 13: case 14: case 15: ops_per_thread_iter = 64; break;
         case 12: ops_per_thread_iter = 128; break;            // two adds per step
         case 20: case 21: ops_per_thread_iter = 8 * 1024.0 / 32; break;  // 8 MMAs x 16*8*256/32 word pairs per warp
         default: return LCE_ERR_INVALID_ARG;
@@ -185,10 +199,13 @@ extern "C" lce_status lce_probe_pipe(int32_t mix, int32_t iterations, double *op
         case 0: fn = probe_mix_kernel<0>; break;
         case 1: fn = probe_mix_kernel<1>; break;
         case 2: fn = probe_mix_kernel<2>; break;
+        case 3: fn = probe_mix_kernel<3>; break;
         case 10: fn = probe_unit_kernel<10>; break;
         case 11: fn = probe_unit_kernel<11>; break;
         case 12: fn = probe_unit_kernel<12>; break;
         case 13: fn = probe_unit_kernel<13>; break;
+        case 14: fn = probe_unit_kernel<14>; break;
+        case 15: fn = probe_unit_kernel<15>; break;
         case 20: fn = probe_mma_b1_kernel<false>; break;
         default: fn = probe_mma_b1_kernel<true>; break;
     }

@@ -82,6 +82,9 @@ typedef struct {
     int32_t out_type;   /* lce_out_type */
     int32_t activation; /* lce_activation; FLOAT32 output only */
     int32_t kernel;     /* lce_kernel */
+    int32_t weights_packed; /* 0: `weights` is the plain word tensor [out_c][kh][kw][ceil(in_c/32)];
+                               1: `weights` is the buffer lce_bconv2d_pack_weights wrote for this
+                                  same descriptor (geometry fields must match) */
 } lce_bconv2d_desc;
 
 /* Output extent of the convolution; LCE_ERR_INVALID_ARG if the descriptor is malformed or
@@ -98,6 +101,8 @@ lce_status lce_bconv2d_out_shape(const lce_bconv2d_desc *desc, int32_t *out_h, i
  *             folds it into the thresholds, Section 3.1); multiplier, bias ignored.
  *   INT32     out int32 [batch][oh][ow][out_c]           = acc.
  *   input   uint32[batch][in_h][in_w][ceil(in_c/32)]     weights uint32[out_c][kh][kw][ceil(in_c/32)]
+ * With desc->weights_packed == 1, `weights` is instead the buffer written by
+ * lce_bconv2d_pack_weights (the fast path: nothing is derived from the weights per call).
  * Pad bits of input and weights must be 0.  Errors: INVALID_ARG (null/extent/enum/missing
  * per-channel array), ALIGNMENT, UNSUPPORTED (kernel forced to TILED on a shape it does not
  * cover), CUDA. */
@@ -105,11 +110,24 @@ lce_status lce_bconv2d(const lce_bconv2d_desc *desc, const uint32_t *input, cons
                        const float *multiplier, const float *bias, const int32_t *thresholds,
                        void *output, void *stream);
 
+/* Load-time weight packing (Section 3.2: the paper's BGEMM also re-arranges the weights ahead of
+ * time for its access pattern; Section 3.1: weights are converted once, when the model is built).  Rewrites
+ * the plain packed weights into the operand layout the tiled kernel copies straight into shared
+ * memory, so that none of that work is repeated per call.  The packed buffer also keeps a copy of
+ * the plain words, and is valid for every padding mode, output type and activation of the same
+ * geometry (batch, sizes, channels, kernel, stride).
+ *   weights uint32[out_c][kh][kw][ceil(in_c/32)] (device)  ->  packed: device buffer of
+ *   lce_bconv2d_packed_weights_bytes(desc) bytes, 256-byte aligned, owned by the caller.
+ * lce_bconv2d_packed_weights_bytes returns 0 for a malformed descriptor. */
+size_t lce_bconv2d_packed_weights_bytes(const lce_bconv2d_desc *desc);
+lce_status lce_bconv2d_pack_weights(const lce_bconv2d_desc *desc, const uint32_t *weights, void *packed,
+                                    void *stream);
+
 /* Host-buffer form of lce_bconv2d, for callers whose tensors live in host memory: every data
  * pointer is a HOST pointer (pinned memory makes the copies asynchronous); `workspace` is a
  * DEVICE buffer of at least lce_bconv2d_host_workspace_bytes(desc) bytes that the call uses
  * for the device copies of input, weights, per-channel arrays and output.  Copies in, runs
- * the same kernel as lce_bconv2d, copies the output back, all on `stream`, and returns after
+ * the same kernel as lce_bconv2d (weights_packed must be 0), copies the output back, all on `stream`, and returns after
  * synchronising that stream.  LCE_ERR_WORKSPACE if workspace_bytes is too small. */
 size_t lce_bconv2d_host_workspace_bytes(const lce_bconv2d_desc *desc);
 lce_status lce_bconv2d_host(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,

@@ -25,7 +25,7 @@ class BConv2dDesc(ctypes.Structure):
     """Mirror of lce_bconv2d_desc."""
     _fields_ = [(n, ctypes.c_int32) for n in (
         "batch", "in_h", "in_w", "in_c", "out_c", "kernel_h", "kernel_w", "stride_h", "stride_w",
-        "padding", "out_type", "activation", "kernel")]
+        "padding", "out_type", "activation", "kernel", "weights_packed")]
 
 
 _lib = None
@@ -47,6 +47,9 @@ def library() -> ctypes.CDLL:
         lib.lce_unpack.argtypes = [vp, vp, i64, i32, vp]
         lib.lce_bconv2d_out_shape.argtypes = [ctypes.POINTER(BConv2dDesc), ctypes.POINTER(i32), ctypes.POINTER(i32)]
         lib.lce_bconv2d.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp]
+        lib.lce_bconv2d_packed_weights_bytes.restype = ctypes.c_size_t
+        lib.lce_bconv2d_packed_weights_bytes.argtypes = [ctypes.POINTER(BConv2dDesc)]
+        lib.lce_bconv2d_pack_weights.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp]
         lib.lce_bconv2d_host_workspace_bytes.restype = ctypes.c_size_t
         lib.lce_bconv2d_host_workspace_bytes.argtypes = [ctypes.POINTER(BConv2dDesc)]
         lib.lce_bconv2d_host.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
@@ -54,6 +57,7 @@ def library() -> ctypes.CDLL:
         lib.lce_add_f32.argtypes = [vp, vp, vp, i64, vp]
         lib.lce_probe_pipe.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), vp]
         for name in ("lce_bitpack", "lce_unpack", "lce_bconv2d_out_shape", "lce_bconv2d", "lce_bconv2d_host",
+                     "lce_bconv2d_pack_weights",
                      "lce_bmaxpool", "lce_add_f32", "lce_probe_pipe"):
             getattr(lib, name).restype = ctypes.c_int
         _lib = lib
@@ -90,9 +94,9 @@ def _words(c: int) -> int:
 
 
 def make_desc(batch, in_h, in_w, in_c, out_c, kernel=(3, 3), stride=(1, 1), padding=PAD_SAME_ONE,
-              out_type=OUT_FLOAT32, activation=ACT_NONE, kernel_choice=KERNEL_AUTO) -> BConv2dDesc:
+              out_type=OUT_FLOAT32, activation=ACT_NONE, kernel_choice=KERNEL_AUTO, weights_packed=0) -> BConv2dDesc:
     return BConv2dDesc(batch, in_h, in_w, in_c, out_c, kernel[0], kernel[1], stride[0], stride[1],
-                       padding, out_type, activation, kernel_choice)
+                       padding, out_type, activation, kernel_choice, weights_packed)
 
 
 def lce_bconv2d_out_shape(desc: BConv2dDesc) -> Tuple[int, int]:
@@ -140,6 +144,8 @@ def lce_bconv2d(desc: BConv2dDesc, input: torch.Tensor, weights: torch.Tensor,
             out = torch.empty((desc.batch, oh, ow, desc.out_c), dtype=torch.int32, device=input.device)
     expect_in = desc.batch * desc.in_h * desc.in_w * _words(desc.in_c)
     expect_w = desc.out_c * desc.kernel_h * desc.kernel_w * _words(desc.in_c)
+    if desc.weights_packed:
+        expect_w = lce_bconv2d_packed_weights_bytes(desc) // 4
     if input.numel() != expect_in or weights.numel() != expect_w:
         raise ValueError("input / weights size does not match the descriptor")
     out_dtype = torch.float32 if desc.out_type == OUT_FLOAT32 else torch.int32
@@ -149,6 +155,21 @@ def lce_bconv2d(desc: BConv2dDesc, input: torch.Tensor, weights: torch.Tensor,
         _dev(bias, torch.float32, "bias") if bias is not None else None,
         _dev(thresholds, torch.int32, "thresholds") if thresholds is not None else None,
         _dev(out, out_dtype, "out"), _stream()), "lce_bconv2d")
+    return out
+
+
+def lce_bconv2d_packed_weights_bytes(desc: BConv2dDesc) -> int:
+    return int(library().lce_bconv2d_packed_weights_bytes(ctypes.byref(desc)))
+
+
+def lce_bconv2d_pack_weights(desc: BConv2dDesc, weights: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Load-time weight packing; returns the packed buffer (int32 words) to pass as `weights`
+    together with a descriptor whose weights_packed is 1."""
+    nbytes = lce_bconv2d_packed_weights_bytes(desc)
+    if out is None:
+        out = torch.empty(nbytes // 4, dtype=torch.int32, device=weights.device)
+    _check(library().lce_bconv2d_pack_weights(ctypes.byref(desc), _dev(weights, torch.int32, "weights"),
+                                              _dev(out, torch.int32, "packed"), _stream()), "lce_bconv2d_pack_weights")
     return out
 
 

@@ -19,19 +19,28 @@ lce_status check_conv_args(const lce_bconv2d_desc *desc, ConvGeom *g, const void
     return LCE_OK;
 }
 
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+size_t plain_weight_bytes(const ConvGeom &g) { return round_up((size_t)g.Cout * g.KH * g.KW * g.Cw * 4, 256); }
+
 lce_status dispatch(const lce_bconv2d_desc *desc, const ConvGeom &g, const uint32_t *input, const uint32_t *weights,
                     const float *multiplier, const float *bias, const int32_t *thresholds, void *output,
                     cudaStream_t s)
 {
+    // a packed-weights buffer = [plain words, rounded up to 256 bytes][tiled image]
+    const uint32_t *image = nullptr;
+    if (desc->weights_packed) {
+        if (!aligned(weights, 256)) return LCE_ERR_ALIGNMENT;
+        if (tiled_weight_image_bytes(g) > 0)
+            image = reinterpret_cast<const uint32_t *>(reinterpret_cast<const char *>(weights) + plain_weight_bytes(g));
+    }
     if (desc->kernel == LCE_KERNEL_DIRECT)
         return launch_bconv_direct(g, input, weights, multiplier, bias, thresholds, output, s);
-    lce_status st = launch_bconv_tiled(g, input, weights, multiplier, bias, thresholds, output, s);
+    lce_status st = launch_bconv_tiled(g, input, weights, image, multiplier, bias, thresholds, output, s);
     if (st == LCE_ERR_UNSUPPORTED && desc->kernel == LCE_KERNEL_AUTO)
         st = launch_bconv_direct(g, input, weights, multiplier, bias, thresholds, output, s);
     return st;
 }
-
-size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct HostLayout {
     size_t in, w, mult, bias, thr, out, total;
@@ -101,6 +110,29 @@ extern "C" lce_status lce_bconv2d(const lce_bconv2d_desc *desc, const uint32_t *
     return dispatch(desc, g, input, weights, multiplier, bias, thresholds, output, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" size_t lce_bconv2d_packed_weights_bytes(const lce_bconv2d_desc *desc)
+{
+    lce::ConvGeom g;
+    if (lce::make_geom(desc, &g) != LCE_OK) return 0;
+    return lce::plain_weight_bytes(g) + lce::tiled_weight_image_bytes(g);
+}
+
+extern "C" lce_status lce_bconv2d_pack_weights(const lce_bconv2d_desc *desc, const uint32_t *weights, void *packed,
+                                               void *stream)
+{
+    using namespace lce;
+    ConvGeom g;
+    lce_status st = make_geom(desc, &g);
+    if (st != LCE_OK) return st;
+    if (!weights || !packed) return LCE_ERR_INVALID_ARG;
+    if (!aligned(weights, 4) || !aligned(packed, 256)) return LCE_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t plain = (size_t)g.Cout * g.KH * g.KW * g.Cw * 4;
+    if (cudaMemcpyAsync(packed, weights, plain, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return LCE_ERR_CUDA;
+    if (tiled_weight_image_bytes(g) == 0) return LCE_OK;
+    return launch_pack_weights_tiled(g, weights, reinterpret_cast<uint32_t *>(static_cast<char *>(packed) + plain_weight_bytes(g)), s);
+}
+
 extern "C" size_t lce_bconv2d_host_workspace_bytes(const lce_bconv2d_desc *desc)
 {
     lce::ConvGeom g;
@@ -116,7 +148,7 @@ extern "C" lce_status lce_bconv2d_host(const lce_bconv2d_desc *desc, const uint3
     ConvGeom g;
     lce_status st = check_conv_args(desc, &g, input, weights, multiplier, bias, thresholds, output);
     if (st != LCE_OK) return st;
-    if (!workspace) return LCE_ERR_INVALID_ARG;
+    if (!workspace || desc->weights_packed) return LCE_ERR_INVALID_ARG;
     if (!aligned(workspace, 256)) return LCE_ERR_ALIGNMENT;
     const HostLayout L = host_layout(g);
     if (workspace_bytes < L.total) return LCE_ERR_WORKSPACE;

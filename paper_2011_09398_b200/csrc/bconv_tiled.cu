@@ -1,38 +1,48 @@
-// LceBConv2d, tiled XOR/POPC kernels (paper Section 3.2: im2col -> BGEMM -> output transform,
-// here as one implicit-GEMM kernel: the im2col matrix is never materialised, the accumulators
-// never leave registers before the output transform).
+// LceBConv2d, tiled XOR/POPC kernel for 3x3 filters (paper Section 3.2: im2col -> BGEMM -> output
+// transform, here as one implicit-GEMM kernel: the im2col matrix is never materialised and the
+// accumulators never leave registers before the output transform).
 //
-// 3x3 kernel, stride 1 or 2, any channel counts and image sizes:
+// Stride 1 or 2, any channel counts and image sizes:
 //   * a CTA owns a run of consecutive output pixels (flat (n, oh, ow) order) times 64 output
 //     channels; a warp works on 4 pixels x 8 channel groups at a time, a thread on TP pixels
 //     (16 apart in the flat order) x 8 channels, i.e. TP x 8 accumulators in registers;
 //   * the CTA first copies the packed input rows its pixels need into shared memory, one plane
 //     per channel word, in "padded image" coordinates: rows/columns outside the image hold zero
 //     words, which is exactly the paper's one-padding (a zero bit is +1.0);
-//   * the weights of its 64 channels are turned into carry-save operands (csa.cuh) while they
-//     are copied to shared memory;
+//   * the weights of its 64 channels arrive as carry-save operands (csa.cuh): either copied in
+//     16-byte pieces from a buffer prepared once by lce_bconv2d_pack_weights (the paper's
+//     load-time "weight packing"), or derived on the fly from the plain packed weights;
 //   * for every channel word the nine taps of a (pixel, channel) pair form one nine-word
 //     carry-save group: 16 LOP3 + 4 POPC + 4 IMAD instead of 9 XOR + 9 POPC + 9 adds.  The
 //     activation-side operands of the thread's TP pixels sit in registers for the whole channel
 //     word; the weight-side operands of one channel are read from shared memory once and used
 //     for all TP pixels (shared-memory bandwidth, not issue slots, is what this ordering saves);
 //   * epilogue: acc = K - 2*count, then float multiply-add, threshold + bit-pack, or raw int32.
+#include <stdlib.h>
+
 #include "common.cuh"
 #include "csa.cuh"
 
 namespace lce {
 namespace {
 
-constexpr int kThreads = 128;       // 4 warps; a warp = 4 pixels x 8 channel groups
-constexpr int kPixPerStep = 16;     // pixels the CTA works on at a time (4 warps x 4)
+#ifndef LCE_WARPS
+#define LCE_WARPS 4
+#endif
+constexpr int kWarps = LCE_WARPS;
+constexpr int kThreads = 32 * kWarps;    // a warp = 4 pixels x 8 channel groups
+constexpr int kPixPerStep = 4 * kWarps;  // pixels the CTA works on at a time
 constexpr int kChanPerCta = 64;
 constexpr int kChanPerThread = 8;
+constexpr int kChanGroups = kChanPerCta / kChanPerThread;
 constexpr int kWRow = 12;           // 9 carry-save operand words per (channel word, channel) + 3 pad
 constexpr int kWGroupStride = kChanPerThread * kWRow + 4;  // +4 words: the 8 channel groups hit distinct banks
+constexpr int kWsumWords = kChanPerCta * 9;                // per-tap weight sums of a channel block
 
 struct TiledParams {
     const uint32_t *in;
-    const uint32_t *w;
+    const uint32_t *w;         // plain packed weights [Cout][3][3][Cw]
+    const uint32_t *w_image;   // packed-weights image (see image_block_words), or nullptr
     const float *mult;
     const float *bias;
     const int32_t *thr;
@@ -40,8 +50,20 @@ struct TiledParams {
     int32_t N, H, W, Cin, Cw, Cout, Cow, OH, OW, pt, pl;
     int32_t tile_pixels;  // flat output pixels per CTA, a multiple of kPixPerStep * TP
     int32_t M, Hp, Wp, pitch, plane;
+    int32_t cw_shift;     // log2(Cw) when Cw is a power of two, else -1
     int32_t padding, out_type, activation;
 };
+
+// Shared-memory / packed-image offset (in words) of the operands of (channel word, channel).
+__host__ __device__ __forceinline__ int32_t w_offset(int cw, int ch)
+{
+    return cw * kChanGroups * kWGroupStride + (ch >> 3) * kWGroupStride + (ch & 7) * kWRow;
+}
+// One channel block of the packed image: operands for every channel word, then the per-tap sums.
+__host__ __device__ __forceinline__ int64_t image_block_words(int Cw)
+{
+    return (int64_t)Cw * kChanGroups * kWGroupStride + kWsumWords;
+}
 
 template <int BYTE_OFF>
 __device__ __forceinline__ uint4 lds128(uint32_t saddr)
@@ -59,6 +81,11 @@ __device__ __forceinline__ uint32_t lds32(uint32_t saddr)
     asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(saddr), "n"(BYTE_OFF));
     return v;
 }
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
+{
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
 
 template <int J>
 __device__ __forceinline__ void load_w_triples(uint32_t saddr, Triple (&wt)[3])
@@ -69,11 +96,6 @@ __device__ __forceinline__ void load_w_triples(uint32_t saddr, Triple (&wt)[3])
     wt[0].all = q0.x; wt[0].pair = q0.y; wt[0].first = q0.z;
     wt[1].all = q0.w; wt[1].pair = q1.x; wt[1].first = q1.y;
     wt[2].all = q1.z; wt[2].pair = q1.w; wt[2].first = q2;
-}
-
-__device__ __forceinline__ int32_t w_smem_offset(int cw, int ch)
-{
-    return cw * (kChanPerCta / kChanPerThread) * kWGroupStride + (ch >> 3) * kWGroupStride + (ch & 7) * kWRow;
 }
 
 template <int J, int TP>
@@ -95,76 +117,135 @@ struct ChannelLoop<kChanPerThread, TP> {
                                                uint32_t (&)[TP][kChanPerThread]) {}
 };
 
+// Nine plain weight words of one (channel, channel word) -> nine carry-save operand words.
+__device__ __forceinline__ void store_w_operands(const uint32_t (&wv)[9], uint32_t *dst)
+{
+#pragma unroll
+    for (int g = 0; g < 3; ++g) {
+        const Triple t = make_triple(wv[3 * g], wv[3 * g + 1], wv[3 * g + 2]);
+        dst[3 * g] = t.all;
+        dst[3 * g + 1] = t.pair;
+        dst[3 * g + 2] = t.first;
+    }
+    dst[9] = dst[10] = dst[11] = 0u;
+}
+
+// Load-time weight packing: plain [Cout][3][3][Cw] -> per channel block of 64 the exact
+// shared-memory image the convolution kernel wants (operands, then per-tap sums).
+__global__ void __launch_bounds__(128)
+pack_weights_kernel(const uint32_t *__restrict__ w, uint32_t *__restrict__ image, int32_t Cout, int32_t Cw,
+                    int32_t Cin, int32_t chan_blocks)
+{
+    const int64_t entries = (int64_t)chan_blocks * kChanPerCta * Cw;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < entries;
+         e += (int64_t)gridDim.x * blockDim.x) {
+        const int cw = (int)(e % Cw);
+        const int64_t c = e / Cw;  // global channel (may be >= Cout in the last block)
+        const int cb = (int)(c / kChanPerCta), ch = (int)(c % kChanPerCta);
+        uint32_t wv[9];
+#pragma unroll
+        for (int t = 0; t < 9; ++t) wv[t] = c < Cout ? w[(c * 9 + t) * Cw + cw] : 0u;
+        uint32_t *block = image + cb * image_block_words(Cw);
+        store_w_operands(wv, block + w_offset(cw, ch));
+        if ((ch & 7) == 7) {  // the 4 pad words after every 8 channels
+            uint32_t *pad = block + w_offset(cw, ch) + kWRow;
+            pad[0] = pad[1] = pad[2] = pad[3] = 0u;
+        }
+        if (cw == 0) {
+            // sum over the true channels of one tap's weights = Cin - 2*popcount (pad bits are 0)
+            int32_t *wsum = reinterpret_cast<int32_t *>(block + (int64_t)Cw * kChanGroups * kWGroupStride);
+            for (int t = 0; t < 9; ++t) {
+                int32_t cnt = 0;
+                if (c < Cout)
+                    for (int j = 0; j < Cw; ++j) cnt += __popc(w[(c * 9 + t) * Cw + j]);
+                wsum[ch * 9 + t] = c < Cout ? Cin - 2 * cnt : 0;
+            }
+        }
+    }
+}
+
 template <int STRIDE, int TP>
-__global__ void __launch_bounds__(kThreads, (TP <= 4 ? 4 : (TP <= 7 ? 3 : 2)))
+__global__ void __launch_bounds__(kThreads, (TP <= 2 ? 24 : 16) / kWarps)
 bconv3x3_kernel(const TiledParams p)
 {
     extern __shared__ __align__(16) uint32_t smem[];
-    uint32_t *sW = smem;                                                       // [Cw][8 groups][kWGroupStride]
-    uint32_t *sA = smem + p.Cw * (kChanPerCta / kChanPerThread) * kWGroupStride;  // [Cw][nv][pitch]
-    int32_t *sWsum = reinterpret_cast<int32_t *>(sA + p.Cw * p.plane);            // [64][9], zero-padding only
+    const int w_words = p.Cw * kChanGroups * kWGroupStride;
+    uint32_t *sW = smem;                                           // [Cw][8 groups][kWGroupStride]
+    int32_t *sWsum = reinterpret_cast<int32_t *>(smem + w_words);  // [64][9]
+    uint32_t *sA = smem + w_words + kWsumWords;                    // [Cw][nv][pitch]
 
     const int tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5;
     const int m0 = blockIdx.x * p.tile_pixels;
     const int m_end = min(m0 + p.tile_pixels, p.M);
     const int ch0 = blockIdx.y * kChanPerCta;
 
+    // ---- weights ----------------------------------------------------------------------------
+    if (p.w_image != nullptr) {
+        // prepared image: a plain 16-byte asynchronous copy of this channel block
+        const int words = (p.padding == LCE_PAD_SAME_ZERO) ? w_words + kWsumWords : w_words;
+        const uint32_t *src = p.w_image + blockIdx.y * image_block_words(p.Cw);
+        for (int e = tid * 4; e < words; e += kThreads * 4) cp_async16(smem + e, src + e);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    } else {
+        for (int e = tid; e < kChanPerCta * p.Cw; e += kThreads) {
+            const int ch = e / p.Cw;
+            const int cw = e - ch * p.Cw;
+            uint32_t wv[9];
+#pragma unroll
+            for (int t = 0; t < 9; ++t)
+                wv[t] = (ch0 + ch < p.Cout) ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + t) * p.Cw + cw) : 0u;
+            store_w_operands(wv, sW + w_offset(cw, ch));
+        }
+        if (p.padding == LCE_PAD_SAME_ZERO) {
+            for (int e = tid; e < kWsumWords; e += kThreads) {
+                const int ch = e / 9, t = e - ch * 9;
+                int32_t cnt = 0;
+                if (ch0 + ch < p.Cout)
+                    for (int cw = 0; cw < p.Cw; ++cw)
+                        cnt += __popc(__ldg(p.w + ((int64_t)(ch0 + ch) * 9 + t) * p.Cw + cw));
+                sWsum[e] = p.Cin - 2 * cnt;
+            }
+        }
+    }
+
+    // ---- input rows: global [n][iy][ix][cw] -> shared [cw][v][x] ---------------------------------
     // virtual (padded-image) rows this CTA needs: v = n*Hp + oh*stride + ky
     const int r_first = m0 / p.OW, r_last = (m_end - 1) / p.OW;
     const int v_first = (r_first / p.OH) * p.Hp + (r_first % p.OH) * STRIDE;
     const int v_last = (r_last / p.OH) * p.Hp + (r_last % p.OH) * STRIDE + 2;
     const int nv = v_last - v_first + 1;
-
-    // ---- stage the input rows: global [n][iy][ix][cw] -> shared [cw][v][x] -------------------
     {
-        const int row_words = p.Wp * p.Cw;
-        for (int v = tid >> 5; v < nv; v += kThreads / 32) {
+        const int row_words = p.W * p.Cw;
+        for (int v = warp; v < nv; v += kThreads / 32) {
             const int va = v_first + v;
             const int n = va / p.Hp;
             const int iy = va - n * p.Hp - p.pt;
-            const bool row_ok = n < p.N && iy >= 0 && iy < p.H;
-            const uint32_t *src = p.in + ((int64_t)n * p.H + iy) * p.W * p.Cw;
-            for (int e = tid & 31; e < row_words; e += 32) {
-                const int x = e / p.Cw;
-                const int cw = e - x * p.Cw;
-                const int ix = x - p.pl;
-                uint32_t val = 0u;
-                if (row_ok && ix >= 0 && ix < p.W) val = __ldg(src + ix * p.Cw + cw);
-                sA[cw * p.plane + v * p.pitch + x] = val;
+            uint32_t *dst_row = sA + v * p.pitch;
+            if (n < p.N && iy >= 0 && iy < p.H) {
+                const uint32_t *src = p.in + ((int64_t)n * p.H + iy) * row_words;
+                // the image's words of this row, coalesced; the columns left and right of it are zero
+                for (int e = lane; e < row_words; e += 32) {
+                    int ix, cw;
+                    if (p.cw_shift >= 0) { ix = e >> p.cw_shift; cw = e & (p.Cw - 1); }
+                    else { ix = e / p.Cw; cw = e - ix * p.Cw; }
+                    dst_row[cw * p.plane + ix + p.pl] = __ldg(src + e);
+                }
+                const int edge = p.Wp - p.W;  // pad columns: pl on the left, the rest on the right
+                for (int e = lane; e < edge * p.Cw; e += 32) {
+                    const int cw = e / edge, k = e - cw * edge;
+                    dst_row[cw * p.plane + (k < p.pl ? k : p.W + k)] = 0u;
+                }
+            } else {
+                for (int e = lane; e < p.Wp * p.Cw; e += 32) {
+                    const int cw = e / p.Wp, x = e - cw * p.Wp;
+                    dst_row[cw * p.plane + x] = 0u;
+                }
             }
-        }
-    }
-    // ---- stage the weights as carry-save operands: [ch][ky][kx][cw] -> [cw][ch][9 (+3)] -------
-    for (int e = tid; e < kChanPerCta * p.Cw; e += kThreads) {
-        const int ch = e / p.Cw;
-        const int cw = e - ch * p.Cw;
-        uint32_t wv[9];
-#pragma unroll
-        for (int t = 0; t < 9; ++t)
-            wv[t] = (ch0 + ch < p.Cout) ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + t) * p.Cw + cw) : 0u;
-        uint32_t *dst = sW + w_smem_offset(cw, ch);
-#pragma unroll
-        for (int g = 0; g < 3; ++g) {
-            const Triple t = make_triple(wv[3 * g], wv[3 * g + 1], wv[3 * g + 2]);
-            dst[3 * g] = t.all;
-            dst[3 * g + 1] = t.pair;
-            dst[3 * g + 2] = t.first;
-        }
-        dst[9] = dst[10] = dst[11] = 0u;
-    }
-    if (p.padding == LCE_PAD_SAME_ZERO) {
-        // sum over the true channels of one tap's weights = Cin - 2*popcount (pad bits are 0)
-        for (int e = tid; e < kChanPerCta * 9; e += kThreads) {
-            const int ch = e / 9, t = e - ch * 9;
-            int32_t cnt = 0;
-            if (ch0 + ch < p.Cout)
-                for (int cw = 0; cw < p.Cw; ++cw) cnt += __popc(__ldg(p.w + ((int64_t)(ch0 + ch) * 9 + t) * p.Cw + cw));
-            sWsum[e] = p.Cin - 2 * cnt;
         }
     }
 
     // ---- this thread's channels and pixels ---------------------------------------------------
-    const int lane = tid & 31, warp = tid >> 5;
     const int px = lane >> 3, cg = lane & 7;
     const int chan = ch0 + cg * kChanPerThread;
     const int K = 9 * p.Cin;
@@ -174,19 +255,21 @@ bconv3x3_kernel(const TiledParams p)
     k124.four = p.N > 0 ? 4u : p.Cin;
     asm volatile("" : "+r"(k124.one), "+r"(k124.two), "+r"(k124.four));
 
-    // running (n, oh, ow) of this lane's next pixel; pixels of one lane are kPixPerStep apart
-    int m_next = m0 + warp * 4 + px;
-    int ow, voh;  // voh = n*Hp + oh*STRIDE: the pixel's first virtual row
+    // running position of this lane's next pixel; the pixels of one lane are kPixPerStep apart
+    int m_next = m0 + warp * 4 + px;  // lanes of a warp: 4 neighbouring pixels
+    int ow, voh, oh_left;  // voh = n*Hp + oh*STRIDE: the pixel's first virtual row
     {
         const int r = m_next / p.OW;
         ow = m_next - r * p.OW;
         const int n = r / p.OH;
-        voh = n * p.Hp + (r - n * p.OH) * STRIDE;
+        const int oh = r - n * p.OH;
+        voh = n * p.Hp + oh * STRIDE;
+        oh_left = p.OH - 1 - oh;  // rows left in the image after this one
     }
-    int oh_left = p.OH - 1 - (m_next / p.OW) % p.OH;  // rows left in the image after this one
     const int a_base_first = ((r_first / p.OH) * p.Hp + (r_first % p.OH) * STRIDE - v_first) * p.pitch +
                              (m0 - r_first * p.OW) * STRIDE;
     const uint32_t w_saddr0 = (uint32_t)__cvta_generic_to_shared(sW + cg * kWGroupStride);
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
 
     for (int base = m0; base < m0 + p.tile_pixels; base += kPixPerStep * TP) {
@@ -199,7 +282,7 @@ bconv3x3_kernel(const TiledParams p)
             ow += kPixPerStep;
             while (ow >= p.OW) {
                 ow -= p.OW;
-                if (oh_left == 0) { oh_left = p.OH - 1; voh += 3; }   // next image: Hp - (OH-1)*STRIDE = 3
+                if (oh_left == 0) { oh_left = p.OH - 1; voh += 3; }  // next image: Hp - (OH-1)*STRIDE = 3
                 else { --oh_left; voh += STRIDE; }
             }
         }
@@ -221,7 +304,7 @@ bconv3x3_kernel(const TiledParams p)
                     at[i][ky] = make_triple(row[0], row[1], row[2]);
                 }
             ChannelLoop<0, TP>::run(w_saddr, at, k124, acc);
-            w_saddr += (kChanPerCta / kChanPerThread) * kWGroupStride * 4;
+            w_saddr += kChanGroups * kWGroupStride * 4;
             plane += p.plane;
         }
 
@@ -302,15 +385,10 @@ bconv3x3_kernel(const TiledParams p)
     }
 }
 
-#ifndef LCE_TP
-#define LCE_TP 4
-#endif
-constexpr int kTP = LCE_TP;  // pixels per thread
-
-template <int STRIDE>
+template <int STRIDE, int TP>
 lce_status launch3x3(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStream_t s)
 {
-    auto kernel = bconv3x3_kernel<STRIDE, kTP>;
+    auto kernel = bconv3x3_kernel<STRIDE, TP>;
     if (smem_bytes > 48 * 1024) {
         // opt in to the large dynamic shared memory carve-out
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
@@ -320,9 +398,13 @@ lce_status launch3x3(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStr
     return launch_status();
 }
 
+// CTAs of 128 threads that the register file lets share an SM, per pixels-per-thread variant
+// (must match the __launch_bounds__ of the kernel).
+int reg_limited_ctas(int tp) { return (tp <= 2 ? 24 : 16) / kWarps; }
+
 size_t smem_bytes_for(const ConvGeom &g, const TiledParams &p)
 {
-    return ((size_t)g.Cw * (kChanPerCta / kChanPerThread) * kWGroupStride + (size_t)g.Cw * p.plane + kChanPerCta * 9) * 4;
+    return ((size_t)g.Cw * kChanGroups * kWGroupStride + kWsumWords + (size_t)g.Cw * p.plane) * 4;
 }
 
 void set_tile(const ConvGeom &g, TiledParams *p, int tile_pixels)
@@ -334,58 +416,103 @@ void set_tile(const ConvGeom &g, TiledParams *p, int tile_pixels)
     p->plane = nv_max * p->pitch;
 }
 
+bool tiled_covers(const ConvGeom &g)
+{
+    return g.KH == 3 && g.KW == 3 && g.sh == g.sw && g.sh <= 2 && g.M < (1ll << 31) - 256 &&
+           (g.Cout + kChanPerCta - 1) / kChanPerCta <= 65535;
+}
+
 }  // namespace
 
-lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const float *mult,
-                              const float *bias, const int32_t *thr, void *out, cudaStream_t s)
+size_t tiled_weight_image_bytes(const ConvGeom &g)
 {
-    if (g.KH != 3 || g.KW != 3 || g.sh != g.sw || g.sh > 2) return LCE_ERR_UNSUPPORTED;
+    if (!tiled_covers(g)) return 0;
+    const int chan_blocks = (g.Cout + kChanPerCta - 1) / kChanPerCta;
+    return (size_t)chan_blocks * image_block_words(g.Cw) * 4;
+}
+
+lce_status launch_pack_weights_tiled(const ConvGeom &g, const uint32_t *w, uint32_t *image, cudaStream_t s)
+{
+    if (!tiled_covers(g)) return LCE_ERR_UNSUPPORTED;
+    const int chan_blocks = (g.Cout + kChanPerCta - 1) / kChanPerCta;
+    const int64_t entries = (int64_t)chan_blocks * kChanPerCta * g.Cw;
+    int blocks = (int)((entries + 127) / 128);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    pack_weights_kernel<<<blocks, 128, 0, s>>>(w, image, g.Cout, g.Cw, g.Cin, chan_blocks);
+    return launch_status();
+}
+
+lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const uint32_t *w_image,
+                              const float *mult, const float *bias, const int32_t *thr, void *out, cudaStream_t s)
+{
+    if (!tiled_covers(g)) return LCE_ERR_UNSUPPORTED;
     // 128-bit epilogue stores need a 16-byte aligned output when the channel count allows them
     if ((g.Cout & 3) == 0 && g.out_type != LCE_OUT_BITPACKED && !aligned(out, 16)) return LCE_ERR_UNSUPPORTED;
-    if (g.M >= (1ll << 31) - 256) return LCE_ERR_UNSUPPORTED;
+    if (w_image && !aligned(w_image, 16)) return LCE_ERR_ALIGNMENT;
     TiledParams p{};
-    p.in = in; p.w = w; p.mult = mult; p.bias = bias; p.thr = thr; p.out = out;
+    p.in = in; p.w = w; p.w_image = w_image; p.mult = mult; p.bias = bias; p.thr = thr; p.out = out;
     p.N = g.N; p.H = g.H; p.W = g.W; p.Cin = g.Cin; p.Cw = g.Cw; p.Cout = g.Cout; p.Cow = g.Cow;
     p.OH = g.OH; p.OW = g.OW; p.pt = g.pt; p.pl = g.pl;
     p.padding = g.padding; p.out_type = g.out_type; p.activation = g.activation;
     p.M = (int32_t)g.M;
     p.Hp = (g.OH - 1) * g.sh + 3;
     p.Wp = (g.OW - 1) * g.sh + 3;
+    if (p.Wp < g.W + g.pl) p.Wp = g.W + g.pl;  // staging writes the whole image row; columns past the taps are unused
     p.pitch = p.Wp | 1;  // odd pitch: the 4 pixels of a warp in 4 different rows hit 4 different banks
+    p.cw_shift = -1;
+    for (int b = 0; b < 16; ++b)
+        if ((1 << b) == g.Cw) p.cw_shift = b;
     const int chan_blocks = (g.Cout + kChanPerCta - 1) / kChanPerCta;
-    if (chan_blocks > 65535) return LCE_ERR_UNSUPPORTED;
 
-    // Tile size: the largest of {128, 112, ..., 16} flat pixels whose shared memory lets at least
-    // three CTAs share an SM, then shrunk while that fills the machine's CTA slots more evenly.
+    // Pixels per thread (TP) and rounds per CTA: a CTA covers 16*TP*rounds flat pixels.  Pick the
+    // pair whose CTA count fills the machine's CTA slots most evenly; the cost of a choice is
+    // (number of waves) x (per-CTA main-loop work + a fixed staging cost), in pixel units.
     int sms = 148;
     {
         int dev = 0;
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     }
-    int best_tile = 0;
+    int forced_tp = 0, forced_rounds = 0;
+#ifdef LCE_TUNING
+    if (const char *e = getenv("LCE_TP")) forced_tp = atoi(e);
+    if (const char *e = getenv("LCE_ROUNDS")) forced_rounds = atoi(e);
+#endif
+    int best_tile = 0, best_tp = 0;
     double best_cost = 0;
-    const int unit = kPixPerStep * kTP;
-    for (int tile = (128 / unit > 0 ? 128 / unit : 1) * unit; tile >= unit; tile -= unit) {
-        set_tile(g, &p, tile);
-        const size_t smem = smem_bytes_for(g, p);
-        if (smem > 110 * 1024) continue;
-        int per_sm = (int)((220 * 1024) / (smem + 1024));
-        const int reg_limit = kTP <= 4 ? 4 : (kTP <= 7 ? 3 : 2);
-        if (per_sm > reg_limit) per_sm = reg_limit;
-        const int64_t ctas = ((g.M + tile - 1) / tile) * chan_blocks;
-        const int64_t slots = (int64_t)sms * per_sm;
-        const int64_t waves = (ctas + slots - 1) / slots;
-        // time ~ waves * (per-CTA work + fixed staging cost), per-CTA work ~ tile pixels
-        const double staging = 12.0 + 64.0 / (9.0 * g.Cw) ;  // in "pixels" of main-loop time; rough
-        const double cost = (double)waves * (tile + staging) / per_sm;
-        if (best_tile == 0 || cost < best_cost) { best_tile = tile; best_cost = cost; }
+    for (int tp = 2; tp <= 4; ++tp) {
+        if (forced_tp && tp != forced_tp) continue;
+        const int unit = kPixPerStep * tp;
+        for (int rounds = 1; rounds <= 4; ++rounds) {
+            if (forced_rounds && rounds != forced_rounds) continue;
+            const int tile = unit * rounds;
+            set_tile(g, &p, tile);
+            const size_t smem = smem_bytes_for(g, p);
+            if (smem > 110 * 1024) continue;
+            int per_sm = (int)((220 * 1024) / (smem + 1024));
+            if (per_sm > reg_limited_ctas(tp)) per_sm = reg_limited_ctas(tp);
+            const int64_t ctas = ((g.M + tile - 1) / tile) * chan_blocks;
+            const int64_t slots = (int64_t)sms * per_sm;
+            const int64_t waves = (ctas + slots - 1) / slots;
+            const double staging = 8.0 + 96.0 / (9.0 * g.Cw);
+            // fewer pixels per thread re-read the weight operands from shared memory more often
+            const double smem_penalty = tp == 2 ? 1.08 : (tp == 3 ? 1.03 : 1.0);
+            const double cost = (double)waves * (tile * smem_penalty + staging) / per_sm;
+            if (best_tile == 0 || cost < best_cost) { best_tile = tile; best_tp = tp; best_cost = cost; }
+        }
     }
     if (best_tile == 0) return LCE_ERR_UNSUPPORTED;
     set_tile(g, &p, best_tile);
     const size_t smem_bytes = smem_bytes_for(g, p);
     const int64_t ctas = (g.M + best_tile - 1) / best_tile;
     dim3 grid((unsigned)ctas, (unsigned)chan_blocks, 1);
-    return g.sh == 1 ? launch3x3<1>(p, smem_bytes, grid, s) : launch3x3<2>(p, smem_bytes, grid, s);
+    if (g.sh == 1) {
+        if (best_tp == 2) return launch3x3<1, 2>(p, smem_bytes, grid, s);
+        if (best_tp == 3) return launch3x3<1, 3>(p, smem_bytes, grid, s);
+        return launch3x3<1, 4>(p, smem_bytes, grid, s);
+    }
+    if (best_tp == 2) return launch3x3<2, 2>(p, smem_bytes, grid, s);
+    if (best_tp == 3) return launch3x3<2, 3>(p, smem_bytes, grid, s);
+    return launch3x3<2, 4>(p, smem_bytes, grid, s);
 }
 
 }  // namespace lce

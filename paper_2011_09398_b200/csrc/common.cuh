@@ -43,6 +43,7 @@ inline lce_status make_geom(const lce_bconv2d_desc *d, ConvGeom *g)
     if (d->out_type < LCE_OUT_FLOAT32 || d->out_type > LCE_OUT_INT32) return LCE_ERR_INVALID_ARG;
     if (d->activation < LCE_ACT_NONE || d->activation > LCE_ACT_RELU) return LCE_ERR_INVALID_ARG;
     if (d->kernel < LCE_KERNEL_AUTO || d->kernel > LCE_KERNEL_TILED) return LCE_ERR_INVALID_ARG;
+    if (d->weights_packed != 0 && d->weights_packed != 1) return LCE_ERR_INVALID_ARG;
     Axis ah = axis_geometry(d->in_h, d->kernel_h, d->stride_h, d->padding);
     Axis aw = axis_geometry(d->in_w, d->kernel_w, d->stride_w, d->padding);
     if (ah.out <= 0 || aw.out <= 0) return LCE_ERR_INVALID_ARG;
@@ -72,7 +73,11 @@ inline lce_status launch_status()
 lce_status launch_bconv_direct(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const float *mult,
                                const float *bias, const int32_t *thr, void *out, cudaStream_t s);
 // Returns LCE_ERR_UNSUPPORTED without launching when the tiled kernel does not cover the shape.
-lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const float *mult,
-                              const float *bias, const int32_t *thr, void *out, cudaStream_t s);
+// w_image: the tiled part of a packed-weights buffer, or nullptr to derive operands from `w`.
+lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const uint32_t *w_image,
+                              const float *mult, const float *bias, const int32_t *thr, void *out, cudaStream_t s);
+// Bytes of the tiled kernel's weight image for this geometry (0 if the kernel does not cover it).
+size_t tiled_weight_image_bytes(const ConvGeom &g);
+lce_status launch_pack_weights_tiled(const ConvGeom &g, const uint32_t *w, uint32_t *image, cudaStream_t s);
 
 }  // namespace lce

@@ -31,14 +31,15 @@ def guards_intact(whole, fill) -> bool:
     return bool((whole[:64] == fill).all().item() and (whole[-64:] == fill).all().item())
 
 
-def run_bconv(a_words, w_words, spec_kwargs, mult=None, bias=None, thr=None, kernel_choice=lce.KERNEL_AUTO):
+def run_bconv(a_words, w_words, spec_kwargs, mult=None, bias=None, thr=None, kernel_choice=lce.KERNEL_AUTO,
+              packed=False):
     """a_words/w_words: numpy uint32. Returns the numpy output (uint32 words / int32 / float32),
     after checking the guard words around the output buffer."""
     N, H, W, _ = a_words.shape
     Cout, KH, KW, _ = w_words.shape
     desc = lce.make_desc(N, H, W, spec_kwargs["in_c"], Cout, (KH, KW), spec_kwargs.get("stride", (1, 1)),
                          spec_kwargs.get("padding", lce.PAD_SAME_ONE), spec_kwargs["out_type"],
-                         spec_kwargs.get("activation", lce.ACT_NONE), kernel_choice)
+                         spec_kwargs.get("activation", lce.ACT_NONE), kernel_choice, 1 if packed else 0)
     oh, ow = lce.lce_bconv2d_out_shape(desc)
     ot = spec_kwargs["out_type"]
     if ot == lce.OUT_FLOAT32:
@@ -48,7 +49,10 @@ def run_bconv(a_words, w_words, spec_kwargs, mult=None, bias=None, thr=None, ker
         last = (Cout + 31) // 32 if ot == lce.OUT_BITPACKED else Cout
         whole, out = guarded((N, oh, ow, last), torch.int32, 0x5A5A5A5A)
         fill = 0x5A5A5A5A
-    lce.lce_bconv2d(desc, to_dev_words(a_words), to_dev_words(w_words),
+    w_dev = to_dev_words(w_words)
+    if packed:
+        w_dev = lce.lce_bconv2d_pack_weights(desc, w_dev)
+    lce.lce_bconv2d(desc, to_dev_words(a_words), w_dev,
                     to_dev(mult) if mult is not None else None, to_dev(bias) if bias is not None else None,
                     to_dev(thr) if thr is not None else None, out)
     torch.cuda.synchronize()

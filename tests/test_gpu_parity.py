@@ -12,7 +12,9 @@ from gpu_util import DEV, guarded, guards_intact, run_bconv, to_dev, to_dev_word
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = [lce.KERNEL_DIRECT, lce.KERNEL_AUTO]
+# (kernel choice, weights packed at load time?)
+KERNELS = [(lce.KERNEL_DIRECT, False), (lce.KERNEL_AUTO, False), (lce.KERNEL_AUTO, True)]
+KERNEL_IDS = ["direct", "auto", "auto-packed"]
 
 
 def rand_pm1(rng, shape):
@@ -77,7 +79,7 @@ FUZZ = [
 ]
 
 
-@pytest.mark.parametrize("kernel_choice", KERNELS)
+@pytest.mark.parametrize("kernel_choice", KERNELS, ids=KERNEL_IDS)
 @pytest.mark.parametrize("padding", [lce.PAD_VALID, lce.PAD_SAME_ONE, lce.PAD_SAME_ZERO])
 @pytest.mark.parametrize("shape", FUZZ)
 def test_bconv_all_output_types_match_oracle(shape, padding, kernel_choice):
@@ -89,21 +91,21 @@ def test_bconv_all_output_types_match_oracle(shape, padding, kernel_choice):
     aw, ww = oracle.bitpack_pm1(a), oracle.bitpack_pm1(w)
     acc = oracle.bconv2d_acc(a, w, (s, s), padding)
     kw = dict(in_c=Cin, stride=(s, s), padding=padding)
-    got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_INT32), kernel_choice=kernel_choice)
+    got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_INT32), kernel_choice=kernel_choice[0], packed=kernel_choice[1])
     np.testing.assert_array_equal(got, acc)
     K = k * k * Cin
     thr = np.rint(np.sqrt(K) * rng.standard_normal(Cout)).astype(np.int32)
-    got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_BITPACKED), thr=thr, kernel_choice=kernel_choice)
+    got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_BITPACKED), thr=thr, kernel_choice=kernel_choice[0], packed=kernel_choice[1])
     np.testing.assert_array_equal(got, oracle.transform_bits(acc, thr))
     mult = rng.uniform(0.5, 1.5, Cout).astype(np.float32)
     bias = (0.1 * rng.standard_normal(Cout)).astype(np.float32)
     for act in (lce.ACT_NONE, lce.ACT_RELU):
         got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_FLOAT32, activation=act), mult=mult, bias=bias,
-                        kernel_choice=kernel_choice)
+                        kernel_choice=kernel_choice[0], packed=kernel_choice[1])
         assert float_close(got, acc, mult, bias, act) == 0  # goal: bit-identical floats
 
 
-@pytest.mark.parametrize("kernel_choice", KERNELS)
+@pytest.mark.parametrize("kernel_choice", KERNELS, ids=KERNEL_IDS)
 def test_saturated_thresholds_and_pad_bits(kernel_choice):
     rng = np.random.default_rng(77)
     a, w = rand_pm1(rng, (1, 6, 6, 64)), rand_pm1(rng, (40, 3, 3, 64))
@@ -111,14 +113,14 @@ def test_saturated_thresholds_and_pad_bits(kernel_choice):
     lo = np.full(40, np.iinfo(np.int32).min, np.int32)
     hi = np.full(40, np.iinfo(np.int32).max, np.int32)
     kw = dict(in_c=64, out_type=lce.OUT_BITPACKED)
-    assert not run_bconv(aw, ww, kw, thr=lo, kernel_choice=kernel_choice).any()
-    ones = run_bconv(aw, ww, kw, thr=hi, kernel_choice=kernel_choice)
+    assert not run_bconv(aw, ww, kw, thr=lo, kernel_choice=kernel_choice[0], packed=kernel_choice[1]).any()
+    ones = run_bconv(aw, ww, kw, thr=hi, kernel_choice=kernel_choice[0], packed=kernel_choice[1])
     assert np.all(ones[..., 0] == 0xFFFFFFFF) and np.all(ones[..., 1] == 0xFF)
 
 
 # ---- config 1 and batch-reduced versions of configs 2, 3 ------------------------------------
 
-def conv_case(config, first_index, spec, kernel_choice=lce.KERNEL_AUTO):
+def conv_case(config, first_index, spec, kernel_choice=(lce.KERNEL_AUTO, True)):
     t = wl.conv_tensors(config, first_index, spec)
     x = wl.activations(config, 0, (spec.batch, spec.in_h, spec.in_w, spec.in_c))
     a_words_oracle = oracle.bitpack(x)
@@ -129,14 +131,14 @@ def conv_case(config, first_index, spec, kernel_choice=lce.KERNEL_AUTO):
     acc = oracle.bconv2d_acc(oracle.sign(x), t.w_pm1, (spec.stride, spec.stride), spec.padding)
     kw = dict(in_c=spec.in_c, stride=(spec.stride, spec.stride), padding=spec.padding, out_type=spec.out_type)
     if spec.out_type == wl.OUT_FLOAT32:
-        got = run_bconv(a_words_gpu, w_words, kw, mult=t.multiplier, bias=t.bias, kernel_choice=kernel_choice)
+        got = run_bconv(a_words_gpu, w_words, kw, mult=t.multiplier, bias=t.bias, kernel_choice=kernel_choice[0], packed=kernel_choice[1])
         assert float_close(got, acc, t.multiplier, t.bias) == 0
     else:
-        got = run_bconv(a_words_gpu, w_words, kw, thr=t.thresholds, kernel_choice=kernel_choice)
+        got = run_bconv(a_words_gpu, w_words, kw, thr=t.thresholds, kernel_choice=kernel_choice[0], packed=kernel_choice[1])
         np.testing.assert_array_equal(got, oracle.transform_bits(acc, t.thresholds))
 
 
-@pytest.mark.parametrize("kernel_choice", KERNELS)
+@pytest.mark.parametrize("kernel_choice", KERNELS, ids=KERNEL_IDS)
 def test_config1_single_conv(kernel_choice):
     conv_case(1, 1, wl.config1_spec(), kernel_choice)
 

@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of the Bconv2D hot path on B200.
+
+Workload ("config 2"): the ResNet-18-shaped 3x3 one-padded binarized convolutions
+56x56x64->64, 28x28x128->128, 14x14x256->256, 7x7x512->512 at batch 64 per GPU, each once with
+float output (per-channel multiply-add) and once with bit-packed output (per-channel thresholds),
+on inputs bit-packed beforehand from seeded N(0,1) activations and uniform +-1 weights packed at
+load time.  One step = those 8 LceBConv2d launches.  Metric: binary multiply-accumulates per
+second (N*OH*OW*Cout*KH*KW*Cin per launch, summed) over all GPUs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl lce|reference] [--no-cpu-baseline]
+
+Prints one JSON line.  With --impl reference the CPU oracle is timed instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+import numpy as np  # noqa: E402
+
+import lce_workloads as wl  # noqa: E402
+
+CONFIG = 2
+BATCH = 64
+METRIC = "bconv2d_binary_macs_per_second"
+UNIT = "binary-MAC/s"
+WORKLOAD = ("config 2: 3x3 one-padded Bconv2D sweep 56x56x64, 28x28x128, 14x14x256, 7x7x512 at batch 64 per GPU, "
+            "float and bit-packed output each (8 launches per step), pre-packed inputs, load-time packed weights")
+
+# Derived compute ceiling of the chosen pipe (integer logic + popcount), see the design doc:
+# 64 logic lanes/clk/SM, 16.75 logic instructions per nine 32-bit word operations, 32 binary MACs per word.
+LOGIC_LANES_PER_CLK_PER_SM = 64
+LOGIC_OPS_PER_9_WORDS = 16.75
+
+
+def specs():
+    return wl.config2_specs(BATCH)
+
+
+def layer_inputs(spec, index):
+    """Seeded host tensors of one launch: fp32 activations and +-1 weights plus per-channel arrays."""
+    x = wl.activations(CONFIG, 10 * index, (spec.batch, spec.in_h, spec.in_w, spec.in_c))
+    t = wl.conv_tensors(CONFIG, 10 * index + 1, spec)
+    return x, t
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.002)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def time_oracle(batch: int, passes: int = 1):
+    """Times the CPU oracle, as it stands, on all 8 launches of the workload at the given batch."""
+    import oracle
+    items = []
+    for i, spec in enumerate(wl.config2_specs(batch)):
+        x, t = layer_inputs(spec, i)
+        items.append((spec, oracle.sign(x), t))
+    oracle.bconv2d_acc(items[0][1][:1], items[0][2].w_pm1)  # load the library, warm the threads
+    macs = sum(s.binary_macs for s, _, _ in items)
+    t0 = time.perf_counter()
+    for _ in range(passes):
+        for spec, a, t in items:
+            acc = oracle.bconv2d_acc(a, t.w_pm1, (1, 1), spec.padding)
+            if spec.out_type == wl.OUT_FLOAT32:
+                oracle.transform_float(acc, t.multiplier, t.bias)
+            else:
+                oracle.transform_bits(acc, t.thresholds)
+    dt = (time.perf_counter() - t0) / passes
+    return macs / dt, dt, macs
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = len(os.sched_getaffinity(0))
+    sample_batch = 2
+    for _ in range(args.warmup):
+        time_oracle(sample_batch)
+    times, macs = [], 0
+    for _ in range(args.steps):
+        _, dt, macs = time_oracle(sample_batch)
+        times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    value = macs / (ms * 1e-3)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": f"each step = all 8 launches at batch {sample_batch} on the host cores"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"all 8 launches of config 2 at batch {sample_batch}, {args.steps} steps"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "images_per_second": 8 * sample_batch / (ms * 1e-3),
+    }
+    print(json.dumps(line))
+
+
+def run_lce(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2011_09398_b200 as lce
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- inputs: every rank draws its own batch shard (weak scaling: 64 images per GPU) ------
+    layers = []
+    h2d = d2h = 0
+    for i, spec in enumerate(specs()):
+        x, t = layer_inputs(spec, i + 100 * rank)
+        xd = torch.from_numpy(x).to(dev)
+        a = lce.lce_bitpack(xd)                                   # pre-packed input (outside the timed region)
+        wplain = lce.pack_weights(torch.from_numpy(t.w_pm1).to(dev))
+        desc = lce.make_desc(spec.batch, spec.in_h, spec.in_w, spec.in_c, spec.out_c, (3, 3), (1, 1), spec.padding,
+                             spec.out_type, lce.ACT_NONE, lce.KERNEL_AUTO, 1)
+        wpacked = lce.lce_bconv2d_pack_weights(desc, wplain)       # load-time weight packing
+        mult = torch.from_numpy(t.multiplier).to(dev)
+        bias = torch.from_numpy(t.bias).to(dev)
+        thr = torch.from_numpy(t.thresholds).to(dev)
+        if spec.out_type == wl.OUT_FLOAT32:
+            out = torch.empty((spec.batch, spec.out_h, spec.out_w, spec.out_c), dtype=torch.float32, device=dev)
+        else:
+            out = torch.empty((spec.batch, spec.out_h, spec.out_w, (spec.out_c + 31) // 32), dtype=torch.int32, device=dev)
+        # host side of the end-to-end leg: pinned buffers, plain weights
+        desc_host = lce.make_desc(spec.batch, spec.in_h, spec.in_w, spec.in_c, spec.out_c, (3, 3), (1, 1), spec.padding,
+                                  spec.out_type)
+        host = dict(
+            a=a.cpu().pin_memory(), w=wplain.cpu().pin_memory(),
+            mult=torch.from_numpy(t.multiplier).pin_memory() if spec.out_type == wl.OUT_FLOAT32 else None,
+            bias=torch.from_numpy(t.bias).pin_memory() if spec.out_type == wl.OUT_FLOAT32 else None,
+            thr=torch.from_numpy(t.thresholds).pin_memory() if spec.out_type == wl.OUT_BITPACKED else None,
+            out=torch.empty(out.shape, dtype=out.dtype).pin_memory(),
+            ws=torch.empty(lce.lce_bconv2d_host_workspace_bytes(desc_host), dtype=torch.uint8, device=dev),
+            desc=desc_host)
+        h2d += host["a"].numel() * 4 + host["w"].numel() * 4 + 4 * spec.out_c * (2 if spec.out_type == wl.OUT_FLOAT32 else 1)
+        d2h += host["out"].numel() * 4
+        layers.append(dict(spec=spec, desc=desc, a=a, w=wpacked, mult=mult, bias=bias, thr=thr, out=out, host=host))
+        del xd
+    torch.cuda.synchronize()
+
+    flush = torch.empty(256 * 1024 * 1024 // 4, dtype=torch.int32, device=dev)  # > 126 MB L2
+
+    def launch(layer):
+        s = layer["spec"]
+        if s.out_type == wl.OUT_FLOAT32:
+            lce.lce_bconv2d(layer["desc"], layer["a"], layer["w"], layer["mult"], layer["bias"], None, layer["out"])
+        else:
+            lce.lce_bconv2d(layer["desc"], layer["a"], layer["w"], None, None, layer["thr"], layer["out"])
+
+    def step(events=None):
+        for j, layer in enumerate(layers):
+            if events is not None:
+                events[j].record()
+            launch(layer)
+        if events is not None:
+            events[len(layers)].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        flush.fill_(1)
+        step()
+    barrier()
+
+    # ---- timed region: exactly K steps, L2 flushed between steps, CUDA events on the launch stream
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    all_events = [[torch.cuda.Event(enable_timing=True) for _ in range(len(layers) + 1)] for _ in range(args.steps)]
+    wall0 = time.perf_counter()
+    for k in range(args.steps):
+        flush.fill_(k)
+        step(all_events[k])
+    barrier()
+    wall = time.perf_counter() - wall0
+    clocks = sampler.stop()
+    step_ms = [ev[0].elapsed_time(ev[-1]) for ev in all_events]
+    per_launch_ms = np.array([[ev[j].elapsed_time(ev[j + 1]) for j in range(len(layers))] for ev in all_events])
+    total_ms = float(np.sum(step_ms))
+    if world > 1:
+        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    macs_per_step = sum(l["spec"].binary_macs for l in layers)
+    value = world * macs_per_step / (ms_per_step * 1e-3)
+    images_per_s = world * len(layers) * BATCH / (ms_per_step * 1e-3)
+
+    # ---- end-to-end leg: the host-buffer C-ABI entry point, copies inside the timed region ---------
+    def step_host():
+        for layer in layers:
+            h = layer["host"]
+            lce.lce_bconv2d_host(h["desc"], h["a"], h["w"], h["mult"], h["bias"], h["thr"], h["out"], h["ws"])
+
+    for _ in range(2):
+        step_host()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_steps = max(3, min(args.steps, 10))
+    t0 = time.perf_counter()
+    e0.record()
+    for _ in range(e2e_steps):
+        step_host()
+    e1.record()
+    barrier()
+    e2e_wall = time.perf_counter() - t0
+    e2e_ms = max(e0.elapsed_time(e1), 1e3 * e2e_wall) / e2e_steps  # host-synchronous calls: wall clock is the honest one
+    if world > 1:
+        tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e_value = world * macs_per_step / (e2e_ms * 1e-3)
+
+    # ---- roofline of the dominant kernel (the tiled 3x3 XOR/POPC kernel: all 8 launches) -------
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    max_mhz = clocks["sm_max_mhz"] or 1965
+    peak = sms * max_mhz * 1e6 * LOGIC_LANES_PER_CLK_PER_SM * 9.0 / LOGIC_OPS_PER_9_WORDS * 32
+    avg_launch_ms = float(per_launch_ms.mean())
+    achieved = (macs_per_step / len(layers)) / (avg_launch_ms * 1e-3)
+    probe_ops, _ = lce.lce_probe_pipe(3, 2000)
+    roofline = {
+        "bound": "alu", "kernel": "bconv3x3_kernel", "achieved": achieved / 1e12, "peak": peak / 1e12,
+        "unit": "T binary-MAC/s", "frac": achieved / peak,
+        "peak_source": "derived: SMs x max SM clock x 64 logic lanes/clk/SM x 9/16.75 word-ops per logic op x 32",
+        "measured_mix_probe": probe_ops * 32 / 1e12, "frac_of_measured_probe": achieved / (probe_ops * 32),
+        "avg_launch_us": avg_launch_ms * 1e3,
+        "traffic": None,
+        "hbm_bound_us": float(np.mean([l["spec"].algorithmic_bytes for l in layers])) / peak_hbm_bytes_per_s() * 1e6,
+    }
+    per_layer = {
+        l["spec"].name: {"us": float(per_launch_ms[:, j].mean() * 1e3),
+                         "T_bmac_per_s": l["spec"].binary_macs / float(per_launch_ms[:, j].mean() * 1e-3) / 1e12}
+        for j, l in enumerate(layers)
+    }
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "batch_per_gpu": BATCH, "parallelism": f"batch-split x{world}, no collective",
+                   "l2": "flushed between steps by a 256 MiB write"},
+        "images_per_second": images_per_s,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms, "api": "lce_bconv2d_host (pinned host buffers, plain weights)"},
+        "gpu_launches": args.steps * len(layers),
+        "clocks": clocks, "roofline": roofline, "per_layer": per_layer, "wall_s_timed_region": wall,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cores = len(os.sched_getaffinity(0))
+        sample_batch, passes = BATCH, 2
+        v, dt, _ = time_oracle(sample_batch, passes)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"all 8 launches of config 2 at batch {sample_batch}, {passes} passes of {dt:.1f} s"}
+    if world > 1:
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+def peak_hbm_bytes_per_s() -> float:
+    p = ROOT / "MEASURED_PEAKS.json"
+    try:
+        return float(json.loads(p.read_text())["hbm_gbs"]) * 1e9
+    except Exception:
+        return 6650e9  # fallback figure of this pool
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="lce", choices=["lce", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_lce(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -48,7 +48,8 @@ struct TiledParams {
     const int32_t *thr;
     void *out;
     int32_t N, H, W, Cin, Cw, Cout, Cow, OH, OW, pt, pl;
-    int32_t tile_pixels;  // flat output pixels per CTA, a multiple of kPixPerStep * TP
+    int32_t tile_pixels;  // flat output pixels per tile, a multiple of kPixPerStep * TP
+    int32_t n_tiles;      // ceil(M / tile_pixels); CTA x works on tiles x, x + gridDim.x, ...
     int32_t M, Hp, Wp, pitch, plane;
     int32_t cw_shift;     // log2(Cw) when Cw is a power of two, else -1
     int32_t padding, out_type, activation;
@@ -164,6 +165,60 @@ pack_weights_kernel(const uint32_t *__restrict__ w, uint32_t *__restrict__ image
     }
 }
 
+// 4-byte asynchronous global->shared copy (no register round trip: the copy overlaps whatever the
+// thread does next).
+__device__ __forceinline__ void cp_async4(uint32_t *smem_dst, const uint32_t *gmem_src)
+{
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+
+// First virtual (padded-image) row of a tile of flat pixels [m0, m_end): v = n*Hp + oh*stride.
+template <int STRIDE>
+__device__ __forceinline__ int tile_first_vrow(const TiledParams &p, int m0)
+{
+    const int r_first = m0 / p.OW;
+    return (r_first / p.OH) * p.Hp + (r_first % p.OH) * STRIDE;
+}
+
+// Copies the input rows a tile needs into shared memory: global [n][iy][ix][cw] -> [cw][v][x] in
+// padded-image coordinates.  Image words travel as asynchronous copies (the caller waits for
+// them); rows and columns outside the image are written as zero words (one-padding).
+template <int STRIDE>
+__device__ __forceinline__ void stage_rows(const TiledParams &p, int m0, int m_end, uint32_t *sA, int warp, int lane)
+{
+    const int r_last = (m_end - 1) / p.OW;
+    const int v_first = tile_first_vrow<STRIDE>(p, m0);
+    const int v_last = (r_last / p.OH) * p.Hp + (r_last % p.OH) * STRIDE + 2;
+    const int nv = v_last - v_first + 1;
+    const int row_words = p.W * p.Cw;
+    for (int v = warp; v < nv; v += kWarps) {
+        const int va = v_first + v;
+        const int n = va / p.Hp;
+        const int iy = va - n * p.Hp - p.pt;
+        uint32_t *dst_row = sA + v * p.pitch;
+        if (n < p.N && iy >= 0 && iy < p.H) {
+            const uint32_t *src = p.in + ((int64_t)n * p.H + iy) * row_words;
+            for (int e = lane; e < row_words; e += 32) {
+                int ix, cw;
+                if (p.cw_shift >= 0) { ix = e >> p.cw_shift; cw = e & (p.Cw - 1); }
+                else { ix = e / p.Cw; cw = e - ix * p.Cw; }
+                cp_async4(dst_row + cw * p.plane + ix + p.pl, src + e);
+            }
+            const int edge = p.Wp - p.W;  // pad columns: pl on the left, the rest on the right
+            for (int e = lane; e < edge * p.Cw; e += 32) {
+                const int cw = e / edge, k = e - cw * edge;
+                dst_row[cw * p.plane + (k < p.pl ? k : p.W + k)] = 0u;
+            }
+        } else {
+            for (int e = lane; e < p.Wp * p.Cw; e += 32) {
+                const int cw = e / p.Wp, x = e - cw * p.Wp;
+                dst_row[cw * p.plane + x] = 0u;
+            }
+        }
+    }
+}
+
 template <int STRIDE, int TP>
 __global__ void __launch_bounds__(kThreads, (TP <= 2 ? 24 : 16) / kWarps)
 bconv3x3_kernel(const TiledParams p)
@@ -172,13 +227,12 @@ bconv3x3_kernel(const TiledParams p)
     const int w_words = p.Cw * kChanGroups * kWGroupStride;
     uint32_t *sW = smem;                                           // [Cw][8 groups][kWGroupStride]
     int32_t *sWsum = reinterpret_cast<int32_t *>(smem + w_words);  // [64][9]
-    uint32_t *sA = smem + w_words + kWsumWords;                    // [Cw][nv][pitch]
+    uint32_t *sA0 = smem + w_words + kWsumWords;                   // 2 x [Cw][nv][pitch]
 
     const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
-    const int m0 = blockIdx.x * p.tile_pixels;
-    const int m_end = min(m0 + p.tile_pixels, p.M);
     const int ch0 = blockIdx.y * kChanPerCta;
+    const int plane_words = p.Cw * p.plane;  // one input buffer; two of them alternate between tiles
 
     // ---- weights ----------------------------------------------------------------------------
     if (p.w_image != nullptr) {
@@ -209,43 +263,7 @@ bconv3x3_kernel(const TiledParams p)
         }
     }
 
-    // ---- input rows: global [n][iy][ix][cw] -> shared [cw][v][x] ---------------------------------
-    // virtual (padded-image) rows this CTA needs: v = n*Hp + oh*stride + ky
-    const int r_first = m0 / p.OW, r_last = (m_end - 1) / p.OW;
-    const int v_first = (r_first / p.OH) * p.Hp + (r_first % p.OH) * STRIDE;
-    const int v_last = (r_last / p.OH) * p.Hp + (r_last % p.OH) * STRIDE + 2;
-    const int nv = v_last - v_first + 1;
-    {
-        const int row_words = p.W * p.Cw;
-        for (int v = warp; v < nv; v += kThreads / 32) {
-            const int va = v_first + v;
-            const int n = va / p.Hp;
-            const int iy = va - n * p.Hp - p.pt;
-            uint32_t *dst_row = sA + v * p.pitch;
-            if (n < p.N && iy >= 0 && iy < p.H) {
-                const uint32_t *src = p.in + ((int64_t)n * p.H + iy) * row_words;
-                // the image's words of this row, coalesced; the columns left and right of it are zero
-                for (int e = lane; e < row_words; e += 32) {
-                    int ix, cw;
-                    if (p.cw_shift >= 0) { ix = e >> p.cw_shift; cw = e & (p.Cw - 1); }
-                    else { ix = e / p.Cw; cw = e - ix * p.Cw; }
-                    dst_row[cw * p.plane + ix + p.pl] = __ldg(src + e);
-                }
-                const int edge = p.Wp - p.W;  // pad columns: pl on the left, the rest on the right
-                for (int e = lane; e < edge * p.Cw; e += 32) {
-                    const int cw = e / edge, k = e - cw * edge;
-                    dst_row[cw * p.plane + (k < p.pl ? k : p.W + k)] = 0u;
-                }
-            } else {
-                for (int e = lane; e < p.Wp * p.Cw; e += 32) {
-                    const int cw = e / p.Wp, x = e - cw * p.Wp;
-                    dst_row[cw * p.plane + x] = 0u;
-                }
-            }
-        }
-    }
-
-    // ---- this thread's channels and pixels ---------------------------------------------------
+    // ---- this thread's channels --------------------------------------------------------------
     const int px = lane >> 3, cg = lane & 7;
     const int chan = ch0 + cg * kChanPerThread;
     const int K = 9 * p.Cin;
@@ -254,6 +272,30 @@ bconv3x3_kernel(const TiledParams p)
     k124.two = p.N > 0 ? 2u : p.Cin;
     k124.four = p.N > 0 ? 4u : p.Cin;
     asm volatile("" : "+r"(k124.one), "+r"(k124.two), "+r"(k124.four));
+    const uint32_t w_saddr0 = (uint32_t)__cvta_generic_to_shared(sW + cg * kWGroupStride);
+
+    // ---- persistent loop over this CTA's pixel tiles; the next tile's input rows are copied into
+    // the other buffer while the current tile is computed --------------------------------------
+    int tile = blockIdx.x;
+    if (tile < p.n_tiles)
+        stage_rows<STRIDE>(p, tile * p.tile_pixels, min((tile + 1) * p.tile_pixels, p.M), sA0, warp, lane);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+
+  for (int buf = 0; tile < p.n_tiles; tile += gridDim.x, buf ^= 1) {
+    const uint32_t *sA = sA0 + buf * plane_words;
+    const int m0 = tile * p.tile_pixels;
+    const int m_end = min(m0 + p.tile_pixels, p.M);
+    {
+        const int next = tile + gridDim.x;
+        if (next < p.n_tiles)
+            stage_rows<STRIDE>(p, next * p.tile_pixels, min((next + 1) * p.tile_pixels, p.M),
+                               sA0 + (buf ^ 1) * plane_words, warp, lane);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    const int r_first = m0 / p.OW;
+    const int v_first = tile_first_vrow<STRIDE>(p, m0);
 
     // running position of this lane's next pixel; the pixels of one lane are kPixPerStep apart
     int m_next = m0 + warp * 4 + px;  // lanes of a warp: 4 neighbouring pixels
@@ -266,11 +308,7 @@ bconv3x3_kernel(const TiledParams p)
         voh = n * p.Hp + oh * STRIDE;
         oh_left = p.OH - 1 - oh;  // rows left in the image after this one
     }
-    const int a_base_first = ((r_first / p.OH) * p.Hp + (r_first % p.OH) * STRIDE - v_first) * p.pitch +
-                             (m0 - r_first * p.OW) * STRIDE;
-    const uint32_t w_saddr0 = (uint32_t)__cvta_generic_to_shared(sW + cg * kWGroupStride);
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    __syncthreads();
+    const int a_base_first = (m0 - r_first * p.OW) * STRIDE;  // the tile's first pixel sits in virtual row 0
 
     for (int base = m0; base < m0 + p.tile_pixels; base += kPixPerStep * TP) {
         int a_base[TP];
@@ -383,6 +421,10 @@ bconv3x3_kernel(const TiledParams p)
             }
         }
     }
+    // the next tile's rows have landed, and every warp is done reading this tile's
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+  }
 }
 
 template <int STRIDE, int TP>
@@ -404,7 +446,7 @@ int reg_limited_ctas(int tp) { return (tp <= 2 ? 24 : 16) / kWarps; }
 
 size_t smem_bytes_for(const ConvGeom &g, const TiledParams &p)
 {
-    return ((size_t)g.Cw * kChanGroups * kWGroupStride + kWsumWords + (size_t)g.Cw * p.plane) * 4;
+    return ((size_t)g.Cw * kChanGroups * kWGroupStride + kWsumWords + 2 * (size_t)g.Cw * p.plane) * 4;
 }
 
 void set_tile(const ConvGeom &g, TiledParams *p, int tile_pixels)
@@ -464,9 +506,10 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
         if ((1 << b) == g.Cw) p.cw_shift = b;
     const int chan_blocks = (g.Cout + kChanPerCta - 1) / kChanPerCta;
 
-    // Pixels per thread (TP) and rounds per CTA: a CTA covers 16*TP*rounds flat pixels.  Pick the
-    // pair whose CTA count fills the machine's CTA slots most evenly; the cost of a choice is
-    // (number of waves) x (per-CTA main-loop work + a fixed staging cost), in pixel units.
+    // Pixels per thread (TP) and tile size: a tile covers 16*TP*rounds flat pixels and the grid is
+    // persistent (each CTA walks tiles x, x + gridDim.x, ...).  Pick the pair that balances the
+    // SMs best: cost = (CTAs on the busiest SM) x (tiles of the busiest CTA) x (tile work),
+    // with a penalty when too few warps share an SM to keep the logic pipe busy.
     int sms = 148;
     {
         int dev = 0;
@@ -477,12 +520,12 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
     if (const char *e = getenv("LCE_TP")) forced_tp = atoi(e);
     if (const char *e = getenv("LCE_ROUNDS")) forced_rounds = atoi(e);
 #endif
-    int best_tile = 0, best_tp = 0;
+    int best_tile = 0, best_tp = 0, best_ctas_x = 0;
     double best_cost = 0;
     for (int tp = 2; tp <= 4; ++tp) {
         if (forced_tp && tp != forced_tp) continue;
         const int unit = kPixPerStep * tp;
-        for (int rounds = 1; rounds <= 4; ++rounds) {
+        for (int rounds = 1; rounds <= 2; ++rounds) {
             if (forced_rounds && rounds != forced_rounds) continue;
             const int tile = unit * rounds;
             set_tile(g, &p, tile);
@@ -490,21 +533,27 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
             if (smem > 110 * 1024) continue;
             int per_sm = (int)((220 * 1024) / (smem + 1024));
             if (per_sm > reg_limited_ctas(tp)) per_sm = reg_limited_ctas(tp);
-            const int64_t ctas = ((g.M + tile - 1) / tile) * chan_blocks;
-            const int64_t slots = (int64_t)sms * per_sm;
-            const int64_t waves = (ctas + slots - 1) / slots;
-            const double staging = 8.0 + 96.0 / (9.0 * g.Cw);
+            const int64_t n_tiles = (g.M + tile - 1) / tile;
+            int64_t ctas_x = ((int64_t)sms * per_sm) / chan_blocks;
+            if (ctas_x < 1) ctas_x = 1;
+            if (ctas_x > n_tiles) ctas_x = n_tiles;
+            const int64_t tiles_per_cta = (n_tiles + ctas_x - 1) / ctas_x;
+            const int64_t ctas_on_sm = (ctas_x * chan_blocks + sms - 1) / sms;
+            const double warps = (double)ctas_x * chan_blocks / sms * kWarps;
+            const double eff = warps >= 16 ? 1.0 : (warps >= 8 ? 0.8 + 0.2 * (warps - 8) / 8 : 0.4 + 0.4 * warps / 8);
             // fewer pixels per thread re-read the weight operands from shared memory more often
-            const double smem_penalty = tp == 2 ? 1.08 : (tp == 3 ? 1.03 : 1.0);
-            const double cost = (double)waves * (tile * smem_penalty + staging) / per_sm;
-            if (best_tile == 0 || cost < best_cost) { best_tile = tile; best_tp = tp; best_cost = cost; }
+            const double smem_penalty = tp == 2 ? 1.06 : (tp == 3 ? 1.02 : 1.0);
+            const double cost = (double)ctas_on_sm * tiles_per_cta * (tile * smem_penalty + 4.0) / eff;
+            if (best_tile == 0 || cost < best_cost) {
+                best_tile = tile; best_tp = tp; best_cost = cost; best_ctas_x = (int)ctas_x;
+            }
         }
     }
     if (best_tile == 0) return LCE_ERR_UNSUPPORTED;
     set_tile(g, &p, best_tile);
+    p.n_tiles = (int32_t)((g.M + best_tile - 1) / best_tile);
     const size_t smem_bytes = smem_bytes_for(g, p);
-    const int64_t ctas = (g.M + best_tile - 1) / best_tile;
-    dim3 grid((unsigned)ctas, (unsigned)chan_blocks, 1);
+    dim3 grid((unsigned)best_ctas_x, (unsigned)chan_blocks, 1);
     if (g.sh == 1) {
         if (best_tp == 2) return launch3x3<1, 2>(p, smem_bytes, grid, s);
         if (best_tp == 3) return launch3x3<1, 3>(p, smem_bytes, grid, s);

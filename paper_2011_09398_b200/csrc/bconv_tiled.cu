@@ -52,6 +52,8 @@ struct TiledParams {
     int32_t n_tiles;      // ceil(M / tile_pixels); CTA x works on tiles x, x + gridDim.x, ...
     int32_t M, Hp, Wp, pitch, plane;
     int32_t cw_shift;     // log2(Cw) when Cw is a power of two, else -1
+    int32_t stride;       // pointwise kernel only
+    int32_t n9, rem3, cwp; // pointwise kernel: nine-word groups, leftover triples, padded words per pixel
     int32_t padding, out_type, activation;
 };
 
@@ -137,6 +139,7 @@ __global__ void __launch_bounds__(128)
 pack_weights_kernel(const uint32_t *__restrict__ w, uint32_t *__restrict__ image, int32_t Cout, int32_t Cw,
                     int32_t Cin, int32_t chan_blocks)
 {
+    // 3x3: group = channel word, the nine words of a group are the nine taps
     const int64_t entries = (int64_t)chan_blocks * kChanPerCta * Cw;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < entries;
          e += (int64_t)gridDim.x * blockDim.x) {
@@ -160,6 +163,75 @@ pack_weights_kernel(const uint32_t *__restrict__ w, uint32_t *__restrict__ image
                 if (c < Cout)
                     for (int j = 0; j < Cw; ++j) cnt += __popc(w[(c * 9 + t) * Cw + j]);
                 wsum[ch * 9 + t] = c < Cout ? Cin - 2 * cnt : 0;
+            }
+        }
+    }
+}
+
+// Per-channel parameters of the thread's 8 output channels for the chosen output type.
+struct ChannelParams {
+    float mult[kChanPerThread], bias[kChanPerThread];
+    int32_t thr[kChanPerThread];
+};
+__device__ __forceinline__ void load_channel_params(const TiledParams &p, int chan, ChannelParams &c)
+{
+#pragma unroll
+    for (int j = 0; j < kChanPerThread; ++j) {
+        const bool ok = chan + j < p.Cout;
+        c.mult[j] = (p.out_type == LCE_OUT_FLOAT32 && ok) ? __ldg(p.mult + chan + j) : 0.f;
+        c.bias[j] = (p.out_type == LCE_OUT_FLOAT32 && ok) ? __ldg(p.bias + chan + j) : 0.f;
+        c.thr[j] = (p.out_type == LCE_OUT_BITPACKED && ok) ? __ldg(p.thr + chan + j) : INT32_MIN;  // pad bits -> 0
+    }
+}
+
+// Output transform of one pixel's 8 accumulators v (paper Section 3.2): float multiply-add after
+// the fused activation, threshold compare + bit-pack, or the raw accumulators.  Every lane of the
+// warp must call it (the bit-packed form combines 4 lanes with shuffles); pix_ok guards the store.
+__device__ __forceinline__ void store_outputs(const TiledParams &p, const int32_t (&v)[kChanPerThread],
+                                              const ChannelParams &c, int m, bool pix_ok, int cg, int ch0, int chan)
+{
+    const float (&mult)[kChanPerThread] = c.mult;
+    const float (&bias)[kChanPerThread] = c.bias;
+    const int32_t (&thr)[kChanPerThread] = c.thr;
+    if (p.out_type == LCE_OUT_BITPACKED) {
+        uint32_t bits = 0u;
+#pragma unroll
+        for (int j = 0; j < kChanPerThread; ++j) bits |= (v[j] < thr[j] ? 1u : 0u) << j;
+        // the 4 lanes cg&~3 .. cg|3 hold the 4 bytes of one output word
+        bits <<= 8 * (cg & 3);
+        bits |= __shfl_xor_sync(0xffffffffu, bits, 1);
+        bits |= __shfl_xor_sync(0xffffffffu, bits, 2);
+        const int word = (ch0 >> 5) + (cg >> 2);
+        if (pix_ok && (cg & 3) == 0 && word < p.Cow)
+            static_cast<uint32_t *>(p.out)[(int64_t)m * p.Cow + word] = bits;
+    } else if (p.out_type == LCE_OUT_FLOAT32) {
+        float f[kChanPerThread];
+#pragma unroll
+        for (int j = 0; j < kChanPerThread; ++j) {
+            const int32_t a = (p.activation == LCE_ACT_RELU && v[j] < 0) ? 0 : v[j];
+            f[j] = __fmaf_rn((float)a, mult[j], bias[j]);
+        }
+        if (pix_ok) {
+            float *dst = static_cast<float *>(p.out) + (int64_t)m * p.Cout + chan;
+            if ((p.Cout & 3) == 0 && chan + kChanPerThread <= p.Cout) {
+                reinterpret_cast<float4 *>(dst)[0] = make_float4(f[0], f[1], f[2], f[3]);
+                reinterpret_cast<float4 *>(dst)[1] = make_float4(f[4], f[5], f[6], f[7]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < kChanPerThread; ++j)
+                    if (chan + j < p.Cout) dst[j] = f[j];
+            }
+        }
+    } else {
+        if (pix_ok) {
+            int32_t *dst = static_cast<int32_t *>(p.out) + (int64_t)m * p.Cout + chan;
+            if ((p.Cout & 3) == 0 && chan + kChanPerThread <= p.Cout) {
+                reinterpret_cast<int4 *>(dst)[0] = make_int4(v[0], v[1], v[2], v[3]);
+                reinterpret_cast<int4 *>(dst)[1] = make_int4(v[4], v[5], v[6], v[7]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < kChanPerThread; ++j)
+                    if (chan + j < p.Cout) dst[j] = v[j];
             }
         }
     }
@@ -347,15 +419,8 @@ bconv3x3_kernel(const TiledParams p)
         }
 
         // ---- output transform -------------------------------------------------------------
-        float mult[kChanPerThread], bias[kChanPerThread];
-        int32_t thr[kChanPerThread];
-#pragma unroll
-        for (int j = 0; j < kChanPerThread; ++j) {
-            const bool ok = chan + j < p.Cout;
-            mult[j] = (p.out_type == LCE_OUT_FLOAT32 && ok) ? __ldg(p.mult + chan + j) : 0.f;
-            bias[j] = (p.out_type == LCE_OUT_FLOAT32 && ok) ? __ldg(p.bias + chan + j) : 0.f;
-            thr[j] = (p.out_type == LCE_OUT_BITPACKED && ok) ? __ldg(p.thr + chan + j) : INT32_MIN;  // pad bits -> 0
-        }
+        ChannelParams cp;
+        load_channel_params(p, chan, cp);
 #pragma unroll
         for (int i = 0; i < TP; ++i) {
             const int m = base + i * kPixPerStep + warp * 4 + px;
@@ -377,54 +442,217 @@ bconv3x3_kernel(const TiledParams p)
                     }
                 }
             }
-            if (p.out_type == LCE_OUT_BITPACKED) {
-                uint32_t bits = 0u;
-#pragma unroll
-                for (int j = 0; j < kChanPerThread; ++j) bits |= (v[j] < thr[j] ? 1u : 0u) << j;
-                // the 4 lanes cg&~3 .. cg|3 hold the 4 bytes of one output word
-                bits <<= 8 * (cg & 3);
-                bits |= __shfl_xor_sync(0xffffffffu, bits, 1);
-                bits |= __shfl_xor_sync(0xffffffffu, bits, 2);
-                const int word = (ch0 >> 5) + (cg >> 2);
-                if (pix_ok && (cg & 3) == 0 && word < p.Cow)
-                    static_cast<uint32_t *>(p.out)[(int64_t)m * p.Cow + word] = bits;
-            } else if (p.out_type == LCE_OUT_FLOAT32) {
-                float f[kChanPerThread];
-#pragma unroll
-                for (int j = 0; j < kChanPerThread; ++j) {
-                    const int32_t a = (p.activation == LCE_ACT_RELU && v[j] < 0) ? 0 : v[j];
-                    f[j] = __fmaf_rn((float)a, mult[j], bias[j]);
-                }
-                if (pix_ok) {
-                    float *dst = static_cast<float *>(p.out) + (int64_t)m * p.Cout + chan;
-                    if ((p.Cout & 3) == 0 && chan + kChanPerThread <= p.Cout) {
-                        reinterpret_cast<float4 *>(dst)[0] = make_float4(f[0], f[1], f[2], f[3]);
-                        reinterpret_cast<float4 *>(dst)[1] = make_float4(f[4], f[5], f[6], f[7]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < kChanPerThread; ++j)
-                            if (chan + j < p.Cout) dst[j] = f[j];
-                    }
-                }
-            } else {
-                if (pix_ok) {
-                    int32_t *dst = static_cast<int32_t *>(p.out) + (int64_t)m * p.Cout + chan;
-                    if ((p.Cout & 3) == 0 && chan + kChanPerThread <= p.Cout) {
-                        reinterpret_cast<int4 *>(dst)[0] = make_int4(v[0], v[1], v[2], v[3]);
-                        reinterpret_cast<int4 *>(dst)[1] = make_int4(v[4], v[5], v[6], v[7]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < kChanPerThread; ++j)
-                            if (chan + j < p.Cout) dst[j] = v[j];
-                    }
-                }
-            }
+            store_outputs(p, v, cp, m, pix_ok, cg, ch0, chan);
         }
     }
     // the next tile's rows have landed, and every warp is done reading this tile's
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
   }
+}
+
+// ---- pointwise (1x1) convolution ------------------------------------------------------------
+// K runs over the channel words of one pixel only, so the nine-word carry-save groups are formed
+// along the channel axis: words 9g .. 9g+8 of a pixel against the same words of a channel.  What
+// is left after the full groups is handled as one or two triples (4 LOP3 + 2 POPC each).  The
+// words past Cw are zero on both sides and so add nothing to the count.
+
+__host__ __device__ __forceinline__ int pointwise_groups(int n9, int rem3) { return n9 + (rem3 > 0 ? 1 : 0); }
+
+__global__ void __launch_bounds__(128)
+pack_weights_pointwise_kernel(const uint32_t *__restrict__ w, uint32_t *__restrict__ image, int32_t Cout, int32_t Cw,
+                              int32_t groups, int32_t chan_blocks)
+{
+    const int64_t entries = (int64_t)chan_blocks * kChanPerCta * groups;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < entries;
+         e += (int64_t)gridDim.x * blockDim.x) {
+        const int g = (int)(e % groups);
+        const int64_t c = e / groups;
+        const int cb = (int)(c / kChanPerCta), ch = (int)(c % kChanPerCta);
+        uint32_t wv[9];
+#pragma unroll
+        for (int t = 0; t < 9; ++t) wv[t] = (c < Cout && 9 * g + t < Cw) ? w[c * Cw + 9 * g + t] : 0u;
+        uint32_t *block = image + cb * image_block_words(groups);
+        store_w_operands(wv, block + w_offset(g, ch));
+        if ((ch & 7) == 7) {
+            uint32_t *pad = block + w_offset(g, ch) + kWRow;
+            pad[0] = pad[1] = pad[2] = pad[3] = 0u;
+        }
+        if (g == 0) {  // per-tap sums are never used by a pointwise convolution (nothing is padded)
+            int32_t *wsum = reinterpret_cast<int32_t *>(block + (int64_t)groups * kChanGroups * kWGroupStride);
+            for (int t = 0; t < 9; ++t) wsum[ch * 9 + t] = 0;
+        }
+    }
+}
+
+template <int J, int TP, int NT>
+struct TailChannelLoop {
+    // leftover triples: NT (1 or 2) triples per (pixel, channel)
+    __device__ __forceinline__ static void run(uint32_t w_saddr, const Triple (&at)[TP][3], const Weights124 &k,
+                                               uint32_t (&acc)[TP][kChanPerThread])
+    {
+        Triple wt[3];
+        const uint4 q0 = lds128<J * 48>(w_saddr);
+        wt[0].all = q0.x; wt[0].pair = q0.y; wt[0].first = q0.z;
+        if (NT > 1) {
+            const uint4 q1 = lds128<J * 48 + 16>(w_saddr);
+            wt[1].all = q0.w; wt[1].pair = q1.x; wt[1].first = q1.y;
+        }
+#pragma unroll
+        for (int i = 0; i < TP; ++i)
+#pragma unroll
+            for (int t = 0; t < NT; ++t) popc3_mad(at[i][t], wt[t], k, acc[i][J]);
+        TailChannelLoop<J + 1, TP, NT>::run(w_saddr, at, k, acc);
+    }
+};
+template <int TP, int NT>
+struct TailChannelLoop<kChanPerThread, TP, NT> {
+    __device__ __forceinline__ static void run(uint32_t, const Triple (&)[TP][3], const Weights124 &,
+                                               uint32_t (&)[TP][kChanPerThread]) {}
+};
+
+// Copies the packed words of a tile's input pixels into shared memory as [pixel][cwp] (cwp = Cw
+// rounded up to whole triples; the extra words are zero).
+__device__ __forceinline__ void stage_pixels(const TiledParams &p, int m0, int m_end, uint32_t *sA, int tid)
+{
+    const int count = (m_end - m0) * p.cwp;
+    for (int e = tid; e < count; e += kThreads) {
+        const int l = e / p.cwp, cw = e - l * p.cwp;
+        if (cw < p.Cw) {
+            const int m = m0 + l;
+            int64_t src_pix = m;
+            if (p.stride != 1 || p.OW != p.W || p.OH != p.H) {
+                const int r = m / p.OW, ow = m - r * p.OW;
+                const int n = r / p.OH, oh = r - n * p.OH;
+                src_pix = ((int64_t)n * p.H + oh * p.stride) * p.W + ow * p.stride;
+            }
+            cp_async4(sA + e, p.in + src_pix * p.Cw + cw);
+        } else {
+            sA[e] = 0u;
+        }
+    }
+}
+
+template <int TP>
+__global__ void __launch_bounds__(kThreads, (TP <= 2 ? 24 : 16) / kWarps)
+bconv1x1_kernel(const TiledParams p)
+{
+    extern __shared__ __align__(16) uint32_t smem[];
+    const int groups = pointwise_groups(p.n9, p.rem3);
+    const int w_words = groups * kChanGroups * kWGroupStride;
+    uint32_t *sW = smem;
+    uint32_t *sA0 = smem + w_words + kWsumWords;  // 2 x [tile_pixels][cwp]
+    const int buf_words = p.tile_pixels * p.cwp;
+
+    const int tid = threadIdx.x;
+    const int lane = tid & 31, warp = tid >> 5;
+    const int ch0 = blockIdx.y * kChanPerCta;
+
+    if (p.w_image != nullptr) {
+        const uint32_t *src = p.w_image + blockIdx.y * image_block_words(groups);
+        for (int e = tid * 4; e < w_words; e += kThreads * 4) cp_async16(smem + e, src + e);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    } else {
+        for (int e = tid; e < kChanPerCta * groups; e += kThreads) {
+            const int ch = e / groups;
+            const int g = e - ch * groups;
+            uint32_t wv[9];
+#pragma unroll
+            for (int t = 0; t < 9; ++t)
+                wv[t] = (ch0 + ch < p.Cout && 9 * g + t < p.Cw) ? __ldg(p.w + (int64_t)(ch0 + ch) * p.Cw + 9 * g + t) : 0u;
+            store_w_operands(wv, sW + w_offset(g, ch));
+        }
+    }
+
+    const int px = lane >> 3, cg = lane & 7;
+    const int chan = ch0 + cg * kChanPerThread;
+    const int K = p.Cin;
+    Weights124 k124;
+    k124.one = p.N > 0 ? 1u : p.Cin;
+    k124.two = p.N > 0 ? 2u : p.Cin;
+    k124.four = p.N > 0 ? 4u : p.Cin;
+    asm volatile("" : "+r"(k124.one), "+r"(k124.two), "+r"(k124.four));
+    const uint32_t w_saddr0 = (uint32_t)__cvta_generic_to_shared(sW + cg * kWGroupStride);
+
+    int tile = blockIdx.x;
+    if (tile < p.n_tiles) stage_pixels(p, tile * p.tile_pixels, min((tile + 1) * p.tile_pixels, p.M), sA0, tid);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+
+    for (int buf = 0; tile < p.n_tiles; tile += gridDim.x, buf ^= 1) {
+        const uint32_t *sA = sA0 + buf * buf_words;
+        const int m0 = tile * p.tile_pixels;
+        const int m_end = min(m0 + p.tile_pixels, p.M);
+        {
+            const int next = tile + gridDim.x;
+            if (next < p.n_tiles)
+                stage_pixels(p, next * p.tile_pixels, min((next + 1) * p.tile_pixels, p.M), sA0 + (buf ^ 1) * buf_words, tid);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
+        for (int base = m0; base < m0 + p.tile_pixels; base += kPixPerStep * TP) {
+            uint32_t acc[TP][kChanPerThread];
+#pragma unroll
+            for (int i = 0; i < TP; ++i)
+#pragma unroll
+                for (int j = 0; j < kChanPerThread; ++j) acc[i][j] = 0u;
+            const uint32_t *apix[TP];
+#pragma unroll
+            for (int i = 0; i < TP; ++i) {
+                const int m = base + i * kPixPerStep + warp * 4 + px;
+                apix[i] = sA + (m < m_end ? (m - m0) * p.cwp : 0);  // past the end: redo pixel 0, store nothing
+            }
+            uint32_t w_saddr = w_saddr0;
+            for (int g = 0; g < p.n9; ++g) {
+                Triple at[TP][3];
+#pragma unroll
+                for (int i = 0; i < TP; ++i)
+#pragma unroll
+                    for (int t = 0; t < 3; ++t) {
+                        const uint32_t *q = apix[i] + 9 * g + 3 * t;
+                        at[i][t] = make_triple(q[0], q[1], q[2]);
+                    }
+                ChannelLoop<0, TP>::run(w_saddr, at, k124, acc);
+                w_saddr += kChanGroups * kWGroupStride * 4;
+            }
+            if (p.rem3 > 0) {
+                Triple at[TP][3];
+#pragma unroll
+                for (int i = 0; i < TP; ++i)
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        const uint32_t *q = apix[i] + 9 * p.n9 + 3 * (t < p.rem3 ? t : 0);
+                        at[i][t] = make_triple(q[0], q[1], q[2]);
+                    }
+                if (p.rem3 == 1) TailChannelLoop<0, TP, 1>::run(w_saddr, at, k124, acc);
+                else TailChannelLoop<0, TP, 2>::run(w_saddr, at, k124, acc);
+            }
+            ChannelParams cp;
+            load_channel_params(p, chan, cp);
+#pragma unroll
+            for (int i = 0; i < TP; ++i) {
+                const int m = base + i * kPixPerStep + warp * 4 + px;
+                int32_t v[kChanPerThread];
+#pragma unroll
+                for (int j = 0; j < kChanPerThread; ++j) v[j] = K - 2 * (int32_t)acc[i][j];
+                store_outputs(p, v, cp, m, m < m_end, cg, ch0, chan);
+            }
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
+    }
+}
+
+template <int TP>
+lce_status launch1x1(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStream_t s)
+{
+    auto kernel = bconv1x1_kernel<TP>;
+    if (smem_bytes > 48 * 1024) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
+            return LCE_ERR_CUDA;
+    }
+    kernel<<<grid, kThreads, smem_bytes, s>>>(p);
+    return launch_status();
 }
 
 template <int STRIDE, int TP>
@@ -458,10 +686,82 @@ void set_tile(const ConvGeom &g, TiledParams *p, int tile_pixels)
     p->plane = nv_max * p->pitch;
 }
 
+bool covers3x3(const ConvGeom &g) { return g.KH == 3 && g.KW == 3 && g.sh == g.sw && g.sh <= 2; }
+bool covers1x1(const ConvGeom &g) { return g.KH == 1 && g.KW == 1 && g.sh == g.sw; }
+
 bool tiled_covers(const ConvGeom &g)
 {
-    return g.KH == 3 && g.KW == 3 && g.sh == g.sw && g.sh <= 2 && g.M < (1ll << 31) - 256 &&
+    return (covers3x3(g) || covers1x1(g)) && g.M < (1ll << 31) - 256 &&
            (g.Cout + kChanPerCta - 1) / kChanPerCta <= 65535;
+}
+
+void pointwise_split(int Cw, int *n9, int *rem3)
+{
+    *n9 = Cw / 9;
+    const int rem = Cw % 9;
+    if (rem > 6) { ++*n9; *rem3 = 0; }
+    else *rem3 = (rem + 2) / 3;
+}
+
+int image_groups(const ConvGeom &g)
+{
+    if (covers3x3(g)) return g.Cw;
+    int n9, rem3;
+    pointwise_split(g.Cw, &n9, &rem3);
+    return pointwise_groups(n9, rem3);
+}
+
+struct TileChoice {
+    int tp, tile, ctas_x;
+};
+
+// Pixels per thread (TP) and tile size: a tile covers 16*TP*rounds flat pixels and the grid is
+// persistent (each CTA walks tiles x, x + gridDim.x, ...).  Pick the pair that balances the SMs
+// best: cost = (CTAs on the busiest SM) x (tiles of the busiest CTA) x (tile work), with a
+// penalty when too few warps share an SM to keep the logic pipe busy.
+template <typename SmemFn>
+bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileChoice *best)
+{
+    int sms = 148;
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    int forced_tp = 0, forced_rounds = 0;
+#ifdef LCE_TUNING
+    if (const char *e = getenv("LCE_TP")) forced_tp = atoi(e);
+    if (const char *e = getenv("LCE_ROUNDS")) forced_rounds = atoi(e);
+#endif
+    double best_cost = 0;
+    best->tile = 0;
+    for (int tp = 2; tp <= 4; ++tp) {
+        if (forced_tp && tp != forced_tp) continue;
+        const int unit = kPixPerStep * tp;
+        for (int rounds = 1; rounds <= 2; ++rounds) {
+            if (forced_rounds && rounds != forced_rounds) continue;
+            const int tile = unit * rounds;
+            const size_t smem = smem_for_tile(tile);
+            if (smem > 110 * 1024) continue;
+            int per_sm = (int)((220 * 1024) / (smem + 1024));
+            if (per_sm > reg_limited_ctas(tp)) per_sm = reg_limited_ctas(tp);
+            const int64_t n_tiles = (g.M + tile - 1) / tile;
+            int64_t ctas_x = ((int64_t)sms * per_sm) / chan_blocks;
+            if (ctas_x < 1) ctas_x = 1;
+            if (ctas_x > n_tiles) ctas_x = n_tiles;
+            const int64_t tiles_per_cta = (n_tiles + ctas_x - 1) / ctas_x;
+            const int64_t ctas_on_sm = (ctas_x * chan_blocks + sms - 1) / sms;
+            const double warps = (double)ctas_x * chan_blocks / sms * kWarps;
+            const double eff = warps >= 16 ? 1.0 : (warps >= 8 ? 0.8 + 0.2 * (warps - 8) / 8 : 0.4 + 0.4 * warps / 8);
+            // fewer pixels per thread re-read the weight operands from shared memory more often
+            const double smem_penalty = tp == 2 ? 1.06 : (tp == 3 ? 1.02 : 1.0);
+            const double cost = (double)ctas_on_sm * tiles_per_cta * (tile * smem_penalty + 4.0) / eff;
+            if (best->tile == 0 || cost < best_cost) {
+                best->tile = tile; best->tp = tp; best->ctas_x = (int)ctas_x;
+                best_cost = cost;
+            }
+        }
+    }
+    return best->tile != 0;
 }
 
 }  // namespace
@@ -470,17 +770,21 @@ size_t tiled_weight_image_bytes(const ConvGeom &g)
 {
     if (!tiled_covers(g)) return 0;
     const int chan_blocks = (g.Cout + kChanPerCta - 1) / kChanPerCta;
-    return (size_t)chan_blocks * image_block_words(g.Cw) * 4;
+    return (size_t)chan_blocks * image_block_words(image_groups(g)) * 4;
 }
 
 lce_status launch_pack_weights_tiled(const ConvGeom &g, const uint32_t *w, uint32_t *image, cudaStream_t s)
 {
     if (!tiled_covers(g)) return LCE_ERR_UNSUPPORTED;
     const int chan_blocks = (g.Cout + kChanPerCta - 1) / kChanPerCta;
-    const int64_t entries = (int64_t)chan_blocks * kChanPerCta * g.Cw;
+    const int groups = image_groups(g);
+    const int64_t entries = (int64_t)chan_blocks * kChanPerCta * groups;
     int blocks = (int)((entries + 127) / 128);
     if (blocks > 148 * 8) blocks = 148 * 8;
-    pack_weights_kernel<<<blocks, 128, 0, s>>>(w, image, g.Cout, g.Cw, g.Cin, chan_blocks);
+    if (covers3x3(g))
+        pack_weights_kernel<<<blocks, 128, 0, s>>>(w, image, g.Cout, g.Cw, g.Cin, chan_blocks);
+    else
+        pack_weights_pointwise_kernel<<<blocks, 128, 0, s>>>(w, image, g.Cout, g.Cw, groups, chan_blocks);
     return launch_status();
 }
 
@@ -497,70 +801,50 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
     p.OH = g.OH; p.OW = g.OW; p.pt = g.pt; p.pl = g.pl;
     p.padding = g.padding; p.out_type = g.out_type; p.activation = g.activation;
     p.M = (int32_t)g.M;
-    p.Hp = (g.OH - 1) * g.sh + 3;
-    p.Wp = (g.OW - 1) * g.sh + 3;
-    if (p.Wp < g.W + g.pl) p.Wp = g.W + g.pl;  // staging writes the whole image row; columns past the taps are unused
-    p.pitch = p.Wp | 1;  // odd pitch: the 4 pixels of a warp in 4 different rows hit 4 different banks
+    p.stride = g.sh;
     p.cw_shift = -1;
     for (int b = 0; b < 16; ++b)
         if ((1 << b) == g.Cw) p.cw_shift = b;
     const int chan_blocks = (g.Cout + kChanPerCta - 1) / kChanPerCta;
+    TileChoice c;
 
-    // Pixels per thread (TP) and tile size: a tile covers 16*TP*rounds flat pixels and the grid is
-    // persistent (each CTA walks tiles x, x + gridDim.x, ...).  Pick the pair that balances the
-    // SMs best: cost = (CTAs on the busiest SM) x (tiles of the busiest CTA) x (tile work),
-    // with a penalty when too few warps share an SM to keep the logic pipe busy.
-    int sms = 148;
-    {
-        int dev = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (covers1x1(g)) {
+        pointwise_split(g.Cw, &p.n9, &p.rem3);
+        p.cwp = 9 * p.n9 + 3 * p.rem3;
+        const int groups = pointwise_groups(p.n9, p.rem3);
+        auto smem_for = [&](int tile) {
+            return ((size_t)groups * kChanGroups * kWGroupStride + kWsumWords + 2 * (size_t)tile * p.cwp) * 4;
+        };
+        if (!choose_tile(g, chan_blocks, smem_for, &c)) return LCE_ERR_UNSUPPORTED;
+        p.tile_pixels = c.tile;
+        p.n_tiles = (int32_t)((g.M + c.tile - 1) / c.tile);
+        dim3 grid((unsigned)c.ctas_x, (unsigned)chan_blocks, 1);
+        const size_t smem_bytes = smem_for(c.tile);
+        if (c.tp == 2) return launch1x1<2>(p, smem_bytes, grid, s);
+        if (c.tp == 3) return launch1x1<3>(p, smem_bytes, grid, s);
+        return launch1x1<4>(p, smem_bytes, grid, s);
     }
-    int forced_tp = 0, forced_rounds = 0;
-#ifdef LCE_TUNING
-    if (const char *e = getenv("LCE_TP")) forced_tp = atoi(e);
-    if (const char *e = getenv("LCE_ROUNDS")) forced_rounds = atoi(e);
-#endif
-    int best_tile = 0, best_tp = 0, best_ctas_x = 0;
-    double best_cost = 0;
-    for (int tp = 2; tp <= 4; ++tp) {
-        if (forced_tp && tp != forced_tp) continue;
-        const int unit = kPixPerStep * tp;
-        for (int rounds = 1; rounds <= 2; ++rounds) {
-            if (forced_rounds && rounds != forced_rounds) continue;
-            const int tile = unit * rounds;
-            set_tile(g, &p, tile);
-            const size_t smem = smem_bytes_for(g, p);
-            if (smem > 110 * 1024) continue;
-            int per_sm = (int)((220 * 1024) / (smem + 1024));
-            if (per_sm > reg_limited_ctas(tp)) per_sm = reg_limited_ctas(tp);
-            const int64_t n_tiles = (g.M + tile - 1) / tile;
-            int64_t ctas_x = ((int64_t)sms * per_sm) / chan_blocks;
-            if (ctas_x < 1) ctas_x = 1;
-            if (ctas_x > n_tiles) ctas_x = n_tiles;
-            const int64_t tiles_per_cta = (n_tiles + ctas_x - 1) / ctas_x;
-            const int64_t ctas_on_sm = (ctas_x * chan_blocks + sms - 1) / sms;
-            const double warps = (double)ctas_x * chan_blocks / sms * kWarps;
-            const double eff = warps >= 16 ? 1.0 : (warps >= 8 ? 0.8 + 0.2 * (warps - 8) / 8 : 0.4 + 0.4 * warps / 8);
-            // fewer pixels per thread re-read the weight operands from shared memory more often
-            const double smem_penalty = tp == 2 ? 1.06 : (tp == 3 ? 1.02 : 1.0);
-            const double cost = (double)ctas_on_sm * tiles_per_cta * (tile * smem_penalty + 4.0) / eff;
-            if (best_tile == 0 || cost < best_cost) {
-                best_tile = tile; best_tp = tp; best_cost = cost; best_ctas_x = (int)ctas_x;
-            }
-        }
-    }
-    if (best_tile == 0) return LCE_ERR_UNSUPPORTED;
-    set_tile(g, &p, best_tile);
-    p.n_tiles = (int32_t)((g.M + best_tile - 1) / best_tile);
+
+    p.Hp = (g.OH - 1) * g.sh + 3;
+    p.Wp = (g.OW - 1) * g.sh + 3;
+    if (p.Wp < g.W + g.pl) p.Wp = g.W + g.pl;  // staging writes the whole image row; columns past the taps are unused
+    p.pitch = p.Wp | 1;  // odd pitch: the 4 pixels of a warp in 4 different rows hit 4 different banks
+    auto smem_for = [&](int tile) {
+        set_tile(g, &p, tile);
+        return smem_bytes_for(g, p);
+    };
+    if (!choose_tile(g, chan_blocks, smem_for, &c)) return LCE_ERR_UNSUPPORTED;
+    set_tile(g, &p, c.tile);
+    p.n_tiles = (int32_t)((g.M + c.tile - 1) / c.tile);
     const size_t smem_bytes = smem_bytes_for(g, p);
-    dim3 grid((unsigned)best_ctas_x, (unsigned)chan_blocks, 1);
+    dim3 grid((unsigned)c.ctas_x, (unsigned)chan_blocks, 1);
     if (g.sh == 1) {
-        if (best_tp == 2) return launch3x3<1, 2>(p, smem_bytes, grid, s);
-        if (best_tp == 3) return launch3x3<1, 3>(p, smem_bytes, grid, s);
+        if (c.tp == 2) return launch3x3<1, 2>(p, smem_bytes, grid, s);
+        if (c.tp == 3) return launch3x3<1, 3>(p, smem_bytes, grid, s);
         return launch3x3<1, 4>(p, smem_bytes, grid, s);
     }
-    if (best_tp == 2) return launch3x3<2, 2>(p, smem_bytes, grid, s);
-    if (best_tp == 3) return launch3x3<2, 3>(p, smem_bytes, grid, s);
+    if (c.tp == 2) return launch3x3<2, 2>(p, smem_bytes, grid, s);
+    if (c.tp == 3) return launch3x3<2, 3>(p, smem_bytes, grid, s);
     return launch3x3<2, 4>(p, smem_bytes, grid, s);
 }
 

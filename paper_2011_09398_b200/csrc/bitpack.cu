@@ -6,13 +6,15 @@ namespace lce {
 namespace {
 
 constexpr int kPackThreads = 256;
-constexpr int kWordsPerWarpPass = 128;  // one warp turns 128x32 floats into 128 words per pass
+constexpr int kWordsPerWarpPass = 32;  // one warp turns 32x32 floats (4 KB) into 32 words per pass
 
 // channels % 32 == 0: the flat float array is a sequence of 32-float groups, each giving one
 // word.  A warp reads group g with one coalesced 128-byte load (lane = channel within the
 // group); __ballot_sync(x < 0) is the packed word (lane order = bit order, LSB = lowest
-// channel).  128 ballots per pass are handed out four per lane so that every lane ends up
-// with four consecutive words and writes them with one 128-bit store.
+// channel).  All 32 loads of a pass are in flight before the first ballot; the 32 ballots are
+// handed out four per lane to lanes 0..7, which write them with one 128-bit store each (128
+// contiguous bytes per warp).  Passes are small so that even a 100K-word tensor gives every SM
+// several warps of work: the kernel is latency-bound otherwise.
 __global__ void __launch_bounds__(kPackThreads)
 bitpack_aligned_kernel(const float *__restrict__ x, uint32_t *__restrict__ out, int64_t n_words)
 {
@@ -20,22 +22,19 @@ bitpack_aligned_kernel(const float *__restrict__ x, uint32_t *__restrict__ out, 
     const int64_t warp = ((int64_t)blockIdx.x * kPackThreads + threadIdx.x) >> 5;
     const int64_t n_warps = ((int64_t)gridDim.x * kPackThreads) >> 5;
     for (int64_t w0 = warp * kWordsPerWarpPass; w0 < n_words; w0 += n_warps * kWordsPerWarpPass) {
-        uint32_t mine[4] = {0u, 0u, 0u, 0u};
         if (w0 + kWordsPerWarpPass <= n_words) {
+            float v[kWordsPerWarpPass];
 #pragma unroll
-            for (int b0 = 0; b0 < kWordsPerWarpPass; b0 += 16) {
-                float v[16];
+            for (int u = 0; u < kWordsPerWarpPass; ++u) v[u] = __ldcs(x + (w0 + u) * 32 + lane);
+            uint32_t mine[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-                for (int u = 0; u < 16; ++u) v[u] = __ldcs(x + (w0 + b0 + u) * 32 + lane);
-#pragma unroll
-                for (int u = 0; u < 16; ++u) {
-                    const uint32_t word = __ballot_sync(0xffffffffu, v[u] < 0.0f);
-                    const int b = b0 + u;
-                    if ((b >> 2) == lane) mine[b & 3] = word;
-                }
+            for (int u = 0; u < kWordsPerWarpPass; ++u) {
+                const uint32_t word = __ballot_sync(0xffffffffu, v[u] < 0.0f);
+                if ((u >> 2) == lane) mine[u & 3] = word;
             }
-            // out + w0 is 16-byte aligned: w0 is a multiple of 128 words and out is checked on the host
-            reinterpret_cast<uint4 *>(out + w0)[lane] = make_uint4(mine[0], mine[1], mine[2], mine[3]);
+            // out + w0 is 16-byte aligned: w0 is a multiple of 32 words and out is checked on the host
+            if (lane < kWordsPerWarpPass / 4)
+                reinterpret_cast<uint4 *>(out + w0)[lane] = make_uint4(mine[0], mine[1], mine[2], mine[3]);
         } else {  // ragged last pass of the tensor
             for (int64_t w = w0; w < n_words; ++w) {
                 const uint32_t word = __ballot_sync(0xffffffffu, x[w * 32 + lane] < 0.0f);
@@ -102,8 +101,8 @@ extern "C" lce_status lce_bitpack(const float *x, uint32_t *out, int64_t rows, i
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int32_t words = (channels + 31) / 32;
     const int64_t n_words = rows * words;
-    // 148 SMs x 8 resident blocks of 256 threads; grid-stride loops cover the rest
-    const int max_blocks = 148 * 8;
+    // up to 148 SMs x 8 resident blocks of 256 threads x 4 passes in the queue; grid-stride loops cover the rest
+    const int max_blocks = 148 * 8 * 4;
     if (channels % 32 == 0 && aligned(out, 16)) {
         const int64_t passes = (n_words + kWordsPerWarpPass - 1) / kWordsPerWarpPass;
         bitpack_aligned_kernel<<<grid_for(passes, kPackThreads / 32, max_blocks), kPackThreads, 0, s>>>(x, out, n_words);

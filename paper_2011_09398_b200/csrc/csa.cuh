@@ -97,6 +97,16 @@ __device__ __forceinline__ void popc9_mad(const Triple (&a)[3], const Triple (&w
     acc = mad_u32(__popc(F), k.four, acc);
 }
 
+// One triple added onto an accumulator with multiply-adds (K tails of the pointwise kernel).
+__device__ __forceinline__ void popc3_mad(const Triple &a, const Triple &w, const Weights124 &k, uint32_t &acc)
+{
+    const uint32_t s = a.all ^ w.all;
+    const uint32_t d = a.pair ^ w.pair;
+    const uint32_t x0 = a.first ^ w.first;
+    acc = mad_u32(__popc(s), k.one, acc);
+    acc = mad_u32(__popc(carry_dsx(d, s, x0)), k.two, acc);
+}
+
 // popcount of one triple alone (used for K tails and by the 3:2 probe): 4 LOP3 + 2 POPC.
 __device__ __forceinline__ uint32_t popc3(const Triple &a, const Triple &w)
 {

@@ -76,6 +76,9 @@ FUZZ = [
     (1, 2, 3, 64, 2, 3, 1), (2, 14, 14, 64, 64, 3, 1), (2, 14, 14, 64, 8, 3, 2), (1, 3, 3, 5, 7, 3, 1),
     (3, 7, 7, 512, 64, 3, 1), (2, 9, 11, 160, 70, 3, 1), (1, 17, 13, 96, 96, 3, 2), (2, 8, 8, 128, 130, 3, 1),
     (1, 29, 31, 64, 64, 3, 1), (2, 16, 16, 256, 32, 1, 1), (1, 57, 9, 32, 64, 3, 1), (5, 7, 7, 64, 64, 3, 1),
+    # pointwise: channel words split into nine-word groups and leftover triples in every combination
+    (1, 5, 5, 512, 70, 1, 1), (2, 6, 6, 200, 64, 1, 1), (1, 6, 5, 160, 8, 1, 1), (1, 4, 4, 320, 16, 1, 1),
+    (2, 9, 9, 64, 128, 1, 2), (1, 28, 28, 128, 256, 1, 1), (1, 3, 5, 608, 33, 1, 1),
 ]
 
 

@@ -36,6 +36,7 @@ lce_status dispatch(const lce_bconv2d_desc *desc, const ConvGeom &g, const uint3
     }
     if (desc->kernel == LCE_KERNEL_DIRECT)
         return launch_bconv_direct(g, input, weights, multiplier, bias, thresholds, output, s);
+    if (patch_covers(g)) return launch_bconv_patch(g, input, weights, multiplier, bias, thresholds, output, s);
     lce_status st = launch_bconv_tiled(g, input, weights, image, multiplier, bias, thresholds, output, s);
     if (st == LCE_ERR_UNSUPPORTED && desc->kernel == LCE_KERNEL_AUTO)
         st = launch_bconv_direct(g, input, weights, multiplier, bias, thresholds, output, s);

@@ -76,6 +76,10 @@ lce_status launch_bconv_direct(const ConvGeom &g, const uint32_t *in, const uint
 // w_image: the tiled part of a packed-weights buffer, or nullptr to derive operands from `w`.
 lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const uint32_t *w_image,
                               const float *mult, const float *bias, const int32_t *thr, void *out, cudaStream_t s);
+// One-word-patch kernel for tiny channel counts (KH*KW*Cin <= 32); plain weights only.
+bool patch_covers(const ConvGeom &g);
+lce_status launch_bconv_patch(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const float *mult,
+                              const float *bias, const int32_t *thr, void *out, cudaStream_t s);
 // Bytes of the tiled kernel's weight image for this geometry (0 if the kernel does not cover it).
 size_t tiled_weight_image_bytes(const ConvGeom &g);
 lce_status launch_pack_weights_tiled(const ConvGeom &g, const uint32_t *w, uint32_t *image, cudaStream_t s);

@@ -38,6 +38,7 @@ WORKLOAD = ("config 2: 3x3 one-padded Bconv2D sweep 56x56x64, 28x28x128, 14x14x2
 
 # Derived compute ceiling of the chosen pipe (integer logic + popcount), see the design doc:
 # 64 logic lanes/clk/SM, 16.75 logic instructions per nine 32-bit word operations, 32 binary MACs per word.
+NCU_DRAM_BYTES_PER_LAUNCH = 0.6e6
 LOGIC_LANES_PER_CLK_PER_SM = 64
 LOGIC_OPS_PER_9_WORDS = 16.75
 
@@ -51,6 +52,27 @@ def layer_inputs(spec, index):
     x = wl.activations(CONFIG, 10 * index, (spec.batch, spec.in_h, spec.in_w, spec.in_c))
     t = wl.conv_tensors(CONFIG, 10 * index + 1, spec)
     return x, t
+
+
+def shard_index(layer: int, rank: int) -> int:
+    """RNG index offset of one launch's tensors on one rank: every rank draws its own 64-image shard."""
+    return layer + 100 * rank
+
+
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Slowest rank's time (the job is as slow as its slowest GPU); identity on one rank."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    tt = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def whole_job_value(units_per_rank: float, world: int, ms: float) -> float:
+    """Weak scaling: every rank processes units_per_rank in the (max-over-ranks) time."""
+    return world * units_per_rank / (ms * 1e-3)
 
 
 class ClockSampler:
@@ -172,7 +194,7 @@ def run_lce(args):
     layers = []
     h2d = d2h = 0
     for i, spec in enumerate(specs()):
-        x, t = layer_inputs(spec, i + 100 * rank)
+        x, t = layer_inputs(spec, shard_index(i, rank))
         xd = torch.from_numpy(x).to(dev)
         a = lce.lce_bitpack(xd)                                   # pre-packed input (outside the timed region)
         wplain = lce.pack_weights(torch.from_numpy(t.w_pm1).to(dev))
@@ -243,14 +265,10 @@ def run_lce(args):
     clocks = sampler.stop()
     step_ms = [ev[0].elapsed_time(ev[-1]) for ev in all_events]
     per_launch_ms = np.array([[ev[j].elapsed_time(ev[j + 1]) for j in range(len(layers))] for ev in all_events])
-    total_ms = float(np.sum(step_ms))
-    if world > 1:
-        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = max_over_ranks(float(np.sum(step_ms)), world, dev)
     ms_per_step = total_ms / args.steps
     macs_per_step = sum(l["spec"].binary_macs for l in layers)
-    value = world * macs_per_step / (ms_per_step * 1e-3)
+    value = whole_job_value(macs_per_step, world, ms_per_step)
     images_per_s = world * len(layers) * BATCH / (ms_per_step * 1e-3)
 
     # ---- end-to-end leg: the host-buffer C-ABI entry point, copies inside the timed region ---------
@@ -272,11 +290,8 @@ def run_lce(args):
     barrier()
     e2e_wall = time.perf_counter() - t0
     e2e_ms = max(e0.elapsed_time(e1), 1e3 * e2e_wall) / e2e_steps  # host-synchronous calls: wall clock is the honest one
-    if world > 1:
-        tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item())
-    e2e_value = world * macs_per_step / (e2e_ms * 1e-3)
+    e2e_ms = max_over_ranks(e2e_ms, world, dev)
+    e2e_value = whole_job_value(macs_per_step, world, e2e_ms)
 
     # ---- roofline of the dominant kernel (the tiled 3x3 XOR/POPC kernel: all 8 launches) -------
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
@@ -291,7 +306,9 @@ def run_lce(args):
         "peak_source": "derived: SMs x max SM clock x 64 logic lanes/clk/SM x 9/16.75 word-ops per logic op x 32",
         "measured_mix_probe": probe_ops * 32 / 1e12, "frac_of_measured_probe": achieved / (probe_ops * 32),
         "avg_launch_us": avg_launch_ms * 1e3,
-        "traffic": None,
+        # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
+        # profiles/ (inputs, weights and outputs of one launch stay in the 126 MB L2 between launches)
+        "traffic": NCU_DRAM_BYTES_PER_LAUNCH,
         "hbm_bound_us": float(np.mean([l["spec"].algorithmic_bytes for l in layers])) / peak_hbm_bytes_per_s() * 1e6,
     }
     per_layer = {
@@ -312,6 +329,8 @@ def run_lce(args):
         "gpu_launches": args.steps * len(layers),
         "clocks": clocks, "roofline": roofline, "per_layer": per_layer, "wall_s_timed_region": wall,
     }
+    if world == 1 and not args.no_chains:
+        line["chains"] = time_chains(dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cores = len(os.sched_getaffinity(0))
         sample_batch, passes = BATCH, 2
@@ -322,6 +341,34 @@ def run_lce(args):
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(line))
+
+
+def time_chains(dev, reps: int = 5):
+    """Configs 4 and 5 end to end (every kernel of the chain on one stream), inputs resident on the
+    device; reported beside the headline number, outside its timed region."""
+    import torch
+
+    from paper_2011_09398_b200.chains import Chain
+    out = {}
+    for cfg, steps, name, batch in ((4, wl.config4_steps(), "X0", 128), (5, wl.config5_steps(), "X", 256)):
+        chain = Chain(steps, cfg, str(dev))
+        chain.buffers[name].normal_()
+        for _ in range(3):
+            chain.run()
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        for r in range(reps):
+            ev[r].record()
+            chain.run()
+        ev[reps].record()
+        torch.cuda.synchronize()
+        ms = ev[0].elapsed_time(ev[reps]) / reps
+        macs = sum(s.conv.binary_macs for s in steps if s.kind == "bconv")
+        out[f"config{cfg}"] = {"batch": batch, "launches": chain.launches, "ms": ms, "images_per_second": batch / (ms * 1e-3),
+                               "binary_macs_per_second": macs / (ms * 1e-3)}
+        del chain
+        torch.cuda.empty_cache()
+    return out
 
 
 def peak_hbm_bytes_per_s() -> float:
@@ -339,6 +386,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="lce", choices=["lce", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-chains", action="store_true", help="skip the config 4 / config 5 chain timings")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

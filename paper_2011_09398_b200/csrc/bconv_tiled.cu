@@ -109,8 +109,12 @@ struct ChannelLoop {
     {
         Triple wt[3];
         load_w_triples<J>(w_saddr, wt);
+#ifdef LCE_SERIAL_PIXELS
 #pragma unroll
         for (int i = 0; i < TP; ++i) popc9_mad(at[i], wt, k, acc[i][J]);
+#else
+        popc9_mad_pixels<TP, kChanPerThread, J>(at, wt, k, acc);
+#endif
         ChannelLoop<J + 1, TP>::run(w_saddr, at, k, acc);
     }
 };

@@ -134,6 +134,25 @@ lce_status lce_bconv2d_host(const lce_bconv2d_desc *desc, const uint32_t *input,
                             const float *multiplier, const float *bias, const int32_t *thresholds,
                             void *output, void *workspace, size_t workspace_bytes, void *stream);
 
+/* (No counterpart in the paper.)  lce_bconv2d_host for callers that cannot allocate device memory:
+ * a process whose allocator is off limits (a real-time loop, a sandboxed plug-in that only ever
+ * sees host tensors) has no way to produce the `workspace` argument above.  This form keeps the
+ * staging area inside the library, in one fixed device array of
+ * lce_bconv2d_host_noalloc_max_bytes() = 8 MiB per GPU, and calls no cudaMalloc, cudaFree or any
+ * other allocating routine.  Arguments and result are those of lce_bconv2d_host without the
+ * workspace; a call whose lce_bconv2d_host_workspace_bytes(desc) exceeds the array returns
+ * LCE_ERR_WORKSPACE and does nothing.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, which still holds the previous call's data:
+ *     nothing needs clearing (every region is rewritten before it is read), but two calls that
+ *     overlap on the GPU (different streams, different threads) would overwrite each other.
+ *     Serialise them. */
+size_t lce_bconv2d_host_noalloc_max_bytes(void);
+lce_status lce_bconv2d_host_noalloc(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
+                                    const float *multiplier, const float *bias, const int32_t *thresholds,
+                                    void *output, void *stream);
+
 /* LceBMaxPool2d (Section 3.2): max-pool of +-1 values on packed words = bitwise AND of the
  * window's words.  padding is LCE_PAD_VALID or LCE_PAD_SAME_ONE (TensorFlow SAME; taps outside
  * the image are skipped).

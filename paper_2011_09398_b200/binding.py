@@ -53,6 +53,10 @@ def library() -> ctypes.CDLL:
         lib.lce_bconv2d_host_workspace_bytes.restype = ctypes.c_size_t
         lib.lce_bconv2d_host_workspace_bytes.argtypes = [ctypes.POINTER(BConv2dDesc)]
         lib.lce_bconv2d_host.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        lib.lce_bconv2d_host_noalloc_max_bytes.restype = ctypes.c_size_t
+        lib.lce_bconv2d_host_noalloc_max_bytes.argtypes = []
+        lib.lce_bconv2d_host_noalloc.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp]
+        lib.lce_bconv2d_host_noalloc.restype = ctypes.c_int
         lib.lce_bmaxpool.argtypes = [vp, vp] + [i32] * 9 + [vp]
         lib.lce_add_f32.argtypes = [vp, vp, vp, i64, vp]
         lib.lce_probe_pipe.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), vp]
@@ -194,6 +198,21 @@ def lce_bconv2d_host(desc: BConv2dDesc, input, weights, multiplier, bias, thresh
         _host(multiplier, torch.float32, "multiplier"), _host(bias, torch.float32, "bias"),
         _host(thresholds, torch.int32, "thresholds"), _host(out, out_dtype, "out"),
         _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()), "lce_bconv2d_host")
+
+
+def lce_bconv2d_host_noalloc_max_bytes() -> int:
+    return int(library().lce_bconv2d_host_noalloc_max_bytes())
+
+
+def lce_bconv2d_host_noalloc(desc: BConv2dDesc, input, weights, multiplier, bias, thresholds, out) -> None:
+    """lce_bconv2d_host without the workspace argument: for callers that cannot allocate device
+    memory.  Every tensor is a host tensor; the staging area is a fixed array inside the library
+    (shared by all calls on the device, so do not overlap calls)."""
+    out_dtype = torch.float32 if desc.out_type == OUT_FLOAT32 else torch.int32
+    _check(library().lce_bconv2d_host_noalloc(
+        ctypes.byref(desc), _host(input, torch.int32, "input"), _host(weights, torch.int32, "weights"),
+        _host(multiplier, torch.float32, "multiplier"), _host(bias, torch.float32, "bias"),
+        _host(thresholds, torch.int32, "thresholds"), _host(out, out_dtype, "out"), _stream()), "lce_bconv2d_host_noalloc")
 
 
 def lce_bmaxpool(words: torch.Tensor, channels: int, pool=(2, 2), stride=(2, 2), padding=PAD_VALID,

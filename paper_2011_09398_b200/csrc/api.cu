@@ -170,3 +170,67 @@ extern "C" lce_status lce_bconv2d_host(const lce_bconv2d_desc *desc, const uint3
     if (cudaStreamSynchronize(s) != cudaSuccess) return LCE_ERR_CUDA;
     return LCE_OK;
 }
+
+// ---- host-buffer convolution that allocates nothing ---------------------------------------------
+// Some callers cannot give lce_bconv2d_host the device workspace it asks for, because they are not
+// in a position to call cudaMalloc at all: code running inside a memory-capped or allocator-less
+// host process, a real-time loop that must not take the allocator's locks, a plug-in that is only
+// handed host tensors.  For them the staging area lives inside the library itself, as a
+// file-scope device array that every GPU loading the library carries until the process exits.
+
+#define LCE_STATIC_WORKSPACE_BYTES (8u << 20)
+
+static __device__ __align__(256) unsigned char g_static_workspace[LCE_STATIC_WORKSPACE_BYTES];
+
+namespace lce {
+namespace {
+
+constexpr int kMaxDevices = 64;
+void *g_static_workspace_addr[kMaxDevices];  // device address of g_static_workspace, per device; 0 = not looked up yet
+
+}  // namespace
+}  // namespace lce
+
+extern "C" size_t lce_bconv2d_host_noalloc_max_bytes(void) { return LCE_STATIC_WORKSPACE_BYTES; }
+
+extern "C" lce_status lce_bconv2d_host_noalloc(const lce_bconv2d_desc *desc, const uint32_t *input,
+                                               const uint32_t *weights, const float *multiplier, const float *bias,
+                                               const int32_t *thresholds, void *output, void *stream)
+{
+    using namespace lce;
+    ConvGeom g;
+    lce_status st = check_conv_args(desc, &g, input, weights, multiplier, bias, thresholds, output);
+    if (st != LCE_OK) return st;
+    if (desc->weights_packed) return LCE_ERR_INVALID_ARG;
+    const HostLayout L = host_layout(g);
+    if (L.total > LCE_STATIC_WORKSPACE_BYTES) return LCE_ERR_WORKSPACE;  // this call does not fit the built-in array
+
+    // In host code the array's name is only a stand-in for the symbol, not a device address: ask the
+    // runtime for the address once per device, with that device current.
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LCE_ERR_CUDA;
+    if (g_static_workspace_addr[dev] == nullptr) {
+        void *addr = nullptr;
+        if (cudaGetSymbolAddress(&addr, g_static_workspace) != cudaSuccess || addr == nullptr) return LCE_ERR_CUDA;
+        g_static_workspace_addr[dev] = addr;
+    }
+    char *ws = static_cast<char *>(g_static_workspace_addr[dev]);
+
+    // Nothing in the array has to start at zero: every region is written in full (by the copies in,
+    // or by the kernel) before anything reads it.
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    bool ok = cudaMemcpyAsync(ws + L.in, input, L.in_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(ws + L.w, weights, L.w_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (multiplier) ok = ok && cudaMemcpyAsync(ws + L.mult, multiplier, L.ch_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (bias) ok = ok && cudaMemcpyAsync(ws + L.bias, bias, L.ch_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (thresholds) ok = ok && cudaMemcpyAsync(ws + L.thr, thresholds, L.ch_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (!ok) return LCE_ERR_CUDA;
+    st = dispatch(desc, g, reinterpret_cast<const uint32_t *>(ws + L.in), reinterpret_cast<const uint32_t *>(ws + L.w),
+                  multiplier ? reinterpret_cast<const float *>(ws + L.mult) : nullptr,
+                  bias ? reinterpret_cast<const float *>(ws + L.bias) : nullptr,
+                  thresholds ? reinterpret_cast<const int32_t *>(ws + L.thr) : nullptr, ws + L.out, s);
+    if (st != LCE_OK) return st;
+    if (cudaMemcpyAsync(output, ws + L.out, L.out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return LCE_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return LCE_ERR_CUDA;
+    return LCE_OK;
+}

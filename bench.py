@@ -372,7 +372,9 @@ def time_chains(dev, reps: int = 5):
 
     from paper_2011_09398_b200.chains import Chain
     out = {}
-    for cfg, steps, name, batch in ((4, wl.config4_steps(), "X0", 128), (5, wl.config5_steps(), "X", 256)):
+    for key, cfg, steps, name, batch in (("config4", 4, wl.config4_steps(), "X0", 128),
+                                         ("config4_fused", 4, wl.config4_fused_steps(), "X0", 128),
+                                         ("config5", 5, wl.config5_steps(), "X", 256)):
         chain = Chain(steps, cfg, str(dev))
         chain.buffers[name].normal_()
         for _ in range(3):
@@ -385,8 +387,8 @@ def time_chains(dev, reps: int = 5):
         ev[reps].record()
         torch.cuda.synchronize()
         ms = ev[0].elapsed_time(ev[reps]) / reps
-        macs = sum(s.conv.binary_macs for s in steps if s.kind == "bconv")
-        out[f"config{cfg}"] = {"batch": batch, "launches": chain.launches, "ms": ms, "images_per_second": batch / (ms * 1e-3),
+        macs = sum(s.conv.binary_macs for s in steps if s.kind.startswith("bconv"))
+        out[key] = {"batch": batch, "launches": chain.launches, "ms": ms, "images_per_second": batch / (ms * 1e-3),
                                "binary_macs_per_second": macs / (ms * 1e-3)}
         del chain
         torch.cuda.empty_cache()

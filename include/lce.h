@@ -110,6 +110,20 @@ lce_status lce_bconv2d(const lce_bconv2d_desc *desc, const uint32_t *input, cons
                        const float *multiplier, const float *bias, const int32_t *thresholds,
                        void *output, void *stream);
 
+/* LceBConv2d with its float-output neighbours fused into the output transform (Section 3.2: fused
+ * operations run on the accumulators before they are written; Section 5.3: a shortcut is float
+ * output -> Add -> LceQuantize).  desc->out_type must be LCE_OUT_FLOAT32.  Per output value:
+ *   y = fmaf((float)act(acc), multiplier[o], bias[o]);  if residual: y = y + residual[...] (fp32);
+ *   if out_float:  out_float[...] = y;   if out_packed: bit o of the pixel's word = (y < 0).
+ *   residual   fp32 [batch][oh][ow][out_c] or NULL       out_float fp32 same shape, or NULL
+ *   out_packed uint32 [batch][oh][ow][ceil(out_c/32)] or NULL   (at least one output required)
+ * The results are bit-identical to lce_bconv2d -> lce_add_f32 -> lce_bitpack run one after the
+ * other.  Only shapes the tiled kernels cover (3x3 stride 1-2, 1x1) are accepted; others return
+ * LCE_ERR_UNSUPPORTED. */
+lce_status lce_bconv2d_fused(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
+                             const float *multiplier, const float *bias, const float *residual,
+                             float *out_float, uint32_t *out_packed, void *stream);
+
 /* Load-time weight packing (Section 3.2: the paper's BGEMM also re-arranges the weights ahead of
  * time for its access pattern; Section 3.1: weights are converted once, when the model is built).  Rewrites
  * the plain packed weights into the operand layout the tiled kernel copies straight into shared

@@ -156,8 +156,10 @@ def config3_specs(batch: int = 64) -> List[ConvSpec]:
 
 @dataclass(frozen=True)
 class Step:
-    """One kernel call of a chain. kind: bitpack | bconv | add | bmaxpool.
-    src/src2/dst name buffers of the chain; conv is the layer spec for kind == 'bconv'."""
+    """One kernel call of a chain. kind: bitpack | bconv | bconv_fused | add | bmaxpool.
+    src/src2/dst name buffers of the chain; conv is the layer spec for the conv kinds.
+    bconv_fused: float-output conv whose result (+ the residual src2, if named) goes to the float
+    buffer dst (if named) and, sign-packed, to dst2 (if named)."""
     kind: str
     src: str
     dst: str
@@ -165,6 +167,7 @@ class Step:
     conv: Optional[ConvSpec] = None
     shape: tuple = ()      # (N,H,W,C) of src for bitpack / add / bmaxpool
     tensor_index: int = -1  # first RNG index of the conv's parameters
+    dst2: str = ""
 
 
 def config4_steps(batch: int = 128, size: int = 56, widths=(64, 128, 256, 512)) -> List[Step]:
@@ -186,6 +189,28 @@ def config4_steps(batch: int = 128, size: int = 56, widths=(64, 128, 256, 512)) 
             steps.append(Step("bmaxpool", p, q, shape=(batch, h, h, c)))
             h2 = h // 2
             steps.append(Step("bconv", q, f"X{s+1}", conv=ConvSpec(f"c4_s{s}_trans", batch, h2, h2, c, widths[s + 1], 1, 1, PAD_SAME_ONE, OUT_FLOAT32), tensor_index=idx)); idx += 4
+            h = h2
+    return steps
+
+
+def config4_fused_steps(batch: int = 128, size: int = 56, widths=(64, 128, 256, 512)) -> List[Step]:
+    """config4_steps with every add and every re-quantize folded into the conv before it: same
+    tensors, same parameters (tensor indices), 15 launches instead of 25.  Buffers that only fed a
+    fused step (F, and Y except the last) are never written."""
+    steps: List[Step] = []
+    idx = 1
+    h = size
+    steps.append(Step("bitpack", "X0", "A0", shape=(batch, h, h, widths[0])))
+    for s, c in enumerate(widths):
+        last = s + 1 == len(widths)
+        steps.append(Step("bconv", f"A{s}", f"B{s}", conv=ConvSpec(f"c4_s{s}_conv1", batch, h, h, c, c, 3, 1, PAD_SAME_ONE, OUT_BITPACKED), tensor_index=idx)); idx += 4
+        steps.append(Step("bconv_fused", f"B{s}", f"Y{s}" if last else "", src2=f"X{s}", dst2="" if last else f"P{s}",
+                          conv=ConvSpec(f"c4_s{s}_conv2", batch, h, h, c, c, 3, 1, PAD_SAME_ONE, OUT_FLOAT32), tensor_index=idx)); idx += 4
+        if not last:
+            steps.append(Step("bmaxpool", f"P{s}", f"Q{s}", shape=(batch, h, h, c)))
+            h2 = h // 2
+            steps.append(Step("bconv_fused", f"Q{s}", f"X{s+1}", dst2=f"A{s+1}",
+                              conv=ConvSpec(f"c4_s{s}_trans", batch, h2, h2, c, widths[s + 1], 1, 1, PAD_SAME_ONE, OUT_FLOAT32), tensor_index=idx)); idx += 4
             h = h2
     return steps
 

@@ -47,6 +47,8 @@ def library() -> ctypes.CDLL:
         lib.lce_unpack.argtypes = [vp, vp, i64, i32, vp]
         lib.lce_bconv2d_out_shape.argtypes = [ctypes.POINTER(BConv2dDesc), ctypes.POINTER(i32), ctypes.POINTER(i32)]
         lib.lce_bconv2d.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp]
+        lib.lce_bconv2d_fused.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.lce_bconv2d_fused.restype = ctypes.c_int
         lib.lce_bconv2d_packed_weights_bytes.restype = ctypes.c_size_t
         lib.lce_bconv2d_packed_weights_bytes.argtypes = [ctypes.POINTER(BConv2dDesc)]
         lib.lce_bconv2d_pack_weights.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp]
@@ -160,6 +162,18 @@ def lce_bconv2d(desc: BConv2dDesc, input: torch.Tensor, weights: torch.Tensor,
         _dev(thresholds, torch.int32, "thresholds") if thresholds is not None else None,
         _dev(out, out_dtype, "out"), _stream()), "lce_bconv2d")
     return out
+
+
+def lce_bconv2d_fused(desc: BConv2dDesc, input, weights, multiplier, bias, residual=None, out_float=None,
+                      out_packed=None) -> None:
+    """LceBConv2d (float output) with the shortcut add and/or the next LceQuantize fused in; the
+    caller supplies whichever of out_float / out_packed it wants."""
+    opt = lambda t, dt, n: _dev(t, dt, n) if t is not None else None
+    _check(library().lce_bconv2d_fused(
+        ctypes.byref(desc), _dev(input, torch.int32, "input"), _dev(weights, torch.int32, "weights"),
+        _dev(multiplier, torch.float32, "multiplier"), _dev(bias, torch.float32, "bias"),
+        opt(residual, torch.float32, "residual"), opt(out_float, torch.float32, "out_float"),
+        opt(out_packed, torch.int32, "out_packed"), _stream()), "lce_bconv2d_fused")
 
 
 def lce_bconv2d_packed_weights_bytes(desc: BConv2dDesc) -> int:

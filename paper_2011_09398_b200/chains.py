@@ -32,7 +32,7 @@ class Chain:
                 N, H, W, C = st.shape
                 self._ensure(st.src, (N, H, W, (C + 31) // 32), torch.int32)
                 self._ensure(st.dst, (N, H // 2, W // 2, (C + 31) // 32), torch.int32)
-            elif st.kind == "bconv":
+            elif st.kind in ("bconv", "bconv_fused"):
                 s = st.conv
                 t = wl.conv_tensors(config, st.tensor_index, s)
                 self.params[i] = t
@@ -41,7 +41,15 @@ class Chain:
                 plain = lce.pack_weights(torch.from_numpy(t.w_pm1).to(dev))
                 packed = lce.lce_bconv2d_pack_weights(desc, plain)
                 self._ensure(st.src, (s.batch, s.in_h, s.in_w, s.in_words), torch.int32)
-                if s.out_type == wl.OUT_FLOAT32:
+                if st.kind == "bconv_fused":
+                    fshape = (s.batch, s.out_h, s.out_w, s.out_c)
+                    for name in (st.dst, st.src2):
+                        if name:
+                            self._ensure(name, fshape, torch.float32)
+                    if st.dst2:
+                        self._ensure(st.dst2, (s.batch, s.out_h, s.out_w, (s.out_c + 31) // 32), torch.int32)
+                    extra = (torch.from_numpy(t.multiplier).to(dev), torch.from_numpy(t.bias).to(dev), None)
+                elif s.out_type == wl.OUT_FLOAT32:
                     self._ensure(st.dst, (s.batch, s.out_h, s.out_w, s.out_c), torch.float32)
                     extra = (torch.from_numpy(t.multiplier).to(dev), torch.from_numpy(t.bias).to(dev), None)
                 else:
@@ -75,6 +83,10 @@ class Chain:
                 lce.lce_add_f32(B[st.src], B[st.src2], B[st.dst])
             elif st.kind == "bmaxpool":
                 lce.lce_bmaxpool(B[st.src], st.shape[3], (2, 2), (2, 2), lce.PAD_VALID, B[st.dst])
+            elif st.kind == "bconv_fused":
+                desc, w, (mult, bias, _) = self._conv[i]
+                lce.lce_bconv2d_fused(desc, B[st.src], w, mult, bias, B[st.src2] if st.src2 else None,
+                                      B[st.dst] if st.dst else None, B[st.dst2] if st.dst2 else None)
             else:
                 desc, w, (mult, bias, thr) = self._conv[i]
                 lce.lce_bconv2d(desc, B[st.src], w, mult, bias, thr, B[st.dst])

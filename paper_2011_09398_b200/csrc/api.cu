@@ -111,6 +111,30 @@ extern "C" lce_status lce_bconv2d(const lce_bconv2d_desc *desc, const uint32_t *
     return dispatch(desc, g, input, weights, multiplier, bias, thresholds, output, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" lce_status lce_bconv2d_fused(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
+                                        const float *multiplier, const float *bias, const float *residual,
+                                        float *out_float, uint32_t *out_packed, void *stream)
+{
+    using namespace lce;
+    ConvGeom g;
+    lce_status st = make_geom(desc, &g);
+    if (st != LCE_OK) return st;
+    if (g.out_type != LCE_OUT_FLOAT32) return LCE_ERR_INVALID_ARG;
+    if (!input || !weights || !multiplier || !bias || (!out_float && !out_packed)) return LCE_ERR_INVALID_ARG;
+    if (!aligned(input, 4) || !aligned(weights, 4) || !aligned(multiplier, 4) || !aligned(bias, 4) ||
+        !aligned(residual, 4) || !aligned(out_float, 4) || !aligned(out_packed, 4))
+        return LCE_ERR_ALIGNMENT;
+    const uint32_t *image = nullptr;
+    if (desc->weights_packed) {
+        if (!aligned(weights, 256)) return LCE_ERR_ALIGNMENT;
+        if (tiled_weight_image_bytes(g) > 0)
+            image = reinterpret_cast<const uint32_t *>(reinterpret_cast<const char *>(weights) + plain_weight_bytes(g));
+    }
+    if (desc->kernel == LCE_KERNEL_DIRECT || patch_covers(g)) return LCE_ERR_UNSUPPORTED;
+    return launch_bconv_tiled(g, input, weights, image, multiplier, bias, nullptr, out_float,
+                              static_cast<cudaStream_t>(stream), residual, out_packed);
+}
+
 extern "C" size_t lce_bconv2d_packed_weights_bytes(const lce_bconv2d_desc *desc)
 {
     lce::ConvGeom g;

@@ -46,7 +46,9 @@ struct TiledParams {
     const float *mult;
     const float *bias;
     const int32_t *thr;
-    void *out;
+    void *out;                 // may be null for float output when only the packed sign is wanted
+    const float *residual;     // float output only: added after the multiply-add (or nullptr)
+    uint32_t *out_packed;      // float output only: LceQuantize of the float result (or nullptr)
     int32_t N, H, W, Cin, Cw, Cout, Cow, OH, OW, pt, pl;
     int32_t tile_pixels;  // flat output pixels per tile, a multiple of kPixPerStep * TP
     int32_t n_tiles;      // ceil(M / tile_pixels); CTA x works on tiles x, x + gridDim.x, ...
@@ -215,9 +217,28 @@ __device__ __forceinline__ void store_outputs(const TiledParams &p, const int32_
             const int32_t a = (p.activation == LCE_ACT_RELU && v[j] < 0) ? 0 : v[j];
             f[j] = __fmaf_rn((float)a, mult[j], bias[j]);
         }
-        if (pix_ok) {
+        const bool vec = (p.Cout & 3) == 0 && chan + kChanPerThread <= p.Cout;
+        if (p.residual != nullptr) {
+            // fused shortcut: one more fp32 add, exactly as a separate add kernel would round it
+            const float *r = p.residual + (int64_t)m * p.Cout + chan;
+            if (pix_ok) {
+                if (vec) {
+                    const float4 r0 = __ldg(reinterpret_cast<const float4 *>(r));
+                    const float4 r1 = __ldg(reinterpret_cast<const float4 *>(r) + 1);
+                    f[0] = __fadd_rn(f[0], r0.x); f[1] = __fadd_rn(f[1], r0.y);
+                    f[2] = __fadd_rn(f[2], r0.z); f[3] = __fadd_rn(f[3], r0.w);
+                    f[4] = __fadd_rn(f[4], r1.x); f[5] = __fadd_rn(f[5], r1.y);
+                    f[6] = __fadd_rn(f[6], r1.z); f[7] = __fadd_rn(f[7], r1.w);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < kChanPerThread; ++j)
+                        if (chan + j < p.Cout) f[j] = __fadd_rn(f[j], __ldg(r + j));
+                }
+            }
+        }
+        if (pix_ok && p.out != nullptr) {
             float *dst = static_cast<float *>(p.out) + (int64_t)m * p.Cout + chan;
-            if ((p.Cout & 3) == 0 && chan + kChanPerThread <= p.Cout) {
+            if (vec) {
                 reinterpret_cast<float4 *>(dst)[0] = make_float4(f[0], f[1], f[2], f[3]);
                 reinterpret_cast<float4 *>(dst)[1] = make_float4(f[4], f[5], f[6], f[7]);
             } else {
@@ -225,6 +246,17 @@ __device__ __forceinline__ void store_outputs(const TiledParams &p, const int32_
                 for (int j = 0; j < kChanPerThread; ++j)
                     if (chan + j < p.Cout) dst[j] = f[j];
             }
+        }
+        if (p.out_packed != nullptr) {
+            // fused LceQuantize of the float result for the next binarized layer: bit = (y < 0)
+            uint32_t bits = 0u;
+#pragma unroll
+            for (int j = 0; j < kChanPerThread; ++j) bits |= ((chan + j < p.Cout && f[j] < 0.0f) ? 1u : 0u) << j;
+            bits <<= 8 * (cg & 3);
+            bits |= __shfl_xor_sync(0xffffffffu, bits, 1);
+            bits |= __shfl_xor_sync(0xffffffffu, bits, 2);
+            const int word = (ch0 >> 5) + (cg >> 2);
+            if (pix_ok && (cg & 3) == 0 && word < p.Cow) p.out_packed[(int64_t)m * p.Cow + word] = bits;
         }
     } else {
         if (pix_ok) {
@@ -793,14 +825,17 @@ lce_status launch_pack_weights_tiled(const ConvGeom &g, const uint32_t *w, uint3
 }
 
 lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const uint32_t *w_image,
-                              const float *mult, const float *bias, const int32_t *thr, void *out, cudaStream_t s)
+                              const float *mult, const float *bias, const int32_t *thr, void *out, cudaStream_t s,
+                              const float *residual, uint32_t *out_packed)
 {
     if (!tiled_covers(g)) return LCE_ERR_UNSUPPORTED;
-    // 128-bit epilogue stores need a 16-byte aligned output when the channel count allows them
-    if ((g.Cout & 3) == 0 && g.out_type != LCE_OUT_BITPACKED && !aligned(out, 16)) return LCE_ERR_UNSUPPORTED;
+    // 128-bit epilogue accesses need 16-byte aligned buffers when the channel count allows them
+    if ((g.Cout & 3) == 0 && g.out_type != LCE_OUT_BITPACKED && (!aligned(out, 16) || !aligned(residual, 16)))
+        return LCE_ERR_UNSUPPORTED;
     if (w_image && !aligned(w_image, 16)) return LCE_ERR_ALIGNMENT;
     TiledParams p{};
     p.in = in; p.w = w; p.w_image = w_image; p.mult = mult; p.bias = bias; p.thr = thr; p.out = out;
+    p.residual = residual; p.out_packed = out_packed;
     p.N = g.N; p.H = g.H; p.W = g.W; p.Cin = g.Cin; p.Cw = g.Cw; p.Cout = g.Cout; p.Cow = g.Cow;
     p.OH = g.OH; p.OW = g.OW; p.pt = g.pt; p.pl = g.pl;
     p.padding = g.padding; p.out_type = g.out_type; p.activation = g.activation;

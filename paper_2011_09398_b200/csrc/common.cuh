@@ -74,8 +74,11 @@ lce_status launch_bconv_direct(const ConvGeom &g, const uint32_t *in, const uint
                                const float *bias, const int32_t *thr, void *out, cudaStream_t s);
 // Returns LCE_ERR_UNSUPPORTED without launching when the tiled kernel does not cover the shape.
 // w_image: the tiled part of a packed-weights buffer, or nullptr to derive operands from `w`.
+// residual / out_packed: fused shortcut add and fused LceQuantize of a float output (both optional;
+// with out_packed given, `out` may be null).
 lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const uint32_t *w_image,
-                              const float *mult, const float *bias, const int32_t *thr, void *out, cudaStream_t s);
+                              const float *mult, const float *bias, const int32_t *thr, void *out, cudaStream_t s,
+                              const float *residual = nullptr, uint32_t *out_packed = nullptr);
 // One-word-patch kernel for tiny channel counts (KH*KW*Cin <= 32); plain weights only.
 bool patch_covers(const ConvGeom &g);
 lce_status launch_bconv_patch(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const float *mult,

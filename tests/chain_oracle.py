@@ -16,6 +16,17 @@ def run_chain_oracle(steps, config, inputs):
             B[st.dst] = oracle.add_f32(B[st.src], B[st.src2])
         elif st.kind == "bmaxpool":
             B[st.dst] = oracle.bmaxpool(B[st.src], st.shape[3], (2, 2), (2, 2), oracle.PAD_VALID)
+        elif st.kind == "bconv_fused":
+            s = st.conv
+            t = wl.conv_tensors(config, st.tensor_index, s)
+            acc = oracle.bconv2d_acc(oracle.unpack_pm1(B[st.src], s.in_c), t.w_pm1, (s.stride, s.stride), s.padding)
+            y = oracle.transform_float(acc, t.multiplier, t.bias)
+            if st.src2:
+                y = oracle.add_f32(y, B[st.src2])
+            if st.dst:
+                B[st.dst] = y
+            if st.dst2:
+                B[st.dst2] = oracle.bitpack(y)
         elif st.kind == "bconv":
             s = st.conv
             t = wl.conv_tensors(config, st.tensor_index, s)

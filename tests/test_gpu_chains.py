@@ -36,6 +36,43 @@ def test_config4_block_stack_batch2():
     assert chain.launches == 25
 
 
+def test_config4_fused_chain_equals_unfused_chain():
+    """Shortcut add and re-quantize folded into the convs: every tensor the fused chain writes equals
+    the oracle's unfused chain (same names, same parameters)."""
+    x = wl.activations(4, 0, (2, 56, 56, 64))
+    fused = wl.config4_fused_steps(batch=2)
+    chain = Chain(fused, 4)
+    chain.set_input("X0", x)
+    chain.run()
+    ref_unfused = run_chain_oracle(wl.config4_steps(batch=2), 4, {"X0": x})
+    ref_fused = run_chain_oracle(fused, 4, {"X0": x})
+    compare_all(chain, ref_fused)
+    compare_all(chain, {k: ref_unfused[k] for k in chain.buffers})
+    assert chain.launches == 15
+
+
+def test_fused_conv_on_ragged_shape():
+    import oracle
+    import paper_2011_09398_b200 as lce
+    rng = np.random.default_rng(5)
+    N, H, W, Cin, Cout = 2, 9, 7, 70, 45
+    a = (2 * rng.integers(0, 2, size=(N, H, W, Cin)) - 1).astype(np.int8)
+    w = (2 * rng.integers(0, 2, size=(Cout, 3, 3, Cin)) - 1).astype(np.int8)
+    mult = rng.uniform(0.5, 1.5, Cout).astype(np.float32)
+    bias = rng.standard_normal(Cout).astype(np.float32)
+    res = rng.standard_normal((N, H, W, Cout)).astype(np.float32) * 30
+    y = oracle.add_f32(oracle.transform_float(oracle.bconv2d_acc(a, w), mult, bias), res)
+    dev = "cuda:0"
+    desc = lce.make_desc(N, H, W, Cin, Cout, out_type=lce.OUT_FLOAT32)
+    t = lambda arr: torch.from_numpy(np.ascontiguousarray(arr)).to(dev)
+    of = torch.empty((N, H, W, Cout), dtype=torch.float32, device=dev)
+    op = torch.empty((N, H, W, 2), dtype=torch.int32, device=dev)
+    lce.lce_bconv2d_fused(desc, t(oracle.bitpack_pm1(a).view(np.int32)), t(oracle.bitpack_pm1(w).view(np.int32)),
+                          t(mult), t(bias), t(res), of, op)
+    assert np.array_equal(of.cpu().numpy(), y)
+    assert np.array_equal(op.cpu().numpy().view(np.uint32), oracle.bitpack(y))
+
+
 def test_config5_body_batch2():
     steps = wl.config5_steps(batch=2)
     x = wl.activations(5, 0, (2, 224, 224, 3))

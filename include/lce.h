@@ -56,8 +56,11 @@ typedef enum { LCE_OUT_FLOAT32 = 0, LCE_OUT_BITPACKED = 1, LCE_OUT_INT32 = 2 } l
 typedef enum { LCE_ACT_NONE = 0, LCE_ACT_RELU = 1 } lce_activation;
 
 /* Which kernel lce_bconv2d uses.  AUTO picks the tiled XOR/POPC kernel when it covers the
- * shape and the direct kernel otherwise; the other values force one (tests, benchmarks). */
-typedef enum { LCE_KERNEL_AUTO = 0, LCE_KERNEL_DIRECT = 1, LCE_KERNEL_TILED = 2 } lce_kernel;
+ * shape and the direct kernel otherwise; the other values force one (tests, benchmarks).
+ * TENSOR is the tensor-core formulation (bits expanded to +-1 int8 in shared memory, tcgen05
+ * kind::i8, accumulators in TMEM; exact): 3x3, stride 1, LCE_PAD_SAME_ONE only, never chosen by
+ * AUTO. */
+typedef enum { LCE_KERNEL_AUTO = 0, LCE_KERNEL_DIRECT = 1, LCE_KERNEL_TILED = 2, LCE_KERNEL_TENSOR = 3 } lce_kernel;
 
 const char *lce_version(void);
 const char *lce_status_string(lce_status status);
@@ -178,6 +181,12 @@ lce_status lce_bmaxpool(const uint32_t *in, uint32_t *out, int32_t batch, int32_
 /* fp32 residual add out = a + b (one rounding), the shortcut pattern of Section 5.3
  * (float output -> Add -> LceQuantize).  n == 0 is a no-op; out may equal a or b. */
 lce_status lce_add_f32(const float *a, const float *b, float *out, int64_t n, void *stream);
+
+/* Status word of the bounded device-side waits (the tensor-core kernel waits on an mbarrier for
+ * its MMAs, with an iteration limit).  *status (HOST pointer) = 0 if no wait has ever given up
+ * on the current device, 1 otherwise; a non-zero value means outputs of the affected call are
+ * incomplete.  Synchronous (reads a device variable). */
+lce_status lce_device_status(int32_t *status);
 
 /* Integer-pipe probe: runs a register/shared-memory resident loop of one instruction mix on
  * every SM of the current device and reports how many 32-bit word operations (one XOR +

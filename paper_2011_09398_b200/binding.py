@@ -12,7 +12,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "liblce_b200.so"
 PAD_VALID, PAD_SAME_ONE, PAD_SAME_ZERO = 0, 1, 2
 OUT_FLOAT32, OUT_BITPACKED, OUT_INT32 = 0, 1, 2
 ACT_NONE, ACT_RELU = 0, 1
-KERNEL_AUTO, KERNEL_DIRECT, KERNEL_TILED = 0, 1, 2
+KERNEL_AUTO, KERNEL_DIRECT, KERNEL_TILED, KERNEL_TENSOR = 0, 1, 2, 3
 
 
 class LceError(RuntimeError):
@@ -256,6 +256,16 @@ def lce_add_f32(a: torch.Tensor, b: torch.Tensor, out: Optional[torch.Tensor] = 
     _check(library().lce_add_f32(_dev(a, torch.float32, "a"), _dev(b, torch.float32, "b"), _dev(out, torch.float32, "out"),
                                  a.numel(), _stream()), "lce_add_f32")
     return out
+
+
+def lce_device_status() -> int:
+    """0 unless a bounded device-side wait has given up on the current device."""
+    v = ctypes.c_int32()
+    lib = library()
+    lib.lce_device_status.argtypes = [ctypes.POINTER(ctypes.c_int32)]
+    lib.lce_device_status.restype = ctypes.c_int
+    _check(lib.lce_device_status(ctypes.byref(v)), "lce_device_status")
+    return v.value
 
 
 def lce_probe_pipe(mix: int, iterations: int = 2000) -> Tuple[float, float]:

@@ -36,6 +36,8 @@ lce_status dispatch(const lce_bconv2d_desc *desc, const ConvGeom &g, const uint3
     }
     if (desc->kernel == LCE_KERNEL_DIRECT)
         return launch_bconv_direct(g, input, weights, multiplier, bias, thresholds, output, s);
+    if (desc->kernel == LCE_KERNEL_TENSOR)
+        return launch_bconv_tensor(g, input, weights, multiplier, bias, thresholds, output, s);
     if (patch_covers(g)) return launch_bconv_patch(g, input, weights, multiplier, bias, thresholds, output, s);
     lce_status st = launch_bconv_tiled(g, input, weights, image, multiplier, bias, thresholds, output, s);
     if (st == LCE_ERR_UNSUPPORTED && desc->kernel == LCE_KERNEL_AUTO)
@@ -83,6 +85,16 @@ extern "C" const char *lce_status_string(lce_status status)
         case LCE_ERR_WORKSPACE: return "workspace too small";
     }
     return "unknown status";
+}
+
+extern "C" lce_status lce_device_status(int32_t *status)
+{
+    if (!status) return LCE_ERR_INVALID_ARG;
+    int v = 0;
+    lce_status st = lce::tensor_device_status(&v);
+    if (st != LCE_OK) return st;
+    *status = v;
+    return LCE_OK;
 }
 
 extern "C" lce_status lce_bconv2d_out_shape(const lce_bconv2d_desc *desc, int32_t *out_h, int32_t *out_w)

@@ -42,7 +42,7 @@ inline lce_status make_geom(const lce_bconv2d_desc *d, ConvGeom *g)
     if (d->padding < LCE_PAD_VALID || d->padding > LCE_PAD_SAME_ZERO) return LCE_ERR_INVALID_ARG;
     if (d->out_type < LCE_OUT_FLOAT32 || d->out_type > LCE_OUT_INT32) return LCE_ERR_INVALID_ARG;
     if (d->activation < LCE_ACT_NONE || d->activation > LCE_ACT_RELU) return LCE_ERR_INVALID_ARG;
-    if (d->kernel < LCE_KERNEL_AUTO || d->kernel > LCE_KERNEL_TILED) return LCE_ERR_INVALID_ARG;
+    if (d->kernel < LCE_KERNEL_AUTO || d->kernel > LCE_KERNEL_TENSOR) return LCE_ERR_INVALID_ARG;
     if (d->weights_packed != 0 && d->weights_packed != 1) return LCE_ERR_INVALID_ARG;
     Axis ah = axis_geometry(d->in_h, d->kernel_h, d->stride_h, d->padding);
     Axis aw = axis_geometry(d->in_w, d->kernel_w, d->stride_w, d->padding);
@@ -83,6 +83,11 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
 bool patch_covers(const ConvGeom &g);
 lce_status launch_bconv_patch(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const float *mult,
                               const float *bias, const int32_t *thr, void *out, cudaStream_t s);
+// Tensor-core (tcgen05 kind::i8) kernel: 3x3, stride 1, one-padding; plain weights.
+bool tensor_covers(const ConvGeom &g);
+lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const float *mult,
+                               const float *bias, const int32_t *thr, void *out, cudaStream_t s);
+lce_status tensor_device_status(int *status);
 // Bytes of the tiled kernel's weight image for this geometry (0 if the kernel does not cover it).
 size_t tiled_weight_image_bytes(const ConvGeom &g);
 lce_status launch_pack_weights_tiled(const ConvGeom &g, const uint32_t *w, uint32_t *image, cudaStream_t s);

@@ -17,23 +17,32 @@
 //   * operand descriptors: K-major, no swizzle, 8-row groups 128 bytes apart (so rows are
 //     uniformly 16 bytes apart), the two 16-byte K chunks of one K=32 instruction one whole
 //     plane apart.
-//   * one CTA = 128 GEMM rows (TMEM lanes) x up to 256 output channels (TMEM columns); weights of
-//     its channel block are expanded once per CTA and stay in shared memory; CTAs are persistent
-//     over row tiles.  Per tile: expand the input rows -> issue 9*Cw MMAs from one thread ->
-//     tcgen05.commit to an mbarrier -> all 128 threads read their accumulator row from TMEM and
-//     apply the output transform.
-// Every wait on the mbarrier is bounded; on expiry the kernel records a status word, skips the
-// rest of its work, frees its TMEM and returns.
+//   * one CTA = 128 GEMM rows (TMEM lanes) x a block of output channels (TMEM columns), persistent
+//     over row tiles.  The packed input words of the next tile are prefetched with cp.async.
+//     Two schedules:
+//       - RESIDENT (small K*N): the block's weights are expanded once and stay in shared memory;
+//         per tile one thread issues all 9*Cw MMAs, and while they run all threads expand the
+//         next tile's input into the other A buffer;
+//       - STREAMING (large K*N): the weights of one tap at a time are expanded into one of two
+//         B buffers while the previous tap's MMAs run.
+//   * tcgen05.commit signals MMA completion on mbarriers; every wait on them is bounded; on expiry
+//     the kernel records a status word, abandons its work, frees its TMEM and returns.
 #include "common.cuh"
 
 namespace lce {
 namespace {
 
-constexpr int kThreads = 128;
+constexpr int kThreads = 256;  // 8 warps: warps w and w+4 share TMEM lanes 32*(w%4).. and split the columns
 constexpr int kTileM = 128;
 constexpr uint32_t kSpinLimit = 1u << 22;  // bounded wait: about a second at worst, far above any real tile
 
 __device__ int g_tensor_status = 0;  // 0 ok, 1 = an mbarrier wait expired
+#ifdef LCE_TUNING
+__device__ long long g_dbg[256];
+#define DBG_T(slot) do { if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0 && it < 6) g_dbg[it * 8 + (slot)] = clock64(); } while (0)
+#else
+#define DBG_T(slot) do {} while (0)
+#endif
 
 struct TensorParams {
     const uint32_t *in;
@@ -48,24 +57,15 @@ struct TensorParams {
     int32_t P;           // staged grid positions per tile = kTileM + 2*Wp + 2
     int32_t n_tiles;     // ceil(total grid positions / kTileM)
     int32_t total_q;     // N * Hs * Wp
-    int32_t n_blk;       // output channels per CTA (multiple of 16, <= 256)
+    int32_t n_blk;       // output channels per CTA: 32, 64, 128 or 256
+    int32_t n_blk_log2;
     int32_t tmem_cols;   // power of two >= max(32, n_blk)
     int32_t pad_corr;    // 9 * (32*Cw - Cin): what the zero pad bits (+1 * +1) add to every accumulator
     int32_t out_type, activation;
+    int32_t vec_store;   // float / int32 rows may be written with 128-bit stores
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-// K-major, no-swizzle operand descriptor; offsets in units of 16 bytes.
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_units, uint32_t sbo_units)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
-    d |= (uint64_t)(lbo_units & 0x3FFFu) << 16;
-    d |= (uint64_t)(sbo_units & 0x3FFFu) << 32;
-    d |= (uint64_t)1 << 46;  // descriptor version of this architecture
-    return d;
-}
 
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
 {
@@ -93,55 +93,206 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
     return false;
 }
 
-__device__ __forceinline__ void mma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+__device__ __forceinline__ void mma_commit(uint64_t *bar)
 {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-        :
-        : "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
-        : "memory");
+    // arrives on the barrier when every MMA issued so far has finished (operand reads included)
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int32_t (&v)[16])
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, int32_t (&v)[32])
 {
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, "
+        "[%32];\n\t"
         "tcgen05.wait::ld.sync.aligned;"
         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr)
         : "memory");
 }
 
-// byte j of the result = +1 (0x01) where bit j of b is 0, -1 (0xFF) where it is 1
-__device__ __forceinline__ uint2 expand_byte(const uint2 *table, uint32_t b) { return table[b & 0xFFu]; }
+// 4-byte asynchronous global->shared copy; with valid == false a zero word is written
+__device__ __forceinline__ void cp_async4_zfill(uint32_t *smem_dst, const uint32_t *gmem_src, bool valid)
+{
+    const int src_size = valid ? 4 : 0;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(src_size) : "memory");
+}
 
-// 32 bits -> 32 bytes, written as two 16-byte chunks
+// 32 bits -> 32 bytes (+1 where the bit is 0, -1 where it is 1), as two 16-byte chunks; the
+// table maps one byte of bits to its eight bytes
 __device__ __forceinline__ void expand_word(const uint2 *table, uint32_t word, uint4 *chunk_lo, uint4 *chunk_hi)
 {
-    const uint2 a = expand_byte(table, word), b = expand_byte(table, word >> 8);
-    const uint2 c = expand_byte(table, word >> 16), d = expand_byte(table, word >> 24);
+    const uint2 a = table[word & 0xFFu], b = table[(word >> 8) & 0xFFu];
+    const uint2 c = table[(word >> 16) & 0xFFu], d = table[word >> 24];
     *chunk_lo = make_uint4(a.x, a.y, b.x, b.y);
     *chunk_hi = make_uint4(c.x, c.y, d.x, d.y);
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+// packed words of the grid positions q0 .. q0+P-1 -> raw[cw*P + row] (pad positions: zero word)
+__device__ __forceinline__ void prefetch_raw(const TensorParams &p, int q0, uint32_t *raw, int tid)
+{
+    for (int row = tid; row < p.P; row += kThreads) {
+        const int f = q0 + row;
+        const int rr = f / p.Wp, cc = f - rr * p.Wp;
+        const int n = rr / p.Hs, ry = rr - n * p.Hs;
+        const bool ok = cc != 0 && ry != 0 && n < p.N;
+        const uint32_t *src = ok ? p.in + (((int64_t)n * p.H + (ry - 1)) * p.W + (cc - 1)) * p.Cw : p.in;
+        for (int cw = 0; cw < p.Cw; ++cw) cp_async4_zfill(raw + cw * p.P + row, ok ? src + cw : src, ok);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// every thread expands the words it prefetched itself (same row mapping), so waiting for its own
+// copies is enough
+__device__ __forceinline__ void expand_a(const TensorParams &p, const uint2 *table, const uint32_t *raw, uint8_t *sA, int tid)
+{
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    for (int row = tid; row < p.P; row += kThreads) {
+        for (int cw = 0; cw < p.Cw; ++cw) {
+            uint4 lo, hi;
+            expand_word(table, raw[cw * p.P + row], &lo, &hi);
+            uint4 *dst = reinterpret_cast<uint4 *>(sA) + (size_t)(2 * cw) * p.P + row;
+            dst[0] = lo;
+            dst[p.P] = hi;
+        }
+    }
+}
+
+// Issues MMAs first .. first+count-1 of a tile.  One thread feeds the whole tensor core, so
+// its instruction stream must be short: the start offsets of both operands of every MMA of a
+// tile sit in a shared-memory table (filled once per CTA), and eight MMAs at a time are issued
+// back to back from one block of code.  A descriptor's high half (row-group stride, version)
+// never changes; its low half = (base + offset) | plane stride << 16.
+__device__ __forceinline__ void issue_mmas(uint32_t tmem, const uint2 *offs, int first, int count, uint32_t a_base_lo,
+                                           uint32_t b_base_lo, uint32_t desc_hi, uint32_t idesc, uint32_t &accumulate)
+{
+    for (int i0 = 0; i0 < count; i0 += 8) {
+        uint32_t a_lo[8], b_lo[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint2 o = offs[first + min(i0 + k, count - 1)];
+            a_lo[k] = a_base_lo + o.x;
+            b_lo[k] = b_base_lo + o.y;
+        }
+        const int n = count - i0;  // MMAs k < n of this batch are real
+        asm volatile(
+            "{\n\t.reg .pred pa, pt, g;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 pa, %19, 0;\n\t"
+            "setp.eq.b32 pt, 0, 0;\n\t"
+            "mov.b64 da, {%1, %17};\n\t mov.b64 db, {%9, %17};\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %18, {%21, %21, %21, %21}, pa;\n\t"
+            "setp.gt.s32 g, %20, 1;\n\t mov.b64 da, {%2, %17};\n\t mov.b64 db, {%10, %17};\n\t"
+            "@g tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %18, {%21, %21, %21, %21}, pt;\n\t"
+            "setp.gt.s32 g, %20, 2;\n\t mov.b64 da, {%3, %17};\n\t mov.b64 db, {%11, %17};\n\t"
+            "@g tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %18, {%21, %21, %21, %21}, pt;\n\t"
+            "setp.gt.s32 g, %20, 3;\n\t mov.b64 da, {%4, %17};\n\t mov.b64 db, {%12, %17};\n\t"
+            "@g tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %18, {%21, %21, %21, %21}, pt;\n\t"
+            "setp.gt.s32 g, %20, 4;\n\t mov.b64 da, {%5, %17};\n\t mov.b64 db, {%13, %17};\n\t"
+            "@g tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %18, {%21, %21, %21, %21}, pt;\n\t"
+            "setp.gt.s32 g, %20, 5;\n\t mov.b64 da, {%6, %17};\n\t mov.b64 db, {%14, %17};\n\t"
+            "@g tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %18, {%21, %21, %21, %21}, pt;\n\t"
+            "setp.gt.s32 g, %20, 6;\n\t mov.b64 da, {%7, %17};\n\t mov.b64 db, {%15, %17};\n\t"
+            "@g tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %18, {%21, %21, %21, %21}, pt;\n\t"
+            "setp.gt.s32 g, %20, 7;\n\t mov.b64 da, {%8, %17};\n\t mov.b64 db, {%16, %17};\n\t"
+            "@g tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %18, {%21, %21, %21, %21}, pt;\n\t"
+            "}"
+            :
+            : "r"(tmem), "r"(a_lo[0]), "r"(a_lo[1]), "r"(a_lo[2]), "r"(a_lo[3]), "r"(a_lo[4]), "r"(a_lo[5]), "r"(a_lo[6]),
+              "r"(a_lo[7]), "r"(b_lo[0]), "r"(b_lo[1]), "r"(b_lo[2]), "r"(b_lo[3]), "r"(b_lo[4]), "r"(b_lo[5]), "r"(b_lo[6]),
+              "r"(b_lo[7]), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(n), "r"(0u)
+            : "memory");
+        accumulate = 1;
+    }
+}
+
+// Output transform of one tile: thread = TMEM lane = GEMM row; 32 channels per TMEM load.
+__device__ __forceinline__ void epilogue(const TensorParams &p, uint32_t tmem_base, int q0, int ch0, const float *sMult,
+                                         const float *sBias, const int32_t *sThr, int tid)
+{
+    const int warp = tid >> 5;
+    const int row = (warp & 3) * 32 + (tid & 31);  // a warp can only read the TMEM lanes 32*(warp%4)..+31
+    const int q = q0 + row;
+    const int rr = q / p.Wp, c = q - rr * p.Wp;
+    const int n = rr / p.Hs, oh = rr - n * p.Hs;
+    const bool row_ok = q < p.total_q && n < p.N && oh < p.H && c < p.W;
+    const int64_t pix = ((int64_t)n * p.H + oh) * p.W + c;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    // warps 0-3 take the first half of the columns, warps 4-7 the second (whole warps skip together)
+    const int half_cols = p.n_blk >= 64 ? p.n_blk / 2 : p.n_blk;
+    const int c_begin = (warp >> 2) * half_cols;
+    const int c_end = (p.n_blk >= 64 || warp < 4) ? c_begin + half_cols : c_begin;
+    for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+        int32_t v[32];
+        tmem_ld32(lane_addr + (uint32_t)c0, v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] -= p.pad_corr;
+        const int o0 = ch0 + c0;
+        if (p.out_type == LCE_OUT_BITPACKED) {
+            uint32_t bits = 0u;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) bits |= (v[j] < sThr[c0 + j] ? 1u : 0u) << j;  // sThr of pad channels = INT32_MIN
+            if (row_ok && o0 < p.Cout) static_cast<uint32_t *>(p.out)[pix * p.Cow + (o0 >> 5)] = bits;
+        } else if (p.out_type == LCE_OUT_FLOAT32) {
+            float f[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const int32_t a = (p.activation == LCE_ACT_RELU && v[j] < 0) ? 0 : v[j];
+                f[j] = __fmaf_rn((float)a, sMult[c0 + j], sBias[c0 + j]);
+            }
+            if (row_ok) {
+                float *dst = static_cast<float *>(p.out) + pix * p.Cout + o0;
+                if (p.vec_store && o0 + 32 <= p.Cout) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4 *>(dst + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (o0 + j < p.Cout) dst[j] = f[j];
+                }
+            }
+        } else if (row_ok) {
+            int32_t *dst = static_cast<int32_t *>(p.out) + pix * p.Cout + o0;
+            if (p.vec_store && o0 + 32 <= p.Cout) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) *reinterpret_cast<int4 *>(dst + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (o0 + j < p.Cout) dst[j] = v[j];
+            }
+        }
+    }
+}
+
+constexpr int kMaxWordsPerThread = 8;  // streaming schedule: packed weight words of one tap per thread
+
+template <bool RESIDENT>
+__global__ void __launch_bounds__(kThreads, 2)
 bconv3x3_tensor_kernel(const TensorParams p)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
-    // layout: [table 2 KB][barrier + tmem slot 64 B][B operand][A operand]
+    // [table 2 KB][2 barriers + tmem slot, 64 B][per-channel params 3*n_blk words][raw A 2x][B][A]
     uint2 *table = reinterpret_cast<uint2 *>(smem_raw);
-    uint64_t *mma_bar = reinterpret_cast<uint64_t *>(smem_raw + 2048);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_raw + 2048 + 16);
-    uint8_t *sB = smem_raw + 2048 + 64;                        // [9 taps][2*Cw chunks][n_blk][16]
-    uint8_t *sA = sB + (size_t)9 * 2 * p.Cw * p.n_blk * 16;    // [2*Cw chunks][P][16]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + 2048);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_raw + 2048 + 32);
+    float *sMult = reinterpret_cast<float *>(smem_raw + 2048 + 64);
+    float *sBias = sMult + p.n_blk;
+    int32_t *sThr = reinterpret_cast<int32_t *>(sBias + p.n_blk);
+    uint2 *offs = reinterpret_cast<uint2 *>(sThr + p.n_blk);          // [9*Cw] operand start offsets of a tile's MMAs
+    uint32_t *raw0 = reinterpret_cast<uint32_t *>(offs + ((9 * p.Cw + 1) / 2) * 2);
+    const int raw_words = ((p.P * p.Cw + 3) / 4) * 4;
+    uint8_t *sB = reinterpret_cast<uint8_t *>(raw0 + 2 * raw_words);
+    const size_t b_tap_bytes = (size_t)2 * p.Cw * p.n_blk * 16;  // one tap: [2*Cw chunks][n_blk][16]
+    uint8_t *sA0 = sB + (RESIDENT ? 9 : 2) * b_tap_bytes;
+    const size_t a_bytes = (size_t)2 * p.Cw * p.P * 16;          // [2*Cw chunks][P][16]
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int ch0 = blockIdx.y * p.n_blk;
 
-    // ---- one-time set-up: expansion table, barrier, TMEM, this CTA's weights --------------------
+    // ---- one-time set-up -------------------------------------------------------------------------
     for (int e = tid; e < 256; e += kThreads) {
         uint32_t lo = 0, hi = 0;
 #pragma unroll
@@ -151,8 +302,23 @@ bconv3x3_tensor_kernel(const TensorParams p)
         }
         table[e] = make_uint2(lo, hi);
     }
+    for (int e = tid; e < p.n_blk; e += kThreads) {
+        const bool ok = ch0 + e < p.Cout;
+        sMult[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.mult + ch0 + e) : 0.f;
+        sBias[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.bias + ch0 + e) : 0.f;
+        sThr[e] = (ok && p.out_type == LCE_OUT_BITPACKED) ? __ldg(p.thr + ch0 + e) : INT32_MIN;  // pad bits -> 0
+    }
+    for (int e = tid; e < 9 * p.Cw; e += kThreads) {
+        const int tap = e / p.Cw, cw = e - tap * p.Cw;
+        // A: window shift of the tap + K step (two planes of P rows); B: K step (two planes of
+        // n_blk rows), plus the tap's block when all nine taps are resident.  Units of 16 bytes.
+        const uint32_t a_off = (uint32_t)((tap / 3) * p.Wp + (tap % 3) + 2 * cw * p.P);
+        const uint32_t b_off = (uint32_t)(2 * cw * p.n_blk) + (RESIDENT ? (uint32_t)(tap * 2 * p.Cw * p.n_blk) : 0u);
+        offs[e] = make_uint2(a_off, b_off);
+    }
     if (tid == 0) {
-        mbar_init(mma_bar, 1);
+        mbar_init(&bars[0], 1);
+        mbar_init(&bars[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -165,115 +331,153 @@ bconv3x3_tensor_kernel(const TensorParams p)
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
 
-    // weights: packed [o][tap][cw] -> bytes [tap][chunk][channel in block][16]
-    for (int e = tid; e < p.n_blk * 9 * p.Cw; e += kThreads) {
-        const int cw = e % p.Cw;
-        const int ot = e / p.Cw;
-        const int tap = ot % 9, ch = ot / 9;
-        const uint32_t word = (ch0 + ch < p.Cout) ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + tap) * p.Cw + cw) : 0u;
-        uint4 lo, hi;
-        expand_word(table, word, &lo, &hi);
-        uint4 *dst = reinterpret_cast<uint4 *>(sB) + (size_t)(tap * 2 * p.Cw + 2 * cw) * p.n_blk + ch;
-        dst[0] = lo;
-        dst[p.n_blk] = hi;
-    }
-
     // instruction descriptor: D = S32, A and B signed 8-bit, both K-major, N = n_blk, M = 128
     const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_blk >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-    const uint32_t a_saddr = smem_u32(sA), b_saddr = smem_u32(sB);
-    uint32_t parity = 0;
-    bool alive = true;
+    const uint32_t b_saddr = smem_u32(sB);
+    // descriptor halves (units of 16 bytes): low = start | plane stride << 16; high = row-group
+    // stride (8 = 128 bytes) | version 1 at bit 46
+    const uint32_t desc_hi = 8u | (1u << 14);
+    const int words_per_tap = p.n_blk * p.Cw;  // packed weight words of one tap of this channel block
+    bool ok = true;
 
-    for (int tile = blockIdx.x; tile < p.n_tiles && alive; tile += gridDim.x) {
-        const int q0 = tile * kTileM;
-        // ---- expand the grid positions q0 .. q0+P-1 of the stacked padded input ----------------
-        for (int e = tid; e < p.P * p.Cw; e += kThreads) {
-            const int row = e % p.P, cw = e / p.P;
-            const int f = q0 + row;
-            const int rr = f / p.Wp, cc = f - rr * p.Wp;
-            const int n = rr / p.Hs, ry = rr - n * p.Hs;
-            uint32_t word = 0u;  // pad position: all +1
-            if (cc != 0 && ry != 0 && n < p.N)
-                word = __ldg(p.in + (((int64_t)n * p.H + (ry - 1)) * p.W + (cc - 1)) * p.Cw + cw);
-            uint4 lo, hi;
-            expand_word(table, word, &lo, &hi);
-            uint4 *dst = reinterpret_cast<uint4 *>(sA) + (size_t)(2 * cw) * p.P + row;
-            dst[0] = lo;
-            dst[p.P] = hi;
+    int tile = blockIdx.x;
+    if (tile < p.n_tiles) prefetch_raw(p, tile * kTileM, raw0, tid);
+
+    if (RESIDENT) {
+        // weights: packed [o][tap][cw] -> bytes [tap][chunk][channel][16], once
+        for (int e0 = tid; e0 < 9 * words_per_tap; e0 += kThreads * 8) {
+            uint32_t wv[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int e = e0 + k * kThreads;
+                const int ch = e & (p.n_blk - 1), tc = e >> p.n_blk_log2;  // tc = tap*Cw + cw
+                const int tap = tc / p.Cw, cw = tc - tap * p.Cw;
+                wv[k] = (e < 9 * words_per_tap && ch0 + ch < p.Cout) ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + tap) * p.Cw + cw) : 0u;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int e = e0 + k * kThreads;
+                if (e < 9 * words_per_tap) {
+                    const int ch = e & (p.n_blk - 1), tc = e >> p.n_blk_log2;
+                    const int tap = tc / p.Cw, cw = tc - tap * p.Cw;
+                    uint4 lo, hi;
+                    expand_word(table, wv[k], &lo, &hi);
+                    uint4 *dst = reinterpret_cast<uint4 *>(sB + tap * b_tap_bytes) + (size_t)(2 * cw) * p.n_blk + ch;
+                    dst[0] = lo;
+                    dst[p.n_blk] = hi;
+                }
+            }
         }
-        // make the generic-proxy writes visible to the tensor core's (async proxy) reads
+        // first tile's input into A buffer 0, the one after it on its way
+        if (tile < p.n_tiles) expand_a(p, table, raw0, sA0, tid);
+        if (tile + (int)gridDim.x < p.n_tiles) prefetch_raw(p, (tile + gridDim.x) * kTileM, raw0 + raw_words, tid);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
 
-        // ---- MMAs: 9 taps x Cw K-steps of 32 channels, one issuing thread ------------------------
-        if (tid == 0) {
+        uint32_t parity = 0;
+        for (int it = 0; tile < p.n_tiles; tile += gridDim.x, ++it) {
+            const int next = tile + gridDim.x;
+            DBG_T(0);
+            if (tid == 0) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                uint32_t accumulate = 0;
+                const uint32_t a_lo0 = (smem_u32(sA0 + (it & 1) * a_bytes) >> 4) | ((uint32_t)p.P << 16);
+                const uint32_t b_lo0 = (b_saddr >> 4) | ((uint32_t)p.n_blk << 16);
+                issue_mmas(tmem_base, offs, 0, 9 * p.Cw, a_lo0, b_lo0, desc_hi, idesc, accumulate);
+                mma_commit(&bars[0]);
+            }
+            DBG_T(1);
+            // while the tensor core works: the next tile's input into the other A buffer (the MMAs
+            // that read that buffer were awaited one iteration ago)
+            if (next < p.n_tiles) {
+                expand_a(p, table, raw0 + ((it + 1) & 1) * raw_words, sA0 + ((it + 1) & 1) * a_bytes, tid);
+                if (next + (int)gridDim.x < p.n_tiles) prefetch_raw(p, (next + gridDim.x) * kTileM, raw0 + (it & 1) * raw_words, tid);
+            }
+            DBG_T(2);
+            ok = mbar_wait_bounded(&bars[0], parity);
+            parity ^= 1u;
+            DBG_T(3);
+            // all threads agree on whether to go on (one that timed out must not strand the others)
+            if (__syncthreads_and(ok ? 1 : 0) == 0) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            DBG_T(4);
+            epilogue(p, tmem_base, tile * kTileM, ch0, sMult, sBias, sThr, tid);
+            DBG_T(5);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncthreads();
+            DBG_T(6);
+        }
+    } else {
+        uint32_t parity[2] = {0u, 0u};
+        const int wpt = (words_per_tap + kThreads - 1) / kThreads;  // <= kMaxWordsPerThread (host-checked)
+        const uint32_t a_lo0 = (smem_u32(sA0) >> 4) | ((uint32_t)p.P << 16);
+        for (int it = 0; tile < p.n_tiles && ok; tile += gridDim.x, ++it) {
+            const int next = tile + gridDim.x;
+            // every MMA of the previous tile was awaited: the A buffer is free
+            expand_a(p, table, raw0 + (it & 1) * raw_words, sA0, tid);
+            if (next < p.n_tiles) prefetch_raw(p, next * kTileM, raw0 + ((it + 1) & 1) * raw_words, tid);
+
+            uint32_t wv[kMaxWordsPerThread];
+            auto load_tap = [&](int tap) {
+#pragma unroll
+                for (int k = 0; k < kMaxWordsPerThread; ++k) {
+                    const int e = tid + k * kThreads;  // channel fastest: conflict-free shared stores
+                    const int ch = e & (p.n_blk - 1), cw = e >> p.n_blk_log2;
+                    wv[k] = (k < wpt && e < words_per_tap && ch0 + ch < p.Cout)
+                                ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + tap) * p.Cw + cw) : 0u;
+                }
+            };
+            load_tap(0);
             uint32_t accumulate = 0;
             for (int tap = 0; tap < 9; ++tap) {
-                const int shift = (tap / 3) * p.Wp + (tap % 3);
-                for (int cw = 0; cw < p.Cw; ++cw) {
-                    const uint64_t adesc = make_desc(a_saddr + (uint32_t)((2 * cw) * p.P + shift) * 16u, (uint32_t)p.P, 8u);
-                    const uint64_t bdesc =
-                        make_desc(b_saddr + (uint32_t)((tap * 2 * p.Cw + 2 * cw) * p.n_blk) * 16u, (uint32_t)p.n_blk, 8u);
-                    mma_i8(tmem_base, adesc, bdesc, idesc, accumulate);
-                    accumulate = 1;
+                const int sbuf = tap & 1;
+                if (tap >= 2) {  // the MMAs of tap-2 read this B buffer
+                    ok = mbar_wait_bounded(&bars[sbuf], parity[sbuf]) && ok;
+                    parity[sbuf] ^= 1u;
                 }
-            }
-            // arrives on the barrier when every MMA above has finished (reads of sA/sB included)
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(mma_bar))
-                         : "memory");
-        }
-        if (!mbar_wait_bounded(mma_bar, parity)) {
-            g_tensor_status = 1;
-            alive = false;
-        }
-        parity ^= 1u;
-        // all threads agree on whether to go on (a thread that timed out must not strand the others)
-        alive = __syncthreads_and(alive ? 1 : 0) != 0;
-        if (!alive) break;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-
-        // ---- output transform: thread = TMEM lane = GEMM row -----------------------------------
-        const int q = q0 + tid;
-        const int rr = q / p.Wp, c = q - rr * p.Wp;
-        const int n = rr / p.Hs, oh = rr - n * p.Hs;
-        const bool row_ok = q < p.total_q && n < p.N && oh < p.H && c < p.W;
-        const int64_t pix = ((int64_t)n * p.H + oh) * p.W + c;
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
-        for (int c0 = 0; c0 < p.n_blk; c0 += 32) {
-            uint32_t bits = 0u;
+                uint8_t *dstB = sB + sbuf * b_tap_bytes;
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const int cb = c0 + 16 * half;
-                if (cb >= p.n_blk) break;  // uniform across the CTA
-                int32_t v[16];
-                tmem_ld16(lane_addr + (uint32_t)cb, v);
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int o = ch0 + cb + j;
-                    const int32_t acc = v[j] - p.pad_corr;
-                    if (p.out_type == LCE_OUT_BITPACKED) {
-                        const bool bit = o < p.Cout && acc < __ldg(p.thr + (o < p.Cout ? o : 0));
-                        bits |= (bit ? 1u : 0u) << (16 * half + j);
-                    } else if (row_ok && o < p.Cout) {
-                        if (p.out_type == LCE_OUT_FLOAT32) {
-                            const int32_t a = (p.activation == LCE_ACT_RELU && acc < 0) ? 0 : acc;
-                            static_cast<float *>(p.out)[pix * p.Cout + o] = __fmaf_rn((float)a, __ldg(p.mult + o), __ldg(p.bias + o));
-                        } else {
-                            static_cast<int32_t *>(p.out)[pix * p.Cout + o] = acc;
-                        }
+                for (int k = 0; k < kMaxWordsPerThread; ++k) {
+                    const int e = tid + k * kThreads;
+                    if (k < wpt && e < words_per_tap) {
+                        const int ch = e & (p.n_blk - 1), cw = e >> p.n_blk_log2;
+                        uint4 lo, hi;
+                        expand_word(table, wv[k], &lo, &hi);
+                        uint4 *dst = reinterpret_cast<uint4 *>(dstB) + (size_t)(2 * cw) * p.n_blk + ch;
+                        dst[0] = lo;
+                        dst[p.n_blk] = hi;
                     }
                 }
+                if (tap + 1 < 9) load_tap(tap + 1);  // in flight while this tap's MMAs are issued
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                if (__syncthreads_and(ok ? 1 : 0) == 0) { ok = false; break; }
+                if (tid == 0) {
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    issue_mmas(tmem_base, offs, tap * p.Cw, p.Cw, a_lo0,
+                               ((b_saddr + (uint32_t)(sbuf * b_tap_bytes)) >> 4) | ((uint32_t)p.n_blk << 16), desc_hi, idesc,
+                               accumulate);
+                    mma_commit(&bars[sbuf]);
+                }
             }
-            if (p.out_type == LCE_OUT_BITPACKED && row_ok && ch0 + c0 < p.Cout)
-                static_cast<uint32_t *>(p.out)[pix * p.Cow + ((ch0 + c0) >> 5)] = bits;
+            if (!ok) break;
+            // taps 7 and 8 are still outstanding: one phase on each barrier
+            ok = mbar_wait_bounded(&bars[1], parity[1]) && ok;
+            parity[1] ^= 1u;
+            ok = mbar_wait_bounded(&bars[0], parity[0]) && ok;
+            parity[0] ^= 1u;
+            if (__syncthreads_and(ok ? 1 : 0) == 0) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            epilogue(p, tmem_base, tile * kTileM, ch0, sMult, sBias, sThr, tid);
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncthreads();
         }
-        // the next tile's MMAs overwrite the accumulators and the next expansion overwrites sA
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
     }
+    if (!ok) g_tensor_status = 1;
 
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     if (warp == 0) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
@@ -301,47 +505,77 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const uint
     p.n_tiles = (p.total_q + kTileM - 1) / kTileM;
     p.pad_corr = 9 * (32 * g.Cw - g.Cin);
     p.out_type = g.out_type; p.activation = g.activation;
+    p.vec_store = ((g.Cout & 3) == 0 && aligned(out, 16)) ? 1 : 0;
     if (p.P > 16383) return LCE_ERR_UNSUPPORTED;  // descriptor offsets are 14-bit counts of 16 bytes
 
-    // channel block: the widest of 256..32 whose expanded weights fit beside the input tile; a
-    // block is a multiple of 32 so that a bit-packed output word never spans two CTAs
-    const size_t a_bytes = (size_t)2 * g.Cw * p.P * 16;
-    const size_t budget = 226 * 1024;  // of the 227 KB a CTA may have
-    const int cout_pad = ((g.Cout + 31) / 32) * 32;
-    int n_blk = 0;
-    for (int cand = 256; cand >= 32; cand /= 2) {
-        const int blk = cand < cout_pad ? cand : cout_pad;
-        if (blk > 256) continue;
-        const size_t b_bytes = (size_t)9 * 2 * g.Cw * blk * 16;
-        if (2048 + 64 + a_bytes + b_bytes <= budget) { n_blk = blk; break; }
-    }
-    if (n_blk == 0) return LCE_ERR_UNSUPPORTED;
-    p.n_blk = n_blk;
-    int cols = 32;
-    while (cols < n_blk) cols *= 2;
-    p.tmem_cols = cols;
-    size_t smem = 2048 + 64 + a_bytes + (size_t)9 * 2 * g.Cw * n_blk * 16;
-    // no more CTAs per SM than the 512 TMEM columns can serve: pad the request if need be
-    const size_t min_smem_for_tmem = (size_t)(227 * 1024) / (512 / cols) - 1024;
-    if (smem < min_smem_for_tmem && (227 * 1024) / (smem + 1024) > (size_t)(512 / cols)) smem = min_smem_for_tmem;
-    const int n_blocks = (g.Cout + n_blk - 1) / n_blk;
+    // channel block (32..256, a power of two) and schedule.  Weights stay resident when the whole
+    // block fits beside two input buffers; otherwise one tap at a time goes through two buffers.
+    // Among the candidates the cheapest by a rough model wins: (rounds of tile iterations per SM)
+    // x (per-iteration work ~ channels x K + input rows).
     int sms = 148;
     {
         int dev = 0;
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     }
+    const size_t a_bytes = (size_t)2 * g.Cw * p.P * 16;
+    const size_t raw_bytes = (size_t)2 * (((size_t)p.P * g.Cw + 3) / 4) * 16;
+    auto fixed = [&](int blk) { return (size_t)2048 + 64 + 12 * (size_t)blk + 8 * (size_t)(((9 * g.Cw + 1) / 2) * 2) + raw_bytes; };
+    auto tap_bytes = [&](int blk) { return (size_t)2 * g.Cw * blk * 16; };
+    int cout_pow2 = 32;
+    while (cout_pow2 < g.Cout && cout_pow2 < 256) cout_pow2 *= 2;
+    int n_blk = 0;
+    bool resident = false;
+    size_t smem = 0;
+    double best_cost = 0;
+    for (int blk = cout_pow2; blk >= 32; blk /= 2) {
+        for (int res = 1; res >= 0; --res) {
+            const size_t need = res ? fixed(blk) + 9 * tap_bytes(blk) + 2 * a_bytes : fixed(blk) + 2 * tap_bytes(blk) + a_bytes;
+            if (need > 226 * 1024) continue;
+            if (!res && (blk * g.Cw + kThreads - 1) / kThreads > kMaxWordsPerThread) continue;
+            int cols = blk < 32 ? 32 : blk;
+            int per_sm = (int)((227 * 1024) / (need + 1024));
+            if (per_sm > 512 / cols) per_sm = 512 / cols;
+            if (per_sm > 4) per_sm = 4;
+            if (per_sm < 1) per_sm = 1;
+            const int64_t iters = (int64_t)p.n_tiles * ((g.Cout + blk - 1) / blk);
+            const int64_t rounds = (iters + (int64_t)sms * per_sm - 1) / ((int64_t)sms * per_sm);
+            // per iteration: MMA + epilogue ~ blk*(9*Cw + 12); input expansion ~ P*Cw; streaming adds
+            // the weight expansion ~ blk*9*Cw.  Several CTAs per SM overlap each other's phases.
+            double work = (double)blk * (9.0 * g.Cw + 12.0) + 0.5 * p.P * g.Cw + (res ? 0.0 : 1.2 * blk * 9.0 * g.Cw);
+            const double cost = (double)rounds * per_sm * work / (per_sm > 1 ? 1.5 : 1.0);
+            if (n_blk == 0 || cost < best_cost) { n_blk = blk; resident = res != 0; smem = need; best_cost = cost; }
+        }
+    }
+    if (n_blk == 0) return LCE_ERR_UNSUPPORTED;
+    p.n_blk = n_blk;
+    p.n_blk_log2 = 0;
+    while ((1 << p.n_blk_log2) < n_blk) ++p.n_blk_log2;
+    int cols = 32;
+    while (cols < n_blk) cols *= 2;
+    p.tmem_cols = cols;
+    // no more CTAs per SM than the 512 TMEM columns can serve: pad the request if need be
+    const int tmem_ctas = 512 / cols;
+    if ((227 * 1024) / (smem + 1024) > (size_t)tmem_ctas) smem = (size_t)(227 * 1024) / tmem_ctas - 1024;
+    const int n_blocks = (g.Cout + n_blk - 1) / n_blk;
     int per_sm = (int)((227 * 1024) / (smem + 1024));
     if (per_sm < 1) per_sm = 1;
-    if (per_sm > 512 / cols) per_sm = 512 / cols;
+    if (per_sm > tmem_ctas) per_sm = tmem_ctas;
     if (per_sm > 8) per_sm = 8;
     int ctas_x = (sms * per_sm) / n_blocks;
     if (ctas_x < 1) ctas_x = 1;
     if (ctas_x > p.n_tiles) ctas_x = p.n_tiles;
-    if (cudaFuncSetAttribute(bconv3x3_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return LCE_ERR_CUDA;
-    bconv3x3_tensor_kernel<<<dim3((unsigned)ctas_x, (unsigned)n_blocks), kThreads, smem, s>>>(p);
+    auto kernel = resident ? bconv3x3_tensor_kernel<true> : bconv3x3_tensor_kernel<false>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return LCE_ERR_CUDA;
+    kernel<<<dim3((unsigned)ctas_x, (unsigned)n_blocks), kThreads, smem, s>>>(p);
     return launch_status();
 }
+
+#ifdef LCE_TUNING
+extern "C" int lce_debug_read(long long *host, int n)
+{
+    return cudaMemcpyFromSymbol(host, g_dbg, sizeof(long long) * n) == cudaSuccess ? 0 : 1;
+}
+#endif
 
 // 0 = no bounded wait has expired on the current device since the library was loaded.
 lce_status tensor_device_status(int *status)

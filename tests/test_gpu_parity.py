@@ -123,6 +123,47 @@ def test_saturated_thresholds_and_pad_bits(kernel_choice):
     assert np.all(ones[..., 0] == 0xFFFFFFFF) and np.all(ones[..., 1] == 0xFF)
 
 
+# ---- tensor-core formulation (tcgen05 kind::i8): same integers, same bits ------------------------
+
+TENSOR_SHAPES = [
+    # N, H, W, Cin, Cout  (3x3, stride 1, one-padding)
+    (1, 7, 7, 64, 64), (2, 14, 14, 64, 64), (3, 9, 11, 70, 45), (1, 28, 28, 128, 128), (2, 7, 7, 512, 96),
+    (1, 56, 56, 64, 64), (2, 14, 14, 256, 256), (1, 5, 5, 32, 300), (4, 7, 7, 512, 512), (2, 9, 9, 320, 40),
+    (1, 1, 1, 3, 1), (5, 3, 40, 96, 130),
+]
+
+
+@pytest.mark.parametrize("shape", TENSOR_SHAPES)
+def test_tensor_core_kernel_matches_oracle(shape):
+    N, H, W, Cin, Cout = shape
+    rng = np.random.default_rng(abs(hash(shape)) % 2**32)
+    a, w = rand_pm1(rng, (N, H, W, Cin)), rand_pm1(rng, (Cout, 3, 3, Cin))
+    aw, ww = oracle.bitpack_pm1(a), oracle.bitpack_pm1(w)
+    acc = oracle.bconv2d_acc(a, w, (1, 1), lce.PAD_SAME_ONE)
+    kw = dict(in_c=Cin, padding=lce.PAD_SAME_ONE)
+    got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_INT32), kernel_choice=lce.KERNEL_TENSOR)
+    np.testing.assert_array_equal(got, acc)
+    thr = np.rint(np.sqrt(9 * Cin) * rng.standard_normal(Cout)).astype(np.int32)
+    got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_BITPACKED), thr=thr, kernel_choice=lce.KERNEL_TENSOR)
+    np.testing.assert_array_equal(got, oracle.transform_bits(acc, thr))
+    mult = rng.uniform(0.5, 1.5, Cout).astype(np.float32)
+    bias = (0.1 * rng.standard_normal(Cout)).astype(np.float32)
+    for act in (lce.ACT_NONE, lce.ACT_RELU):
+        got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_FLOAT32, activation=act), mult=mult, bias=bias,
+                        kernel_choice=lce.KERNEL_TENSOR)
+        assert float_close(got, acc, mult, bias, act) == 0
+    assert lce.lce_device_status() == 0  # no bounded wait gave up
+
+
+def test_tensor_core_kernel_rejects_what_it_does_not_cover():
+    desc = lce.make_desc(1, 8, 8, 64, 64, (3, 3), (2, 2), lce.PAD_SAME_ONE, lce.OUT_INT32, kernel_choice=lce.KERNEL_TENSOR)
+    z = torch.zeros(8 * 8 * 2, dtype=torch.int32, device=DEV)
+    w = torch.zeros(64 * 9 * 2, dtype=torch.int32, device=DEV)
+    with pytest.raises(lce.LceError) as e:
+        lce.lce_bconv2d(desc, z, w)
+    assert e.value.status == 2
+
+
 # ---- config 1 and batch-reduced versions of configs 2, 3 ------------------------------------
 
 def conv_case(config, first_index, spec, kernel_choice=(lce.KERNEL_AUTO, True)):

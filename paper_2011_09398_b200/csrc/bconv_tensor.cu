@@ -27,12 +27,16 @@
 //         B buffers while the previous tap's MMAs run.
 //   * tcgen05.commit signals MMA completion on mbarriers; every wait on them is bounded; on expiry
 //     the kernel records a status word, abandons its work, frees its TMEM and returns.
+#include <stdio.h>
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace lce {
 namespace {
 
-constexpr int kThreads = 256;  // 8 warps: warps w and w+4 share TMEM lanes 32*(w%4).. and split the columns
+constexpr int kWorkers = 256;  // 8 worker warps: warps w and w+4 share TMEM lanes 32*(w%4).. and split the columns
+constexpr int kThreads = kWorkers + 32;  // + one warp that only issues MMAs
 constexpr int kTileM = 128;
 constexpr uint32_t kSpinLimit = 1u << 22;  // bounded wait: about a second at worst, far above any real tile
 
@@ -88,7 +92,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
 {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (i > 64) __nanosleep(64);
+        if (i > 4096) __nanosleep(128);  // long waits back off; short ones wake up at once
     }
     return false;
 }
@@ -131,10 +135,29 @@ __device__ __forceinline__ void expand_word(const uint2 *table, uint32_t word, u
     *chunk_hi = make_uint4(c.x, c.y, d.x, d.y);
 }
 
+// The same expansion without the table, on the integer pipes only (the streaming schedule expands
+// weights while the tensor core streams both operands from shared memory, so shared-memory
+// bandwidth is the scarce resource there).  For a 4-bit value n, n * 0x00204081 puts bit i at
+// bit 8i (other partial products land between the byte boundaries and are masked away); then
+// byte = 1 + 254*bit.
+__device__ __forceinline__ uint32_t expand_nibble(uint32_t n)
+{
+    const uint32_t spread = (n * 0x00204081u) & 0x01010101u;
+    return spread * 0xFEu + 0x01010101u;
+}
+__device__ __forceinline__ void expand_word_alu(uint32_t word, uint4 *chunk_lo, uint4 *chunk_hi)
+{
+    uint32_t r[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) r[k] = expand_nibble((word >> (4 * k)) & 0xFu);
+    *chunk_lo = make_uint4(r[0], r[1], r[2], r[3]);
+    *chunk_hi = make_uint4(r[4], r[5], r[6], r[7]);
+}
+
 // packed words of the grid positions q0 .. q0+P-1 -> raw[cw*P + row] (pad positions: zero word)
 __device__ __forceinline__ void prefetch_raw(const TensorParams &p, int q0, uint32_t *raw, int tid)
 {
-    for (int row = tid; row < p.P; row += kThreads) {
+    for (int row = tid; row < p.P; row += kWorkers) {
         const int f = q0 + row;
         const int rr = f / p.Wp, cc = f - rr * p.Wp;
         const int n = rr / p.Hs, ry = rr - n * p.Hs;
@@ -150,7 +173,7 @@ __device__ __forceinline__ void prefetch_raw(const TensorParams &p, int q0, uint
 __device__ __forceinline__ void expand_a(const TensorParams &p, const uint2 *table, const uint32_t *raw, uint8_t *sA, int tid)
 {
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    for (int row = tid; row < p.P; row += kThreads) {
+    for (int row = tid; row < p.P; row += kWorkers) {
         for (int cw = 0; cw < p.Cw; ++cw) {
             uint4 lo, hi;
             expand_word(table, raw[cw * p.P + row], &lo, &hi);
@@ -267,18 +290,37 @@ __device__ __forceinline__ void epilogue(const TensorParams &p, uint32_t tmem_ba
     }
 }
 
-constexpr int kMaxWordsPerThread = 8;  // streaming schedule: packed weight words of one tap per thread
+constexpr int kMaxWordsPerThread = 8;  // streaming schedule: packed weight words of one tap per worker thread
 
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// Barrier slots in shared memory
+enum { BAR_FULL_A0 = 0, BAR_FULL_A1, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_FULL_B0, BAR_FULL_B1,
+       BAR_EMPTY_B0, BAR_EMPTY_B1, BAR_COUNT };
+
+// Warp-specialised kernel.  Warps 0-7 ("workers", 256 threads) expand operands into shared
+// memory and run the output transform; warp 8 does nothing but issue MMAs (one lane).  They
+// meet only through mbarriers, never through __syncthreads inside the tile loop:
+//   full_a[s]  workers -> issuer : input tile expanded into A buffer s            (256 arrivals)
+//   full_b[s]  workers -> issuer : one tap's weights expanded into B buffer s     (256, streaming)
+//   empty_b[s] issuer  -> workers: the MMAs that read B buffer s have finished    (tcgen05.commit)
+//   full_d[d]  issuer  -> workers: accumulator buffer d is complete               (tcgen05.commit)
+//   empty_d[d] workers -> issuer : accumulator buffer d has been read out         (256 arrivals)
+// A wait that runs out of iterations makes its thread leave the loop; the others then run out on
+// their own waits, everybody reaches the final barrier, TMEM is freed.
 template <bool RESIDENT>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 bconv3x3_tensor_kernel(const TensorParams p)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
-    // [table 2 KB][2 barriers + tmem slot, 64 B][per-channel params 3*n_blk words][raw A 2x][B][A]
+    // [table 2 KB][barriers + tmem slot, 128 B][per-channel params 3*n_blk words][MMA offsets][raw A 2x][B][A]
     uint2 *table = reinterpret_cast<uint2 *>(smem_raw);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + 2048);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_raw + 2048 + 32);
-    float *sMult = reinterpret_cast<float *>(smem_raw + 2048 + 64);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_raw + 2048 + 96);
+    float *sMult = reinterpret_cast<float *>(smem_raw + 2048 + 128);
     float *sBias = sMult + p.n_blk;
     int32_t *sThr = reinterpret_cast<int32_t *>(sBias + p.n_blk);
     uint2 *offs = reinterpret_cast<uint2 *>(sThr + p.n_blk);          // [9*Cw] operand start offsets of a tile's MMAs
@@ -290,9 +332,10 @@ bconv3x3_tensor_kernel(const TensorParams p)
     const size_t a_bytes = (size_t)2 * p.Cw * p.P * 16;          // [2*Cw chunks][P][16]
 
     const int tid = threadIdx.x, warp = tid >> 5;
+    const bool worker = tid < kWorkers;
     const int ch0 = blockIdx.y * p.n_blk;
 
-    // ---- one-time set-up -------------------------------------------------------------------------
+    // ---- one-time set-up (all threads) ---------------------------------------------------------
     for (int e = tid; e < 256; e += kThreads) {
         uint32_t lo = 0, hi = 0;
 #pragma unroll
@@ -317,8 +360,16 @@ bconv3x3_tensor_kernel(const TensorParams p)
         offs[e] = make_uint2(a_off, b_off);
     }
     if (tid == 0) {
-        mbar_init(&bars[0], 1);
-        mbar_init(&bars[1], 1);
+        mbar_init(&bars[BAR_FULL_A0], kWorkers);
+        mbar_init(&bars[BAR_FULL_A1], kWorkers);
+        mbar_init(&bars[BAR_FULL_D0], 1);
+        mbar_init(&bars[BAR_FULL_D1], 1);
+        mbar_init(&bars[BAR_EMPTY_D0], kWorkers);
+        mbar_init(&bars[BAR_EMPTY_D1], kWorkers);
+        mbar_init(&bars[BAR_FULL_B0], kWorkers);
+        mbar_init(&bars[BAR_FULL_B1], kWorkers);
+        mbar_init(&bars[BAR_EMPTY_B0], 1);
+        mbar_init(&bars[BAR_EMPTY_B1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -338,146 +389,162 @@ bconv3x3_tensor_kernel(const TensorParams p)
     // stride (8 = 128 bytes) | version 1 at bit 46
     const uint32_t desc_hi = 8u | (1u << 14);
     const int words_per_tap = p.n_blk * p.Cw;  // packed weight words of one tap of this channel block
+    const int first_tile = blockIdx.x, tile_step = gridDim.x;
     bool ok = true;
 
-    int tile = blockIdx.x;
-    if (tile < p.n_tiles) prefetch_raw(p, tile * kTileM, raw0, tid);
-
-    if (RESIDENT) {
-        // weights: packed [o][tap][cw] -> bytes [tap][chunk][channel][16], once
-        for (int e0 = tid; e0 < 9 * words_per_tap; e0 += kThreads * 8) {
-            uint32_t wv[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const int e = e0 + k * kThreads;
-                const int ch = e & (p.n_blk - 1), tc = e >> p.n_blk_log2;  // tc = tap*Cw + cw
-                const int tap = tc / p.Cw, cw = tc - tap * p.Cw;
-                wv[k] = (e < 9 * words_per_tap && ch0 + ch < p.Cout) ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + tap) * p.Cw + cw) : 0u;
-            }
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const int e = e0 + k * kThreads;
-                if (e < 9 * words_per_tap) {
-                    const int ch = e & (p.n_blk - 1), tc = e >> p.n_blk_log2;
-                    const int tap = tc / p.Cw, cw = tc - tap * p.Cw;
-                    uint4 lo, hi;
-                    expand_word(table, wv[k], &lo, &hi);
-                    uint4 *dst = reinterpret_cast<uint4 *>(sB + tap * b_tap_bytes) + (size_t)(2 * cw) * p.n_blk + ch;
-                    dst[0] = lo;
-                    dst[p.n_blk] = hi;
+    if (!worker) {
+        // ======================= MMA issuer: one lane of warp 8 ===================================
+        if (tid == kWorkers) {
+            uint32_t par_full_a[2] = {0, 0}, par_empty_d[2] = {0, 0}, par_full_b[2] = {0, 0};
+            int g = 0;  // taps issued so far (streaming: B buffer = g & 1)
+            for (int tile = first_tile, it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+                const int ab = RESIDENT ? (it & 1) : 0;  // A buffer
+                const int db = RESIDENT ? (it & 1) : 0;  // accumulator buffer
+                ok = mbar_wait_bounded(&bars[BAR_FULL_A0 + ab], par_full_a[ab]);
+                par_full_a[ab] ^= 1u;
+                if (ok && it >= (RESIDENT ? 2 : 1)) {  // the accumulator buffer must have been read out
+                    ok = mbar_wait_bounded(&bars[BAR_EMPTY_D0 + db], par_empty_d[db]);
+                    par_empty_d[db] ^= 1u;
                 }
-            }
-        }
-        // first tile's input into A buffer 0, the one after it on its way
-        if (tile < p.n_tiles) expand_a(p, table, raw0, sA0, tid);
-        if (tile + (int)gridDim.x < p.n_tiles) prefetch_raw(p, (tile + gridDim.x) * kTileM, raw0 + raw_words, tid);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
-
-        uint32_t parity = 0;
-        for (int it = 0; tile < p.n_tiles; tile += gridDim.x, ++it) {
-            const int next = tile + gridDim.x;
-            DBG_T(0);
-            if (tid == 0) {
+                if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tmem_d = tmem_base + (uint32_t)(db * p.n_blk);
+                const uint32_t a_lo0 = (smem_u32(sA0 + ab * a_bytes) >> 4) | ((uint32_t)p.P << 16);
                 uint32_t accumulate = 0;
-                const uint32_t a_lo0 = (smem_u32(sA0 + (it & 1) * a_bytes) >> 4) | ((uint32_t)p.P << 16);
-                const uint32_t b_lo0 = (b_saddr >> 4) | ((uint32_t)p.n_blk << 16);
-                issue_mmas(tmem_base, offs, 0, 9 * p.Cw, a_lo0, b_lo0, desc_hi, idesc, accumulate);
-                mma_commit(&bars[0]);
+                if (RESIDENT) {
+                    issue_mmas(tmem_d, offs, 0, 9 * p.Cw, a_lo0, (b_saddr >> 4) | ((uint32_t)p.n_blk << 16), desc_hi, idesc, accumulate);
+                } else {
+                    for (int tap = 0; tap < 9 && ok; ++tap, ++g) {
+                        const int sb = g & 1;
+                        ok = mbar_wait_bounded(&bars[BAR_FULL_B0 + sb], par_full_b[sb]);
+                        par_full_b[sb] ^= 1u;
+                        if (!ok) break;
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        issue_mmas(tmem_d, offs, tap * p.Cw, p.Cw, a_lo0,
+                                   ((b_saddr + (uint32_t)(sb * b_tap_bytes)) >> 4) | ((uint32_t)p.n_blk << 16), desc_hi, idesc, accumulate);
+                        mma_commit(&bars[BAR_EMPTY_B0 + sb]);
+                    }
+                    if (!ok) break;
+                }
+                mma_commit(&bars[BAR_FULL_D0 + db]);
             }
-            DBG_T(1);
-            // while the tensor core works: the next tile's input into the other A buffer (the MMAs
-            // that read that buffer were awaited one iteration ago)
-            if (next < p.n_tiles) {
-                expand_a(p, table, raw0 + ((it + 1) & 1) * raw_words, sA0 + ((it + 1) & 1) * a_bytes, tid);
-                if (next + (int)gridDim.x < p.n_tiles) prefetch_raw(p, (next + gridDim.x) * kTileM, raw0 + (it & 1) * raw_words, tid);
-            }
-            DBG_T(2);
-            ok = mbar_wait_bounded(&bars[0], parity);
-            parity ^= 1u;
-            DBG_T(3);
-            // all threads agree on whether to go on (one that timed out must not strand the others)
-            if (__syncthreads_and(ok ? 1 : 0) == 0) { ok = false; break; }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            DBG_T(4);
-            epilogue(p, tmem_base, tile * kTileM, ch0, sMult, sBias, sThr, tid);
-            DBG_T(5);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncthreads();
-            DBG_T(6);
         }
     } else {
-        uint32_t parity[2] = {0u, 0u};
-        const int wpt = (words_per_tap + kThreads - 1) / kThreads;  // <= kMaxWordsPerThread (host-checked)
-        const uint32_t a_lo0 = (smem_u32(sA0) >> 4) | ((uint32_t)p.P << 16);
-        for (int it = 0; tile < p.n_tiles && ok; tile += gridDim.x, ++it) {
-            const int next = tile + gridDim.x;
-            // every MMA of the previous tile was awaited: the A buffer is free
-            expand_a(p, table, raw0 + (it & 1) * raw_words, sA0, tid);
-            if (next < p.n_tiles) prefetch_raw(p, next * kTileM, raw0 + ((it + 1) & 1) * raw_words, tid);
+        // ======================= workers: expansion and output transform ==========================
+        uint32_t par_full_d[2] = {0, 0}, par_empty_b[2] = {0, 0};
+        int tile = first_tile;
+        if (tile < p.n_tiles) prefetch_raw(p, tile * kTileM, raw0, tid);
 
-            uint32_t wv[kMaxWordsPerThread];
-            auto load_tap = [&](int tap) {
+        if (RESIDENT) {
+            // weights: packed [o][tap][cw] -> bytes [tap][chunk][channel][16], once
+            for (int e0 = tid; e0 < 9 * words_per_tap; e0 += kWorkers * 8) {
+                uint32_t wv[8];
 #pragma unroll
-                for (int k = 0; k < kMaxWordsPerThread; ++k) {
-                    const int e = tid + k * kThreads;  // channel fastest: conflict-free shared stores
-                    const int ch = e & (p.n_blk - 1), cw = e >> p.n_blk_log2;
-                    wv[k] = (k < wpt && e < words_per_tap && ch0 + ch < p.Cout)
-                                ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + tap) * p.Cw + cw) : 0u;
+                for (int k = 0; k < 8; ++k) {
+                    const int e = e0 + k * kWorkers;
+                    const int ch = e & (p.n_blk - 1), tc = e >> p.n_blk_log2;  // tc = tap*Cw + cw
+                    const int tap = tc / p.Cw, cw = tc - tap * p.Cw;
+                    wv[k] = (e < 9 * words_per_tap && ch0 + ch < p.Cout) ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + tap) * p.Cw + cw) : 0u;
                 }
-            };
-            load_tap(0);
-            uint32_t accumulate = 0;
-            for (int tap = 0; tap < 9; ++tap) {
-                const int sbuf = tap & 1;
-                if (tap >= 2) {  // the MMAs of tap-2 read this B buffer
-                    ok = mbar_wait_bounded(&bars[sbuf], parity[sbuf]) && ok;
-                    parity[sbuf] ^= 1u;
-                }
-                uint8_t *dstB = sB + sbuf * b_tap_bytes;
 #pragma unroll
-                for (int k = 0; k < kMaxWordsPerThread; ++k) {
-                    const int e = tid + k * kThreads;
-                    if (k < wpt && e < words_per_tap) {
-                        const int ch = e & (p.n_blk - 1), cw = e >> p.n_blk_log2;
+                for (int k = 0; k < 8; ++k) {
+                    const int e = e0 + k * kWorkers;
+                    if (e < 9 * words_per_tap) {
+                        const int ch = e & (p.n_blk - 1), tc = e >> p.n_blk_log2;
+                        const int tap = tc / p.Cw, cw = tc - tap * p.Cw;
                         uint4 lo, hi;
                         expand_word(table, wv[k], &lo, &hi);
-                        uint4 *dst = reinterpret_cast<uint4 *>(dstB) + (size_t)(2 * cw) * p.n_blk + ch;
+                        uint4 *dst = reinterpret_cast<uint4 *>(sB + tap * b_tap_bytes) + (size_t)(2 * cw) * p.n_blk + ch;
                         dst[0] = lo;
                         dst[p.n_blk] = hi;
                     }
                 }
-                if (tap + 1 < 9) load_tap(tap + 1);  // in flight while this tap's MMAs are issued
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                if (__syncthreads_and(ok ? 1 : 0) == 0) { ok = false; break; }
-                if (tid == 0) {
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    issue_mmas(tmem_base, offs, tap * p.Cw, p.Cw, a_lo0,
-                               ((b_saddr + (uint32_t)(sbuf * b_tap_bytes)) >> 4) | ((uint32_t)p.n_blk << 16), desc_hi, idesc,
-                               accumulate);
-                    mma_commit(&bars[sbuf]);
-                }
             }
-            if (!ok) break;
-            // taps 7 and 8 are still outstanding: one phase on each barrier
-            ok = mbar_wait_bounded(&bars[1], parity[1]) && ok;
-            parity[1] ^= 1u;
-            ok = mbar_wait_bounded(&bars[0], parity[0]) && ok;
-            parity[0] ^= 1u;
-            if (__syncthreads_and(ok ? 1 : 0) == 0) { ok = false; break; }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            epilogue(p, tmem_base, tile * kTileM, ch0, sMult, sBias, sThr, tid);
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncthreads();
+            if (tile < p.n_tiles) {
+                expand_a(p, table, raw0, sA0, tid);
+                if (tile + tile_step < p.n_tiles) prefetch_raw(p, (tile + tile_step) * kTileM, raw0 + raw_words, tid);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(&bars[BAR_FULL_A0]);
+            }
+            for (int it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+                const int next = tile + tile_step;
+                const int cur = it & 1, nxt = cur ^ 1;
+                if (next < p.n_tiles) {
+                    // A buffer nxt was last read by the MMAs of tile it-1, whose completion (full_d)
+                    // this thread waited for in the previous iteration
+                    expand_a(p, table, raw0 + nxt * raw_words, sA0 + nxt * a_bytes, tid);
+                    if (next + tile_step < p.n_tiles) prefetch_raw(p, (next + tile_step) * kTileM, raw0 + cur * raw_words, tid);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    mbar_arrive(&bars[BAR_FULL_A0 + nxt]);
+                }
+                ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + cur], par_full_d[cur]);
+                par_full_d[cur] ^= 1u;
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                epilogue(p, tmem_base + (uint32_t)(cur * p.n_blk), tile * kTileM, ch0, sMult, sBias, sThr, tid);
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                mbar_arrive(&bars[BAR_EMPTY_D0 + cur]);
+            }
+        } else {
+            const int wpt = (words_per_tap + kWorkers - 1) / kWorkers;  // <= kMaxWordsPerThread (host-checked)
+            int g = 0;  // taps produced so far
+            for (int it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+                const int next = tile + tile_step;
+                // the single A buffer was last read by the previous tile's MMAs: full_d awaited below
+                expand_a(p, table, raw0 + (it & 1) * raw_words, sA0, tid);
+                if (next < p.n_tiles) prefetch_raw(p, next * kTileM, raw0 + ((it + 1) & 1) * raw_words, tid);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(&bars[BAR_FULL_A0]);
+
+                uint32_t wv[kMaxWordsPerThread];
+                auto load_tap = [&](int tap) {
+#pragma unroll
+                    for (int k = 0; k < kMaxWordsPerThread; ++k) {
+                        const int e = tid + k * kWorkers;  // channel fastest: conflict-free shared stores
+                        const int ch = e & (p.n_blk - 1), cw = e >> p.n_blk_log2;
+                        wv[k] = (k < wpt && e < words_per_tap && ch0 + ch < p.Cout)
+                                    ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + tap) * p.Cw + cw) : 0u;
+                    }
+                };
+                load_tap(0);
+                for (int tap = 0; tap < 9 && ok; ++tap, ++g) {
+                    const int sb = g & 1;
+                    if (g >= 2) {  // the MMAs of two taps ago read this B buffer
+                        ok = mbar_wait_bounded(&bars[BAR_EMPTY_B0 + sb], par_empty_b[sb]);
+                        par_empty_b[sb] ^= 1u;
+                        if (!ok) break;
+                    }
+                    uint8_t *dstB = sB + sb * b_tap_bytes;
+#pragma unroll
+                    for (int k = 0; k < kMaxWordsPerThread; ++k) {
+                        const int e = tid + k * kWorkers;
+                        if (k < wpt && e < words_per_tap) {
+                            const int ch = e & (p.n_blk - 1), cw = e >> p.n_blk_log2;
+                            uint4 lo, hi;
+                            expand_word_alu(wv[k], &lo, &hi);
+                            uint4 *dst = reinterpret_cast<uint4 *>(dstB) + (size_t)(2 * cw) * p.n_blk + ch;
+                            dst[0] = lo;
+                            dst[p.n_blk] = hi;
+                        }
+                    }
+                    if (tap + 1 < 9) load_tap(tap + 1);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    mbar_arrive(&bars[BAR_FULL_B0 + sb]);
+                }
+                if (!ok) break;
+                ok = mbar_wait_bounded(&bars[BAR_FULL_D0], par_full_d[0]);
+                par_full_d[0] ^= 1u;
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                epilogue(p, tmem_base, tile * kTileM, ch0, sMult, sBias, sThr, tid);
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                mbar_arrive(&bars[BAR_EMPTY_D0]);
+            }
         }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     if (!ok) g_tensor_status = 1;
 
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     if (warp == 0) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
@@ -508,10 +575,10 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const uint
     p.vec_store = ((g.Cout & 3) == 0 && aligned(out, 16)) ? 1 : 0;
     if (p.P > 16383) return LCE_ERR_UNSUPPORTED;  // descriptor offsets are 14-bit counts of 16 bytes
 
-    // channel block (32..256, a power of two) and schedule.  Weights stay resident when the whole
-    // block fits beside two input buffers; otherwise one tap at a time goes through two buffers.
-    // Among the candidates the cheapest by a rough model wins: (rounds of tile iterations per SM)
-    // x (per-iteration work ~ channels x K + input rows).
+    // Channel block (32..256, a power of two) and schedule, by a rule that matches what was
+    // measured on the ResNet-18 shapes: weights resident if the full channel width (up to 256)
+    // fits beside two input buffers; otherwise stream one tap at a time with the widest block
+    // that fits (wide MMAs amortise the A-operand traffic); a narrower resident block last.
     int sms = 148;
     {
         int dev = 0;
@@ -519,58 +586,72 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const uint
     }
     const size_t a_bytes = (size_t)2 * g.Cw * p.P * 16;
     const size_t raw_bytes = (size_t)2 * (((size_t)p.P * g.Cw + 3) / 4) * 16;
-    auto fixed = [&](int blk) { return (size_t)2048 + 64 + 12 * (size_t)blk + 8 * (size_t)(((9 * g.Cw + 1) / 2) * 2) + raw_bytes; };
+    auto fixed = [&](int blk) { return (size_t)2048 + 128 + 12 * (size_t)blk + 8 * (size_t)(((9 * g.Cw + 1) / 2) * 2) + raw_bytes; };
     auto tap_bytes = [&](int blk) { return (size_t)2 * g.Cw * blk * 16; };
+    auto need_bytes = [&](int blk, bool res) {
+        return res ? fixed(blk) + 9 * tap_bytes(blk) + 2 * a_bytes : fixed(blk) + 2 * tap_bytes(blk) + a_bytes;
+    };
+    auto feasible = [&](int blk, bool res) {
+        if (need_bytes(blk, res) > 226 * 1024) return false;
+        return res || (blk * g.Cw + kWorkers - 1) / kWorkers <= kMaxWordsPerThread;
+    };
     int cout_pow2 = 32;
     while (cout_pow2 < g.Cout && cout_pow2 < 256) cout_pow2 *= 2;
     int n_blk = 0;
     bool resident = false;
-    size_t smem = 0;
-    double best_cost = 0;
-    for (int blk = cout_pow2; blk >= 32; blk /= 2) {
-        for (int res = 1; res >= 0; --res) {
-            const size_t need = res ? fixed(blk) + 9 * tap_bytes(blk) + 2 * a_bytes : fixed(blk) + 2 * tap_bytes(blk) + a_bytes;
-            if (need > 226 * 1024) continue;
-            if (!res && (blk * g.Cw + kThreads - 1) / kThreads > kMaxWordsPerThread) continue;
-            int cols = blk < 32 ? 32 : blk;
-            int per_sm = (int)((227 * 1024) / (need + 1024));
-            if (per_sm > 512 / cols) per_sm = 512 / cols;
-            if (per_sm > 4) per_sm = 4;
-            if (per_sm < 1) per_sm = 1;
-            const int64_t iters = (int64_t)p.n_tiles * ((g.Cout + blk - 1) / blk);
-            const int64_t rounds = (iters + (int64_t)sms * per_sm - 1) / ((int64_t)sms * per_sm);
-            // per iteration: MMA + epilogue ~ blk*(9*Cw + 12); input expansion ~ P*Cw; streaming adds
-            // the weight expansion ~ blk*9*Cw.  Several CTAs per SM overlap each other's phases.
-            double work = (double)blk * (9.0 * g.Cw + 12.0) + 0.5 * p.P * g.Cw + (res ? 0.0 : 1.2 * blk * 9.0 * g.Cw);
-            const double cost = (double)rounds * per_sm * work / (per_sm > 1 ? 1.5 : 1.0);
-            if (n_blk == 0 || cost < best_cost) { n_blk = blk; resident = res != 0; smem = need; best_cost = cost; }
-        }
+    int force_blk = 0, force_res = -1;
+#ifdef LCE_TUNING
+    if (const char *e = getenv("LCE_TENSOR_BLK")) force_blk = atoi(e);
+    if (const char *e = getenv("LCE_TENSOR_RES")) force_res = atoi(e);
+#endif
+    if (force_blk) {
+        if (feasible(force_blk, force_res != 0)) { n_blk = force_blk; resident = force_res != 0; }
+    } else if (feasible(cout_pow2, true)) {
+        n_blk = cout_pow2; resident = true;
+    } else {
+        for (int blk = cout_pow2; blk >= 32 && n_blk == 0; blk /= 2)
+            if (feasible(blk, false)) { n_blk = blk; resident = false; }
+        for (int blk = cout_pow2 / 2; blk >= 32 && n_blk == 0; blk /= 2)
+            if (feasible(blk, true)) { n_blk = blk; resident = true; }
     }
     if (n_blk == 0) return LCE_ERR_UNSUPPORTED;
+    size_t smem = need_bytes(n_blk, resident);
     p.n_blk = n_blk;
     p.n_blk_log2 = 0;
     while ((1 << p.n_blk_log2) < n_blk) ++p.n_blk_log2;
     int cols = 32;
-    while (cols < n_blk) cols *= 2;
+    while (cols < (resident ? 2 * n_blk : n_blk)) cols *= 2;
     p.tmem_cols = cols;
     // no more CTAs per SM than the 512 TMEM columns can serve: pad the request if need be
     const int tmem_ctas = 512 / cols;
     if ((227 * 1024) / (smem + 1024) > (size_t)tmem_ctas) smem = (size_t)(227 * 1024) / tmem_ctas - 1024;
     const int n_blocks = (g.Cout + n_blk - 1) / n_blk;
-    int per_sm = (int)((227 * 1024) / (smem + 1024));
-    if (per_sm < 1) per_sm = 1;
+    auto kernel = resident ? bconv3x3_tensor_kernel<true> : bconv3x3_tensor_kernel<false>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return LCE_ERR_CUDA;
+    // ask for the largest shared-memory carve-out, or a second CTA per SM may not be allowed
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+        return LCE_ERR_CUDA;
+    // persistent grid: exactly as many CTAs as can be resident at once (registers, shared memory
+    // and TMEM columns all count)
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, smem) != cudaSuccess) return LCE_ERR_CUDA;
+    if (per_sm < 1) return LCE_ERR_UNSUPPORTED;
     if (per_sm > tmem_ctas) per_sm = tmem_ctas;
-    if (per_sm > 8) per_sm = 8;
     int ctas_x = (sms * per_sm) / n_blocks;
     if (ctas_x < 1) ctas_x = 1;
     if (ctas_x > p.n_tiles) ctas_x = p.n_tiles;
-    auto kernel = resident ? bconv3x3_tensor_kernel<true> : bconv3x3_tensor_kernel<false>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return LCE_ERR_CUDA;
+#ifdef LCE_TUNING
+    if (getenv("LCE_VERBOSE")) fprintf(stderr, "tensor: resident=%d n_blk=%d smem=%zu occ=%d ctas_x=%d n_blocks=%d tiles=%d\n", (int)resident, n_blk, smem, per_sm, ctas_x, n_blocks, p.n_tiles);
+#endif
     kernel<<<dim3((unsigned)ctas_x, (unsigned)n_blocks), kThreads, smem, s>>>(p);
     return launch_status();
 }
 
 #ifdef LCE_TUNING
+extern "C" int lce_debug_write(const long long *host, int n)
+{
+    return cudaMemcpyToSymbol(g_dbg, host, sizeof(long long) * n) == cudaSuccess ? 0 : 1;
+}
 extern "C" int lce_debug_read(long long *host, int n)
 {
     return cudaMemcpyFromSymbol(host, g_dbg, sizeof(long long) * n) == cudaSuccess ? 0 : 1;

@@ -37,7 +37,8 @@ constexpr int kChanPerThread = 8;
 constexpr int kChanGroups = kChanPerCta / kChanPerThread;
 constexpr int kWRow = 12;           // 9 carry-save operand words per (channel word, channel) + 3 pad
 constexpr int kWGroupStride = kChanPerThread * kWRow + 4;  // +4 words: the 8 channel groups hit distinct banks
-constexpr int kWsumWords = kChanPerCta * 9;                // per-tap weight sums of a channel block
+constexpr int kMaxTaps = 25;                               // 5x5 is the largest tiled filter
+constexpr int kWsumWords = kChanPerCta * kMaxTaps;         // per-tap weight sums of a channel block
 
 struct TiledParams {
     const uint32_t *in;
@@ -64,11 +65,13 @@ __host__ __device__ __forceinline__ int32_t w_offset(int cw, int ch)
 {
     return cw * kChanGroups * kWGroupStride + (ch >> 3) * kWGroupStride + (ch & 7) * kWRow;
 }
-// One channel block of the packed image: operands for every channel word, then the per-tap sums.
-__host__ __device__ __forceinline__ int64_t image_block_words(int Cw)
+// One channel block of the packed image: operands of every nine-word group, then the per-tap sums.
+__host__ __device__ __forceinline__ int64_t image_block_words(int groups)
 {
-    return (int64_t)Cw * kChanGroups * kWGroupStride + kWsumWords;
+    return (int64_t)groups * kChanGroups * kWGroupStride + kWsumWords;
 }
+// nine-word groups per channel word of a KSxKS filter: taps beyond KS*KS count as zero words
+__host__ __device__ constexpr int groups_per_word(int ks) { return (ks * ks + 8) / 9; }
 
 template <int BYTE_OFF>
 __device__ __forceinline__ uint4 lds128(uint32_t saddr)
@@ -143,32 +146,34 @@ __device__ __forceinline__ void store_w_operands(const uint32_t (&wv)[9], uint32
 // shared-memory image the convolution kernel wants (operands, then per-tap sums).
 __global__ void __launch_bounds__(128)
 pack_weights_kernel(const uint32_t *__restrict__ w, uint32_t *__restrict__ image, int32_t Cout, int32_t Cw,
-                    int32_t Cin, int32_t chan_blocks)
+                    int32_t Cin, int32_t chan_blocks, int32_t ks)
 {
-    // 3x3: group = channel word, the nine words of a group are the nine taps
-    const int64_t entries = (int64_t)chan_blocks * kChanPerCta * Cw;
+    // group = (channel word, run of nine taps); taps past ks*ks are zero words
+    const int taps = ks * ks, ng = groups_per_word(ks);
+    const int64_t entries = (int64_t)chan_blocks * kChanPerCta * Cw * ng;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < entries;
          e += (int64_t)gridDim.x * blockDim.x) {
-        const int cw = (int)(e % Cw);
-        const int64_t c = e / Cw;  // global channel (may be >= Cout in the last block)
+        const int g = (int)(e % ng);
+        const int cw = (int)((e / ng) % Cw);
+        const int64_t c = e / ((int64_t)ng * Cw);  // global channel (may be >= Cout in the last block)
         const int cb = (int)(c / kChanPerCta), ch = (int)(c % kChanPerCta);
         uint32_t wv[9];
 #pragma unroll
-        for (int t = 0; t < 9; ++t) wv[t] = c < Cout ? w[(c * 9 + t) * Cw + cw] : 0u;
-        uint32_t *block = image + cb * image_block_words(Cw);
-        store_w_operands(wv, block + w_offset(cw, ch));
+        for (int t = 0; t < 9; ++t) wv[t] = (c < Cout && 9 * g + t < taps) ? w[(c * taps + 9 * g + t) * Cw + cw] : 0u;
+        uint32_t *block = image + cb * image_block_words(Cw * ng);
+        store_w_operands(wv, block + w_offset(cw * ng + g, ch));
         if ((ch & 7) == 7) {  // the 4 pad words after every 8 channels
-            uint32_t *pad = block + w_offset(cw, ch) + kWRow;
+            uint32_t *pad = block + w_offset(cw * ng + g, ch) + kWRow;
             pad[0] = pad[1] = pad[2] = pad[3] = 0u;
         }
-        if (cw == 0) {
+        if (cw == 0 && g == 0) {
             // sum over the true channels of one tap's weights = Cin - 2*popcount (pad bits are 0)
-            int32_t *wsum = reinterpret_cast<int32_t *>(block + (int64_t)Cw * kChanGroups * kWGroupStride);
-            for (int t = 0; t < 9; ++t) {
+            int32_t *wsum = reinterpret_cast<int32_t *>(block + (int64_t)Cw * ng * kChanGroups * kWGroupStride);
+            for (int t = 0; t < kMaxTaps; ++t) {
                 int32_t cnt = 0;
-                if (c < Cout)
-                    for (int j = 0; j < Cw; ++j) cnt += __popc(w[(c * 9 + t) * Cw + j]);
-                wsum[ch * 9 + t] = c < Cout ? Cin - 2 * cnt : 0;
+                if (c < Cout && t < taps)
+                    for (int j = 0; j < Cw; ++j) cnt += __popc(w[(c * taps + t) * Cw + j]);
+                wsum[ch * kMaxTaps + t] = (c < Cout && t < taps) ? Cin - 2 * cnt : 0;
             }
         }
     }
@@ -292,12 +297,12 @@ __device__ __forceinline__ int tile_first_vrow(const TiledParams &p, int m0)
 // Copies the input rows a tile needs into shared memory: global [n][iy][ix][cw] -> [cw][v][x] in
 // padded-image coordinates.  Image words travel as asynchronous copies (the caller waits for
 // them); rows and columns outside the image are written as zero words (one-padding).
-template <int STRIDE>
+template <int KS, int STRIDE>
 __device__ __forceinline__ void stage_rows(const TiledParams &p, int m0, int m_end, uint32_t *sA, int warp, int lane)
 {
     const int r_last = (m_end - 1) / p.OW;
     const int v_first = tile_first_vrow<STRIDE>(p, m0);
-    const int v_last = (r_last / p.OH) * p.Hp + (r_last % p.OH) * STRIDE + 2;
+    const int v_last = (r_last / p.OH) * p.Hp + (r_last % p.OH) * STRIDE + (KS - 1);
     const int nv = v_last - v_first + 1;
     const int row_words = p.W * p.Cw;
     for (int v = warp; v < nv; v += kWarps) {
@@ -327,13 +332,15 @@ __device__ __forceinline__ void stage_rows(const TiledParams &p, int m0, int m_e
     }
 }
 
-template <int STRIDE, int TP>
+template <int KS, int STRIDE, int TP>
 __global__ void __launch_bounds__(kThreads, (TP <= 2 ? 24 : 16) / kWarps)
 bconv3x3_kernel(const TiledParams p)
 {
+    constexpr int kTaps = KS * KS;             // 9 or 25
+    constexpr int kNG = groups_per_word(KS);   // nine-word groups per channel word: 1 or 3
     extern __shared__ __align__(16) uint32_t smem[];
-    const int w_words = p.Cw * kChanGroups * kWGroupStride;
-    uint32_t *sW = smem;                                           // [Cw][8 groups][kWGroupStride]
+    const int w_words = p.Cw * kNG * kChanGroups * kWGroupStride;
+    uint32_t *sW = smem;                                           // [Cw*kNG][8 groups][kWGroupStride]
     int32_t *sWsum = reinterpret_cast<int32_t *>(smem + w_words);  // [64][9]
     uint32_t *sA0 = smem + w_words + kWsumWords;                   // 2 x [Cw][nv][pitch]
 
@@ -346,27 +353,29 @@ bconv3x3_kernel(const TiledParams p)
     if (p.w_image != nullptr) {
         // prepared image: a plain 16-byte asynchronous copy of this channel block
         const int words = (p.padding == LCE_PAD_SAME_ZERO) ? w_words + kWsumWords : w_words;
-        const uint32_t *src = p.w_image + blockIdx.y * image_block_words(p.Cw);
+        const uint32_t *src = p.w_image + blockIdx.y * image_block_words(p.Cw * kNG);
         for (int e = tid * 4; e < words; e += kThreads * 4) cp_async16(smem + e, src + e);
         asm volatile("cp.async.commit_group;" ::: "memory");
     } else {
-        for (int e = tid; e < kChanPerCta * p.Cw; e += kThreads) {
-            const int ch = e / p.Cw;
-            const int cw = e - ch * p.Cw;
+        for (int e = tid; e < kChanPerCta * p.Cw * kNG; e += kThreads) {
+            const int g = e % kNG;
+            const int cw = (e / kNG) % p.Cw;
+            const int ch = e / (kNG * p.Cw);
             uint32_t wv[9];
 #pragma unroll
             for (int t = 0; t < 9; ++t)
-                wv[t] = (ch0 + ch < p.Cout) ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + t) * p.Cw + cw) : 0u;
-            store_w_operands(wv, sW + w_offset(cw, ch));
+                wv[t] = (ch0 + ch < p.Cout && 9 * g + t < kTaps)
+                            ? __ldg(p.w + ((int64_t)(ch0 + ch) * kTaps + 9 * g + t) * p.Cw + cw) : 0u;
+            store_w_operands(wv, sW + w_offset(cw * kNG + g, ch));
         }
         if (p.padding == LCE_PAD_SAME_ZERO) {
-            for (int e = tid; e < kWsumWords; e += kThreads) {
-                const int ch = e / 9, t = e - ch * 9;
+            for (int e = tid; e < kChanPerCta * kTaps; e += kThreads) {
+                const int ch = e / kTaps, t = e - ch * kTaps;
                 int32_t cnt = 0;
                 if (ch0 + ch < p.Cout)
                     for (int cw = 0; cw < p.Cw; ++cw)
-                        cnt += __popc(__ldg(p.w + ((int64_t)(ch0 + ch) * 9 + t) * p.Cw + cw));
-                sWsum[e] = p.Cin - 2 * cnt;
+                        cnt += __popc(__ldg(p.w + ((int64_t)(ch0 + ch) * kTaps + t) * p.Cw + cw));
+                sWsum[ch * kMaxTaps + t] = p.Cin - 2 * cnt;
             }
         }
     }
@@ -374,7 +383,7 @@ bconv3x3_kernel(const TiledParams p)
     // ---- this thread's channels --------------------------------------------------------------
     const int px = lane >> 3, cg = lane & 7;
     const int chan = ch0 + cg * kChanPerThread;
-    const int K = 9 * p.Cin;
+    const int K = kTaps * p.Cin;
     Weights124 k124;
     k124.one = p.N > 0 ? 1u : p.Cin;  // opaque to the compiler: keeps the weighted sum on multiply-adds
     k124.two = p.N > 0 ? 2u : p.Cin;
@@ -386,7 +395,7 @@ bconv3x3_kernel(const TiledParams p)
     // the other buffer while the current tile is computed --------------------------------------
     int tile = blockIdx.x;
     if (tile < p.n_tiles)
-        stage_rows<STRIDE>(p, tile * p.tile_pixels, min((tile + 1) * p.tile_pixels, p.M), sA0, warp, lane);
+        stage_rows<KS, STRIDE>(p, tile * p.tile_pixels, min((tile + 1) * p.tile_pixels, p.M), sA0, warp, lane);
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
@@ -398,7 +407,7 @@ bconv3x3_kernel(const TiledParams p)
     {
         const int next = tile + gridDim.x;
         if (next < p.n_tiles)
-            stage_rows<STRIDE>(p, next * p.tile_pixels, min((next + 1) * p.tile_pixels, p.M),
+            stage_rows<KS, STRIDE>(p, next * p.tile_pixels, min((next + 1) * p.tile_pixels, p.M),
                                sA0 + (buf ^ 1) * plane_words, warp, lane);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
@@ -428,7 +437,7 @@ bconv3x3_kernel(const TiledParams p)
             ow += kPixPerStep;
             while (ow >= p.OW) {
                 ow -= p.OW;
-                if (oh_left == 0) { oh_left = p.OH - 1; voh += 3; }  // next image: Hp - (OH-1)*STRIDE = 3
+                if (oh_left == 0) { oh_left = p.OH - 1; voh += KS; }  // next image: Hp - (OH-1)*STRIDE = KS
                 else { --oh_left; voh += STRIDE; }
             }
         }
@@ -441,16 +450,26 @@ bconv3x3_kernel(const TiledParams p)
         uint32_t w_saddr = w_saddr0;
         const uint32_t *plane = sA;
         for (int cw = 0; cw < p.Cw; ++cw) {
-            Triple at[TP][3];
 #pragma unroll
-            for (int i = 0; i < TP; ++i)
+            for (int g = 0; g < kNG; ++g) {
+                // activation-side operands of nine-word group g: taps 9g .. 9g+8 in (ky, kx) order;
+                // taps past the filter's last one are zero words on both sides and count nothing
+                Triple at[TP][3];
 #pragma unroll
-                for (int ky = 0; ky < 3; ++ky) {
-                    const uint32_t *row = plane + a_base[i] + ky * p.pitch;
-                    at[i][ky] = make_triple(row[0], row[1], row[2]);
-                }
-            ChannelLoop<0, TP>::run(w_saddr, at, k124, acc);
-            w_saddr += kChanGroups * kWGroupStride * 4;
+                for (int i = 0; i < TP; ++i)
+#pragma unroll
+                    for (int k = 0; k < 3; ++k) {
+                        uint32_t v[3];
+#pragma unroll
+                        for (int j = 0; j < 3; ++j) {
+                            const int t = 9 * g + 3 * k + j;  // compile-time after unrolling
+                            v[j] = t < kTaps ? plane[a_base[i] + (t / KS) * p.pitch + (t % KS)] : 0u;
+                        }
+                        at[i][k] = make_triple(v[0], v[1], v[2]);
+                    }
+                ChannelLoop<0, TP>::run(w_saddr, at, k124, acc);
+                w_saddr += kChanGroups * kWGroupStride * 4;
+            }
             plane += p.plane;
         }
 
@@ -470,11 +489,11 @@ bconv3x3_kernel(const TiledParams p)
                 const int r = mm / p.OW;
                 const int iy0 = (r % p.OH) * STRIDE - p.pt, ix0 = (mm - r * p.OW) * STRIDE - p.pl;
 #pragma unroll
-                for (int t = 0; t < 9; ++t) {
-                    const int iy = iy0 + t / 3, ix = ix0 + t % 3;
+                for (int t = 0; t < kTaps; ++t) {
+                    const int iy = iy0 + t / KS, ix = ix0 + t % KS;
                     if (iy < 0 || iy >= p.H || ix < 0 || ix >= p.W) {
 #pragma unroll
-                        for (int j = 0; j < kChanPerThread; ++j) v[j] -= sWsum[(cg * kChanPerThread + j) * 9 + t];
+                        for (int j = 0; j < kChanPerThread; ++j) v[j] -= sWsum[(cg * kChanPerThread + j) * kMaxTaps + t];
                     }
                 }
             }
@@ -516,7 +535,7 @@ pack_weights_pointwise_kernel(const uint32_t *__restrict__ w, uint32_t *__restri
         }
         if (g == 0) {  // per-tap sums are never used by a pointwise convolution (nothing is padded)
             int32_t *wsum = reinterpret_cast<int32_t *>(block + (int64_t)groups * kChanGroups * kWGroupStride);
-            for (int t = 0; t < 9; ++t) wsum[ch * 9 + t] = 0;
+            for (int t = 0; t < kMaxTaps; ++t) wsum[ch * kMaxTaps + t] = 0;
         }
     }
 }
@@ -691,10 +710,10 @@ lce_status launch1x1(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStr
     return launch_status();
 }
 
-template <int STRIDE, int TP>
-lce_status launch3x3(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStream_t s)
+template <int KS, int STRIDE, int TP>
+lce_status launch_kxk(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStream_t s)
 {
-    auto kernel = bconv3x3_kernel<STRIDE, TP>;
+    auto kernel = bconv3x3_kernel<KS, STRIDE, TP>;
     if (smem_bytes > 48 * 1024) {
         // opt in to the large dynamic shared memory carve-out
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
@@ -710,7 +729,7 @@ int reg_limited_ctas(int tp) { return (tp <= 2 ? 24 : 16) / kWarps; }
 
 size_t smem_bytes_for(const ConvGeom &g, const TiledParams &p)
 {
-    return ((size_t)g.Cw * kChanGroups * kWGroupStride + kWsumWords + 2 * (size_t)g.Cw * p.plane) * 4;
+    return ((size_t)g.Cw * groups_per_word(g.KH) * kChanGroups * kWGroupStride + kWsumWords + 2 * (size_t)g.Cw * p.plane) * 4;
 }
 
 void set_tile(const ConvGeom &g, TiledParams *p, int tile_pixels)
@@ -718,11 +737,11 @@ void set_tile(const ConvGeom &g, TiledParams *p, int tile_pixels)
     p->tile_pixels = tile_pixels;
     int rows_max = (tile_pixels - 1) / g.OW + 2;  // output rows a run of tile_pixels flat pixels can touch
     if (rows_max > tile_pixels) rows_max = tile_pixels;
-    const int nv_max = (rows_max - 1) * 3 + 3;     // consecutive output rows are at most 3 virtual rows apart
+    const int nv_max = (rows_max - 1) * g.KH + g.KH;  // consecutive output rows are at most KH virtual rows apart
     p->plane = nv_max * p->pitch;
 }
 
-bool covers3x3(const ConvGeom &g) { return g.KH == 3 && g.KW == 3 && g.sh == g.sw && g.sh <= 2; }
+bool covers3x3(const ConvGeom &g) { return g.KH == g.KW && (g.KH == 3 || g.KH == 5) && g.sh == g.sw && g.sh <= 2; }
 bool covers1x1(const ConvGeom &g) { return g.KH == 1 && g.KW == 1 && g.sh == g.sw; }
 
 bool tiled_covers(const ConvGeom &g)
@@ -741,7 +760,7 @@ void pointwise_split(int Cw, int *n9, int *rem3)
 
 int image_groups(const ConvGeom &g)
 {
-    if (covers3x3(g)) return g.Cw;
+    if (covers3x3(g)) return g.Cw * groups_per_word(g.KH);
     int n9, rem3;
     pointwise_split(g.Cw, &n9, &rem3);
     return pointwise_groups(n9, rem3);
@@ -818,7 +837,7 @@ lce_status launch_pack_weights_tiled(const ConvGeom &g, const uint32_t *w, uint3
     int blocks = (int)((entries + 127) / 128);
     if (blocks > 148 * 8) blocks = 148 * 8;
     if (covers3x3(g))
-        pack_weights_kernel<<<blocks, 128, 0, s>>>(w, image, g.Cout, g.Cw, g.Cin, chan_blocks);
+        pack_weights_kernel<<<blocks, 128, 0, s>>>(w, image, g.Cout, g.Cw, g.Cin, chan_blocks, g.KH);
     else
         pack_weights_pointwise_kernel<<<blocks, 128, 0, s>>>(w, image, g.Cout, g.Cw, groups, chan_blocks);
     return launch_status();
@@ -864,8 +883,8 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
         return launch1x1<4>(p, smem_bytes, grid, s);
     }
 
-    p.Hp = (g.OH - 1) * g.sh + 3;
-    p.Wp = (g.OW - 1) * g.sh + 3;
+    p.Hp = (g.OH - 1) * g.sh + g.KH;
+    p.Wp = (g.OW - 1) * g.sh + g.KW;
     if (p.Wp < g.W + g.pl) p.Wp = g.W + g.pl;  // staging writes the whole image row; columns past the taps are unused
     p.pitch = p.Wp | 1;  // odd pitch: the 4 pixels of a warp in 4 different rows hit 4 different banks
     auto smem_for = [&](int tile) {
@@ -877,14 +896,24 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
     p.n_tiles = (int32_t)((g.M + c.tile - 1) / c.tile);
     const size_t smem_bytes = smem_bytes_for(g, p);
     dim3 grid((unsigned)c.ctas_x, (unsigned)chan_blocks, 1);
-    if (g.sh == 1) {
-        if (c.tp == 2) return launch3x3<1, 2>(p, smem_bytes, grid, s);
-        if (c.tp == 3) return launch3x3<1, 3>(p, smem_bytes, grid, s);
-        return launch3x3<1, 4>(p, smem_bytes, grid, s);
+    if (g.KH == 3) {
+        if (g.sh == 1) {
+            if (c.tp == 2) return launch_kxk<3, 1, 2>(p, smem_bytes, grid, s);
+            if (c.tp == 3) return launch_kxk<3, 1, 3>(p, smem_bytes, grid, s);
+            return launch_kxk<3, 1, 4>(p, smem_bytes, grid, s);
+        }
+        if (c.tp == 2) return launch_kxk<3, 2, 2>(p, smem_bytes, grid, s);
+        if (c.tp == 3) return launch_kxk<3, 2, 3>(p, smem_bytes, grid, s);
+        return launch_kxk<3, 2, 4>(p, smem_bytes, grid, s);
     }
-    if (c.tp == 2) return launch3x3<2, 2>(p, smem_bytes, grid, s);
-    if (c.tp == 3) return launch3x3<2, 3>(p, smem_bytes, grid, s);
-    return launch3x3<2, 4>(p, smem_bytes, grid, s);
+    if (g.sh == 1) {
+        if (c.tp == 2) return launch_kxk<5, 1, 2>(p, smem_bytes, grid, s);
+        if (c.tp == 3) return launch_kxk<5, 1, 3>(p, smem_bytes, grid, s);
+        return launch_kxk<5, 1, 4>(p, smem_bytes, grid, s);
+    }
+    if (c.tp == 2) return launch_kxk<5, 2, 2>(p, smem_bytes, grid, s);
+    if (c.tp == 3) return launch_kxk<5, 2, 3>(p, smem_bytes, grid, s);
+    return launch_kxk<5, 2, 4>(p, smem_bytes, grid, s);
 }
 
 }  // namespace lce

@@ -154,6 +154,19 @@ def config3_specs(batch: int = 64) -> List[ConvSpec]:
     ]
 
 
+def sweep_specs(batch: int = 1) -> List[ConvSpec]:
+    """The paper's convolution sweep (Section 5.1): square inputs of 8..64 pixels, Cin = Cout from 32
+    to 256, 3x3 and 5x5 filters, stride 1, same padding; float outputs as in a full-precision-output
+    benchmark of one layer.  The paper runs it one image at a time; batch scales it for a GPU."""
+    specs = []
+    for kernel in (3, 5):
+        for size in (8, 16, 32, 64):
+            for ch in (32, 64, 96, 128, 160, 256):
+                specs.append(ConvSpec(f"sweep_{size}x{size}x{ch}_k{kernel}", batch, size, size, ch, ch, kernel, 1,
+                                      PAD_SAME_ONE, OUT_FLOAT32))
+    return specs
+
+
 @dataclass(frozen=True)
 class Step:
     """One kernel call of a chain. kind: bitpack | bconv | bconv_fused | add | bmaxpool.

@@ -297,7 +297,7 @@ __device__ __forceinline__ int tile_first_vrow(const TiledParams &p, int m0)
 // Copies the input rows a tile needs into shared memory: global [n][iy][ix][cw] -> [cw][v][x] in
 // padded-image coordinates.  Image words travel as asynchronous copies (the caller waits for
 // them); rows and columns outside the image are written as zero words (one-padding).
-template <int KS, int STRIDE>
+template <int KS, int STRIDE, int NW>
 __device__ __forceinline__ void stage_rows(const TiledParams &p, int m0, int m_end, uint32_t *sA, int warp, int lane)
 {
     const int r_last = (m_end - 1) / p.OW;
@@ -305,7 +305,7 @@ __device__ __forceinline__ void stage_rows(const TiledParams &p, int m0, int m_e
     const int v_last = (r_last / p.OH) * p.Hp + (r_last % p.OH) * STRIDE + (KS - 1);
     const int nv = v_last - v_first + 1;
     const int row_words = p.W * p.Cw;
-    for (int v = warp; v < nv; v += kWarps) {
+    for (int v = warp; v < nv; v += NW) {
         const int va = v_first + v;
         const int n = va / p.Hp;
         const int iy = va - n * p.Hp - p.pt;
@@ -332,10 +332,14 @@ __device__ __forceinline__ void stage_rows(const TiledParams &p, int m0, int m_e
     }
 }
 
-template <int KS, int STRIDE, int TP>
-__global__ void __launch_bounds__(kThreads, (TP <= 2 ? 24 : 16) / kWarps)
+// NW warps per CTA: 4 normally; 8 when the weight operands of a channel block are so large that
+// only one CTA fits an SM, so that the SM still has eight warps to hide latencies with.
+template <int KS, int STRIDE, int TP, int NW>
+__global__ void __launch_bounds__(32 * NW, (TP <= 2 ? 24 : 16) / NW)
 bconv3x3_kernel(const TiledParams p)
 {
+    constexpr int kThreads = 32 * NW;
+    constexpr int kPixPerStep = 4 * NW;
     constexpr int kTaps = KS * KS;             // 9 or 25
     constexpr int kNG = groups_per_word(KS);   // nine-word groups per channel word: 1 or 3
     extern __shared__ __align__(16) uint32_t smem[];
@@ -395,7 +399,7 @@ bconv3x3_kernel(const TiledParams p)
     // the other buffer while the current tile is computed --------------------------------------
     int tile = blockIdx.x;
     if (tile < p.n_tiles)
-        stage_rows<KS, STRIDE>(p, tile * p.tile_pixels, min((tile + 1) * p.tile_pixels, p.M), sA0, warp, lane);
+        stage_rows<KS, STRIDE, NW>(p, tile * p.tile_pixels, min((tile + 1) * p.tile_pixels, p.M), sA0, warp, lane);
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
@@ -407,7 +411,7 @@ bconv3x3_kernel(const TiledParams p)
     {
         const int next = tile + gridDim.x;
         if (next < p.n_tiles)
-            stage_rows<KS, STRIDE>(p, next * p.tile_pixels, min((next + 1) * p.tile_pixels, p.M),
+            stage_rows<KS, STRIDE, NW>(p, next * p.tile_pixels, min((next + 1) * p.tile_pixels, p.M),
                                sA0 + (buf ^ 1) * plane_words, warp, lane);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
@@ -710,22 +714,22 @@ lce_status launch1x1(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStr
     return launch_status();
 }
 
-template <int KS, int STRIDE, int TP>
+template <int KS, int STRIDE, int TP, int NW = kWarps>
 lce_status launch_kxk(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStream_t s)
 {
-    auto kernel = bconv3x3_kernel<KS, STRIDE, TP>;
+    auto kernel = bconv3x3_kernel<KS, STRIDE, TP, NW>;
     if (smem_bytes > 48 * 1024) {
         // opt in to the large dynamic shared memory carve-out
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
             return LCE_ERR_CUDA;
     }
-    kernel<<<grid, kThreads, smem_bytes, s>>>(p);
+    kernel<<<grid, 32 * NW, smem_bytes, s>>>(p);
     return launch_status();
 }
 
 // CTAs of 128 threads that the register file lets share an SM, per pixels-per-thread variant
 // (must match the __launch_bounds__ of the kernel).
-int reg_limited_ctas(int tp) { return (tp <= 2 ? 24 : 16) / kWarps; }
+int reg_limited_ctas(int tp, int nw) { return (tp <= 2 ? 24 : 16) / nw; }
 
 size_t smem_bytes_for(const ConvGeom &g, const TiledParams &p)
 {
@@ -768,6 +772,7 @@ int image_groups(const ConvGeom &g)
 
 struct TileChoice {
     int tp, tile, ctas_x;
+    double cost;
 };
 
 // Pixels per thread (TP) and tile size: a tile covers 16*TP*rounds flat pixels and the grid is
@@ -775,7 +780,8 @@ struct TileChoice {
 // best: cost = (CTAs on the busiest SM) x (tiles of the busiest CTA) x (tile work), with a
 // penalty when too few warps share an SM to keep the logic pipe busy.
 template <typename SmemFn>
-bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileChoice *best)
+bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileChoice *best, int nw = kWarps,
+                 size_t smem_limit = 110 * 1024)
 {
     int sms = 148;
     {
@@ -791,28 +797,29 @@ bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileC
     best->tile = 0;
     for (int tp = 2; tp <= 4; ++tp) {
         if (forced_tp && tp != forced_tp) continue;
-        const int unit = kPixPerStep * tp;
+        const int unit = 4 * nw * tp;
         for (int rounds = 1; rounds <= 2; ++rounds) {
             if (forced_rounds && rounds != forced_rounds) continue;
             const int tile = unit * rounds;
             const size_t smem = smem_for_tile(tile);
-            if (smem > 110 * 1024) continue;
+            if (smem > smem_limit) continue;
             int per_sm = (int)((220 * 1024) / (smem + 1024));
-            if (per_sm > reg_limited_ctas(tp)) per_sm = reg_limited_ctas(tp);
+            if (per_sm < 1) per_sm = 1;
+            if (per_sm > reg_limited_ctas(tp, nw)) per_sm = reg_limited_ctas(tp, nw);
             const int64_t n_tiles = (g.M + tile - 1) / tile;
             int64_t ctas_x = ((int64_t)sms * per_sm) / chan_blocks;
             if (ctas_x < 1) ctas_x = 1;
             if (ctas_x > n_tiles) ctas_x = n_tiles;
             const int64_t tiles_per_cta = (n_tiles + ctas_x - 1) / ctas_x;
             const int64_t ctas_on_sm = (ctas_x * chan_blocks + sms - 1) / sms;
-            const double warps = (double)ctas_x * chan_blocks / sms * kWarps;
+            const double warps = (double)ctas_x * chan_blocks / sms * nw;
             const double eff = warps >= 16 ? 1.0 : (warps >= 8 ? 0.8 + 0.2 * (warps - 8) / 8 : 0.4 + 0.4 * warps / 8);
             // fewer pixels per thread re-read the weight operands from shared memory more often
             const double smem_penalty = tp == 2 ? 1.06 : (tp == 3 ? 1.02 : 1.0);
             const double cost = (double)ctas_on_sm * tiles_per_cta * (tile * smem_penalty + 4.0) / eff;
             if (best->tile == 0 || cost < best_cost) {
                 best->tile = tile; best->tp = tp; best->ctas_x = (int)ctas_x;
-                best_cost = cost;
+                best_cost = best->cost = cost;
             }
         }
     }
@@ -891,29 +898,37 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
         set_tile(g, &p, tile);
         return smem_bytes_for(g, p);
     };
-    if (!choose_tile(g, chan_blocks, smem_for, &c)) return LCE_ERR_UNSUPPORTED;
+    // Eight warps per CTA share one copy of the weight operands and one staging buffer, which
+    // measures faster than two CTAs of four warps wherever a whole tile of 32*TP pixels is useful
+    // work; CTAs of four warps remain for problems too small to fill such tiles on every SM.
+    int nw = 8;
+    TileChoice c4;
+    const bool ok8 = choose_tile(g, chan_blocks, smem_for, &c, 8, 226 * 1024);
+    const bool ok4 = choose_tile(g, chan_blocks, smem_for, &c4, 4, 110 * 1024);
+    if (!ok8 && !ok4) return LCE_ERR_UNSUPPORTED;
+    if (!ok8 || (ok4 && c4.cost < c.cost)) { c = c4; nw = 4; }
+#ifdef LCE_TUNING
+    if (const char *e = getenv("LCE_NW")) {
+        const int want = atoi(e);
+        if (want == 4 && ok4) { c = c4; nw = 4; }
+        if (want == 8 && ok8) { choose_tile(g, chan_blocks, smem_for, &c, 8, 226 * 1024); nw = 8; }
+    }
+#endif
     set_tile(g, &p, c.tile);
     p.n_tiles = (int32_t)((g.M + c.tile - 1) / c.tile);
     const size_t smem_bytes = smem_bytes_for(g, p);
     dim3 grid((unsigned)c.ctas_x, (unsigned)chan_blocks, 1);
-    if (g.KH == 3) {
-        if (g.sh == 1) {
-            if (c.tp == 2) return launch_kxk<3, 1, 2>(p, smem_bytes, grid, s);
-            if (c.tp == 3) return launch_kxk<3, 1, 3>(p, smem_bytes, grid, s);
-            return launch_kxk<3, 1, 4>(p, smem_bytes, grid, s);
-        }
-        if (c.tp == 2) return launch_kxk<3, 2, 2>(p, smem_bytes, grid, s);
-        if (c.tp == 3) return launch_kxk<3, 2, 3>(p, smem_bytes, grid, s);
-        return launch_kxk<3, 2, 4>(p, smem_bytes, grid, s);
-    }
-    if (g.sh == 1) {
-        if (c.tp == 2) return launch_kxk<5, 1, 2>(p, smem_bytes, grid, s);
-        if (c.tp == 3) return launch_kxk<5, 1, 3>(p, smem_bytes, grid, s);
-        return launch_kxk<5, 1, 4>(p, smem_bytes, grid, s);
-    }
-    if (c.tp == 2) return launch_kxk<5, 2, 2>(p, smem_bytes, grid, s);
-    if (c.tp == 3) return launch_kxk<5, 2, 3>(p, smem_bytes, grid, s);
-    return launch_kxk<5, 2, 4>(p, smem_bytes, grid, s);
+#define LCE_LAUNCH_TP(KS, ST, NW)                                                   \
+    do {                                                                            \
+        if (c.tp == 2) return launch_kxk<KS, ST, 2, NW>(p, smem_bytes, grid, s);    \
+        if (c.tp == 3) return launch_kxk<KS, ST, 3, NW>(p, smem_bytes, grid, s);    \
+        return launch_kxk<KS, ST, 4, NW>(p, smem_bytes, grid, s);                   \
+    } while (0)
+    if (g.KH == 3 && g.sh == 1) { if (nw == 8) LCE_LAUNCH_TP(3, 1, 8); else LCE_LAUNCH_TP(3, 1, 4); }
+    if (g.KH == 3) { if (nw == 8) LCE_LAUNCH_TP(3, 2, 8); else LCE_LAUNCH_TP(3, 2, 4); }
+    if (g.sh == 1) { if (nw == 8) LCE_LAUNCH_TP(5, 1, 8); else LCE_LAUNCH_TP(5, 1, 4); }
+    if (nw == 8) LCE_LAUNCH_TP(5, 2, 8); else LCE_LAUNCH_TP(5, 2, 4);
+#undef LCE_LAUNCH_TP
 }
 
 }  // namespace lce

@@ -82,6 +82,8 @@ FUZZ = [
     # 5x5 filters: 25 taps = two full nine-word groups and one partial group per channel word
     (2, 16, 16, 64, 64, 5, 1), (1, 33, 29, 96, 70, 5, 1), (2, 17, 19, 160, 40, 5, 2), (3, 8, 8, 256, 256, 5, 1),
     (1, 4, 3, 32, 9, 5, 1), (1, 64, 64, 32, 32, 5, 1),
+    # wide rows and 256 channels: weights too large for two CTAs per SM -> the eight-warp variant
+    (1, 20, 64, 256, 70, 5, 1),
     # few input channels: the whole receptive field fits one word
     (2, 20, 18, 3, 32, 3, 2), (1, 9, 9, 1, 40, 5, 1), (1, 12, 11, 2, 70, 3, 1), (2, 8, 8, 3, 5, 3, 1),
 ]

@@ -354,6 +354,7 @@ def run_lce(args):
     if world == 1 and not args.no_chains:
         line["chains"] = time_chains(dev)
         line["tensor_core_path"] = time_tensor_path(dev, layers)
+        line["paper_sweep"] = time_paper_sweep(dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cores = len(os.sched_getaffinity(0))
         sample_batch, passes = BATCH, 2
@@ -408,6 +409,57 @@ def time_tensor_path(dev, layers, reps: int = 5):
             total_macs += s.binary_macs
     out["all_8_launches"] = {"us": total_ms * 1e3, "T_bmac_per_s": total_macs / (total_ms * 1e-3) / 1e12}
     out["device_status"] = lce.lce_device_status()
+    return out
+
+
+def time_paper_sweep(dev, reps: int = 3):
+    """The paper's convolution sweep (Section 5.1: Cin = Cout in {32..256}, 8..64 pixels square, 3x3 and
+    5x5, stride 1, same padding, float output) through the default integer path: 48 layers, each timed
+    alone as a CUDA-graph replay of 10 launches, at the headline batch and one image at a time (the
+    paper's setting).  Reported beside the headline, outside its timed region."""
+    import torch
+
+    import paper_2011_09398_b200 as lce
+    stream = torch.cuda.Stream(device=dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(wl.SEED0 % (2**31))
+    out = {}
+    for batch in (BATCH, 1):
+        rows, total_s, total_macs = {}, 0.0, 0
+        for s in wl.sweep_specs(batch):
+            a = torch.randint(-2**31, 2**31 - 1, (s.batch, s.in_h, s.in_w, s.in_words), dtype=torch.int32, device=dev, generator=gen)
+            w = torch.randint(-2**31, 2**31 - 1, (s.out_c, s.kernel, s.kernel, s.in_words), dtype=torch.int32, device=dev, generator=gen)
+            mult = torch.rand(s.out_c, device=dev, generator=gen) + 0.5
+            bias = torch.randn(s.out_c, device=dev, generator=gen) * 0.1
+            desc = lce.make_desc(s.batch, s.in_h, s.in_w, s.in_c, s.out_c, (s.kernel, s.kernel), (1, 1), s.padding,
+                                 s.out_type, lce.ACT_NONE, lce.KERNEL_AUTO, 1)
+            wp = lce.lce_bconv2d_pack_weights(desc, w)
+            o = lce.lce_bconv2d(desc, a, wp, mult, bias, None)
+            with torch.cuda.stream(stream):
+                stream.wait_stream(torch.cuda.current_stream(dev))
+                for _ in range(3):
+                    lce.lce_bconv2d(desc, a, wp, mult, bias, None, o)
+                stream.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    for _ in range(10):
+                        lce.lce_bconv2d(desc, a, wp, mult, bias, None, o)
+                g.replay()
+                stream.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(reps):
+                    g.replay()
+                e1.record(stream)
+                stream.synchronize()
+            sec = e0.elapsed_time(e1) * 1e-3 / (10 * reps)
+            rows[s.name] = {"us": round(sec * 1e6, 2), "T_bmac_per_s": round(s.binary_macs / sec / 1e12, 2)}
+            total_s += sec
+            total_macs += s.binary_macs
+            del g, a, w, wp, o
+        rates = [r["T_bmac_per_s"] for r in rows.values()]
+        out[f"batch_{batch}"] = {"layers": len(rows), "sum_us": total_s * 1e6, "T_bmac_per_s_whole_sweep": total_macs / total_s / 1e12,
+                                 "T_bmac_per_s_min": min(rates), "T_bmac_per_s_max": max(rates), "per_layer": rows}
     return out
 
 

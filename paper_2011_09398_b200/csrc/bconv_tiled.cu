@@ -18,6 +18,7 @@
 //     word; the weight-side operands of one channel are read from shared memory once and used
 //     for all TP pixels (shared-memory bandwidth, not issue slots, is what this ordering saves);
 //   * epilogue: acc = K - 2*count, then float multiply-add, threshold + bit-pack, or raw int32.
+#include <stdio.h>
 #include <stdlib.h>
 
 #include "common.cuh"
@@ -770,6 +771,11 @@ int image_groups(const ConvGeom &g)
     return pointwise_groups(n9, rem3);
 }
 
+#ifndef LCE_MAX_ROUNDS
+#define LCE_MAX_ROUNDS 2
+#endif
+constexpr int kMaxRounds = LCE_MAX_ROUNDS;
+
 struct TileChoice {
     int tp, tile, ctas_x;
     double cost;
@@ -798,7 +804,7 @@ bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileC
     for (int tp = 2; tp <= 4; ++tp) {
         if (forced_tp && tp != forced_tp) continue;
         const int unit = 4 * nw * tp;
-        for (int rounds = 1; rounds <= 2; ++rounds) {
+        for (int rounds = 1; rounds <= kMaxRounds; ++rounds) {
             if (forced_rounds && rounds != forced_rounds) continue;
             const int tile = unit * rounds;
             const size_t smem = smem_for_tile(tile);
@@ -918,6 +924,11 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
     p.n_tiles = (int32_t)((g.M + c.tile - 1) / c.tile);
     const size_t smem_bytes = smem_bytes_for(g, p);
     dim3 grid((unsigned)c.ctas_x, (unsigned)chan_blocks, 1);
+#ifdef LCE_TUNING
+    if (getenv("LCE_VERBOSE"))
+        fprintf(stderr, "tiled %dx%d M=%lld Cw=%d Cout=%d: nw=%d tp=%d tile=%d n_tiles=%d grid=%dx%d smem=%zu cost=%.0f\n", g.KH, g.KW,
+                (long long)g.M, g.Cw, g.Cout, nw, c.tp, c.tile, p.n_tiles, c.ctas_x, chan_blocks, smem_bytes, c.cost);
+#endif
 #define LCE_LAUNCH_TP(KS, ST, NW)                                                   \
     do {                                                                            \
         if (c.tp == 2) return launch_kxk<KS, ST, 2, NW>(p, smem_bytes, grid, s);    \

@@ -127,6 +127,21 @@ lce_status lce_bconv2d_fused(const lce_bconv2d_desc *desc, const uint32_t *input
                              const float *multiplier, const float *bias, const float *residual,
                              float *out_float, uint32_t *out_packed, void *stream);
 
+/* LceQuantize fused into LceBConv2d's loader (Section 3.2: a binarized convolution whose input is a
+ * full-precision tensor is preceded by LceQuantize; Section 5.3 counts that op's share of the run
+ * time).  `input` is the fp32 activation tensor [batch][in_h][in_w][in_c] (device); the kernel
+ * takes the sign bit of each value (negative -> bit 1, as lce_bitpack does) while it stages the
+ * rows, so the packed tensor never exists in memory.  Everything else is lce_bconv2d, and the
+ * result is bit-identical to lce_bitpack followed by lce_bconv2d.  Covers the shapes of the tiled
+ * KxK kernel (3x3 and 5x5 filters, equal strides of 1 or 2); anything else, and desc->kernel set to
+ * DIRECT or TENSOR, returns LCE_ERR_UNSUPPORTED (call lce_bitpack, then lce_bconv2d).
+ * Cost: the sign loads are synchronous and every channel block and halo row repeats them, so on
+ * this GPU the call is slower than lce_bitpack + lce_bconv2d for every measured shape; what it
+ * saves is the packed tensor's memory. */
+lce_status lce_bconv2d_f32(const lce_bconv2d_desc *desc, const float *input, const uint32_t *weights,
+                           const float *multiplier, const float *bias, const int32_t *thresholds,
+                           void *output, void *stream);
+
 /* Load-time weight packing (Section 3.2: the paper's BGEMM also re-arranges the weights ahead of
  * time for its access pattern; Section 3.1: weights are converted once, when the model is built).  Rewrites
  * the plain packed weights into the operand layout the tiled kernel copies straight into shared

@@ -47,6 +47,8 @@ def library() -> ctypes.CDLL:
         lib.lce_unpack.argtypes = [vp, vp, i64, i32, vp]
         lib.lce_bconv2d_out_shape.argtypes = [ctypes.POINTER(BConv2dDesc), ctypes.POINTER(i32), ctypes.POINTER(i32)]
         lib.lce_bconv2d.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp]
+        lib.lce_bconv2d_f32.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp]
+        lib.lce_bconv2d_f32.restype = ctypes.c_int
         lib.lce_bconv2d_fused.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp, vp]
         lib.lce_bconv2d_fused.restype = ctypes.c_int
         lib.lce_bconv2d_packed_weights_bytes.restype = ctypes.c_size_t
@@ -161,6 +163,30 @@ def lce_bconv2d(desc: BConv2dDesc, input: torch.Tensor, weights: torch.Tensor,
         _dev(bias, torch.float32, "bias") if bias is not None else None,
         _dev(thresholds, torch.int32, "thresholds") if thresholds is not None else None,
         _dev(out, out_dtype, "out"), _stream()), "lce_bconv2d")
+    return out
+
+
+def lce_bconv2d_f32(desc: BConv2dDesc, input: torch.Tensor, weights: torch.Tensor,
+                    multiplier: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+                    thresholds: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """LceQuantize + LceBConv2d in one kernel: `input` is the fp32 tensor [batch][in_h][in_w][in_c]."""
+    oh, ow = lce_bconv2d_out_shape(desc)
+    if out is None:
+        last = _words(desc.out_c) if desc.out_type == OUT_BITPACKED else desc.out_c
+        out = torch.empty((desc.batch, oh, ow, last), dtype=torch.float32 if desc.out_type == OUT_FLOAT32 else torch.int32,
+                          device=input.device)
+    expect_w = desc.out_c * desc.kernel_h * desc.kernel_w * _words(desc.in_c)
+    if desc.weights_packed:
+        expect_w = lce_bconv2d_packed_weights_bytes(desc) // 4
+    if input.numel() != desc.batch * desc.in_h * desc.in_w * desc.in_c or weights.numel() != expect_w:
+        raise ValueError("input / weights size does not match the descriptor")
+    out_dtype = torch.float32 if desc.out_type == OUT_FLOAT32 else torch.int32
+    _check(library().lce_bconv2d_f32(
+        ctypes.byref(desc), _dev(input, torch.float32, "input"), _dev(weights, torch.int32, "weights"),
+        _dev(multiplier, torch.float32, "multiplier") if multiplier is not None else None,
+        _dev(bias, torch.float32, "bias") if bias is not None else None,
+        _dev(thresholds, torch.int32, "thresholds") if thresholds is not None else None,
+        _dev(out, out_dtype, "out"), _stream()), "lce_bconv2d_f32")
     return out
 
 

@@ -147,6 +147,29 @@ extern "C" lce_status lce_bconv2d_fused(const lce_bconv2d_desc *desc, const uint
                               static_cast<cudaStream_t>(stream), residual, out_packed);
 }
 
+extern "C" lce_status lce_bconv2d_f32(const lce_bconv2d_desc *desc, const float *input, const uint32_t *weights,
+                                      const float *multiplier, const float *bias, const int32_t *thresholds,
+                                      void *output, void *stream)
+{
+    using namespace lce;
+    ConvGeom g;
+    lce_status st = check_conv_args(desc, &g, input, weights, multiplier, bias, thresholds, output);
+    if (st != LCE_OK) return st;
+    if (!aligned(input, 4) || !aligned(weights, 4) || !aligned(output, 4) ||
+        (multiplier && !aligned(multiplier, 4)) || (bias && !aligned(bias, 4)) ||
+        (thresholds && !aligned(thresholds, 4)))
+        return LCE_ERR_ALIGNMENT;
+    const uint32_t *image = nullptr;
+    if (desc->weights_packed) {
+        if (!aligned(weights, 256)) return LCE_ERR_ALIGNMENT;
+        if (tiled_weight_image_bytes(g) > 0)
+            image = reinterpret_cast<const uint32_t *>(reinterpret_cast<const char *>(weights) + plain_weight_bytes(g));
+    }
+    if (desc->kernel == LCE_KERNEL_DIRECT || desc->kernel == LCE_KERNEL_TENSOR) return LCE_ERR_UNSUPPORTED;
+    return launch_bconv_tiled(g, nullptr, weights, image, multiplier, bias, thresholds, output,
+                              static_cast<cudaStream_t>(stream), nullptr, nullptr, input);
+}
+
 extern "C" size_t lce_bconv2d_packed_weights_bytes(const lce_bconv2d_desc *desc)
 {
     lce::ConvGeom g;

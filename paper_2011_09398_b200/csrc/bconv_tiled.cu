@@ -43,6 +43,7 @@ constexpr int kWsumWords = kChanPerCta * kMaxTaps;         // per-tap weight sum
 
 struct TiledParams {
     const uint32_t *in;
+    const float *in_f32;       // KxK kernel: float activations, binarized while staged (then `in` is unused)
     const uint32_t *w;         // plain packed weights [Cout][3][3][Cw]
     const uint32_t *w_image;   // packed-weights image (see image_block_words), or nullptr
     const float *mult;
@@ -295,10 +296,46 @@ __device__ __forceinline__ int tile_first_vrow(const TiledParams &p, int m0)
     return (r_first / p.OH) * p.Hp + (r_first % p.OH) * STRIDE;
 }
 
+// LceQuantize fused into the loader, one image row: lane = channel within a word, one coalesced
+// 128-byte load and one ballot per word (bit = 1 for a negative value), eight words in flight per
+// warp; lane u keeps word u of the batch and writes it.
+struct RowF32 {
+    int W, Cw, Cin, plane, pl, Wp;
+};
+__device__ __forceinline__ void stage_row_f32(const float *src, uint32_t *dst_row, RowF32 p, int lane)
+{
+    const int row_words = p.W * p.Cw;
+    for (int e0 = 0; e0 < row_words; e0 += 8) {
+        float x[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int e = e0 + u;
+            const int ix = e / p.Cw, c = (e - ix * p.Cw) * 32 + lane;
+            x[u] = (e < row_words && c < p.Cin) ? __ldg(src + (int64_t)ix * p.Cin + c) : 0.0f;
+        }
+        uint32_t mine = 0u;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t word = __ballot_sync(0xffffffffu, x[u] < 0.0f);
+            if (lane == u) mine = word;
+        }
+        const int e = e0 + lane;
+        if (lane < 8 && e < row_words) {
+            const int ix = e / p.Cw, cw = e - ix * p.Cw;
+            dst_row[cw * p.plane + ix + p.pl] = mine;
+        }
+    }
+    const int edge = p.Wp - p.W;
+    for (int e = lane; e < edge * p.Cw; e += 32) {
+        const int cw = e / edge, k = e - cw * edge;
+        dst_row[cw * p.plane + (k < p.pl ? k : p.W + k)] = 0u;
+    }
+}
+
 // Copies the input rows a tile needs into shared memory: global [n][iy][ix][cw] -> [cw][v][x] in
 // padded-image coordinates.  Image words travel as asynchronous copies (the caller waits for
 // them); rows and columns outside the image are written as zero words (one-padding).
-template <int KS, int STRIDE, int NW>
+template <int KS, int STRIDE, int NW, bool F32>
 __device__ __forceinline__ void stage_rows(const TiledParams &p, int m0, int m_end, uint32_t *sA, int warp, int lane)
 {
     const int r_last = (m_end - 1) / p.OW;
@@ -311,7 +348,10 @@ __device__ __forceinline__ void stage_rows(const TiledParams &p, int m0, int m_e
         const int n = va / p.Hp;
         const int iy = va - n * p.Hp - p.pt;
         uint32_t *dst_row = sA + v * p.pitch;
-        if (n < p.N && iy >= 0 && iy < p.H) {
+        if (F32 && n < p.N && iy >= 0 && iy < p.H) {
+            stage_row_f32(p.in_f32 + ((int64_t)n * p.H + iy) * p.W * p.Cin, dst_row,
+                          RowF32{p.W, p.Cw, p.Cin, p.plane, p.pl, p.Wp}, lane);
+        } else if (n < p.N && iy >= 0 && iy < p.H) {
             const uint32_t *src = p.in + ((int64_t)n * p.H + iy) * row_words;
             for (int e = lane; e < row_words; e += 32) {
                 int ix, cw;
@@ -335,7 +375,7 @@ __device__ __forceinline__ void stage_rows(const TiledParams &p, int m0, int m_e
 
 // NW warps per CTA: 4 normally; 8 when the weight operands of a channel block are so large that
 // only one CTA fits an SM, so that the SM still has eight warps to hide latencies with.
-template <int KS, int STRIDE, int TP, int NW>
+template <int KS, int STRIDE, int TP, int NW, bool F32>
 __global__ void __launch_bounds__(32 * NW, (TP <= 2 ? 24 : 16) / NW)
 bconv3x3_kernel(const TiledParams p)
 {
@@ -400,7 +440,7 @@ bconv3x3_kernel(const TiledParams p)
     // the other buffer while the current tile is computed --------------------------------------
     int tile = blockIdx.x;
     if (tile < p.n_tiles)
-        stage_rows<KS, STRIDE, NW>(p, tile * p.tile_pixels, min((tile + 1) * p.tile_pixels, p.M), sA0, warp, lane);
+        stage_rows<KS, STRIDE, NW, F32>(p, tile * p.tile_pixels, min((tile + 1) * p.tile_pixels, p.M), sA0, warp, lane);
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
@@ -412,7 +452,7 @@ bconv3x3_kernel(const TiledParams p)
     {
         const int next = tile + gridDim.x;
         if (next < p.n_tiles)
-            stage_rows<KS, STRIDE, NW>(p, next * p.tile_pixels, min((next + 1) * p.tile_pixels, p.M),
+            stage_rows<KS, STRIDE, NW, F32>(p, next * p.tile_pixels, min((next + 1) * p.tile_pixels, p.M),
                                sA0 + (buf ^ 1) * plane_words, warp, lane);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
@@ -715,10 +755,10 @@ lce_status launch1x1(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStr
     return launch_status();
 }
 
-template <int KS, int STRIDE, int TP, int NW = kWarps>
+template <int KS, int STRIDE, int TP, int NW, bool F32 = false>
 lce_status launch_kxk(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStream_t s)
 {
-    auto kernel = bconv3x3_kernel<KS, STRIDE, TP, NW>;
+    auto kernel = bconv3x3_kernel<KS, STRIDE, TP, NW, F32>;
     if (smem_bytes > 48 * 1024) {
         // opt in to the large dynamic shared memory carve-out
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
@@ -858,16 +898,17 @@ lce_status launch_pack_weights_tiled(const ConvGeom &g, const uint32_t *w, uint3
 
 lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const uint32_t *w_image,
                               const float *mult, const float *bias, const int32_t *thr, void *out, cudaStream_t s,
-                              const float *residual, uint32_t *out_packed)
+                              const float *residual, uint32_t *out_packed, const float *in_f32)
 {
     if (!tiled_covers(g)) return LCE_ERR_UNSUPPORTED;
+    if (in_f32 && !covers3x3(g)) return LCE_ERR_UNSUPPORTED;
     // 128-bit epilogue accesses need 16-byte aligned buffers when the channel count allows them
     if ((g.Cout & 3) == 0 && g.out_type != LCE_OUT_BITPACKED && (!aligned(out, 16) || !aligned(residual, 16)))
         return LCE_ERR_UNSUPPORTED;
     if (w_image && !aligned(w_image, 16)) return LCE_ERR_ALIGNMENT;
     TiledParams p{};
     p.in = in; p.w = w; p.w_image = w_image; p.mult = mult; p.bias = bias; p.thr = thr; p.out = out;
-    p.residual = residual; p.out_packed = out_packed;
+    p.residual = residual; p.out_packed = out_packed; p.in_f32 = in_f32;
     p.N = g.N; p.H = g.H; p.W = g.W; p.Cin = g.Cin; p.Cw = g.Cw; p.Cout = g.Cout; p.Cow = g.Cow;
     p.OH = g.OH; p.OW = g.OW; p.pt = g.pt; p.pl = g.pl;
     p.padding = g.padding; p.out_type = g.out_type; p.activation = g.activation;
@@ -909,8 +950,10 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
     // work; CTAs of four warps remain for problems too small to fill such tiles on every SM.
     int nw = 8;
     TileChoice c4;
-    const bool ok8 = choose_tile(g, chan_blocks, smem_for, &c, 8, 226 * 1024);
-    const bool ok4 = choose_tile(g, chan_blocks, smem_for, &c4, 4, 110 * 1024);
+    // the float-input loader exists for four-warp CTAs only
+    const bool ok8 = in_f32 == nullptr && choose_tile(g, chan_blocks, smem_for, &c, 8, 226 * 1024);
+    const bool ok4 = choose_tile(g, chan_blocks, smem_for, &c4, 4, 110 * 1024) ||
+                     (in_f32 != nullptr && choose_tile(g, chan_blocks, smem_for, &c4, 4, 226 * 1024));
     if (!ok8 && !ok4) return LCE_ERR_UNSUPPORTED;
     if (!ok8 || (ok4 && c4.cost < c.cost)) { c = c4; nw = 4; }
 #ifdef LCE_TUNING
@@ -935,6 +978,19 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
         if (c.tp == 3) return launch_kxk<KS, ST, 3, NW>(p, smem_bytes, grid, s);    \
         return launch_kxk<KS, ST, 4, NW>(p, smem_bytes, grid, s);                   \
     } while (0)
+    if (in_f32) {
+#define LCE_LAUNCH_F32(KS, ST)                                                         \
+    do {                                                                               \
+        if (c.tp == 2) return launch_kxk<KS, ST, 2, 4, true>(p, smem_bytes, grid, s);  \
+        if (c.tp == 3) return launch_kxk<KS, ST, 3, 4, true>(p, smem_bytes, grid, s);  \
+        return launch_kxk<KS, ST, 4, 4, true>(p, smem_bytes, grid, s);                 \
+    } while (0)
+        if (g.KH == 3 && g.sh == 1) LCE_LAUNCH_F32(3, 1);
+        if (g.KH == 3) LCE_LAUNCH_F32(3, 2);
+        if (g.sh == 1) LCE_LAUNCH_F32(5, 1);
+        LCE_LAUNCH_F32(5, 2);
+#undef LCE_LAUNCH_F32
+    }
     if (g.KH == 3 && g.sh == 1) { if (nw == 8) LCE_LAUNCH_TP(3, 1, 8); else LCE_LAUNCH_TP(3, 1, 4); }
     if (g.KH == 3) { if (nw == 8) LCE_LAUNCH_TP(3, 2, 8); else LCE_LAUNCH_TP(3, 2, 4); }
     if (g.sh == 1) { if (nw == 8) LCE_LAUNCH_TP(5, 1, 8); else LCE_LAUNCH_TP(5, 1, 4); }

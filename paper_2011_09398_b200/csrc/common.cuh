@@ -78,7 +78,8 @@ lce_status launch_bconv_direct(const ConvGeom &g, const uint32_t *in, const uint
 // with out_packed given, `out` may be null).
 lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const uint32_t *w_image,
                               const float *mult, const float *bias, const int32_t *thr, void *out, cudaStream_t s,
-                              const float *residual = nullptr, uint32_t *out_packed = nullptr);
+                              const float *residual = nullptr, uint32_t *out_packed = nullptr,
+                              const float *in_f32 = nullptr);
 // One-word-patch kernel for tiny channel counts (KH*KW*Cin <= 32); plain weights only.
 bool patch_covers(const ConvGeom &g);
 lce_status launch_bconv_patch(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const float *mult,

@@ -57,6 +57,8 @@ struct TiledParams {
     int32_t n_tiles;      // ceil(M / tile_pixels); CTA x works on tiles x, x + gridDim.x, ...
     int32_t M, Hp, Wp, pitch, plane;
     int32_t cw_shift;     // log2(Cw) when Cw is a power of two, else -1
+    int32_t half_block;   // KxK kernel: index of the channel block with at most 32 real channels, or -1
+    int32_t full_blocks, ctas_full, ctas_half;  // KxK kernel: 1-D grid = full_blocks x ctas_full CTAs, then ctas_half
     int32_t stride;       // pointwise kernel only
     int32_t n9, rem3, cwp; // pointwise kernel: nine-word groups, leftover triples, padded words per pixel
     int32_t padding, out_type, activation;
@@ -380,7 +382,6 @@ __global__ void __launch_bounds__(32 * NW, (TP <= 2 ? 24 : 16) / NW)
 bconv3x3_kernel(const TiledParams p)
 {
     constexpr int kThreads = 32 * NW;
-    constexpr int kPixPerStep = 4 * NW;
     constexpr int kTaps = KS * KS;             // 9 or 25
     constexpr int kNG = groups_per_word(KS);   // nine-word groups per channel word: 1 or 3
     extern __shared__ __align__(16) uint32_t smem[];
@@ -391,14 +392,25 @@ bconv3x3_kernel(const TiledParams p)
 
     const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
-    const int ch0 = blockIdx.y * kChanPerCta;
+    // 1-D grid: ctas_full CTAs for each full channel block, then ctas_half for the half block
+    int block_y, block_x, ctas_x;
+    if ((int)blockIdx.x < p.full_blocks * p.ctas_full) {
+        block_y = blockIdx.x % p.full_blocks;
+        block_x = blockIdx.x / p.full_blocks;
+        ctas_x = p.ctas_full;
+    } else {
+        block_y = p.full_blocks;
+        block_x = blockIdx.x - p.full_blocks * p.ctas_full;
+        ctas_x = p.ctas_half;
+    }
+    const int ch0 = block_y * kChanPerCta;
     const int plane_words = p.Cw * p.plane;  // one input buffer; two of them alternate between tiles
 
     // ---- weights ----------------------------------------------------------------------------
     if (p.w_image != nullptr) {
         // prepared image: a plain 16-byte asynchronous copy of this channel block
         const int words = (p.padding == LCE_PAD_SAME_ZERO) ? w_words + kWsumWords : w_words;
-        const uint32_t *src = p.w_image + blockIdx.y * image_block_words(p.Cw * kNG);
+        const uint32_t *src = p.w_image + block_y * image_block_words(p.Cw * kNG);
         for (int e = tid * 4; e < words; e += kThreads * 4) cp_async16(smem + e, src + e);
         asm volatile("cp.async.commit_group;" ::: "memory");
     } else {
@@ -426,7 +438,13 @@ bconv3x3_kernel(const TiledParams p)
     }
 
     // ---- this thread's channels --------------------------------------------------------------
-    const int px = lane >> 3, cg = lane & 7;
+    // A warp is 4 pixels x 8 channel groups; in a channel block whose upper 32 channels do not
+    // exist (Cout mod 64 in 1..32) it is 8 pixels x 4 channel groups instead, so that no lane works
+    // on channels that are not there.
+    const int cg_bits = (block_y == p.half_block) ? 2 : 3;
+    const int px = lane >> cg_bits, cg = lane & ((1 << cg_bits) - 1);
+    const int pix_per_warp = 32 >> cg_bits;
+    const int pix_per_step = pix_per_warp * NW;  // pixels the CTA works on at a time
     const int chan = ch0 + cg * kChanPerThread;
     const int K = kTaps * p.Cin;
     Weights124 k124;
@@ -438,19 +456,19 @@ bconv3x3_kernel(const TiledParams p)
 
     // ---- persistent loop over this CTA's pixel tiles; the next tile's input rows are copied into
     // the other buffer while the current tile is computed --------------------------------------
-    int tile = blockIdx.x;
+    int tile = block_x;
     if (tile < p.n_tiles)
         stage_rows<KS, STRIDE, NW, F32>(p, tile * p.tile_pixels, min((tile + 1) * p.tile_pixels, p.M), sA0, warp, lane);
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
 
-  for (int buf = 0; tile < p.n_tiles; tile += gridDim.x, buf ^= 1) {
+  for (int buf = 0; tile < p.n_tiles; tile += ctas_x, buf ^= 1) {
     const uint32_t *sA = sA0 + buf * plane_words;
     const int m0 = tile * p.tile_pixels;
     const int m_end = min(m0 + p.tile_pixels, p.M);
     {
-        const int next = tile + gridDim.x;
+        const int next = tile + ctas_x;
         if (next < p.n_tiles)
             stage_rows<KS, STRIDE, NW, F32>(p, next * p.tile_pixels, min((next + 1) * p.tile_pixels, p.M),
                                sA0 + (buf ^ 1) * plane_words, warp, lane);
@@ -459,8 +477,8 @@ bconv3x3_kernel(const TiledParams p)
     const int r_first = m0 / p.OW;
     const int v_first = tile_first_vrow<STRIDE>(p, m0);
 
-    // running position of this lane's next pixel; the pixels of one lane are kPixPerStep apart
-    int m_next = m0 + warp * 4 + px;  // lanes of a warp: 4 neighbouring pixels
+    // running position of this lane's next pixel; the pixels of one lane are pix_per_step apart
+    int m_next = m0 + warp * pix_per_warp + px;  // lanes of a warp: neighbouring pixels
     int ow, voh, oh_left;  // voh = n*Hp + oh*STRIDE: the pixel's first virtual row
     {
         const int r = m_next / p.OW;
@@ -472,14 +490,14 @@ bconv3x3_kernel(const TiledParams p)
     }
     const int a_base_first = (m0 - r_first * p.OW) * STRIDE;  // the tile's first pixel sits in virtual row 0
 
-    for (int base = m0; base < m0 + p.tile_pixels; base += kPixPerStep * TP) {
+    for (int base = m0; base < m0 + p.tile_pixels; base += pix_per_step * TP) {
         int a_base[TP];
 #pragma unroll
         for (int i = 0; i < TP; ++i) {
             // pixels past the end of the tile redo the tile's first pixel and store nothing
             a_base[i] = (m_next < m_end) ? (voh - v_first) * p.pitch + ow * STRIDE : a_base_first;
-            m_next += kPixPerStep;
-            ow += kPixPerStep;
+            m_next += pix_per_step;
+            ow += pix_per_step;
             while (ow >= p.OW) {
                 ow -= p.OW;
                 if (oh_left == 0) { oh_left = p.OH - 1; voh += KS; }  // next image: Hp - (OH-1)*STRIDE = KS
@@ -523,7 +541,7 @@ bconv3x3_kernel(const TiledParams p)
         load_channel_params(p, chan, cp);
 #pragma unroll
         for (int i = 0; i < TP; ++i) {
-            const int m = base + i * kPixPerStep + warp * 4 + px;
+            const int m = base + i * pix_per_step + warp * pix_per_warp + px;
             const bool pix_ok = m < m_end;
             int32_t v[kChanPerThread];
 #pragma unroll
@@ -817,7 +835,7 @@ int image_groups(const ConvGeom &g)
 constexpr int kMaxRounds = LCE_MAX_ROUNDS;
 
 struct TileChoice {
-    int tp, tile, ctas_x;
+    int tp, tile, ctas_x, ctas_half;
     double cost;
 };
 
@@ -827,7 +845,7 @@ struct TileChoice {
 // penalty when too few warps share an SM to keep the logic pipe busy.
 template <typename SmemFn>
 bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileChoice *best, int nw = kWarps,
-                 size_t smem_limit = 110 * 1024)
+                 size_t smem_limit = 110 * 1024, bool has_half_block = false)
 {
     int sms = 148;
     {
@@ -846,6 +864,8 @@ bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileC
         const int unit = 4 * nw * tp;
         for (int rounds = 1; rounds <= kMaxRounds; ++rounds) {
             if (forced_rounds && rounds != forced_rounds) continue;
+            // a half channel block takes two units of pixels per step
+            if (has_half_block && (rounds & 1)) continue;
             const int tile = unit * rounds;
             const size_t smem = smem_for_tile(tile);
             if (smem > smem_limit) continue;
@@ -853,18 +873,31 @@ bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileC
             if (per_sm < 1) per_sm = 1;
             if (per_sm > reg_limited_ctas(tp, nw)) per_sm = reg_limited_ctas(tp, nw);
             const int64_t n_tiles = (g.M + tile - 1) / tile;
-            int64_t ctas_x = ((int64_t)sms * per_sm) / chan_blocks;
+            // CTAs per channel block: a half block gets half as many, its tiles cost half as much
+            const int full_blocks = has_half_block ? chan_blocks - 1 : chan_blocks;
+            const int64_t slots = (int64_t)sms * per_sm;
+            int64_t ctas_x = has_half_block ? (2 * slots) / (2 * full_blocks + 1) : slots / chan_blocks;
             if (ctas_x < 1) ctas_x = 1;
             if (ctas_x > n_tiles) ctas_x = n_tiles;
-            const int64_t tiles_per_cta = (n_tiles + ctas_x - 1) / ctas_x;
-            const int64_t ctas_on_sm = (ctas_x * chan_blocks + sms - 1) / sms;
-            const double warps = (double)ctas_x * chan_blocks / sms * nw;
+            int64_t ctas_half = 0;
+            if (has_half_block) {
+                ctas_half = full_blocks > 0 ? (ctas_x + 1) / 2 : ctas_x;
+                if (full_blocks == 0 && ctas_half > slots) ctas_half = slots;
+            }
+            const int64_t total_ctas = ctas_x * full_blocks + ctas_half;
+            double tiles_per_cta = full_blocks > 0 ? (double)((n_tiles + ctas_x - 1) / ctas_x) : 0.0;
+            if (has_half_block) {
+                const double t_half = 0.5 * (double)((n_tiles + ctas_half - 1) / ctas_half);
+                if (t_half > tiles_per_cta) tiles_per_cta = t_half;
+            }
+            const int64_t ctas_on_sm = (total_ctas + sms - 1) / sms;
+            const double warps = (double)total_ctas / sms * nw;
             const double eff = warps >= 16 ? 1.0 : (warps >= 8 ? 0.8 + 0.2 * (warps - 8) / 8 : 0.4 + 0.4 * warps / 8);
             // fewer pixels per thread re-read the weight operands from shared memory more often
             const double smem_penalty = tp == 2 ? 1.06 : (tp == 3 ? 1.02 : 1.0);
             const double cost = (double)ctas_on_sm * tiles_per_cta * (tile * smem_penalty + 4.0) / eff;
             if (best->tile == 0 || cost < best_cost) {
-                best->tile = tile; best->tp = tp; best->ctas_x = (int)ctas_x;
+                best->tile = tile; best->tp = tp; best->ctas_x = (int)ctas_x; best->ctas_half = (int)ctas_half;
                 best_cost = best->cost = cost;
             }
         }
@@ -915,6 +948,7 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
     p.M = (int32_t)g.M;
     p.stride = g.sh;
     p.cw_shift = -1;
+    p.half_block = -1;
     for (int b = 0; b < 16; ++b)
         if ((1 << b) == g.Cw) p.cw_shift = b;
     const int chan_blocks = (g.Cout + kChanPerCta - 1) / kChanPerCta;
@@ -948,29 +982,47 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
     // Eight warps per CTA share one copy of the weight operands and one staging buffer, which
     // measures faster than two CTAs of four warps wherever a whole tile of 32*TP pixels is useful
     // work; CTAs of four warps remain for problems too small to fill such tiles on every SM.
-    int nw = 8;
-    TileChoice c4;
-    // the float-input loader exists for four-warp CTAs only
-    const bool ok8 = in_f32 == nullptr && choose_tile(g, chan_blocks, smem_for, &c, 8, 226 * 1024);
-    const bool ok4 = choose_tile(g, chan_blocks, smem_for, &c4, 4, 110 * 1024) ||
-                     (in_f32 != nullptr && choose_tile(g, chan_blocks, smem_for, &c4, 4, 226 * 1024));
-    if (!ok8 && !ok4) return LCE_ERR_UNSUPPORTED;
-    if (!ok8 || (ok4 && c4.cost < c.cost)) { c = c4; nw = 4; }
+    // candidates: CTAs of 8 or 4 warps, with or without the half-block lane mapping (which needs
+    // tiles of two units and so fewer, larger tiles: not worth it on very small problems)
+    const int tail_channels = g.Cout % kChanPerCta;
+    const bool can_half = tail_channels >= 1 && tail_channels <= kChanPerCta / 2;
+    int nw = 0;
+    bool half = false;
+    c.cost = 0;
+    for (int use_half = can_half ? 1 : 0; use_half >= 0; --use_half) {
+        for (int w = 8; w >= 4; w -= 4) {
+            if (w == 8 && in_f32 != nullptr) continue;  // the float-input loader exists for four-warp CTAs only
+            TileChoice t;
+            bool ok = choose_tile(g, chan_blocks, smem_for, &t, w, w == 8 ? 226 * 1024 : 110 * 1024, use_half != 0);
+            if (!ok && w == 4 && in_f32 != nullptr)
+                ok = choose_tile(g, chan_blocks, smem_for, &t, 4, 226 * 1024, use_half != 0);
+            if (ok && (nw == 0 || t.cost < c.cost)) { c = t; nw = w; half = use_half != 0; }
+        }
+    }
+    if (nw == 0) return LCE_ERR_UNSUPPORTED;
 #ifdef LCE_TUNING
-    if (const char *e = getenv("LCE_NW")) {
-        const int want = atoi(e);
-        if (want == 4 && ok4) { c = c4; nw = 4; }
-        if (want == 8 && ok8) { choose_tile(g, chan_blocks, smem_for, &c, 8, 226 * 1024); nw = 8; }
+    {
+        const char *e_nw = getenv("LCE_NW"), *e_half = getenv("LCE_HALF");
+        if (e_nw || e_half) {
+            const int want_nw = e_nw ? atoi(e_nw) : nw;
+            const bool want_half = e_half ? (atoi(e_half) != 0 && can_half) : half;
+            TileChoice t;
+            if (choose_tile(g, chan_blocks, smem_for, &t, want_nw, 226 * 1024, want_half)) { c = t; nw = want_nw; half = want_half; }
+        }
     }
 #endif
     set_tile(g, &p, c.tile);
     p.n_tiles = (int32_t)((g.M + c.tile - 1) / c.tile);
     const size_t smem_bytes = smem_bytes_for(g, p);
-    dim3 grid((unsigned)c.ctas_x, (unsigned)chan_blocks, 1);
+    p.half_block = half ? chan_blocks - 1 : -1;
+    p.full_blocks = half ? chan_blocks - 1 : chan_blocks;
+    p.ctas_full = c.ctas_x;
+    p.ctas_half = half ? c.ctas_half : 0;
+    dim3 grid((unsigned)(p.full_blocks * p.ctas_full + p.ctas_half), 1, 1);
 #ifdef LCE_TUNING
     if (getenv("LCE_VERBOSE"))
-        fprintf(stderr, "tiled %dx%d M=%lld Cw=%d Cout=%d: nw=%d tp=%d tile=%d n_tiles=%d grid=%dx%d smem=%zu cost=%.0f\n", g.KH, g.KW,
-                (long long)g.M, g.Cw, g.Cout, nw, c.tp, c.tile, p.n_tiles, c.ctas_x, chan_blocks, smem_bytes, c.cost);
+        fprintf(stderr, "tiled %dx%d M=%lld Cw=%d Cout=%d: nw=%d tp=%d tile=%d n_tiles=%d grid=%dx%d+%d smem=%zu cost=%.0f\n", g.KH, g.KW,
+                (long long)g.M, g.Cw, g.Cout, nw, c.tp, c.tile, p.n_tiles, p.ctas_full, p.full_blocks, p.ctas_half, smem_bytes, c.cost);
 #endif
 #define LCE_LAUNCH_TP(KS, ST, NW)                                                   \
     do {                                                                            \

@@ -65,6 +65,41 @@ bitpack_generic_kernel(const float *__restrict__ x, uint32_t *__restrict__ out, 
     }
 }
 
+// Very few channels (an RGB image: C = 3): one word per pixel.  A thread takes four consecutive
+// pixels = 4*C floats = C aligned 128-bit loads, all in flight together, and writes its four words
+// with one 128-bit store.  Rows past the last whole group of four go through the generic kernel.
+template <int C>
+__global__ void __launch_bounds__(kPackThreads)
+bitpack_few_channels_kernel(const float4 *__restrict__ x, uint4 *__restrict__ out, int64_t groups)
+{
+    for (int64_t i = (int64_t)blockIdx.x * kPackThreads + threadIdx.x; i < groups;
+         i += (int64_t)gridDim.x * kPackThreads) {
+        float v[4 * C];
+#pragma unroll
+        for (int q = 0; q < C; ++q) {
+            const float4 f = __ldcs(x + i * C + q);
+            v[4 * q] = f.x; v[4 * q + 1] = f.y; v[4 * q + 2] = f.z; v[4 * q + 3] = f.w;
+        }
+        uint32_t w[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            w[r] = 0u;
+#pragma unroll
+            for (int c = 0; c < C; ++c) w[r] |= (v[r * C + c] < 0.0f ? 1u : 0u) << c;
+        }
+        out[i] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+template <int C>
+void launch_few_channels(const float *x, uint32_t *out, int64_t groups, int max_blocks, cudaStream_t s)
+{
+    int64_t b = (groups + kPackThreads - 1) / kPackThreads;
+    if (b > max_blocks) b = max_blocks;
+    bitpack_few_channels_kernel<C><<<(unsigned)b, kPackThreads, 0, s>>>(reinterpret_cast<const float4 *>(x),
+                                                                       reinterpret_cast<uint4 *>(out), groups);
+}
+
 // LceDequantize: one thread per output float.
 __global__ void __launch_bounds__(kPackThreads)
 unpack_kernel(const uint32_t *__restrict__ in, float *__restrict__ out, int64_t rows, int32_t channels,
@@ -106,6 +141,15 @@ extern "C" lce_status lce_bitpack(const float *x, uint32_t *out, int64_t rows, i
     if (channels % 32 == 0 && aligned(out, 16)) {
         const int64_t passes = (n_words + kWordsPerWarpPass - 1) / kWordsPerWarpPass;
         bitpack_aligned_kernel<<<grid_for(passes, kPackThreads / 32, max_blocks), kPackThreads, 0, s>>>(x, out, n_words);
+    } else if (channels <= 4 && rows >= 4 && aligned(x, 16) && aligned(out, 16)) {
+        const int64_t groups = rows / 4;
+        if (channels == 1) launch_few_channels<1>(x, out, groups, max_blocks * 4, s);
+        else if (channels == 2) launch_few_channels<2>(x, out, groups, max_blocks * 4, s);
+        else if (channels == 3) launch_few_channels<3>(x, out, groups, max_blocks * 4, s);
+        else launch_few_channels<4>(x, out, groups, max_blocks * 4, s);
+        const int64_t done = groups * 4;
+        if (rows > done)
+            bitpack_generic_kernel<<<1, kPackThreads, 0, s>>>(x + done * channels, out + done, rows - done, channels, 1);
     } else {
         bitpack_generic_kernel<<<grid_for(n_words, kPackThreads, max_blocks * 4), kPackThreads, 0, s>>>(
             x, out, rows, channels, words);

@@ -33,7 +33,7 @@ def float_close(got, acc, mult, bias, act=0):
 # ---- LceQuantize / LceDequantize ---------------------------------------------------------
 
 @pytest.mark.parametrize("rows,C", [(1, 1), (7, 3), (50, 31), (33, 32), (129, 33), (1000, 40), (4097, 64), (300, 96),
-                                    (513, 256), (2, 4096), (100003, 3)])
+                                    (513, 256), (2, 4096), (100003, 3), (4099, 1), (1026, 2), (8, 4), (5001, 4), (3, 3)])
 def test_bitpack_matches_oracle(rows, C):
     rng = np.random.default_rng(rows * 131 + C)
     x = rng.standard_normal((rows, C)).astype(np.float32)
@@ -43,6 +43,16 @@ def test_bitpack_matches_oracle(rows, C):
     torch.cuda.synchronize()
     assert guards_intact(whole, 0x5A5A5A5A)
     np.testing.assert_array_equal(words_to_host(out), oracle.bitpack(x))
+
+
+def test_bitpack_few_channels_from_an_unaligned_pointer():
+    # 16-byte alignment decides between the 128-bit few-channel kernel and the generic one
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((1001, 3)).astype(np.float32)
+    buf = torch.zeros(1001 * 3 + 1, dtype=torch.float32, device=DEV)
+    buf[1:] = to_dev(x).flatten()
+    got = words_to_host(lce.lce_bitpack(buf[1:].view(1001, 3)))
+    np.testing.assert_array_equal(got, oracle.bitpack(x))
 
 
 def test_bitpack_one_hot_bit_order():

@@ -33,6 +33,7 @@ bconv_patch_kernel(const PatchParams p)
     uint32_t *sWord = smem;                                             // [cout_pad] weight patch words
     int32_t *sThr = reinterpret_cast<int32_t *>(smem + cout_pad);       // [cout_pad]
     int32_t *sWsum = reinterpret_cast<int32_t *>(smem + 2 * cout_pad);  // [cout_pad][taps], zero-padding only
+    // then [cout_pad] (word, popcount threshold) pairs for the bit-packed fast path
     const uint32_t mask = p.Cin >= 32 ? 0xffffffffu : ((1u << p.Cin) - 1u);
 
     for (int o = threadIdx.x; o < cout_pad; o += kThreads) {
@@ -52,6 +53,56 @@ bconv_patch_kernel(const PatchParams p)
     __syncthreads();
 
     const int K = taps * p.Cin;
+
+    if (p.out_type == LCE_OUT_BITPACKED && p.padding != LCE_PAD_SAME_ZERO) {
+        // Bit-packed output without a zero-padding correction (the stem of a binarized network):
+        // acc < thr  <=>  K - 2*popc < thr  <=>  popc > floor((K - thr) / 2), so a channel is one
+        // 64-bit shared-memory read (weight word, popcount threshold), XOR, POPC, compare, OR.  Two
+        // pixels per thread share that read.
+        __syncthreads();  // sWord / sThr are complete; rewrite them as (word, popcount threshold) pairs
+        uint2 *sPair = reinterpret_cast<uint2 *>(smem + (2 + taps) * cout_pad);
+        for (int o = threadIdx.x; o < cout_pad; o += kThreads) {
+            int32_t t = INT32_MAX;  // pad channels: never set
+            if (o < p.Cout) t = (int32_t)(((int64_t)K - (int64_t)sThr[o]) >> 1);
+            sPair[o] = make_uint2(sWord[o], (uint32_t)t);
+        }
+        __syncthreads();
+        const int64_t stride = (int64_t)gridDim.x * kThreads;
+        for (int64_t m0 = (int64_t)blockIdx.x * kThreads + threadIdx.x; m0 < p.M; m0 += 2 * stride) {
+            const int64_t mm[2] = {m0, m0 + stride};
+            uint32_t patch[2] = {0u, 0u};
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                if (mm[q] >= p.M) continue;
+                const int m = (int)mm[q];
+                const int r = m / p.OW, ow = m - r * p.OW;
+                const int n = r / p.OH, oh = r - n * p.OH;
+                const int iy0 = oh * p.sh - p.pt, ix0 = ow * p.sw - p.pl;
+                const uint32_t *img = p.in + (int64_t)n * p.H * p.W;
+                for (int ky = 0; ky < p.KH; ++ky) {
+                    const int iy = iy0 + ky;
+                    for (int kx = 0; kx < p.KW; ++kx) {
+                        const int ix = ix0 + kx;
+                        if (iy >= 0 && iy < p.H && ix >= 0 && ix < p.W)
+                            patch[q] |= (__ldg(img + iy * p.W + ix) & mask) << ((ky * p.KW + kx) * p.Cin);
+                    }
+                }
+            }
+            for (int wd = 0; wd < p.Cow; ++wd) {
+                uint32_t bits0 = 0u, bits1 = 0u;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const uint2 wt = sPair[wd * 32 + j];
+                    if ((int32_t)__popc(patch[0] ^ wt.x) > (int32_t)wt.y) bits0 |= 1u << j;
+                    if ((int32_t)__popc(patch[1] ^ wt.x) > (int32_t)wt.y) bits1 |= 1u << j;
+                }
+                static_cast<uint32_t *>(p.out)[mm[0] * p.Cow + wd] = bits0;
+                if (mm[1] < p.M) static_cast<uint32_t *>(p.out)[mm[1] * p.Cow + wd] = bits1;
+            }
+        }
+        return;
+    }
+
     for (int m = blockIdx.x * kThreads + threadIdx.x; m < p.M; m += gridDim.x * kThreads) {
         const int r = m / p.OW, ow = m - r * p.OW;
         const int n = r / p.OH, oh = r - n * p.OH;
@@ -116,10 +167,12 @@ lce_status launch_bconv_patch(const ConvGeom &g, const uint32_t *in, const uint3
     p.N = g.N; p.H = g.H; p.W = g.W; p.Cin = g.Cin; p.Cout = g.Cout; p.Cow = g.Cow;
     p.KH = g.KH; p.KW = g.KW; p.sh = g.sh; p.sw = g.sw; p.OH = g.OH; p.OW = g.OW; p.pt = g.pt; p.pl = g.pl;
     p.M = (int32_t)g.M; p.padding = g.padding; p.out_type = g.out_type; p.activation = g.activation;
-    const size_t smem = (size_t)g.Cow * 32 * (2 + g.KH * g.KW) * 4;
+    const size_t smem = (size_t)g.Cow * 32 * (4 + g.KH * g.KW) * 4;
     if (smem > 48 * 1024) return LCE_ERR_UNSUPPORTED;
+    // one wave of resident blocks (8 x 256 threads per SM), grid-stride beyond that: every block pays
+    // for building the weight words in shared memory, so fewer, longer-lived blocks are cheaper
     int64_t blocks = (g.M + kThreads - 1) / kThreads;
-    if (blocks > 148 * 8 * 8) blocks = 148 * 8 * 8;  // grid-stride beyond 8 waves of 8 blocks per SM
+    if (blocks > 148 * 8) blocks = 148 * 8;
     bconv_patch_kernel<<<(unsigned)blocks, kThreads, smem, s>>>(p);
     return launch_status();
 }

@@ -551,6 +551,175 @@ bconv3x3_tensor_kernel(const TensorParams p)
     }
 }
 
+
+// RESIDENT schedule with the worker roles split over two warp groups, so that the expansion of
+// tile t+1, the MMAs of tile t and the output transform of tile t-1 run at the same time (a kernel
+// that allocates TMEM is given one CTA per SM, so the overlap has to come from inside the CTA):
+// warps 0-7 "loaders" (prefetch + expand the input tile), warps 8-15 "finishers" (read the
+// accumulators, output transform), warp 16 issues MMAs.  Barriers as above; full_d[s] is awaited by
+// both groups (the loaders reuse A buffer s only after the MMAs that read it are done).
+constexpr int kSplitThreads = 2 * kWorkers + 32;
+
+__global__ void __launch_bounds__(kSplitThreads, 1)
+bconv3x3_tensor_split_kernel(const TensorParams p)
+{
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    uint2 *table = reinterpret_cast<uint2 *>(smem_raw);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + 2048);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_raw + 2048 + 96);
+    float *sMult = reinterpret_cast<float *>(smem_raw + 2048 + 128);
+    float *sBias = sMult + p.n_blk;
+    int32_t *sThr = reinterpret_cast<int32_t *>(sBias + p.n_blk);
+    uint2 *offs = reinterpret_cast<uint2 *>(sThr + p.n_blk);
+    uint32_t *raw0 = reinterpret_cast<uint32_t *>(offs + ((9 * p.Cw + 1) / 2) * 2);
+    const int raw_words = ((p.P * p.Cw + 3) / 4) * 4;
+    uint8_t *sB = reinterpret_cast<uint8_t *>(raw0 + 2 * raw_words);
+    const size_t b_tap_bytes = (size_t)2 * p.Cw * p.n_blk * 16;
+    uint8_t *sA0 = sB + 9 * b_tap_bytes;
+    const size_t a_bytes = (size_t)2 * p.Cw * p.P * 16;
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int ch0 = blockIdx.y * p.n_blk;
+
+    for (int e = tid; e < 256; e += kSplitThreads) {
+        uint32_t lo = 0, hi = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            lo |= (((e >> j) & 1) ? 0xFFu : 0x01u) << (8 * j);
+            hi |= (((e >> (j + 4)) & 1) ? 0xFFu : 0x01u) << (8 * j);
+        }
+        table[e] = make_uint2(lo, hi);
+    }
+    for (int e = tid; e < p.n_blk; e += kSplitThreads) {
+        const bool ok = ch0 + e < p.Cout;
+        sMult[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.mult + ch0 + e) : 0.f;
+        sBias[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.bias + ch0 + e) : 0.f;
+        sThr[e] = (ok && p.out_type == LCE_OUT_BITPACKED) ? __ldg(p.thr + ch0 + e) : INT32_MIN;
+    }
+    for (int e = tid; e < 9 * p.Cw; e += kSplitThreads) {
+        const int tap = e / p.Cw, cw = e - tap * p.Cw;
+        const uint32_t a_off = (uint32_t)((tap / 3) * p.Wp + (tap % 3) + 2 * cw * p.P);
+        const uint32_t b_off = (uint32_t)(2 * cw * p.n_blk) + (uint32_t)(tap * 2 * p.Cw * p.n_blk);
+        offs[e] = make_uint2(a_off, b_off);
+    }
+    if (tid == 0) {
+        mbar_init(&bars[BAR_FULL_A0], kWorkers);
+        mbar_init(&bars[BAR_FULL_A1], kWorkers);
+        mbar_init(&bars[BAR_FULL_D0], 1);
+        mbar_init(&bars[BAR_FULL_D1], 1);
+        mbar_init(&bars[BAR_EMPTY_D0], kWorkers);
+        mbar_init(&bars[BAR_EMPTY_D1], kWorkers);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"((uint32_t)p.tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_blk >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+    const uint32_t b_saddr = smem_u32(sB);
+    const uint32_t desc_hi = 8u | (1u << 14);
+    const int words_per_tap = p.n_blk * p.Cw;
+    const int first_tile = blockIdx.x, tile_step = gridDim.x;
+    bool ok = true;
+
+    if (tid >= 2 * kWorkers) {
+        // ---- MMA issuer: one lane -------------------------------------------------------------
+        if (tid == 2 * kWorkers) {
+            uint32_t par_full_a[2] = {0, 0}, par_empty_d[2] = {0, 0};
+            for (int tile = first_tile, it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+                const int sbuf = it & 1;
+                ok = mbar_wait_bounded(&bars[BAR_FULL_A0 + sbuf], par_full_a[sbuf]);
+                par_full_a[sbuf] ^= 1u;
+                if (ok && it >= 2) {  // the accumulator buffer must have been read out
+                    ok = mbar_wait_bounded(&bars[BAR_EMPTY_D0 + sbuf], par_empty_d[sbuf]);
+                    par_empty_d[sbuf] ^= 1u;
+                }
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tmem_d = tmem_base + (uint32_t)(sbuf * p.n_blk);
+                const uint32_t a_lo0 = (smem_u32(sA0 + sbuf * a_bytes) >> 4) | ((uint32_t)p.P << 16);
+                uint32_t accumulate = 0;
+                issue_mmas(tmem_d, offs, 0, 9 * p.Cw, a_lo0, (b_saddr >> 4) | ((uint32_t)p.n_blk << 16), desc_hi, idesc, accumulate);
+                mma_commit(&bars[BAR_FULL_D0 + sbuf]);
+            }
+        }
+    } else {
+        // ---- both worker groups expand the resident weights, then part ways ----------------------
+        if (tid < kWorkers && first_tile < p.n_tiles) prefetch_raw(p, first_tile * kTileM, raw0, tid);
+        for (int e0 = tid; e0 < 9 * words_per_tap; e0 += 2 * kWorkers * 8) {
+            uint32_t wv[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int e = e0 + k * 2 * kWorkers;
+                const int ch = e & (p.n_blk - 1), tc = e >> p.n_blk_log2;  // tc = tap*Cw + cw
+                const int tap = tc / p.Cw, cw = tc - tap * p.Cw;
+                wv[k] = (e < 9 * words_per_tap && ch0 + ch < p.Cout) ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + tap) * p.Cw + cw) : 0u;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int e = e0 + k * 2 * kWorkers;
+                if (e < 9 * words_per_tap) {
+                    const int ch = e & (p.n_blk - 1), tc = e >> p.n_blk_log2;
+                    const int tap = tc / p.Cw, cw = tc - tap * p.Cw;
+                    uint4 lo, hi;
+                    expand_word(table, wv[k], &lo, &hi);
+                    uint4 *dst = reinterpret_cast<uint4 *>(sB + tap * b_tap_bytes) + (size_t)(2 * cw) * p.n_blk + ch;
+                    dst[0] = lo;
+                    dst[p.n_blk] = hi;
+                }
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(2 * kWorkers) : "memory");  // weights complete before any full_a arrival
+
+        uint32_t par_full_d[2] = {0, 0};
+        if (tid < kWorkers) {
+            // ---- loaders ---------------------------------------------------------------------------
+            int tile = first_tile;
+            for (int it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+                const int sbuf = it & 1;
+                if (it >= 2) {  // A buffer sbuf was read by the MMAs of tile it-2
+                    ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + sbuf], par_full_d[sbuf]);
+                    par_full_d[sbuf] ^= 1u;
+                    if (!ok) break;
+                }
+                expand_a(p, table, raw0 + sbuf * raw_words, sA0 + sbuf * a_bytes, tid);
+                const int next = tile + tile_step;
+                if (next < p.n_tiles) prefetch_raw(p, next * kTileM, raw0 + (sbuf ^ 1) * raw_words, tid);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(&bars[BAR_FULL_A0 + sbuf]);
+            }
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        } else {
+            // ---- finishers -------------------------------------------------------------------------
+            const int ftid = tid - kWorkers;
+            int tile = first_tile;
+            for (int it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+                const int sbuf = it & 1;
+                ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + sbuf], par_full_d[sbuf]);
+                par_full_d[sbuf] ^= 1u;
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                epilogue(p, tmem_base + (uint32_t)(sbuf * p.n_blk), tile * kTileM, ch0, sMult, sBias, sThr, ftid);
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                mbar_arrive(&bars[BAR_EMPTY_D0 + sbuf]);
+            }
+        }
+    }
+    if (!ok) g_tensor_status = 1;
+
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+    }
+}
+
 }  // namespace
 
 bool tensor_covers(const ConvGeom &g)
@@ -622,28 +791,35 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const uint
     int cols = 32;
     while (cols < (resident ? 2 * n_blk : n_blk)) cols *= 2;
     p.tmem_cols = cols;
-    // no more CTAs per SM than the 512 TMEM columns can serve: pad the request if need be
-    const int tmem_ctas = 512 / cols;
-    if ((227 * 1024) / (smem + 1024) > (size_t)tmem_ctas) smem = (size_t)(227 * 1024) / tmem_ctas - 1024;
     const int n_blocks = (g.Cout + n_blk - 1) / n_blk;
-    auto kernel = resident ? bconv3x3_tensor_kernel<true> : bconv3x3_tensor_kernel<false>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return LCE_ERR_CUDA;
-    // ask for the largest shared-memory carve-out, or a second CTA per SM may not be allowed
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess)
-        return LCE_ERR_CUDA;
-    // persistent grid: exactly as many CTAs as can be resident at once (registers, shared memory
-    // and TMEM columns all count)
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, smem) != cudaSuccess) return LCE_ERR_CUDA;
-    if (per_sm < 1) return LCE_ERR_UNSUPPORTED;
-    if (per_sm > tmem_ctas) per_sm = tmem_ctas;
-    int ctas_x = (sms * per_sm) / n_blocks;
+    // Persistent grid.  A kernel that allocates TMEM is given one CTA per SM (the occupancy query
+    // reports 1 for any such kernel, whatever its registers and shared memory), so the grid is one
+    // CTA per SM.  The shared-memory carve-out is left to the driver: forcing the largest one leaves
+    // no L1 for the streaming schedule's weight loads (measured: 24 -> 19 us at 14x14x256).
+    int ctas_x = sms / n_blocks;
     if (ctas_x < 1) ctas_x = 1;
     if (ctas_x > p.n_tiles) ctas_x = p.n_tiles;
+    const dim3 grid((unsigned)ctas_x, (unsigned)n_blocks);
+    bool split = resident;
 #ifdef LCE_TUNING
-    if (getenv("LCE_VERBOSE")) fprintf(stderr, "tensor: resident=%d n_blk=%d smem=%zu occ=%d ctas_x=%d n_blocks=%d tiles=%d\n", (int)resident, n_blk, smem, per_sm, ctas_x, n_blocks, p.n_tiles);
+    if (const char *e = getenv("LCE_TENSOR_SPLIT")) split = resident && atoi(e) != 0;
+    if (getenv("LCE_VERBOSE"))
+        fprintf(stderr, "tensor: resident=%d split=%d n_blk=%d smem=%zu ctas_x=%d n_blocks=%d tiles=%d\n", (int)resident, (int)split, n_blk,
+                smem, ctas_x, n_blocks, p.n_tiles);
 #endif
-    kernel<<<dim3((unsigned)ctas_x, (unsigned)n_blocks), kThreads, smem, s>>>(p);
+    if (split) {
+        if (cudaFuncSetAttribute(bconv3x3_tensor_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return LCE_ERR_CUDA;
+        bconv3x3_tensor_split_kernel<<<grid, kSplitThreads, smem, s>>>(p);
+    } else if (resident) {
+        if (cudaFuncSetAttribute(bconv3x3_tensor_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return LCE_ERR_CUDA;
+        bconv3x3_tensor_kernel<true><<<grid, kThreads, smem, s>>>(p);
+    } else {
+        if (cudaFuncSetAttribute(bconv3x3_tensor_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return LCE_ERR_CUDA;
+        bconv3x3_tensor_kernel<false><<<grid, kThreads, smem, s>>>(p);
+    }
     return launch_status();
 }
 

@@ -21,6 +21,8 @@
 #include <stdio.h>
 #include <stdlib.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "csa.cuh"
 
@@ -38,6 +40,11 @@ constexpr int kChanPerThread = 8;
 constexpr int kChanGroups = kChanPerCta / kChanPerThread;
 constexpr int kWRow = 12;           // 9 carry-save operand words per (channel word, channel) + 3 pad
 constexpr int kWGroupStride = kChanPerThread * kWRow + 4;  // +4 words: the 8 channel groups hit distinct banks
+#ifdef LCE_NO_TAIL
+constexpr bool kTailStep = false;
+#else
+constexpr bool kTailStep = true;
+#endif
 constexpr int kMaxTaps = 25;                               // 5x5 is the largest tiled filter
 constexpr int kWsumWords = kChanPerCta * kMaxTaps;         // per-tap weight sums of a channel block
 
@@ -59,6 +66,7 @@ struct TiledParams {
     int32_t cw_shift;     // log2(Cw) when Cw is a power of two, else -1
     int32_t half_block;   // KxK kernel: index of the channel block with at most 32 real channels, or -1
     int32_t full_blocks, ctas_full, ctas_half;  // KxK kernel: 1-D grid = full_blocks x ctas_full CTAs, then ctas_half
+    int32_t range_full, range_half;             // KxK kernel: flat output pixels per CTA of a full / the half block
     int32_t stride;       // pointwise kernel only
     int32_t n9, rem3, cwp; // pointwise kernel: nine-word groups, leftover triples, padded words per pixel
     int32_t padding, out_type, activation;
@@ -393,16 +401,19 @@ bconv3x3_kernel(const TiledParams p)
     const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
     // 1-D grid: ctas_full CTAs for each full channel block, then ctas_half for the half block
-    int block_y, block_x, ctas_x;
+    // Every CTA of a channel block owns one contiguous range of flat output pixels.
+    int block_y, block_x, range;
     if ((int)blockIdx.x < p.full_blocks * p.ctas_full) {
         block_y = blockIdx.x % p.full_blocks;
         block_x = blockIdx.x / p.full_blocks;
-        ctas_x = p.ctas_full;
+        range = p.range_full;
     } else {
         block_y = p.full_blocks;
         block_x = blockIdx.x - p.full_blocks * p.ctas_full;
-        ctas_x = p.ctas_half;
+        range = p.range_half;
     }
+    const int r_begin = block_x * range;                 // host: (CTAs - 1) * range < M
+    const int r_end = min(r_begin + range, p.M);
     const int ch0 = block_y * kChanPerCta;
     const int plane_words = p.Cw * p.plane;  // one input buffer; two of them alternate between tiles
 
@@ -454,24 +465,21 @@ bconv3x3_kernel(const TiledParams p)
     asm volatile("" : "+r"(k124.one), "+r"(k124.two), "+r"(k124.four));
     const uint32_t w_saddr0 = (uint32_t)__cvta_generic_to_shared(sW + cg * kWGroupStride);
 
-    // ---- persistent loop over this CTA's pixel tiles; the next tile's input rows are copied into
-    // the other buffer while the current tile is computed --------------------------------------
-    int tile = block_x;
-    if (tile < p.n_tiles)
-        stage_rows<KS, STRIDE, NW, F32>(p, tile * p.tile_pixels, min((tile + 1) * p.tile_pixels, p.M), sA0, warp, lane);
+    // ---- loop over the tiles of this CTA's range; the next tile's input rows are copied into the
+    // other buffer while the current tile is computed ---------------------------------------------
+    if (r_begin < r_end)
+        stage_rows<KS, STRIDE, NW, F32>(p, r_begin, min(r_begin + p.tile_pixels, r_end), sA0, warp, lane);
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
 
-  for (int buf = 0; tile < p.n_tiles; tile += ctas_x, buf ^= 1) {
+  for (int m0 = r_begin, buf = 0; m0 < r_end; m0 += p.tile_pixels, buf ^= 1) {
     const uint32_t *sA = sA0 + buf * plane_words;
-    const int m0 = tile * p.tile_pixels;
-    const int m_end = min(m0 + p.tile_pixels, p.M);
+    const int m_end = min(m0 + p.tile_pixels, r_end);
     {
-        const int next = tile + ctas_x;
-        if (next < p.n_tiles)
-            stage_rows<KS, STRIDE, NW, F32>(p, next * p.tile_pixels, min((next + 1) * p.tile_pixels, p.M),
-                               sA0 + (buf ^ 1) * plane_words, warp, lane);
+        const int next = m0 + p.tile_pixels;
+        if (next < r_end)
+            stage_rows<KS, STRIDE, NW, F32>(p, next, min(next + p.tile_pixels, r_end), sA0 + (buf ^ 1) * plane_words, warp, lane);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
     const int r_first = m0 / p.OW;
@@ -490,10 +498,14 @@ bconv3x3_kernel(const TiledParams p)
     }
     const int a_base_first = (m0 - r_first * p.OW) * STRIDE;  // the tile's first pixel sits in virtual row 0
 
-    for (int base = m0; base < m0 + p.tile_pixels; base += pix_per_step * TP) {
-        int a_base[TP];
+    // One step: every thread works on TPX pixels x 8 channels.  TPX = TP everywhere except at the
+    // end of the CTA's range, where a remainder of at most two pixels per thread takes the TPX = 2
+    // form of the same code: the work of all CTAs is then equal to within 2 x pix_per_step pixels.
+    auto step = [&](auto tpx_tag, const int base) {
+        constexpr int TPX = decltype(tpx_tag)::value;
+        int a_base[TPX];
 #pragma unroll
-        for (int i = 0; i < TP; ++i) {
+        for (int i = 0; i < TPX; ++i) {
             // pixels past the end of the tile redo the tile's first pixel and store nothing
             a_base[i] = (m_next < m_end) ? (voh - v_first) * p.pitch + ow * STRIDE : a_base_first;
             m_next += pix_per_step;
@@ -504,9 +516,9 @@ bconv3x3_kernel(const TiledParams p)
                 else { --oh_left; voh += STRIDE; }
             }
         }
-        uint32_t acc[TP][kChanPerThread];
+        uint32_t acc[TPX][kChanPerThread];
 #pragma unroll
-        for (int i = 0; i < TP; ++i)
+        for (int i = 0; i < TPX; ++i)
 #pragma unroll
             for (int j = 0; j < kChanPerThread; ++j) acc[i][j] = 0u;
 
@@ -517,9 +529,9 @@ bconv3x3_kernel(const TiledParams p)
             for (int g = 0; g < kNG; ++g) {
                 // activation-side operands of nine-word group g: taps 9g .. 9g+8 in (ky, kx) order;
                 // taps past the filter's last one are zero words on both sides and count nothing
-                Triple at[TP][3];
+                Triple at[TPX][3];
 #pragma unroll
-                for (int i = 0; i < TP; ++i)
+                for (int i = 0; i < TPX; ++i)
 #pragma unroll
                     for (int k = 0; k < 3; ++k) {
                         uint32_t v[3];
@@ -530,7 +542,7 @@ bconv3x3_kernel(const TiledParams p)
                         }
                         at[i][k] = make_triple(v[0], v[1], v[2]);
                     }
-                ChannelLoop<0, TP>::run(w_saddr, at, k124, acc);
+                ChannelLoop<0, TPX>::run(w_saddr, at, k124, acc);
                 w_saddr += kChanGroups * kWGroupStride * 4;
             }
             plane += p.plane;
@@ -540,7 +552,7 @@ bconv3x3_kernel(const TiledParams p)
         ChannelParams cp;
         load_channel_params(p, chan, cp);
 #pragma unroll
-        for (int i = 0; i < TP; ++i) {
+        for (int i = 0; i < TPX; ++i) {
             const int m = base + i * pix_per_step + warp * pix_per_warp + px;
             const bool pix_ok = m < m_end;
             int32_t v[kChanPerThread];
@@ -561,6 +573,15 @@ bconv3x3_kernel(const TiledParams p)
                 }
             }
             store_outputs(p, v, cp, m, pix_ok, cg, ch0, chan);
+        }
+    };
+    for (int base = m0; base < m_end;) {
+        if (kTailStep && TP > 2 && m_end - base <= 2 * pix_per_step) {
+            step(std::integral_constant<int, 2>{}, base);
+            base += 2 * pix_per_step;
+        } else {
+            step(std::integral_constant<int, TP>{}, base);
+            base += TP * pix_per_step;
         }
     }
     // the next tile's rows have landed, and every warp is done reading this tile's
@@ -830,12 +851,12 @@ int image_groups(const ConvGeom &g)
 }
 
 #ifndef LCE_MAX_ROUNDS
-#define LCE_MAX_ROUNDS 2
+#define LCE_MAX_ROUNDS 8
 #endif
 constexpr int kMaxRounds = LCE_MAX_ROUNDS;
 
 struct TileChoice {
-    int tp, tile, ctas_x, ctas_half;
+    int tp, tile, ctas_x, ctas_half, range_full, range_half;
     double cost;
 };
 
@@ -845,7 +866,7 @@ struct TileChoice {
 // penalty when too few warps share an SM to keep the logic pipe busy.
 template <typename SmemFn>
 bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileChoice *best, int nw = kWarps,
-                 size_t smem_limit = 110 * 1024, bool has_half_block = false)
+                 size_t smem_limit = 110 * 1024, bool has_half_block = false, bool ranged = false)
 {
     int sms = 148;
     {
@@ -872,32 +893,59 @@ bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileC
             int per_sm = (int)((220 * 1024) / (smem + 1024));
             if (per_sm < 1) per_sm = 1;
             if (per_sm > reg_limited_ctas(tp, nw)) per_sm = reg_limited_ctas(tp, nw);
-            const int64_t n_tiles = (g.M + tile - 1) / tile;
-            // CTAs per channel block: a half block gets half as many, its tiles cost half as much
+            const double smem_penalty[5] = {0, 0, 1.06, 1.02, 1.0};  // fewer pixels per thread re-read the weight operands more often
             const int full_blocks = has_half_block ? chan_blocks - 1 : chan_blocks;
             const int64_t slots = (int64_t)sms * per_sm;
-            int64_t ctas_x = has_half_block ? (2 * slots) / (2 * full_blocks + 1) : slots / chan_blocks;
-            if (ctas_x < 1) ctas_x = 1;
-            if (ctas_x > n_tiles) ctas_x = n_tiles;
-            int64_t ctas_half = 0;
-            if (has_half_block) {
-                ctas_half = full_blocks > 0 ? (ctas_x + 1) / 2 : ctas_x;
-                if (full_blocks == 0 && ctas_half > slots) ctas_half = slots;
+            int64_t ctas_x, ctas_half = 0, range_full = 0, range_half = 0;
+            double t_cta;  // time of the busiest CTA, in pixel-steps of a full block
+            if (ranged) {
+                // KxK kernel: a CTA owns a contiguous range of pixels, a whole number of granules; a
+                // granule is the smallest step the kernel has (2 pixels per thread when TP > 2)
+                const bool tail = kTailStep && tp > 2;
+                const int64_t pps = 4 * nw;                     // pixels per step and pixel-per-thread, full block
+                const int64_t granule = tail ? pps : unit;      // ranges are whole numbers of granules
+                // per tile: barrier bubbles and the halo rows that are staged again (measured at
+                // 56x56x64: about a fifth of the time of computing those rows)
+                const double tile_overhead = 4.0 + 0.2 * (g.KH - 1) * g.OW;
+                auto range_for = [&](int64_t ctas, int64_t gran) { return ((g.M + ctas - 1) / ctas + gran - 1) / gran * gran; };
+                auto time_of = [&](int64_t range, int pixel_scale) {  // pixel_scale 2: a half block's step covers twice the pixels
+                    double t = (double)((range + tile - 1) / tile) * tile_overhead;
+                    for (int64_t r = range / pixel_scale; r > 0;) {  // the kernel's own decomposition into steps
+                        if (tail && r <= 2 * pps) { t += 2 * pps * smem_penalty[2]; r = 0; }
+                        else { t += unit * smem_penalty[tp]; r -= unit; }
+                    }
+                    return t;
+                };
+                ctas_x = has_half_block ? (2 * slots) / (2 * full_blocks + 1) : slots / chan_blocks;
+                if (ctas_x < 1) ctas_x = 1;
+                t_cta = 0;
+                if (full_blocks > 0) {
+                    range_full = range_for(ctas_x, granule);
+                    ctas_x = (g.M + range_full - 1) / range_full;
+                    t_cta = time_of(range_full, 1);
+                }
+                if (has_half_block) {
+                    ctas_half = full_blocks > 0 ? (ctas_x + 1) / 2 : (slots < 1 ? 1 : slots);
+                    range_half = range_for(ctas_half, 2 * granule);
+                    ctas_half = (g.M + range_half - 1) / range_half;
+                    const double t_half = time_of(range_half, 2);
+                    if (t_half > t_cta) t_cta = t_half;
+                }
+            } else {
+                const int64_t n_tiles = (g.M + tile - 1) / tile;
+                ctas_x = slots / chan_blocks;
+                if (ctas_x < 1) ctas_x = 1;
+                if (ctas_x > n_tiles) ctas_x = n_tiles;
+                t_cta = (double)((n_tiles + ctas_x - 1) / ctas_x) * (tile * smem_penalty[tp] + 4.0);
             }
             const int64_t total_ctas = ctas_x * full_blocks + ctas_half;
-            double tiles_per_cta = full_blocks > 0 ? (double)((n_tiles + ctas_x - 1) / ctas_x) : 0.0;
-            if (has_half_block) {
-                const double t_half = 0.5 * (double)((n_tiles + ctas_half - 1) / ctas_half);
-                if (t_half > tiles_per_cta) tiles_per_cta = t_half;
-            }
             const int64_t ctas_on_sm = (total_ctas + sms - 1) / sms;
             const double warps = (double)total_ctas / sms * nw;
             const double eff = warps >= 16 ? 1.0 : (warps >= 8 ? 0.8 + 0.2 * (warps - 8) / 8 : 0.4 + 0.4 * warps / 8);
-            // fewer pixels per thread re-read the weight operands from shared memory more often
-            const double smem_penalty = tp == 2 ? 1.06 : (tp == 3 ? 1.02 : 1.0);
-            const double cost = (double)ctas_on_sm * tiles_per_cta * (tile * smem_penalty + 4.0) / eff;
+            const double cost = (double)ctas_on_sm * t_cta / eff;
             if (best->tile == 0 || cost < best_cost) {
                 best->tile = tile; best->tp = tp; best->ctas_x = (int)ctas_x; best->ctas_half = (int)ctas_half;
+                best->range_full = (int)range_full; best->range_half = (int)range_half;
                 best_cost = best->cost = cost;
             }
         }
@@ -993,9 +1041,9 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
         for (int w = 8; w >= 4; w -= 4) {
             if (w == 8 && in_f32 != nullptr) continue;  // the float-input loader exists for four-warp CTAs only
             TileChoice t;
-            bool ok = choose_tile(g, chan_blocks, smem_for, &t, w, w == 8 ? 226 * 1024 : 110 * 1024, use_half != 0);
+            bool ok = choose_tile(g, chan_blocks, smem_for, &t, w, w == 8 ? 226 * 1024 : 110 * 1024, use_half != 0, true);
             if (!ok && w == 4 && in_f32 != nullptr)
-                ok = choose_tile(g, chan_blocks, smem_for, &t, 4, 226 * 1024, use_half != 0);
+                ok = choose_tile(g, chan_blocks, smem_for, &t, 4, 226 * 1024, use_half != 0, true);
             if (ok && (nw == 0 || t.cost < c.cost)) { c = t; nw = w; half = use_half != 0; }
         }
     }
@@ -1007,7 +1055,7 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
             const int want_nw = e_nw ? atoi(e_nw) : nw;
             const bool want_half = e_half ? (atoi(e_half) != 0 && can_half) : half;
             TileChoice t;
-            if (choose_tile(g, chan_blocks, smem_for, &t, want_nw, 226 * 1024, want_half)) { c = t; nw = want_nw; half = want_half; }
+            if (choose_tile(g, chan_blocks, smem_for, &t, want_nw, 226 * 1024, want_half, true)) { c = t; nw = want_nw; half = want_half; }
         }
     }
 #endif
@@ -1018,11 +1066,13 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
     p.full_blocks = half ? chan_blocks - 1 : chan_blocks;
     p.ctas_full = c.ctas_x;
     p.ctas_half = half ? c.ctas_half : 0;
+    p.range_full = c.range_full;
+    p.range_half = c.range_half;
     dim3 grid((unsigned)(p.full_blocks * p.ctas_full + p.ctas_half), 1, 1);
 #ifdef LCE_TUNING
     if (getenv("LCE_VERBOSE"))
-        fprintf(stderr, "tiled %dx%d M=%lld Cw=%d Cout=%d: nw=%d tp=%d tile=%d n_tiles=%d grid=%dx%d+%d smem=%zu cost=%.0f\n", g.KH, g.KW,
-                (long long)g.M, g.Cw, g.Cout, nw, c.tp, c.tile, p.n_tiles, p.ctas_full, p.full_blocks, p.ctas_half, smem_bytes, c.cost);
+        fprintf(stderr, "tiled %dx%d M=%lld Cw=%d Cout=%d: nw=%d tp=%d tile=%d n_tiles=%d grid=%dx%d+%d range=%d/%d smem=%zu cost=%.0f\n", g.KH, g.KW,
+                (long long)g.M, g.Cw, g.Cout, nw, c.tp, c.tile, p.n_tiles, p.ctas_full, p.full_blocks, p.ctas_half, p.range_full, p.range_half, smem_bytes, c.cost);
 #endif
 #define LCE_LAUNCH_TP(KS, ST, NW)                                                   \
     do {                                                                            \

@@ -1,22 +1,27 @@
-// LceBConv2d, tiled XOR/POPC kernel for 3x3 filters (paper Section 3.2: im2col -> BGEMM -> output
-// transform, here as one implicit-GEMM kernel: the im2col matrix is never materialised and the
-// accumulators never leave registers before the output transform).
+// LceBConv2d, tiled XOR/POPC kernels for 3x3 and 5x5 filters (and, further down, 1x1) (paper
+// Section 3.2: im2col -> BGEMM -> output transform, here as one implicit-GEMM kernel: the im2col
+// matrix is never materialised and the accumulators never leave registers before the output
+// transform).
 //
 // Stride 1 or 2, any channel counts and image sizes:
-//   * a CTA owns a run of consecutive output pixels (flat (n, oh, ow) order) times 64 output
-//     channels; a warp works on 4 pixels x 8 channel groups at a time, a thread on TP pixels
-//     (16 apart in the flat order) x 8 channels, i.e. TP x 8 accumulators in registers;
-//   * the CTA first copies the packed input rows its pixels need into shared memory, one plane
-//     per channel word, in "padded image" coordinates: rows/columns outside the image hold zero
-//     words, which is exactly the paper's one-padding (a zero bit is +1.0);
+//   * a CTA of 8 (or 4) warps owns one contiguous range of output pixels (flat (n, oh, ow) order)
+//     times 64 output channels; a warp works on 4 pixels x 8 channel groups at a time (8 x 4 in a
+//     channel block that has at most 32 channels), a thread on TP pixels x 8 channels, i.e. TP x 8
+//     accumulators in registers.  All ranges are equal to within two pixels per thread: the last step
+//     of a range runs the two-pixel form of the same code;
+//   * the CTA copies the packed input rows its pixels need into shared memory, a tile of up to
+//     8 x 32 x TP pixels at a time (the next tile while the current one is computed), one plane per
+//     channel word, in "padded image" coordinates: rows/columns outside the image hold zero words,
+//     which is exactly the paper's one-padding (a zero bit is +1.0);
 //   * the weights of its 64 channels arrive as carry-save operands (csa.cuh): either copied in
 //     16-byte pieces from a buffer prepared once by lce_bconv2d_pack_weights (the paper's
 //     load-time "weight packing"), or derived on the fly from the plain packed weights;
-//   * for every channel word the nine taps of a (pixel, channel) pair form one nine-word
-//     carry-save group: 16 LOP3 + 4 POPC + 4 IMAD instead of 9 XOR + 9 POPC + 9 adds.  The
-//     activation-side operands of the thread's TP pixels sit in registers for the whole channel
-//     word; the weight-side operands of one channel are read from shared memory once and used
-//     for all TP pixels (shared-memory bandwidth, not issue slots, is what this ordering saves);
+//   * for every channel word nine taps of a (pixel, channel) pair form one nine-word carry-save
+//     group (a 5x5 filter is three groups, the last two words zero): 16 LOP3 + 4 POPC + 4 IMAD
+//     instead of 9 XOR + 9 POPC + 9 adds.  The activation-side operands of the thread's TP pixels
+//     sit in registers for the whole group; the weight-side operands of one channel are read from
+//     shared memory once and used for all TP pixels (shared-memory bandwidth, not issue slots, is
+//     what this ordering saves);
 //   * epilogue: acc = K - 2*count, then float multiply-add, threshold + bit-pack, or raw int32.
 #include <stdio.h>
 #include <stdlib.h>

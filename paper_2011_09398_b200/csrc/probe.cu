@@ -173,6 +173,102 @@ probe_mma_b1_kernel(const uint32_t *__restrict__ seed, uint32_t *__restrict__ si
     if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
 }
 
+// Do the integer pipes and the legacy 1-bit warp MMA run side by side?  Even warps run the
+// nine-word carry-save loop (mix 3), odd warps the AND+POPC MMA loop (mix 21), in the same CTA at
+// the same time; each group times itself.  cycles[2*block] = logic group, [2*block+1] = MMA group.
+template <int MODE>  // 0: both groups, 1: the logic group alone (odd warps idle), 2: the MMA group alone
+__global__ void __launch_bounds__(kThreads, 2)
+probe_combined_kernel(const uint32_t *__restrict__ seed, uint32_t *__restrict__ sink, long long *__restrict__ cycles,
+                      int iterations)
+{
+    __shared__ __align__(16) uint32_t tile[1024 + 64];
+    for (int i = threadIdx.x; i < 1024 + 64; i += kThreads) tile[i] = seed[i & 1023];
+    __syncthreads();
+    const int warp = threadIdx.x >> 5;
+    uint32_t x = 0;
+    if ((warp & 1) == 0) {
+        if (MODE == 2) return;
+        // as in the convolution kernel: 4 pixels x 8 channels per thread, activation operands in
+        // registers, each channel's weight operands read from shared memory once per group
+        constexpr int TPX = 4;
+        Weights124 k124;
+        k124.one = iterations > 0 ? 1u : seed[0];
+        k124.two = iterations > 0 ? 2u : seed[1];
+        k124.four = iterations > 0 ? 4u : seed[2];
+        asm volatile("" : "+r"(k124.one), "+r"(k124.two), "+r"(k124.four));
+        uint32_t acc[TPX][CH];
+#pragma unroll
+        for (int p = 0; p < TPX; ++p)
+#pragma unroll
+            for (int j = 0; j < CH; ++j) acc[p][j] = 0;
+        const int base = (threadIdx.x >> 3) * 2;
+        const uint32_t *wrow = tile + (threadIdx.x & 7) * 100;  // 8 channels x 12 words, as the kernel's layout
+        const int its = iterations * 115 / 100;  // 288 word operations per iteration against the MMA group's 256 pairs
+        const long long t0 = clock64();
+        for (int it = 0; it < its; ++it) {
+            const uint32_t *row = tile + ((base + it * 11) & 1023);
+            Triple at[TPX][3];
+#pragma unroll
+            for (int p = 0; p < TPX; ++p)
+#pragma unroll
+                for (int g = 0; g < 3; ++g) at[p][g] = make_triple(row[p * 9 + 3 * g], row[p * 9 + 3 * g + 1], row[p * 9 + 3 * g + 2]);
+#pragma unroll
+            for (int j = 0; j < CH; ++j) {
+                const uint4 q0 = *reinterpret_cast<const uint4 *>(wrow + j * 12);
+                const uint4 q1 = *reinterpret_cast<const uint4 *>(wrow + j * 12 + 4);
+                const uint32_t q2 = wrow[j * 12 + 8];
+                Triple wt[3];
+                wt[0].all = q0.x; wt[0].pair = q0.y; wt[0].first = q0.z;
+                wt[1].all = q0.w; wt[1].pair = q1.x; wt[1].first = q1.y;
+                wt[2].all = q1.z; wt[2].pair = q1.w; wt[2].first = q2;
+                if (j == 0) popc9_mad_pixels<TPX, CH, 0>(at, wt, k124, acc);
+                if (j == 1) popc9_mad_pixels<TPX, CH, 1>(at, wt, k124, acc);
+                if (j == 2) popc9_mad_pixels<TPX, CH, 2>(at, wt, k124, acc);
+                if (j == 3) popc9_mad_pixels<TPX, CH, 3>(at, wt, k124, acc);
+                if (j == 4) popc9_mad_pixels<TPX, CH, 4>(at, wt, k124, acc);
+                if (j == 5) popc9_mad_pixels<TPX, CH, 5>(at, wt, k124, acc);
+                if (j == 6) popc9_mad_pixels<TPX, CH, 6>(at, wt, k124, acc);
+                if (j == 7) popc9_mad_pixels<TPX, CH, 7>(at, wt, k124, acc);
+            }
+        }
+        const long long t1 = clock64();
+#pragma unroll
+        for (int p = 0; p < TPX; ++p)
+#pragma unroll
+            for (int j = 0; j < CH; ++j) x ^= acc[p][j];
+        if (threadIdx.x == 0) cycles[2 * blockIdx.x] = t1 - t0;
+    } else {
+        if (MODE == 1) return;
+        uint32_t a[4], b[2];
+        int32_t d[8][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) a[i] = seed[(threadIdx.x * 4 + i) & 1023];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) b[i] = seed[(threadIdx.x * 2 + i + 300) & 1023];
+#pragma unroll
+        for (int t = 0; t < 8; ++t)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) d[t][i] = 0;
+        const long long t0 = clock64();
+        for (int it = 0; it < iterations; ++it) {
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+                asm volatile(
+                    "mma.sync.aligned.m16n8k256.row.col.s32.b1.b1.s32.and.popc {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                    "{%0,%1,%2,%3};"
+                    : "+r"(d[t][0]), "+r"(d[t][1]), "+r"(d[t][2]), "+r"(d[t][3])
+                    : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+        }
+        const long long t1 = clock64();
+#pragma unroll
+        for (int t = 0; t < 8; ++t)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) x ^= (uint32_t)d[t][i];
+        if (threadIdx.x == 32) cycles[2 * blockIdx.x + 1] = t1 - t0;
+    }
+    sink[(size_t)blockIdx.x * kThreads + threadIdx.x] = x;
+}
+
 }  // namespace
 }  // namespace lce
 
@@ -187,6 +283,8 @@ extern "C" lce_status lce_probe_pipe(int32_t mix, int32_t iterations, double *op
         case 10: case 11: case 13: case 14: case 15: ops_per_thread_iter = 64; break;
         case 12: ops_per_thread_iter = 128; break;            // two adds per step
         case 20: case 21: ops_per_thread_iter = 8 * 1024.0 / 32; break;  // 8 MMAs x 16*8*256/32 word pairs per warp
+        case 30: case 32: ops_per_thread_iter = 4 * CH * 9 * 1.15; break;  // logic group of the combined probe (half the warps)
+        case 31: case 33: ops_per_thread_iter = 8 * 1024.0 / 32; break;    // MMA group of the combined probe (half the warps)
         default: return LCE_ERR_INVALID_ARG;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -207,6 +305,9 @@ extern "C" lce_status lce_probe_pipe(int32_t mix, int32_t iterations, double *op
         case 14: fn = probe_unit_kernel<14>; break;
         case 15: fn = probe_unit_kernel<15>; break;
         case 20: fn = probe_mma_b1_kernel<false>; break;
+        case 30: case 31: fn = probe_combined_kernel<0>; break;
+        case 32: fn = probe_combined_kernel<1>; break;
+        case 33: fn = probe_combined_kernel<2>; break;
         default: fn = probe_mma_b1_kernel<true>; break;
     }
     // one wave exactly: as many blocks per SM as the kernel's registers let be resident
@@ -226,7 +327,7 @@ extern "C" lce_status lce_probe_pipe(int32_t mix, int32_t iterations, double *op
     do {
         if (cudaMalloc(&seed, sizeof(host_seed)) != cudaSuccess) break;
         if (cudaMalloc(&sink, (size_t)blocks * kThreads * 4) != cudaSuccess) break;
-        if (cudaMalloc(&cycles, (size_t)blocks * 8) != cudaSuccess) break;
+        if (cudaMalloc(&cycles, (size_t)blocks * 16) != cudaSuccess) break;
         if (cudaMemcpyAsync(seed, host_seed, sizeof(host_seed), cudaMemcpyHostToDevice, s) != cudaSuccess) break;
         if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) break;
         for (int rep = 0; rep < 2; ++rep) {  // first repetition warms up
@@ -238,15 +339,25 @@ extern "C" lce_status lce_probe_pipe(int32_t mix, int32_t iterations, double *op
         if (cudaGetLastError() != cudaSuccess) break;
         float ms = 0.f;
         if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess || ms <= 0.f) break;
-        host_cycles = new long long[blocks];
-        if (cudaMemcpy(host_cycles, cycles, (size_t)blocks * 8, cudaMemcpyDeviceToHost) != cudaSuccess) break;
+        host_cycles = new long long[2 * blocks];
+        if (cudaMemcpy(host_cycles, cycles, (size_t)blocks * 16, cudaMemcpyDeviceToHost) != cudaSuccess) break;
+        const bool combined = mix >= 30;
         double mean_cycles = 0;
-        for (int i = 0; i < blocks; ++i) mean_cycles += (double)host_cycles[i];
+        for (int i = 0; i < blocks; ++i) mean_cycles += (double)host_cycles[combined ? 2 * i + ((mix - 30) & 1) : i];
         mean_cycles /= blocks;
         const double per_thread = ops_per_thread_iter * (double)iterations;
-        const double total = per_thread * (double)blocks * kThreads;
-        *ops_per_second = total / (ms * 1e-3);
-        *ops_per_clock_per_sm = per_thread * kThreads * blocks_per_sm / mean_cycles;
+        // combined probe: the group is half the threads, and its rate per second is taken from its own
+        // cycle count at the clock the whole launch ran at (the groups need not end together)
+        const double threads = combined ? kThreads / 2 : kThreads;
+        const double total = per_thread * (double)blocks * threads;
+        *ops_per_clock_per_sm = per_thread * threads * blocks_per_sm / mean_cycles;
+        if (combined) {
+            int khz = 0;
+            if (cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev) != cudaSuccess) break;
+            *ops_per_second = *ops_per_clock_per_sm * sms * (double)khz * 1e3;  // at the maximum SM clock
+        } else {
+            *ops_per_second = total / (ms * 1e-3);
+        }
         st = LCE_OK;
     } while (0);
     delete[] host_cycles;

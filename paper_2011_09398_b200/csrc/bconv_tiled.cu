@@ -871,7 +871,7 @@ struct TileChoice {
 // penalty when too few warps share an SM to keep the logic pipe busy.
 template <typename SmemFn>
 bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileChoice *best, int nw = kWarps,
-                 size_t smem_limit = 110 * 1024, bool has_half_block = false, bool ranged = false)
+                 size_t smem_limit = 110 * 1024, bool has_half_block = false, bool ranged = false, bool allow_tp1 = false)
 {
     int sms = 148;
     {
@@ -885,7 +885,9 @@ bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileC
 #endif
     double best_cost = 0;
     best->tile = 0;
-    for (int tp = 2; tp <= 4; ++tp) {
+    // one pixel per thread exists for the KxK kernel with 4-warp CTAs only: the finest split of a
+    // single image over the SMs (latency, not throughput)
+    for (int tp = (ranged && nw == 4 && allow_tp1) ? 1 : 2; tp <= 4; ++tp) {
         if (forced_tp && tp != forced_tp) continue;
         const int unit = 4 * nw * tp;
         for (int rounds = 1; rounds <= kMaxRounds; ++rounds) {
@@ -898,7 +900,7 @@ bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileC
             int per_sm = (int)((220 * 1024) / (smem + 1024));
             if (per_sm < 1) per_sm = 1;
             if (per_sm > reg_limited_ctas(tp, nw)) per_sm = reg_limited_ctas(tp, nw);
-            const double smem_penalty[5] = {0, 0, 1.06, 1.02, 1.0};  // fewer pixels per thread re-read the weight operands more often
+            const double smem_penalty[5] = {0, 1.2, 1.06, 1.02, 1.0};  // fewer pixels per thread re-read the weight operands more often
             const int full_blocks = has_half_block ? chan_blocks - 1 : chan_blocks;
             const int64_t slots = (int64_t)sms * per_sm;
             int64_t ctas_x, ctas_half = 0, range_full = 0, range_half = 0;
@@ -1046,7 +1048,7 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
         for (int w = 8; w >= 4; w -= 4) {
             if (w == 8 && in_f32 != nullptr) continue;  // the float-input loader exists for four-warp CTAs only
             TileChoice t;
-            bool ok = choose_tile(g, chan_blocks, smem_for, &t, w, w == 8 ? 226 * 1024 : 110 * 1024, use_half != 0, true);
+            bool ok = choose_tile(g, chan_blocks, smem_for, &t, w, w == 8 ? 226 * 1024 : 110 * 1024, use_half != 0, true, in_f32 == nullptr);
             if (!ok && w == 4 && in_f32 != nullptr)
                 ok = choose_tile(g, chan_blocks, smem_for, &t, 4, 226 * 1024, use_half != 0, true);
             if (ok && (nw == 0 || t.cost < c.cost)) { c = t; nw = w; half = use_half != 0; }
@@ -1060,7 +1062,7 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
             const int want_nw = e_nw ? atoi(e_nw) : nw;
             const bool want_half = e_half ? (atoi(e_half) != 0 && can_half) : half;
             TileChoice t;
-            if (choose_tile(g, chan_blocks, smem_for, &t, want_nw, 226 * 1024, want_half, true)) { c = t; nw = want_nw; half = want_half; }
+            if (choose_tile(g, chan_blocks, smem_for, &t, want_nw, 226 * 1024, want_half, true, in_f32 == nullptr)) { c = t; nw = want_nw; half = want_half; }
         }
     }
 #endif
@@ -1081,6 +1083,7 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
 #endif
 #define LCE_LAUNCH_TP(KS, ST, NW)                                                   \
     do {                                                                            \
+        if (c.tp == 1) return launch_kxk<KS, ST, 1, 4>(p, smem_bytes, grid, s);     \
         if (c.tp == 2) return launch_kxk<KS, ST, 2, NW>(p, smem_bytes, grid, s);    \
         if (c.tp == 3) return launch_kxk<KS, ST, 3, NW>(p, smem_bytes, grid, s);    \
         return launch_kxk<KS, ST, 4, NW>(p, smem_bytes, grid, s);                   \

@@ -293,24 +293,30 @@ def run_lce(args):
     images_per_s = world * len(layers) * BATCH / (ms_per_step * 1e-3)
 
     # ---- end-to-end leg: the host-buffer C-ABI entry point, copies inside the timed region ---------
+    # Every step copies each layer's inputs in from pinned host memory, runs the kernel and copies the
+    # result back, through lce_bconv2d_host_async on two streams (layers alternate, each with its own
+    # workspace), so that one layer's copy back overlaps the next layer's copies in and kernel; the
+    # step ends when both streams are synchronised, i.e. when all eight results are in host memory.
+    host_streams = [torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)]
+
     def step_host():
-        for layer in layers:
+        for j, layer in enumerate(layers):
             h = layer["host"]
-            lce.lce_bconv2d_host(h["desc"], h["a"], h["w"], h["mult"], h["bias"], h["thr"], h["out"], h["ws"])
+            with torch.cuda.stream(host_streams[j % 2]):
+                lce.lce_bconv2d_host_async(h["desc"], h["a"], h["w"], h["mult"], h["bias"], h["thr"], h["out"], h["ws"])
+        for st in host_streams:
+            st.synchronize()
 
     for _ in range(2):
         step_host()
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2e_steps = max(3, min(args.steps, 10))
     t0 = time.perf_counter()
-    e0.record()
     for _ in range(e2e_steps):
         step_host()
-    e1.record()
     barrier()
     e2e_wall = time.perf_counter() - t0
-    e2e_ms = max(e0.elapsed_time(e1), 1e3 * e2e_wall) / e2e_steps  # host-synchronous calls: wall clock is the honest one
+    e2e_ms = 1e3 * e2e_wall / e2e_steps  # every step ends with a host synchronisation: wall clock is the honest one
     e2e_ms = max_over_ranks(e2e_ms, world, dev)
     e2e_value = whole_job_value(macs_per_step, world, e2e_ms)
 
@@ -347,7 +353,7 @@ def run_lce(args):
                    "l2": "flushed between steps by a 256 MiB write", "launch": "one CUDA graph replay per step"},
         "images_per_second": images_per_s,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_ms, "api": "lce_bconv2d_host (pinned host buffers, plain weights)"},
+                "ms_per_step": e2e_ms, "api": "lce_bconv2d_host_async on two streams, synchronised every step (pinned host buffers, plain weights)"},
         "gpu_launches": args.steps * len(layers),
         "clocks": clocks, "roofline": roofline, "per_layer": per_layer, "wall_s_timed_region": wall,
     }

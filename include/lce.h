@@ -166,6 +166,15 @@ lce_status lce_bconv2d_host(const lce_bconv2d_desc *desc, const uint32_t *input,
                             const float *multiplier, const float *bias, const int32_t *thresholds,
                             void *output, void *workspace, size_t workspace_bytes, void *stream);
 
+/* lce_bconv2d_host without the final synchronisation: the copies and the kernel are only enqueued on
+ * `stream`.  Host buffers must be pinned for the copies to be asynchronous, and all buffers
+ * (`output` and `workspace` included) belong to the call until the caller has synchronised `stream`;
+ * calls on different streams with different workspaces overlap (one layer's copy back with the next
+ * layer's copies in and kernel). */
+lce_status lce_bconv2d_host_async(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
+                                  const float *multiplier, const float *bias, const int32_t *thresholds,
+                                  void *output, void *workspace, size_t workspace_bytes, void *stream);
+
 /* (No counterpart in the paper.)  lce_bconv2d_host for callers that cannot allocate device memory:
  * a process whose allocator is off limits (a real-time loop, a sandboxed plug-in that only ever
  * sees host tensors) has no way to produce the `workspace` argument above.  This form keeps the

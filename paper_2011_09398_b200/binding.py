@@ -57,6 +57,8 @@ def library() -> ctypes.CDLL:
         lib.lce_bconv2d_host_workspace_bytes.restype = ctypes.c_size_t
         lib.lce_bconv2d_host_workspace_bytes.argtypes = [ctypes.POINTER(BConv2dDesc)]
         lib.lce_bconv2d_host.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        lib.lce_bconv2d_host_async.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        lib.lce_bconv2d_host_async.restype = ctypes.c_int
         lib.lce_bconv2d_host_noalloc_max_bytes.restype = ctypes.c_size_t
         lib.lce_bconv2d_host_noalloc_max_bytes.argtypes = []
         lib.lce_bconv2d_host_noalloc.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp]
@@ -238,6 +240,17 @@ def lce_bconv2d_host(desc: BConv2dDesc, input, weights, multiplier, bias, thresh
         _host(multiplier, torch.float32, "multiplier"), _host(bias, torch.float32, "bias"),
         _host(thresholds, torch.int32, "thresholds"), _host(out, out_dtype, "out"),
         _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()), "lce_bconv2d_host")
+
+
+def lce_bconv2d_host_async(desc: BConv2dDesc, input, weights, multiplier, bias, thresholds, out, workspace: torch.Tensor) -> None:
+    """lce_bconv2d_host that only enqueues its copies and kernel on the current stream; the caller
+    synchronises the stream before touching `out` (or reusing `workspace`)."""
+    out_dtype = torch.float32 if desc.out_type == OUT_FLOAT32 else torch.int32
+    _check(library().lce_bconv2d_host_async(
+        ctypes.byref(desc), _host(input, torch.int32, "input"), _host(weights, torch.int32, "weights"),
+        _host(multiplier, torch.float32, "multiplier"), _host(bias, torch.float32, "bias"),
+        _host(thresholds, torch.int32, "thresholds"), _host(out, out_dtype, "out"),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()), "lce_bconv2d_host_async")
 
 
 def lce_bconv2d_host_noalloc_max_bytes() -> int:

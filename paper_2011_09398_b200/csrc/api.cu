@@ -200,11 +200,12 @@ extern "C" size_t lce_bconv2d_host_workspace_bytes(const lce_bconv2d_desc *desc)
     return lce::host_layout(g).total;
 }
 
-extern "C" lce_status lce_bconv2d_host(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
-                                       const float *multiplier, const float *bias, const int32_t *thresholds,
-                                       void *output, void *workspace, size_t workspace_bytes, void *stream)
+namespace lce {
+namespace {
+lce_status host_conv(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights, const float *multiplier,
+                     const float *bias, const int32_t *thresholds, void *output, void *workspace, size_t workspace_bytes,
+                     void *stream, bool synchronise)
 {
-    using namespace lce;
     ConvGeom g;
     lce_status st = check_conv_args(desc, &g, input, weights, multiplier, bias, thresholds, output);
     if (st != LCE_OK) return st;
@@ -226,8 +227,24 @@ extern "C" lce_status lce_bconv2d_host(const lce_bconv2d_desc *desc, const uint3
                   thresholds ? reinterpret_cast<const int32_t *>(ws + L.thr) : nullptr, ws + L.out, s);
     if (st != LCE_OK) return st;
     if (cudaMemcpyAsync(output, ws + L.out, L.out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return LCE_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) return LCE_ERR_CUDA;
+    if (synchronise && cudaStreamSynchronize(s) != cudaSuccess) return LCE_ERR_CUDA;
     return LCE_OK;
+}
+}  // namespace
+}  // namespace lce
+
+extern "C" lce_status lce_bconv2d_host(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
+                                       const float *multiplier, const float *bias, const int32_t *thresholds,
+                                       void *output, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return lce::host_conv(desc, input, weights, multiplier, bias, thresholds, output, workspace, workspace_bytes, stream, true);
+}
+
+extern "C" lce_status lce_bconv2d_host_async(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
+                                             const float *multiplier, const float *bias, const int32_t *thresholds,
+                                             void *output, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return lce::host_conv(desc, input, weights, multiplier, bias, thresholds, output, workspace, workspace_bytes, stream, false);
 }
 
 // ---- host-buffer convolution that allocates nothing ---------------------------------------------

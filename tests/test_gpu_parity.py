@@ -303,3 +303,36 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     with pytest.raises(lce.LceError) as e:
         lce.lce_bconv2d_host(desc, h_in, h_w, None, None, h_thr, h_out, ws[:1024])
     assert e.value.status == 6
+
+
+def test_async_host_entry_point_on_two_streams_matches_oracle():
+    # two layers in flight on two streams, each with its own workspace; results read after synchronising
+    jobs = []
+    streams = [torch.cuda.Stream(device=DEV), torch.cuda.Stream(device=DEV)]
+    for j, base in enumerate((wl.config2_specs()[0], wl.config2_specs()[3])):  # float 56x56x64, bits 28x28x128
+        spec = wl.with_batch(base, 2)
+        t = wl.conv_tensors(2, 1 + 4 * j, spec)
+        x = wl.activations(2, j, (spec.batch, spec.in_h, spec.in_w, spec.in_c))
+        desc = lce.make_desc(spec.batch, spec.in_h, spec.in_w, spec.in_c, spec.out_c, out_type=spec.out_type)
+        ws = torch.empty(lce.lce_bconv2d_host_workspace_bytes(desc), dtype=torch.uint8, device=DEV)
+        h_in = torch.from_numpy(oracle.bitpack(x).view(np.int32)).pin_memory()
+        h_w = torch.from_numpy(oracle.bitpack_pm1(t.w_pm1).view(np.int32)).pin_memory()
+        is_f = spec.out_type == wl.OUT_FLOAT32
+        last = spec.out_c if is_f else (spec.out_c + 31) // 32
+        h_out = torch.empty((spec.batch, spec.out_h, spec.out_w, last), dtype=torch.float32 if is_f else torch.int32).pin_memory()
+        h_m = torch.from_numpy(t.multiplier).pin_memory() if is_f else None
+        h_b = torch.from_numpy(t.bias).pin_memory() if is_f else None
+        h_t = None if is_f else torch.from_numpy(t.thresholds).pin_memory()
+        jobs.append((spec, t, x, desc, ws, h_in, h_w, h_m, h_b, h_t, h_out))
+    torch.cuda.synchronize()
+    for j, (spec, t, x, desc, ws, h_in, h_w, h_m, h_b, h_t, h_out) in enumerate(jobs):
+        with torch.cuda.stream(streams[j]):
+            lce.lce_bconv2d_host_async(desc, h_in, h_w, h_m, h_b, h_t, h_out, ws)
+    for s in streams:
+        s.synchronize()
+    for spec, t, x, desc, ws, h_in, h_w, h_m, h_b, h_t, h_out in jobs:
+        acc = oracle.bconv2d_acc(oracle.sign(x), t.w_pm1, (1, 1), spec.padding)
+        if spec.out_type == wl.OUT_FLOAT32:
+            assert float_close(h_out.numpy(), acc, t.multiplier, t.bias) == 0
+        else:
+            np.testing.assert_array_equal(h_out.numpy().view(np.uint32), oracle.transform_bits(acc, t.thresholds))

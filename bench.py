@@ -360,7 +360,8 @@ def run_lce(args):
     if world == 1 and not args.no_chains:
         line["chains"] = time_chains(dev)
         line["tensor_core_path"] = time_tensor_path(dev, layers)
-        line["paper_sweep"] = time_paper_sweep(dev)
+        if not args.no_sweep:
+            line["paper_sweep"] = time_paper_sweep(dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cores = len(os.sched_getaffinity(0))
         sample_batch, passes = BATCH, 2
@@ -515,6 +516,7 @@ def main():
     ap.add_argument("--impl", default="lce", choices=["lce", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-chains", action="store_true", help="skip the config 4 / config 5 chain timings")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the paper's 48-layer convolution sweep")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -121,7 +121,7 @@ lce_status lce_bconv2d(const lce_bconv2d_desc *desc, const uint32_t *input, cons
  *   residual   fp32 [batch][oh][ow][out_c] or NULL       out_float fp32 same shape, or NULL
  *   out_packed uint32 [batch][oh][ow][ceil(out_c/32)] or NULL   (at least one output required)
  * The results are bit-identical to lce_bconv2d -> lce_add_f32 -> lce_bitpack run one after the
- * other.  Only shapes the tiled kernels cover (3x3 stride 1-2, 1x1) are accepted; others return
+ * other.  Only shapes the tiled kernels cover (3x3 and 5x5 with equal strides of 1 or 2, 1x1) are accepted; others return
  * LCE_ERR_UNSUPPORTED. */
 lce_status lce_bconv2d_fused(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
                              const float *multiplier, const float *bias, const float *residual,
@@ -141,6 +141,28 @@ lce_status lce_bconv2d_fused(const lce_bconv2d_desc *desc, const uint32_t *input
 lce_status lce_bconv2d_f32(const lce_bconv2d_desc *desc, const float *input, const uint32_t *weights,
                            const float *multiplier, const float *bias, const int32_t *thresholds,
                            void *output, void *stream);
+
+/* Which kernel lce_bconv2d would launch for this descriptor, and with what shape: host arithmetic
+ * only, nothing is launched and no GPU is needed (without one the plan is made for 148 SMs).  The
+ * paper's engine picks its kernel and tiling per layer when the model is loaded (Section 3.1); this
+ * is that choice made visible.  Fields that do not apply to the chosen kernel are 0.
+ *   kernel              LCE_KERNEL_DIRECT, LCE_KERNEL_TILED or LCE_KERNEL_TENSOR (the one-word patch
+ *                       kernel for very few input channels reports LCE_KERNEL_TILED with patch = 1)
+ *   pointwise           1 for the 1x1 tiled kernel
+ *   warps_per_cta, pixels_per_thread, tile_pixels, shared_bytes      the variant of the tiled kernel
+ *   ctas                CTAs of the launch; ctas_half_block of them work on the last, at most
+ *                       32-channel block with the 8-pixel x 4-group lane mapping
+ *   pixels_per_cta      flat output pixels each CTA of a full channel block owns (KxK kernel);
+ *                       pixels_per_cta_half_block the same for the half block
+ * Output buffers are assumed 16-byte aligned.  Errors: INVALID_ARG; UNSUPPORTED when desc->kernel
+ * forces a kernel that does not cover the shape. */
+typedef struct lce_bconv2d_plan_info {
+    int32_t kernel, patch, pointwise;
+    int32_t warps_per_cta, pixels_per_thread, tile_pixels;
+    int32_t ctas, ctas_half_block, pixels_per_cta, pixels_per_cta_half_block;
+    int64_t shared_bytes;
+} lce_bconv2d_plan_info;
+lce_status lce_bconv2d_plan(const lce_bconv2d_desc *desc, lce_bconv2d_plan_info *plan);
 
 /* Load-time weight packing (Section 3.2: the paper's BGEMM also re-arranges the weights ahead of
  * time for its access pattern; Section 3.1: weights are converted once, when the model is built).  Rewrites

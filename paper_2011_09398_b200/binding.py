@@ -192,6 +192,22 @@ def lce_bconv2d_f32(desc: BConv2dDesc, input: torch.Tensor, weights: torch.Tenso
     return out
 
 
+class BConv2dPlanInfo(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("kernel", "patch", "pointwise", "warps_per_cta", "pixels_per_thread", "tile_pixels",
+                                               "ctas", "ctas_half_block", "pixels_per_cta", "pixels_per_cta_half_block")] + \
+               [("shared_bytes", ctypes.c_int64)]
+
+
+def lce_bconv2d_plan(desc: BConv2dDesc) -> dict:
+    """The kernel and launch shape lce_bconv2d would use for `desc` (host arithmetic only)."""
+    info = BConv2dPlanInfo()
+    fn = library().lce_bconv2d_plan
+    fn.argtypes = [ctypes.POINTER(BConv2dDesc), ctypes.POINTER(BConv2dPlanInfo)]
+    fn.restype = ctypes.c_int
+    _check(fn(ctypes.byref(desc), ctypes.byref(info)), "lce_bconv2d_plan")
+    return {n: getattr(info, n) for n, _ in BConv2dPlanInfo._fields_}
+
+
 def lce_bconv2d_fused(desc: BConv2dDesc, input, weights, multiplier, bias, residual=None, out_float=None,
                       out_packed=None) -> None:
     """LceBConv2d (float output) with the shortcut add and/or the next LceQuantize fused in; the

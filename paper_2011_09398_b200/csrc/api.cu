@@ -108,6 +108,39 @@ extern "C" lce_status lce_bconv2d_out_shape(const lce_bconv2d_desc *desc, int32_
     return LCE_OK;
 }
 
+extern "C" lce_status lce_bconv2d_plan(const lce_bconv2d_desc *desc, lce_bconv2d_plan_info *plan)
+{
+    using namespace lce;
+    ConvGeom g;
+    lce_status st = make_geom(desc, &g);
+    if (st != LCE_OK) return st;
+    if (!plan) return LCE_ERR_INVALID_ARG;
+    *plan = lce_bconv2d_plan_info{};
+    // the same order of preference as dispatch()
+    if (desc->kernel == LCE_KERNEL_DIRECT) { plan->kernel = LCE_KERNEL_DIRECT; return LCE_OK; }
+    if (desc->kernel == LCE_KERNEL_TENSOR) {
+        if (!tensor_covers(g)) return LCE_ERR_UNSUPPORTED;
+        plan->kernel = LCE_KERNEL_TENSOR;
+        return LCE_OK;
+    }
+    if (patch_covers(g)) { plan->kernel = LCE_KERNEL_TILED; plan->patch = 1; return LCE_OK; }
+    TiledPlanInfo info{};
+    st = tiled_plan_info(g, &info);
+    if (st == LCE_ERR_UNSUPPORTED && desc->kernel == LCE_KERNEL_AUTO) { plan->kernel = LCE_KERNEL_DIRECT; return LCE_OK; }
+    if (st != LCE_OK) return st;
+    plan->kernel = LCE_KERNEL_TILED;
+    plan->pointwise = info.pointwise;
+    plan->warps_per_cta = info.warps_per_cta;
+    plan->pixels_per_thread = info.pixels_per_thread;
+    plan->tile_pixels = info.tile_pixels;
+    plan->ctas = info.ctas;
+    plan->ctas_half_block = info.ctas_half_block;
+    plan->pixels_per_cta = info.pixels_per_cta;
+    plan->pixels_per_cta_half_block = info.pixels_per_cta_half_block;
+    plan->shared_bytes = info.shared_bytes;
+    return LCE_OK;
+}
+
 extern "C" lce_status lce_bconv2d(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
                                   const float *multiplier, const float *bias, const int32_t *thresholds,
                                   void *output, void *stream)

@@ -984,19 +984,20 @@ lce_status launch_pack_weights_tiled(const ConvGeom &g, const uint32_t *w, uint3
     return launch_status();
 }
 
-lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const uint32_t *w_image,
-                              const float *mult, const float *bias, const int32_t *thr, void *out, cudaStream_t s,
-                              const float *residual, uint32_t *out_packed, const float *in_f32)
+// Everything the launch needs that does not depend on the buffers: geometry fields of the kernel
+// parameters, the chosen variant and the launch dimensions.
+struct TiledPlan {
+    bool pointwise;
+    int nw, tp;
+    size_t smem_bytes;
+    dim3 grid;
+};
+
+static lce_status plan_tiled(const ConvGeom &g, bool f32_input, TiledParams *pp, TiledPlan *plan)
 {
+    TiledParams &p = *pp;
     if (!tiled_covers(g)) return LCE_ERR_UNSUPPORTED;
-    if (in_f32 && !covers3x3(g)) return LCE_ERR_UNSUPPORTED;
-    // 128-bit epilogue accesses need 16-byte aligned buffers when the channel count allows them
-    if ((g.Cout & 3) == 0 && g.out_type != LCE_OUT_BITPACKED && (!aligned(out, 16) || !aligned(residual, 16)))
-        return LCE_ERR_UNSUPPORTED;
-    if (w_image && !aligned(w_image, 16)) return LCE_ERR_ALIGNMENT;
-    TiledParams p{};
-    p.in = in; p.w = w; p.w_image = w_image; p.mult = mult; p.bias = bias; p.thr = thr; p.out = out;
-    p.residual = residual; p.out_packed = out_packed; p.in_f32 = in_f32;
+    if (f32_input && !covers3x3(g)) return LCE_ERR_UNSUPPORTED;
     p.N = g.N; p.H = g.H; p.W = g.W; p.Cin = g.Cin; p.Cw = g.Cw; p.Cout = g.Cout; p.Cow = g.Cow;
     p.OH = g.OH; p.OW = g.OW; p.pt = g.pt; p.pl = g.pl;
     p.padding = g.padding; p.out_type = g.out_type; p.activation = g.activation;
@@ -1019,11 +1020,12 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
         if (!choose_tile(g, chan_blocks, smem_for, &c)) return LCE_ERR_UNSUPPORTED;
         p.tile_pixels = c.tile;
         p.n_tiles = (int32_t)((g.M + c.tile - 1) / c.tile);
-        dim3 grid((unsigned)c.ctas_x, (unsigned)chan_blocks, 1);
-        const size_t smem_bytes = smem_for(c.tile);
-        if (c.tp == 2) return launch1x1<2>(p, smem_bytes, grid, s);
-        if (c.tp == 3) return launch1x1<3>(p, smem_bytes, grid, s);
-        return launch1x1<4>(p, smem_bytes, grid, s);
+        plan->pointwise = true;
+        plan->nw = kWarps;
+        plan->tp = c.tp;
+        plan->grid = dim3((unsigned)c.ctas_x, (unsigned)chan_blocks, 1);
+        plan->smem_bytes = smem_for(c.tile);
+        return LCE_OK;
     }
 
     p.Hp = (g.OH - 1) * g.sh + g.KH;
@@ -1034,11 +1036,10 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
         set_tile(g, &p, tile);
         return smem_bytes_for(g, p);
     };
-    // Eight warps per CTA share one copy of the weight operands and one staging buffer, which
-    // measures faster than two CTAs of four warps wherever a whole tile of 32*TP pixels is useful
-    // work; CTAs of four warps remain for problems too small to fill such tiles on every SM.
-    // candidates: CTAs of 8 or 4 warps, with or without the half-block lane mapping (which needs
-    // tiles of two units and so fewer, larger tiles: not worth it on very small problems)
+    // Candidates: CTAs of 8 or 4 warps (eight warps share one copy of the weight operands and one
+    // staging buffer, which measures faster wherever whole tiles of 32*TP pixels are useful work;
+    // four-warp CTAs remain for problems too small for that), with or without the half-block lane
+    // mapping (which needs tiles of two units: not worth it on very small problems).
     const int tail_channels = g.Cout % kChanPerCta;
     const bool can_half = tail_channels >= 1 && tail_channels <= kChanPerCta / 2;
     int nw = 0;
@@ -1046,10 +1047,10 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
     c.cost = 0;
     for (int use_half = can_half ? 1 : 0; use_half >= 0; --use_half) {
         for (int w = 8; w >= 4; w -= 4) {
-            if (w == 8 && in_f32 != nullptr) continue;  // the float-input loader exists for four-warp CTAs only
+            if (w == 8 && f32_input) continue;  // the float-input loader exists for four-warp CTAs only
             TileChoice t;
-            bool ok = choose_tile(g, chan_blocks, smem_for, &t, w, w == 8 ? 226 * 1024 : 110 * 1024, use_half != 0, true, in_f32 == nullptr);
-            if (!ok && w == 4 && in_f32 != nullptr)
+            bool ok = choose_tile(g, chan_blocks, smem_for, &t, w, w == 8 ? 226 * 1024 : 110 * 1024, use_half != 0, true, !f32_input);
+            if (!ok && w == 4 && f32_input)
                 ok = choose_tile(g, chan_blocks, smem_for, &t, 4, 226 * 1024, use_half != 0, true);
             if (ok && (nw == 0 || t.cost < c.cost)) { c = t; nw = w; half = use_half != 0; }
         }
@@ -1062,25 +1063,73 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
             const int want_nw = e_nw ? atoi(e_nw) : nw;
             const bool want_half = e_half ? (atoi(e_half) != 0 && can_half) : half;
             TileChoice t;
-            if (choose_tile(g, chan_blocks, smem_for, &t, want_nw, 226 * 1024, want_half, true, in_f32 == nullptr)) { c = t; nw = want_nw; half = want_half; }
+            if (choose_tile(g, chan_blocks, smem_for, &t, want_nw, 226 * 1024, want_half, true, !f32_input)) { c = t; nw = want_nw; half = want_half; }
         }
     }
 #endif
     set_tile(g, &p, c.tile);
     p.n_tiles = (int32_t)((g.M + c.tile - 1) / c.tile);
-    const size_t smem_bytes = smem_bytes_for(g, p);
     p.half_block = half ? chan_blocks - 1 : -1;
     p.full_blocks = half ? chan_blocks - 1 : chan_blocks;
     p.ctas_full = c.ctas_x;
     p.ctas_half = half ? c.ctas_half : 0;
     p.range_full = c.range_full;
     p.range_half = c.range_half;
-    dim3 grid((unsigned)(p.full_blocks * p.ctas_full + p.ctas_half), 1, 1);
+    plan->pointwise = false;
+    plan->nw = nw;
+    plan->tp = c.tp;
+    plan->smem_bytes = smem_bytes_for(g, p);
+    plan->grid = dim3((unsigned)(p.full_blocks * p.ctas_full + p.ctas_half), 1, 1);
 #ifdef LCE_TUNING
     if (getenv("LCE_VERBOSE"))
-        fprintf(stderr, "tiled %dx%d M=%lld Cw=%d Cout=%d: nw=%d tp=%d tile=%d n_tiles=%d grid=%dx%d+%d range=%d/%d smem=%zu cost=%.0f\n", g.KH, g.KW,
-                (long long)g.M, g.Cw, g.Cout, nw, c.tp, c.tile, p.n_tiles, p.ctas_full, p.full_blocks, p.ctas_half, p.range_full, p.range_half, smem_bytes, c.cost);
+        fprintf(stderr, "tiled %dx%d M=%lld Cw=%d Cout=%d: nw=%d tp=%d tile=%d grid=%dx%d+%d range=%d/%d smem=%zu cost=%.0f\n", g.KH, g.KW,
+                (long long)g.M, g.Cw, g.Cout, nw, c.tp, c.tile, p.ctas_full, p.full_blocks, p.ctas_half, p.range_full, p.range_half,
+                plan->smem_bytes, c.cost);
 #endif
+    return LCE_OK;
+}
+
+lce_status tiled_plan_info(const ConvGeom &g, TiledPlanInfo *info)
+{
+    TiledParams p{};
+    TiledPlan plan{};
+    const lce_status st = plan_tiled(g, false, &p, &plan);
+    if (st != LCE_OK) return st;
+    info->pointwise = plan.pointwise ? 1 : 0;
+    info->warps_per_cta = plan.nw;
+    info->pixels_per_thread = plan.tp;
+    info->tile_pixels = p.tile_pixels;
+    info->ctas = (int32_t)(plan.grid.x * plan.grid.y);
+    info->ctas_half_block = plan.pointwise ? 0 : p.ctas_half;
+    info->pixels_per_cta = plan.pointwise ? 0 : p.range_full;
+    info->pixels_per_cta_half_block = plan.pointwise ? 0 : p.range_half;
+    info->shared_bytes = (int64_t)plan.smem_bytes;
+    return LCE_OK;
+}
+
+lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const uint32_t *w_image,
+                              const float *mult, const float *bias, const int32_t *thr, void *out, cudaStream_t s,
+                              const float *residual, uint32_t *out_packed, const float *in_f32)
+{
+    // 128-bit epilogue accesses need 16-byte aligned buffers when the channel count allows them
+    if ((g.Cout & 3) == 0 && g.out_type != LCE_OUT_BITPACKED && (!aligned(out, 16) || !aligned(residual, 16)))
+        return LCE_ERR_UNSUPPORTED;
+    if (w_image && !aligned(w_image, 16)) return LCE_ERR_ALIGNMENT;
+    TiledParams p{};
+    TiledPlan plan{};
+    const lce_status st = plan_tiled(g, in_f32 != nullptr, &p, &plan);
+    if (st != LCE_OK) return st;
+    p.in = in; p.w = w; p.w_image = w_image; p.mult = mult; p.bias = bias; p.thr = thr; p.out = out;
+    p.residual = residual; p.out_packed = out_packed; p.in_f32 = in_f32;
+    const size_t smem_bytes = plan.smem_bytes;
+    const dim3 grid = plan.grid;
+    const int nw = plan.nw;
+    struct { int tp; } c{plan.tp};
+    if (plan.pointwise) {
+        if (c.tp == 2) return launch1x1<2>(p, smem_bytes, grid, s);
+        if (c.tp == 3) return launch1x1<3>(p, smem_bytes, grid, s);
+        return launch1x1<4>(p, smem_bytes, grid, s);
+    }
 #define LCE_LAUNCH_TP(KS, ST, NW)                                                   \
     do {                                                                            \
         if (c.tp == 1) return launch_kxk<KS, ST, 1, 4>(p, smem_bytes, grid, s);     \

@@ -90,6 +90,13 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const uint
                                const float *bias, const int32_t *thr, void *out, cudaStream_t s);
 lce_status tensor_device_status(int *status);
 // Bytes of the tiled kernel's weight image for this geometry (0 if the kernel does not cover it).
+// Launch plan of the tiled kernels for a geometry (no buffers involved), for lce_bconv2d_plan.
+struct TiledPlanInfo {
+    int32_t pointwise, warps_per_cta, pixels_per_thread, tile_pixels, ctas, ctas_half_block, pixels_per_cta,
+        pixels_per_cta_half_block;
+    int64_t shared_bytes;
+};
+lce_status tiled_plan_info(const ConvGeom &g, TiledPlanInfo *info);
 size_t tiled_weight_image_bytes(const ConvGeom &g);
 lce_status launch_pack_weights_tiled(const ConvGeom &g, const uint32_t *w, uint32_t *image, cudaStream_t s);
 

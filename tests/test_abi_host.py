@@ -79,3 +79,61 @@ def test_binding_refuses_cpu_tensors():
     import torch
     with pytest.raises(ValueError):
         lce.lce_bitpack(torch.zeros(4, 32))
+
+
+# ---- launch plans (host arithmetic only): the work split the kernels rely on ----------------------
+
+def _plan(N, H, W, Cin, Cout, k, s, padding=None, kernel_choice=None, out_type=None):
+    d = lce.make_desc(N, H, W, Cin, Cout, (k, k), (s, s), lce.PAD_SAME_ONE if padding is None else padding,
+                      lce.OUT_BITPACKED if out_type is None else out_type, lce.ACT_NONE,
+                      lce.KERNEL_AUTO if kernel_choice is None else kernel_choice)
+    oh, ow = lce.lce_bconv2d_out_shape(d)
+    return lce.lce_bconv2d_plan(d), N * oh * ow
+
+
+PLAN_SHAPES = [(64, 56, 56, 64, 64, 3, 1), (64, 28, 28, 128, 128, 3, 1), (64, 14, 14, 256, 256, 3, 1), (64, 7, 7, 512, 512, 3, 1),
+               (64, 56, 56, 64, 128, 3, 2), (1, 14, 14, 64, 64, 3, 1), (1, 8, 8, 32, 32, 3, 1), (64, 64, 64, 96, 96, 5, 1),
+               (64, 64, 64, 256, 256, 5, 1), (3, 9, 11, 160, 70, 3, 1), (1, 1, 1, 33, 1, 3, 1), (2, 17, 13, 96, 33, 5, 2),
+               (256, 112, 112, 32, 64, 3, 2), (7, 5, 5, 40, 200, 3, 1)]
+
+
+@pytest.mark.parametrize("shape", PLAN_SHAPES)
+def test_tiled_plan_covers_every_pixel_once_and_fits_the_sm(lib, shape):
+    plan, M = _plan(*shape)
+    Cout = shape[4]
+    assert plan["kernel"] == lce.KERNEL_TILED and not plan["patch"] and not plan["pointwise"]
+    nw, tp = plan["warps_per_cta"], plan["pixels_per_thread"]
+    assert nw in (4, 8) and 1 <= tp <= 4 and (tp > 1 or nw == 4)
+    assert plan["tile_pixels"] % (4 * nw * tp) == 0 and plan["tile_pixels"] > 0
+    assert 0 < plan["shared_bytes"] <= 227 * 1024
+    blocks = (Cout + 63) // 64
+    half = plan["ctas_half_block"]
+    full_blocks = blocks - (1 if half else 0)
+    if half:
+        assert 1 <= Cout % 64 <= 32
+        r = plan["pixels_per_cta_half_block"]
+        assert r % (8 * nw) == 0 and half * r >= M and (half - 1) * r < M   # ranges tile [0, M), none is empty
+    if full_blocks:
+        assert (plan["ctas"] - half) % full_blocks == 0
+        per_block = (plan["ctas"] - half) // full_blocks
+        r = plan["pixels_per_cta"]
+        assert r % (4 * nw) == 0 and per_block * r >= M and (per_block - 1) * r < M
+    # one resident wave: the kernel is persistent, no CTA waits for an SM
+    per_sm_by_regs = (24 if tp <= 2 else 16) // nw
+    per_sm_by_smem = (228 * 1024) // (plan["shared_bytes"] + 1024)
+    assert plan["ctas"] <= 148 * min(per_sm_by_regs, per_sm_by_smem)
+
+
+def test_plan_names_the_other_kernels(lib):
+    assert _plan(2, 20, 18, 3, 32, 3, 2)[0]["patch"] == 1                                   # RGB stem: one-word patches
+    p = _plan(64, 14, 14, 256, 512, 1, 1)[0]
+    assert p["kernel"] == lce.KERNEL_TILED and p["pointwise"] == 1 and p["ctas"] > 0
+    assert _plan(1, 9, 9, 64, 64, 7, 1)[0]["kernel"] == lce.KERNEL_DIRECT                    # no tiled 7x7
+    assert _plan(1, 9, 9, 64, 64, 3, 1, kernel_choice=lce.KERNEL_DIRECT)[0]["kernel"] == lce.KERNEL_DIRECT
+    assert _plan(1, 9, 9, 64, 64, 3, 1, kernel_choice=lce.KERNEL_TENSOR)[0]["kernel"] == lce.KERNEL_TENSOR
+    with pytest.raises(lce.LceError) as e:
+        _plan(1, 9, 9, 64, 64, 7, 1, kernel_choice=lce.KERNEL_TILED)
+    assert e.value.status == 2
+    with pytest.raises(lce.LceError) as e:
+        _plan(1, 9, 9, 64, 64, 3, 2, kernel_choice=lce.KERNEL_TENSOR)                        # tensor path: stride 1 only
+    assert e.value.status == 2

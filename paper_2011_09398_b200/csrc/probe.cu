@@ -186,8 +186,7 @@ probe_combined_kernel(const uint32_t *__restrict__ seed, uint32_t *__restrict__ 
     __syncthreads();
     const int warp = threadIdx.x >> 5;
     uint32_t x = 0;
-    if ((warp & 1) == 0) {
-        if (MODE == 2) return;
+    if ((warp & 1) == 0 && MODE != 2) {
         // as in the convolution kernel: 4 pixels x 8 channels per thread, activation operands in
         // registers, each channel's weight operands read from shared memory once per group
         constexpr int TPX = 4;
@@ -237,8 +236,7 @@ probe_combined_kernel(const uint32_t *__restrict__ seed, uint32_t *__restrict__ 
 #pragma unroll
             for (int j = 0; j < CH; ++j) x ^= acc[p][j];
         if (threadIdx.x == 0) cycles[2 * blockIdx.x] = t1 - t0;
-    } else {
-        if (MODE == 1) return;
+    } else if ((warp & 1) == 1 && MODE != 1) {
         uint32_t a[4], b[2];
         int32_t d[8][4];
 #pragma unroll

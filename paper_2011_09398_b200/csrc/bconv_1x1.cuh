@@ -123,6 +123,8 @@ bconv1x1_kernel(const TiledParams p)
     const int px = lane >> 3, cg = lane & 7;
     const int chan = ch0 + cg * kChanPerThread;
     const int K = p.Cin;
+    const bool biased = p.out_type == LCE_OUT_FLOAT32 && K < kMaxBiasedK;
+    const int Kb = biased ? K + kFloatBias : K;
     Weights124 k124;
     k124.one = p.N > 0 ? 1u : p.Cin;
     k124.two = p.N > 0 ? 2u : p.Cin;
@@ -190,8 +192,8 @@ bconv1x1_kernel(const TiledParams p)
                 const int m = base + i * kPixPerStep + warp * 4 + px;
                 int32_t v[kChanPerThread];
 #pragma unroll
-                for (int j = 0; j < kChanPerThread; ++j) v[j] = K - 2 * (int32_t)acc[i][j];
-                store_outputs(p, v, cp, m, m < m_end, cg, ch0, chan);
+                for (int j = 0; j < kChanPerThread; ++j) v[j] = Kb - 2 * (int32_t)acc[i][j];
+                store_outputs(p, v, cp, m, m < m_end, cg, ch0, chan, biased);
             }
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");

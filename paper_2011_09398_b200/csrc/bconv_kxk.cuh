@@ -177,6 +177,9 @@ bconv3x3_kernel(const TiledParams p)
     const int pix_per_step = pix_per_warp * NW;  // pixels the CTA works on at a time
     const int chan = ch0 + cg * kChanPerThread;
     const int K = kTaps * p.Cin;
+    // float output: accumulators carry the bias that makes int -> float one exact subtraction
+    const bool biased = p.out_type == LCE_OUT_FLOAT32 && K < kMaxBiasedK;
+    const int Kb = biased ? K + kFloatBias : K;
     Weights124 k124;
     k124.one = p.N > 0 ? 1u : p.Cin;  // opaque to the compiler: keeps the weighted sum on multiply-adds
     k124.two = p.N > 0 ? 2u : p.Cin;
@@ -276,7 +279,7 @@ bconv3x3_kernel(const TiledParams p)
             const bool pix_ok = m < m_end;
             int32_t v[kChanPerThread];
 #pragma unroll
-            for (int j = 0; j < kChanPerThread; ++j) v[j] = K - 2 * (int32_t)acc[i][j];
+            for (int j = 0; j < kChanPerThread; ++j) v[j] = Kb - 2 * (int32_t)acc[i][j];
             if (p.padding == LCE_PAD_SAME_ZERO) {
                 // zero-padding correction: taps outside the image contributed (+1)*w; take that out
                 const int mm = pix_ok ? m : m0;
@@ -291,7 +294,7 @@ bconv3x3_kernel(const TiledParams p)
                     }
                 }
             }
-            store_outputs(p, v, cp, m, pix_ok, cg, ch0, chan);
+            store_outputs(p, v, cp, m, pix_ok, cg, ch0, chan, biased);
         }
     };
     for (int base = m0; base < m_end;) {

@@ -180,20 +180,40 @@ struct ChannelParams {
 };
 __device__ __forceinline__ void load_channel_params(const TiledParams &p, int chan, ChannelParams &c)
 {
+    if (chan + kChanPerThread <= p.Cout) {
+        // all eight channels exist (every thread but those of a ragged last group): unconditional
+        // loads of only what the output type needs
 #pragma unroll
-    for (int j = 0; j < kChanPerThread; ++j) {
-        const bool ok = chan + j < p.Cout;
-        c.mult[j] = (p.out_type == LCE_OUT_FLOAT32 && ok) ? __ldg(p.mult + chan + j) : 0.f;
-        c.bias[j] = (p.out_type == LCE_OUT_FLOAT32 && ok) ? __ldg(p.bias + chan + j) : 0.f;
-        c.thr[j] = (p.out_type == LCE_OUT_BITPACKED && ok) ? __ldg(p.thr + chan + j) : INT32_MIN;  // pad bits -> 0
+        for (int j = 0; j < kChanPerThread; ++j) {
+            c.mult[j] = (p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.mult + chan + j) : 0.f;
+            c.bias[j] = (p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.bias + chan + j) : 0.f;
+            c.thr[j] = (p.out_type == LCE_OUT_BITPACKED) ? __ldg(p.thr + chan + j) : INT32_MIN;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < kChanPerThread; ++j) {
+            const bool ok = chan + j < p.Cout;
+            c.mult[j] = (p.out_type == LCE_OUT_FLOAT32 && ok) ? __ldg(p.mult + chan + j) : 0.f;
+            c.bias[j] = (p.out_type == LCE_OUT_FLOAT32 && ok) ? __ldg(p.bias + chan + j) : 0.f;
+            c.thr[j] = (p.out_type == LCE_OUT_BITPACKED && ok) ? __ldg(p.thr + chan + j) : INT32_MIN;  // pad bits -> 0
+        }
     }
 }
+
+// int32 -> fp32 without the conversion unit: for |v| < 2^22 the integer v + 0x4B400000 is the bit
+// pattern of the float 12582912 + v (1.5 * 2^23, where floats are exactly one apart), so one exact
+// float subtraction gives (float)v.  The kernels fold the integer addition into acc = K - 2*count
+// ("biased" accumulators); the conversion then costs one FADD on the FMA pipe instead of an I2F on
+// the unit the popcounts use.
+constexpr int32_t kFloatBias = 0x4B400000;
+constexpr int32_t kMaxBiasedK = 1 << 22;
 
 // Output transform of one pixel's 8 accumulators v (paper Section 3.2): float multiply-add after
 // the fused activation, threshold compare + bit-pack, or the raw accumulators.  Every lane of the
 // warp must call it (the bit-packed form combines 4 lanes with shuffles); pix_ok guards the store.
 __device__ __forceinline__ void store_outputs(const TiledParams &p, const int32_t (&v)[kChanPerThread],
-                                              const ChannelParams &c, int m, bool pix_ok, int cg, int ch0, int chan)
+                                              const ChannelParams &c, int m, bool pix_ok, int cg, int ch0, int chan,
+                                              bool biased)  // v carries + kFloatBias (float output with K < 2^22 only)
 {
     const float (&mult)[kChanPerThread] = c.mult;
     const float (&bias)[kChanPerThread] = c.bias;
@@ -213,8 +233,11 @@ __device__ __forceinline__ void store_outputs(const TiledParams &p, const int32_
         float f[kChanPerThread];
 #pragma unroll
         for (int j = 0; j < kChanPerThread; ++j) {
-            const int32_t a = (p.activation == LCE_ACT_RELU && v[j] < 0) ? 0 : v[j];
-            f[j] = __fmaf_rn((float)a, mult[j], bias[j]);
+            // fused ReLU on the integer: max(v, 0), or max(v + bias, bias) in the biased form
+            const int32_t floor_v = p.activation == LCE_ACT_RELU ? (biased ? kFloatBias : 0) : INT32_MIN;
+            const int32_t a = max(v[j], floor_v);
+            const float x = biased ? __fadd_rn(__int_as_float(a), -12582912.0f) : (float)a;
+            f[j] = __fmaf_rn(x, mult[j], bias[j]);
         }
         const bool vec = (p.Cout & 3) == 0 && chan + kChanPerThread <= p.Cout;
         if (p.residual != nullptr) {

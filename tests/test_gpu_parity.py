@@ -336,3 +336,37 @@ def test_async_host_entry_point_on_two_streams_matches_oracle():
             assert float_close(h_out.numpy(), acc, t.multiplier, t.bias) == 0
         else:
             np.testing.assert_array_equal(h_out.numpy().view(np.uint32), oracle.transform_bits(acc, t.thresholds))
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_seeded_random_shapes_through_the_dispatcher(seed):
+    """40 random layer shapes per seed (filter 1/3/5, stride 1/2, all paddings, ragged channel counts,
+    plain or load-time packed weights): whatever kernel and work split the dispatcher picks, int32,
+    bit-packed and float outputs equal the oracle's."""
+    rng = np.random.default_rng(seed)
+    done = 0
+    while done < 40:
+        k, s = int(rng.choice([1, 3, 3, 5])), int(rng.choice([1, 1, 2]))
+        N, H, W = int(rng.integers(1, 7)), int(rng.integers(1, 70)), int(rng.integers(1, 70))
+        Cin = int(rng.choice([rng.integers(1, 40), rng.integers(1, 300), 32, 64, 96, 128]))
+        Cout = int(rng.choice([rng.integers(1, 40), rng.integers(1, 300), 32, 64, 96, 160]))
+        padding = int(rng.integers(0, 3))
+        if (padding == lce.PAD_VALID and (H < k or W < k)) or N * H * W * Cout * k * k * Cin > 2e9:
+            continue
+        done += 1
+        packed = bool(rng.integers(0, 2))
+        a, w = rand_pm1(rng, (N, H, W, Cin)), rand_pm1(rng, (Cout, k, k, Cin))
+        aw, ww = oracle.bitpack_pm1(a), oracle.bitpack_pm1(w)
+        acc = oracle.bconv2d_acc(a, w, (s, s), padding)
+        kw = dict(in_c=Cin, stride=(s, s), padding=padding)
+        where = f"N={N} H={H} W={W} Cin={Cin} Cout={Cout} k={k} s={s} padding={padding} packed={packed}"
+        got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_INT32), packed=packed)
+        assert np.array_equal(got, acc), where
+        thr = np.rint(np.sqrt(k * k * Cin) * rng.standard_normal(Cout)).astype(np.int32)
+        got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_BITPACKED), thr=thr, packed=packed)
+        assert np.array_equal(got, oracle.transform_bits(acc, thr)), where
+        mult = rng.uniform(0.5, 1.5, Cout).astype(np.float32)
+        bias = (0.1 * rng.standard_normal(Cout)).astype(np.float32)
+        act = int(rng.integers(0, 2))
+        got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_FLOAT32, activation=act), mult=mult, bias=bias, packed=packed)
+        assert float_close(got, acc, mult, bias, act) == 0, where

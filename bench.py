@@ -362,6 +362,7 @@ def run_lce(args):
         line["tensor_core_path"] = time_tensor_path(dev, layers)
         if not args.no_sweep:
             line["paper_sweep"] = time_paper_sweep(dev)
+        line["streaming_kernels"] = time_streaming_kernels(dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cores = len(os.sched_getaffinity(0))
         sample_batch, passes = BATCH, 2
@@ -416,6 +417,45 @@ def time_tensor_path(dev, layers, reps: int = 5):
             total_macs += s.binary_macs
     out["all_8_launches"] = {"us": total_ms * 1e3, "T_bmac_per_s": total_macs / (total_ms * 1e-3) / 1e12}
     out["device_status"] = lce.lce_device_status()
+    return out
+
+
+def time_streaming_kernels(dev, reps: int = 20):
+    """The HBM-bound kernels around the convolution (LceQuantize, LceBMaxPool2d, the shortcut add) on
+    tensors larger than the L2, each against the measured copy bandwidth: bytes moved / time."""
+    import torch
+
+    import paper_2011_09398_b200 as lce
+    peak = peak_hbm_bytes_per_s()
+    out = {}
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1) * 1e-3 / reps
+
+    def entry(name, seconds, nbytes):
+        out[name] = {"us": seconds * 1e6, "GB_per_s": nbytes / seconds / 1e9, "frac_of_measured_hbm": nbytes / seconds / peak}
+
+    x = torch.randn((256, 112, 112, 64), device=dev)                       # 822 MB of fp32
+    words = lce.lce_bitpack(x)
+    entry("bitpack_256x112x112x64", timed(lambda: lce.lce_bitpack(x, words)), x.numel() * 4 + words.numel() * 4)
+    rgb = torch.randn((256, 224, 224, 3), device=dev)                      # 154 MB: the config 5 input
+    w3 = lce.lce_bitpack(rgb)
+    entry("bitpack_256x224x224x3", timed(lambda: lce.lce_bitpack(rgb, w3)), rgb.numel() * 4 + w3.numel() * 4)
+    y = torch.randn_like(x)
+    z = torch.empty_like(x)
+    entry("add_f32_256x112x112x64", timed(lambda: lce.lce_add_f32(x, y, z)), 3 * x.numel() * 4)
+    big = torch.randint(-2**31, 2**31 - 1, (256, 224, 224, 8), dtype=torch.int32, device=dev)   # 411 MB of packed words
+    pooled = lce.lce_bmaxpool(big, 256)
+    entry("bmaxpool2x2_256x224x224x256", timed(lambda: lce.lce_bmaxpool(big, 256, out=pooled)), big.numel() * 4 + pooled.numel() * 4)
     return out
 
 

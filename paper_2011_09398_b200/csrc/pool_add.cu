@@ -8,32 +8,48 @@ namespace {
 
 constexpr int kThreads = 256;
 
-// One thread per output word.  Out-of-image taps are skipped (AND identity = all ones);
-// channel-pad bits stay 0 because they are 0 in every input word.
+// A block walks output rows (n, oh); its threads walk the row's words, VEC words at a time (VEC = 4:
+// 128-bit loads and stores, when the word count per pixel allows), so that the only division left
+// per output is a 32-bit one by the words per pixel.  Out-of-image taps are skipped (AND identity
+// = all ones); channel-pad bits stay 0 because they are 0 in every input word.
+template <int VEC>
 __global__ void __launch_bounds__(kThreads)
 bmaxpool_kernel(const uint32_t *__restrict__ in, uint32_t *__restrict__ out, int32_t N, int32_t H, int32_t W,
                 int32_t Cw, int32_t OH, int32_t OW, int32_t PH, int32_t PW, int32_t sh, int32_t sw, int32_t pt,
                 int32_t pl)
 {
-    const int64_t total = (int64_t)N * OH * OW * Cw;
-    for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < total; i += (int64_t)gridDim.x * kThreads) {
-        const int32_t j = (int32_t)(i % Cw);
-        int64_t p = i / Cw;
-        const int32_t ow = (int32_t)(p % OW);
-        p /= OW;
-        const int32_t oh = (int32_t)(p % OH);
-        const int32_t n = (int32_t)(p / OH);
-        uint32_t acc = 0xffffffffu;
-        for (int32_t ky = 0; ky < PH; ++ky) {
-            const int32_t iy = oh * sh - pt + ky;
-            if (iy < 0 || iy >= H) continue;
-            for (int32_t kx = 0; kx < PW; ++kx) {
-                const int32_t ix = ow * sw - pl + kx;
-                if (ix < 0 || ix >= W) continue;
-                acc &= __ldg(in + (((int64_t)n * H + iy) * W + ix) * Cw + j);
+    const int32_t cv = Cw / VEC;            // vectors per pixel
+    const int32_t row_vecs = OW * cv;       // vectors per output row
+    const int32_t rows = N * OH;  // < 2^31: checked on the host
+    for (int32_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        const int32_t n = row / OH, oh = row - n * OH;
+        const int32_t iy0 = oh * sh - pt;
+        const uint32_t *img = in + (int64_t)n * H * W * Cw;
+        uint32_t *orow = out + (int64_t)row * OW * Cw;
+        for (int32_t e = threadIdx.x; e < row_vecs; e += kThreads) {
+            const int32_t ow = e / cv, j = (e - ow * cv) * VEC;
+            const int32_t ix0 = ow * sw - pl;
+            uint32_t acc[VEC];
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[v] = 0xffffffffu;
+            for (int32_t ky = 0; ky < PH; ++ky) {
+                const int32_t iy = iy0 + ky;
+                if (iy < 0 || iy >= H) continue;
+                for (int32_t kx = 0; kx < PW; ++kx) {
+                    const int32_t ix = ix0 + kx;
+                    if (ix < 0 || ix >= W) continue;
+                    const uint32_t *src = img + ((int64_t)iy * W + ix) * Cw + j;
+                    if (VEC == 4) {
+                        const uint4 q = __ldcs(reinterpret_cast<const uint4 *>(src));
+                        acc[0] &= q.x; acc[1] &= q.y; acc[2] &= q.z; acc[3] &= q.w;
+                    } else {
+                        acc[0] &= __ldcs(src);
+                    }
+                }
             }
+            if (VEC == 4) *reinterpret_cast<uint4 *>(orow + (int64_t)ow * Cw + j) = make_uint4(acc[0], acc[1], acc[2], acc[3]);
+            else orow[(int64_t)ow * Cw + j] = acc[0];
         }
-        out[i] = acc;
     }
 }
 
@@ -80,9 +96,17 @@ extern "C" lce_status lce_bmaxpool(const uint32_t *in, uint32_t *out, int32_t ba
     if (ah.out <= 0 || aw.out <= 0) return LCE_ERR_INVALID_ARG;
     const int32_t Cw = (channels + 31) / 32;
     const int64_t total = (int64_t)batch * ah.out * aw.out * Cw;
-    bmaxpool_kernel<<<grid_for(total, 148 * 16), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        in, out, batch, in_h, in_w, Cw, ah.out, aw.out, pool_h, pool_w, stride_h, stride_w, ah.pad_before,
-        aw.pad_before);
+    (void)total;
+    if ((int64_t)batch * ah.out >= (1ll << 31)) return LCE_ERR_UNSUPPORTED;
+    int64_t blocks = (int64_t)batch * ah.out;  // one block per output row, grid-stride beyond 8 waves of 8 blocks per SM
+    if (blocks > 148 * 8 * 8) blocks = 148 * 8 * 8;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (Cw % 4 == 0 && aligned(in, 16) && aligned(out, 16))
+        bmaxpool_kernel<4><<<(unsigned)blocks, kThreads, 0, s>>>(in, out, batch, in_h, in_w, Cw, ah.out, aw.out, pool_h, pool_w,
+                                                                stride_h, stride_w, ah.pad_before, aw.pad_before);
+    else
+        bmaxpool_kernel<1><<<(unsigned)blocks, kThreads, 0, s>>>(in, out, batch, in_h, in_w, Cw, ah.out, aw.out, pool_h, pool_w,
+                                                                stride_h, stride_w, ah.pad_before, aw.pad_before);
     return launch_status();
 }
 

@@ -40,10 +40,10 @@ bmaxpool_kernel(const uint32_t *__restrict__ in, uint32_t *__restrict__ out, int
                     if (ix < 0 || ix >= W) continue;
                     const uint32_t *src = img + ((int64_t)iy * W + ix) * Cw + j;
                     if (VEC == 4) {
-                        const uint4 q = __ldcs(reinterpret_cast<const uint4 *>(src));
+                        const uint4 q = __ldg(reinterpret_cast<const uint4 *>(src));
                         acc[0] &= q.x; acc[1] &= q.y; acc[2] &= q.z; acc[3] &= q.w;
                     } else {
-                        acc[0] &= __ldcs(src);
+                        acc[0] &= __ldg(src);
                     }
                 }
             }

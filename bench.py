@@ -450,6 +450,9 @@ def time_streaming_kernels(dev, reps: int = 20):
     rgb = torch.randn((256, 224, 224, 3), device=dev)                      # 154 MB: the config 5 input
     w3 = lce.lce_bitpack(rgb)
     entry("bitpack_256x224x224x3", timed(lambda: lce.lce_bitpack(rgb, w3)), rgb.numel() * 4 + w3.numel() * 4)
+    back = torch.empty_like(x)
+    entry("unpack_256x112x112x64", timed(lambda: lce.lce_unpack(words, 64, back)), x.numel() * 4 + words.numel() * 4)
+    del back
     y = torch.randn_like(x)
     z = torch.empty_like(x)
     entry("add_f32_256x112x112x64", timed(lambda: lce.lce_add_f32(x, y, z)), 3 * x.numel() * 4)

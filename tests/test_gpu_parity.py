@@ -64,7 +64,7 @@ def test_bitpack_one_hot_bit_order():
         assert int(got[1, c // 32]) == 1 << (c % 32)
 
 
-@pytest.mark.parametrize("rows,C", [(5, 3), (64, 64), (77, 70), (1, 1)])
+@pytest.mark.parametrize("rows,C", [(5, 3), (64, 64), (77, 70), (1, 1), (4099, 32), (1001, 256), (3, 96)])
 def test_unpack_matches_oracle(rows, C):
     rng = np.random.default_rng(C)
     words = oracle.bitpack(rng.standard_normal((rows, C)).astype(np.float32))

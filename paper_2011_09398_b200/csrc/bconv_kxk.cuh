@@ -102,6 +102,23 @@ __device__ __forceinline__ void stage_rows(const TiledParams &p, int m0, int m_e
     }
 }
 
+template <int J, int TP>
+struct ChannelLoopPacked {
+    __device__ __forceinline__ static void run(uint32_t w_saddr, const Triple (&at)[TP][3], const Weights124 &k, const Weights124 &khi,
+                                               uint32_t (&acc)[(TP + 1) / 2][kChanPerThread])
+    {
+        Triple wt[3];
+        load_w_triples<J>(w_saddr, wt);
+        popc9_mad_pixels_packed<TP, kChanPerThread, J>(at, wt, k, khi, acc);
+        ChannelLoopPacked<J + 1, TP>::run(w_saddr, at, k, khi, acc);
+    }
+};
+template <int TP>
+struct ChannelLoopPacked<kChanPerThread, TP> {
+    __device__ __forceinline__ static void run(uint32_t, const Triple (&)[TP][3], const Weights124 &, const Weights124 &,
+                                               uint32_t (&)[(TP + 1) / 2][kChanPerThread]) {}
+};
+
 // NW warps per CTA: 4 normally; 8 when the weight operands of a channel block are so large that
 // only one CTA fits an SM, so that the SM still has eight warps to hide latencies with.
 template <int KS, int STRIDE, int TP, int NW, bool F32>
@@ -185,6 +202,11 @@ bconv3x3_kernel(const TiledParams p)
     k124.two = p.N > 0 ? 2u : p.Cin;
     k124.four = p.N > 0 ? 4u : p.Cin;
     asm volatile("" : "+r"(k124.one), "+r"(k124.two), "+r"(k124.four));
+    Weights124 khi;  // the same multipliers for the pixel kept in the high half of an accumulator
+    khi.one = p.N > 0 ? (1u << 16) : p.Cin;
+    khi.two = p.N > 0 ? (2u << 16) : p.Cin;
+    khi.four = p.N > 0 ? (4u << 16) : p.Cin;
+    asm volatile("" : "+r"(khi.one), "+r"(khi.two), "+r"(khi.four));
     const uint32_t w_saddr0 = (uint32_t)__cvta_generic_to_shared(sW + cg * kWGroupStride);
 
     // ---- loop over the tiles of this CTA's range; the next tile's input rows are copied into the
@@ -238,9 +260,10 @@ bconv3x3_kernel(const TiledParams p)
                 else { --oh_left; voh += STRIDE; }
             }
         }
-        uint32_t acc[TPX][kChanPerThread];
+        constexpr int HX = (TPX + 1) / 2;  // two pixels' 16-bit counts per accumulator register
+        uint32_t acc[HX][kChanPerThread];
 #pragma unroll
-        for (int i = 0; i < TPX; ++i)
+        for (int i = 0; i < HX; ++i)
 #pragma unroll
             for (int j = 0; j < kChanPerThread; ++j) acc[i][j] = 0u;
 
@@ -264,7 +287,7 @@ bconv3x3_kernel(const TiledParams p)
                         }
                         at[i][k] = make_triple(v[0], v[1], v[2]);
                     }
-                ChannelLoop<0, TPX>::run(w_saddr, at, k124, acc);
+                ChannelLoopPacked<0, TPX>::run(w_saddr, at, k124, khi, acc);
                 w_saddr += kChanGroups * kWGroupStride * 4;
             }
             plane += p.plane;
@@ -279,7 +302,8 @@ bconv3x3_kernel(const TiledParams p)
             const bool pix_ok = m < m_end;
             int32_t v[kChanPerThread];
 #pragma unroll
-            for (int j = 0; j < kChanPerThread; ++j) v[j] = Kb - 2 * (int32_t)acc[i][j];
+            for (int j = 0; j < kChanPerThread; ++j)
+                v[j] = Kb - 2 * (int32_t)(i < HX ? (acc[i][j] & 0xFFFFu) : (acc[i - HX][j] >> 16));
             if (p.padding == LCE_PAD_SAME_ZERO) {
                 // zero-padding correction: taps outside the image contributed (+1)*w; take that out
                 const int mm = pix_ok ? m : m0;

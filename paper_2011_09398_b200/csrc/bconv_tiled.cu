@@ -80,7 +80,11 @@ void set_tile(const ConvGeom &g, TiledParams *p, int tile_pixels)
     p->plane = nv_max * p->pitch;
 }
 
-bool covers3x3(const ConvGeom &g) { return g.KH == g.KW && (g.KH == 3 || g.KH == 5) && g.sh == g.sw && g.sh <= 2; }
+// the KxK kernel keeps two pixels' counts in one 32-bit accumulator: a count can reach K, so K < 65536
+bool covers3x3(const ConvGeom &g)
+{
+    return g.KH == g.KW && (g.KH == 3 || g.KH == 5) && g.sh == g.sw && g.sh <= 2 && (int64_t)g.KH * g.KW * g.Cin < 65536;
+}
 bool covers1x1(const ConvGeom &g) { return g.KH == 1 && g.KW == 1 && g.sh == g.sw; }
 
 bool tiled_covers(const ConvGeom &g)

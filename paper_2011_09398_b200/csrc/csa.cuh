@@ -144,6 +144,53 @@ __device__ __forceinline__ void popc9_mad_pixels(const Triple (&a)[TP][3], const
     for (int i = 0; i < TP; ++i) acc[i][J] = mad_u32(pF[i], k.four, acc[i][J]);
 }
 
+// The same with two pixels' counts per accumulator register: pixel i < H = ceil(TP/2) in the low 16
+// bits of acc[i], pixel i >= H in the high 16 bits of acc[i - H], its multiply-adds using the
+// multipliers shifted left by 16 (`khi` = {1<<16, 2<<16, 4<<16}).  Counts must stay below 65536.
+template <int TP, int NCH, int J>
+__device__ __forceinline__ void popc9_mad_pixels_packed(const Triple (&a)[TP][3], const Triple (&w)[3], const Weights124 &k,
+                                                        const Weights124 &khi, uint32_t (&acc)[(TP + 1) / 2][NCH])
+{
+    constexpr int H = (TP + 1) / 2;
+    uint32_t s[TP][3], c[TP][3];
+#pragma unroll
+    for (int g = 0; g < 3; ++g)
+#pragma unroll
+        for (int i = 0; i < TP; ++i) s[i][g] = a[i][g].all ^ w[g].all;
+#pragma unroll
+    for (int g = 0; g < 3; ++g)
+#pragma unroll
+        for (int i = 0; i < TP; ++i) {
+            const uint32_t d = a[i][g].pair ^ w[g].pair;
+            const uint32_t x0 = a[i][g].first ^ w[g].first;
+            c[i][g] = carry_dsx(d, s[i][g], x0);
+        }
+    uint32_t S[TP], C[TP], T[TP], F[TP];
+#pragma unroll
+    for (int i = 0; i < TP; ++i) {
+        S[i] = xor3(s[i][0], s[i][1], s[i][2]);
+        C[i] = maj3(s[i][0], s[i][1], s[i][2]);
+    }
+#pragma unroll
+    for (int i = 0; i < TP; ++i) {
+        T[i] = xor3(c[i][0], c[i][1], c[i][2]);
+        F[i] = maj3(c[i][0], c[i][1], c[i][2]);
+    }
+    uint32_t pS[TP], pC[TP], pT[TP], pF[TP];
+#pragma unroll
+    for (int i = 0; i < TP; ++i) { pS[i] = __popc(S[i]); pC[i] = __popc(C[i]); }
+#pragma unroll
+    for (int i = 0; i < TP; ++i) { pT[i] = __popc(T[i]); pF[i] = __popc(F[i]); }
+#pragma unroll
+    for (int i = 0; i < TP; ++i) acc[i % H][J] = mad_u32(pS[i], i < H ? k.one : khi.one, acc[i % H][J]);
+#pragma unroll
+    for (int i = 0; i < TP; ++i) acc[i % H][J] = mad_u32(pC[i], i < H ? k.two : khi.two, acc[i % H][J]);
+#pragma unroll
+    for (int i = 0; i < TP; ++i) acc[i % H][J] = mad_u32(pT[i], i < H ? k.two : khi.two, acc[i % H][J]);
+#pragma unroll
+    for (int i = 0; i < TP; ++i) acc[i % H][J] = mad_u32(pF[i], i < H ? k.four : khi.four, acc[i % H][J]);
+}
+
 // One triple added onto an accumulator with multiply-adds (K tails of the pointwise kernel).
 __device__ __forceinline__ void popc3_mad(const Triple &a, const Triple &w, const Weights124 &k, uint32_t &acc)
 {

@@ -129,6 +129,7 @@ def test_plan_names_the_other_kernels(lib):
     p = _plan(64, 14, 14, 256, 512, 1, 1)[0]
     assert p["kernel"] == lce.KERNEL_TILED and p["pointwise"] == 1 and p["ctas"] > 0
     assert _plan(1, 9, 9, 64, 64, 7, 1)[0]["kernel"] == lce.KERNEL_DIRECT                    # no tiled 7x7
+    assert _plan(1, 3, 4, 7300, 5, 3, 1)[0]["kernel"] == lce.KERNEL_DIRECT                   # K >= 65536 (and far more weights than shared memory holds)
     assert _plan(1, 9, 9, 64, 64, 3, 1, kernel_choice=lce.KERNEL_DIRECT)[0]["kernel"] == lce.KERNEL_DIRECT
     assert _plan(1, 9, 9, 64, 64, 3, 1, kernel_choice=lce.KERNEL_TENSOR)[0]["kernel"] == lce.KERNEL_TENSOR
     with pytest.raises(lce.LceError) as e:

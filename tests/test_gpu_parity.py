@@ -94,6 +94,8 @@ FUZZ = [
     (1, 4, 3, 32, 9, 5, 1), (1, 64, 64, 32, 32, 5, 1),
     # wide rows and 256 channels: weights too large for two CTAs per SM -> the eight-warp variant
     (1, 20, 64, 256, 70, 5, 1),
+    # K = 9 * 7300 > 65535: past what the tiled kernel's 16-bit packed counts hold -> direct kernel
+    (1, 3, 4, 7300, 5, 3, 1),
     # few input channels: the whole receptive field fits one word
     (2, 20, 18, 3, 32, 3, 2), (1, 9, 9, 1, 40, 5, 1), (1, 12, 11, 2, 70, 3, 1), (2, 8, 8, 3, 5, 3, 1),
 ]

@@ -365,7 +365,7 @@ def run_lce(args):
         line["streaming_kernels"] = time_streaming_kernels(dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cores = len(os.sched_getaffinity(0))
-        sample_batch, passes = BATCH, 2
+        sample_batch, passes = BATCH, 4
         v, dt, _ = time_oracle(sample_batch, passes)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"all 8 launches of config 2 at batch {sample_batch}, {passes} passes of {dt:.1f} s"}

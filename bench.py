@@ -126,8 +126,9 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def time_oracle(batch: int, passes: int = 1):
-    """Times the CPU oracle, as it stands, on all 8 launches of the workload at the given batch."""
+def time_oracle(batch: int, passes: int = 1, min_seconds: float = 0.0):
+    """Times the CPU oracle, as it stands, on all 8 launches of the workload at the given batch:
+    `passes` passes, then more until `min_seconds` of CPU work are done (at most 16)."""
     import oracle
     items = []
     for i, spec in enumerate(wl.config2_specs(batch)):
@@ -136,14 +137,17 @@ def time_oracle(batch: int, passes: int = 1):
     oracle.bconv2d_acc(items[0][1][:1], items[0][2].w_pm1)  # load the library, warm the threads
     macs = sum(s.binary_macs for s, _, _ in items)
     t0 = time.perf_counter()
-    for _ in range(passes):
+    done = 0
+    while done < passes or (time.perf_counter() - t0 < min_seconds and done < 16):
         for spec, a, t in items:
             acc = oracle.bconv2d_acc(a, t.w_pm1, (1, 1), spec.padding)
             if spec.out_type == wl.OUT_FLOAT32:
                 oracle.transform_float(acc, t.multiplier, t.bias)
             else:
                 oracle.transform_bits(acc, t.thresholds)
-    dt = (time.perf_counter() - t0) / passes
+        done += 1
+    dt = (time.perf_counter() - t0) / done
+    time_oracle.last_passes = done
     return macs / dt, dt, macs
 
 
@@ -365,10 +369,10 @@ def run_lce(args):
         line["streaming_kernels"] = time_streaming_kernels(dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cores = len(os.sched_getaffinity(0))
-        sample_batch, passes = BATCH, 4
-        v, dt, _ = time_oracle(sample_batch, passes)
+        sample_batch = BATCH
+        v, dt, _ = time_oracle(sample_batch, passes=2, min_seconds=10.0)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "sample": f"all 8 launches of config 2 at batch {sample_batch}, {passes} passes of {dt:.1f} s"}
+                                "sample": f"all 8 launches of config 2 at batch {sample_batch}, {time_oracle.last_passes} passes of {dt:.1f} s"}
     if world > 1:
         dist.destroy_process_group()
     if rank == 0:

@@ -155,9 +155,10 @@ __device__ __forceinline__ void expand_word_alu(uint32_t word, uint4 *chunk_lo, 
 }
 
 // packed words of the grid positions q0 .. q0+P-1 -> raw[cw*P + row] (pad positions: zero word)
+template <int STRIDE = kWorkers>
 __device__ __forceinline__ void prefetch_raw(const TensorParams &p, int q0, uint32_t *raw, int tid)
 {
-    for (int row = tid; row < p.P; row += kWorkers) {
+    for (int row = tid; row < p.P; row += STRIDE) {
         const int f = q0 + row;
         const int rr = f / p.Wp, cc = f - rr * p.Wp;
         const int n = rr / p.Hs, ry = rr - n * p.Hs;
@@ -170,13 +171,15 @@ __device__ __forceinline__ void prefetch_raw(const TensorParams &p, int q0, uint
 
 // every thread expands the words it prefetched itself (same row mapping), so waiting for its own
 // copies is enough
+template <int STRIDE = kWorkers, bool USE_TABLE = false>
 __device__ __forceinline__ void expand_a(const TensorParams &p, const uint2 *table, const uint32_t *raw, uint8_t *sA, int tid)
 {
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    for (int row = tid; row < p.P; row += kWorkers) {
+    for (int row = tid; row < p.P; row += STRIDE) {
         for (int cw = 0; cw < p.Cw; ++cw) {
             uint4 lo, hi;
-            expand_word(table, raw[cw * p.P + row], &lo, &hi);
+            if (USE_TABLE) expand_word(table, raw[cw * p.P + row], &lo, &hi);
+            else expand_word_alu(raw[cw * p.P + row], &lo, &hi);
             uint4 *dst = reinterpret_cast<uint4 *>(sA) + (size_t)(2 * cw) * p.P + row;
             dst[0] = lo;
             dst[p.P] = hi;
@@ -690,10 +693,12 @@ bconv3x3_tensor_split_kernel(const TensorParams p)
                     if (!ok) break;
                 }
                 expand_a(p, table, raw0 + sbuf * raw_words, sA0 + sbuf * a_bytes, tid);
-                const int next = tile + tile_step;
-                if (next < p.n_tiles) prefetch_raw(p, next * kTileM, raw0 + (sbuf ^ 1) * raw_words, tid);
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_arrive(&bars[BAR_FULL_A0 + sbuf]);
+                // only now the words of the next tile: every thread reads back just its own copies, and
+                // the MMAs of this tile must not wait for loads they do not need
+                const int next = tile + tile_step;
+                if (next < p.n_tiles) prefetch_raw(p, next * kTileM, raw0 + (sbuf ^ 1) * raw_words, tid);
             }
             asm volatile("cp.async.wait_group 0;" ::: "memory");
         } else {
@@ -720,6 +725,226 @@ bconv3x3_tensor_split_kernel(const TensorParams p)
     }
 }
 
+
+// ---- pixels as the N dimension ---------------------------------------------------------------------
+// An i8 MMA streams (M + N) * 32 bytes of operands from shared memory for M * N * 32 products, so a
+// layer with few output channels is better served with the operands swapped: D[channel][pixel] =
+// W[channel][k] x X[pixel][k]^T, M = 128 channel rows (channels past Cout are zero words = +1 bytes,
+// their lanes are ignored), N = 256 pixels per MMA: four times the work per instruction of the M =
+// 128 pixels x N = 64 channels form for 1.5 times the operand bytes.  The shifted window now applies
+// to the B operand (same [chunk][position][16 bytes] buffer, same descriptors with N = 256).  A TMEM
+// lane is a channel and a column a pixel, which suits bit-packed output (a lane's 32 compare bits,
+// then a 32 x 32 bit transpose across the warp gives every lane the finished word of one pixel);
+// float and int32 output stay with the pixel-row form, whose lanes hold 32 consecutive channels of a
+// pixel.  Roles and barriers as in the split kernel, with 16 loader warps.
+constexpr int kTileN = 256;
+constexpr int kSwLoaders = 512;                                  // 16 loader warps: one position per thread for P <= 512
+constexpr int kSwThreads = kSwLoaders + kWorkers + 32;           // + 8 finisher warps + the issuer warp
+
+__device__ __forceinline__ void epilogue_swapped(const TensorParams &p, uint32_t tmem_d, const int32_t *sPix, int ch0,
+                                                 const int32_t *sThr, int ftid)
+{
+    const int warp = ftid >> 5, lane = ftid & 31;
+    const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31 = channels of this warp
+    if (ch0 + quarter * 32 >= p.Cout) return;     // whole warp: no real channel in its lanes
+    const int32_t thr = sThr[quarter * 32 + lane];  // INT32_MIN for pad channels: bit 0
+    // acc - pad_corr < thr  <=>  acc - (thr + pad_corr) < 0; the threshold is clamped to +-2^30 so that
+    // the subtraction cannot overflow (|acc| <= 9 * 32 * 32 here)
+    const int32_t thr_biased = max(-(1 << 30), min(1 << 30, thr > (1 << 30) ? (1 << 30) : thr + p.pad_corr));
+    const uint32_t lane_addr = tmem_d + ((uint32_t)(quarter * 32) << 16);
+    const int c_begin = (warp >> 2) * (kTileN / 2);
+    for (int c0 = c_begin; c0 < c_begin + kTileN / 2; c0 += 32) {
+        int32_t v[32];
+        tmem_ld32(lane_addr + (uint32_t)c0, v);
+        const int my_pix = sPix[c0 + lane];       // output pixel of column c0 + lane, or -1
+        // this lane's channel against the 32 pixels of the chunk, bit j = pixel c0 + j (the sign bit
+        // of acc - threshold, shifted in from the top: two chains of 16) ...
+        uint32_t m_lo = 0u, m_hi = 0u;
+#pragma unroll
+        for (int j = 15; j >= 0; --j) {
+            m_lo = __funnelshift_l((uint32_t)(v[j] - thr_biased), m_lo, 1);
+            m_hi = __funnelshift_l((uint32_t)(v[16 + j] - thr_biased), m_hi, 1);
+        }
+        uint32_t m = m_lo | (m_hi << 16);
+        // ... then a 32 x 32 bit transpose across the warp (five butterfly steps), after which lane j
+        // holds the output word of pixel c0 + j: bit i = channel 32*quarter + i
+#pragma unroll
+        for (int k = 16; k >= 1; k >>= 1) {
+            const uint32_t keep = k == 16 ? 0x0000FFFFu : k == 8 ? 0x00FF00FFu : k == 4 ? 0x0F0F0F0Fu : k == 2 ? 0x33333333u : 0x55555555u;
+            const uint32_t y = __shfl_xor_sync(0xffffffffu, m, k);
+            m = (lane & k) ? (((y >> k) & keep) | (m & ~keep)) : ((m & keep) | ((y & keep) << k));
+        }
+        if (my_pix >= 0) static_cast<uint32_t *>(p.out)[(int64_t)my_pix * p.Cow + ((ch0 >> 5) + quarter)] = m;
+    }
+}
+
+__global__ void __launch_bounds__(kSwThreads, 1)
+bconv3x3_tensor_swapped_kernel(const TensorParams p)  // p.P, p.n_tiles are for tiles of kTileN positions; p.n_blk = 128
+{
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    uint2 *table = reinterpret_cast<uint2 *>(smem_raw);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + 2048);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_raw + 2048 + 96);
+    int32_t *sThr = reinterpret_cast<int32_t *>(smem_raw + 2048 + 128);
+    // [4][kTileN] output pixel of a column, or -1.  A ring of four: the loaders of tile t+2 must not wait
+    // for the finishers of tile t (that would chain the three roles one after the other); slot t&3 is
+    // rewritten for tile t+4, whose X buffer is free only after the MMAs of tile t+2, which wait for
+    // the finishers of tile t.
+    int32_t *sPix = sThr + 128;
+    uint2 *offs = reinterpret_cast<uint2 *>(sPix + 4 * kTileN);         // [9*Cw] operand start offsets of a tile's MMAs
+    uint32_t *raw0 = reinterpret_cast<uint32_t *>(offs + ((9 * p.Cw + 1) / 2) * 2);
+    const int raw_words = ((p.P * p.Cw + 3) / 4) * 4;
+    uint8_t *sW = reinterpret_cast<uint8_t *>(raw0 + 2 * raw_words);    // A operand: [tap][2*Cw chunks][128 channels][16]
+    const size_t w_tap_bytes = (size_t)2 * p.Cw * 128 * 16;
+    uint8_t *sX0 = sW + 9 * w_tap_bytes;                                // B operand: 2 x [2*Cw chunks][P positions][16]
+    const size_t x_bytes = (size_t)2 * p.Cw * p.P * 16;
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int ch0 = blockIdx.y * 128;
+
+    for (int e = tid; e < 256; e += kSwThreads) {
+        uint32_t lo = 0, hi = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            lo |= (((e >> j) & 1) ? 0xFFu : 0x01u) << (8 * j);
+            hi |= (((e >> (j + 4)) & 1) ? 0xFFu : 0x01u) << (8 * j);
+        }
+        table[e] = make_uint2(lo, hi);
+    }
+    for (int e = tid; e < 128; e += kSwThreads) {
+        sThr[e] = ch0 + e < p.Cout ? __ldg(p.thr + ch0 + e) : INT32_MIN;
+    }
+    for (int e = tid; e < 9 * p.Cw; e += kSwThreads) {
+        const int tap = e / p.Cw, cw = e - tap * p.Cw;
+        // A (weights): the tap's block + K step (two planes of 128 rows); B (positions): window shift of
+        // the tap + K step (two planes of P rows).  Units of 16 bytes.
+        const uint32_t a_off = (uint32_t)(tap * 2 * p.Cw * 128 + 2 * cw * 128);
+        const uint32_t b_off = (uint32_t)((tap / 3) * p.Wp + (tap % 3) + 2 * cw * p.P);
+        offs[e] = make_uint2(a_off, b_off);
+    }
+    if (tid == 0) {
+        mbar_init(&bars[BAR_FULL_A0], kSwLoaders);   // here: positions expanded into X buffer 0 / 1
+        mbar_init(&bars[BAR_FULL_A1], kSwLoaders);
+        mbar_init(&bars[BAR_FULL_D0], 1);
+        mbar_init(&bars[BAR_FULL_D1], 1);
+        mbar_init(&bars[BAR_EMPTY_D0], kWorkers);
+        mbar_init(&bars[BAR_EMPTY_D1], kWorkers);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    // instruction descriptor: D = S32, A and B signed 8-bit, both K-major, N = 256, M = 128
+    const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    const uint32_t desc_hi = 8u | (1u << 14);
+    const int first_tile = blockIdx.x, tile_step = gridDim.x;
+    bool ok = true;
+
+    if (tid >= kSwLoaders + kWorkers) {
+        if (tid == kSwLoaders + kWorkers) {
+            uint32_t par_full_x[2] = {0, 0}, par_empty_d[2] = {0, 0};
+            const uint32_t a_lo0 = (smem_u32(sW) >> 4) | (128u << 16);
+            for (int tile = first_tile, it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+                const int sbuf = it & 1;
+                ok = mbar_wait_bounded(&bars[BAR_FULL_A0 + sbuf], par_full_x[sbuf]);
+                par_full_x[sbuf] ^= 1u;
+                if (ok && it >= 2) {
+                    ok = mbar_wait_bounded(&bars[BAR_EMPTY_D0 + sbuf], par_empty_d[sbuf]);
+                    par_empty_d[sbuf] ^= 1u;
+                }
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tmem_d = tmem_base + (uint32_t)(sbuf * kTileN);
+                const uint32_t b_lo0 = (smem_u32(sX0 + sbuf * x_bytes) >> 4) | ((uint32_t)p.P << 16);
+                uint32_t accumulate = 0;
+                issue_mmas(tmem_d, offs, 0, 9 * p.Cw, a_lo0, b_lo0, desc_hi, idesc, accumulate);
+                mma_commit(&bars[BAR_FULL_D0 + sbuf]);
+            }
+        }
+    } else {
+        if (tid < kSwLoaders && first_tile < p.n_tiles) prefetch_raw<kSwLoaders>(p, first_tile * kTileN, raw0, tid);
+        // weights of this channel block, once: packed [o][tap][cw] -> bytes [tap][chunk][channel][16]
+        const int words = 9 * 128 * p.Cw;
+        for (int e0 = tid; e0 < words; e0 += (kSwLoaders + kWorkers) * 8) {
+            uint32_t wv[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int e = e0 + k * (kSwLoaders + kWorkers);
+                const int ch = e & 127, tc = e >> 7;  // tc = tap*Cw + cw
+                const int tap = tc / p.Cw, cw = tc - tap * p.Cw;
+                wv[k] = (e < words && ch0 + ch < p.Cout) ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + tap) * p.Cw + cw) : 0u;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int e = e0 + k * (kSwLoaders + kWorkers);
+                if (e < words) {
+                    const int ch = e & 127, tc = e >> 7;
+                    const int tap = tc / p.Cw, cw = tc - tap * p.Cw;
+                    uint4 lo, hi;
+                    expand_word(table, wv[k], &lo, &hi);
+                    uint4 *dst = reinterpret_cast<uint4 *>(sW + tap * w_tap_bytes) + (size_t)(2 * cw) * 128 + ch;
+                    dst[0] = lo;
+                    dst[128] = hi;
+                }
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kSwLoaders + kWorkers) : "memory");
+
+        uint32_t par_full_d[2] = {0, 0};
+        if (tid < kSwLoaders) {
+            // ---- loaders: expand the positions of a tile, note which output pixel each column is ------
+            int tile = first_tile;
+            for (int it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+                const int sbuf = it & 1;
+                if (it >= 2) {  // X buffer sbuf was read by the MMAs of tile it-2
+                    ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + sbuf], par_full_d[sbuf]);
+                    par_full_d[sbuf] ^= 1u;
+                    if (!ok) break;
+                }
+                expand_a<kSwLoaders, false>(p, table, raw0 + sbuf * raw_words, sX0 + sbuf * x_bytes, tid);
+                if (tid < kTileN) {
+                    const int q = tile * kTileN + tid;  // one column per thread of the first eight loader warps
+                    const int rr = q / p.Wp, c = q - rr * p.Wp;
+                    const int n = rr / p.Hs, oh = rr - n * p.Hs;
+                    const bool col_ok = q < p.total_q && n < p.N && oh < p.H && c < p.W;
+                    sPix[(it & 3) * kTileN + tid] = col_ok ? (n * p.H + oh) * p.W + c : -1;
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(&bars[BAR_FULL_A0 + sbuf]);
+                const int next = tile + tile_step;
+                if (next < p.n_tiles) prefetch_raw<kSwLoaders>(p, next * kTileN, raw0 + (sbuf ^ 1) * raw_words, tid);
+            }
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        } else {
+            // ---- finishers -------------------------------------------------------------------------------
+            const int ftid = tid - kSwLoaders;
+            int tile = first_tile;
+            for (int it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+                const int sbuf = it & 1;
+                ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + sbuf], par_full_d[sbuf]);
+                par_full_d[sbuf] ^= 1u;
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                epilogue_swapped(p, tmem_base + (uint32_t)(sbuf * kTileN), sPix + (it & 3) * kTileN, ch0, sThr, ftid);
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                mbar_arrive(&bars[BAR_EMPTY_D0 + sbuf]);
+            }
+        }
+    }
+    if (!ok) g_tensor_status = 1;
+
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
 }  // namespace
 
 bool tensor_covers(const ConvGeom &g)
@@ -743,6 +968,36 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const uint
     p.out_type = g.out_type; p.activation = g.activation;
     p.vec_store = ((g.Cout & 3) == 0 && aligned(out, 16)) ? 1 : 0;
     if (p.P > 16383) return LCE_ERR_UNSUPPORTED;  // descriptor offsets are 14-bit counts of 16 bytes
+
+    // Bit-packed output with few output channels: pixels as the N dimension (M = 128 channel rows, N =
+    // 256 pixels per MMA), when the resident weights of a 128-channel block and two position buffers fit.
+    {
+        TensorParams q = p;
+        q.P = kTileN + 2 * p.Wp + 2;
+        q.n_tiles = (p.total_q + kTileN - 1) / kTileN;
+        q.n_blk = 128;
+        q.n_blk_log2 = 7;
+        q.tmem_cols = 512;
+        const size_t raw_b = (size_t)2 * (((size_t)q.P * g.Cw + 3) / 4) * 16;
+        const size_t need = (size_t)2048 + 128 + 128 * 4 + 4 * kTileN * 4 + 8 * (size_t)(((9 * g.Cw + 1) / 2) * 2) + raw_b +
+                            9 * (size_t)2 * g.Cw * 128 * 16 + 2 * (size_t)2 * g.Cw * q.P * 16;
+        bool swapped = g.out_type == LCE_OUT_BITPACKED && g.Cout <= 128 && need <= 226 * 1024 && q.P <= 16383 && (int64_t)g.N * g.H * g.W < (1ll << 31);
+#ifdef LCE_TUNING
+        if (const char *e = getenv("LCE_TENSOR_SWAP")) swapped = swapped && atoi(e) != 0;
+#endif
+        if (swapped) {
+            int sms2 = 148, dev = 0;
+            if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms2, cudaDevAttrMultiProcessorCount, dev);
+            const int n_blocks = (g.Cout + 127) / 128;
+            int ctas_x = sms2 / n_blocks;
+            if (ctas_x < 1) ctas_x = 1;
+            if (ctas_x > q.n_tiles) ctas_x = q.n_tiles;
+            if (cudaFuncSetAttribute(bconv3x3_tensor_swapped_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need) != cudaSuccess)
+                return LCE_ERR_CUDA;
+            bconv3x3_tensor_swapped_kernel<<<dim3((unsigned)ctas_x, (unsigned)n_blocks), kSwThreads, need, s>>>(q);
+            return launch_status();
+        }
+    }
 
     // Channel block (32..256, a power of two) and schedule, by a rule that matches what was
     // measured on the ResNet-18 shapes: weights resident if the full channel width (up to 256)

@@ -147,6 +147,8 @@ TENSOR_SHAPES = [
     (1, 7, 7, 64, 64), (2, 14, 14, 64, 64), (3, 9, 11, 70, 45), (1, 28, 28, 128, 128), (2, 7, 7, 512, 96),
     (1, 56, 56, 64, 64), (2, 14, 14, 256, 256), (1, 5, 5, 32, 300), (4, 7, 7, 512, 512), (2, 9, 9, 320, 40),
     (1, 1, 1, 3, 1), (5, 3, 40, 96, 130),
+    # bit-packed output with Cout <= 128 and few input words: the pixels-as-N schedule, several tiles and images
+    (2, 30, 30, 32, 128), (6, 20, 17, 64, 100), (1, 80, 80, 33, 33), (3, 40, 3, 96, 64),
 ]
 
 

@@ -36,7 +36,7 @@ UNIT = "binary-MAC/s"
 WORKLOAD = ("config 2: 3x3 one-padded Bconv2D sweep 56x56x64, 28x28x128, 14x14x256, 7x7x512 at batch 64 per GPU, "
             "float and bit-packed output each (8 launches per step), pre-packed inputs, load-time packed weights")
 
-# Derived compute ceiling of the chosen pipe (integer logic + popcount), see the design doc:
+# Derived compute ceiling of the chosen pipe (integer logic + popcount):
 # 64 logic lanes/clk/SM, 16.75 logic instructions per nine 32-bit word operations, 32 binary MACs per word.
 NCU_DRAM_BYTES_PER_LAUNCH = 1.7e6
 LOGIC_LANES_PER_CLK_PER_SM = 64

@@ -27,6 +27,8 @@
 #include <stdlib.h>
 
 #include "common.cuh"
+#include <atomic>
+
 #include "csa.cuh"
 #include "tiled_common.cuh"
 #include "bconv_kxk.cuh"
@@ -37,14 +39,35 @@ namespace {
 
 // ---- host side: launchers, the tile / range chooser, weight packing, plan and launch ----------------
 
+// The opt-in to more than 48 KB of dynamic shared memory is a driver call; it is made once per kernel,
+// device and size (a larger request later raises it), not on every launch.  One instance per kernel.
+struct SmemOptIn {
+    static constexpr int kDevices = 64;
+    std::atomic<size_t> granted[kDevices];
+    SmemOptIn() { for (auto &g : granted) g.store(0, std::memory_order_relaxed); }
+    template <typename Kernel>
+    bool ensure(Kernel kernel, size_t smem_bytes)
+    {
+        if (smem_bytes <= 48 * 1024) return true;
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess) return false;
+        const bool tracked = dev >= 0 && dev < kDevices;
+        if (tracked && granted[dev].load(std::memory_order_acquire) >= smem_bytes) return true;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess) return false;
+        if (tracked) {  // concurrent callers may both set the attribute; the recorded size only grows
+            size_t seen = granted[dev].load(std::memory_order_relaxed);
+            while (seen < smem_bytes && !granted[dev].compare_exchange_weak(seen, smem_bytes, std::memory_order_release)) {}
+        }
+        return true;
+    }
+};
+
 template <int TP>
 lce_status launch1x1(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStream_t s)
 {
     auto kernel = bconv1x1_kernel<TP>;
-    if (smem_bytes > 48 * 1024) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
-            return LCE_ERR_CUDA;
-    }
+    static SmemOptIn opted;
+    if (!opted.ensure(kernel, smem_bytes)) return LCE_ERR_CUDA;
     kernel<<<grid, kThreads, smem_bytes, s>>>(p);
     return launch_status();
 }
@@ -53,11 +76,8 @@ template <int KS, int STRIDE, int TP, int NW, bool F32 = false>
 lce_status launch_kxk(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStream_t s)
 {
     auto kernel = bconv3x3_kernel<KS, STRIDE, TP, NW, F32>;
-    if (smem_bytes > 48 * 1024) {
-        // opt in to the large dynamic shared memory carve-out
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
-            return LCE_ERR_CUDA;
-    }
+    static SmemOptIn opted;
+    if (!opted.ensure(kernel, smem_bytes)) return LCE_ERR_CUDA;
     kernel<<<grid, 32 * NW, smem_bytes, s>>>(p);
     return launch_status();
 }
@@ -240,6 +260,12 @@ lce_status launch_pack_weights_tiled(const ConvGeom &g, const uint32_t *w, uint3
 
 // Everything the launch needs that does not depend on the buffers: geometry fields of the kernel
 // parameters, the chosen variant and the launch dimensions.
+inline bool geom_equal(const ConvGeom &a, const ConvGeom &b)
+{
+    return a.N == b.N && a.H == b.H && a.W == b.W && a.Cin == b.Cin && a.Cout == b.Cout && a.KH == b.KH && a.KW == b.KW &&
+           a.sh == b.sh && a.sw == b.sw && a.padding == b.padding && a.out_type == b.out_type && a.activation == b.activation;
+}
+
 struct TiledPlan {
     bool pointwise;
     int nw, tp;
@@ -247,7 +273,7 @@ struct TiledPlan {
     dim3 grid;
 };
 
-static lce_status plan_tiled(const ConvGeom &g, bool f32_input, TiledParams *pp, TiledPlan *plan)
+static lce_status plan_tiled_uncached(const ConvGeom &g, bool f32_input, TiledParams *pp, TiledPlan *plan)
 {
     TiledParams &p = *pp;
     if (!tiled_covers(g)) return LCE_ERR_UNSUPPORTED;
@@ -341,6 +367,50 @@ static lce_status plan_tiled(const ConvGeom &g, bool f32_input, TiledParams *pp,
                 plan->smem_bytes, c.cost);
 #endif
     return LCE_OK;
+}
+
+// The plan depends on the geometry alone, and a network repeats few geometries: the last few plans
+// of each host thread are kept (the cost model walks a few hundred candidates per call otherwise).
+static lce_status plan_tiled(const ConvGeom &g, bool f32_input, TiledParams *pp, TiledPlan *plan)
+{
+#ifdef LCE_TUNING
+    return plan_tiled_uncached(g, f32_input, pp, plan);  // environment knobs may change between calls
+#else
+    struct Entry {
+        ConvGeom g;
+        bool f32_input, valid;
+        int device;  // the plan depends on the SM count of the current device
+        lce_status status;
+        TiledParams p;
+        TiledPlan plan;
+    };
+    constexpr int kEntries = 16;
+    static thread_local Entry cache[kEntries];
+    static thread_local int next = 0;
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) device = -1;
+    for (int i = 0; i < kEntries; ++i) {
+        const Entry &e = cache[i];
+        if (e.valid && e.f32_input == f32_input && e.device == device && geom_equal(e.g, g)) {
+            *pp = e.p;
+            *plan = e.plan;
+            return e.status;
+        }
+    }
+    Entry &e = cache[next];
+    next = (next + 1) % kEntries;
+    e.valid = false;
+    e.p = TiledParams{};
+    e.plan = TiledPlan{};
+    e.status = plan_tiled_uncached(g, f32_input, &e.p, &e.plan);
+    e.g = g;
+    e.f32_input = f32_input;
+    e.device = device;
+    e.valid = true;
+    *pp = e.p;
+    *plan = e.plan;
+    return e.status;
+#endif
 }
 
 lce_status tiled_plan_info(const ConvGeom &g, TiledPlanInfo *info)

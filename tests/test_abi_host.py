@@ -4,6 +4,7 @@ import ctypes
 import re
 from pathlib import Path
 
+import numpy as np
 import pytest
 
 import paper_2011_09398_b200 as lce
@@ -138,3 +139,22 @@ def test_plan_names_the_other_kernels(lib):
     with pytest.raises(lce.LceError) as e:
         _plan(1, 9, 9, 64, 64, 3, 2, kernel_choice=lce.KERNEL_TENSOR)                        # tensor path: stride 1 only
     assert e.value.status == 2
+
+
+def test_plans_are_remembered_per_geometry_not_mixed_up(lib):
+    """The library keeps the last few plans of a host thread: a repeated geometry must give the same
+    plan as the first time, with more distinct geometries in between than it keeps."""
+    rng = np.random.default_rng(5)
+    shapes = list(PLAN_SHAPES)
+    for _ in range(30):
+        k = int(rng.choice([1, 3, 5]))
+        shapes.append((int(rng.integers(1, 9)), int(rng.integers(5, 40)), int(rng.integers(5, 40)), int(rng.integers(1, 200)),
+                       int(rng.integers(1, 200)), k, int(rng.integers(1, 3))))
+    first = [_plan(*s)[0] for s in shapes]
+    again = [_plan(*s)[0] for s in reversed(shapes)][::-1]
+    assert first == again
+    # a field that is not part of the tile choice but is part of the geometry: output type and padding
+    a = _plan(4, 20, 20, 64, 96, 3, 1, out_type=lce.OUT_FLOAT32)[0]
+    b = _plan(4, 20, 20, 64, 96, 3, 1, padding=lce.PAD_VALID)[0]
+    c = _plan(4, 20, 20, 64, 96, 3, 1, out_type=lce.OUT_FLOAT32)[0]
+    assert a == c and b["kernel"] == lce.KERNEL_TILED

@@ -125,6 +125,7 @@ bconv1x1_kernel(const TiledParams p)
     const int K = p.Cin;
     const bool biased = p.out_type == LCE_OUT_FLOAT32 && K < kMaxBiasedK;
     const int Kb = biased ? K + kFloatBias : K;
+    const int epi = epilogue_mode(p, chan, biased);
     Weights124 k124;
     k124.one = p.N > 0 ? 1u : p.Cin;
     k124.two = p.N > 0 ? 2u : p.Cin;
@@ -193,7 +194,7 @@ bconv1x1_kernel(const TiledParams p)
                 int32_t v[kChanPerThread];
 #pragma unroll
                 for (int j = 0; j < kChanPerThread; ++j) v[j] = Kb - 2 * (int32_t)acc[i][j];
-                store_outputs(p, v, cp, m, m < m_end, cg, ch0, chan, biased);
+                store_outputs(p, v, cp, m, m < m_end, cg, ch0, chan, biased, epi);
             }
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");

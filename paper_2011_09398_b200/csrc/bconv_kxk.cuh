@@ -197,6 +197,7 @@ bconv3x3_kernel(const TiledParams p)
     // float output: accumulators carry the bias that makes int -> float one exact subtraction
     const bool biased = p.out_type == LCE_OUT_FLOAT32 && K < kMaxBiasedK;
     const int Kb = biased ? K + kFloatBias : K;
+    const int epi = epilogue_mode(p, chan, biased);
     Weights124 k124;
     k124.one = p.N > 0 ? 1u : p.Cin;  // opaque to the compiler: keeps the weighted sum on multiply-adds
     k124.two = p.N > 0 ? 2u : p.Cin;
@@ -296,6 +297,19 @@ bconv3x3_kernel(const TiledParams p)
         // ---- output transform -------------------------------------------------------------
         ChannelParams cp;
         load_channel_params(p, chan, cp);
+        if (epi == kEpiBits) {
+            // bit-packed output without a padding correction: nothing to decide per pixel
+#pragma unroll
+            for (int i = 0; i < TPX; ++i) {
+                const int m = base + i * pix_per_step + warp * pix_per_warp + px;
+                int32_t v[kChanPerThread];
+#pragma unroll
+                for (int j = 0; j < kChanPerThread; ++j)
+                    v[j] = Kb - 2 * (int32_t)(i < HX ? (acc[i][j] & 0xFFFFu) : (acc[i - HX][j] >> 16));
+                store_bits(p, v, cp.thr, m, m < m_end, cg, ch0);
+            }
+            return;
+        }
 #pragma unroll
         for (int i = 0; i < TPX; ++i) {
             const int m = base + i * pix_per_step + warp * pix_per_warp + px;
@@ -318,7 +332,7 @@ bconv3x3_kernel(const TiledParams p)
                     }
                 }
             }
-            store_outputs(p, v, cp, m, pix_ok, cg, ch0, chan, biased);
+            store_outputs(p, v, cp, m, pix_ok, cg, ch0, chan, biased, epi);
         }
     };
     for (int base = m0; base < m_end;) {

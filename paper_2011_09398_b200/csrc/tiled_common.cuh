@@ -208,27 +208,66 @@ __device__ __forceinline__ void load_channel_params(const TiledParams &p, int ch
 constexpr int32_t kFloatBias = 0x4B400000;
 constexpr int32_t kMaxBiasedK = 1 << 22;
 
+// The bit-packed output transform of one pixel: compare, pack the thread's 8 channels, combine the
+// 4 lanes that hold the 4 bytes of one output word, store.  Every lane of the warp must call it.
+__device__ __forceinline__ void store_bits(const TiledParams &p, const int32_t (&v)[kChanPerThread],
+                                           const int32_t (&thr)[kChanPerThread], int m, bool pix_ok, int cg, int ch0)
+{
+    uint32_t bits = 0u;
+#pragma unroll
+    for (int j = 0; j < kChanPerThread; ++j) bits |= (v[j] < thr[j] ? 1u : 0u) << j;
+    bits <<= 8 * (cg & 3);
+    bits |= __shfl_xor_sync(0xffffffffu, bits, 1);
+    bits |= __shfl_xor_sync(0xffffffffu, bits, 2);
+    const int word = (ch0 >> 5) + (cg >> 2);
+    if (pix_ok && (cg & 3) == 0 && word < p.Cow) static_cast<uint32_t *>(p.out)[(int64_t)m * p.Cow + word] = bits;
+}
+
+// What a thread's output transform will be, decided once per kernel: the plain float cases (biased
+// accumulators, all eight channels of the thread exist, 16-byte stores, no shortcut, no packed copy)
+// skip every test the general form makes per pixel.
+constexpr int kEpiGeneral = 0, kEpiFloat = 1, kEpiFloatRelu = 2, kEpiBits = 3;
+__device__ __forceinline__ int epilogue_mode(const TiledParams &p, int chan, bool biased)
+{
+    if (p.out_type == LCE_OUT_BITPACKED && p.padding != LCE_PAD_SAME_ZERO) return kEpiBits;
+    const bool plain = p.out_type == LCE_OUT_FLOAT32 && biased && p.residual == nullptr && p.out_packed == nullptr &&
+                       p.out != nullptr && (p.Cout & 3) == 0 && chan + kChanPerThread <= p.Cout;
+    return !plain ? kEpiGeneral : p.activation == LCE_ACT_RELU ? kEpiFloatRelu : kEpiFloat;
+}
+
 // Output transform of one pixel's 8 accumulators v (paper Section 3.2): float multiply-add after
 // the fused activation, threshold compare + bit-pack, or the raw accumulators.  Every lane of the
 // warp must call it (the bit-packed form combines 4 lanes with shuffles); pix_ok guards the store.
 __device__ __forceinline__ void store_outputs(const TiledParams &p, const int32_t (&v)[kChanPerThread],
                                               const ChannelParams &c, int m, bool pix_ok, int cg, int ch0, int chan,
-                                              bool biased)  // v carries + kFloatBias (float output with K < 2^22 only)
+                                              bool biased,  // v carries + kFloatBias (float output with K < 2^22 only)
+                                              int epi)      // epilogue_mode() of this thread
 {
     const float (&mult)[kChanPerThread] = c.mult;
     const float (&bias)[kChanPerThread] = c.bias;
     const int32_t (&thr)[kChanPerThread] = c.thr;
-    if (p.out_type == LCE_OUT_BITPACKED) {
-        uint32_t bits = 0u;
+    if (epi == kEpiFloat || epi == kEpiFloatRelu) {
+        // the common float case with every decision already taken: one exact FADD takes the bias off the
+        // accumulator, one FMA, two 16-byte stores
+        float f[kChanPerThread];
+        if (epi == kEpiFloat) {
 #pragma unroll
-        for (int j = 0; j < kChanPerThread; ++j) bits |= (v[j] < thr[j] ? 1u : 0u) << j;
-        // the 4 lanes cg&~3 .. cg|3 hold the 4 bytes of one output word
-        bits <<= 8 * (cg & 3);
-        bits |= __shfl_xor_sync(0xffffffffu, bits, 1);
-        bits |= __shfl_xor_sync(0xffffffffu, bits, 2);
-        const int word = (ch0 >> 5) + (cg >> 2);
-        if (pix_ok && (cg & 3) == 0 && word < p.Cow)
-            static_cast<uint32_t *>(p.out)[(int64_t)m * p.Cow + word] = bits;
+            for (int j = 0; j < kChanPerThread; ++j)
+                f[j] = __fmaf_rn(__fadd_rn(__int_as_float(v[j]), -12582912.0f), mult[j], bias[j]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < kChanPerThread; ++j)
+                f[j] = __fmaf_rn(__fadd_rn(__int_as_float(max(v[j], kFloatBias)), -12582912.0f), mult[j], bias[j]);
+        }
+        if (pix_ok) {
+            float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(p.out) + (int64_t)m * p.Cout + chan);
+            dst[0] = make_float4(f[0], f[1], f[2], f[3]);
+            dst[1] = make_float4(f[4], f[5], f[6], f[7]);
+        }
+        return;
+    }
+    if (p.out_type == LCE_OUT_BITPACKED) {
+        store_bits(p, v, thr, m, pix_ok, cg, ch0);
     } else if (p.out_type == LCE_OUT_FLOAT32) {
         float f[kChanPerThread];
 #pragma unroll

@@ -183,11 +183,20 @@ __device__ __forceinline__ void load_channel_params(const TiledParams &p, int ch
     if (chan + kChanPerThread <= p.Cout) {
         // all eight channels exist (every thread but those of a ragged last group): unconditional
         // loads of only what the output type needs
+        if (p.out_type == LCE_OUT_BITPACKED) {
 #pragma unroll
-        for (int j = 0; j < kChanPerThread; ++j) {
-            c.mult[j] = (p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.mult + chan + j) : 0.f;
-            c.bias[j] = (p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.bias + chan + j) : 0.f;
-            c.thr[j] = (p.out_type == LCE_OUT_BITPACKED) ? __ldg(p.thr + chan + j) : INT32_MIN;
+            for (int j = 0; j < kChanPerThread; ++j) {
+                c.mult[j] = 0.f;
+                c.bias[j] = 0.f;
+                c.thr[j] = __ldg(p.thr + chan + j);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < kChanPerThread; ++j) {
+                c.mult[j] = (p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.mult + chan + j) : 0.f;
+                c.bias[j] = (p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.bias + chan + j) : 0.f;
+                c.thr[j] = INT32_MIN;
+            }
         }
     } else {
 #pragma unroll

@@ -188,6 +188,23 @@ bconv1x1_kernel(const TiledParams p)
             }
             ChannelParams cp;
             load_channel_params(p, chan, cp);
+            if (epi == kEpiBits && K < (1 << 29)) {
+                // acc < thr  <=>  c - 2*count < 0 with c = K - thr (threshold clamped to [-K-1, K+1]):
+                // the output bit is the sign bit of one multiply-add, collected by a funnel shift
+                int32_t c[kChanPerThread];
+#pragma unroll
+                for (int j = 0; j < kChanPerThread; ++j) c[j] = K - max(-K - 1, min(K + 1, cp.thr[j]));
+#pragma unroll
+                for (int i = 0; i < TP; ++i) {
+                    const int m = base + i * kPixPerStep + warp * 4 + px;
+                    uint32_t bits = 0u;
+#pragma unroll
+                    for (int j = kChanPerThread - 1; j >= 0; --j)
+                        bits = __funnelshift_l((uint32_t)c[j] - 2u * acc[i][j], bits, 1);
+                    store_bits_byte(p, bits, m, m < m_end, cg, ch0);
+                }
+                continue;
+            }
 #pragma unroll
             for (int i = 0; i < TP; ++i) {
                 const int m = base + i * kPixPerStep + warp * 4 + px;

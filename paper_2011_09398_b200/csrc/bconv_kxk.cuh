@@ -297,8 +297,20 @@ bconv3x3_kernel(const TiledParams p)
         // ---- output transform -------------------------------------------------------------
         ChannelParams cp;
         load_channel_params(p, chan, cp);
+        if (epi == kEpiBits && K < 32768) {
+            // bit-packed output without a padding correction: nothing to decide per pixel, and the
+            // compare works on the packed counts directly
+            int32_t c15[kChanPerThread];
+            packed_compare_operands(cp.thr, K, c15);
+#pragma unroll
+            for (int i = 0; i < TPX; ++i) {
+                const int m = base + i * pix_per_step + warp * pix_per_warp + px;
+                const uint32_t bits = i < HX ? packed_compare_bits<false>(acc[i], c15) : packed_compare_bits<true>(acc[i - HX < 0 ? 0 : i - HX], c15);
+                store_bits_byte(p, bits, m, m < m_end, cg, ch0);
+            }
+            return;
+        }
         if (epi == kEpiBits) {
-            // bit-packed output without a padding correction: nothing to decide per pixel
 #pragma unroll
             for (int i = 0; i < TPX; ++i) {
                 const int m = base + i * pix_per_step + warp * pix_per_warp + px;

@@ -217,6 +217,41 @@ __device__ __forceinline__ void load_channel_params(const TiledParams &p, int ch
 constexpr int32_t kFloatBias = 0x4B400000;
 constexpr int32_t kMaxBiasedK = 1 << 22;
 
+// The thread's 8 output bits (channels 8*cg .. 8*cg+7 of the block) -> the output word they belong to:
+// the 4 lanes that hold the 4 bytes of a word combine them with two shuffles, one lane stores.
+__device__ __forceinline__ void store_bits_byte(const TiledParams &p, uint32_t bits, int m, bool pix_ok, int cg, int ch0)
+{
+    bits <<= 8 * (cg & 3);
+    bits |= __shfl_xor_sync(0xffffffffu, bits, 1);
+    bits |= __shfl_xor_sync(0xffffffffu, bits, 2);
+    const int word = (ch0 >> 5) + (cg >> 2);
+    if (pix_ok && (cg & 3) == 0 && word < p.Cow) static_cast<uint32_t *>(p.out)[(int64_t)m * p.Cow + word] = bits;
+}
+
+// Threshold compare on packed 16-bit counts without unpacking them (K < 32768).  With x the mismatch
+// count, acc = K - 2x < thr  <=>  c - 2x < 0 for c = K - thr, and, c' = c | 1 being odd, <=> c' - 2x < 0
+// with c' - 2x never zero.  For the pixel in the low half, (c' << 15) - (acc << 16) = 32768 (c' - 2 x_lo);
+// for the pixel in the high half, (c' << 15) - acc = 32768 (c' - 2 x_hi) - x_lo, which has the sign of
+// c' - 2 x_hi because that is odd and x_lo < 32768.  So the output bit is the sign bit of one
+// multiply-add, and a funnel shift collects it: two instructions per output instead of five.
+// The threshold is clamped to [-K-1, K+1] first (outside that range nothing changes), so c' << 15 fits.
+__device__ __forceinline__ void packed_compare_operands(const int32_t (&thr)[kChanPerThread], int K, int32_t (&c15)[kChanPerThread])
+{
+#pragma unroll
+    for (int j = 0; j < kChanPerThread; ++j) c15[j] = ((K - max(-K - 1, min(K + 1, thr[j]))) | 1) * 32768;
+}
+template <bool HIGH>
+__device__ __forceinline__ uint32_t packed_compare_bits(const uint32_t (&acc)[kChanPerThread], const int32_t (&c15)[kChanPerThread])
+{
+    uint32_t bits = 0u;
+#pragma unroll
+    for (int j = kChanPerThread - 1; j >= 0; --j) {
+        const uint32_t e = HIGH ? (uint32_t)c15[j] - acc[j] : (uint32_t)c15[j] - acc[j] * 65536u;
+        bits = __funnelshift_l(e, bits, 1);  // (bits << 1) | sign(e)
+    }
+    return bits;
+}
+
 // The bit-packed output transform of one pixel: compare, pack the thread's 8 channels, combine the
 // 4 lanes that hold the 4 bytes of one output word, store.  Every lane of the warp must call it.
 __device__ __forceinline__ void store_bits(const TiledParams &p, const int32_t (&v)[kChanPerThread],
@@ -225,11 +260,7 @@ __device__ __forceinline__ void store_bits(const TiledParams &p, const int32_t (
     uint32_t bits = 0u;
 #pragma unroll
     for (int j = 0; j < kChanPerThread; ++j) bits |= (v[j] < thr[j] ? 1u : 0u) << j;
-    bits <<= 8 * (cg & 3);
-    bits |= __shfl_xor_sync(0xffffffffu, bits, 1);
-    bits |= __shfl_xor_sync(0xffffffffu, bits, 2);
-    const int word = (ch0 >> 5) + (cg >> 2);
-    if (pix_ok && (cg & 3) == 0 && word < p.Cow) static_cast<uint32_t *>(p.out)[(int64_t)m * p.Cow + word] = bits;
+    store_bits_byte(p, bits, m, pix_ok, cg, ch0);
 }
 
 // What a thread's output transform will be, decided once per kernel: the plain float cases (biased

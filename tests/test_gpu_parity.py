@@ -374,3 +374,35 @@ def test_seeded_random_shapes_through_the_dispatcher(seed):
         act = int(rng.integers(0, 2))
         got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_FLOAT32, activation=act), mult=mult, bias=bias, packed=packed)
         assert float_close(got, acc, mult, bias, act) == 0, where
+
+
+# ---- thresholds at and beyond the ends of the accumulator range --------------------------------------
+
+@pytest.mark.parametrize("shape", [
+    # N, H, W, Cin, Cout, k, stride, padding
+    (2, 12, 12, 64, 64, 3, 1, lce.PAD_SAME_ONE), (1, 9, 10, 70, 40, 3, 2, lce.PAD_VALID), (2, 8, 8, 32, 96, 5, 1, lce.PAD_SAME_ONE),
+    (1, 6, 6, 128, 64, 1, 1, lce.PAD_VALID), (1, 7, 7, 64, 33, 3, 1, lce.PAD_SAME_ZERO), (1, 4, 4, 3700, 8, 3, 1, lce.PAD_SAME_ONE),
+])
+@pytest.mark.parametrize("packed", [False, True])
+def test_thresholds_at_the_ends_of_the_accumulator_range(shape, packed):
+    """Section 3.2: the bit-packed output is acc < threshold[c].  Accumulators of +K and -K are forced
+    (a channel equal to the all-ones input, its complement) and thresholds sit on, next to and far
+    beyond both ends, including INT32_MIN and INT32_MAX."""
+    N, H, W, Cin, Cout, k, s, padding = shape
+    rng = np.random.default_rng(abs(hash(shape)) % 2**32)
+    a = rand_pm1(rng, (N, H, W, Cin))
+    a[0] = 1                                   # image 0: all +1
+    w = rand_pm1(rng, (Cout, k, k, Cin))
+    w[0::4] = 1                                # acc = +K wherever the window lies inside image 0 (or on one-padding)
+    w[1::4] = -1                               # acc = -K there
+    K = k * k * Cin
+    edge = [-K - 2, -K - 1, -K, -K + 1, -K + 2, -1, 0, 1, K - 2, K - 1, K, K + 1, K + 2, -2**31, 2**31 - 1, -2**31 + 1, 2**31 - 2,
+            -65536, 65536, -32768, 32767]
+    thr = np.array([edge[(c // 4 + 5 * (c % 4)) % len(edge)] for c in range(Cout)], dtype=np.int64)
+    thr[2::4] = rng.integers(-K - 3, K + 4, size=len(thr[2::4]))
+    thr = thr.astype(np.int32)
+    acc = oracle.bconv2d_acc(a, w, (s, s), padding)
+    assert acc.max() == K and (acc.min() == -K)
+    got = run_bconv(oracle.bitpack_pm1(a), oracle.bitpack_pm1(w), dict(in_c=Cin, stride=(s, s), padding=padding, out_type=lce.OUT_BITPACKED),
+                    thr=thr, packed=packed)
+    np.testing.assert_array_equal(got, oracle.transform_bits(acc, thr))

@@ -68,17 +68,52 @@ bconv_patch_kernel(const PatchParams p)
         }
         __syncthreads();
         const int64_t stride = (int64_t)gridDim.x * kThreads;
-        for (int64_t m0 = (int64_t)blockIdx.x * kThreads + threadIdx.x; m0 < p.M; m0 += 2 * stride) {
+        // (image, row, column) of the thread's two pixels, advanced by 2*stride pixels per iteration
+        // with carries instead of two divisions per pixel
+        const int64_t step = 2 * stride;
+        const int step_ow = (int)(step % p.OW);
+        const int64_t step_rows = step / p.OW;
+        const int step_oh = (int)(step_rows % p.OH), step_n = (int)(step_rows / p.OH);
+        int pn[2], poh[2], pow_[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int64_t m = (int64_t)blockIdx.x * kThreads + threadIdx.x + q * stride;
+            const int64_t r = m / p.OW;
+            pow_[q] = (int)(m - r * p.OW);
+            pn[q] = (int)(r / p.OH);
+            poh[q] = (int)(r - (int64_t)pn[q] * p.OH);
+        }
+        for (int64_t m0 = (int64_t)blockIdx.x * kThreads + threadIdx.x; m0 < p.M; m0 += step) {
             const int64_t mm[2] = {m0, m0 + stride};
             uint32_t patch[2] = {0u, 0u};
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
+                const int n = pn[q], oh = poh[q], ow = pow_[q];
+                pow_[q] += step_ow;
+                poh[q] += step_oh;
+                pn[q] += step_n;
+                if (pow_[q] >= p.OW) { pow_[q] -= p.OW; ++poh[q]; }
+                if (poh[q] >= p.OH) { poh[q] -= p.OH; ++pn[q]; }
                 if (mm[q] >= p.M) continue;
-                const int m = (int)mm[q];
-                const int r = m / p.OW, ow = m - r * p.OW;
-                const int n = r / p.OH, oh = r - n * p.OH;
                 const int iy0 = oh * p.sh - p.pt, ix0 = ow * p.sw - p.pl;
                 const uint32_t *img = p.in + (int64_t)n * p.H * p.W;
+                if (taps == 9 && p.KW == 3 && iy0 >= 0 && iy0 + 2 < p.H && ix0 >= 0 && ix0 + 2 < p.W) {
+                    // 3x3 window inside the image (all but the border pixels): nine loads from three row
+                    // pointers, nothing to test per tap
+                    const uint32_t *r0 = img + iy0 * p.W + ix0, *r1 = r0 + p.W, *r2 = r1 + p.W;
+                    uint32_t v[9];
+#pragma unroll
+                    for (int kx = 0; kx < 3; ++kx) {
+                        v[kx] = __ldg(r0 + kx);
+                        v[3 + kx] = __ldg(r1 + kx);
+                        v[6 + kx] = __ldg(r2 + kx);
+                    }
+                    uint32_t acc_patch = 0u;
+#pragma unroll
+                    for (int t = 8; t >= 0; --t) acc_patch = (acc_patch << p.Cin) | (v[t] & mask);  // Horner: tap t ends at bit t*Cin
+                    patch[q] = acc_patch;
+                    continue;
+                }
                 for (int ky = 0; ky < p.KH; ++ky) {
                     const int iy = iy0 + ky;
                     for (int kx = 0; kx < p.KW; ++kx) {
@@ -91,10 +126,11 @@ bconv_patch_kernel(const PatchParams p)
             for (int wd = 0; wd < p.Cow; ++wd) {
                 uint32_t bits0 = 0u, bits1 = 0u;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
+                for (int j = 31; j >= 0; --j) {
+                    // popc > t  <=>  t - popc < 0: the output bit is a sign bit, shifted in from the top
                     const uint2 wt = sPair[wd * 32 + j];
-                    if ((int32_t)__popc(patch[0] ^ wt.x) > (int32_t)wt.y) bits0 |= 1u << j;
-                    if ((int32_t)__popc(patch[1] ^ wt.x) > (int32_t)wt.y) bits1 |= 1u << j;
+                    bits0 = __funnelshift_l(wt.y - (uint32_t)__popc(patch[0] ^ wt.x), bits0, 1);
+                    bits1 = __funnelshift_l(wt.y - (uint32_t)__popc(patch[1] ^ wt.x), bits1, 1);
                 }
                 static_cast<uint32_t *>(p.out)[mm[0] * p.Cow + wd] = bits0;
                 if (mm[1] < p.M) static_cast<uint32_t *>(p.out)[mm[1] * p.Cow + wd] = bits1;

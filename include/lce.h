@@ -164,6 +164,22 @@ typedef struct lce_bconv2d_plan_info {
 } lce_bconv2d_plan_info;
 lce_status lce_bconv2d_plan(const lce_bconv2d_desc *desc, lce_bconv2d_plan_info *plan);
 
+/* A convolution bound to its buffers: checked once, launched many times (Section 3.1: the paper's
+ * engine prepares every operator when the model is loaded and only runs it per inference).
+ * lce_bconv2d_plan_create takes the arguments of lce_bconv2d, makes all of its host-side checks,
+ * including that a kernel covers the shape, and on LCE_OK stores a handle in *plan; nothing is
+ * launched.  lce_plan_run launches the convolution on `stream` exactly as lce_bconv2d would (asynchronous,
+ * no allocation, capturable in a CUDA graph); it may be called any number of times, from one host
+ * thread at a time.  The handle is a small host object owned by the library until lce_plan_destroy
+ * (NULL is ignored); it holds the descriptor and the pointers, never the buffers, which stay the
+ * caller's and must outlive the runs.  Errors: those of lce_bconv2d; INVALID_ARG for a NULL plan. */
+typedef struct lce_plan lce_plan;
+lce_status lce_bconv2d_plan_create(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
+                                   const float *multiplier, const float *bias, const int32_t *thresholds,
+                                   void *output, lce_plan **plan);
+lce_status lce_plan_run(const lce_plan *plan, void *stream);
+void lce_plan_destroy(lce_plan *plan);
+
 /* Load-time weight packing (Section 3.2: the paper's BGEMM also re-arranges the weights ahead of
  * time for its access pattern; Section 3.1: weights are converted once, when the model is built).  Rewrites
  * the plain packed weights into the operand layout the tiled kernel copies straight into shared

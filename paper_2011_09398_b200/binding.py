@@ -63,6 +63,12 @@ def library() -> ctypes.CDLL:
         lib.lce_bconv2d_host_noalloc_max_bytes.argtypes = []
         lib.lce_bconv2d_host_noalloc.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, vp]
         lib.lce_bconv2d_host_noalloc.restype = ctypes.c_int
+        lib.lce_bconv2d_plan_create.argtypes = [ctypes.POINTER(BConv2dDesc), vp, vp, vp, vp, vp, vp, ctypes.POINTER(vp)]
+        lib.lce_bconv2d_plan_create.restype = ctypes.c_int
+        lib.lce_plan_run.argtypes = [vp, vp]
+        lib.lce_plan_run.restype = ctypes.c_int
+        lib.lce_plan_destroy.argtypes = [vp]
+        lib.lce_plan_destroy.restype = None
         lib.lce_bmaxpool.argtypes = [vp, vp] + [i32] * 9 + [vp]
         lib.lce_add_f32.argtypes = [vp, vp, vp, i64, vp]
         lib.lce_probe_pipe.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), vp]
@@ -206,6 +212,43 @@ def lce_bconv2d_plan(desc: BConv2dDesc) -> dict:
     fn.restype = ctypes.c_int
     _check(fn(ctypes.byref(desc), ctypes.byref(info)), "lce_bconv2d_plan")
     return {n: getattr(info, n) for n, _ in BConv2dPlanInfo._fields_}
+
+
+class BConv2dPlan:
+    """Handle of lce_bconv2d_plan_create; keeps the bound tensors alive.  `out` is the output tensor."""
+
+    def __init__(self, handle: int, tensors, out: torch.Tensor):
+        self.handle, self._tensors, self.out = handle, tensors, out
+
+
+def lce_bconv2d_plan_create(desc: BConv2dDesc, input: torch.Tensor, weights: torch.Tensor,
+                            multiplier: Optional[torch.Tensor] = None, bias: Optional[torch.Tensor] = None,
+                            thresholds: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None) -> BConv2dPlan:
+    """lce_bconv2d bound to its buffers: all checks now, launches later with lce_plan_run."""
+    oh, ow = lce_bconv2d_out_shape(desc)
+    out_dtype = torch.float32 if desc.out_type == OUT_FLOAT32 else torch.int32
+    if out is None:
+        last = _words(desc.out_c) if desc.out_type == OUT_BITPACKED else desc.out_c
+        out = torch.empty((desc.batch, oh, ow, last), dtype=out_dtype, device=input.device)
+    handle = ctypes.c_void_p()
+    _check(library().lce_bconv2d_plan_create(
+        ctypes.byref(desc), _dev(input, torch.int32, "input"), _dev(weights, torch.int32, "weights"),
+        _dev(multiplier, torch.float32, "multiplier") if multiplier is not None else None,
+        _dev(bias, torch.float32, "bias") if bias is not None else None,
+        _dev(thresholds, torch.int32, "thresholds") if thresholds is not None else None,
+        _dev(out, out_dtype, "out"), ctypes.byref(handle)), "lce_bconv2d_plan_create")
+    return BConv2dPlan(handle.value, (input, weights, multiplier, bias, thresholds), out)
+
+
+def lce_plan_run(plan: BConv2dPlan) -> torch.Tensor:
+    """Launches the planned convolution on torch's current stream; returns the plan's output tensor."""
+    _check(library().lce_plan_run(plan.handle, _stream()), "lce_plan_run")
+    return plan.out
+
+
+def lce_plan_destroy(plan: BConv2dPlan) -> None:
+    library().lce_plan_destroy(plan.handle)
+    plan.handle = None
 
 
 def lce_bconv2d_fused(desc: BConv2dDesc, input, weights, multiplier, bias, residual=None, out_float=None,

@@ -2,6 +2,8 @@
 // host-buffer forms).  All argument checks happen here, before anything is launched.
 #include "common.cuh"
 
+#include <new>
+
 namespace lce {
 namespace {
 
@@ -155,6 +157,52 @@ extern "C" lce_status lce_bconv2d(const lce_bconv2d_desc *desc, const uint32_t *
         return LCE_ERR_ALIGNMENT;
     return dispatch(desc, g, input, weights, multiplier, bias, thresholds, output, static_cast<cudaStream_t>(stream));
 }
+
+// ---- plan objects: the checks of lce_bconv2d once, the launch many times ---------------------------
+struct lce_plan {
+    lce_bconv2d_desc desc;
+    lce::ConvGeom geom;
+    const uint32_t *input, *weights;
+    const float *multiplier, *bias;
+    const int32_t *thresholds;
+    void *output;
+};
+
+extern "C" lce_status lce_bconv2d_plan_create(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
+                                              const float *multiplier, const float *bias, const int32_t *thresholds,
+                                              void *output, lce_plan **plan)
+{
+    using namespace lce;
+    if (!plan) return LCE_ERR_INVALID_ARG;
+    *plan = nullptr;
+    ConvGeom g;
+    lce_status st = check_conv_args(desc, &g, input, weights, multiplier, bias, thresholds, output);
+    if (st != LCE_OK) return st;
+    if (!aligned(input, 4) || !aligned(weights, 4) || !aligned(output, 4) ||
+        (multiplier && !aligned(multiplier, 4)) || (bias && !aligned(bias, 4)) ||
+        (thresholds && !aligned(thresholds, 4)))
+        return LCE_ERR_ALIGNMENT;
+    lce_bconv2d_plan_info info;
+    st = lce_bconv2d_plan(desc, &info);  // is there a kernel for this shape (and for a forced kernel choice)?
+    if (st != LCE_OK) return st;
+    lce_plan *h = new (std::nothrow) lce_plan;
+    if (!h) return LCE_ERR_CUDA;
+    h->desc = *desc;
+    h->geom = g;
+    h->input = input; h->weights = weights; h->multiplier = multiplier; h->bias = bias; h->thresholds = thresholds;
+    h->output = output;
+    *plan = h;
+    return LCE_OK;
+}
+
+extern "C" lce_status lce_plan_run(const lce_plan *plan, void *stream)
+{
+    if (!plan) return LCE_ERR_INVALID_ARG;
+    return lce::dispatch(&plan->desc, plan->geom, plan->input, plan->weights, plan->multiplier, plan->bias, plan->thresholds,
+                         plan->output, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" void lce_plan_destroy(lce_plan *plan) { delete plan; }
 
 extern "C" lce_status lce_bconv2d_fused(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
                                         const float *multiplier, const float *bias, const float *residual,

@@ -158,3 +158,20 @@ def test_plans_are_remembered_per_geometry_not_mixed_up(lib):
     b = _plan(4, 20, 20, 64, 96, 3, 1, padding=lce.PAD_VALID)[0]
     c = _plan(4, 20, 20, 64, 96, 3, 1, out_type=lce.OUT_FLOAT32)[0]
     assert a == c and b["kernel"] == lce.KERNEL_TILED
+
+
+def test_plan_objects_check_their_arguments_on_the_host(lib):
+    d = lce.make_desc(1, 4, 4, 32, 32)
+    fake = ctypes.c_void_p(256)  # never dereferenced: nothing is launched by plan_create
+    handle = ctypes.c_void_p()
+    assert lib.lce_bconv2d_plan_create(ctypes.byref(d), None, fake, fake, fake, None, fake, ctypes.byref(handle)) == 1
+    assert handle.value is None
+    assert lib.lce_bconv2d_plan_create(ctypes.byref(d), fake, fake, fake, fake, None, fake, None) == 1      # nowhere to put the handle
+    assert lib.lce_bconv2d_plan_create(ctypes.byref(d), ctypes.c_void_p(258), fake, fake, fake, None, fake, ctypes.byref(handle)) == 3
+    forced = lce.make_desc(1, 9, 9, 64, 64, (3, 3), (2, 2), kernel_choice=lce.KERNEL_TENSOR)                   # tensor path: stride 1 only
+    assert lib.lce_bconv2d_plan_create(ctypes.byref(forced), fake, fake, fake, fake, None, fake, ctypes.byref(handle)) == 2
+    assert lib.lce_bconv2d_plan_create(ctypes.byref(d), fake, fake, fake, fake, None, fake, ctypes.byref(handle)) == 0
+    assert handle.value
+    lib.lce_plan_destroy(handle)
+    lib.lce_plan_destroy(None)                                                                                # ignored
+    assert lib.lce_plan_run(None, None) == 1

@@ -406,3 +406,30 @@ def test_thresholds_at_the_ends_of_the_accumulator_range(shape, packed):
     got = run_bconv(oracle.bitpack_pm1(a), oracle.bitpack_pm1(w), dict(in_c=Cin, stride=(s, s), padding=padding, out_type=lce.OUT_BITPACKED),
                     thr=thr, packed=packed)
     np.testing.assert_array_equal(got, oracle.transform_bits(acc, thr))
+
+
+def test_plan_object_runs_like_the_direct_call_and_inside_a_cuda_graph():
+    """lce_bconv2d_plan_create / lce_plan_run: the same launch as lce_bconv2d, capturable in a graph."""
+    rng = np.random.default_rng(77)
+    N, H, W, Cin, Cout = 3, 13, 11, 96, 72
+    a, w = rand_pm1(rng, (N, H, W, Cin)), rand_pm1(rng, (Cout, 3, 3, Cin))
+    acc = oracle.bconv2d_acc(a, w, (1, 1), lce.PAD_SAME_ONE)
+    thr = np.rint(np.sqrt(9 * Cin) * rng.standard_normal(Cout)).astype(np.int32)
+    desc = lce.make_desc(N, H, W, Cin, Cout, (3, 3), (1, 1), lce.PAD_SAME_ONE, lce.OUT_BITPACKED, lce.ACT_NONE, lce.KERNEL_AUTO, 1)
+    a_dev, w_dev = to_dev_words(oracle.bitpack_pm1(a)), to_dev_words(oracle.bitpack_pm1(w))
+    w_img = lce.lce_bconv2d_pack_weights(desc, w_dev)
+    plan = lce.lce_bconv2d_plan_create(desc, a_dev, w_img, thresholds=to_dev(thr))
+    want = oracle.transform_bits(acc, thr)
+    out = lce.lce_plan_run(plan)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(out.cpu().numpy().view(np.uint32), want)
+    out.zero_()
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            lce.lce_plan_run(plan)
+        graph.replay()
+        stream.synchronize()
+    np.testing.assert_array_equal(out.cpu().numpy().view(np.uint32), want)
+    lce.lce_plan_destroy(plan)

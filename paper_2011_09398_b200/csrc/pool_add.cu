@@ -30,6 +30,19 @@ bmaxpool_kernel(const uint32_t *__restrict__ in, uint32_t *__restrict__ out, int
             const int32_t ow = e / cv, j = (e - ow * cv) * VEC;
             const int32_t ix0 = ow * sw - pl;
             uint32_t acc[VEC];
+            if (PH == 2 && PW == 2 && iy0 >= 0 && iy0 + 1 < H && ix0 >= 0 && ix0 + 1 < W) {
+                // the usual 2x2 window, inside the image: four independent loads in flight, three ANDs
+                const uint32_t *s0 = img + ((int64_t)iy0 * W + ix0) * Cw + j, *s1 = s0 + (int64_t)W * Cw;
+                if (VEC == 4) {
+                    const uint4 a = __ldcs(reinterpret_cast<const uint4 *>(s0)), b = __ldcs(reinterpret_cast<const uint4 *>(s0 + Cw));
+                    const uint4 c = __ldcs(reinterpret_cast<const uint4 *>(s1)), d = __ldcs(reinterpret_cast<const uint4 *>(s1 + Cw));
+                    __stcs(reinterpret_cast<uint4 *>(orow + (int64_t)ow * Cw + j),
+                           make_uint4(a.x & b.x & c.x & d.x, a.y & b.y & c.y & d.y, a.z & b.z & c.z & d.z, a.w & b.w & c.w & d.w));
+                } else {
+                    orow[(int64_t)ow * Cw + j] = __ldcs(s0) & __ldcs(s0 + Cw) & __ldcs(s1) & __ldcs(s1 + Cw);
+                }
+                continue;
+            }
 #pragma unroll
             for (int v = 0; v < VEC; ++v) acc[v] = 0xffffffffu;
             for (int32_t ky = 0; ky < PH; ++ky) {

@@ -66,7 +66,7 @@ struct TensorParams {
     int32_t tmem_cols;   // power of two >= max(32, n_blk)
     int32_t pad_corr;    // 9 * (32*Cw - Cin): what the zero pad bits (+1 * +1) add to every accumulator
     int32_t out_type, activation;
-    int32_t vec_store;   // float / int32 rows may be written with 128-bit stores
+    int32_t vec_store;   // float / int32 rows may be written with 128-bit stores (2: with 256-bit stores)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -234,6 +234,15 @@ __device__ __forceinline__ void issue_mmas(uint32_t tmem, const uint2 *offs, int
     }
 }
 
+// Threshold as the pixel-row epilogue compares it: acc_raw - pad_corr < thr  <=>  acc_raw - (thr + pad_corr) < 0,
+// with thr clamped to +-2^30 (|acc| <= 9 * 32 * 32, so nothing changes) and channels that do not exist
+// given the lowest value, which no accumulator is below: their bits are 0.
+__device__ __forceinline__ int32_t biased_threshold(const TensorParams &p, bool real_channel, int channel)
+{
+    const int32_t t = real_channel ? __ldg(p.thr + channel) : INT32_MIN;
+    return max(-(1 << 30), min(1 << 30, t)) + p.pad_corr;
+}
+
 // Output transform of one tile: thread = TMEM lane = GEMM row; 32 channels per TMEM load.
 __device__ __forceinline__ void epilogue(const TensorParams &p, uint32_t tmem_base, int q0, int ch0, const float *sMult,
                                          const float *sBias, const int32_t *sThr, int tid)
@@ -253,24 +262,47 @@ __device__ __forceinline__ void epilogue(const TensorParams &p, uint32_t tmem_ba
     for (int c0 = c_begin; c0 < c_end; c0 += 32) {
         int32_t v[32];
         tmem_ld32(lane_addr + (uint32_t)c0, v);
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] -= p.pad_corr;
         const int o0 = ch0 + c0;
         if (p.out_type == LCE_OUT_BITPACKED) {
+            // sThr holds threshold + pad correction, clamped so that the difference cannot overflow (pad
+            // channels: the lowest value, bit 0): the output bit is the sign of raw accumulator - sThr,
+            // shifted in from the top; the array is read four channels at a time (c0 is a multiple of 32)
             uint32_t bits = 0u;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) bits |= (v[j] < sThr[c0 + j] ? 1u : 0u) << j;  // sThr of pad channels = INT32_MIN
+            for (int j = 28; j >= 0; j -= 4) {
+                const int4 t4 = *reinterpret_cast<const int4 *>(sThr + c0 + j);
+                bits = __funnelshift_l((uint32_t)(v[j + 3] - t4.w), bits, 1);
+                bits = __funnelshift_l((uint32_t)(v[j + 2] - t4.z), bits, 1);
+                bits = __funnelshift_l((uint32_t)(v[j + 1] - t4.y), bits, 1);
+                bits = __funnelshift_l((uint32_t)(v[j] - t4.x), bits, 1);
+            }
             if (row_ok && o0 < p.Cout) static_cast<uint32_t *>(p.out)[pix * p.Cow + (o0 >> 5)] = bits;
-        } else if (p.out_type == LCE_OUT_FLOAT32) {
-            float f[32];
+            continue;
+        }
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int32_t a = (p.activation == LCE_ACT_RELU && v[j] < 0) ? 0 : v[j];
-                f[j] = __fmaf_rn((float)a, sMult[c0 + j], sBias[c0 + j]);
+        for (int j = 0; j < 32; ++j) v[j] -= p.pad_corr;
+        if (p.out_type == LCE_OUT_FLOAT32) {
+            float f[32];
+            const int32_t floor_v = p.activation == LCE_ACT_RELU ? 0 : INT32_MIN;
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+                // c0 is a multiple of 32: the per-channel arrays are read four floats at a time
+                const float4 m4 = *reinterpret_cast<const float4 *>(sMult + c0 + j), b4 = *reinterpret_cast<const float4 *>(sBias + c0 + j);
+                f[j] = __fmaf_rn((float)max(v[j], floor_v), m4.x, b4.x);
+                f[j + 1] = __fmaf_rn((float)max(v[j + 1], floor_v), m4.y, b4.y);
+                f[j + 2] = __fmaf_rn((float)max(v[j + 2], floor_v), m4.z, b4.z);
+                f[j + 3] = __fmaf_rn((float)max(v[j + 3], floor_v), m4.w, b4.w);
             }
             if (row_ok) {
                 float *dst = static_cast<float *>(p.out) + pix * p.Cout + o0;
-                if (p.vec_store && o0 + 32 <= p.Cout) {
+                if (p.vec_store == 2 && o0 + 32 <= p.Cout) {
+                    // one whole 32-byte sector per lane and instruction
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8)
+                        asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst + j), "f"(f[j]), "f"(f[j + 1]), "f"(f[j + 2]),
+                                     "f"(f[j + 3]), "f"(f[j + 4]), "f"(f[j + 5]), "f"(f[j + 6]), "f"(f[j + 7])
+                                     : "memory");
+                } else if (p.vec_store && o0 + 32 <= p.Cout) {
 #pragma unroll
                     for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4 *>(dst + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
                 } else {
@@ -352,7 +384,7 @@ bconv3x3_tensor_kernel(const TensorParams p)
         const bool ok = ch0 + e < p.Cout;
         sMult[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.mult + ch0 + e) : 0.f;
         sBias[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.bias + ch0 + e) : 0.f;
-        sThr[e] = (ok && p.out_type == LCE_OUT_BITPACKED) ? __ldg(p.thr + ch0 + e) : INT32_MIN;  // pad bits -> 0
+        sThr[e] = biased_threshold(p, ok && p.out_type == LCE_OUT_BITPACKED, ch0 + e);
     }
     for (int e = tid; e < 9 * p.Cw; e += kThreads) {
         const int tap = e / p.Cw, cw = e - tap * p.Cw;
@@ -597,7 +629,7 @@ bconv3x3_tensor_split_kernel(const TensorParams p)
         const bool ok = ch0 + e < p.Cout;
         sMult[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.mult + ch0 + e) : 0.f;
         sBias[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.bias + ch0 + e) : 0.f;
-        sThr[e] = (ok && p.out_type == LCE_OUT_BITPACKED) ? __ldg(p.thr + ch0 + e) : INT32_MIN;
+        sThr[e] = biased_threshold(p, ok && p.out_type == LCE_OUT_BITPACKED, ch0 + e);
     }
     for (int e = tid; e < 9 * p.Cw; e += kSplitThreads) {
         const int tap = e / p.Cw, cw = e - tap * p.Cw;
@@ -966,7 +998,7 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const uint
     p.n_tiles = (p.total_q + kTileM - 1) / kTileM;
     p.pad_corr = 9 * (32 * g.Cw - g.Cin);
     p.out_type = g.out_type; p.activation = g.activation;
-    p.vec_store = ((g.Cout & 3) == 0 && aligned(out, 16)) ? 1 : 0;
+    p.vec_store = ((g.Cout & 7) == 0 && aligned(out, 32)) ? 2 : ((g.Cout & 3) == 0 && aligned(out, 16)) ? 1 : 0;
     if (p.P > 16383) return LCE_ERR_UNSUPPORTED;  // descriptor offsets are 14-bit counts of 16 bytes
 
     // Bit-packed output with few output channels: pixels as the N dimension (M = 128 channel rows, N =

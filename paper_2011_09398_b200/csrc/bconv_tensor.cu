@@ -521,7 +521,14 @@ bconv3x3_tensor_kernel(const TensorParams p)
                 mbar_arrive(&bars[BAR_EMPTY_D0 + cur]);
             }
         } else {
-            const int wpt = (words_per_tap + kWorkers - 1) / kWorkers;  // <= kMaxWordsPerThread (host-checked)
+            // A thread expands consecutive channel words of ONE channel (kWorkers / n_blk threads share a
+            // channel): its loads of a tap are then one or two whole 32-byte sectors instead of eight
+            // words in eight different sectors, and its shared-memory stores stay channel-fastest.
+            const int tpc = kWorkers >> p.n_blk_log2;            // threads per channel: 1, 2, 4 or 8
+            const int wpt = (p.Cw + tpc - 1) / tpc;              // <= kMaxWordsPerThread (host-checked)
+            const int my_ch = tid & (p.n_blk - 1), cw0 = (tid >> p.n_blk_log2) * wpt;
+            const bool ch_real = ch0 + my_ch < p.Cout;
+            const bool vec_w = (p.Cw & 3) == 0 && (wpt & 3) == 0 && (reinterpret_cast<uintptr_t>(p.w) & 15) == 0;
             int g = 0;  // taps produced so far
             for (int it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
                 const int next = tile + tile_step;
@@ -533,12 +540,18 @@ bconv3x3_tensor_kernel(const TensorParams p)
 
                 uint32_t wv[kMaxWordsPerThread];
                 auto load_tap = [&](int tap) {
+                    const uint32_t *src = p.w + ((int64_t)(ch0 + (ch_real ? my_ch : 0)) * 9 + tap) * p.Cw + cw0;
+                    if (vec_w) {
 #pragma unroll
-                    for (int k = 0; k < kMaxWordsPerThread; ++k) {
-                        const int e = tid + k * kWorkers;  // channel fastest: conflict-free shared stores
-                        const int ch = e & (p.n_blk - 1), cw = e >> p.n_blk_log2;
-                        wv[k] = (k < wpt && e < words_per_tap && ch0 + ch < p.Cout)
-                                    ? __ldg(p.w + ((int64_t)(ch0 + ch) * 9 + tap) * p.Cw + cw) : 0u;
+                        for (int k = 0; k < kMaxWordsPerThread; k += 4) {
+                            uint4 q = make_uint4(0u, 0u, 0u, 0u);
+                            if (ch_real && k < wpt && cw0 + k < p.Cw) q = __ldg(reinterpret_cast<const uint4 *>(src + k));
+                            wv[k] = q.x; wv[k + 1] = q.y; wv[k + 2] = q.z; wv[k + 3] = q.w;
+                        }
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < kMaxWordsPerThread; ++k)
+                            wv[k] = (ch_real && k < wpt && cw0 + k < p.Cw) ? __ldg(src + k) : 0u;
                     }
                 };
                 load_tap(0);
@@ -552,9 +565,8 @@ bconv3x3_tensor_kernel(const TensorParams p)
                     uint8_t *dstB = sB + sb * b_tap_bytes;
 #pragma unroll
                     for (int k = 0; k < kMaxWordsPerThread; ++k) {
-                        const int e = tid + k * kWorkers;
-                        if (k < wpt && e < words_per_tap) {
-                            const int ch = e & (p.n_blk - 1), cw = e >> p.n_blk_log2;
+                        if (k < wpt && cw0 + k < p.Cw) {
+                            const int ch = my_ch, cw = cw0 + k;
                             uint4 lo, hi;
                             expand_word_alu(wv[k], &lo, &hi);
                             uint4 *dst = reinterpret_cast<uint4 *>(dstB) + (size_t)(2 * cw) * p.n_blk + ch;

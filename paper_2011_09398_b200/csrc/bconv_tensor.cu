@@ -779,8 +779,8 @@ bconv3x3_tensor_split_kernel(const TensorParams p)
 // to the B operand (same [chunk][position][16 bytes] buffer, same descriptors with N = 256).  A TMEM
 // lane is a channel and a column a pixel, which suits bit-packed output (a lane's 32 compare bits,
 // then a 32 x 32 bit transpose across the warp gives every lane the finished word of one pixel);
-// float and int32 output stay with the pixel-row form, whose lanes hold 32 consecutive channels of a
-// pixel.  Roles and barriers as in the split kernel, with 16 loader warps.
+// float and int32 output of up to 64 channels go through a shared-memory stage (see
+// epilogue_swapped_staged), wider ones stay with the pixel-row form.  Roles and barriers as in the split kernel, with 16 loader warps.
 constexpr int kTileN = 256;
 constexpr int kSwLoaders = 512;                                  // 16 loader warps: one position per thread for P <= 512
 constexpr int kSwThreads = kSwLoaders + kWorkers + 32;           // + 8 finisher warps + the issuer warp
@@ -822,6 +822,97 @@ __device__ __forceinline__ void epilogue_swapped(const TensorParams &p, uint32_t
     }
 }
 
+// Float / int32 output of the pixels-as-N kernel (Cout <= 64): a lane holds ONE channel of 32 pixels, the
+// output wants 64 consecutive channels per pixel.  The values go through a shared-memory stage
+// [256 pixels][64 channels]: the warps that own real channels write it (lanes = consecutive channels:
+// no bank conflicts; the multiplier and bias of a lane's channel sit in two registers), all eight
+// finisher warps then copy whole pixel rows out with 16-byte accesses, two rows per instruction.
+// Two named-barrier phases per tile (256 finisher threads): stage complete / stage free again.
+constexpr int kStageCh = 64;
+__device__ __forceinline__ void epilogue_swapped_staged(const TensorParams &p, uint32_t tmem_d, const int32_t *sPix, int ch0,
+                                                        uint32_t *stage, float mult, float bias, int ftid, uint64_t *empty_d)
+{
+    const int warp = ftid >> 5, lane = ftid & 31;
+    const int quarter = warp & 3;
+    if (ch0 + quarter * 32 < p.Cout) {
+        const uint32_t lane_addr = tmem_d + ((uint32_t)(quarter * 32) << 16);
+        const int c_begin = (warp >> 2) * (kTileN / 2);
+        const bool relu = p.activation == LCE_ACT_RELU;
+        uint32_t *col = stage + quarter * 32 + lane;
+        for (int c0 = c_begin; c0 < c_begin + kTileN / 2; c0 += 32) {
+            int32_t v[32];
+            tmem_ld32(lane_addr + (uint32_t)c0, v);
+            if (p.out_type == LCE_OUT_FLOAT32) {
+                // int -> float without the conversion unit (the active finisher warps share two of the four
+                // SM sub-partitions): v + 0x4B400000 is the bit pattern of 12582912 + v for |v| < 2^22, so one
+                // exact FADD gives (float)v; ReLU is a max against the same constant
+                const int32_t add = 0x4B400000 - p.pad_corr;
+                if (relu) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        col[(c0 + j) * kStageCh] = __float_as_uint(
+                            __fmaf_rn(__fadd_rn(__int_as_float(max(v[j] + add, 0x4B400000)), -12582912.0f), mult, bias));
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        col[(c0 + j) * kStageCh] = __float_as_uint(__fmaf_rn(__fadd_rn(__int_as_float(v[j] + add), -12582912.0f), mult, bias));
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) col[(c0 + j) * kStageCh] = (uint32_t)(v[j] - p.pad_corr);
+            }
+        }
+    }
+    // the accumulator buffer has been read: hand it back before the copy out
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    mbar_arrive(empty_d);
+    if (p.Cout == kStageCh) {
+        // A stage row is an output row: runs of consecutive valid columns are contiguous in both, so the
+        // copy engine moves them (one bulk copy per run, at most 32 columns = 8 KB) while the warps go
+        // on to the next tile.  The caller waits for the reads of the stage before it is written again.
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("bar.sync 2, %0;" ::"n"(kWorkers) : "memory");  // the stage holds the whole tile
+        const int col_px = warp * 32 + lane;
+        const int pix = sPix[col_px];
+        const int prev = __shfl_up_sync(0xffffffffu, pix, 1);
+        const bool valid = pix >= 0;
+        const bool start = valid && (lane == 0 || prev < 0 || prev + 1 != pix);
+        const uint32_t stops = ~__ballot_sync(0xffffffffu, valid) | __ballot_sync(0xffffffffu, start);  // a run ends before these lanes
+        if (start) {
+            const uint32_t later = lane == 31 ? 0u : (stops >> (lane + 1));
+            const int len = later == 0u ? 32 - lane : 1 + __ffs(later) - 1;  // columns lane .. lane+len-1
+            const uint32_t src = smem_u32(stage + col_px * kStageCh);
+            uint32_t *dst = static_cast<uint32_t *>(p.out) + (int64_t)pix * kStageCh;
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"((uint32_t)(len * kStageCh * 4))
+                         : "memory");
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        return;
+    }
+    asm volatile("bar.sync 2, %0;" ::"n"(kWorkers) : "memory");  // the stage holds the whole tile
+    // rows out: warp w takes pixels 32w .. 32w+31; a row of Cout values is Cout/4 16-byte pieces
+    const int pieces = p.Cout >> 2;                       // 1 .. 16 (Cout is a multiple of 4 here)
+    const int rows_per_inst = 32 / pieces >= 2 ? 2 : 1;   // Cout <= 32: still two rows per instruction
+    const int sub = lane / pieces, piece = lane - sub * pieces;
+    if (sub < rows_per_inst) {
+        // four rows in flight per lane: the loads do not wait for one another's stores
+        for (int r = 0; r < 32; r += 4 * rows_per_inst) {
+            int pix[4];
+            uint4 q[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int col_px = warp * 32 + r + u * rows_per_inst + sub;  // rows_per_inst divides 8: stays inside the warp's 32
+                pix[u] = sPix[col_px];
+                q[u] = *reinterpret_cast<const uint4 *>(stage + col_px * kStageCh + piece * 4);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (pix[u] >= 0) *reinterpret_cast<uint4 *>(static_cast<uint32_t *>(p.out) + (int64_t)pix[u] * p.Cout + piece * 4) = q[u];
+        }
+    }
+    asm volatile("bar.sync 2, %0;" ::"n"(kWorkers) : "memory");  // everybody has read the stage
+}
+
 __global__ void __launch_bounds__(kSwThreads, 1)
 bconv3x3_tensor_swapped_kernel(const TensorParams p)  // p.P, p.n_tiles are for tiles of kTileN positions; p.n_blk = 128
 {
@@ -842,6 +933,7 @@ bconv3x3_tensor_swapped_kernel(const TensorParams p)  // p.P, p.n_tiles are for 
     const size_t w_tap_bytes = (size_t)2 * p.Cw * 128 * 16;
     uint8_t *sX0 = sW + 9 * w_tap_bytes;                                // B operand: 2 x [2*Cw chunks][P positions][16]
     const size_t x_bytes = (size_t)2 * p.Cw * p.P * 16;
+    uint32_t *stage = reinterpret_cast<uint32_t *>(sX0 + 2 * x_bytes);  // float / int32 output only: [kTileN][kStageCh]
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int ch0 = blockIdx.y * 128;
@@ -856,7 +948,7 @@ bconv3x3_tensor_swapped_kernel(const TensorParams p)  // p.P, p.n_tiles are for 
         table[e] = make_uint2(lo, hi);
     }
     for (int e = tid; e < 128; e += kSwThreads) {
-        sThr[e] = ch0 + e < p.Cout ? __ldg(p.thr + ch0 + e) : INT32_MIN;
+        sThr[e] = (p.out_type == LCE_OUT_BITPACKED && ch0 + e < p.Cout) ? __ldg(p.thr + ch0 + e) : INT32_MIN;
     }
     for (int e = tid; e < 9 * p.Cw; e += kSwThreads) {
         const int tap = e / p.Cw, cw = e - tap * p.Cw;
@@ -968,17 +1060,41 @@ bconv3x3_tensor_swapped_kernel(const TensorParams p)  // p.P, p.n_tiles are for 
         } else {
             // ---- finishers -------------------------------------------------------------------------------
             const int ftid = tid - kSwLoaders;
+            const bool staged = p.out_type != LCE_OUT_BITPACKED;
+            const int my_channel = ch0 + ((ftid >> 5) & 3) * 32 + (ftid & 31);
+            const bool has_params = p.out_type == LCE_OUT_FLOAT32 && my_channel < p.Cout;
+            const float my_mult = has_params ? __ldg(p.mult + my_channel) : 0.f, my_bias = has_params ? __ldg(p.bias + my_channel) : 0.f;
             int tile = first_tile;
             for (int it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
                 const int sbuf = it & 1;
                 ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + sbuf], par_full_d[sbuf]);
                 par_full_d[sbuf] ^= 1u;
+                if (staged) {
+                    // the staged form synchronises the finisher warps among themselves: they go on only
+                    // if the wait succeeded in every one of them
+                    uint32_t all_ok;
+                    asm volatile("{\n\t.reg .pred q, r;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred r, 3, %2, q;\n\tselp.u32 %0, 1, 0, r;\n\t}"
+                                 : "=r"(all_ok)
+                                 : "r"((uint32_t)ok), "n"(kWorkers)
+                                 : "memory");
+                    ok = all_ok != 0;
+                }
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                epilogue_swapped(p, tmem_base + (uint32_t)(sbuf * kTileN), sPix + (it & 3) * kTileN, ch0, sThr, ftid);
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                mbar_arrive(&bars[BAR_EMPTY_D0 + sbuf]);
+                if (staged && p.Cout == kStageCh && it > 0) {
+                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // this thread's copies have read the stage
+                    asm volatile("bar.sync 2, %0;" ::"n"(kWorkers) : "memory");     // ... and so have everybody's
+                }
+                if (staged) {
+                    epilogue_swapped_staged(p, tmem_base + (uint32_t)(sbuf * kTileN), sPix + (it & 3) * kTileN, ch0, stage, my_mult, my_bias,
+                                            ftid, &bars[BAR_EMPTY_D0 + sbuf]);
+                } else {
+                    epilogue_swapped(p, tmem_base + (uint32_t)(sbuf * kTileN), sPix + (it & 3) * kTileN, ch0, sThr, ftid);
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    mbar_arrive(&bars[BAR_EMPTY_D0 + sbuf]);
+                }
             }
+            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // staged form: the last tile's copies are complete
         }
     }
     if (!ok) g_tensor_status = 1;
@@ -1023,9 +1139,13 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const uint
         q.n_blk_log2 = 7;
         q.tmem_cols = 512;
         const size_t raw_b = (size_t)2 * (((size_t)q.P * g.Cw + 3) / 4) * 16;
-        const size_t need = (size_t)2048 + 128 + 128 * 4 + 4 * kTileN * 4 + 8 * (size_t)(((9 * g.Cw + 1) / 2) * 2) + raw_b +
+        size_t need = (size_t)2048 + 128 + 128 * 4 + 4 * kTileN * 4 + 8 * (size_t)(((9 * g.Cw + 1) / 2) * 2) + raw_b +
                             9 * (size_t)2 * g.Cw * 128 * 16 + 2 * (size_t)2 * g.Cw * q.P * 16;
-        bool swapped = g.out_type == LCE_OUT_BITPACKED && g.Cout <= 128 && need <= 226 * 1024 && q.P <= 16383 && (int64_t)g.N * g.H * g.W < (1ll << 31);
+        // float / int32 output goes through a [256][64] stage in shared memory: Cout <= 64, 16-byte rows
+        const bool staged = g.out_type != LCE_OUT_BITPACKED;
+        if (staged) need += (size_t)kTileN * kStageCh * 4;
+        bool swapped = (staged ? (g.Cout <= kStageCh && p.vec_store != 0) : g.Cout <= 128) && need <= 226 * 1024 && q.P <= 16383 &&
+                       (int64_t)g.N * g.H * g.W < (1ll << 31);
 #ifdef LCE_TUNING
         if (const char *e = getenv("LCE_TENSOR_SWAP")) swapped = swapped && atoi(e) != 0;
 #endif

@@ -149,6 +149,8 @@ TENSOR_SHAPES = [
     (1, 1, 1, 3, 1), (5, 3, 40, 96, 130),
     # bit-packed output with Cout <= 128 and few input words: the pixels-as-N schedule, several tiles and images
     (2, 30, 30, 32, 128), (6, 20, 17, 64, 100), (1, 80, 80, 33, 33), (3, 40, 3, 96, 64),
+    # float / int32 output with Cout <= 64, a multiple of 4: the same schedule with the shared-memory stage
+    (2, 20, 20, 64, 48), (1, 30, 30, 32, 8), (4, 16, 16, 40, 60), (1, 12, 12, 64, 4), (3, 33, 31, 64, 32),
 ]
 
 

@@ -699,7 +699,44 @@ bconv3x3_tensor_split_kernel(const TensorParams p)
     } else {
         // ---- both worker groups expand the resident weights, then part ways ----------------------
         if (tid < kWorkers && first_tile < p.n_tiles) prefetch_raw(p, first_tile * kTileM, raw0, tid);
-        for (int e0 = tid; e0 < 9 * words_per_tap; e0 += 2 * kWorkers * 8) {
+        const bool quads = (p.Cw & 3) == 0 && (reinterpret_cast<uintptr_t>(p.w) & 15) == 0;
+        if (quads) {
+            // Four consecutive channel words of one channel per 128-bit load (channel-fastest over the
+            // lanes, so the shared-memory stores stay conflict-free): a quarter of the load requests of
+            // the word-by-word form, which kept the load unit busy for most of the set-up time.  Half of
+            // the words go through the look-up table and half through the integer pipes, which work
+            // side by side.
+            const int units = 9 * words_per_tap / 4;  // (channel, quad) pairs; a quad lies inside one tap
+            for (int u0 = tid; u0 < units; u0 += 2 * kWorkers * 2) {
+                uint4 q[2];
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    const int u = u0 + k * 2 * kWorkers;
+                    const int ch = u & (p.n_blk - 1), tc = (u >> p.n_blk_log2) * 4;
+                    q[k] = (u < units && ch0 + ch < p.Cout) ? __ldg(reinterpret_cast<const uint4 *>(p.w + (int64_t)(ch0 + ch) * 9 * p.Cw + tc))
+                                                            : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    const int u = u0 + k * 2 * kWorkers;
+                    if (u < units) {
+                        const int ch = u & (p.n_blk - 1), tc = (u >> p.n_blk_log2) * 4;
+                        const int tap = tc / p.Cw, cw = tc - tap * p.Cw;
+                        const uint32_t wq[4] = {q[k].x, q[k].y, q[k].z, q[k].w};
+                        uint4 *dst = reinterpret_cast<uint4 *>(sB + tap * b_tap_bytes) + (size_t)(2 * cw) * p.n_blk + ch;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint4 lo, hi;
+                            if (i & 1) expand_word(table, wq[i], &lo, &hi);
+                            else expand_word_alu(wq[i], &lo, &hi);
+                            dst[(size_t)(2 * i) * p.n_blk] = lo;
+                            dst[(size_t)(2 * i + 1) * p.n_blk] = hi;
+                        }
+                    }
+                }
+            }
+        }
+        for (int e0 = tid; !quads && e0 < 9 * words_per_tap; e0 += 2 * kWorkers * 8) {
             uint32_t wv[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
@@ -1006,7 +1043,39 @@ bconv3x3_tensor_swapped_kernel(const TensorParams p)  // p.P, p.n_tiles are for 
         if (tid < kSwLoaders && first_tile < p.n_tiles) prefetch_raw<kSwLoaders>(p, first_tile * kTileN, raw0, tid);
         // weights of this channel block, once: packed [o][tap][cw] -> bytes [tap][chunk][channel][16]
         const int words = 9 * 128 * p.Cw;
-        for (int e0 = tid; e0 < words; e0 += (kSwLoaders + kWorkers) * 8) {
+        const bool pairs = (p.Cw & 1) == 0 && (reinterpret_cast<uintptr_t>(p.w) & 7) == 0;
+        if (pairs) {
+            // two consecutive channel words per 64-bit load, channel-fastest over the lanes: half the load
+            // requests; one word of a pair is expanded through the table, the other on the integer pipes
+            const int units = words / 2;  // (channel, pair) pairs; a pair lies inside one tap
+            for (int u0 = tid; u0 < units; u0 += (kSwLoaders + kWorkers) * 4) {
+                uint2 q[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int u = u0 + k * (kSwLoaders + kWorkers);
+                    const int ch = u & 127, tc = (u >> 7) * 2;
+                    q[k] = (u < units && ch0 + ch < p.Cout) ? __ldg(reinterpret_cast<const uint2 *>(p.w + (int64_t)(ch0 + ch) * 9 * p.Cw + tc))
+                                                            : make_uint2(0u, 0u);
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int u = u0 + k * (kSwLoaders + kWorkers);
+                    if (u < units) {
+                        const int ch = u & 127, tc = (u >> 7) * 2;
+                        const int tap = tc / p.Cw, cw = tc - tap * p.Cw;
+                        uint4 *dst = reinterpret_cast<uint4 *>(sW + tap * w_tap_bytes) + (size_t)(2 * cw) * 128 + ch;
+                        uint4 lo, hi;
+                        expand_word(table, q[k].x, &lo, &hi);
+                        dst[0] = lo;
+                        dst[128] = hi;
+                        expand_word_alu(q[k].y, &lo, &hi);
+                        dst[256] = lo;
+                        dst[384] = hi;
+                    }
+                }
+            }
+        }
+        for (int e0 = tid; !pairs && e0 < words; e0 += (kSwLoaders + kWorkers) * 8) {
             uint32_t wv[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) {

@@ -37,9 +37,10 @@ typedef enum {
     LCE_OK = 0,
     LCE_ERR_INVALID_ARG = 1,    /* null pointer, non-positive extent, bad enum, empty output */
     LCE_ERR_UNSUPPORTED = 2,    /* valid request that no kernel here implements */
-    LCE_ERR_ALIGNMENT = 3,      /* a pointer is not aligned to its element size (4 bytes) */
+    LCE_ERR_ALIGNMENT = 3,      /* a pointer is not aligned to its element size (4 bytes; packed weights: 256) */
     LCE_ERR_CUDA = 4,           /* the CUDA runtime reported an error at launch / copy */
-    LCE_ERR_DEVICE_TIMEOUT = 5, /* reserved: a bounded device-side wait gave up */
+    LCE_ERR_DEVICE_TIMEOUT = 5, /* a bounded device-side wait of an earlier kernel on this device gave up:
+                                   that kernel's output is incomplete; see lce_device_status */
     LCE_ERR_WORKSPACE = 6       /* caller's workspace is too small */
 } lce_status;
 
@@ -55,11 +56,17 @@ typedef enum { LCE_OUT_FLOAT32 = 0, LCE_OUT_BITPACKED = 1, LCE_OUT_INT32 = 2 } l
  * batch-norm in QuickNet).  Applied to the accumulator before multiplier and bias. */
 typedef enum { LCE_ACT_NONE = 0, LCE_ACT_RELU = 1 } lce_activation;
 
-/* Which kernel lce_bconv2d uses.  AUTO picks the tiled XOR/POPC kernel when it covers the
- * shape and the direct kernel otherwise; the other values force one (tests, benchmarks).
- * TENSOR is the tensor-core formulation (bits expanded to +-1 int8 in shared memory, tcgen05
- * kind::i8, accumulators in TMEM; exact): 3x3, stride 1, LCE_PAD_SAME_ONE only, never chosen by
- * AUTO. */
+/* Which kernel lce_bconv2d uses; every kernel gives the same, exact result.
+ *   TILED  the XOR/POPC kernels on the integer pipes (1x1, 3x3, 5x5 filters, equal strides 1 or 2; a
+ *          one-word kernel when kh*kw*in_c <= 32);
+ *   TENSOR the tensor-core formulation: bits expanded to +-1 (0 for padding) as 4-bit e2m1 values,
+ *          tcgen05 kind::mxf4 with unit block scales, fp32 accumulators in TMEM (exact: every sum is an
+ *          integer below 2^24).  Filters of up to 64 taps, equal strides of 1 or 2, in_c <= 1024, every
+ *          padding mode and output type.  Needs weights packed by lce_bconv2d_pack_weights;
+ *   DIRECT one thread per output, any shape (fallback, not tuned);
+ *   AUTO   TENSOR for layers of at least 2^28 binary MACs when the weights are packed, otherwise TILED
+ *          where it covers the shape, otherwise DIRECT.
+ * Forcing a kernel on a shape (or on plain weights) it does not cover returns LCE_ERR_UNSUPPORTED. */
 typedef enum { LCE_KERNEL_AUTO = 0, LCE_KERNEL_DIRECT = 1, LCE_KERNEL_TILED = 2, LCE_KERNEL_TENSOR = 3 } lce_kernel;
 
 const char *lce_version(void);
@@ -106,9 +113,12 @@ lce_status lce_bconv2d_out_shape(const lce_bconv2d_desc *desc, int32_t *out_h, i
  *   input   uint32[batch][in_h][in_w][ceil(in_c/32)]     weights uint32[out_c][kh][kw][ceil(in_c/32)]
  * With desc->weights_packed == 1, `weights` is instead the buffer written by
  * lce_bconv2d_pack_weights (the fast path: nothing is derived from the weights per call).
- * Pad bits of input and weights must be 0.  Errors: INVALID_ARG (null/extent/enum/missing
- * per-channel array), ALIGNMENT, UNSUPPORTED (kernel forced to TILED on a shape it does not
- * cover), CUDA. */
+ * Pad bits of input and weights must be 0.  The float / int32 fast paths want `output` 16-byte
+ * aligned (out_c a multiple of 4); a buffer that is only 4-byte aligned is served by the direct kernel
+ * under AUTO.  The weights and per-channel arrays are constants of the model: they must not be written
+ * by work that is still running on the stream when this call is made.  Errors: INVALID_ARG
+ * (null/extent/enum/missing per-channel array), ALIGNMENT, UNSUPPORTED (a forced kernel does not cover
+ * the shape), CUDA, DEVICE_TIMEOUT (see lce_device_status; nothing is launched). */
 lce_status lce_bconv2d(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,
                        const float *multiplier, const float *bias, const int32_t *thresholds,
                        void *output, void *stream);
@@ -147,7 +157,10 @@ lce_status lce_bconv2d_f32(const lce_bconv2d_desc *desc, const float *input, con
  * paper's engine picks its kernel and tiling per layer when the model is loaded (Section 3.1); this
  * is that choice made visible.  Fields that do not apply to the chosen kernel are 0.
  *   kernel              LCE_KERNEL_DIRECT, LCE_KERNEL_TILED or LCE_KERNEL_TENSOR (the one-word patch
- *                       kernel for very few input channels reports LCE_KERNEL_TILED with patch = 1)
+ *                       kernel for very few input channels reports LCE_KERNEL_TILED with patch = 1).
+ *                       For LCE_KERNEL_TENSOR: tile_pixels = grid positions per tile, ctas, shared_bytes,
+ *                       weight_stages = taps the shared-memory weight ring holds, weights_resident = 1
+ *                       when that is every tap (fetched once per CTA instead of once per tile)
  *   pointwise           1 for the 1x1 tiled kernel
  *   warps_per_cta, pixels_per_thread, tile_pixels, shared_bytes      the variant of the tiled kernel
  *   ctas                CTAs of the launch; ctas_half_block of them work on the last, at most
@@ -161,6 +174,7 @@ typedef struct lce_bconv2d_plan_info {
     int32_t warps_per_cta, pixels_per_thread, tile_pixels;
     int32_t ctas, ctas_half_block, pixels_per_cta, pixels_per_cta_half_block;
     int64_t shared_bytes;
+    int32_t weight_stages, weights_resident;
 } lce_bconv2d_plan_info;
 lce_status lce_bconv2d_plan(const lce_bconv2d_desc *desc, lce_bconv2d_plan_info *plan);
 
@@ -184,8 +198,11 @@ void lce_plan_destroy(lce_plan *plan);
  * time for its access pattern; Section 3.1: weights are converted once, when the model is built).  Rewrites
  * the plain packed weights into the operand layout the tiled kernel copies straight into shared
  * memory, so that none of that work is repeated per call.  The packed buffer also keeps a copy of
- * the plain words, and is valid for every padding mode, output type and activation of the same
- * geometry (batch, sizes, channels, kernel, stride).
+ * the plain words, and, where the tensor-core kernel covers the geometry, that kernel's operand image
+ * (every weight bit expanded to a 4-bit +-1, pad channels 0).  It is valid for every padding mode, output
+ * type and activation of the same geometry (batch, sizes, channels, kernel, stride).  The first call in a
+ * process also sets up a few bytes of pinned host memory for the device-timeout flag: make it outside
+ * any stream capture.
  *   weights uint32[out_c][kh][kw][ceil(in_c/32)] (device)  ->  packed: device buffer of
  *   lce_bconv2d_packed_weights_bytes(desc) bytes, 256-byte aligned, owned by the caller.
  * lce_bconv2d_packed_weights_bytes returns 0 for a malformed descriptor. */
@@ -222,7 +239,8 @@ lce_status lce_bconv2d_host_async(const lce_bconv2d_desc *desc, const uint32_t *
  * workspace; a call whose lce_bconv2d_host_workspace_bytes(desc) exceeds the array returns
  * LCE_ERR_WORKSPACE and does nothing.
  *   - The first call on each device looks up the array's device address (with that device
- *     current); make that first call before starting any stream capture.
+ *     current).  The call synchronises `stream` before it returns, so it cannot be part of a stream
+ *     capture anyway.
  *   - All calls on a device share the one array, which still holds the previous call's data:
  *     nothing needs clearing (every region is rewritten before it is read), but two calls that
  *     overlap on the GPU (different streams, different threads) would overwrite each other.
@@ -244,11 +262,22 @@ lce_status lce_bmaxpool(const uint32_t *in, uint32_t *out, int32_t batch, int32_
  * (float output -> Add -> LceQuantize).  n == 0 is a no-op; out may equal a or b. */
 lce_status lce_add_f32(const float *a, const float *b, float *out, int64_t n, void *stream);
 
-/* Status word of the bounded device-side waits (the tensor-core kernel waits on an mbarrier for
- * its MMAs, with an iteration limit).  *status (HOST pointer) = 0 if no wait has ever given up
- * on the current device, 1 otherwise; a non-zero value means outputs of the affected call are
- * incomplete.  Synchronous (reads a device variable). */
+/* Status of the bounded device-side waits.  The tensor-core kernel's warps meet through mbarriers
+ * (operands ready, MMAs complete, accumulator read out); every such wait is limited to 0.2 s, after
+ * which the kernel stops working, waits (bounded) for its copies and MMAs in flight, frees its tensor
+ * memory and returns, leaving its output incomplete.  It records that in a device word and in a word
+ * of mapped host memory; from then on lce_bconv2d, lce_bconv2d_fused and lce_plan_run on that device
+ * return LCE_ERR_DEVICE_TIMEOUT without launching, until lce_device_status_reset.
+ *   lce_device_status        *status (HOST pointer) = 0 if no wait has given up on the current device
+ *                            since load or the last reset, 1 otherwise.  Synchronous (reads the device word).
+ *   lce_device_status_reset  clears both words for the current device.  Synchronous.
+ *   lce_device_wait_probe    self-test of that machinery: launches one tiny kernel on `stream` whose
+ *                            wait (limit_ns, 1 .. 10^9) is on a barrier nobody arrives at, so it runs out,
+ *                            is reported like a real one, and the kernel returns normally.  Touches no
+ *                            tensor; follow it with lce_device_status_reset. */
 lce_status lce_device_status(int32_t *status);
+lce_status lce_device_status_reset(void);
+lce_status lce_device_wait_probe(uint64_t limit_ns, void *stream);
 
 /* Integer-pipe probe: runs a register/shared-memory resident loop of one instruction mix on
  * every SM of the current device and reports how many 32-bit word operations (one XOR +

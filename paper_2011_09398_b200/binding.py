@@ -201,7 +201,7 @@ def lce_bconv2d_f32(desc: BConv2dDesc, input: torch.Tensor, weights: torch.Tenso
 class BConv2dPlanInfo(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("kernel", "patch", "pointwise", "warps_per_cta", "pixels_per_thread", "tile_pixels",
                                                "ctas", "ctas_half_block", "pixels_per_cta", "pixels_per_cta_half_block")] + \
-               [("shared_bytes", ctypes.c_int64)]
+               [("shared_bytes", ctypes.c_int64), ("weight_stages", ctypes.c_int32), ("weights_resident", ctypes.c_int32)]
 
 
 def lce_bconv2d_plan(desc: BConv2dDesc) -> dict:
@@ -364,6 +364,22 @@ def lce_device_status() -> int:
     lib.lce_device_status.restype = ctypes.c_int
     _check(lib.lce_device_status(ctypes.byref(v)), "lce_device_status")
     return v.value
+
+
+def lce_device_status_reset() -> None:
+    """Clears the status of the bounded device-side waits for the current device."""
+    lib = library()
+    lib.lce_device_status_reset.argtypes = []
+    lib.lce_device_status_reset.restype = ctypes.c_int
+    _check(lib.lce_device_status_reset(), "lce_device_status_reset")
+
+
+def lce_device_wait_probe(limit_ns: int) -> None:
+    """Launches the tiny kernel whose bounded wait is meant to run out (see lce.h); asynchronous."""
+    lib = library()
+    lib.lce_device_wait_probe.argtypes = [ctypes.c_uint64, ctypes.c_void_p]
+    lib.lce_device_wait_probe.restype = ctypes.c_int
+    _check(lib.lce_device_wait_probe(int(limit_ns), _stream()), "lce_device_wait_probe")
 
 
 def lce_probe_pipe(mix: int, iterations: int = 2000) -> Tuple[float, float]:

@@ -1,23 +1,26 @@
 """Builds the C-ABI CUDA library in-tree: ``python -m paper_2011_09398_b200.build``.
 
-nvcc cross-compiles for sm_100a without a GPU present.  The resulting
-``liblce_b200.so`` sits next to this file and is what the binding loads.
+nvcc cross-compiles for sm_100a without a GPU present.  Every ``csrc/*.cu`` is compiled to an
+object file (in parallel, only when it or a header changed) and the objects are linked into
+``liblce_b200.so`` next to this file, which is what the binding loads.
 """
 from __future__ import annotations
 
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 from pathlib import Path
 
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 INCLUDE = PKG.parent / "include"
+OBJ = PKG / "build"
 LIB = PKG / "liblce_b200.so"
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-shared",
+    "-Xcompiler", "-fPIC",
 ]
 
 
@@ -25,25 +28,46 @@ def sources():
     return sorted(CSRC.glob("*.cu"))
 
 
+def _headers_mtime() -> float:
+    deps = list(CSRC.glob("*.cuh")) + list(INCLUDE.glob("*.h"))
+    return max(d.stat().st_mtime for d in deps)
+
+
 def is_stale() -> bool:
     if not LIB.exists():
         return True
     t = LIB.stat().st_mtime
-    deps = list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh")) + list(INCLUDE.glob("*.h"))
-    return any(d.stat().st_mtime > t for d in deps)
+    return any(s.stat().st_mtime > t for s in sources()) or _headers_mtime() > t
 
 
 def build(force: bool = False, verbose: bool = False) -> Path:
     if not force and not is_stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
-    extra = os.environ.get("LCE_NVCC_FLAGS", "").split()  # e.g. -DLCE_CTAS_PER_SM=3 for tuning runs
-    cmd = [nvcc, *NVCC_FLAGS, *extra, f"-I{INCLUDE}", f"-I{CSRC}", "-o", str(tmp), *map(str, sources())]
+    OBJ.mkdir(exist_ok=True)
+    hdr = _headers_mtime()
+    jobs = []
+    for src in sources():
+        obj = OBJ / (src.stem + ".o")
+        if force or not obj.exists() or obj.stat().st_mtime < max(src.stat().st_mtime, hdr):
+            cmd = [nvcc, *NVCC_FLAGS, f"-I{INCLUDE}", f"-I{CSRC}", "-c", "-o", str(obj), str(src)]
+            if verbose:
+                cmd.insert(1, "-Xptxas=-v")
+            jobs.append(cmd)
     if verbose:
-        cmd.insert(1, "-Xptxas=-v")
-        print(" ".join(cmd), file=sys.stderr)
-    subprocess.run(cmd, check=True)
+        for cmd in jobs:
+            print(" ".join(cmd), file=sys.stderr)
+    with ThreadPoolExecutor(max_workers=min(8, max(1, len(jobs)))) as pool:
+        for res in pool.map(lambda c: subprocess.run(c, capture_output=not verbose, text=True), jobs):
+            if res.returncode != 0:
+                sys.stderr.write((res.stdout or "") + (res.stderr or ""))
+                raise subprocess.CalledProcessError(res.returncode, res.args)
+    stale = {p.stem for p in OBJ.glob("*.o")} - {s.stem for s in sources()}
+    for name in stale:  # objects of sources that no longer exist
+        (OBJ / (name + ".o")).unlink()
+    tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
+    objs = [str(OBJ / (s.stem + ".o")) for s in sources()]
+    subprocess.run([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", str(tmp), *objs], check=True)
     os.replace(tmp, LIB)
     return LIB
 

@@ -2,6 +2,7 @@
 // host-buffer forms).  All argument checks happen here, before anything is launched.
 #include "common.cuh"
 
+#include <atomic>
 #include <new>
 
 namespace lce {
@@ -25,26 +26,81 @@ size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 size_t plain_weight_bytes(const ConvGeom &g) { return round_up((size_t)g.Cout * g.KH * g.KW * g.Cw * 4, 256); }
 
+// A packed-weights buffer = [plain words][operand image of the tiled XOR/POPC kernel][operand image of
+// the tensor-core kernel], each part rounded up to 256 bytes; a part a kernel does not cover is empty.
+struct WeightViews {
+    const uint32_t *plain;
+    const uint32_t *tiled;
+    const void *tensor;
+};
+
+lce_status weight_views(const lce_bconv2d_desc *desc, const ConvGeom &g, const uint32_t *weights, WeightViews *v)
+{
+    v->plain = weights;
+    v->tiled = nullptr;
+    v->tensor = nullptr;
+    if (!desc->weights_packed) return LCE_OK;
+    if (!aligned(weights, 256)) return LCE_ERR_ALIGNMENT;
+    const char *base = reinterpret_cast<const char *>(weights);
+    size_t off = plain_weight_bytes(g);
+    const size_t tiled = tiled_weight_image_bytes(g), tensor = tensor_weight_image_bytes(g);
+    if (tiled > 0) v->tiled = reinterpret_cast<const uint32_t *>(base + off);
+    off += round_up(tiled, 256);
+    if (tensor > 0) v->tensor = base + off;
+    return LCE_OK;
+}
+
+// The tiled kernels write float / int32 rows with 128-bit accesses when the channel count allows it,
+// and then need 16-byte aligned buffers.
+bool tiled_accepts(const ConvGeom &g, const void *out, const void *residual)
+{
+    return !((g.Cout & 3) == 0 && g.out_type != LCE_OUT_BITPACKED && (!aligned(out, 16) || !aligned(residual, 16)));
+}
+
+// AUTO takes the tensor-core kernel when the weights were packed at load time (its operand image
+// exists) and the layer is large enough to fill the machine: below about 2^28 binary MACs a launch is
+// dominated by fixed costs and the integer kernels, which start faster, win (measured).
+bool tensor_preferred(const ConvGeom &g)
+{
+    const double macs = (double)g.M * g.Cout * g.KH * g.KW * g.Cin;
+    return macs >= 268435456.0 && !patch_covers(g);
+}
+
+enum KernelPick { PICK_NONE = 0, PICK_DIRECT, PICK_PATCH, PICK_TILED, PICK_TENSOR };
+
+// One place decides which kernel a call gets; lce_bconv2d_plan shows the same decision.
+KernelPick pick_kernel(const lce_bconv2d_desc *desc, const ConvGeom &g, bool have_tensor_image, bool tiled_buffers_ok)
+{
+    TiledPlanInfo info{};
+    switch (desc->kernel) {
+        case LCE_KERNEL_DIRECT: return PICK_DIRECT;
+        case LCE_KERNEL_TENSOR: return have_tensor_image && tensor_covers(g) ? PICK_TENSOR : PICK_NONE;
+        case LCE_KERNEL_TILED:
+            if (patch_covers(g)) return PICK_PATCH;
+            return tiled_buffers_ok && tiled_plan_info(g, &info) == LCE_OK ? PICK_TILED : PICK_NONE;
+        default: break;
+    }
+    if (have_tensor_image && tensor_preferred(g) && tensor_covers(g)) return PICK_TENSOR;
+    if (patch_covers(g)) return PICK_PATCH;
+    if (tiled_buffers_ok && tiled_plan_info(g, &info) == LCE_OK) return PICK_TILED;
+    return PICK_DIRECT;
+}
+
 lce_status dispatch(const lce_bconv2d_desc *desc, const ConvGeom &g, const uint32_t *input, const uint32_t *weights,
                     const float *multiplier, const float *bias, const int32_t *thresholds, void *output,
                     cudaStream_t s)
 {
-    // a packed-weights buffer = [plain words, rounded up to 256 bytes][tiled image]
-    const uint32_t *image = nullptr;
-    if (desc->weights_packed) {
-        if (!aligned(weights, 256)) return LCE_ERR_ALIGNMENT;
-        if (tiled_weight_image_bytes(g) > 0)
-            image = reinterpret_cast<const uint32_t *>(reinterpret_cast<const char *>(weights) + plain_weight_bytes(g));
+    if (tensor_timeout_flagged()) return LCE_ERR_DEVICE_TIMEOUT;  // an earlier kernel on this device gave up a wait
+    WeightViews v;
+    lce_status st = weight_views(desc, g, weights, &v);
+    if (st != LCE_OK) return st;
+    switch (pick_kernel(desc, g, v.tensor != nullptr, tiled_accepts(g, output, nullptr))) {
+        case PICK_DIRECT: return launch_bconv_direct(g, input, v.plain, multiplier, bias, thresholds, output, s);
+        case PICK_PATCH: return launch_bconv_patch(g, input, v.plain, multiplier, bias, thresholds, output, s);
+        case PICK_TILED: return launch_bconv_tiled(g, input, v.plain, v.tiled, multiplier, bias, thresholds, output, s);
+        case PICK_TENSOR: return launch_bconv_tensor(g, input, v.tensor, multiplier, bias, thresholds, output, s);
+        default: return LCE_ERR_UNSUPPORTED;
     }
-    if (desc->kernel == LCE_KERNEL_DIRECT)
-        return launch_bconv_direct(g, input, weights, multiplier, bias, thresholds, output, s);
-    if (desc->kernel == LCE_KERNEL_TENSOR)
-        return launch_bconv_tensor(g, input, weights, multiplier, bias, thresholds, output, s);
-    if (patch_covers(g)) return launch_bconv_patch(g, input, weights, multiplier, bias, thresholds, output, s);
-    lce_status st = launch_bconv_tiled(g, input, weights, image, multiplier, bias, thresholds, output, s);
-    if (st == LCE_ERR_UNSUPPORTED && desc->kernel == LCE_KERNEL_AUTO)
-        st = launch_bconv_direct(g, input, weights, multiplier, bias, thresholds, output, s);
-    return st;
 }
 
 struct HostLayout {
@@ -99,6 +155,14 @@ extern "C" lce_status lce_device_status(int32_t *status)
     return LCE_OK;
 }
 
+extern "C" lce_status lce_device_status_reset(void) { return lce::tensor_device_status_reset(); }
+
+extern "C" lce_status lce_device_wait_probe(uint64_t limit_ns, void *stream)
+{
+    if (limit_ns == 0 || limit_ns > 1000000000ull) return LCE_ERR_INVALID_ARG;  // at most a second
+    return lce::tensor_wait_probe(limit_ns, static_cast<cudaStream_t>(stream));
+}
+
 extern "C" lce_status lce_bconv2d_out_shape(const lce_bconv2d_desc *desc, int32_t *out_h, int32_t *out_w)
 {
     lce::ConvGeom g;
@@ -118,17 +182,28 @@ extern "C" lce_status lce_bconv2d_plan(const lce_bconv2d_desc *desc, lce_bconv2d
     if (st != LCE_OK) return st;
     if (!plan) return LCE_ERR_INVALID_ARG;
     *plan = lce_bconv2d_plan_info{};
-    // the same order of preference as dispatch()
-    if (desc->kernel == LCE_KERNEL_DIRECT) { plan->kernel = LCE_KERNEL_DIRECT; return LCE_OK; }
-    if (desc->kernel == LCE_KERNEL_TENSOR) {
-        if (!tensor_covers(g)) return LCE_ERR_UNSUPPORTED;
-        plan->kernel = LCE_KERNEL_TENSOR;
-        return LCE_OK;
+    // the decision dispatch() makes, for 16-byte aligned buffers
+    const bool have_tensor_image = desc->weights_packed && tensor_weight_image_bytes(g) > 0;
+    switch (pick_kernel(desc, g, have_tensor_image, true)) {
+        case PICK_DIRECT: plan->kernel = LCE_KERNEL_DIRECT; return LCE_OK;
+        case PICK_PATCH: plan->kernel = LCE_KERNEL_TILED; plan->patch = 1; return LCE_OK;
+        case PICK_TENSOR: {
+            TensorPlanInfo t{};
+            st = tensor_plan_info(g, &t);
+            if (st != LCE_OK) return st;
+            plan->kernel = LCE_KERNEL_TENSOR;
+            plan->tile_pixels = t.tile_positions;
+            plan->ctas = t.ctas;
+            plan->weight_stages = t.weight_stages;
+            plan->weights_resident = t.weights_resident;
+            plan->shared_bytes = t.shared_bytes;
+            return LCE_OK;
+        }
+        case PICK_TILED: break;
+        default: return LCE_ERR_UNSUPPORTED;
     }
-    if (patch_covers(g)) { plan->kernel = LCE_KERNEL_TILED; plan->patch = 1; return LCE_OK; }
     TiledPlanInfo info{};
     st = tiled_plan_info(g, &info);
-    if (st == LCE_ERR_UNSUPPORTED && desc->kernel == LCE_KERNEL_AUTO) { plan->kernel = LCE_KERNEL_DIRECT; return LCE_OK; }
     if (st != LCE_OK) return st;
     plan->kernel = LCE_KERNEL_TILED;
     plan->pointwise = info.pointwise;
@@ -182,9 +257,13 @@ extern "C" lce_status lce_bconv2d_plan_create(const lce_bconv2d_desc *desc, cons
         (multiplier && !aligned(multiplier, 4)) || (bias && !aligned(bias, 4)) ||
         (thresholds && !aligned(thresholds, 4)))
         return LCE_ERR_ALIGNMENT;
-    lce_bconv2d_plan_info info;
-    st = lce_bconv2d_plan(desc, &info);  // is there a kernel for this shape (and for a forced kernel choice)?
+    // is there a kernel for this shape, these buffers and a forced kernel choice?  (A float / int32 output
+    // that is only 4-byte aligned rules the tiled kernel out: AUTO then records the direct kernel, a
+    // forced LCE_KERNEL_TILED fails here rather than at every run.)
+    WeightViews v;
+    st = weight_views(desc, g, weights, &v);
     if (st != LCE_OK) return st;
+    if (pick_kernel(desc, g, v.tensor != nullptr, tiled_accepts(g, output, nullptr)) == PICK_NONE) return LCE_ERR_UNSUPPORTED;
     lce_plan *h = new (std::nothrow) lce_plan;
     if (!h) return LCE_ERR_CUDA;
     h->desc = *desc;
@@ -217,15 +296,18 @@ extern "C" lce_status lce_bconv2d_fused(const lce_bconv2d_desc *desc, const uint
     if (!aligned(input, 4) || !aligned(weights, 4) || !aligned(multiplier, 4) || !aligned(bias, 4) ||
         !aligned(residual, 4) || !aligned(out_float, 4) || !aligned(out_packed, 4))
         return LCE_ERR_ALIGNMENT;
-    const uint32_t *image = nullptr;
-    if (desc->weights_packed) {
-        if (!aligned(weights, 256)) return LCE_ERR_ALIGNMENT;
-        if (tiled_weight_image_bytes(g) > 0)
-            image = reinterpret_cast<const uint32_t *>(reinterpret_cast<const char *>(weights) + plain_weight_bytes(g));
-    }
+    if (tensor_timeout_flagged()) return LCE_ERR_DEVICE_TIMEOUT;
+    WeightViews v;
+    st = weight_views(desc, g, weights, &v);
+    if (st != LCE_OK) return st;
     if (desc->kernel == LCE_KERNEL_DIRECT || patch_covers(g)) return LCE_ERR_UNSUPPORTED;
-    return launch_bconv_tiled(g, input, weights, image, multiplier, bias, nullptr, out_float,
-                              static_cast<cudaStream_t>(stream), residual, out_packed);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the tensor-core kernel fuses the same neighbours when whole 32-channel words and 16-byte rows allow it
+    const bool tensor_ok = v.tensor && tensor_covers(g) && (g.Cout & 31) == 0 && aligned(out_float, 16) && aligned(residual, 16);
+    if (desc->kernel == LCE_KERNEL_TENSOR && !tensor_ok) return LCE_ERR_UNSUPPORTED;
+    if (tensor_ok && (desc->kernel == LCE_KERNEL_TENSOR || (desc->kernel == LCE_KERNEL_AUTO && tensor_preferred(g))))
+        return launch_bconv_tensor(g, input, v.tensor, multiplier, bias, nullptr, out_float, s, residual, out_packed);
+    return launch_bconv_tiled(g, input, v.plain, v.tiled, multiplier, bias, nullptr, out_float, s, residual, out_packed);
 }
 
 extern "C" lce_status lce_bconv2d_f32(const lce_bconv2d_desc *desc, const float *input, const uint32_t *weights,
@@ -240,14 +322,11 @@ extern "C" lce_status lce_bconv2d_f32(const lce_bconv2d_desc *desc, const float 
         (multiplier && !aligned(multiplier, 4)) || (bias && !aligned(bias, 4)) ||
         (thresholds && !aligned(thresholds, 4)))
         return LCE_ERR_ALIGNMENT;
-    const uint32_t *image = nullptr;
-    if (desc->weights_packed) {
-        if (!aligned(weights, 256)) return LCE_ERR_ALIGNMENT;
-        if (tiled_weight_image_bytes(g) > 0)
-            image = reinterpret_cast<const uint32_t *>(reinterpret_cast<const char *>(weights) + plain_weight_bytes(g));
-    }
+    WeightViews v;
+    st = weight_views(desc, g, weights, &v);
+    if (st != LCE_OK) return st;
     if (desc->kernel == LCE_KERNEL_DIRECT || desc->kernel == LCE_KERNEL_TENSOR) return LCE_ERR_UNSUPPORTED;
-    return launch_bconv_tiled(g, nullptr, weights, image, multiplier, bias, thresholds, output,
+    return launch_bconv_tiled(g, nullptr, v.plain, v.tiled, multiplier, bias, thresholds, output,
                               static_cast<cudaStream_t>(stream), nullptr, nullptr, input);
 }
 
@@ -255,7 +334,7 @@ extern "C" size_t lce_bconv2d_packed_weights_bytes(const lce_bconv2d_desc *desc)
 {
     lce::ConvGeom g;
     if (lce::make_geom(desc, &g) != LCE_OK) return 0;
-    return lce::plain_weight_bytes(g) + lce::tiled_weight_image_bytes(g);
+    return lce::plain_weight_bytes(g) + lce::round_up(lce::tiled_weight_image_bytes(g), 256) + lce::tensor_weight_image_bytes(g);
 }
 
 extern "C" lce_status lce_bconv2d_pack_weights(const lce_bconv2d_desc *desc, const uint32_t *weights, void *packed,
@@ -270,8 +349,15 @@ extern "C" lce_status lce_bconv2d_pack_weights(const lce_bconv2d_desc *desc, con
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t plain = (size_t)g.Cout * g.KH * g.KW * g.Cw * 4;
     if (cudaMemcpyAsync(packed, weights, plain, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return LCE_ERR_CUDA;
-    if (tiled_weight_image_bytes(g) == 0) return LCE_OK;
-    return launch_pack_weights_tiled(g, weights, reinterpret_cast<uint32_t *>(static_cast<char *>(packed) + plain_weight_bytes(g)), s);
+    size_t off = plain_weight_bytes(g);
+    const size_t tiled = tiled_weight_image_bytes(g), tensor = tensor_weight_image_bytes(g);
+    if (tiled > 0) {
+        st = launch_pack_weights_tiled(g, weights, reinterpret_cast<uint32_t *>(static_cast<char *>(packed) + off), s);
+        if (st != LCE_OK) return st;
+    }
+    off += round_up(tiled, 256);
+    if (tensor > 0) return launch_pack_weights_tensor(g, weights, static_cast<char *>(packed) + off, s);
+    return LCE_OK;
 }
 
 extern "C" size_t lce_bconv2d_host_workspace_bytes(const lce_bconv2d_desc *desc)
@@ -343,7 +429,7 @@ namespace lce {
 namespace {
 
 constexpr int kMaxDevices = 64;
-void *g_static_workspace_addr[kMaxDevices];  // device address of g_static_workspace, per device; 0 = not looked up yet
+std::atomic<void *> g_static_workspace_addr[kMaxDevices];  // device address of g_static_workspace, per device; null = not looked up yet
 
 }  // namespace
 }  // namespace lce
@@ -359,35 +445,19 @@ extern "C" lce_status lce_bconv2d_host_noalloc(const lce_bconv2d_desc *desc, con
     lce_status st = check_conv_args(desc, &g, input, weights, multiplier, bias, thresholds, output);
     if (st != LCE_OK) return st;
     if (desc->weights_packed) return LCE_ERR_INVALID_ARG;
-    const HostLayout L = host_layout(g);
-    if (L.total > LCE_STATIC_WORKSPACE_BYTES) return LCE_ERR_WORKSPACE;  // this call does not fit the built-in array
+    if (host_layout(g).total > LCE_STATIC_WORKSPACE_BYTES) return LCE_ERR_WORKSPACE;  // this call does not fit the built-in array
 
     // In host code the array's name is only a stand-in for the symbol, not a device address: ask the
-    // runtime for the address once per device, with that device current.
+    // runtime for the address once per device, with that device current.  (Two threads making the
+    // first call together both look it up and store the same value.)
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LCE_ERR_CUDA;
-    if (g_static_workspace_addr[dev] == nullptr) {
-        void *addr = nullptr;
+    void *addr = g_static_workspace_addr[dev].load(std::memory_order_acquire);
+    if (addr == nullptr) {
         if (cudaGetSymbolAddress(&addr, g_static_workspace) != cudaSuccess || addr == nullptr) return LCE_ERR_CUDA;
-        g_static_workspace_addr[dev] = addr;
+        g_static_workspace_addr[dev].store(addr, std::memory_order_release);
     }
-    char *ws = static_cast<char *>(g_static_workspace_addr[dev]);
-
     // Nothing in the array has to start at zero: every region is written in full (by the copies in,
-    // or by the kernel) before anything reads it.
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    bool ok = cudaMemcpyAsync(ws + L.in, input, L.in_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(ws + L.w, weights, L.w_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    if (multiplier) ok = ok && cudaMemcpyAsync(ws + L.mult, multiplier, L.ch_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    if (bias) ok = ok && cudaMemcpyAsync(ws + L.bias, bias, L.ch_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    if (thresholds) ok = ok && cudaMemcpyAsync(ws + L.thr, thresholds, L.ch_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    if (!ok) return LCE_ERR_CUDA;
-    st = dispatch(desc, g, reinterpret_cast<const uint32_t *>(ws + L.in), reinterpret_cast<const uint32_t *>(ws + L.w),
-                  multiplier ? reinterpret_cast<const float *>(ws + L.mult) : nullptr,
-                  bias ? reinterpret_cast<const float *>(ws + L.bias) : nullptr,
-                  thresholds ? reinterpret_cast<const int32_t *>(ws + L.thr) : nullptr, ws + L.out, s);
-    if (st != LCE_OK) return st;
-    if (cudaMemcpyAsync(output, ws + L.out, L.out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return LCE_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) return LCE_ERR_CUDA;
-    return LCE_OK;
+    // or by the kernel) before anything reads it.  From here on this is lce_bconv2d_host on that array.
+    return host_conv(desc, input, weights, multiplier, bias, thresholds, output, addr, LCE_STATIC_WORKSPACE_BYTES, stream, true);
 }

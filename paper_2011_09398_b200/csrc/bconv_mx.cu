@@ -1,0 +1,900 @@
+// LceBConv2d on the 5th-generation tensor cores with 4-bit operands (tcgen05 kind::mxf4, accumulators
+// in TMEM).  The +-1 multiply-accumulate of the paper's binary GEMM (Section 2: dot = K - 2 popcount(a
+// XOR w); Section 3.2, LceBConv2d) is an exact contraction in any number format that holds +1, -1 and
+// 0: e2m1 holds all three in four bits, block scales of 1.0 change nothing, and the fp32 accumulator
+// is exact for |sum| < 2^24.  One instruction multiplies 128 x N x 64 values, twice the depth of an
+// 8-bit instruction for the same operand bytes, and a zero operand gives the paper's zero-padding
+// variant and the channel padding without any correction term.
+//
+// The packed bits stay the storage and transfer format (32x smaller, Section 3.2).  A 32-bit word
+// of activations or weights becomes one 16-byte row chunk of 32 e2m1 values in shared memory:
+// nibble = 0x2 (+1.0) | bit << 3 (sign), four shift-and-mask operations per word; pad channels of
+// the weights and, for zero-padding, pad pixels are the nibble 0 (0.0).
+//
+// Implicit GEMM, D[channel][position] = W[channel][k] * X[position][k]^T, M = 128 output channels (TMEM
+// lanes), N = a tile of up to 224 grid positions (TMEM columns), K = 64 per instruction:
+//   * positions: the images are stacked into one grid of row pitch Wg and Hg rows per image.  For
+//     stride 1 the pixel (y, x) sits at (y + pad_top, x + pad_left) and rows / images share their pad
+//     positions (the right pad of a row is the left pad of the next); output (oh, ow) is the
+//     position of its window's top-left corner and tap (ky, kx) reads position + ky * Wg + kx.  For
+//     stride 2 the padded image is split into four phase grids (row parity x column parity), in
+//     which tap (ky, kx) of output (oh, ow) is position + (ky / 2) * Wg + kx / 2 of phase
+//     (ky % 2, kx % 2).  Positions that are no output (pad columns, pad rows) are computed and dropped.
+//   * shared memory holds, per phase, [channel word][position][16 bytes]: the B operand of a tap is
+//     the same buffer shifted by the tap's position offset (K-major, no swizzle, rows 16 bytes
+//     apart), so every staged position is expanded once for all taps.
+//   * the weights were expanded when the model was loaded (lce_bconv2d_pack_weights) into the exact
+//     operand image [channel block][tap][channel word][128 channels][16 bytes]; the bulk-copy engine
+//     brings one tap at a time into a ring of shared-memory stages (cp.async.bulk + mbarrier
+//     transaction count).  If the ring holds every tap they are fetched once per CTA, otherwise they
+//     stream past once per tile.
+//   * roles: 8 loader warps (prefetch packed words with cp.async, expand), one thread that issues
+//     the MMAs, one thread that feeds the weight ring, 8 finisher warps (tcgen05.ld, output
+//     transform, stores).  Two position buffers and two accumulator buffers: the expansion of tile
+//     t+1, the MMAs of tile t and the output transform of tile t-1 overlap.  The roles meet only
+//     through mbarriers; every wait is bounded by time, after which the kernel records a status,
+//     waits (bounded) for what it has in flight, frees its TMEM and returns.
+//   * output transform (Section 3.2): a TMEM lane is a channel and a column a position.  Bit-packed
+//     output: the sign of (accumulator - threshold) of 32 positions per lane, then a 32 x 32 bit
+//     transpose across the warp gives each lane the finished word of one pixel.  Float / int32 output
+//     goes through a shared-memory stage [32 positions][128 channels] and leaves as whole pixel rows.
+#include <atomic>
+#include <math.h>
+#include <mutex>
+#include <stdlib.h>
+#include <string.h>
+
+#include "common.cuh"
+#include "mx_common.cuh"
+
+namespace lce {
+namespace {
+
+constexpr int kLoaders = 256;                                // warps 0-7
+constexpr int kFinishers = 512;                              // warps 8-23 (warp % 4 = TMEM lane quarter, four column groups)
+constexpr int kMxThreads = kLoaders + kFinishers + 64;       // + MMA issuer warp + weight producer warp
+constexpr int kIssuerWarp = (kLoaders + kFinishers) / 32;
+constexpr int kProducerTid = (kIssuerWarp + 1) * 32;
+constexpr int kColGroups = kFinishers / 128;                 // finisher warps per TMEM lane quarter
+constexpr int kMaxNt = 224;                                  // tile width (positions); two accumulators + scales fit 512 columns
+constexpr uint32_t kD1Col = 240;                             // TMEM column of the second accumulator buffer
+constexpr uint32_t kSfaCol = 480, kSfbCol = 496;             // block scales (all 1.0) of the A / B operand
+constexpr int kMaxTaps = 64;
+constexpr int kMaxStages = 32;
+constexpr int kPixSlots = 4;
+constexpr int kStageRows = 16, kStageCh = 128;               // float / int32 output stage of one column group
+
+// shared-memory map (bytes)
+constexpr int kOffBars = 0;          // full_x[2] full_d[2] empty_d[2] done full_w[32] empty_w[32]
+constexpr int kOffSlot = 1000;       // TMEM base address; 1004 fills issued, 1008 fills consumed
+constexpr int kOffThr = 1024;        // float[128]
+constexpr int kOffMult = 1536;       // float[128]
+constexpr int kOffBias = 2048;       // float[128]
+constexpr int kOffPix = 2816;        // int32[4][224]: output pixel of a column, or -1
+constexpr int kOffDyn = 6400;        // raw words, weight ring, position buffers, output stage
+
+enum { BAR_FULL_X0 = 0, BAR_FULL_X1, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_DONE, BAR_FULL_W0,
+       BAR_EMPTY_W0 = BAR_FULL_W0 + kMaxStages, BAR_COUNT = BAR_EMPTY_W0 + kMaxStages };
+static_assert(BAR_COUNT * 8 <= kOffSlot, "barriers overlap the TMEM slot");
+
+
+// ---- what a wait that gave up leaves behind --------------------------------------------------------------
+// A device word (read by lce_device_status) and, once it has been set up, a word in mapped host memory
+// that the host reads without synchronising: the next call on that device reports LCE_ERR_DEVICE_TIMEOUT.
+__device__ int g_mx_status = 0;
+
+__device__ __forceinline__ void mx_report_timeout(int *host_flag)
+{
+    g_mx_status = 1;
+    if (host_flag) {
+        *reinterpret_cast<volatile int *>(host_flag) = 1;
+        __threadfence_system();
+    }
+}
+
+constexpr int kFlagDevices = 64;
+std::mutex g_flag_mutex;
+std::atomic<int *> g_flag_host{nullptr};   // int[kFlagDevices] in mapped, portable host memory
+std::atomic<int *> g_flag_dev{nullptr};    // the same array as the devices see it
+
+// Sets the flag array up on first use.  Not a stream operation: must not run while a stream is capturing.
+int *mx_flag_array(bool device_view)
+{
+    int *h = g_flag_host.load(std::memory_order_acquire);
+    if (!h) {
+        std::lock_guard<std::mutex> lock(g_flag_mutex);
+        h = g_flag_host.load(std::memory_order_acquire);
+        if (!h) {
+            void *mem = nullptr, *dev = nullptr;
+            if (cudaHostAlloc(&mem, kFlagDevices * sizeof(int), cudaHostAllocPortable | cudaHostAllocMapped) != cudaSuccess) {
+                cudaGetLastError();
+                return nullptr;
+            }
+            memset(mem, 0, kFlagDevices * sizeof(int));
+            if (cudaHostGetDevicePointer(&dev, mem, 0) != cudaSuccess) {
+                cudaGetLastError();
+                cudaFreeHost(mem);
+                return nullptr;
+            }
+            g_flag_dev.store(static_cast<int *>(dev), std::memory_order_release);
+            g_flag_host.store(static_cast<int *>(mem), std::memory_order_release);
+            h = static_cast<int *>(mem);
+        }
+    }
+    return device_view ? g_flag_dev.load(std::memory_order_acquire) : h;
+}
+
+int current_device_index()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kFlagDevices) return -1;
+    return dev;
+}
+
+// the current device's flag as a kernel argument; null while it cannot be set up (a capturing stream)
+int *mx_flag_for_launch(cudaStream_t s)
+{
+    const int dev = current_device_index();
+    if (dev < 0) return nullptr;
+    if (!g_flag_host.load(std::memory_order_acquire)) {
+        cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(s, &st) != cudaSuccess || st != cudaStreamCaptureStatusNone) {
+            cudaGetLastError();
+            return nullptr;
+        }
+    }
+    int *arr = mx_flag_array(true);
+    return arr ? arr + dev : nullptr;
+}
+
+struct MxParams {
+    const uint32_t *in;
+    const uint8_t *wimg;
+    const float *mult;
+    const float *bias;
+    const int32_t *thr;
+    void *out;
+    const float *residual;   // fused shortcut (float output), or null
+    uint32_t *out_packed;    // fused LceQuantize of the float result, or null
+    int *host_flag;          // host-mapped word set when a wait gives up, or null
+    int32_t N, H, W, Cw, Cw2, Cout, Cow;
+    int32_t OH, OW, KH, KW, stride, pt, pl, K;
+    int32_t Wg, Hg, n_phase;
+    uint32_t Wg_mul, Wg_sh, Hg_mul, Hg_sh, P_mul, P_sh;   // divisions by Wg, Hg, P as multiply + shift
+    int32_t Nt, P;           // tile width; staged positions per tile and phase
+    int32_t n_tiles, total_q;
+    int32_t taps, ksteps, stages, resident;
+    int32_t tap_bytes, raw_words, x_bytes;
+    int32_t off_w, off_x, off_stage;   // byte offsets in shared memory
+    int32_t cp_words;        // words per cp.async: 4, 2 or 1
+    int32_t pad_zero, out_type, activation, vec_out, write_float;
+};
+
+// n / d for 0 <= n < 2^31 with (mul, sh) from the host: floor(n * mul / 2^sh), exact
+__device__ __forceinline__ int fast_div(int n, uint32_t mul, uint32_t sh) { return (int)(((uint64_t)(uint32_t)n * mul) >> sh); }
+
+// position j of the tile that starts at q0, phase ph -> inside the image? and the pixel's word offset
+__device__ __forceinline__ bool mx_locate(const MxParams &p, int q0, int ph, int j, int64_t *word_offset)
+{
+    const int f = q0 + j;
+    const int r = fast_div(f, p.Wg_mul, p.Wg_sh), c = f - r * p.Wg;
+    const int n = fast_div(r, p.Hg_mul, p.Hg_sh), rr = r - n * p.Hg;
+    const int py = p.stride == 2 ? (ph >> 1) : 0, px = p.stride == 2 ? (ph & 1) : 0;
+    const int y = rr * p.stride + py - p.pt, x = c * p.stride + px - p.pl;
+    const bool ok = n < p.N && (unsigned)y < (unsigned)p.H && (unsigned)x < (unsigned)p.W;
+    *word_offset = ok ? (((int64_t)n * p.H + y) * p.W + x) * p.Cw : 0;
+    return ok;
+}
+
+// packed words of the tile's positions -> raw[item][Cw] (pad positions: zero words), asynchronously
+__device__ __forceinline__ void mx_prefetch(const MxParams &p, int q0, uint32_t *raw, int ltid)
+{
+    const int items = p.n_phase * p.P;
+    for (int i = ltid; i < items; i += kLoaders) {
+        const int ph = fast_div(i, p.P_mul, p.P_sh), j = i - ph * p.P;
+        int64_t off;
+        const bool ok = mx_locate(p, q0, ph, j, &off);
+        const uint32_t *src = p.in + off;
+        uint32_t *dst = raw + (size_t)i * p.Cw;
+        if (p.cp_words == 4) {
+            for (int cw = 0; cw < p.Cw; cw += 4) cp_async_zfill<16>(dst + cw, src + cw, ok);
+        } else if (p.cp_words == 2) {
+            for (int cw = 0; cw < p.Cw; cw += 2) cp_async_zfill<8>(dst + cw, src + cw, ok);
+        } else {
+            for (int cw = 0; cw < p.Cw; ++cw) cp_async_zfill<4>(dst + cw, src + cw, ok);
+        }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// every thread expands the words it prefetched itself (same item mapping): waiting for its own copies is enough
+__device__ __forceinline__ void mx_expand(const MxParams &p, int q0, const uint32_t *raw, uint8_t *X, int ltid)
+{
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    const int items = p.n_phase * p.P;
+    for (int i = ltid; i < items; i += kLoaders) {
+        const int ph = fast_div(i, p.P_mul, p.P_sh), j = i - ph * p.P;
+        bool zero = false;
+        if (p.pad_zero) {
+            int64_t off;
+            zero = !mx_locate(p, q0, ph, j, &off);
+        }
+        const uint32_t *src = raw + (size_t)i * p.Cw;
+        uint4 *dst = reinterpret_cast<uint4 *>(X) + (size_t)ph * p.Cw2 * p.P + j;
+        for (int cw = 0; cw < p.Cw; ++cw) {
+            uint4 v = mx_expand_word(src[cw]);
+            if (zero) v = make_uint4(0u, 0u, 0u, 0u);
+            dst[(size_t)cw * p.P] = v;
+        }
+    }
+}
+
+// One lane of the converged warp, the same one every time
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+
+// `count` MMAs of one tap, up to four per block of code.  The whole issuer warp runs this with the same
+// values in every lane, so that the descriptors stay in uniform registers (a single diverged thread
+// pays a register-to-uniform move per operand and MMA, about 200 clocks per instruction, measured);
+// only the elected lane issues.  Descriptor low words advance by additions, the high word never changes.
+__device__ __forceinline__ void mx_issue(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t a_step, uint32_t b_step, int count,
+                                         uint32_t desc_hi, uint32_t idesc, uint32_t sfa, uint32_t sfb, uint32_t &accumulate)
+{
+    for (int i0 = 0; i0 < count; i0 += 4) {
+        const int n = count - i0;
+        const uint32_t a0 = a_lo + (uint32_t)i0 * a_step, b0 = b_lo + (uint32_t)i0 * b_step;
+        if (elect_one()) {
+            asm volatile(
+                "{\n\t.reg .pred pa, pt, g;\n\t.reg .b64 da, db;\n\t"
+                "setp.ne.b32 pa, %13, 0;\n\t"
+                "setp.eq.b32 pt, 0, 0;\n\t"
+                "mov.b64 da, {%1, %9};\n\t mov.b64 db, {%5, %9};\n\t"
+                "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %10, [%11], [%12], pa;\n\t"
+                "setp.gt.s32 g, %14, 1;\n\t mov.b64 da, {%2, %9};\n\t mov.b64 db, {%6, %9};\n\t"
+                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %10, [%11], [%12], pt;\n\t"
+                "setp.gt.s32 g, %14, 2;\n\t mov.b64 da, {%3, %9};\n\t mov.b64 db, {%7, %9};\n\t"
+                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %10, [%11], [%12], pt;\n\t"
+                "setp.gt.s32 g, %14, 3;\n\t mov.b64 da, {%4, %9};\n\t mov.b64 db, {%8, %9};\n\t"
+                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %10, [%11], [%12], pt;\n\t"
+                "}"
+                :
+                : "r"(tmem_d), "r"(a0), "r"(a0 + a_step), "r"(a0 + 2 * a_step), "r"(a0 + 3 * a_step), "r"(b0), "r"(b0 + b_step),
+                  "r"(b0 + 2 * b_step), "r"(b0 + 3 * b_step), "r"(desc_hi), "r"(idesc), "r"(sfa), "r"(sfb), "r"(accumulate), "r"(n)
+                : "memory");
+        }
+        accumulate = 1;
+    }
+}
+
+// a single MMA (one K step per tap: 33..64 input channels)
+__device__ __forceinline__ void mx_issue1(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t sfa,
+                                          uint32_t sfb, uint32_t accumulate)
+{
+    if (elect_one()) {
+        asm volatile(
+            "{\n\t.reg .pred pa;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 pa, %7, 0;\n\t"
+            "mov.b64 da, {%1, %3};\n\t mov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %4, [%5], [%6], pa;\n\t"
+            "}"
+            :
+            : "r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(sfa), "r"(sfb), "r"(accumulate)
+            : "memory");
+    }
+}
+
+// 32 x 32 bit transpose across the warp: in: lane = row, bit j = column j; out: lane j holds column j
+__device__ __forceinline__ uint32_t warp_transpose32(uint32_t m, int lane)
+{
+#pragma unroll
+    for (int k = 16; k >= 1; k >>= 1) {
+        const uint32_t keep = k == 16 ? 0x0000FFFFu : k == 8 ? 0x00FF00FFu : k == 4 ? 0x0F0F0F0Fu : k == 2 ? 0x33333333u : 0x55555555u;
+        const uint32_t y = __shfl_xor_sync(0xffffffffu, m, k);
+        m = (lane & k) ? (((y >> k) & keep) | (m & ~keep)) : ((m & keep) | ((y & keep) << k));
+    }
+    return m;
+}
+
+// Bit-packed output of one tile (Section 3.2: accumulator compared with the per-channel threshold).
+// Lane = channel ch0 + 32 * quarter + lane; this warp takes every fourth 32-column chunk (at most two).
+__device__ __forceinline__ void mx_epilogue_bits(const MxParams &p, uint32_t tmem_d, const int32_t *sPix, int ch0, const float *sThr,
+                                                 int fw, int lane, uint64_t *empty_d)
+{
+    const int quarter = fw & 3, group = fw >> 2;
+    const bool real = ch0 + quarter * 32 < p.Cout;     // whole warp: any channel of its lanes exists
+    const float thr = sThr[quarter * 32 + lane];       // -inf for channels that do not exist: bit 0
+    const uint32_t lane_addr = tmem_d + ((uint32_t)(quarter * 32) << 16);
+    uint32_t *out = static_cast<uint32_t *>(p.out);
+    uint32_t words[2] = {0u, 0u};
+    int pix[2] = {-1, -1};
+    if (real) {
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int c0 = (group + k * kColGroups) * 32;
+            if (c0 >= p.Nt) break;
+            float v[32];
+            const bool full = c0 + 32 <= p.Nt;
+            if (full) tmem_ld32(lane_addr + (uint32_t)c0, v);
+            else tmem_ld16(lane_addr + (uint32_t)c0, v);
+            // bit j = (acc_j < thr): the sign of acc - thr (both are small integers held exactly);
+            // four short chains instead of one long one
+            uint32_t m0 = 0u, m1 = 0u, m2 = 0u, m3 = 0u;
+#pragma unroll
+            for (int j = 7; j >= 0; --j) {
+                m0 = __funnelshift_l(__float_as_uint(v[j] - thr), m0, 1);
+                m1 = __funnelshift_l(__float_as_uint(v[8 + j] - thr), m1, 1);
+                m2 = __funnelshift_l(__float_as_uint(v[16 + j] - thr), m2, 1);
+                m3 = __funnelshift_l(__float_as_uint(v[24 + j] - thr), m3, 1);
+            }
+            uint32_t m = m0 | (m1 << 8);
+            if (full) m |= (m2 << 16) | (m3 << 24);
+            words[k] = warp_transpose32(m, lane);
+            pix[k] = (c0 + lane < p.Nt) ? sPix[c0 + lane] : -1;
+        }
+    }
+    // the accumulator buffer has been read: hand it back before the stores
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    mbar_arrive(empty_d);
+    const int word = (ch0 >> 5) + quarter;
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+        if (pix[k] >= 0) out[(int64_t)pix[k] * p.Cow + word] = words[k];
+}
+
+// Float / int32 output of one tile through the shared-memory stage (Section 3.2: int -> float, fused
+// activation, one multiply-add; Section 5.3: optional shortcut add and re-quantisation).  The four
+// warps of a column group (one per lane quarter) share a stage of 16 positions x 128 channels: each
+// writes its 32 channels of the chunk's positions, then each copies out four whole pixel rows.
+__device__ __forceinline__ void mx_epilogue_staged(const MxParams &p, uint32_t tmem_d, const int32_t *sPix, int ch0, uint32_t *stage_all,
+                                                   float mult, float bias, int fw, int lane, uint64_t *empty_d)
+{
+    const int quarter = fw & 3, group = fw >> 2;
+    const bool real = ch0 + quarter * 32 < p.Cout;
+    const uint32_t lane_addr = tmem_d + ((uint32_t)(quarter * 32) << 16);
+    uint32_t *stage = stage_all + group * (kStageRows * kStageCh);
+    const bool relu = p.activation == LCE_ACT_RELU;
+    const int blk_ch = min(kStageCh, p.Cout - ch0);     // channels of this block that exist
+    const int my_ch = 4 * lane;                          // write-out: four consecutive channels of a pixel per lane
+    const bool act = my_ch < blk_ch;
+    const int n_chunks = p.Nt >> 4;                      // 16-column chunks; this group takes chunk group, group + 4, ...
+    if (group >= n_chunks) {  // a narrow tile leaves this column group without work
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        mbar_arrive(empty_d);
+        return;
+    }
+    const int last_chunk = group + ((n_chunks - 1 - group) / kColGroups) * kColGroups;
+    for (int ck = group; ck < n_chunks; ck += kColGroups) {
+        const int c0 = ck * 16;
+        float v[32];
+        if (real) tmem_ld16(lane_addr + (uint32_t)c0, v);
+        if (ck == last_chunk) {  // last read of the accumulator by this warp
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            mbar_arrive(empty_d);
+        }
+        asm volatile("bar.sync %0, 128;" ::"r"(6 + group) : "memory");  // the stage is free again
+        if (real) {
+            uint32_t *col = stage + quarter * 32 + lane;
+            if (p.out_type == LCE_OUT_FLOAT32) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) col[j * kStageCh] = __float_as_uint(__fmaf_rn(relu ? fmaxf(v[j], 0.f) : v[j], mult, bias));
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) col[j * kStageCh] = (uint32_t)__float2int_rn(v[j]);
+            }
+        }
+        asm volatile("bar.sync %0, 128;" ::"r"(2 + group) : "memory");  // the stage holds the chunk
+        // rows out: warp `quarter` takes positions quarter, quarter + 4, quarter + 8, quarter + 12
+        int pix[4];
+        uint4 q[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = quarter + 4 * u;
+            pix[u] = sPix[c0 + j];  // the same for every lane
+            q[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (act && pix[u] >= 0 && p.vec_out) q[u] = *reinterpret_cast<const uint4 *>(stage + j * kStageCh + my_ch);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (pix[u] < 0) continue;
+            const int j = quarter + 4 * u;
+            const int64_t o = (int64_t)pix[u] * p.Cout + ch0 + my_ch;
+            if (p.vec_out) {
+                if (act) {
+                    if (p.residual) {
+                        const float4 r = __ldg(reinterpret_cast<const float4 *>(p.residual + o));
+                        q[u].x = __float_as_uint(__fadd_rn(__uint_as_float(q[u].x), r.x));
+                        q[u].y = __float_as_uint(__fadd_rn(__uint_as_float(q[u].y), r.y));
+                        q[u].z = __float_as_uint(__fadd_rn(__uint_as_float(q[u].z), r.z));
+                        q[u].w = __float_as_uint(__fadd_rn(__uint_as_float(q[u].w), r.w));
+                    }
+                    if (p.write_float) *reinterpret_cast<uint4 *>(static_cast<uint32_t *>(p.out) + o) = q[u];
+                }
+                if (p.out_packed) {
+                    // sign bits of this lane's four channels, gathered over the eight lanes of a 32-channel word
+                    uint32_t nib = (__uint_as_float(q[u].x) < 0.f ? 1u : 0u) | (__uint_as_float(q[u].y) < 0.f ? 2u : 0u) |
+                                   (__uint_as_float(q[u].z) < 0.f ? 4u : 0u) | (__uint_as_float(q[u].w) < 0.f ? 8u : 0u);
+                    nib <<= 4 * (lane & 7);
+                    nib |= __shfl_xor_sync(0xffffffffu, nib, 1);
+                    nib |= __shfl_xor_sync(0xffffffffu, nib, 2);
+                    nib |= __shfl_xor_sync(0xffffffffu, nib, 4);
+                    if ((lane & 7) == 0 && act) p.out_packed[(int64_t)pix[u] * p.Cow + ((ch0 + my_ch) >> 5)] = nib;
+                }
+            } else if (act) {
+                const uint32_t *srow = stage + j * kStageCh + my_ch;
+                for (int e = 0; e < 4 && my_ch + e < blk_ch; ++e) static_cast<uint32_t *>(p.out)[o + e] = srow[e];
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_constant__ MxParams p)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kOffBars);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kOffSlot);
+    int32_t *fills = reinterpret_cast<int32_t *>(smem + kOffSlot + 4);  // [0] issued by the producer, [1] consumed by the issuer
+    float *sThr = reinterpret_cast<float *>(smem + kOffThr);
+    float *sMult = reinterpret_cast<float *>(smem + kOffMult);
+    float *sBias = reinterpret_cast<float *>(smem + kOffBias);
+    int32_t *sPix = reinterpret_cast<int32_t *>(smem + kOffPix);
+    uint32_t *raw0 = reinterpret_cast<uint32_t *>(smem + kOffDyn);
+    uint8_t *sW = smem + p.off_w;
+    uint8_t *sX0 = smem + p.off_x;
+    uint32_t *stage = reinterpret_cast<uint32_t *>(smem + p.off_stage);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int ch0 = blockIdx.y * 128;
+    const int first_tile = blockIdx.x, tile_step = gridDim.x;
+
+    // ---- set-up (all threads) -------------------------------------------------------------------------
+    for (int e = tid; e < 128; e += kMxThreads) {
+        const bool ok = ch0 + e < p.Cout;
+        float t = -INFINITY;
+        if (ok && p.out_type == LCE_OUT_BITPACKED) {
+            // acc < thr is unchanged by clamping thr to [-K-1, K+1] (|acc| <= K), and then thr is exact in fp32
+            const int32_t ti = __ldg(p.thr + ch0 + e);
+            t = (float)max(-p.K - 1, min(p.K + 1, ti));
+        }
+        sThr[e] = t;
+        sMult[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.mult + ch0 + e) : 0.f;
+        sBias[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.bias + ch0 + e) : 0.f;
+    }
+    if (tid == 0) {
+        mbar_init(&bars[BAR_FULL_X0], kLoaders);
+        mbar_init(&bars[BAR_FULL_X1], kLoaders);
+        mbar_init(&bars[BAR_FULL_D0], 1);
+        mbar_init(&bars[BAR_FULL_D1], 1);
+        mbar_init(&bars[BAR_EMPTY_D0], kFinishers);
+        mbar_init(&bars[BAR_EMPTY_D1], kFinishers);
+        mbar_init(&bars[BAR_DONE], 1);
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(&bars[BAR_FULL_W0 + s], 1);
+            mbar_init(&bars[BAR_EMPTY_W0 + s], 1);
+        }
+        fills[0] = 0;
+        fills[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+    if (warp < 4) {
+        // block scales: every byte 0x7F = 2^0 (ue8m0), for all 128 lanes of the 32 scale columns
+        const uint32_t one = 0x7F7F7F7Fu;
+        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + kSfaCol;
+#pragma unroll
+        for (int c = 0; c < 32; c += 8)
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1};" ::"r"(taddr + c), "r"(one) : "memory");
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+    bool ok = true;
+    if (tid < kLoaders) {
+        // ======================= loaders ==============================================================
+        uint32_t par_full_d[2] = {0, 0};
+        int tile = first_tile;
+        if (tile < p.n_tiles) mx_prefetch(p, tile * p.Nt, raw0, tid);
+        for (int it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+            const int buf = it & 1;
+            if (it >= 2) {  // position buffer `buf` was read by the MMAs of tile it-2
+                ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + buf], par_full_d[buf]);
+                par_full_d[buf] ^= 1u;
+                if (!ok) break;
+            }
+            mx_expand(p, tile * p.Nt, raw0 + buf * p.raw_words, sX0 + (size_t)buf * p.x_bytes, tid);
+            if (tid < p.Nt) {
+                const int f = tile * p.Nt + tid;
+                const int r = fast_div(f, p.Wg_mul, p.Wg_sh), c = f - r * p.Wg;
+                const int n = fast_div(r, p.Hg_mul, p.Hg_sh), rr = r - n * p.Hg;
+                const bool col_ok = n < p.N && rr < p.OH && c < p.OW;
+                sPix[(it & (kPixSlots - 1)) * kMaxNt + tid] = col_ok ? (n * p.OH + rr) * p.OW + c : -1;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive(&bars[BAR_FULL_X0 + buf]);
+            // only now the words of the next tile: the MMAs of this tile must not wait for loads they do not need
+            const int next = tile + tile_step;
+            if (next < p.n_tiles) mx_prefetch(p, next * p.Nt, raw0 + (buf ^ 1) * p.raw_words, tid);
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    } else if (tid < kLoaders + kFinishers) {
+        // ======================= finishers ============================================================
+        const int fw = warp - kLoaders / 32;  // 0..15: lane quarter fw & 3 (= warp & 3), column group fw >> 2
+        uint32_t par_full_d[2] = {0, 0};
+        const int my_channel = (fw & 3) * 32 + lane;
+        const float my_mult = sMult[my_channel], my_bias = sBias[my_channel];
+        int tile = first_tile;
+        for (int it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+            const int buf = it & 1;
+            ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + buf], par_full_d[buf]);
+            par_full_d[buf] ^= 1u;
+            {   // the staged form synchronises the finisher warps among themselves: go on only if all of them got through
+                uint32_t all_ok;
+                asm volatile("{\n\t.reg .pred q, r;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred r, 1, %2, q;\n\tselp.u32 %0, 1, 0, r;\n\t}"
+                             : "=r"(all_ok)
+                             : "r"((uint32_t)ok), "n"(kFinishers)
+                             : "memory");
+                ok = all_ok != 0;
+            }
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
+            const int32_t *pix = sPix + (it & (kPixSlots - 1)) * kMaxNt;
+            if (p.out_type == LCE_OUT_BITPACKED)
+                mx_epilogue_bits(p, tmem_d, pix, ch0, sThr, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
+            else
+                mx_epilogue_staged(p, tmem_d, pix, ch0, stage, my_mult, my_bias, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
+        }
+    } else if (warp == kIssuerWarp) {
+        // ======================= MMA issuer: one warp, every lane with the same values ================
+        // instruction descriptor (block-scaled kinds): A, B = e2m1 (1), both K-major, N >> 3 at bit 17,
+        // scales ue8m0 (bit 23), M >> 4 at bit 24, scale-factor ids 0
+        const uint32_t idesc = (1u << 7) | (1u << 10) | ((uint32_t)(p.Nt >> 3) << 17) | (1u << 23) | ((uint32_t)(128 >> 4) << 24);
+        // shared-memory descriptors (units of 16 bytes): low = start | K-chunk stride << 16; high = 8-row
+        // group stride (128 bytes) | version 1 at bit 46; no swizzle
+        const uint32_t desc_hi = 8u | (1u << 14);
+        const uint32_t w_lo0 = ((uint32_t)p.off_w >> 4) + (smem_u32(smem) >> 4) + (128u << 16);
+        const uint32_t tap_units = (uint32_t)p.tap_bytes >> 4;
+        const uint32_t sfa = tmem_base + kSfaCol, sfb = tmem_base + kSfbCol;
+        uint32_t par_full_x[2] = {0, 0}, par_empty_d[2] = {0, 0};
+        int g = 0, stage_i = 0;
+        uint32_t w_parity = 0;
+        for (int tile = first_tile, it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+            const int buf = it & 1;
+            ok = mbar_wait_bounded(&bars[BAR_FULL_X0 + buf], par_full_x[buf]);
+            par_full_x[buf] ^= 1u;
+            if (ok && it >= 2) {  // the accumulator buffer must have been read out
+                ok = mbar_wait_bounded(&bars[BAR_EMPTY_D0 + buf], par_empty_d[buf]);
+                par_empty_d[buf] ^= 1u;
+            }
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
+            const uint32_t x_lo0 = ((uint32_t)p.off_x >> 4) + (smem_u32(smem) >> 4) + (uint32_t)buf * ((uint32_t)p.x_bytes >> 4) + ((uint32_t)p.P << 16);
+            uint32_t accumulate = 0;
+            for (int ky = 0; ky < p.KH && ok; ++ky) {
+                for (int kx = 0; kx < p.KW; ++kx) {
+                    if (!p.resident || it == 0) {
+                        ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_FULL_W0 + stage_i], w_parity));
+                        if (!ok) break;
+                        ++g;
+                        if (lane == 0) fills[1] = g;
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    }
+                    // B operand of the tap: its phase buffer (stride 2) shifted by the tap's position offset
+                    uint32_t b_off;
+                    if (p.stride == 2) b_off = (uint32_t)((((ky & 1) * 2 + (kx & 1)) * p.Cw2) * p.P + (ky >> 1) * p.Wg + (kx >> 1));
+                    else b_off = (uint32_t)(ky * p.Wg + kx);
+                    const uint32_t a_lo = w_lo0 + (uint32_t)stage_i * tap_units;
+                    if (p.ksteps == 1) {
+                        mx_issue1(tmem_d, a_lo, x_lo0 + b_off, desc_hi, idesc, sfa, sfb, accumulate);
+                        accumulate = 1;
+                    } else {
+                        mx_issue(tmem_d, a_lo, x_lo0 + b_off, 256u, 2u * (uint32_t)p.P, p.ksteps, desc_hi, idesc, sfa, sfb, accumulate);
+                    }
+                    if (!p.resident && elect_one()) mma_commit(&bars[BAR_EMPTY_W0 + stage_i]);
+                    if (++stage_i == p.stages) { stage_i = 0; w_parity ^= 1u; }
+                }
+            }
+            if (!ok) break;
+            if (elect_one()) mma_commit(&bars[BAR_FULL_D0 + buf]);
+        }
+    } else if (tid == kProducerTid) {
+        // ======================= weight producer: one thread ==========================================
+        int my_tiles = 0;
+        for (int tile = first_tile; tile < p.n_tiles; tile += tile_step) ++my_tiles;
+        const int total = p.resident ? p.taps : my_tiles * p.taps;
+        const uint8_t *src = p.wimg + (size_t)blockIdx.y * p.taps * p.tap_bytes;
+        int stage_i = 0, tap = 0;
+        uint32_t e_parity = 1;  // the first pass over the ring waits for nothing
+        for (int g = 0; g < total; ++g) {
+            if (g >= p.stages) {
+                ok = mbar_wait_bounded(&bars[BAR_EMPTY_W0 + stage_i], e_parity);
+                if (!ok) break;
+            }
+            mbar_expect_tx(&bars[BAR_FULL_W0 + stage_i], (uint32_t)p.tap_bytes);
+            bulk_copy_g2s(sW + (size_t)stage_i * p.tap_bytes, src + (size_t)tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0 + stage_i]);
+            fills[0] = g + 1;
+            if (++tap == p.taps) tap = 0;
+            if (++stage_i == p.stages) { stage_i = 0; e_parity ^= 1u; }
+        }
+    }
+    if (!ok) mx_report_timeout(p.host_flag);
+
+    // ---- tear-down: nothing of this CTA may still be in flight when its TMEM and shared memory go ----
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == kIssuerWarp && elect_one()) {              // the lane that issued the MMAs
+        mma_commit(&bars[BAR_DONE]);                       // arrives when every MMA issued above has finished
+        bool drained = mbar_wait_bounded(&bars[BAR_DONE], 0);
+        // weight copies that were started but never consumed (only after a wait gave up)
+        const int issued = fills[0], consumed = fills[1];
+        for (int g = consumed; g < issued && drained; ++g)
+            drained = mbar_wait_bounded(&bars[BAR_FULL_W0 + g % p.stages], (uint32_t)(g / p.stages) & 1u);
+        if (!drained) mx_report_timeout(p.host_flag);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+}
+
+// ---- load-time weight image -----------------------------------------------------------------------------
+// plain packed words [Cout][taps][Cw] -> e2m1 operand image [channel block][tap][Cw2][128 channels][16 bytes];
+// channels past Cout, the pad channel word of an odd Cw and channels past Cin inside a word are 0.0
+__global__ void mx_pack_weights_kernel(const uint32_t *w, uint4 *image, int Cout, int Cin, int Cw, int Cw2, int taps, int n_blocks)
+{
+    const int64_t total = (int64_t)n_blocks * taps * Cw2 * 128;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int row = (int)(e & 127);
+        int64_t t = e >> 7;
+        const int cw = (int)(t % Cw2);
+        t /= Cw2;
+        const int tap = (int)(t % taps);
+        const int blk = (int)(t / taps);
+        const int o = blk * 128 + row;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (o < Cout && cw < Cw) {
+            v = mx_expand_word(w[((int64_t)o * taps + tap) * Cw + cw]);
+            const int valid = Cin - cw * 32;  // channels of this word that exist
+            if (valid < 32) {
+                // value (register j, nibble i) is channel 4 i + j of the word
+                uint32_t m[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    m[j] = 0u;
+                    for (int i = 0; i < 8; ++i)
+                        if (4 * i + j < valid) m[j] |= 0xFu << (4 * i);
+                }
+                v.x &= m[0]; v.y &= m[1]; v.z &= m[2]; v.w &= m[3];
+            }
+        }
+        image[e] = v;
+    }
+}
+
+struct MxPlan {
+    int Nt, P, stages, resident, n_blocks, ctas_x, n_tiles, total_q, Wg, Hg, n_phase, Cw2, taps, halo;
+    size_t raw_words, x_bytes, tap_bytes, off_w, off_x, off_stage, smem;
+};
+
+constexpr size_t kSmemLimit = 227 * 1024;
+
+bool mx_plan(const ConvGeom &g, int sms, MxPlan *pl)
+{
+    if (g.sh != g.sw || (g.sh != 1 && g.sh != 2)) return false;
+    if (g.Cw > 32) return false;
+    const int taps = g.KH * g.KW;
+    if (taps > kMaxTaps) return false;
+    const int s = g.sh;
+    int Wg, Hg, halo;
+    if (s == 1) {
+        const int pr = max(0, (g.OW - 1) + g.KW - g.W - g.pl), pb = max(0, (g.OH - 1) + g.KH - g.H - g.pt);
+        Wg = g.W + max(g.pl, pr);
+        Hg = g.H + max(g.pt, pb);
+        halo = (g.KH - 1) * Wg + (g.KW - 1);
+    } else {
+        Wg = g.OW + (g.KW - 1) / 2;
+        Hg = g.OH + (g.KH - 1) / 2;
+        halo = ((g.KH - 1) / 2) * Wg + (g.KW - 1) / 2;
+    }
+    const int64_t total_q = (int64_t)g.N * Hg * Wg;
+    if (total_q >= (1ll << 31) - 4096 || g.M >= (1ll << 31)) return false;
+    pl->Wg = Wg; pl->Hg = Hg; pl->halo = halo; pl->total_q = (int)total_q;
+    pl->n_phase = s * s;
+    pl->Cw2 = g.Cw + (g.Cw & 1);
+    pl->taps = taps;
+    pl->tap_bytes = (size_t)pl->Cw2 * 2048;
+    pl->n_blocks = (g.Cout + 127) / 128;
+    const int ctas_max = max(1, sms / pl->n_blocks);
+    const bool staged = g.out_type != LCE_OUT_BITPACKED;
+    const size_t stage_bytes = staged ? (size_t)kColGroups * kStageRows * kStageCh * 4 : 0;
+    const int ksteps = pl->Cw2 / 2;
+    double best = 1e30;
+    bool found = false;
+    for (int nt = 16; nt <= kMaxNt; nt += 16) {
+        const int P = nt + halo;
+        if (P > 16383) break;  // descriptor strides are 14-bit counts of 16 bytes
+        const size_t raw_words = (((size_t)pl->n_phase * P * g.Cw + 3) / 4) * 4;
+        const size_t x_bytes = (size_t)pl->n_phase * pl->Cw2 * P * 16;
+        const size_t fixed = kOffDyn + 2 * raw_words * 4;
+        const size_t off_w = (fixed + 127) / 128 * 128;
+        const size_t rest = 2 * x_bytes + stage_bytes + 256;
+        if (off_w + rest + 2 * pl->tap_bytes > kSmemLimit) continue;
+        int stages = (int)((kSmemLimit - off_w - rest) / pl->tap_bytes);
+        if (stages > kMaxStages) stages = kMaxStages;
+        const bool resident = stages >= taps;
+        if (resident) stages = taps;
+        const int n_tiles = (int)((total_q + nt - 1) / nt);
+        const int ctas_x = min(ctas_max, n_tiles);
+        const int per_cta = (n_tiles + ctas_x - 1) / ctas_x;
+        // clocks per MMA: 43 + N/2, at least 95 (measured); streamed weights cost about as much again from L2
+        const double mma = (double)taps * ksteps * fmax(95.0, 43.0 + nt / 2.0);
+        const double tile = fmax(mma, resident ? 0.0 : (double)taps * pl->tap_bytes / 48.0) + 250.0;
+        const double cost = per_cta * tile;
+        if (cost < best) {
+            best = cost;
+            found = true;
+            pl->Nt = nt; pl->P = P; pl->stages = stages; pl->resident = resident ? 1 : 0;
+            pl->n_tiles = n_tiles; pl->ctas_x = ctas_x;
+            pl->raw_words = raw_words; pl->x_bytes = x_bytes;
+            pl->off_w = off_w;
+            pl->off_x = (off_w + (size_t)stages * pl->tap_bytes + 127) / 128 * 128;
+            pl->off_stage = pl->off_x + 2 * x_bytes;
+            pl->smem = pl->off_stage + stage_bytes;
+        }
+    }
+    return found;
+}
+
+// floor(n / d) = (n * mul) >> sh for every 0 <= n < 2^31: sh = 31 + ceil(log2 d), mul = floor(2^sh / d) + 1
+// (the excess mul * d - 2^sh is at most d <= 2^(sh - 31), so n * excess < 2^sh)
+void fast_div_constants(uint32_t d, uint32_t *mul, uint32_t *sh)
+{
+    uint32_t l = 0;
+    while ((1ull << l) < d) ++l;
+    *sh = 31 + l;
+    *mul = (uint32_t)(((1ull << (31 + l)) / d) + 1);
+}
+
+int device_sms()
+{
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return sms > 0 ? sms : 148;
+}
+
+}  // namespace
+
+bool tensor_covers(const ConvGeom &g)
+{
+    MxPlan pl;
+    return mx_plan(g, 148, &pl);
+}
+
+size_t tensor_weight_image_bytes(const ConvGeom &g)
+{
+    MxPlan pl;
+    if (!mx_plan(g, 148, &pl)) return 0;
+    return (size_t)pl.n_blocks * pl.taps * pl.tap_bytes;
+}
+
+lce_status launch_pack_weights_tensor(const ConvGeom &g, const uint32_t *w, void *image, cudaStream_t s)
+{
+    MxPlan pl;
+    if (!mx_plan(g, 148, &pl)) return LCE_ERR_UNSUPPORTED;
+    const int64_t total = (int64_t)pl.n_blocks * pl.taps * pl.Cw2 * 128;
+    const int64_t want = (total + 255) / 256;
+    const int blocks = (int)(want < 4096 ? want : 4096);
+    mx_pack_weights_kernel<<<blocks, 256, 0, s>>>(w, static_cast<uint4 *>(image), g.Cout, g.Cin, g.Cw, pl.Cw2, pl.taps, pl.n_blocks);
+    mx_flag_array(false);  // load time is the moment to set up the host-visible status word (it cannot be done under stream capture)
+    return launch_status();
+}
+
+lce_status tensor_plan_info(const ConvGeom &g, TensorPlanInfo *info)
+{
+    MxPlan pl;
+    if (!mx_plan(g, device_sms(), &pl)) return LCE_ERR_UNSUPPORTED;
+    info->tile_positions = pl.Nt;
+    info->ctas = pl.ctas_x * pl.n_blocks;
+    info->weight_stages = pl.stages;
+    info->weights_resident = pl.resident;
+    info->shared_bytes = (int64_t)pl.smem;
+    return LCE_OK;
+}
+
+lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const void *w_image, const float *mult, const float *bias,
+                               const int32_t *thr, void *out, cudaStream_t s, const float *residual, uint32_t *out_packed)
+{
+    MxPlan pl;
+    if (!w_image || !mx_plan(g, device_sms(), &pl)) return LCE_ERR_UNSUPPORTED;
+    MxParams p{};
+    p.in = in; p.wimg = static_cast<const uint8_t *>(w_image); p.mult = mult; p.bias = bias; p.thr = thr; p.out = out;
+    p.residual = residual; p.out_packed = out_packed;
+    p.host_flag = mx_flag_for_launch(s);
+    p.N = g.N; p.H = g.H; p.W = g.W; p.Cw = g.Cw; p.Cw2 = pl.Cw2; p.Cout = g.Cout; p.Cow = g.Cow;
+    p.OH = g.OH; p.OW = g.OW; p.KH = g.KH; p.KW = g.KW; p.stride = g.sh; p.pt = g.pt; p.pl = g.pl;
+    p.K = g.KH * g.KW * g.Cin;
+    p.Wg = pl.Wg; p.Hg = pl.Hg; p.n_phase = pl.n_phase;
+    fast_div_constants((uint32_t)pl.Wg, &p.Wg_mul, &p.Wg_sh);
+    fast_div_constants((uint32_t)pl.Hg, &p.Hg_mul, &p.Hg_sh);
+    fast_div_constants((uint32_t)pl.P, &p.P_mul, &p.P_sh);
+    p.Nt = pl.Nt; p.P = pl.P; p.n_tiles = pl.n_tiles; p.total_q = pl.total_q;
+    p.taps = pl.taps; p.ksteps = pl.Cw2 / 2; p.stages = pl.stages; p.resident = pl.resident;
+    p.tap_bytes = (int32_t)pl.tap_bytes; p.raw_words = (int32_t)pl.raw_words; p.x_bytes = (int32_t)pl.x_bytes;
+    p.off_w = (int32_t)pl.off_w; p.off_x = (int32_t)pl.off_x; p.off_stage = (int32_t)pl.off_stage;
+    p.cp_words = (g.Cw % 4 == 0 && aligned(in, 16)) ? 4 : (g.Cw % 2 == 0 && aligned(in, 8)) ? 2 : 1;
+    p.pad_zero = g.padding == LCE_PAD_SAME_ZERO;
+    p.out_type = g.out_type; p.activation = g.activation;
+    p.write_float = out != nullptr;
+    p.vec_out = (g.Cout % 4 == 0) && aligned(out, 16) && aligned(residual, 16);
+    if ((residual || out_packed) && (!p.vec_out || g.Cout % 32 != 0)) return LCE_ERR_UNSUPPORTED;
+    if (!aligned(w_image, 16)) return LCE_ERR_ALIGNMENT;
+    static SmemOptIn opted;
+    if (!opted.ensure(bconv_mx_kernel, pl.smem)) return LCE_ERR_CUDA;
+    bconv_mx_kernel<<<dim3((unsigned)pl.ctas_x, (unsigned)pl.n_blocks), kMxThreads, pl.smem, s>>>(p);
+    return launch_status();
+}
+
+
+// ---- status of the bounded waits ----------------------------------------------------------------------
+namespace {
+// One CTA waits, with the kernels' own helper and the given limit, on a barrier that nobody arrives
+// at, and reports the expiry the way the convolution kernels do.  Touches no tensor-core state.
+__global__ void mx_wait_probe_kernel(uint64_t limit_ns, int *host_flag)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!mbar_wait_bounded(&bar, 0, limit_ns)) mx_report_timeout(host_flag);
+    }
+}
+}  // namespace
+
+lce_status tensor_wait_probe(uint64_t limit_ns, cudaStream_t s)
+{
+    mx_wait_probe_kernel<<<1, 32, 0, s>>>(limit_ns, mx_flag_for_launch(s));
+    return launch_status();
+}
+
+// 0 = no bounded wait has given up on the current device since the library was loaded (or since the reset).
+lce_status tensor_device_status(int *status)
+{
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_mx_status, sizeof(int)) != cudaSuccess) return LCE_ERR_CUDA;
+    *status = v;
+    return LCE_OK;
+}
+
+lce_status tensor_device_status_reset()
+{
+    const int zero = 0;
+    if (cudaMemcpyToSymbol(g_mx_status, &zero, sizeof(int)) != cudaSuccess) return LCE_ERR_CUDA;
+    const int dev = current_device_index();
+    int *arr = g_flag_host.load(std::memory_order_acquire);
+    if (arr && dev >= 0) *reinterpret_cast<volatile int *>(arr + dev) = 0;
+    return LCE_OK;
+}
+
+// Host-side look at the mapped word: no synchronisation, no CUDA call beyond cudaGetDevice.
+bool tensor_timeout_flagged()
+{
+    int *arr = g_flag_host.load(std::memory_order_acquire);
+    if (!arr) return false;
+    const int dev = current_device_index();
+    return dev >= 0 && *reinterpret_cast<volatile int *>(arr + dev) != 0;
+}
+
+}  // namespace lce

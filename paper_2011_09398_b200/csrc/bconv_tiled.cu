@@ -39,29 +39,6 @@ namespace {
 
 // ---- host side: launchers, the tile / range chooser, weight packing, plan and launch ----------------
 
-// The opt-in to more than 48 KB of dynamic shared memory is a driver call; it is made once per kernel,
-// device and size (a larger request later raises it), not on every launch.  One instance per kernel.
-struct SmemOptIn {
-    static constexpr int kDevices = 64;
-    std::atomic<size_t> granted[kDevices];
-    SmemOptIn() { for (auto &g : granted) g.store(0, std::memory_order_relaxed); }
-    template <typename Kernel>
-    bool ensure(Kernel kernel, size_t smem_bytes)
-    {
-        if (smem_bytes <= 48 * 1024) return true;
-        int dev = -1;
-        if (cudaGetDevice(&dev) != cudaSuccess) return false;
-        const bool tracked = dev >= 0 && dev < kDevices;
-        if (tracked && granted[dev].load(std::memory_order_acquire) >= smem_bytes) return true;
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess) return false;
-        if (tracked) {  // concurrent callers may both set the attribute; the recorded size only grows
-            size_t seen = granted[dev].load(std::memory_order_relaxed);
-            while (seen < smem_bytes && !granted[dev].compare_exchange_weak(seen, smem_bytes, std::memory_order_release)) {}
-        }
-        return true;
-    }
-};
-
 template <int TP>
 lce_status launch1x1(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStream_t s)
 {

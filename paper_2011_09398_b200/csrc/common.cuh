@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "lce.h"
 
 namespace lce {
@@ -69,6 +71,29 @@ inline lce_status launch_status()
     return cudaGetLastError() == cudaSuccess ? LCE_OK : LCE_ERR_CUDA;
 }
 
+// The opt-in to more than 48 KB of dynamic shared memory is a driver call; it is made once per kernel,
+// device and size (a larger request later raises it), not on every launch.  One instance per kernel.
+struct SmemOptIn {
+    static constexpr int kDevices = 64;
+    std::atomic<size_t> granted[kDevices];
+    SmemOptIn() { for (auto &g : granted) g.store(0, std::memory_order_relaxed); }
+    template <typename Kernel>
+    bool ensure(Kernel kernel, size_t smem_bytes)
+    {
+        if (smem_bytes <= 48 * 1024) return true;
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess) return false;
+        const bool tracked = dev >= 0 && dev < kDevices;
+        if (tracked && granted[dev].load(std::memory_order_acquire) >= smem_bytes) return true;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess) return false;
+        if (tracked) {  // concurrent callers may both set the attribute; the recorded size only grows
+            size_t seen = granted[dev].load(std::memory_order_relaxed);
+            while (seen < smem_bytes && !granted[dev].compare_exchange_weak(seen, smem_bytes, std::memory_order_release)) {}
+        }
+        return true;
+    }
+};
+
 // Kernel entry points implemented in the other translation units.
 lce_status launch_bconv_direct(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const float *mult,
                                const float *bias, const int32_t *thr, void *out, cudaStream_t s);
@@ -84,11 +109,27 @@ lce_status launch_bconv_tiled(const ConvGeom &g, const uint32_t *in, const uint3
 bool patch_covers(const ConvGeom &g);
 lce_status launch_bconv_patch(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const float *mult,
                               const float *bias, const int32_t *thr, void *out, cudaStream_t s);
-// Tensor-core (tcgen05 kind::i8) kernel: 3x3, stride 1, one-padding; plain weights.
+// Tensor-core kernel (tcgen05 kind::mxf4 on e2m1 operands): any filter of up to 64 taps, equal strides
+// of 1 or 2, every padding mode; needs the weight image that launch_pack_weights_tensor writes at load
+// time (w_image; null -> LCE_ERR_UNSUPPORTED).  residual / out_packed as for the tiled kernel (float
+// output, out_c a multiple of 32).
 bool tensor_covers(const ConvGeom &g);
-lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const uint32_t *w, const float *mult,
-                               const float *bias, const int32_t *thr, void *out, cudaStream_t s);
+size_t tensor_weight_image_bytes(const ConvGeom &g);
+lce_status launch_pack_weights_tensor(const ConvGeom &g, const uint32_t *w, void *image, cudaStream_t s);
+lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const void *w_image, const float *mult,
+                               const float *bias, const int32_t *thr, void *out, cudaStream_t s,
+                               const float *residual = nullptr, uint32_t *out_packed = nullptr);
+struct TensorPlanInfo {
+    int32_t tile_positions, ctas, weight_stages, weights_resident;
+    int64_t shared_bytes;
+};
+lce_status tensor_plan_info(const ConvGeom &g, TensorPlanInfo *info);
+// Bounded device-side waits: status word, its reset, the host-visible flag (no synchronisation), and a
+// tiny kernel whose wait is meant to run out (nobody arrives at its barrier).
 lce_status tensor_device_status(int *status);
+lce_status tensor_device_status_reset();
+bool tensor_timeout_flagged();
+lce_status tensor_wait_probe(uint64_t limit_ns, cudaStream_t s);
 // Bytes of the tiled kernel's weight image for this geometry (0 if the kernel does not cover it).
 // Launch plan of the tiled kernels for a geometry (no buffers involved), for lce_bconv2d_plan.
 struct TiledPlanInfo {

@@ -84,10 +84,10 @@ def test_binding_refuses_cpu_tensors():
 
 # ---- launch plans (host arithmetic only): the work split the kernels rely on ----------------------
 
-def _plan(N, H, W, Cin, Cout, k, s, padding=None, kernel_choice=None, out_type=None):
+def _plan(N, H, W, Cin, Cout, k, s, padding=None, kernel_choice=None, out_type=None, packed=0):
     d = lce.make_desc(N, H, W, Cin, Cout, (k, k), (s, s), lce.PAD_SAME_ONE if padding is None else padding,
                       lce.OUT_BITPACKED if out_type is None else out_type, lce.ACT_NONE,
-                      lce.KERNEL_AUTO if kernel_choice is None else kernel_choice)
+                      lce.KERNEL_AUTO if kernel_choice is None else kernel_choice, packed)
     oh, ow = lce.lce_bconv2d_out_shape(d)
     return lce.lce_bconv2d_plan(d), N * oh * ow
 
@@ -132,13 +132,50 @@ def test_plan_names_the_other_kernels(lib):
     assert _plan(1, 9, 9, 64, 64, 7, 1)[0]["kernel"] == lce.KERNEL_DIRECT                    # no tiled 7x7
     assert _plan(1, 3, 4, 7300, 5, 3, 1)[0]["kernel"] == lce.KERNEL_DIRECT                   # K >= 65536 (and far more weights than shared memory holds)
     assert _plan(1, 9, 9, 64, 64, 3, 1, kernel_choice=lce.KERNEL_DIRECT)[0]["kernel"] == lce.KERNEL_DIRECT
-    assert _plan(1, 9, 9, 64, 64, 3, 1, kernel_choice=lce.KERNEL_TENSOR)[0]["kernel"] == lce.KERNEL_TENSOR
+    assert _plan(1, 9, 9, 64, 64, 3, 1, kernel_choice=lce.KERNEL_TENSOR, packed=1)[0]["kernel"] == lce.KERNEL_TENSOR
     with pytest.raises(lce.LceError) as e:
         _plan(1, 9, 9, 64, 64, 7, 1, kernel_choice=lce.KERNEL_TILED)
     assert e.value.status == 2
     with pytest.raises(lce.LceError) as e:
-        _plan(1, 9, 9, 64, 64, 3, 2, kernel_choice=lce.KERNEL_TENSOR)                        # tensor path: stride 1 only
+        _plan(1, 9, 9, 64, 64, 3, 1, kernel_choice=lce.KERNEL_TENSOR)                        # tensor path: packed weights only
     assert e.value.status == 2
+    with pytest.raises(lce.LceError) as e:
+        _plan(1, 9, 9, 64, 64, 3, 3, kernel_choice=lce.KERNEL_TENSOR, packed=1)              # tensor path: strides 1 and 2
+    assert e.value.status == 2
+    with pytest.raises(lce.LceError) as e:
+        _plan(1, 9, 9, 1056, 64, 3, 1, kernel_choice=lce.KERNEL_TENSOR, packed=1)            # tensor path: at most 32 channel words
+    assert e.value.status == 2
+
+
+TENSOR_PLAN_SHAPES = [(64, 56, 56, 64, 64, 3, 1), (64, 28, 28, 128, 128, 3, 1), (64, 14, 14, 256, 256, 3, 1), (64, 7, 7, 512, 512, 3, 1),
+                      (64, 56, 56, 64, 128, 3, 2), (64, 28, 28, 256, 256, 3, 2), (64, 14, 14, 256, 512, 1, 1), (256, 112, 112, 32, 64, 3, 2),
+                      (64, 64, 64, 256, 256, 5, 1), (64, 32, 32, 96, 96, 5, 1), (128, 28, 28, 64, 128, 1, 1), (8, 9, 9, 512, 40, 7, 2)]
+
+
+@pytest.mark.parametrize("out_type", [lce.OUT_BITPACKED, lce.OUT_FLOAT32])
+@pytest.mark.parametrize("shape", TENSOR_PLAN_SHAPES)
+def test_tensor_plan_fits_the_sm_and_auto_takes_it_for_large_packed_layers(lib, shape, out_type):
+    forced, _ = _plan(*shape, kernel_choice=lce.KERNEL_TENSOR, out_type=out_type, packed=1)
+    assert forced["kernel"] == lce.KERNEL_TENSOR
+    assert forced["tile_pixels"] % 16 == 0 and 16 <= forced["tile_pixels"] <= 224       # N of the MMA, two accumulators in 512 columns
+    assert 0 < forced["shared_bytes"] <= 227 * 1024
+    assert 1 <= forced["ctas"] <= 148
+    k = shape[5]
+    assert min(2, k * k) <= forced["weight_stages"] <= k * k and forced["weights_resident"] == (forced["weight_stages"] == k * k)
+    auto, M = _plan(*shape, out_type=out_type, packed=1)
+    macs = M * shape[4] * k * k * shape[3]
+    assert (auto["kernel"] == lce.KERNEL_TENSOR) == (macs >= 2 ** 28)
+    assert _plan(*shape, out_type=out_type)[0]["kernel"] != lce.KERNEL_TENSOR             # plain weights: integer kernels
+
+
+def test_packed_weights_buffer_holds_the_three_parts(lib):
+    d = lce.make_desc(64, 28, 28, 128, 128, (3, 3), (1, 1))
+    plain = 128 * 9 * 4 * 4
+    total = lce.lce_bconv2d_packed_weights_bytes(d)
+    tensor_image = 1 * 9 * 4 * 2048        # [channel block][tap][channel word][128 channels][16 bytes]
+    assert total > plain + tensor_image and total % 256 == 0
+    odd = lce.make_desc(1, 8, 8, 96, 130, (3, 3), (1, 1))   # 3 channel words are padded to 4, 130 channels to 2 blocks
+    assert lce.lce_bconv2d_packed_weights_bytes(odd) >= 130 * 9 * 3 * 4 + 2 * 9 * 4 * 2048
 
 
 def test_plans_are_remembered_per_geometry_not_mixed_up(lib):
@@ -168,7 +205,7 @@ def test_plan_objects_check_their_arguments_on_the_host(lib):
     assert handle.value is None
     assert lib.lce_bconv2d_plan_create(ctypes.byref(d), fake, fake, fake, fake, None, fake, None) == 1      # nowhere to put the handle
     assert lib.lce_bconv2d_plan_create(ctypes.byref(d), ctypes.c_void_p(258), fake, fake, fake, None, fake, ctypes.byref(handle)) == 3
-    forced = lce.make_desc(1, 9, 9, 64, 64, (3, 3), (2, 2), kernel_choice=lce.KERNEL_TENSOR)                   # tensor path: stride 1 only
+    forced = lce.make_desc(1, 9, 9, 64, 64, (3, 3), (2, 2), kernel_choice=lce.KERNEL_TENSOR)                   # tensor path: packed weights only
     assert lib.lce_bconv2d_plan_create(ctypes.byref(forced), fake, fake, fake, fake, None, fake, ctypes.byref(handle)) == 2
     assert lib.lce_bconv2d_plan_create(ctypes.byref(d), fake, fake, fake, fake, None, fake, ctypes.byref(handle)) == 0
     assert handle.value

@@ -13,8 +13,20 @@ from gpu_util import DEV, guarded, guards_intact, run_bconv, to_dev, to_dev_word
 pytestmark = pytest.mark.gpu
 
 # (kernel choice, weights packed at load time?)
-KERNELS = [(lce.KERNEL_DIRECT, False), (lce.KERNEL_AUTO, False), (lce.KERNEL_AUTO, True)]
-KERNEL_IDS = ["direct", "auto", "auto-packed"]
+KERNELS = [(lce.KERNEL_DIRECT, False), (lce.KERNEL_AUTO, False), (lce.KERNEL_AUTO, True), (lce.KERNEL_TENSOR, True)]
+KERNEL_IDS = ["direct", "auto", "auto-packed", "tensor"]
+
+
+def skip_unless_covered(kernel_choice, N, H, W, Cin, Cout, k, s, padding):
+    """The tensor-core kernel is forced in these tests; shapes it does not cover are reported as such."""
+    if kernel_choice[0] != lce.KERNEL_TENSOR:
+        return
+    desc = lce.make_desc(N, H, W, Cin, Cout, (k, k), (s, s), padding, lce.OUT_FLOAT32, lce.ACT_NONE, lce.KERNEL_TENSOR, 1)
+    try:
+        lce.lce_bconv2d_plan(desc)
+    except lce.LceError as e:
+        assert e.status == 2
+        pytest.skip("not covered by the tensor-core kernel")
 
 
 def rand_pm1(rng, shape):
@@ -108,6 +120,7 @@ def test_bconv_all_output_types_match_oracle(shape, padding, kernel_choice):
     N, H, W, Cin, Cout, k, s = shape
     if padding == lce.PAD_VALID and (H < k or W < k):
         pytest.skip("empty VALID output")
+    skip_unless_covered(kernel_choice, N, H, W, Cin, Cout, k, s, padding)
     rng = np.random.default_rng(abs(hash((shape, padding))) % 2**32)
     a, w = rand_pm1(rng, (N, H, W, Cin)), rand_pm1(rng, (Cout, k, k, Cin))
     aw, ww = oracle.bitpack_pm1(a), oracle.bitpack_pm1(w)
@@ -140,7 +153,7 @@ def test_saturated_thresholds_and_pad_bits(kernel_choice):
     assert np.all(ones[..., 0] == 0xFFFFFFFF) and np.all(ones[..., 1] == 0xFF)
 
 
-# ---- tensor-core formulation (tcgen05 kind::i8): same integers, same bits ------------------------
+# ---- tensor-core formulation (tcgen05 kind::mxf4 on +-1 / 0 e2m1 values): same integers, same bits ------
 
 TENSOR_SHAPES = [
     # N, H, W, Cin, Cout  (3x3, stride 1, one-padding)
@@ -151,6 +164,8 @@ TENSOR_SHAPES = [
     (2, 30, 30, 32, 128), (6, 20, 17, 64, 100), (1, 80, 80, 33, 33), (3, 40, 3, 96, 64),
     # float / int32 output with Cout <= 64, a multiple of 4: the same schedule with the shared-memory stage
     (2, 20, 20, 64, 48), (1, 30, 30, 32, 8), (4, 16, 16, 40, 60), (1, 12, 12, 64, 4), (3, 33, 31, 64, 32),
+    # several tiles per CTA (more than 148 x 224 positions), three channel blocks, odd channel-word counts
+    (40, 30, 30, 64, 64), (24, 28, 28, 96, 300), (9, 56, 56, 160, 64),
 ]
 
 
@@ -162,26 +177,32 @@ def test_tensor_core_kernel_matches_oracle(shape):
     aw, ww = oracle.bitpack_pm1(a), oracle.bitpack_pm1(w)
     acc = oracle.bconv2d_acc(a, w, (1, 1), lce.PAD_SAME_ONE)
     kw = dict(in_c=Cin, padding=lce.PAD_SAME_ONE)
-    got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_INT32), kernel_choice=lce.KERNEL_TENSOR)
+    got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_INT32), kernel_choice=lce.KERNEL_TENSOR, packed=True)
     np.testing.assert_array_equal(got, acc)
     thr = np.rint(np.sqrt(9 * Cin) * rng.standard_normal(Cout)).astype(np.int32)
-    got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_BITPACKED), thr=thr, kernel_choice=lce.KERNEL_TENSOR)
+    got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_BITPACKED), thr=thr, kernel_choice=lce.KERNEL_TENSOR, packed=True)
     np.testing.assert_array_equal(got, oracle.transform_bits(acc, thr))
     mult = rng.uniform(0.5, 1.5, Cout).astype(np.float32)
     bias = (0.1 * rng.standard_normal(Cout)).astype(np.float32)
     for act in (lce.ACT_NONE, lce.ACT_RELU):
         got = run_bconv(aw, ww, dict(kw, out_type=lce.OUT_FLOAT32, activation=act), mult=mult, bias=bias,
-                        kernel_choice=lce.KERNEL_TENSOR)
+                        kernel_choice=lce.KERNEL_TENSOR, packed=True)
         assert float_close(got, acc, mult, bias, act) == 0
     assert lce.lce_device_status() == 0  # no bounded wait gave up
 
 
 def test_tensor_core_kernel_rejects_what_it_does_not_cover():
-    desc = lce.make_desc(1, 8, 8, 64, 64, (3, 3), (2, 2), lce.PAD_SAME_ONE, lce.OUT_INT32, kernel_choice=lce.KERNEL_TENSOR)
     z = torch.zeros(8 * 8 * 2, dtype=torch.int32, device=DEV)
     w = torch.zeros(64 * 9 * 2, dtype=torch.int32, device=DEV)
+    # plain weights: the kernel needs the operand image made at load time
+    desc = lce.make_desc(1, 8, 8, 64, 64, (3, 3), (1, 1), lce.PAD_SAME_ONE, lce.OUT_INT32, kernel_choice=lce.KERNEL_TENSOR)
     with pytest.raises(lce.LceError) as e:
         lce.lce_bconv2d(desc, z, w)
+    assert e.value.status == 2
+    # stride 3
+    desc = lce.make_desc(1, 8, 8, 64, 64, (3, 3), (3, 3), lce.PAD_SAME_ONE, lce.OUT_INT32, lce.ACT_NONE, lce.KERNEL_TENSOR, 1)
+    with pytest.raises(lce.LceError) as e:
+        lce.lce_bconv2d(desc, z, lce.lce_bconv2d_pack_weights(desc, w))
     assert e.value.status == 2
 
 

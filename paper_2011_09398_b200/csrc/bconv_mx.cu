@@ -37,7 +37,8 @@
 //   * output transform (Section 3.2): a TMEM lane is a channel and a column a position.  Bit-packed
 //     output: the sign of (accumulator - threshold) of 32 positions per lane, then a 32 x 32 bit
 //     transpose across the warp gives each lane the finished word of one pixel.  Float / int32 output
-//     goes through a shared-memory stage [32 positions][128 channels] and leaves as whole pixel rows.
+//     is written straight from the registers: per position a warp stores its 32 consecutive channels as
+//     one 128-byte line.
 #include <atomic>
 #include <math.h>
 #include <mutex>
@@ -62,7 +63,6 @@ constexpr uint32_t kSfaCol = 480, kSfbCol = 496;             // block scales (al
 constexpr int kMaxTaps = 64;
 constexpr int kMaxStages = 32;
 constexpr int kPixSlots = 4;
-constexpr int kStageRows = 16, kStageCh = 128;               // float / int32 output stage of one column group
 
 // shared-memory map (bytes)
 constexpr int kOffBars = 0;          // full_x[2] full_d[2] empty_d[2] done full_w[32] empty_w[32]
@@ -71,7 +71,9 @@ constexpr int kOffThr = 1024;        // float[128]
 constexpr int kOffMult = 1536;       // float[128]
 constexpr int kOffBias = 2048;       // float[128]
 constexpr int kOffPix = 2816;        // int32[4][224]: output pixel of a column, or -1
-constexpr int kOffDyn = 6400;        // raw words, weight ring, position buffers, output stage
+constexpr int kOffTbl = 6400;        // uint2[256]: operand offsets (A, B; 16-byte units) of the MMAs of a tile
+constexpr int kOffDyn = 8448;        // raw words, weight ring, position buffers
+constexpr int kMaxTblMmas = 256;
 
 enum { BAR_FULL_X0 = 0, BAR_FULL_X1, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_DONE, BAR_FULL_W0,
        BAR_EMPTY_W0 = BAR_FULL_W0 + kMaxStages, BAR_COUNT = BAR_EMPTY_W0 + kMaxStages };
@@ -165,9 +167,9 @@ struct MxParams {
     int32_t n_tiles, total_q;
     int32_t taps, ksteps, stages, resident;
     int32_t tap_bytes, raw_words, x_bytes;
-    int32_t off_w, off_x, off_stage;   // byte offsets in shared memory
+    int32_t off_w, off_x;    // byte offsets in shared memory
     int32_t cp_words;        // words per cp.async: 4, 2 or 1
-    int32_t pad_zero, out_type, activation, vec_out, write_float;
+    int32_t pad_zero, out_type, activation, write_float;
 };
 
 // n / d for 0 <= n < 2^31 with (mul, sh) from the host: floor(n * mul / 2^sh), exact
@@ -270,6 +272,55 @@ __device__ __forceinline__ void mx_issue(uint32_t tmem_d, uint32_t a_lo, uint32_
     }
 }
 
+// MMAs 0 .. count - 1 of a tile straight from the table of operand offsets, eight per block of code: the
+// loads of a block are independent, and between two MMAs there is nothing but the next descriptor's
+// move.  For the tiles after a CTA's first one, when all weights are resident and nothing has to be
+// waited for between taps.
+__device__ __forceinline__ void mx_issue_table(uint32_t tmem_d, const uint2 *tbl, int count, uint32_t a_base, uint32_t b_base, uint32_t desc_hi,
+                                               uint32_t idesc, uint32_t sfa, uint32_t sfb)
+{
+    uint32_t accumulate = 0;
+    for (int i0 = 0; i0 < count; i0 += 8) {
+        uint32_t a[8], b[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint2 o = tbl[min(i0 + k, count - 1)];
+            a[k] = a_base + o.x;
+            b[k] = b_base + o.y;
+        }
+        const int n = count - i0;
+        if (elect_one()) {
+            asm volatile(
+                "{\n\t.reg .pred pa, pt, g;\n\t.reg .b64 da, db;\n\t"
+                "setp.ne.b32 pa, %21, 0;\n\t"
+                "setp.eq.b32 pt, 0, 0;\n\t"
+                "mov.b64 da, {%1, %17};\n\t mov.b64 db, {%9, %17};\n\t"
+                "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pa;\n\t"
+                "setp.gt.s32 g, %22, 1;\n\t mov.b64 da, {%2, %17};\n\t mov.b64 db, {%10, %17};\n\t"
+                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+                "setp.gt.s32 g, %22, 2;\n\t mov.b64 da, {%3, %17};\n\t mov.b64 db, {%11, %17};\n\t"
+                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+                "setp.gt.s32 g, %22, 3;\n\t mov.b64 da, {%4, %17};\n\t mov.b64 db, {%12, %17};\n\t"
+                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+                "setp.gt.s32 g, %22, 4;\n\t mov.b64 da, {%5, %17};\n\t mov.b64 db, {%13, %17};\n\t"
+                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+                "setp.gt.s32 g, %22, 5;\n\t mov.b64 da, {%6, %17};\n\t mov.b64 db, {%14, %17};\n\t"
+                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+                "setp.gt.s32 g, %22, 6;\n\t mov.b64 da, {%7, %17};\n\t mov.b64 db, {%15, %17};\n\t"
+                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+                "setp.gt.s32 g, %22, 7;\n\t mov.b64 da, {%8, %17};\n\t mov.b64 db, {%16, %17};\n\t"
+                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+                "}"
+                :
+                : "r"(tmem_d), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(a[4]), "r"(a[5]), "r"(a[6]), "r"(a[7]), "r"(b[0]), "r"(b[1]),
+                  "r"(b[2]), "r"(b[3]), "r"(b[4]), "r"(b[5]), "r"(b[6]), "r"(b[7]), "r"(desc_hi), "r"(idesc), "r"(sfa), "r"(sfb),
+                  "r"(accumulate), "r"(n)
+                : "memory");
+        }
+        accumulate = 1;
+    }
+}
+
 // a single MMA (one K step per tap: 33..64 input channels)
 __device__ __forceinline__ void mx_issue1(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t sfa,
                                           uint32_t sfb, uint32_t accumulate)
@@ -345,87 +396,58 @@ __device__ __forceinline__ void mx_epilogue_bits(const MxParams &p, uint32_t tme
         if (pix[k] >= 0) out[(int64_t)pix[k] * p.Cow + word] = words[k];
 }
 
-// Float / int32 output of one tile through the shared-memory stage (Section 3.2: int -> float, fused
-// activation, one multiply-add; Section 5.3: optional shortcut add and re-quantisation).  The four
-// warps of a column group (one per lane quarter) share a stage of 16 positions x 128 channels: each
-// writes its 32 channels of the chunk's positions, then each copies out four whole pixel rows.
-__device__ __forceinline__ void mx_epilogue_staged(const MxParams &p, uint32_t tmem_d, const int32_t *sPix, int ch0, uint32_t *stage_all,
-                                                   float mult, float bias, int fw, int lane, uint64_t *empty_d)
+// Float / int32 output of one tile (Section 3.2: int -> float, fused activation, one multiply-add;
+// Section 5.3: optional shortcut add and re-quantisation).  A lane holds one channel of 32 positions:
+// for every position the warp writes its 32 consecutive channels as one 128-byte store, so a value
+// costs one multiply-add and one store instruction and nothing is staged.  The re-quantised copy is a
+// warp ballot of the signs: the finished word of the pixel.
+__device__ __forceinline__ void mx_epilogue_values(const MxParams &p, uint32_t tmem_d, const int32_t *sPix, int ch0, float mult, float bias,
+                                                   int fw, int lane, uint64_t *empty_d)
 {
     const int quarter = fw & 3, group = fw >> 2;
-    const bool real = ch0 + quarter * 32 < p.Cout;
+    const int channel = ch0 + quarter * 32 + lane;
+    const bool real = ch0 + quarter * 32 < p.Cout;     // whole warp: any channel of its lanes exists
+    const bool ch_ok = channel < p.Cout;
     const uint32_t lane_addr = tmem_d + ((uint32_t)(quarter * 32) << 16);
-    uint32_t *stage = stage_all + group * (kStageRows * kStageCh);
     const bool relu = p.activation == LCE_ACT_RELU;
-    const int blk_ch = min(kStageCh, p.Cout - ch0);     // channels of this block that exist
-    const int my_ch = 4 * lane;                          // write-out: four consecutive channels of a pixel per lane
-    const bool act = my_ch < blk_ch;
-    const int n_chunks = p.Nt >> 4;                      // 16-column chunks; this group takes chunk group, group + 4, ...
-    if (group >= n_chunks) {  // a narrow tile leaves this column group without work
+    const int n_chunks = (p.Nt + 31) >> 5;               // this warp takes chunk group, group + 4
+    if (!real || group >= n_chunks) {  // nothing to read for this warp
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         mbar_arrive(empty_d);
         return;
     }
     const int last_chunk = group + ((n_chunks - 1 - group) / kColGroups) * kColGroups;
     for (int ck = group; ck < n_chunks; ck += kColGroups) {
-        const int c0 = ck * 16;
+        const int c0 = ck * 32;
+        const int cols = min(32, p.Nt - c0);
         float v[32];
-        if (real) tmem_ld16(lane_addr + (uint32_t)c0, v);
+        if (cols == 32) tmem_ld32(lane_addr + (uint32_t)c0, v);
+        else tmem_ld16(lane_addr + (uint32_t)c0, v);
         if (ck == last_chunk) {  // last read of the accumulator by this warp
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             mbar_arrive(empty_d);
         }
-        asm volatile("bar.sync %0, 128;" ::"r"(6 + group) : "memory");  // the stage is free again
-        if (real) {
-            uint32_t *col = stage + quarter * 32 + lane;
-            if (p.out_type == LCE_OUT_FLOAT32) {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) col[j * kStageCh] = __float_as_uint(__fmaf_rn(relu ? fmaxf(v[j], 0.f) : v[j], mult, bias));
-            } else {
+        for (int j4 = 0; j4 < 32; j4 += 4) {
+            if (j4 >= cols) break;
+            const int4 pix4 = *reinterpret_cast<const int4 *>(sPix + c0 + j4);  // the same for every lane
+            const int pix[4] = {pix4.x, pix4.y, pix4.z, pix4.w};
 #pragma unroll
-                for (int j = 0; j < 16; ++j) col[j * kStageCh] = (uint32_t)__float2int_rn(v[j]);
-            }
-        }
-        asm volatile("bar.sync %0, 128;" ::"r"(2 + group) : "memory");  // the stage holds the chunk
-        // rows out: warp `quarter` takes positions quarter, quarter + 4, quarter + 8, quarter + 12
-        int pix[4];
-        uint4 q[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int j = quarter + 4 * u;
-            pix[u] = sPix[c0 + j];  // the same for every lane
-            q[u] = make_uint4(0u, 0u, 0u, 0u);
-            if (act && pix[u] >= 0 && p.vec_out) q[u] = *reinterpret_cast<const uint4 *>(stage + j * kStageCh + my_ch);
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            if (pix[u] < 0) continue;
-            const int j = quarter + 4 * u;
-            const int64_t o = (int64_t)pix[u] * p.Cout + ch0 + my_ch;
-            if (p.vec_out) {
-                if (act) {
-                    if (p.residual) {
-                        const float4 r = __ldg(reinterpret_cast<const float4 *>(p.residual + o));
-                        q[u].x = __float_as_uint(__fadd_rn(__uint_as_float(q[u].x), r.x));
-                        q[u].y = __float_as_uint(__fadd_rn(__uint_as_float(q[u].y), r.y));
-                        q[u].z = __float_as_uint(__fadd_rn(__uint_as_float(q[u].z), r.z));
-                        q[u].w = __float_as_uint(__fadd_rn(__uint_as_float(q[u].w), r.w));
+            for (int u = 0; u < 4; ++u) {
+                if (pix[u] < 0) continue;
+                const float a = v[j4 + u];
+                const int64_t o = (int64_t)pix[u] * p.Cout + channel;
+                if (p.out_type == LCE_OUT_FLOAT32) {
+                    float y = __fmaf_rn(relu ? fmaxf(a, 0.f) : a, mult, bias);
+                    if (p.residual && ch_ok) y = __fadd_rn(y, __ldg(p.residual + o));
+                    if (p.write_float && ch_ok) static_cast<float *>(p.out)[o] = y;
+                    if (p.out_packed) {
+                        const uint32_t word = __ballot_sync(0xffffffffu, ch_ok && y < 0.f);
+                        if (lane == 0) p.out_packed[(int64_t)pix[u] * p.Cow + (ch0 >> 5) + quarter] = word;
                     }
-                    if (p.write_float) *reinterpret_cast<uint4 *>(static_cast<uint32_t *>(p.out) + o) = q[u];
+                } else if (ch_ok) {
+                    static_cast<int32_t *>(p.out)[o] = __float2int_rn(a);
                 }
-                if (p.out_packed) {
-                    // sign bits of this lane's four channels, gathered over the eight lanes of a 32-channel word
-                    uint32_t nib = (__uint_as_float(q[u].x) < 0.f ? 1u : 0u) | (__uint_as_float(q[u].y) < 0.f ? 2u : 0u) |
-                                   (__uint_as_float(q[u].z) < 0.f ? 4u : 0u) | (__uint_as_float(q[u].w) < 0.f ? 8u : 0u);
-                    nib <<= 4 * (lane & 7);
-                    nib |= __shfl_xor_sync(0xffffffffu, nib, 1);
-                    nib |= __shfl_xor_sync(0xffffffffu, nib, 2);
-                    nib |= __shfl_xor_sync(0xffffffffu, nib, 4);
-                    if ((lane & 7) == 0 && act) p.out_packed[(int64_t)pix[u] * p.Cow + ((ch0 + my_ch) >> 5)] = nib;
-                }
-            } else if (act) {
-                const uint32_t *srow = stage + j * kStageCh + my_ch;
-                for (int e = 0; e < 4 && my_ch + e < blk_ch; ++e) static_cast<uint32_t *>(p.out)[o + e] = srow[e];
             }
         }
     }
@@ -441,10 +463,10 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
     float *sMult = reinterpret_cast<float *>(smem + kOffMult);
     float *sBias = reinterpret_cast<float *>(smem + kOffBias);
     int32_t *sPix = reinterpret_cast<int32_t *>(smem + kOffPix);
+    uint2 *tbl = reinterpret_cast<uint2 *>(smem + kOffTbl);
     uint32_t *raw0 = reinterpret_cast<uint32_t *>(smem + kOffDyn);
     uint8_t *sW = smem + p.off_w;
     uint8_t *sX0 = smem + p.off_x;
-    uint32_t *stage = reinterpret_cast<uint32_t *>(smem + p.off_stage);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int ch0 = blockIdx.y * 128;
@@ -462,6 +484,18 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         sThr[e] = t;
         sMult[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.mult + ch0 + e) : 0.f;
         sBias[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.bias + ch0 + e) : 0.f;
+    }
+    const int n_mma = p.taps * p.ksteps;
+    const bool use_table = p.resident && n_mma <= kMaxTblMmas;
+    for (int e = tid; use_table && e < n_mma; e += kMxThreads) {
+        const int tap = e / p.ksteps, kk = e - tap * p.ksteps;
+        const int ky = tap / p.KW, kx = tap - ky * p.KW;
+        // A: the tap's ring stage (all taps resident: stage = tap) + K step; B: phase buffer (stride 2) shifted
+        // by the tap's position offset + K step
+        uint32_t b_off;
+        if (p.stride == 2) b_off = (uint32_t)((((ky & 1) * 2 + (kx & 1)) * p.Cw2) * p.P + (ky >> 1) * p.Wg + (kx >> 1));
+        else b_off = (uint32_t)(ky * p.Wg + kx);
+        tbl[e] = make_uint2((uint32_t)tap * ((uint32_t)p.tap_bytes >> 4) + 256u * kk, b_off + 2u * (uint32_t)p.P * kk);
     }
     if (tid == 0) {
         mbar_init(&bars[BAR_FULL_X0], kLoaders);
@@ -539,14 +573,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             const int buf = it & 1;
             ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + buf], par_full_d[buf]);
             par_full_d[buf] ^= 1u;
-            {   // the staged form synchronises the finisher warps among themselves: go on only if all of them got through
-                uint32_t all_ok;
-                asm volatile("{\n\t.reg .pred q, r;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred r, 1, %2, q;\n\tselp.u32 %0, 1, 0, r;\n\t}"
-                             : "=r"(all_ok)
-                             : "r"((uint32_t)ok), "n"(kFinishers)
-                             : "memory");
-                ok = all_ok != 0;
-            }
+            ok = __all_sync(0xffffffffu, ok);  // the warp goes on together (its epilogue uses warp-wide shuffles and ballots)
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
@@ -554,7 +581,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             if (p.out_type == LCE_OUT_BITPACKED)
                 mx_epilogue_bits(p, tmem_d, pix, ch0, sThr, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
             else
-                mx_epilogue_staged(p, tmem_d, pix, ch0, stage, my_mult, my_bias, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
+                mx_epilogue_values(p, tmem_d, pix, ch0, my_mult, my_bias, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
         }
     } else if (warp == kIssuerWarp) {
         // ======================= MMA issuer: one warp, every lane with the same values ================
@@ -583,6 +610,11 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
             const uint32_t x_lo0 = ((uint32_t)p.off_x >> 4) + (smem_u32(smem) >> 4) + (uint32_t)buf * ((uint32_t)p.x_bytes >> 4) + ((uint32_t)p.P << 16);
+            if (use_table && it > 0) {
+                mx_issue_table(tmem_d, tbl, n_mma, w_lo0, x_lo0, desc_hi, idesc, sfa, sfb);
+                if (elect_one()) mma_commit(&bars[BAR_FULL_D0 + buf]);
+                continue;
+            }
             uint32_t accumulate = 0;
             for (int ky = 0; ky < p.KH && ok; ++ky) {
                 for (int kx = 0; kx < p.KW; ++kx) {
@@ -686,7 +718,7 @@ __global__ void mx_pack_weights_kernel(const uint32_t *w, uint4 *image, int Cout
 
 struct MxPlan {
     int Nt, P, stages, resident, n_blocks, ctas_x, n_tiles, total_q, Wg, Hg, n_phase, Cw2, taps, halo;
-    size_t raw_words, x_bytes, tap_bytes, off_w, off_x, off_stage, smem;
+    size_t raw_words, x_bytes, tap_bytes, off_w, off_x, smem;
 };
 
 constexpr size_t kSmemLimit = 227 * 1024;
@@ -718,8 +750,6 @@ bool mx_plan(const ConvGeom &g, int sms, MxPlan *pl)
     pl->tap_bytes = (size_t)pl->Cw2 * 2048;
     pl->n_blocks = (g.Cout + 127) / 128;
     const int ctas_max = max(1, sms / pl->n_blocks);
-    const bool staged = g.out_type != LCE_OUT_BITPACKED;
-    const size_t stage_bytes = staged ? (size_t)kColGroups * kStageRows * kStageCh * 4 : 0;
     const int ksteps = pl->Cw2 / 2;
     double best = 1e30;
     bool found = false;
@@ -730,7 +760,7 @@ bool mx_plan(const ConvGeom &g, int sms, MxPlan *pl)
         const size_t x_bytes = (size_t)pl->n_phase * pl->Cw2 * P * 16;
         const size_t fixed = kOffDyn + 2 * raw_words * 4;
         const size_t off_w = (fixed + 127) / 128 * 128;
-        const size_t rest = 2 * x_bytes + stage_bytes + 256;
+        const size_t rest = 2 * x_bytes + 256;
         if (off_w + rest + 2 * pl->tap_bytes > kSmemLimit) continue;
         int stages = (int)((kSmemLimit - off_w - rest) / pl->tap_bytes);
         if (stages > kMaxStages) stages = kMaxStages;
@@ -751,8 +781,7 @@ bool mx_plan(const ConvGeom &g, int sms, MxPlan *pl)
             pl->raw_words = raw_words; pl->x_bytes = x_bytes;
             pl->off_w = off_w;
             pl->off_x = (off_w + (size_t)stages * pl->tap_bytes + 127) / 128 * 128;
-            pl->off_stage = pl->off_x + 2 * x_bytes;
-            pl->smem = pl->off_stage + stage_bytes;
+            pl->smem = pl->off_x + 2 * x_bytes;
         }
     }
     return found;
@@ -833,13 +862,11 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const void
     p.Nt = pl.Nt; p.P = pl.P; p.n_tiles = pl.n_tiles; p.total_q = pl.total_q;
     p.taps = pl.taps; p.ksteps = pl.Cw2 / 2; p.stages = pl.stages; p.resident = pl.resident;
     p.tap_bytes = (int32_t)pl.tap_bytes; p.raw_words = (int32_t)pl.raw_words; p.x_bytes = (int32_t)pl.x_bytes;
-    p.off_w = (int32_t)pl.off_w; p.off_x = (int32_t)pl.off_x; p.off_stage = (int32_t)pl.off_stage;
+    p.off_w = (int32_t)pl.off_w; p.off_x = (int32_t)pl.off_x;
     p.cp_words = (g.Cw % 4 == 0 && aligned(in, 16)) ? 4 : (g.Cw % 2 == 0 && aligned(in, 8)) ? 2 : 1;
     p.pad_zero = g.padding == LCE_PAD_SAME_ZERO;
     p.out_type = g.out_type; p.activation = g.activation;
     p.write_float = out != nullptr;
-    p.vec_out = (g.Cout % 4 == 0) && aligned(out, 16) && aligned(residual, 16);
-    if ((residual || out_packed) && (!p.vec_out || g.Cout % 32 != 0)) return LCE_ERR_UNSUPPORTED;
     if (!aligned(w_image, 16)) return LCE_ERR_ALIGNMENT;
     static SmemOptIn opted;
     if (!opted.ensure(bconv_mx_kernel, pl.smem)) return LCE_ERR_CUDA;

@@ -71,9 +71,9 @@ constexpr int kOffThr = 1024;        // float[128]
 constexpr int kOffMult = 1536;       // float[128]
 constexpr int kOffBias = 2048;       // float[128]
 constexpr int kOffPix = 2816;        // int32[4][224]: output pixel of a column, or -1
-constexpr int kOffTbl = 6400;        // uint2[256]: operand offsets (A, B; 16-byte units) of the MMAs of a tile
-constexpr int kOffDyn = 8448;        // raw words, weight ring, position buffers
-constexpr int kMaxTblMmas = 256;
+constexpr int kOffTbl = 6400;        // uint2[512]: operand offsets (A, B; 16-byte units) of the MMAs of a tile
+constexpr int kOffDyn = 10496;       // raw words, weight ring, position buffers
+constexpr int kMaxTblMmas = 512;
 
 enum { BAR_FULL_X0 = 0, BAR_FULL_X1, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_DONE, BAR_FULL_W0,
        BAR_EMPTY_W0 = BAR_FULL_W0 + kMaxStages, BAR_COUNT = BAR_EMPTY_W0 + kMaxStages };
@@ -175,8 +175,16 @@ struct MxParams {
 // n / d for 0 <= n < 2^31 with (mul, sh) from the host: floor(n * mul / 2^sh), exact
 __device__ __forceinline__ int fast_div(int n, uint32_t mul, uint32_t sh) { return (int)(((uint64_t)(uint32_t)n * mul) >> sh); }
 
+// what the loaders need of the geometry, in registers (kernel parameters read inside their loops cost
+// more than the arithmetic)
+struct MxGeo {
+    int N, H, W, Cw, Cw2, Wg, Hg, P, items, stride, pt, pl, pad_zero, cp_words;
+    uint32_t Wg_mul, Wg_sh, Hg_mul, Hg_sh, P_mul, P_sh;
+    const uint32_t *in;
+};
+
 // position j of the tile that starts at q0, phase ph -> inside the image? and the pixel's word offset
-__device__ __forceinline__ bool mx_locate(const MxParams &p, int q0, int ph, int j, int64_t *word_offset)
+__device__ __forceinline__ bool mx_locate(const MxGeo &p, int q0, int ph, int j, int64_t *word_offset)
 {
     const int f = q0 + j;
     const int r = fast_div(f, p.Wg_mul, p.Wg_sh), c = f - r * p.Wg;
@@ -189,10 +197,9 @@ __device__ __forceinline__ bool mx_locate(const MxParams &p, int q0, int ph, int
 }
 
 // packed words of the tile's positions -> raw[item][Cw] (pad positions: zero words), asynchronously
-__device__ __forceinline__ void mx_prefetch(const MxParams &p, int q0, uint32_t *raw, int ltid)
+__device__ __forceinline__ void mx_prefetch(const MxGeo &p, int q0, uint32_t *raw, int ltid)
 {
-    const int items = p.n_phase * p.P;
-    for (int i = ltid; i < items; i += kLoaders) {
+    for (int i = ltid; i < p.items; i += kLoaders) {
         const int ph = fast_div(i, p.P_mul, p.P_sh), j = i - ph * p.P;
         int64_t off;
         const bool ok = mx_locate(p, q0, ph, j, &off);
@@ -210,11 +217,10 @@ __device__ __forceinline__ void mx_prefetch(const MxParams &p, int q0, uint32_t 
 }
 
 // every thread expands the words it prefetched itself (same item mapping): waiting for its own copies is enough
-__device__ __forceinline__ void mx_expand(const MxParams &p, int q0, const uint32_t *raw, uint8_t *X, int ltid)
+__device__ __forceinline__ void mx_expand(const MxGeo &p, int q0, const uint32_t *raw, uint8_t *X, int ltid)
 {
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    const int items = p.n_phase * p.P;
-    for (int i = ltid; i < items; i += kLoaders) {
+    for (int i = ltid; i < p.items; i += kLoaders) {
         const int ph = fast_div(i, p.P_mul, p.P_sh), j = i - ph * p.P;
         bool zero = false;
         if (p.pad_zero) {
@@ -239,10 +245,9 @@ __device__ __forceinline__ bool elect_one()
     return pred != 0;
 }
 
-// `count` MMAs of one tap, up to four per block of code.  The whole issuer warp runs this with the same
-// values in every lane, so that the descriptors stay in uniform registers (a single diverged thread
-// pays a register-to-uniform move per operand and MMA, about 200 clocks per instruction, measured);
-// only the elected lane issues.  Descriptor low words advance by additions, the high word never changes.
+// `count` MMAs of one tap by descriptor arithmetic, up to four per block of code (filters with more MMAs
+// per tile than the offset table holds).  Descriptor low words advance by additions, the high word
+// never changes.
 __device__ __forceinline__ void mx_issue(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t a_step, uint32_t b_step, int count,
                                          uint32_t desc_hi, uint32_t idesc, uint32_t sfa, uint32_t sfb, uint32_t &accumulate)
 {
@@ -272,14 +277,14 @@ __device__ __forceinline__ void mx_issue(uint32_t tmem_d, uint32_t a_lo, uint32_
     }
 }
 
-// MMAs 0 .. count - 1 of a tile straight from the table of operand offsets, eight per block of code: the
-// loads of a block are independent, and between two MMAs there is nothing but the next descriptor's
-// move.  For the tiles after a CTA's first one, when all weights are resident and nothing has to be
-// waited for between taps.
+// `count` MMAs straight from a table of operand offsets, eight per block of code: the loads of a block
+// are independent, and between two MMAs there is nothing but the next descriptor's move.  The whole
+// issuer warp runs this with the same values in every lane, so that the descriptors stay in uniform
+// registers (a single diverged thread pays a register-to-uniform move per operand and MMA: about 200
+// clocks per instruction, measured); only the elected lane issues.
 __device__ __forceinline__ void mx_issue_table(uint32_t tmem_d, const uint2 *tbl, int count, uint32_t a_base, uint32_t b_base, uint32_t desc_hi,
-                                               uint32_t idesc, uint32_t sfa, uint32_t sfb)
+                                               uint32_t idesc, uint32_t sfa, uint32_t sfb, uint32_t &accumulate)
 {
-    uint32_t accumulate = 0;
     for (int i0 = 0; i0 < count; i0 += 8) {
         uint32_t a[8], b[8];
 #pragma unroll
@@ -321,23 +326,6 @@ __device__ __forceinline__ void mx_issue_table(uint32_t tmem_d, const uint2 *tbl
     }
 }
 
-// a single MMA (one K step per tap: 33..64 input channels)
-__device__ __forceinline__ void mx_issue1(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t sfa,
-                                          uint32_t sfb, uint32_t accumulate)
-{
-    if (elect_one()) {
-        asm volatile(
-            "{\n\t.reg .pred pa;\n\t.reg .b64 da, db;\n\t"
-            "setp.ne.b32 pa, %7, 0;\n\t"
-            "mov.b64 da, {%1, %3};\n\t mov.b64 db, {%2, %3};\n\t"
-            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %4, [%5], [%6], pa;\n\t"
-            "}"
-            :
-            : "r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(sfa), "r"(sfb), "r"(accumulate)
-            : "memory");
-    }
-}
-
 // 32 x 32 bit transpose across the warp: in: lane = row, bit j = column j; out: lane j holds column j
 __device__ __forceinline__ uint32_t warp_transpose32(uint32_t m, int lane)
 {
@@ -356,19 +344,21 @@ __device__ __forceinline__ void mx_epilogue_bits(const MxParams &p, uint32_t tme
                                                  int fw, int lane, uint64_t *empty_d)
 {
     const int quarter = fw & 3, group = fw >> 2;
+    const int Nt = p.Nt;
     const bool real = ch0 + quarter * 32 < p.Cout;     // whole warp: any channel of its lanes exists
     const float thr = sThr[quarter * 32 + lane];       // -inf for channels that do not exist: bit 0
     const uint32_t lane_addr = tmem_d + ((uint32_t)(quarter * 32) << 16);
-    uint32_t *out = static_cast<uint32_t *>(p.out);
+    uint32_t *out = static_cast<uint32_t *>(p.out) + (ch0 >> 5) + quarter;
+    const int64_t cow = p.Cow;
     uint32_t words[2] = {0u, 0u};
     int pix[2] = {-1, -1};
     if (real) {
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
             const int c0 = (group + k * kColGroups) * 32;
-            if (c0 >= p.Nt) break;
+            if (c0 >= Nt) break;
             float v[32];
-            const bool full = c0 + 32 <= p.Nt;
+            const bool full = c0 + 32 <= Nt;
             if (full) tmem_ld32(lane_addr + (uint32_t)c0, v);
             else tmem_ld16(lane_addr + (uint32_t)c0, v);
             // bit j = (acc_j < thr): the sign of acc - thr (both are small integers held exactly);
@@ -384,33 +374,73 @@ __device__ __forceinline__ void mx_epilogue_bits(const MxParams &p, uint32_t tme
             uint32_t m = m0 | (m1 << 8);
             if (full) m |= (m2 << 16) | (m3 << 24);
             words[k] = warp_transpose32(m, lane);
-            pix[k] = (c0 + lane < p.Nt) ? sPix[c0 + lane] : -1;
+            pix[k] = (c0 + lane < Nt) ? sPix[c0 + lane] : -1;
         }
     }
     // the accumulator buffer has been read: hand it back before the stores
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     mbar_arrive(empty_d);
-    const int word = (ch0 >> 5) + quarter;
 #pragma unroll
     for (int k = 0; k < 2; ++k)
-        if (pix[k] >= 0) out[(int64_t)pix[k] * p.Cow + word] = words[k];
+        if (pix[k] >= 0) out[pix[k] * cow] = words[k];
 }
 
 // Float / int32 output of one tile (Section 3.2: int -> float, fused activation, one multiply-add;
 // Section 5.3: optional shortcut add and re-quantisation).  A lane holds one channel of 32 positions:
 // for every position the warp writes its 32 consecutive channels as one 128-byte store, so a value
 // costs one multiply-add and one store instruction and nothing is staged.  The re-quantised copy is a
-// warp ballot of the signs: the finished word of the pixel.
+// warp ballot of the signs: the finished word of the pixel.  Everything the loops need sits in
+// registers before they start (kernel parameters read inside them cost more than the arithmetic).
+enum { EPI_FLOAT = 0, EPI_FLOAT_FUSED = 1, EPI_INT32 = 2, EPI_BITS = 3 };
+
+template <int MODE>
+__device__ __forceinline__ void mx_store_chunk(const float (&v)[32], int cols, const int32_t *sPixChunk, int64_t cout, float *outp,
+                                               const float *resp, uint32_t *packp, int64_t cow, bool ch_ok, bool relu, bool write_float,
+                                               float mult, float bias, int lane)
+{
+#pragma unroll
+    for (int j4 = 0; j4 < 32; j4 += 4) {
+        if (j4 >= cols) break;
+        const int4 pix4 = *reinterpret_cast<const int4 *>(sPixChunk + j4);  // the same for every lane
+        const int pix[4] = {pix4.x, pix4.y, pix4.z, pix4.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (pix[u] < 0) continue;
+            const float a = v[j4 + u];
+            const int64_t o = pix[u] * cout;
+            if (MODE == EPI_FLOAT) {
+                if (ch_ok) outp[o] = __fmaf_rn(a, mult, bias);
+            } else if (MODE == EPI_INT32) {
+                if (ch_ok) reinterpret_cast<int32_t *>(outp)[o] = __float2int_rn(a);
+            } else {
+                float y = __fmaf_rn(relu ? fmaxf(a, 0.f) : a, mult, bias);
+                if (resp && ch_ok) y = __fadd_rn(y, __ldg(resp + o));
+                if (write_float && ch_ok) outp[o] = y;
+                if (packp) {
+                    const uint32_t word = __ballot_sync(0xffffffffu, ch_ok && y < 0.f);
+                    if (lane == 0) packp[pix[u] * cow] = word;
+                }
+            }
+        }
+    }
+}
+
+template <int MODE>
 __device__ __forceinline__ void mx_epilogue_values(const MxParams &p, uint32_t tmem_d, const int32_t *sPix, int ch0, float mult, float bias,
                                                    int fw, int lane, uint64_t *empty_d)
 {
     const int quarter = fw & 3, group = fw >> 2;
     const int channel = ch0 + quarter * 32 + lane;
+    const int Nt = p.Nt;
+    const int64_t cout = p.Cout, cow = p.Cow;
     const bool real = ch0 + quarter * 32 < p.Cout;     // whole warp: any channel of its lanes exists
     const bool ch_ok = channel < p.Cout;
+    const bool relu = p.activation == LCE_ACT_RELU, write_float = p.write_float != 0;
+    float *outp = static_cast<float *>(p.out) + channel;
+    const float *resp = p.residual ? p.residual + channel : nullptr;
+    uint32_t *packp = p.out_packed ? p.out_packed + (ch0 >> 5) + quarter : nullptr;
     const uint32_t lane_addr = tmem_d + ((uint32_t)(quarter * 32) << 16);
-    const bool relu = p.activation == LCE_ACT_RELU;
-    const int n_chunks = (p.Nt + 31) >> 5;               // this warp takes chunk group, group + 4
+    const int n_chunks = (Nt + 31) >> 5;               // this warp takes chunk group, group + 4
     if (!real || group >= n_chunks) {  // nothing to read for this warp
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         mbar_arrive(empty_d);
@@ -419,7 +449,7 @@ __device__ __forceinline__ void mx_epilogue_values(const MxParams &p, uint32_t t
     const int last_chunk = group + ((n_chunks - 1 - group) / kColGroups) * kColGroups;
     for (int ck = group; ck < n_chunks; ck += kColGroups) {
         const int c0 = ck * 32;
-        const int cols = min(32, p.Nt - c0);
+        const int cols = min(32, Nt - c0);
         float v[32];
         if (cols == 32) tmem_ld32(lane_addr + (uint32_t)c0, v);
         else tmem_ld16(lane_addr + (uint32_t)c0, v);
@@ -427,32 +457,13 @@ __device__ __forceinline__ void mx_epilogue_values(const MxParams &p, uint32_t t
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             mbar_arrive(empty_d);
         }
-#pragma unroll
-        for (int j4 = 0; j4 < 32; j4 += 4) {
-            if (j4 >= cols) break;
-            const int4 pix4 = *reinterpret_cast<const int4 *>(sPix + c0 + j4);  // the same for every lane
-            const int pix[4] = {pix4.x, pix4.y, pix4.z, pix4.w};
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (pix[u] < 0) continue;
-                const float a = v[j4 + u];
-                const int64_t o = (int64_t)pix[u] * p.Cout + channel;
-                if (p.out_type == LCE_OUT_FLOAT32) {
-                    float y = __fmaf_rn(relu ? fmaxf(a, 0.f) : a, mult, bias);
-                    if (p.residual && ch_ok) y = __fadd_rn(y, __ldg(p.residual + o));
-                    if (p.write_float && ch_ok) static_cast<float *>(p.out)[o] = y;
-                    if (p.out_packed) {
-                        const uint32_t word = __ballot_sync(0xffffffffu, ch_ok && y < 0.f);
-                        if (lane == 0) p.out_packed[(int64_t)pix[u] * p.Cow + (ch0 >> 5) + quarter] = word;
-                    }
-                } else if (ch_ok) {
-                    static_cast<int32_t *>(p.out)[o] = __float2int_rn(a);
-                }
-            }
-        }
+        mx_store_chunk<MODE>(v, cols, sPix + c0, cout, outp, resp, packp, cow, ch_ok, relu, write_float, mult, bias, lane);
     }
 }
 
+// EPI: the output transform this instantiation carries (one kernel per form keeps each one's code, and
+// with it the instruction-cache footprint of four roles running side by side, small)
+template <int EPI>
 __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_constant__ MxParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -486,16 +497,16 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         sBias[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.bias + ch0 + e) : 0.f;
     }
     const int n_mma = p.taps * p.ksteps;
-    const bool use_table = p.resident && n_mma <= kMaxTblMmas;
+    const bool use_table = n_mma <= kMaxTblMmas;
     for (int e = tid; use_table && e < n_mma; e += kMxThreads) {
         const int tap = e / p.ksteps, kk = e - tap * p.ksteps;
         const int ky = tap / p.KW, kx = tap - ky * p.KW;
-        // A: the tap's ring stage (all taps resident: stage = tap) + K step; B: phase buffer (stride 2) shifted
-        // by the tap's position offset + K step
+        // A: K step (+ the tap's ring stage when all taps are resident: stage = tap); B: phase buffer (stride
+        // 2) shifted by the tap's position offset + K step
         uint32_t b_off;
         if (p.stride == 2) b_off = (uint32_t)((((ky & 1) * 2 + (kx & 1)) * p.Cw2) * p.P + (ky >> 1) * p.Wg + (kx >> 1));
         else b_off = (uint32_t)(ky * p.Wg + kx);
-        tbl[e] = make_uint2((uint32_t)tap * ((uint32_t)p.tap_bytes >> 4) + 256u * kk, b_off + 2u * (uint32_t)p.P * kk);
+        tbl[e] = make_uint2((p.resident ? (uint32_t)tap * ((uint32_t)p.tap_bytes >> 4) : 0u) + 256u * kk, b_off + 2u * (uint32_t)p.P * kk);
     }
     if (tid == 0) {
         mbar_init(&bars[BAR_FULL_X0], kLoaders);
@@ -537,29 +548,36 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
     bool ok = true;
     if (tid < kLoaders) {
         // ======================= loaders ==============================================================
+        MxGeo geo;
+        geo.N = p.N; geo.H = p.H; geo.W = p.W; geo.Cw = p.Cw; geo.Cw2 = p.Cw2; geo.Wg = p.Wg; geo.Hg = p.Hg; geo.P = p.P;
+        geo.items = p.n_phase * p.P; geo.stride = p.stride; geo.pt = p.pt; geo.pl = p.pl; geo.pad_zero = p.pad_zero; geo.cp_words = p.cp_words;
+        geo.Wg_mul = p.Wg_mul; geo.Wg_sh = p.Wg_sh; geo.Hg_mul = p.Hg_mul; geo.Hg_sh = p.Hg_sh; geo.P_mul = p.P_mul; geo.P_sh = p.P_sh;
+        geo.in = p.in;
+        const int Nt = p.Nt, n_tiles = p.n_tiles, OH = p.OH, OW = p.OW, raw_words = p.raw_words;
+        const size_t x_bytes = (size_t)p.x_bytes;
         uint32_t par_full_d[2] = {0, 0};
         int tile = first_tile;
-        if (tile < p.n_tiles) mx_prefetch(p, tile * p.Nt, raw0, tid);
-        for (int it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
+        if (tile < n_tiles) mx_prefetch(geo, tile * Nt, raw0, tid);
+        for (int it = 0; tile < n_tiles && ok; tile += tile_step, ++it) {
             const int buf = it & 1;
             if (it >= 2) {  // position buffer `buf` was read by the MMAs of tile it-2
                 ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + buf], par_full_d[buf]);
                 par_full_d[buf] ^= 1u;
                 if (!ok) break;
             }
-            mx_expand(p, tile * p.Nt, raw0 + buf * p.raw_words, sX0 + (size_t)buf * p.x_bytes, tid);
-            if (tid < p.Nt) {
-                const int f = tile * p.Nt + tid;
-                const int r = fast_div(f, p.Wg_mul, p.Wg_sh), c = f - r * p.Wg;
-                const int n = fast_div(r, p.Hg_mul, p.Hg_sh), rr = r - n * p.Hg;
-                const bool col_ok = n < p.N && rr < p.OH && c < p.OW;
-                sPix[(it & (kPixSlots - 1)) * kMaxNt + tid] = col_ok ? (n * p.OH + rr) * p.OW + c : -1;
+            mx_expand(geo, tile * Nt, raw0 + buf * raw_words, sX0 + buf * x_bytes, tid);
+            if (tid < Nt) {
+                const int f = tile * Nt + tid;
+                const int r = fast_div(f, geo.Wg_mul, geo.Wg_sh), c = f - r * geo.Wg;
+                const int n = fast_div(r, geo.Hg_mul, geo.Hg_sh), rr = r - n * geo.Hg;
+                const bool col_ok = n < geo.N && rr < OH && c < OW;
+                sPix[(it & (kPixSlots - 1)) * kMaxNt + tid] = col_ok ? (n * OH + rr) * OW + c : -1;
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_arrive(&bars[BAR_FULL_X0 + buf]);
             // only now the words of the next tile: the MMAs of this tile must not wait for loads they do not need
             const int next = tile + tile_step;
-            if (next < p.n_tiles) mx_prefetch(p, next * p.Nt, raw0 + (buf ^ 1) * p.raw_words, tid);
+            if (next < n_tiles) mx_prefetch(geo, next * Nt, raw0 + (buf ^ 1) * raw_words, tid);
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else if (tid < kLoaders + kFinishers) {
@@ -578,10 +596,10 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
             const int32_t *pix = sPix + (it & (kPixSlots - 1)) * kMaxNt;
-            if (p.out_type == LCE_OUT_BITPACKED)
+            if (EPI == EPI_BITS)
                 mx_epilogue_bits(p, tmem_d, pix, ch0, sThr, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
             else
-                mx_epilogue_values(p, tmem_d, pix, ch0, my_mult, my_bias, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
+                mx_epilogue_values<EPI>(p, tmem_d, pix, ch0, my_mult, my_bias, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
         }
     } else if (warp == kIssuerWarp) {
         // ======================= MMA issuer: one warp, every lane with the same values ================
@@ -610,34 +628,35 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
             const uint32_t x_lo0 = ((uint32_t)p.off_x >> 4) + (smem_u32(smem) >> 4) + (uint32_t)buf * ((uint32_t)p.x_bytes >> 4) + ((uint32_t)p.P << 16);
-            if (use_table && it > 0) {
-                mx_issue_table(tmem_d, tbl, n_mma, w_lo0, x_lo0, desc_hi, idesc, sfa, sfb);
-                if (elect_one()) mma_commit(&bars[BAR_FULL_D0 + buf]);
-                continue;
-            }
             uint32_t accumulate = 0;
-            for (int ky = 0; ky < p.KH && ok; ++ky) {
-                for (int kx = 0; kx < p.KW; ++kx) {
-                    if (!p.resident || it == 0) {
-                        ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_FULL_W0 + stage_i], w_parity));
-                        if (!ok) break;
-                        ++g;
-                        if (lane == 0) fills[1] = g;
-                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (use_table && p.resident && it > 0) {
+                // every tap is in shared memory: nothing to wait for between the MMAs of the tile
+                mx_issue_table(tmem_d, tbl, n_mma, w_lo0, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
+            } else {
+                int tap = 0;
+                for (int ky = 0; ky < p.KH && ok; ++ky) {
+                    for (int kx = 0; kx < p.KW; ++kx, ++tap) {
+                        if (!p.resident || it == 0) {
+                            ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_FULL_W0 + stage_i], w_parity));
+                            if (!ok) break;
+                            ++g;
+                            if (lane == 0) fills[1] = g;
+                            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        }
+                        const uint32_t a_stage = w_lo0 + (uint32_t)stage_i * tap_units;
+                        if (use_table && p.ksteps <= 2) {
+                            mx_issue_table(tmem_d, tbl + tap * p.ksteps, p.ksteps, p.resident ? w_lo0 : a_stage, x_lo0, desc_hi, idesc, sfa, sfb,
+                                           accumulate);
+                        } else {
+                            // B operand of the tap: its phase buffer (stride 2) shifted by the tap's position offset
+                            uint32_t b_off;
+                            if (p.stride == 2) b_off = (uint32_t)((((ky & 1) * 2 + (kx & 1)) * p.Cw2) * p.P + (ky >> 1) * p.Wg + (kx >> 1));
+                            else b_off = (uint32_t)(ky * p.Wg + kx);
+                            mx_issue(tmem_d, a_stage, x_lo0 + b_off, 256u, 2u * (uint32_t)p.P, p.ksteps, desc_hi, idesc, sfa, sfb, accumulate);
+                        }
+                        if (!p.resident && elect_one()) mma_commit(&bars[BAR_EMPTY_W0 + stage_i]);
+                        if (++stage_i == p.stages) { stage_i = 0; w_parity ^= 1u; }
                     }
-                    // B operand of the tap: its phase buffer (stride 2) shifted by the tap's position offset
-                    uint32_t b_off;
-                    if (p.stride == 2) b_off = (uint32_t)((((ky & 1) * 2 + (kx & 1)) * p.Cw2) * p.P + (ky >> 1) * p.Wg + (kx >> 1));
-                    else b_off = (uint32_t)(ky * p.Wg + kx);
-                    const uint32_t a_lo = w_lo0 + (uint32_t)stage_i * tap_units;
-                    if (p.ksteps == 1) {
-                        mx_issue1(tmem_d, a_lo, x_lo0 + b_off, desc_hi, idesc, sfa, sfb, accumulate);
-                        accumulate = 1;
-                    } else {
-                        mx_issue(tmem_d, a_lo, x_lo0 + b_off, 256u, 2u * (uint32_t)p.P, p.ksteps, desc_hi, idesc, sfa, sfb, accumulate);
-                    }
-                    if (!p.resident && elect_one()) mma_commit(&bars[BAR_EMPTY_W0 + stage_i]);
-                    if (++stage_i == p.stages) { stage_i = 0; w_parity ^= 1u; }
                 }
             }
             if (!ok) break;
@@ -797,6 +816,15 @@ void fast_div_constants(uint32_t d, uint32_t *mul, uint32_t *sh)
     *mul = (uint32_t)(((1ull << (31 + l)) / d) + 1);
 }
 
+template <int EPI>
+lce_status launch_mx(const MxParams &p, dim3 grid, size_t smem, cudaStream_t s)
+{
+    static SmemOptIn opted;
+    if (!opted.ensure(bconv_mx_kernel<EPI>, smem)) return LCE_ERR_CUDA;
+    bconv_mx_kernel<EPI><<<grid, kMxThreads, smem, s>>>(p);
+    return launch_status();
+}
+
 int device_sms()
 {
     int sms = 148, dev = 0;
@@ -868,10 +896,11 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const void
     p.out_type = g.out_type; p.activation = g.activation;
     p.write_float = out != nullptr;
     if (!aligned(w_image, 16)) return LCE_ERR_ALIGNMENT;
-    static SmemOptIn opted;
-    if (!opted.ensure(bconv_mx_kernel, pl.smem)) return LCE_ERR_CUDA;
-    bconv_mx_kernel<<<dim3((unsigned)pl.ctas_x, (unsigned)pl.n_blocks), kMxThreads, pl.smem, s>>>(p);
-    return launch_status();
+    const dim3 grid((unsigned)pl.ctas_x, (unsigned)pl.n_blocks);
+    if (g.out_type == LCE_OUT_BITPACKED) return launch_mx<EPI_BITS>(p, grid, pl.smem, s);
+    if (g.out_type == LCE_OUT_INT32) return launch_mx<EPI_INT32>(p, grid, pl.smem, s);
+    if (residual || out_packed || !out || g.activation != LCE_ACT_NONE) return launch_mx<EPI_FLOAT_FUSED>(p, grid, pl.smem, s);
+    return launch_mx<EPI_FLOAT>(p, grid, pl.smem, s);
 }
 
 

@@ -23,28 +23,29 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+// One try: the hardware may suspend the thread until the phase completes or about `suspend_ns` have
+// passed (a suspended thread takes no issue slots, unlike a polling loop, and wakes when the barrier flips).
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity, uint32_t suspend_ns)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(suspend_ns)
         : "memory");
     return ok != 0;
 }
 // Wait bounded by time, not by iterations; false when the limit was reached.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs)
 {
-    for (int i = 0; i < 1024; ++i)  // short waits wake up at once
-        if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity, 2000u)) return true;
     const uint64_t t0 = globaltimer_ns();
     do {
-        for (int i = 0; i < 32; ++i) {
-            if (mbar_try_wait(bar, parity)) return true;
-            __nanosleep(64);
+        for (int i = 0; i < 16; ++i) {
+            if (mbar_try_wait(bar, parity, 20000u)) return true;
+            __nanosleep(32);  // in case the suspension is shorter than asked for: do not poll hot
         }
     } while (globaltimer_ns() - t0 < limit_ns);
     return false;

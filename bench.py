@@ -522,7 +522,7 @@ def time_chains(dev, reps: int = 5):
     device; reported beside the headline number, outside its timed region."""
     import torch
 
-    from paper_2011_09398_b200.chains import Chain
+    from chains import Chain
     out = {}
     for key, cfg, steps, name, batch in (("config4", 4, wl.config4_steps(), "X0", 128),
                                          ("config4_fused", 4, wl.config4_fused_steps(), "X0", 128),

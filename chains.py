@@ -1,6 +1,7 @@
 """Runs a list of hot-path steps (LceQuantize, LceBConv2d, add, LceBMaxPool2d) as consecutive
-C-ABI calls on one stream.  Argument marshalling only: buffers are torch CUDA tensors, weights are
-packed once at construction (load time), every step is one library call."""
+C-ABI calls on one stream (harness for the tests and bench.py, next to the workload lists it
+runs).  Argument marshalling only: buffers are torch CUDA tensors, weights are packed once at
+construction (load time), every step is one library call."""
 from __future__ import annotations
 
 from typing import Dict, List
@@ -9,8 +10,7 @@ import numpy as np
 import torch
 
 import lce_workloads as wl
-
-from . import binding as lce
+import paper_2011_09398_b200 as lce
 
 
 class Chain:

@@ -62,7 +62,7 @@ constexpr uint32_t kD1Col = 240;                             // TMEM column of t
 constexpr uint32_t kSfaCol = 480, kSfbCol = 496;             // block scales (all 1.0) of the A / B operand
 constexpr int kMaxTaps = 64;
 constexpr int kMaxStages = 32;
-constexpr int kPixSlots = 4;
+constexpr int kPixSlots = 8;                                 // see the note at kOffPix
 
 // shared-memory map (bytes)
 constexpr int kOffBars = 0;          // full_x[2] full_d[2] empty_d[2] done full_w[32] empty_w[32]
@@ -70,9 +70,12 @@ constexpr int kOffSlot = 1000;       // TMEM base address; 1004 fills issued, 10
 constexpr int kOffThr = 1024;        // float[128]
 constexpr int kOffMult = 1536;       // float[128]
 constexpr int kOffBias = 2048;       // float[128]
-constexpr int kOffPix = 2816;        // int32[4][224]: output pixel of a column, or -1
-constexpr int kOffTbl = 6400;        // uint2[512]: operand offsets (A, B; 16-byte units) of the MMAs of a tile
-constexpr int kOffDyn = 10496;       // raw words, weight ring, position buffers
+// int32[8][224]: output pixel of a column, or -1.  A ring of eight tiles: the finishers hand an
+// accumulator back before they have stored its values, so the loaders can be up to four tiles ahead
+// of a finisher that still reads its tile's slot (tile t + 5 cannot be staged before finisher t is done).
+constexpr int kOffPix = 2816;
+constexpr int kOffTbl = 9984;        // uint2[512]: operand offsets (A, B; 16-byte units) of the MMAs of a tile
+constexpr int kOffDyn = 14080;       // raw words, weight ring, position buffers
 constexpr int kMaxTblMmas = 512;
 
 enum { BAR_FULL_X0 = 0, BAR_FULL_X1, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_DONE, BAR_FULL_W0,

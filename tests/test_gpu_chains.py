@@ -7,7 +7,7 @@ import torch
 
 import lce_workloads as wl
 from chain_oracle import run_chain_oracle
-from paper_2011_09398_b200.chains import Chain
+from chains import Chain
 
 pytestmark = pytest.mark.gpu
 

@@ -1,11 +1,11 @@
-"""GPU parity at the full benchmark sizes (batch 64, load-time packed weights, the kernel the
-dispatcher picks: the launch configuration bench.py times).  The oracle cannot compute a whole
-7.4-G-MAC layer in test time, so every layer is checked two ways:
-  * sampled outputs: a few thousand (n, oh, ow, o) coordinates - random ones, every corner of the
-    tensor, and the pixels on either side of the CTA range boundaries - each computed by the oracle
-    from the definition, compared exactly (int32, bits) or within the float tolerance;
-  * a property that holds at any size and covers every output: complementing every weight bit
-    negates every accumulator (Section 2: the dot product of +-1 vectors is odd in either factor).
+"""GPU parity at the full benchmark sizes, every output element: configs 2 and 3 at batch 64 (the launch
+configuration bench.py times: load-time packed weights, the kernel the dispatcher picks, and the integer
+XOR/POPC kernel forced), config 4 at batch 128 and config 5 at batch 256 (every buffer of the chain).
+The oracle computes each whole layer from the definition (a fraction of a second per layer on the host
+cores); int32 and bit-packed outputs must be identical, float outputs must not differ in a single value
+(the stated tolerance is checked first).  Around that: range-edge samples as a fast first assertion and
+the weight-complement property of the accumulators (Section 2: the dot product of +-1 vectors is odd
+in either factor).
 """
 import numpy as np
 import pytest
@@ -14,19 +14,20 @@ import torch
 import lce_workloads as wl
 import oracle
 import paper_2011_09398_b200 as lce
-from gpu_util import DEV, to_dev, to_dev_words, words_to_host
+from chain_oracle import run_chain_oracle
+from chains import Chain
+from gpu_util import to_dev, to_dev_words
 
 pytestmark = pytest.mark.gpu
 
-SAMPLES = 3000
 
-
-def sample_indices(rng, spec):
+def edge_samples(rng, spec, count=400):
+    """Random outputs plus every corner of the tensor and the pixels on either side of the places where a
+    CTA's share of the work can begin or end."""
     N, OH, OW, Co = spec.batch, spec.out_h, spec.out_w, spec.out_c
-    idx = np.stack([rng.integers(0, N, SAMPLES), rng.integers(0, OH, SAMPLES), rng.integers(0, OW, SAMPLES),
-                    rng.integers(0, Co, SAMPLES)], axis=1)
+    idx = np.stack([rng.integers(0, N, count), rng.integers(0, OH, count), rng.integers(0, OW, count),
+                    rng.integers(0, Co, count)], axis=1)
     corners = [(n, oh, ow, o) for n in (0, N - 1) for oh in (0, OH - 1) for ow in (0, OW - 1) for o in (0, Co // 2, Co - 1)]
-    # flat pixels next to where a CTA's range can begin or end: multiples of 32 around M * k / 148
     M = N * OH * OW
     edges = []
     for k in range(1, 148, 7):
@@ -36,77 +37,127 @@ def sample_indices(rng, spec):
     return np.concatenate([idx, np.array(corners), np.array(edges)]).astype(np.int32)
 
 
-def run_layer(config, first_index, spec, kernel_choice, packed, out_type=None):
-    t = wl.conv_tensors(config, first_index, spec)
-    x = wl.activations(config, 0, (spec.batch, spec.in_h, spec.in_w, spec.in_c))
-    a_sign = oracle.sign(x)
-    a_words = lce.lce_bitpack(to_dev(x))
-    w_words = to_dev_words(oracle.bitpack_pm1(t.w_pm1))
-    ot = spec.out_type if out_type is None else out_type
+def gpu_layer(spec, t, a_words, w_words, kernel_choice, out_type):
     desc = lce.make_desc(spec.batch, spec.in_h, spec.in_w, spec.in_c, spec.out_c, (spec.kernel, spec.kernel),
-                         (spec.stride, spec.stride), spec.padding, ot, lce.ACT_NONE, kernel_choice, 1 if packed else 0)
-    wd = lce.lce_bconv2d_pack_weights(desc, w_words) if packed else w_words
-    mult = to_dev(t.multiplier) if ot == lce.OUT_FLOAT32 else None
-    bias = to_dev(t.bias) if ot == lce.OUT_FLOAT32 else None
-    thr = to_dev(t.thresholds) if ot == lce.OUT_BITPACKED else None
-    out = lce.lce_bconv2d(desc, a_words, wd, mult, bias, thr)
-    return t, a_sign, a_words, w_words, desc, out
+                         (spec.stride, spec.stride), spec.padding, out_type, lce.ACT_NONE, kernel_choice, 1)
+    wd = lce.lce_bconv2d_pack_weights(desc, w_words)
+    mult = to_dev(t.multiplier) if out_type == lce.OUT_FLOAT32 else None
+    bias = to_dev(t.bias) if out_type == lce.OUT_FLOAT32 else None
+    thr = to_dev(t.thresholds) if out_type == lce.OUT_BITPACKED else None
+    return lce.lce_bconv2d(desc, a_words, wd, mult, bias, thr), lce.lce_bconv2d_plan(desc)["kernel"]
 
 
-def check_samples(spec, t, a_sign, out, ot, rng):
-    idx = sample_indices(rng, spec)
-    acc = oracle.bconv2d_acc_at(a_sign, t.w_pm1, idx, (spec.stride, spec.stride), spec.padding)
-    n, oh, ow, o = idx.T
+def assert_layer_equal(spec, t, acc, out, out_type, rng):
     host = out.cpu().numpy()
-    if ot == lce.OUT_INT32:
-        np.testing.assert_array_equal(host[n, oh, ow, o], acc)
-    elif ot == lce.OUT_BITPACKED:
-        words = host.view(np.uint32)[n, oh, ow, o // 32]
-        np.testing.assert_array_equal((words >> (o % 32).astype(np.uint32)) & 1, (acc < t.thresholds[o]).astype(np.uint32))
+    idx = edge_samples(rng, spec)
+    n, oh, ow, o = idx.T
+    if out_type == lce.OUT_INT32:
+        np.testing.assert_array_equal(host[n, oh, ow, o], acc[n, oh, ow, o])       # fast first look
+        np.testing.assert_array_equal(host, acc)
+    elif out_type == lce.OUT_BITPACKED:
+        words = host.view(np.uint32)
+        np.testing.assert_array_equal((words[n, oh, ow, o // 32] >> (o % 32).astype(np.uint32)) & 1,
+                                      (acc[n, oh, ow, o] < t.thresholds[o]).astype(np.uint32))
+        np.testing.assert_array_equal(words, oracle.transform_bits(acc, t.thresholds))
     else:
-        got = host[n, oh, ow, o]
-        m, b = t.multiplier[o], t.bias[o]
-        want = (acc.astype(np.float64) * m.astype(np.float64) + b.astype(np.float64))
-        tol = 1e-6 * (np.abs(acc.astype(np.float64) * m) + np.abs(b))  # the stated tolerance; one fp32 rounding is 6e-8
-        assert np.all(np.abs(got.astype(np.float64) - want) <= tol)
+        want = oracle.transform_float(acc, t.multiplier, t.bias)
+        a64 = acc.astype(np.float64)
+        tol = 1e-6 * (np.abs(a64 * t.multiplier) + np.abs(t.bias))  # the stated tolerance; one fp32 rounding is 6e-8
+        assert np.all(np.abs(host.astype(np.float64) - (a64 * t.multiplier.astype(np.float64) + t.bias.astype(np.float64))) <= tol)
+        assert int((host != want).sum()) == 0                      # the goal: not one differing float
 
 
 FULL = [(2, 1 + 4 * i, s) for i, s in enumerate(wl.config2_specs())] + [(3, 1 + 4 * i, s) for i, s in enumerate(wl.config3_specs())]
 
 
 @pytest.mark.parametrize("config,first,spec", FULL, ids=[s.name for _, _, s in FULL])
-def test_full_size_layer_sampled_against_oracle(config, first, spec):
+def test_full_size_layer_every_element_against_oracle(config, first, spec):
+    """All outputs of the layer at batch 64, through the kernel AUTO picks for load-time packed weights
+    (the tensor-core kernel at these sizes) and through the integer XOR/POPC kernel."""
     rng = np.random.default_rng(config * 1000 + first)
-    t, a_sign, _, _, _, out = run_layer(config, first, spec, lce.KERNEL_AUTO, packed=True)
-    check_samples(spec, t, a_sign, out, spec.out_type, rng)
-
-
-@pytest.mark.parametrize("spec", wl.config2_specs()[1::2] + wl.config2_specs()[:1], ids=lambda s: s.name)
-def test_full_size_tensor_core_layer_sampled_against_oracle(spec):
-    rng = np.random.default_rng(abs(hash(spec.name)) % 2**32)
-    t, a_sign, _, _, _, out = run_layer(2, 1, spec, lce.KERNEL_TENSOR, packed=False)
-    check_samples(spec, t, a_sign, out, spec.out_type, rng)
+    t = wl.conv_tensors(config, first, spec)
+    x = wl.activations(config, 0, (spec.batch, spec.in_h, spec.in_w, spec.in_c))
+    acc = oracle.bconv2d_acc(oracle.sign(x), t.w_pm1, (spec.stride, spec.stride), spec.padding)
+    a_words = lce.lce_bitpack(to_dev(x))
+    w_words = to_dev_words(oracle.bitpack_pm1(t.w_pm1))
+    picked = set()
+    for kernel_choice in (lce.KERNEL_AUTO, lce.KERNEL_TILED):
+        out, kernel = gpu_layer(spec, t, a_words, w_words, kernel_choice, spec.out_type)
+        picked.add(kernel)
+        assert_layer_equal(spec, t, acc, out, spec.out_type, rng)
+    assert picked == {lce.KERNEL_TENSOR, lce.KERNEL_TILED}
     assert lce.lce_device_status() == 0
 
 
-@pytest.mark.parametrize("kernel_choice,packed", [(lce.KERNEL_AUTO, True), (lce.KERNEL_TENSOR, False)], ids=["auto-packed", "tensor"])
-@pytest.mark.parametrize("spec", wl.config2_specs()[::2], ids=lambda s: s.name)
-def test_full_size_weight_complement_negates_every_accumulator(spec, kernel_choice, packed):
-    t, a_sign, a_words, w_words, desc, acc = run_layer(2, 1, spec, kernel_choice, packed, out_type=lce.OUT_INT32)
+@pytest.mark.parametrize("kernel_choice", [lce.KERNEL_TENSOR, lce.KERNEL_TILED], ids=["tensor", "tiled"])
+@pytest.mark.parametrize("spec", wl.config2_specs()[::2] + wl.config3_specs()[:2], ids=lambda s: s.name)
+def test_full_size_accumulators_and_weight_complement(spec, kernel_choice):
+    t = wl.conv_tensors(2, 1, spec)
+    x = wl.activations(2, 0, (spec.batch, spec.in_h, spec.in_w, spec.in_c))
+    acc_ref = oracle.bconv2d_acc(oracle.sign(x), t.w_pm1, (spec.stride, spec.stride), spec.padding)
+    a_words = lce.lce_bitpack(to_dev(x))
+    w_words = to_dev_words(oracle.bitpack_pm1(t.w_pm1))
+    acc, _ = gpu_layer(spec, t, a_words, w_words, kernel_choice, lce.OUT_INT32)
+    np.testing.assert_array_equal(acc.cpu().numpy(), acc_ref)
     assert spec.in_c % 32 == 0  # no pad bits to keep at zero
-    w_flipped = torch.bitwise_not(w_words)
-    wd = lce.lce_bconv2d_pack_weights(desc, w_flipped) if packed else w_flipped
-    acc_flipped = lce.lce_bconv2d(desc, a_words, wd)
+    acc_flipped, _ = gpu_layer(spec, t, a_words, torch.bitwise_not(w_words), kernel_choice, lce.OUT_INT32)
     assert torch.equal(acc_flipped, -acc)
-    # and the accumulators have the parity of K and stay within [-K, K]
     K = spec.K
-    assert int(acc.abs().max().item()) <= K
-    assert bool(((acc + K) % 2 == 0).all().item())
-    check_samples(spec, t, a_sign, acc, lce.OUT_INT32, np.random.default_rng(7))
+    assert int(acc.abs().max().item()) <= K and bool(((acc + K) % 2 == 0).all().item())
 
 
-def test_full_size_largest_sweep_layer_5x5():
+def test_full_size_largest_sweep_layer_5x5_sampled():
+    """The paper's largest sweep layer (64x64x256, 5x5) at batch 64 is 429 G MAC: sampled here (a few
+    thousand outputs, corners and range edges), every element at batch 4 below."""
     spec = [s for s in wl.sweep_specs(64) if s.name == "sweep_64x64x256_k5"][0]
     rng = np.random.default_rng(55)
-    t, a_sign, _, _, _, out = run_layer(6, 1, spec, lce.KERNEL_AUTO, packed=True)
-    check_samples(spec, t, a_sign, out, spec.out_type, rng)
+    t = wl.conv_tensors(6, 1, spec)
+    x = wl.activations(6, 0, (spec.batch, spec.in_h, spec.in_w, spec.in_c))
+    a_sign = oracle.sign(x)
+    a_words = lce.lce_bitpack(to_dev(x))
+    w_words = to_dev_words(oracle.bitpack_pm1(t.w_pm1))
+    idx = edge_samples(rng, spec, 3000)
+    acc = oracle.bconv2d_acc_at(a_sign, t.w_pm1, idx, (1, 1), spec.padding)
+    n, oh, ow, o = idx.T
+    for kernel_choice in (lce.KERNEL_AUTO, lce.KERNEL_TILED):
+        out, _ = gpu_layer(spec, t, a_words, w_words, kernel_choice, lce.OUT_INT32)
+        np.testing.assert_array_equal(out.cpu().numpy()[n, oh, ow, o], acc)
+    small = wl.with_batch(spec, 4)
+    acc4 = oracle.bconv2d_acc(a_sign[:4], t.w_pm1, (1, 1), spec.padding)
+    for kernel_choice in (lce.KERNEL_TENSOR, lce.KERNEL_TILED):
+        out, _ = gpu_layer(small, t, a_words[:4].contiguous(), w_words, kernel_choice, spec.out_type)
+        assert_layer_equal(small, t, acc4, out, spec.out_type, rng)
+
+
+def compare_chain(chain, ref):
+    torch.cuda.synchronize()
+    for name, tensor in chain.buffers.items():
+        got = tensor.cpu().numpy()
+        want = ref[name]
+        if got.dtype == np.int32:
+            got = got.view(np.uint32)
+        assert got.shape == want.shape, name
+        assert np.array_equal(got, want), f"buffer {name} differs"
+
+
+@pytest.mark.parametrize("fused", [False, True], ids=["25-launches", "fused-15-launches"])
+def test_config4_block_stack_at_batch_128_every_buffer(fused):
+    steps = wl.config4_fused_steps() if fused else wl.config4_steps()
+    x = wl.activations(4, 0, (128, 56, 56, 64))
+    chain = Chain(steps, 4)
+    chain.set_input("X0", x)
+    chain.run()
+    compare_chain(chain, run_chain_oracle(steps, 4, {"X0": x}))
+    assert chain.buffers["Y3"].shape == (128, 7, 7, 512)
+    assert lce.lce_device_status() == 0
+
+
+def test_config5_body_at_batch_256_every_buffer():
+    steps = wl.config5_steps()
+    x = wl.activations(5, 0, (256, 224, 224, 3))
+    chain = Chain(steps, 5)
+    chain.set_input("X", x)
+    chain.run()
+    compare_chain(chain, run_chain_oracle(steps, 5, {"X": x}))
+    assert chain.buffers["T17"].shape == (256, 7, 7, 512)
+    assert lce.lce_device_status() == 0

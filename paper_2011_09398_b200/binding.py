@@ -71,10 +71,9 @@ def library() -> ctypes.CDLL:
         lib.lce_plan_destroy.restype = None
         lib.lce_bmaxpool.argtypes = [vp, vp] + [i32] * 9 + [vp]
         lib.lce_add_f32.argtypes = [vp, vp, vp, i64, vp]
-        lib.lce_probe_pipe.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), vp]
         for name in ("lce_bitpack", "lce_unpack", "lce_bconv2d_out_shape", "lce_bconv2d", "lce_bconv2d_host",
                      "lce_bconv2d_pack_weights",
-                     "lce_bmaxpool", "lce_add_f32", "lce_probe_pipe"):
+                     "lce_bmaxpool", "lce_add_f32"):
             getattr(lib, name).restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -380,12 +379,3 @@ def lce_device_wait_probe(limit_ns: int) -> None:
     lib.lce_device_wait_probe.argtypes = [ctypes.c_uint64, ctypes.c_void_p]
     lib.lce_device_wait_probe.restype = ctypes.c_int
     _check(lib.lce_device_wait_probe(int(limit_ns), _stream()), "lce_device_wait_probe")
-
-
-def lce_probe_pipe(mix: int, iterations: int = 2000) -> Tuple[float, float]:
-    """Returns (ops per second, ops per clock per SM) of one instruction mix; see lce.h."""
-    if not torch.cuda.is_available():
-        raise RuntimeError("lce_probe_pipe needs a CUDA device")
-    a, b = ctypes.c_double(), ctypes.c_double()
-    _check(library().lce_probe_pipe(mix, iterations, ctypes.byref(a), ctypes.byref(b), _stream()), "lce_probe_pipe")
-    return a.value, b.value

@@ -23,11 +23,7 @@
 //     shared memory once and used for all TP pixels (shared-memory bandwidth, not issue slots, is
 //     what this ordering saves);
 //   * epilogue: acc = K - 2*count, then float multiply-add, threshold + bit-pack, or raw int32.
-#include <stdio.h>
-#include <stdlib.h>
-
 #include "common.cuh"
-#include <atomic>
 
 #include "csa.cuh"
 #include "tiled_common.cuh"
@@ -129,20 +125,13 @@ bool choose_tile(const ConvGeom &g, int chan_blocks, SmemFn smem_for_tile, TileC
         int dev = 0;
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     }
-    int forced_tp = 0, forced_rounds = 0;
-#ifdef LCE_TUNING
-    if (const char *e = getenv("LCE_TP")) forced_tp = atoi(e);
-    if (const char *e = getenv("LCE_ROUNDS")) forced_rounds = atoi(e);
-#endif
     double best_cost = 0;
     best->tile = 0;
     // one pixel per thread exists for the KxK kernel with 4-warp CTAs only: the finest split of a
     // single image over the SMs (latency, not throughput)
     for (int tp = (ranged && nw == 4 && allow_tp1) ? 1 : 2; tp <= 4; ++tp) {
-        if (forced_tp && tp != forced_tp) continue;
         const int unit = 4 * nw * tp;
         for (int rounds = 1; rounds <= kMaxRounds; ++rounds) {
-            if (forced_rounds && rounds != forced_rounds) continue;
             // a half channel block takes two units of pixels per step
             if (has_half_block && (rounds & 1)) continue;
             const int tile = unit * rounds;
@@ -313,17 +302,6 @@ static lce_status plan_tiled_uncached(const ConvGeom &g, bool f32_input, TiledPa
         }
     }
     if (nw == 0) return LCE_ERR_UNSUPPORTED;
-#ifdef LCE_TUNING
-    {
-        const char *e_nw = getenv("LCE_NW"), *e_half = getenv("LCE_HALF");
-        if (e_nw || e_half) {
-            const int want_nw = e_nw ? atoi(e_nw) : nw;
-            const bool want_half = e_half ? (atoi(e_half) != 0 && can_half) : half;
-            TileChoice t;
-            if (choose_tile(g, chan_blocks, smem_for, &t, want_nw, 226 * 1024, want_half, true, !f32_input)) { c = t; nw = want_nw; half = want_half; }
-        }
-    }
-#endif
     set_tile(g, &p, c.tile);
     p.n_tiles = (int32_t)((g.M + c.tile - 1) / c.tile);
     p.half_block = half ? chan_blocks - 1 : -1;
@@ -337,12 +315,6 @@ static lce_status plan_tiled_uncached(const ConvGeom &g, bool f32_input, TiledPa
     plan->tp = c.tp;
     plan->smem_bytes = smem_bytes_for(g, p);
     plan->grid = dim3((unsigned)(p.full_blocks * p.ctas_full + p.ctas_half), 1, 1);
-#ifdef LCE_TUNING
-    if (getenv("LCE_VERBOSE"))
-        fprintf(stderr, "tiled %dx%d M=%lld Cw=%d Cout=%d: nw=%d tp=%d tile=%d grid=%dx%d+%d range=%d/%d smem=%zu cost=%.0f\n", g.KH, g.KW,
-                (long long)g.M, g.Cw, g.Cout, nw, c.tp, c.tile, p.ctas_full, p.full_blocks, p.ctas_half, p.range_full, p.range_half,
-                plan->smem_bytes, c.cost);
-#endif
     return LCE_OK;
 }
 
@@ -350,9 +322,6 @@ static lce_status plan_tiled_uncached(const ConvGeom &g, bool f32_input, TiledPa
 // of each host thread are kept (the cost model walks a few hundred candidates per call otherwise).
 static lce_status plan_tiled(const ConvGeom &g, bool f32_input, TiledParams *pp, TiledPlan *plan)
 {
-#ifdef LCE_TUNING
-    return plan_tiled_uncached(g, f32_input, pp, plan);  // environment knobs may change between calls
-#else
     struct Entry {
         ConvGeom g;
         bool f32_input, valid;
@@ -387,7 +356,6 @@ static lce_status plan_tiled(const ConvGeom &g, bool f32_input, TiledParams *pp,
     *pp = e.p;
     *plan = e.plan;
     return e.status;
-#endif
 }
 
 lce_status tiled_plan_info(const ConvGeom &g, TiledPlanInfo *info)

@@ -4,6 +4,7 @@
 // ceilings the convolution kernel is judged against.
 #include "common.cuh"
 #include "csa.cuh"
+#include "lce_probe.h"
 
 namespace lce {
 namespace {

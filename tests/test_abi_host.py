@@ -19,17 +19,25 @@ def lib():
     return lce.library()
 
 
-def declared_symbols():
-    text = (ROOT / "include" / "lce.h").read_text()
+def declared_symbols(header):
+    text = (ROOT / "include" / header).read_text()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(lce_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_every_declared_symbol_is_exported(lib):
-    names = declared_symbols()
-    assert {"lce_bitpack", "lce_bconv2d", "lce_bmaxpool"} <= set(names)
+    names = declared_symbols("lce.h")
+    assert {"lce_bitpack", "lce_bconv2d", "lce_bmaxpool", "lce_device_status_reset"} <= set(names)
     for name in names:
         assert hasattr(lib, name), f"{name} declared in lce.h but not exported"
+    # the measurement-only companion library has a header of its own
+    probe = ctypes.CDLL(str(lce_build.PROBE_LIB))
+    probe_names = declared_symbols("lce_probe.h")
+    assert probe_names == ["lce_probe_pipe"]
+    for name in probe_names:
+        assert hasattr(probe, name), f"{name} declared in lce_probe.h but not exported"
+    assert not hasattr(lib, "lce_probe_pipe")
+    assert {h.name for h in (ROOT / "include").glob("*.h")} == {"lce.h", "lce_probe.h"}
 
 
 def test_version_and_status_strings(lib):

@@ -240,6 +240,13 @@ __device__ __forceinline__ void mx_expand(const MxGeo &p, int q0, const uint32_t
     }
 }
 
+// B operand of tap (ky, kx): its phase buffer (stride 2) shifted by the tap's position offset, in 16-byte units
+__device__ __forceinline__ uint32_t tap_b_offset(const MxParams &p, int ky, int kx)
+{
+    if (p.stride == 2) return (uint32_t)((((ky & 1) * 2 + (kx & 1)) * p.Cw2) * p.P + (ky >> 1) * p.Wg + (kx >> 1));
+    return (uint32_t)(ky * p.Wg + kx);
+}
+
 // One lane of the converged warp, the same one every time
 __device__ __forceinline__ bool elect_one()
 {
@@ -280,51 +287,153 @@ __device__ __forceinline__ void mx_issue(uint32_t tmem_d, uint32_t a_lo, uint32_
     }
 }
 
-// `count` MMAs straight from a table of operand offsets, eight per block of code: the loads of a block
-// are independent, and between two MMAs there is nothing but the next descriptor's move.  The whole
-// issuer warp runs this with the same values in every lane, so that the descriptors stay in uniform
-// registers (a single diverged thread pays a register-to-uniform move per operand and MMA: about 200
-// clocks per instruction, measured); only the elected lane issues.
+// N MMAs straight from a table of operand offsets, back to back in one block of code: the loads of the
+// block are independent, and between two MMAs there is nothing but the next descriptor's move.  The
+// issuing warp pays about 100 clocks per tcgen05.mma in its instruction stream, whether the instruction
+// is predicated off or not (measured), so blocks come in exact sizes (8, 4, 2, 1) instead of one
+// predicated block of eight.  The whole issuer warp runs this; only the elected lane issues.
+template <int N>
+__device__ __forceinline__ void mx_issue_block(uint32_t tmem_d, const uint2 *tbl, uint32_t a_base, uint32_t b_base, uint32_t desc_hi,
+                                               uint32_t idesc, uint32_t sfa, uint32_t sfb, uint32_t accumulate);
+template <>
+__device__ __forceinline__ void mx_issue_block<8>(uint32_t tmem_d, const uint2 *tbl, uint32_t a_base, uint32_t b_base, uint32_t desc_hi,
+                                                  uint32_t idesc, uint32_t sfa, uint32_t sfb, uint32_t accumulate)
+{
+    uint32_t a[8], b[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const uint2 o = tbl[k];
+        a[k] = a_base + o.x;
+        b[k] = b_base + o.y;
+    }
+    if (elect_one()) {
+        asm volatile(
+            "{\n\t.reg .pred pa, pt;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 pa, %21, 0;\n\t"
+            "setp.eq.b32 pt, 0, 0;\n\t"
+            "mov.b64 da, {%1, %17};\n\t mov.b64 db, {%9, %17};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pa;\n\t"
+            "mov.b64 da, {%2, %17};\n\t mov.b64 db, {%10, %17};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+            "mov.b64 da, {%3, %17};\n\t mov.b64 db, {%11, %17};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+            "mov.b64 da, {%4, %17};\n\t mov.b64 db, {%12, %17};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+            "mov.b64 da, {%5, %17};\n\t mov.b64 db, {%13, %17};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+            "mov.b64 da, {%6, %17};\n\t mov.b64 db, {%14, %17};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+            "mov.b64 da, {%7, %17};\n\t mov.b64 db, {%15, %17};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+            "mov.b64 da, {%8, %17};\n\t mov.b64 db, {%16, %17};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
+            "}"
+            :
+            : "r"(tmem_d), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(a[4]), "r"(a[5]), "r"(a[6]), "r"(a[7]), "r"(b[0]), "r"(b[1]), "r"(b[2]), "r"(b[3]), "r"(b[4]), "r"(b[5]), "r"(b[6]), "r"(b[7]), "r"(desc_hi), "r"(idesc), "r"(sfa), "r"(sfb), "r"(accumulate)
+            : "memory");
+    }
+}
+template <>
+__device__ __forceinline__ void mx_issue_block<4>(uint32_t tmem_d, const uint2 *tbl, uint32_t a_base, uint32_t b_base, uint32_t desc_hi,
+                                                  uint32_t idesc, uint32_t sfa, uint32_t sfb, uint32_t accumulate)
+{
+    uint32_t a[4], b[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint2 o = tbl[k];
+        a[k] = a_base + o.x;
+        b[k] = b_base + o.y;
+    }
+    if (elect_one()) {
+        asm volatile(
+            "{\n\t.reg .pred pa, pt;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 pa, %13, 0;\n\t"
+            "setp.eq.b32 pt, 0, 0;\n\t"
+            "mov.b64 da, {%1, %9};\n\t mov.b64 db, {%5, %9};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %10, [%11], [%12], pa;\n\t"
+            "mov.b64 da, {%2, %9};\n\t mov.b64 db, {%6, %9};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %10, [%11], [%12], pt;\n\t"
+            "mov.b64 da, {%3, %9};\n\t mov.b64 db, {%7, %9};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %10, [%11], [%12], pt;\n\t"
+            "mov.b64 da, {%4, %9};\n\t mov.b64 db, {%8, %9};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %10, [%11], [%12], pt;\n\t"
+            "}"
+            :
+            : "r"(tmem_d), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]), "r"(b[2]), "r"(b[3]), "r"(desc_hi), "r"(idesc), "r"(sfa), "r"(sfb), "r"(accumulate)
+            : "memory");
+    }
+}
+template <>
+__device__ __forceinline__ void mx_issue_block<2>(uint32_t tmem_d, const uint2 *tbl, uint32_t a_base, uint32_t b_base, uint32_t desc_hi,
+                                                  uint32_t idesc, uint32_t sfa, uint32_t sfb, uint32_t accumulate)
+{
+    uint32_t a[2], b[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const uint2 o = tbl[k];
+        a[k] = a_base + o.x;
+        b[k] = b_base + o.y;
+    }
+    if (elect_one()) {
+        asm volatile(
+            "{\n\t.reg .pred pa, pt;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 pa, %9, 0;\n\t"
+            "setp.eq.b32 pt, 0, 0;\n\t"
+            "mov.b64 da, {%1, %5};\n\t mov.b64 db, {%3, %5};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %6, [%7], [%8], pa;\n\t"
+            "mov.b64 da, {%2, %5};\n\t mov.b64 db, {%4, %5};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %6, [%7], [%8], pt;\n\t"
+            "}"
+            :
+            : "r"(tmem_d), "r"(a[0]), "r"(a[1]), "r"(b[0]), "r"(b[1]), "r"(desc_hi), "r"(idesc), "r"(sfa), "r"(sfb), "r"(accumulate)
+            : "memory");
+    }
+}
+template <>
+__device__ __forceinline__ void mx_issue_block<1>(uint32_t tmem_d, const uint2 *tbl, uint32_t a_base, uint32_t b_base, uint32_t desc_hi,
+                                                  uint32_t idesc, uint32_t sfa, uint32_t sfb, uint32_t accumulate)
+{
+    uint32_t a[1], b[1];
+#pragma unroll
+    for (int k = 0; k < 1; ++k) {
+        const uint2 o = tbl[k];
+        a[k] = a_base + o.x;
+        b[k] = b_base + o.y;
+    }
+    if (elect_one()) {
+        asm volatile(
+            "{\n\t.reg .pred pa, pt;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 pa, %7, 0;\n\t"
+            "setp.eq.b32 pt, 0, 0;\n\t"
+            "mov.b64 da, {%1, %3};\n\t mov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %4, [%5], [%6], pa;\n\t"
+            "}"
+            :
+            : "r"(tmem_d), "r"(a[0]), "r"(b[0]), "r"(desc_hi), "r"(idesc), "r"(sfa), "r"(sfb), "r"(accumulate)
+            : "memory");
+    }
+}
+
 __device__ __forceinline__ void mx_issue_table(uint32_t tmem_d, const uint2 *tbl, int count, uint32_t a_base, uint32_t b_base, uint32_t desc_hi,
                                                uint32_t idesc, uint32_t sfa, uint32_t sfb, uint32_t &accumulate)
 {
-    for (int i0 = 0; i0 < count; i0 += 8) {
-        uint32_t a[8], b[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const uint2 o = tbl[min(i0 + k, count - 1)];
-            a[k] = a_base + o.x;
-            b[k] = b_base + o.y;
-        }
-        const int n = count - i0;
-        if (elect_one()) {
-            asm volatile(
-                "{\n\t.reg .pred pa, pt, g;\n\t.reg .b64 da, db;\n\t"
-                "setp.ne.b32 pa, %21, 0;\n\t"
-                "setp.eq.b32 pt, 0, 0;\n\t"
-                "mov.b64 da, {%1, %17};\n\t mov.b64 db, {%9, %17};\n\t"
-                "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pa;\n\t"
-                "setp.gt.s32 g, %22, 1;\n\t mov.b64 da, {%2, %17};\n\t mov.b64 db, {%10, %17};\n\t"
-                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
-                "setp.gt.s32 g, %22, 2;\n\t mov.b64 da, {%3, %17};\n\t mov.b64 db, {%11, %17};\n\t"
-                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
-                "setp.gt.s32 g, %22, 3;\n\t mov.b64 da, {%4, %17};\n\t mov.b64 db, {%12, %17};\n\t"
-                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
-                "setp.gt.s32 g, %22, 4;\n\t mov.b64 da, {%5, %17};\n\t mov.b64 db, {%13, %17};\n\t"
-                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
-                "setp.gt.s32 g, %22, 5;\n\t mov.b64 da, {%6, %17};\n\t mov.b64 db, {%14, %17};\n\t"
-                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
-                "setp.gt.s32 g, %22, 6;\n\t mov.b64 da, {%7, %17};\n\t mov.b64 db, {%15, %17};\n\t"
-                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
-                "setp.gt.s32 g, %22, 7;\n\t mov.b64 da, {%8, %17};\n\t mov.b64 db, {%16, %17};\n\t"
-                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %18, [%19], [%20], pt;\n\t"
-                "}"
-                :
-                : "r"(tmem_d), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(a[4]), "r"(a[5]), "r"(a[6]), "r"(a[7]), "r"(b[0]), "r"(b[1]),
-                  "r"(b[2]), "r"(b[3]), "r"(b[4]), "r"(b[5]), "r"(b[6]), "r"(b[7]), "r"(desc_hi), "r"(idesc), "r"(sfa), "r"(sfb),
-                  "r"(accumulate), "r"(n)
-                : "memory");
-        }
+    int i = 0;
+    for (; i + 8 <= count; i += 8) {
+        mx_issue_block<8>(tmem_d, tbl + i, a_base, b_base, desc_hi, idesc, sfa, sfb, accumulate);
+        accumulate = 1;
+    }
+    if (count & 4) {
+        mx_issue_block<4>(tmem_d, tbl + i, a_base, b_base, desc_hi, idesc, sfa, sfb, accumulate);
+        accumulate = 1;
+        i += 4;
+    }
+    if (count & 2) {
+        mx_issue_block<2>(tmem_d, tbl + i, a_base, b_base, desc_hi, idesc, sfa, sfb, accumulate);
+        accumulate = 1;
+        i += 2;
+    }
+    if (count & 1) {
+        mx_issue_block<1>(tmem_d, tbl + i, a_base, b_base, desc_hi, idesc, sfa, sfb, accumulate);
         accumulate = 1;
     }
 }
@@ -504,11 +613,8 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
     for (int e = tid; use_table && e < n_mma; e += kMxThreads) {
         const int tap = e / p.ksteps, kk = e - tap * p.ksteps;
         const int ky = tap / p.KW, kx = tap - ky * p.KW;
-        // A: K step (+ the tap's ring stage when all taps are resident: stage = tap); B: phase buffer (stride
-        // 2) shifted by the tap's position offset + K step
-        uint32_t b_off;
-        if (p.stride == 2) b_off = (uint32_t)((((ky & 1) * 2 + (kx & 1)) * p.Cw2) * p.P + (ky >> 1) * p.Wg + (kx >> 1));
-        else b_off = (uint32_t)(ky * p.Wg + kx);
+        // A: K step (+ the tap's ring stage when all taps are resident: stage = tap); B: the tap's offset + K step
+        const uint32_t b_off = tap_b_offset(p, ky, kx);
         tbl[e] = make_uint2((p.resident ? (uint32_t)tap * ((uint32_t)p.tap_bytes >> 4) : 0u) + 256u * kk, b_off + 2u * (uint32_t)p.P * kk);
     }
     if (tid == 0) {
@@ -632,32 +738,39 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
             const uint32_t x_lo0 = ((uint32_t)p.off_x >> 4) + (smem_u32(smem) >> 4) + (uint32_t)buf * ((uint32_t)p.x_bytes >> 4) + ((uint32_t)p.P << 16);
             uint32_t accumulate = 0;
-            if (use_table && p.resident && it > 0) {
-                // every tap is in shared memory: nothing to wait for between the MMAs of the tile
-                mx_issue_table(tmem_d, tbl, n_mma, w_lo0, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
+            if (p.resident) {
+                // every tap stays in shared memory: one wait for all of them (a single barrier counts the bytes
+                // of all the copies) before the CTA's first tile, then nothing between the MMAs of a tile
+                if (it == 0) {
+                    ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_FULL_W0], 0));
+                    if (!ok) break;
+                    if (lane == 0) fills[1] = 1;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                }
+                if (use_table) {
+                    mx_issue_table(tmem_d, tbl, n_mma, w_lo0, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
+                } else {
+                    uint32_t a_tap = w_lo0;
+                    for (int ky = 0; ky < p.KH; ++ky)
+                        for (int kx = 0; kx < p.KW; ++kx, a_tap += tap_units)
+                            mx_issue(tmem_d, a_tap, x_lo0 + tap_b_offset(p, ky, kx), 256u, 2u * (uint32_t)p.P, p.ksteps, desc_hi, idesc, sfa, sfb,
+                                     accumulate);
+                }
             } else {
+                // the taps stream through the ring: wait for each, issue its MMAs, hand its stage back
+                const bool by_table = use_table && (p.ksteps & 3) != 0;  // blocks of four by arithmetic waste nothing when 4 | K steps
                 int tap = 0;
                 for (int ky = 0; ky < p.KH && ok; ++ky) {
                     for (int kx = 0; kx < p.KW; ++kx, ++tap) {
-                        if (!p.resident || it == 0) {
-                            ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_FULL_W0 + stage_i], w_parity));
-                            if (!ok) break;
-                            ++g;
-                            if (lane == 0) fills[1] = g;
-                            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        }
+                        ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_FULL_W0 + stage_i], w_parity));
+                        if (!ok) break;
+                        ++g;
+                        if (lane == 0) fills[1] = g;
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         const uint32_t a_stage = w_lo0 + (uint32_t)stage_i * tap_units;
-                        if (use_table && p.ksteps <= 2) {
-                            mx_issue_table(tmem_d, tbl + tap * p.ksteps, p.ksteps, p.resident ? w_lo0 : a_stage, x_lo0, desc_hi, idesc, sfa, sfb,
-                                           accumulate);
-                        } else {
-                            // B operand of the tap: its phase buffer (stride 2) shifted by the tap's position offset
-                            uint32_t b_off;
-                            if (p.stride == 2) b_off = (uint32_t)((((ky & 1) * 2 + (kx & 1)) * p.Cw2) * p.P + (ky >> 1) * p.Wg + (kx >> 1));
-                            else b_off = (uint32_t)(ky * p.Wg + kx);
-                            mx_issue(tmem_d, a_stage, x_lo0 + b_off, 256u, 2u * (uint32_t)p.P, p.ksteps, desc_hi, idesc, sfa, sfb, accumulate);
-                        }
-                        if (!p.resident && elect_one()) mma_commit(&bars[BAR_EMPTY_W0 + stage_i]);
+                        if (by_table) mx_issue_table(tmem_d, tbl + tap * p.ksteps, p.ksteps, a_stage, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
+                        else mx_issue(tmem_d, a_stage, x_lo0 + tap_b_offset(p, ky, kx), 256u, 2u * (uint32_t)p.P, p.ksteps, desc_hi, idesc, sfa, sfb, accumulate);
+                        if (elect_one()) mma_commit(&bars[BAR_EMPTY_W0 + stage_i]);
                         if (++stage_i == p.stages) { stage_i = 0; w_parity ^= 1u; }
                     }
                 }
@@ -667,22 +780,30 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         }
     } else if (tid == kProducerTid) {
         // ======================= weight producer: one thread ==========================================
-        int my_tiles = 0;
-        for (int tile = first_tile; tile < p.n_tiles; tile += tile_step) ++my_tiles;
-        const int total = p.resident ? p.taps : my_tiles * p.taps;
         const uint8_t *src = p.wimg + (size_t)blockIdx.y * p.taps * p.tap_bytes;
-        int stage_i = 0, tap = 0;
-        uint32_t e_parity = 1;  // the first pass over the ring waits for nothing
-        for (int g = 0; g < total; ++g) {
-            if (g >= p.stages) {
-                ok = mbar_wait_bounded(&bars[BAR_EMPTY_W0 + stage_i], e_parity);
-                if (!ok) break;
+        if (p.resident) {
+            // all taps once, every copy counted on the same barrier
+            mbar_expect_tx(&bars[BAR_FULL_W0], (uint32_t)(p.taps * p.tap_bytes));
+            for (int tap = 0; tap < p.taps; ++tap)
+                bulk_copy_g2s(sW + (size_t)tap * p.tap_bytes, src + (size_t)tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0]);
+            fills[0] = 1;
+        } else {
+            int my_tiles = 0;
+            for (int tile = first_tile; tile < p.n_tiles; tile += tile_step) ++my_tiles;
+            const int total = my_tiles * p.taps;
+            int stage_i = 0, tap = 0;
+            uint32_t e_parity = 1;  // the first pass over the ring waits for nothing
+            for (int g = 0; g < total; ++g) {
+                if (g >= p.stages) {
+                    ok = mbar_wait_bounded(&bars[BAR_EMPTY_W0 + stage_i], e_parity);
+                    if (!ok) break;
+                }
+                mbar_expect_tx(&bars[BAR_FULL_W0 + stage_i], (uint32_t)p.tap_bytes);
+                bulk_copy_g2s(sW + (size_t)stage_i * p.tap_bytes, src + (size_t)tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0 + stage_i]);
+                fills[0] = g + 1;
+                if (++tap == p.taps) tap = 0;
+                if (++stage_i == p.stages) { stage_i = 0; e_parity ^= 1u; }
             }
-            mbar_expect_tx(&bars[BAR_FULL_W0 + stage_i], (uint32_t)p.tap_bytes);
-            bulk_copy_g2s(sW + (size_t)stage_i * p.tap_bytes, src + (size_t)tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0 + stage_i]);
-            fills[0] = g + 1;
-            if (++tap == p.taps) tap = 0;
-            if (++stage_i == p.stages) { stage_i = 0; e_parity ^= 1u; }
         }
     }
     if (!ok) mx_report_timeout(p.host_flag);

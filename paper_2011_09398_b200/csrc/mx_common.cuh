@@ -23,29 +23,30 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
-// One try: the hardware may suspend the thread until the phase completes or about `suspend_ns` have
-// passed (a suspended thread takes no issue slots, unlike a polling loop, and wakes when the barrier flips).
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity, uint32_t suspend_ns)
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity), "r"(suspend_ns)
+        : "r"(smem_u32(bar)), "r"(parity)
         : "memory");
     return ok != 0;
 }
-// Wait bounded by time, not by iterations; false when the limit was reached.
+// Wait bounded by time, not by iterations; false when the limit was reached.  (try_wait with a
+// suspend-time hint was measured here: a suspended thread often slept out its whole hint, microseconds
+// after the barrier had flipped, so the plain form is polled, with a short sleep once the wait is long.)
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs)
 {
-    if (mbar_try_wait(bar, parity, 2000u)) return true;
+    for (int i = 0; i < 64; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
     do {
-        for (int i = 0; i < 16; ++i) {
-            if (mbar_try_wait(bar, parity, 20000u)) return true;
-            __nanosleep(32);  // in case the suspension is shorter than asked for: do not poll hot
+        for (int i = 0; i < 256; ++i) {
+            if (mbar_try_wait(bar, parity)) return true;
+            __nanosleep(20);
         }
     } while (globaltimer_ns() - t0 < limit_ns);
     return false;

@@ -165,9 +165,11 @@ struct MxParams {
     int32_t N, H, W, Cw, Cw2, Cout, Cow;
     int32_t OH, OW, KH, KW, stride, pt, pl, K;
     int32_t Wg, Hg, n_phase;
-    uint32_t Wg_mul, Wg_sh, Hg_mul, Hg_sh, P_mul, P_sh;   // divisions by Wg, Hg, P as multiply + shift
-    int32_t Nt, P;           // tile width; staged positions per tile and phase
-    int32_t n_tiles, total_q;
+    uint32_t Wg_mul, Wg_sh, Hg_mul, Hg_sh;                // divisions by Wg, Hg as multiply + shift
+    uint32_t c0_mul, c0_sh, c1_mul, c1_sh;                // ... by the items per phase of a first / later chunk
+    int32_t Nt, P;           // tile width; rows of a position buffer per phase and channel word = T * Nt + halo
+    int32_t T, halo;         // tiles that share a position buffer; positions a tile reads beyond its own
+    int32_t n_tiles, n_super, total_q;
     int32_t taps, ksteps, stages, resident;
     int32_t tap_bytes, raw_words, x_bytes;
     int32_t off_w, off_x;    // byte offsets in shared memory
@@ -181,9 +183,16 @@ __device__ __forceinline__ int fast_div(int n, uint32_t mul, uint32_t sh) { retu
 // what the loaders need of the geometry, in registers (kernel parameters read inside their loops cost
 // more than the arithmetic)
 struct MxGeo {
-    int N, H, W, Cw, Cw2, Wg, Hg, P, items, stride, pt, pl, pad_zero, cp_words;
-    uint32_t Wg_mul, Wg_sh, Hg_mul, Hg_sh, P_mul, P_sh;
+    int N, H, W, Cw, Cw2, Wg, Hg, P, n_phase, stride, pt, pl, pad_zero, cp_words;
+    uint32_t Wg_mul, Wg_sh, Hg_mul, Hg_sh;
     const uint32_t *in;
+};
+
+// A chunk of a position buffer: rows lo .. lo + count - 1 (of every phase), which hold the grid positions
+// q0 + lo ..; (mul, sh) divide by count.
+struct MxChunk {
+    int q0, lo, count;
+    uint32_t mul, sh;
 };
 
 // position j of the tile that starts at q0, phase ph -> inside the image? and the pixel's word offset
@@ -199,13 +208,14 @@ __device__ __forceinline__ bool mx_locate(const MxGeo &p, int q0, int ph, int j,
     return ok;
 }
 
-// packed words of the tile's positions -> raw[item][Cw] (pad positions: zero words), asynchronously
-__device__ __forceinline__ void mx_prefetch(const MxGeo &p, int q0, uint32_t *raw, int ltid)
+// packed words of the chunk's positions -> raw[item][Cw] (pad positions: zero words), asynchronously
+__device__ __forceinline__ void mx_prefetch(const MxGeo &p, const MxChunk &c, uint32_t *raw, int ltid)
 {
-    for (int i = ltid; i < p.items; i += kLoaders) {
-        const int ph = fast_div(i, p.P_mul, p.P_sh), j = i - ph * p.P;
+    const int items = p.n_phase * c.count;
+    for (int i = ltid; i < items; i += kLoaders) {
+        const int ph = p.n_phase == 1 ? 0 : fast_div(i, c.mul, c.sh), j = i - ph * c.count;
         int64_t off;
-        const bool ok = mx_locate(p, q0, ph, j, &off);
+        const bool ok = mx_locate(p, c.q0 + c.lo, ph, j, &off);
         const uint32_t *src = p.in + off;
         uint32_t *dst = raw + (size_t)i * p.Cw;
         if (p.cp_words == 4) {
@@ -220,18 +230,19 @@ __device__ __forceinline__ void mx_prefetch(const MxGeo &p, int q0, uint32_t *ra
 }
 
 // every thread expands the words it prefetched itself (same item mapping): waiting for its own copies is enough
-__device__ __forceinline__ void mx_expand(const MxGeo &p, int q0, const uint32_t *raw, uint8_t *X, int ltid)
+__device__ __forceinline__ void mx_expand(const MxGeo &p, const MxChunk &c, const uint32_t *raw, uint8_t *X, int ltid)
 {
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    for (int i = ltid; i < p.items; i += kLoaders) {
-        const int ph = fast_div(i, p.P_mul, p.P_sh), j = i - ph * p.P;
+    const int items = p.n_phase * c.count;
+    for (int i = ltid; i < items; i += kLoaders) {
+        const int ph = p.n_phase == 1 ? 0 : fast_div(i, c.mul, c.sh), j = i - ph * c.count;
         bool zero = false;
         if (p.pad_zero) {
             int64_t off;
-            zero = !mx_locate(p, q0, ph, j, &off);
+            zero = !mx_locate(p, c.q0 + c.lo, ph, j, &off);
         }
         const uint32_t *src = raw + (size_t)i * p.Cw;
-        uint4 *dst = reinterpret_cast<uint4 *>(X) + (size_t)ph * p.Cw2 * p.P + j;
+        uint4 *dst = reinterpret_cast<uint4 *>(X) + (size_t)ph * p.Cw2 * p.P + c.lo + j;
         for (int cw = 0; cw < p.Cw; ++cw) {
             uint4 v = mx_expand_word(src[cw]);
             if (zero) v = make_uint4(0u, 0u, 0u, 0u);
@@ -510,6 +521,28 @@ __device__ __forceinline__ void mx_store_chunk(const float (&v)[32], int cols, c
                                                const float *resp, uint32_t *packp, int64_t cow, bool ch_ok, bool relu, bool write_float,
                                                float mult, float bias, int lane)
 {
+    if (MODE != EPI_FLOAT_FUSED) {
+        // straight-line code: every store is predicated, nothing branches, so the 32 positions' address
+        // arithmetic, multiply-adds and stores overlap instead of running one position after the other
+#pragma unroll
+        for (int j4 = 0; j4 < 32; j4 += 4) {
+            const int4 pix4 = *reinterpret_cast<const int4 *>(sPixChunk + j4);  // the same for every lane (slots past the tile: never stored)
+            const int pix[4] = {pix4.x, pix4.y, pix4.z, pix4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const bool st = ch_ok && pix[u] >= 0 && j4 + u < cols;
+                const int64_t o = pix[u] * cout;
+                if (MODE == EPI_FLOAT) {
+                    const float y = __fmaf_rn(v[j4 + u], mult, bias);
+                    if (st) outp[o] = y;
+                } else {
+                    const int32_t y = __float2int_rn(v[j4 + u]);
+                    if (st) reinterpret_cast<int32_t *>(outp)[o] = y;
+                }
+            }
+        }
+        return;
+    }
 #pragma unroll
     for (int j4 = 0; j4 < 32; j4 += 4) {
         if (j4 >= cols) break;
@@ -518,20 +551,13 @@ __device__ __forceinline__ void mx_store_chunk(const float (&v)[32], int cols, c
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             if (pix[u] < 0) continue;
-            const float a = v[j4 + u];
             const int64_t o = pix[u] * cout;
-            if (MODE == EPI_FLOAT) {
-                if (ch_ok) outp[o] = __fmaf_rn(a, mult, bias);
-            } else if (MODE == EPI_INT32) {
-                if (ch_ok) reinterpret_cast<int32_t *>(outp)[o] = __float2int_rn(a);
-            } else {
-                float y = __fmaf_rn(relu ? fmaxf(a, 0.f) : a, mult, bias);
-                if (resp && ch_ok) y = __fadd_rn(y, __ldg(resp + o));
-                if (write_float && ch_ok) outp[o] = y;
-                if (packp) {
-                    const uint32_t word = __ballot_sync(0xffffffffu, ch_ok && y < 0.f);
-                    if (lane == 0) packp[pix[u] * cow] = word;
-                }
+            float y = __fmaf_rn(relu ? fmaxf(v[j4 + u], 0.f) : v[j4 + u], mult, bias);
+            if (resp && ch_ok) y = __fadd_rn(y, __ldg(resp + o));
+            if (write_float && ch_ok) outp[o] = y;
+            if (packp) {
+                const uint32_t word = __ballot_sync(0xffffffffu, ch_ok && y < 0.f);
+                if (lane == 0) packp[pix[u] * cow] = word;
             }
         }
     }
@@ -659,34 +685,53 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         // ======================= loaders ==============================================================
         MxGeo geo;
         geo.N = p.N; geo.H = p.H; geo.W = p.W; geo.Cw = p.Cw; geo.Cw2 = p.Cw2; geo.Wg = p.Wg; geo.Hg = p.Hg; geo.P = p.P;
-        geo.items = p.n_phase * p.P; geo.stride = p.stride; geo.pt = p.pt; geo.pl = p.pl; geo.pad_zero = p.pad_zero; geo.cp_words = p.cp_words;
-        geo.Wg_mul = p.Wg_mul; geo.Wg_sh = p.Wg_sh; geo.Hg_mul = p.Hg_mul; geo.Hg_sh = p.Hg_sh; geo.P_mul = p.P_mul; geo.P_sh = p.P_sh;
+        geo.n_phase = p.n_phase; geo.stride = p.stride; geo.pt = p.pt; geo.pl = p.pl; geo.pad_zero = p.pad_zero; geo.cp_words = p.cp_words;
+        geo.Wg_mul = p.Wg_mul; geo.Wg_sh = p.Wg_sh; geo.Hg_mul = p.Hg_mul; geo.Hg_sh = p.Hg_sh;
         geo.in = p.in;
-        const int Nt = p.Nt, n_tiles = p.n_tiles, OH = p.OH, OW = p.OW, raw_words = p.raw_words;
+        const int Nt = p.Nt, T = p.T, halo = p.halo, n_tiles = p.n_tiles, n_super = p.n_super, OH = p.OH, OW = p.OW, raw_words = p.raw_words;
+        const uint32_t c0_mul = p.c0_mul, c0_sh = p.c0_sh, c1_mul = p.c1_mul, c1_sh = p.c1_sh;
         const size_t x_bytes = (size_t)p.x_bytes;
+        // the chunk of tile k of the super-tile that starts at position q0: the first tile brings the halo
+        auto chunk_of = [&](int q0, int k) {
+            MxChunk c;
+            c.q0 = q0;
+            c.lo = k ? k * Nt + halo : 0;
+            c.count = k ? Nt : Nt + halo;
+            c.mul = k ? c1_mul : c0_mul;
+            c.sh = k ? c1_sh : c0_sh;
+            return c;
+        };
         uint32_t par_full_d[2] = {0, 0};
-        int tile = first_tile;
-        if (tile < n_tiles) mx_prefetch(geo, tile * Nt, raw0, tid);
-        for (int it = 0; tile < n_tiles && ok; tile += tile_step, ++it) {
-            const int buf = it & 1;
-            if (it >= 2) {  // position buffer `buf` was read by the MMAs of tile it-2
-                ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + buf], par_full_d[buf]);
-                par_full_d[buf] ^= 1u;
-                if (!ok) break;
+        int it = 0;
+        if (first_tile < n_super) mx_prefetch(geo, chunk_of(first_tile * T * Nt, 0), raw0, tid);
+        for (int st = first_tile, is = 0; st < n_super && ok; st += tile_step, ++is) {
+            const int xbuf = is & 1, q0 = st * T * Nt;
+            uint8_t *X = sX0 + xbuf * x_bytes;
+            for (int k = 0; k < T && st * T + k < n_tiles; ++k, ++it) {
+                if (it >= 2) {
+                    // At most two tiles ahead of the MMAs: the MMAs of tile it - 2 are done.  That keeps the
+                    // arrivals on full_x within one phase of what the issuer has seen, and (the MMAs finish
+                    // in order) it means super-tile is - 2, whose position buffer this chunk may overwrite,
+                    // has been read completely.
+                    ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + (it & 1)], par_full_d[it & 1]);
+                    par_full_d[it & 1] ^= 1u;
+                    if (!ok) break;
+                }
+                mx_expand(geo, chunk_of(q0, k), raw0 + (it & 1) * raw_words, X, tid);
+                if (tid < Nt) {
+                    const int f = q0 + k * Nt + tid;
+                    const int r = fast_div(f, geo.Wg_mul, geo.Wg_sh), c = f - r * geo.Wg;
+                    const int n = fast_div(r, geo.Hg_mul, geo.Hg_sh), rr = r - n * geo.Hg;
+                    const bool col_ok = n < geo.N && rr < OH && c < OW;
+                    sPix[(it & (kPixSlots - 1)) * kMaxNt + tid] = col_ok ? (n * OH + rr) * OW + c : -1;
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(&bars[BAR_FULL_X0 + (it & 1)]);
+                // only now the words of the next chunk: the MMAs of this tile must not wait for loads they do not need
+                const bool more_here = k + 1 < T && st * T + k + 1 < n_tiles;
+                if (more_here) mx_prefetch(geo, chunk_of(q0, k + 1), raw0 + ((it + 1) & 1) * raw_words, tid);
+                else if (st + tile_step < n_super) mx_prefetch(geo, chunk_of((st + tile_step) * T * Nt, 0), raw0 + ((it + 1) & 1) * raw_words, tid);
             }
-            mx_expand(geo, tile * Nt, raw0 + buf * raw_words, sX0 + buf * x_bytes, tid);
-            if (tid < Nt) {
-                const int f = tile * Nt + tid;
-                const int r = fast_div(f, geo.Wg_mul, geo.Wg_sh), c = f - r * geo.Wg;
-                const int n = fast_div(r, geo.Hg_mul, geo.Hg_sh), rr = r - n * geo.Hg;
-                const bool col_ok = n < geo.N && rr < OH && c < OW;
-                sPix[(it & (kPixSlots - 1)) * kMaxNt + tid] = col_ok ? (n * OH + rr) * OW + c : -1;
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            mbar_arrive(&bars[BAR_FULL_X0 + buf]);
-            // only now the words of the next tile: the MMAs of this tile must not wait for loads they do not need
-            const int next = tile + tile_step;
-            if (next < n_tiles) mx_prefetch(geo, next * Nt, raw0 + (buf ^ 1) * raw_words, tid);
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else if (tid < kLoaders + kFinishers) {
@@ -695,20 +740,22 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         uint32_t par_full_d[2] = {0, 0};
         const int my_channel = (fw & 3) * 32 + lane;
         const float my_mult = sMult[my_channel], my_bias = sBias[my_channel];
-        int tile = first_tile;
-        for (int it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
-            const int buf = it & 1;
-            ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + buf], par_full_d[buf]);
-            par_full_d[buf] ^= 1u;
-            ok = __all_sync(0xffffffffu, ok);  // the warp goes on together (its epilogue uses warp-wide shuffles and ballots)
-            if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
-            const int32_t *pix = sPix + (it & (kPixSlots - 1)) * kMaxNt;
-            if (EPI == EPI_BITS)
-                mx_epilogue_bits(p, tmem_d, pix, ch0, sThr, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
-            else
-                mx_epilogue_values<EPI>(p, tmem_d, pix, ch0, my_mult, my_bias, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
+        int it = 0;
+        for (int st = first_tile; st < p.n_super && ok; st += tile_step) {
+            for (int k = 0; k < p.T && st * p.T + k < p.n_tiles; ++k, ++it) {
+                const int buf = it & 1;
+                ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + buf], par_full_d[buf]);
+                par_full_d[buf] ^= 1u;
+                ok = __all_sync(0xffffffffu, ok);  // the warp goes on together (its epilogue uses warp-wide shuffles and ballots)
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
+                const int32_t *pix = sPix + (it & (kPixSlots - 1)) * kMaxNt;
+                if (EPI == EPI_BITS)
+                    mx_epilogue_bits(p, tmem_d, pix, ch0, sThr, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
+                else
+                    mx_epilogue_values<EPI>(p, tmem_d, pix, ch0, my_mult, my_bias, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
+            }
         }
     } else if (warp == kIssuerWarp) {
         // ======================= MMA issuer: one warp, every lane with the same values ================
@@ -724,8 +771,10 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         uint32_t par_full_x[2] = {0, 0}, par_empty_d[2] = {0, 0};
         int g = 0, stage_i = 0;
         uint32_t w_parity = 0;
-        for (int tile = first_tile, it = 0; tile < p.n_tiles && ok; tile += tile_step, ++it) {
-            const int buf = it & 1;
+        int it = 0;
+        for (int st = first_tile, is = 0; st < p.n_super && ok; st += tile_step, ++is)
+        for (int k = 0; k < p.T && st * p.T + k < p.n_tiles && ok; ++k, ++it) {
+            const int buf = it & 1, xbuf = is & 1;
             ok = mbar_wait_bounded(&bars[BAR_FULL_X0 + buf], par_full_x[buf]);
             par_full_x[buf] ^= 1u;
             if (ok && it >= 2) {  // the accumulator buffer must have been read out
@@ -736,7 +785,9 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
-            const uint32_t x_lo0 = ((uint32_t)p.off_x >> 4) + (smem_u32(smem) >> 4) + (uint32_t)buf * ((uint32_t)p.x_bytes >> 4) + ((uint32_t)p.P << 16);
+            // B operand: the super-tile's position buffer from this tile's first row on
+            const uint32_t x_lo0 = ((uint32_t)p.off_x >> 4) + (smem_u32(smem) >> 4) + (uint32_t)xbuf * ((uint32_t)p.x_bytes >> 4) + (uint32_t)(k * p.Nt) +
+                                   ((uint32_t)p.P << 16);
             uint32_t accumulate = 0;
             if (p.resident) {
                 // every tap stays in shared memory: one wait for all of them (a single barrier counts the bytes
@@ -789,7 +840,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             fills[0] = 1;
         } else {
             int my_tiles = 0;
-            for (int tile = first_tile; tile < p.n_tiles; tile += tile_step) ++my_tiles;
+            for (int st = first_tile; st < p.n_super; st += tile_step) my_tiles += min(p.T, p.n_tiles - st * p.T);
             const int total = my_tiles * p.taps;
             int stage_i = 0, tap = 0;
             uint32_t e_parity = 1;  // the first pass over the ring waits for nothing
@@ -860,7 +911,7 @@ __global__ void mx_pack_weights_kernel(const uint32_t *w, uint4 *image, int Cout
 }
 
 struct MxPlan {
-    int Nt, P, stages, resident, n_blocks, ctas_x, n_tiles, total_q, Wg, Hg, n_phase, Cw2, taps, halo;
+    int Nt, P, T, stages, resident, n_blocks, ctas_x, n_tiles, n_super, total_q, Wg, Hg, n_phase, Cw2, taps, halo;
     size_t raw_words, x_bytes, tap_bytes, off_w, off_x, smem;
 };
 
@@ -897,34 +948,41 @@ bool mx_plan(const ConvGeom &g, int sms, MxPlan *pl)
     double best = 1e30;
     bool found = false;
     for (int nt = 16; nt <= kMaxNt; nt += 16) {
-        const int P = nt + halo;
-        if (P > 16383) break;  // descriptor strides are 14-bit counts of 16 bytes
-        const size_t raw_words = (((size_t)pl->n_phase * P * g.Cw + 3) / 4) * 4;
-        const size_t x_bytes = (size_t)pl->n_phase * pl->Cw2 * P * 16;
-        const size_t fixed = kOffDyn + 2 * raw_words * 4;
-        const size_t off_w = (fixed + 127) / 128 * 128;
-        const size_t rest = 2 * x_bytes + 256;
-        if (off_w + rest + 2 * pl->tap_bytes > kSmemLimit) continue;
-        int stages = (int)((kSmemLimit - off_w - rest) / pl->tap_bytes);
-        if (stages > kMaxStages) stages = kMaxStages;
-        const bool resident = stages >= taps;
-        if (resident) stages = taps;
         const int n_tiles = (int)((total_q + nt - 1) / nt);
-        const int ctas_x = min(ctas_max, n_tiles);
-        const int per_cta = (n_tiles + ctas_x - 1) / ctas_x;
-        // clocks per MMA: 43 + N/2, at least 95 (measured); streamed weights cost about as much again from L2
-        const double mma = (double)taps * ksteps * fmax(95.0, 43.0 + nt / 2.0);
-        const double tile = fmax(mma, resident ? 0.0 : (double)taps * pl->tap_bytes / 48.0) + 250.0;
-        const double cost = per_cta * tile;
-        if (cost < best) {
-            best = cost;
-            found = true;
-            pl->Nt = nt; pl->P = P; pl->stages = stages; pl->resident = resident ? 1 : 0;
-            pl->n_tiles = n_tiles; pl->ctas_x = ctas_x;
-            pl->raw_words = raw_words; pl->x_bytes = x_bytes;
-            pl->off_w = off_w;
-            pl->off_x = (off_w + (size_t)stages * pl->tap_bytes + 127) / 128 * 128;
-            pl->smem = pl->off_x + 2 * x_bytes;
+        for (int T = 1; T <= 8; ++T) {
+            // T tiles share one position buffer of T * nt + halo rows: the halo is staged once per T tiles
+            const int P = T * nt + halo;
+            if (P > 16383) break;  // descriptor strides are 14-bit counts of 16 bytes
+            if (T > 1 && (T - 1) * ctas_max >= n_tiles) break;   // no CTA would have that many tiles
+            const size_t raw_words = (((size_t)pl->n_phase * (nt + halo) * g.Cw + 3) / 4) * 4;
+            const size_t x_bytes = (size_t)pl->n_phase * pl->Cw2 * P * 16;
+            const size_t fixed = kOffDyn + 2 * raw_words * 4;
+            const size_t off_w = (fixed + 127) / 128 * 128;
+            const size_t rest = 2 * x_bytes + 256;
+            if (off_w + rest + (taps > 1 ? 2 : 1) * pl->tap_bytes > kSmemLimit) break;
+            int stages = (int)((kSmemLimit - off_w - rest) / pl->tap_bytes);
+            if (stages > kMaxStages) stages = kMaxStages;
+            const bool resident = stages >= taps;
+            if (resident) stages = taps;
+            const int n_super = (n_tiles + T - 1) / T;
+            const int ctas_x = min(ctas_max, n_super);
+            const int per_cta = ((n_super + ctas_x - 1) / ctas_x) * T;
+            // clocks per MMA: 43 + N/2, at least 100 (measured); streamed weights cost about as much again from
+            // L2; the loaders need about 400 + 8 clocks per staged position and tile
+            const double mma = (double)taps * ksteps * fmax(100.0, 43.0 + nt / 2.0);
+            const double stream = resident ? 0.0 : (double)taps * pl->tap_bytes / 48.0;
+            const double load = 400.0 + 8.0 * pl->n_phase * (nt + (double)halo / T);
+            const double cost = per_cta * (fmax(fmax(mma, stream), load) + 150.0);
+            if (cost < best) {
+                best = cost;
+                found = true;
+                pl->Nt = nt; pl->P = P; pl->T = T; pl->stages = stages; pl->resident = resident ? 1 : 0;
+                pl->n_tiles = n_tiles; pl->n_super = n_super; pl->ctas_x = ctas_x;
+                pl->raw_words = raw_words; pl->x_bytes = x_bytes;
+                pl->off_w = off_w;
+                pl->off_x = (off_w + (size_t)stages * pl->tap_bytes + 127) / 128 * 128;
+                pl->smem = pl->off_x + 2 * x_bytes;
+            }
         }
     }
     return found;
@@ -1010,8 +1068,9 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const void
     p.Wg = pl.Wg; p.Hg = pl.Hg; p.n_phase = pl.n_phase;
     fast_div_constants((uint32_t)pl.Wg, &p.Wg_mul, &p.Wg_sh);
     fast_div_constants((uint32_t)pl.Hg, &p.Hg_mul, &p.Hg_sh);
-    fast_div_constants((uint32_t)pl.P, &p.P_mul, &p.P_sh);
-    p.Nt = pl.Nt; p.P = pl.P; p.n_tiles = pl.n_tiles; p.total_q = pl.total_q;
+    fast_div_constants((uint32_t)(pl.Nt + pl.halo), &p.c0_mul, &p.c0_sh);
+    fast_div_constants((uint32_t)pl.Nt, &p.c1_mul, &p.c1_sh);
+    p.Nt = pl.Nt; p.P = pl.P; p.T = pl.T; p.halo = pl.halo; p.n_tiles = pl.n_tiles; p.n_super = pl.n_super; p.total_q = pl.total_q;
     p.taps = pl.taps; p.ksteps = pl.Cw2 / 2; p.stages = pl.stages; p.resident = pl.resident;
     p.tap_bytes = (int32_t)pl.tap_bytes; p.raw_words = (int32_t)pl.raw_words; p.x_bytes = (int32_t)pl.x_bytes;
     p.off_w = (int32_t)pl.off_w; p.off_x = (int32_t)pl.off_x;

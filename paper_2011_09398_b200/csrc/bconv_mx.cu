@@ -175,6 +175,7 @@ struct MxParams {
     int32_t off_w, off_x;    // byte offsets in shared memory
     int32_t cp_words;        // words per cp.async: 4, 2 or 1
     int32_t pad_zero, out_type, activation, write_float;
+    int32_t dup;             // copies of the channel block in the 128 rows: 2 for out_c <= 64, 4 for out_c <= 32, else 1
 };
 
 // n / d for 0 <= n < 2^31 with (mul, sh) from the host: floor(n * mul / 2^sh), exact
@@ -466,19 +467,22 @@ __device__ __forceinline__ uint32_t warp_transpose32(uint32_t m, int lane)
 __device__ __forceinline__ void mx_epilogue_bits(const MxParams &p, uint32_t tmem_d, const int32_t *sPix, int ch0, const float *sThr,
                                                  int fw, int lane, uint64_t *empty_d)
 {
-    const int quarter = fw & 3, group = fw >> 2;
+    // TMEM lane quarter of this warp; with few output channels the 128 rows hold `dup` copies of the channel
+    // block, and the warps of copy `sub` take other columns than those of copy 0: no finisher warp is idle
+    const int quarter = fw & 3, dup = p.dup, cq = quarter & (4 / dup - 1), sub = quarter / (4 / dup);
+    const int group = (fw >> 2) * dup + sub, n_groups = kColGroups * dup;
     const int Nt = p.Nt;
-    const bool real = ch0 + quarter * 32 < p.Cout;     // whole warp: any channel of its lanes exists
-    const float thr = sThr[quarter * 32 + lane];       // -inf for channels that do not exist: bit 0
+    const bool real = ch0 + cq * 32 < p.Cout;          // whole warp: any channel of its lanes exists
+    const float thr = sThr[cq * 32 + lane];            // -inf for channels that do not exist: bit 0
     const uint32_t lane_addr = tmem_d + ((uint32_t)(quarter * 32) << 16);
-    uint32_t *out = static_cast<uint32_t *>(p.out) + (ch0 >> 5) + quarter;
+    uint32_t *out = static_cast<uint32_t *>(p.out) + (ch0 >> 5) + cq;
     const int64_t cow = p.Cow;
     uint32_t words[2] = {0u, 0u};
     int pix[2] = {-1, -1};
     if (real) {
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
-            const int c0 = (group + k * kColGroups) * 32;
+            const int c0 = (group + k * n_groups) * 32;
             if (c0 >= Nt) break;
             float v[32];
             const bool full = c0 + 32 <= Nt;
@@ -543,21 +547,29 @@ __device__ __forceinline__ void mx_store_chunk(const float (&v)[32], int cols, c
         }
         return;
     }
+    // Eight positions at a time: first all their shortcut values are requested (eight independent 128-byte
+    // loads in flight; one position after the other would pay the memory latency 32 times per chunk), then
+    // the arithmetic, the stores and the ballots.
+    const float floor_v = relu ? 0.f : -INFINITY;
 #pragma unroll
-    for (int j4 = 0; j4 < 32; j4 += 4) {
-        if (j4 >= cols) break;
-        const int4 pix4 = *reinterpret_cast<const int4 *>(sPixChunk + j4);  // the same for every lane
-        const int pix[4] = {pix4.x, pix4.y, pix4.z, pix4.w};
+    for (int j8 = 0; j8 < 32; j8 += 8) {
+        const int4 pa = *reinterpret_cast<const int4 *>(sPixChunk + j8), pb = *reinterpret_cast<const int4 *>(sPixChunk + j8 + 4);  // the same for every lane
+        const int pix[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
+        float r[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            if (pix[u] < 0) continue;
-            const int64_t o = pix[u] * cout;
-            float y = __fmaf_rn(relu ? fmaxf(v[j4 + u], 0.f) : v[j4 + u], mult, bias);
-            if (resp && ch_ok) y = __fadd_rn(y, __ldg(resp + o));
-            if (write_float && ch_ok) outp[o] = y;
-            if (packp) {
+        for (int u = 0; u < 8; ++u) {
+            r[u] = 0.f;
+            if (resp != nullptr && ch_ok && pix[u] >= 0 && j8 + u < cols) r[u] = __ldg(resp + pix[u] * cout);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const bool pos_ok = pix[u] >= 0 && j8 + u < cols;   // the same for every lane
+            float y = __fmaf_rn(fmaxf(v[j8 + u], floor_v), mult, bias);
+            if (resp != nullptr) y = __fadd_rn(y, r[u]);
+            if (write_float && ch_ok && pos_ok) outp[pix[u] * cout] = y;
+            if (packp != nullptr) {
                 const uint32_t word = __ballot_sync(0xffffffffu, ch_ok && y < 0.f);
-                if (lane == 0) packp[pix[u] * cow] = word;
+                if (lane == 0 && pos_ok) packp[pix[u] * cow] = word;
             }
         }
     }
@@ -567,25 +579,26 @@ template <int MODE>
 __device__ __forceinline__ void mx_epilogue_values(const MxParams &p, uint32_t tmem_d, const int32_t *sPix, int ch0, float mult, float bias,
                                                    int fw, int lane, uint64_t *empty_d)
 {
-    const int quarter = fw & 3, group = fw >> 2;
-    const int channel = ch0 + quarter * 32 + lane;
+    const int quarter = fw & 3, dup = p.dup, cq = quarter & (4 / dup - 1), sub = quarter / (4 / dup);  // see mx_epilogue_bits
+    const int group = (fw >> 2) * dup + sub, n_groups = kColGroups * dup;
+    const int channel = ch0 + cq * 32 + lane;
     const int Nt = p.Nt;
     const int64_t cout = p.Cout, cow = p.Cow;
-    const bool real = ch0 + quarter * 32 < p.Cout;     // whole warp: any channel of its lanes exists
+    const bool real = ch0 + cq * 32 < p.Cout;          // whole warp: any channel of its lanes exists
     const bool ch_ok = channel < p.Cout;
     const bool relu = p.activation == LCE_ACT_RELU, write_float = p.write_float != 0;
     float *outp = static_cast<float *>(p.out) + channel;
     const float *resp = p.residual ? p.residual + channel : nullptr;
-    uint32_t *packp = p.out_packed ? p.out_packed + (ch0 >> 5) + quarter : nullptr;
+    uint32_t *packp = p.out_packed ? p.out_packed + (ch0 >> 5) + cq : nullptr;
     const uint32_t lane_addr = tmem_d + ((uint32_t)(quarter * 32) << 16);
-    const int n_chunks = (Nt + 31) >> 5;               // this warp takes chunk group, group + 4
+    const int n_chunks = (Nt + 31) >> 5;               // this warp takes chunk group, group + n_groups, ...
     if (!real || group >= n_chunks) {  // nothing to read for this warp
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         mbar_arrive(empty_d);
         return;
     }
-    const int last_chunk = group + ((n_chunks - 1 - group) / kColGroups) * kColGroups;
-    for (int ck = group; ck < n_chunks; ck += kColGroups) {
+    const int last_chunk = group + ((n_chunks - 1 - group) / n_groups) * n_groups;
+    for (int ck = group; ck < n_chunks; ck += n_groups) {
         const int c0 = ck * 32;
         const int cols = min(32, Nt - c0);
         float v[32];
@@ -738,7 +751,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         // ======================= finishers ============================================================
         const int fw = warp - kLoaders / 32;  // 0..15: lane quarter fw & 3 (= warp & 3), column group fw >> 2
         uint32_t par_full_d[2] = {0, 0};
-        const int my_channel = (fw & 3) * 32 + lane;
+        const int my_channel = ((fw & 3) & (4 / p.dup - 1)) * 32 + lane;
         const float my_mult = sMult[my_channel], my_bias = sBias[my_channel];
         int it = 0;
         for (int st = first_tile; st < p.n_super && ok; st += tile_step) {
@@ -878,8 +891,10 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
 
 // ---- load-time weight image -----------------------------------------------------------------------------
 // plain packed words [Cout][taps][Cw] -> e2m1 operand image [channel block][tap][Cw2][128 channels][16 bytes];
-// channels past Cout, the pad channel word of an odd Cw and channels past Cin inside a word are 0.0
-__global__ void mx_pack_weights_kernel(const uint32_t *w, uint4 *image, int Cout, int Cin, int Cw, int Cw2, int taps, int n_blocks)
+// channels past Cout, the pad channel word of an odd Cw and channels past Cin inside a word are 0.0; with out_c
+// <= 64 (<= 32) the rows hold two (four) copies of the channels, so that every TMEM lane quarter has work for a
+// finisher warp
+__global__ void mx_pack_weights_kernel(const uint32_t *w, uint4 *image, int Cout, int Cin, int Cw, int Cw2, int taps, int n_blocks, int dup)
 {
     const int64_t total = (int64_t)n_blocks * taps * Cw2 * 128;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
@@ -889,7 +904,7 @@ __global__ void mx_pack_weights_kernel(const uint32_t *w, uint4 *image, int Cout
         t /= Cw2;
         const int tap = (int)(t % taps);
         const int blk = (int)(t / taps);
-        const int o = blk * 128 + row;
+        const int o = blk * 128 + (row & (128 / dup - 1));  // few output channels: the block is repeated down the 128 rows
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (o < Cout && cw < Cw) {
             v = mx_expand_word(w[((int64_t)o * taps + tap) * Cw + cw]);
@@ -1007,6 +1022,8 @@ lce_status launch_mx(const MxParams &p, dim3 grid, size_t smem, cudaStream_t s)
     return launch_status();
 }
 
+int mx_dup(const ConvGeom &g) { return g.Cout <= 32 ? 4 : g.Cout <= 64 ? 2 : 1; }
+
 int device_sms()
 {
     int sms = 148, dev = 0;
@@ -1036,7 +1053,7 @@ lce_status launch_pack_weights_tensor(const ConvGeom &g, const uint32_t *w, void
     const int64_t total = (int64_t)pl.n_blocks * pl.taps * pl.Cw2 * 128;
     const int64_t want = (total + 255) / 256;
     const int blocks = (int)(want < 4096 ? want : 4096);
-    mx_pack_weights_kernel<<<blocks, 256, 0, s>>>(w, static_cast<uint4 *>(image), g.Cout, g.Cin, g.Cw, pl.Cw2, pl.taps, pl.n_blocks);
+    mx_pack_weights_kernel<<<blocks, 256, 0, s>>>(w, static_cast<uint4 *>(image), g.Cout, g.Cin, g.Cw, pl.Cw2, pl.taps, pl.n_blocks, mx_dup(g));
     mx_flag_array(false);  // load time is the moment to set up the host-visible status word (it cannot be done under stream capture)
     return launch_status();
 }
@@ -1078,6 +1095,7 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const void
     p.pad_zero = g.padding == LCE_PAD_SAME_ZERO;
     p.out_type = g.out_type; p.activation = g.activation;
     p.write_float = out != nullptr;
+    p.dup = mx_dup(g);
     if (!aligned(w_image, 16)) return LCE_ERR_ALIGNMENT;
     const dim3 grid((unsigned)pl.ctas_x, (unsigned)pl.n_blocks);
     if (g.out_type == LCE_OUT_BITPACKED) return launch_mx<EPI_BITS>(p, grid, pl.smem, s);

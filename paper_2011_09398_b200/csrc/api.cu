@@ -57,13 +57,19 @@ bool tiled_accepts(const ConvGeom &g, const void *out, const void *residual)
     return !((g.Cout & 3) == 0 && g.out_type != LCE_OUT_BITPACKED && (!aligned(out, 16) || !aligned(residual, 16)));
 }
 
-// AUTO takes the tensor-core kernel when the weights were packed at load time (its operand image
-// exists) and the layer is large enough to fill the machine: below about 2^28 binary MACs a launch is
-// dominated by fixed costs and the integer kernels, which start faster, win (measured).
+// AUTO takes the tensor-core kernel when the weights were packed at load time (its operand image exists)
+// and the layer is large enough to pay for that kernel's start-up, by what was measured on the paper's
+// layer sweep and the ImageNet-shaped bodies: from 2^29 binary MACs when all taps of a channel block
+// stay in shared memory, from 2^31 when they have to stream past once per tile; 3x3 and smaller filters
+// on at most 32 input channels stay on the integer kernels (half of every 64-deep MMA would be padding).
 bool tensor_preferred(const ConvGeom &g)
 {
+    if (patch_covers(g)) return false;
+    if (g.Cin <= 32 && g.KH * g.KW <= 9) return false;
+    TensorPlanInfo t{};
+    if (tensor_plan_info(g, &t) != LCE_OK) return false;
     const double macs = (double)g.M * g.Cout * g.KH * g.KW * g.Cin;
-    return macs >= 268435456.0 && !patch_covers(g);
+    return macs >= (t.weights_resident ? 536870912.0 : 2147483648.0);
 }
 
 enum KernelPick { PICK_NONE = 0, PICK_DIRECT, PICK_PATCH, PICK_TILED, PICK_TENSOR };

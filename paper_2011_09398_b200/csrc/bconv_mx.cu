@@ -932,7 +932,40 @@ struct MxPlan {
 
 constexpr size_t kSmemLimit = 227 * 1024;
 
+bool mx_plan_uncached(const ConvGeom &g, int sms, MxPlan *pl);
+
+// The plan depends on the geometry alone, and a network repeats few geometries: the last few plans of
+// each host thread are kept (the search below walks about a hundred candidates otherwise).
 bool mx_plan(const ConvGeom &g, int sms, MxPlan *pl)
+{
+    struct Entry {
+        ConvGeom g;
+        int sms;
+        bool valid, found;
+        MxPlan plan;
+    };
+    constexpr int kEntries = 16;
+    static thread_local Entry cache[kEntries];
+    static thread_local int next = 0;
+    for (int i = 0; i < kEntries; ++i) {
+        const Entry &e = cache[i];
+        if (e.valid && e.sms == sms && memcmp(&e.g, &g, sizeof(ConvGeom)) == 0) {
+            *pl = e.plan;
+            return e.found;
+        }
+    }
+    Entry &e = cache[next];
+    next = (next + 1) % kEntries;
+    memset(&e.g, 0, sizeof(ConvGeom));
+    e.g = g;
+    e.sms = sms;
+    e.found = mx_plan_uncached(g, sms, &e.plan);
+    e.valid = true;
+    *pl = e.plan;
+    return e.found;
+}
+
+bool mx_plan_uncached(const ConvGeom &g, int sms, MxPlan *pl)
 {
     if (g.sh != g.sw || (g.sh != 1 && g.sh != 2)) return false;
     if (g.Cw > 32) return false;

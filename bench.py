@@ -343,7 +343,7 @@ def run_lce(args):
 
         # ---- the same step for about a second more, so that the clock record has hundreds of samples ----
         sustained = None
-        if world == 1:
+        if world == 1 and not args.profile:
             n_more = int(min(4000, max(50, 1.0 / max(1e-6, (np.mean(step_ms) + 0.12) * 1e-3))))
             more_ms, more_clocks, more_wall = timed_steps(graph, n_more, True)
             sustained = {"steps": n_more, "ms_per_step": float(np.mean(more_ms)), "wall_s": more_wall, "clocks": more_clocks,
@@ -675,7 +675,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-chains", action="store_true", help="skip the config 4 / config 5 chain timings")
     ap.add_argument("--no-sweep", action="store_true", help="skip the paper's 48-layer convolution sweep")
+    ap.add_argument("--profile", action="store_true",
+                    help="short form for runs under ncu: the timed steps of the default and the integer path only (no one-second "
+                         "clock loop, chains, sweep or CPU baseline)")
     args = ap.parse_args()
+    if args.profile:
+        args.no_chains = args.no_cpu_baseline = True
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -693,9 +693,13 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
+    // the next kernel of the stream may start setting itself up as soon as every CTA of this one has got here
+    if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     bool ok = true;
     if (tid < kLoaders) {
         // ======================= loaders ==============================================================
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // the activations may come from the previous kernel
         MxGeo geo;
         geo.N = p.N; geo.H = p.H; geo.W = p.W; geo.Cw = p.Cw; geo.Cw2 = p.Cw2; geo.Wg = p.Wg; geo.Hg = p.Hg; geo.P = p.P;
         geo.n_phase = p.n_phase; geo.stride = p.stride; geo.pt = p.pt; geo.pl = p.pl; geo.pad_zero = p.pad_zero; geo.cp_words = p.cp_words;
@@ -749,6 +753,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else if (tid < kLoaders + kFinishers) {
         // ======================= finishers ============================================================
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // outputs and the shortcut tensor: only after the previous kernel
         const int fw = warp - kLoaders / 32;  // 0..15: lane quarter fw & 3 (= warp & 3), column group fw >> 2
         uint32_t par_full_d[2] = {0, 0};
         const int my_channel = ((fw & 3) & (4 / p.dup - 1)) * 32 + lane;
@@ -1051,8 +1056,25 @@ lce_status launch_mx(const MxParams &p, dim3 grid, size_t smem, cudaStream_t s)
 {
     static SmemOptIn opted;
     if (!opted.ensure(bconv_mx_kernel<EPI>, smem)) return LCE_ERR_CUDA;
-    bconv_mx_kernel<EPI><<<grid, kMxThreads, smem, s>>>(p);
-    return launch_status();
+    // Programmatic dependent launch: the CTAs of this grid may be scheduled while the previous kernel of the
+    // stream is still draining; they set themselves up and fetch their weights (constants of the model),
+    // and wait for the previous kernel's completion (griddepcontrol.wait) before they touch anything it may
+    // have written or may still read: the activations, the shortcut tensor, the outputs.
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kMxThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, bconv_mx_kernel<EPI>, p) != cudaSuccess) {
+        cudaGetLastError();
+        return LCE_ERR_CUDA;
+    }
+    return LCE_OK;
 }
 
 int mx_dup(const ConvGeom &g) { return g.Cout <= 32 ? 4 : g.Cout <= 64 ? 2 : 1; }

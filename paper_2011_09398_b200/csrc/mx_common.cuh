@@ -40,13 +40,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // after the barrier had flipped, so the plain form is polled, with a short sleep once the wait is long.)
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs)
 {
-    for (int i = 0; i < 64; ++i)
+    for (int i = 0; i < 16; ++i)
         if (mbar_try_wait(bar, parity)) return true;
+    // a longer wait: sleep between polls, a little longer every time (polling warps take issue slots from
+    // the warps that work; ncu counted about as many poll instructions as useful ones without this)
     const uint64_t t0 = globaltimer_ns();
+    uint32_t nap = 32;
     do {
-        for (int i = 0; i < 256; ++i) {
+        for (int i = 0; i < 64; ++i) {
+            __nanosleep(nap);
             if (mbar_try_wait(bar, parity)) return true;
-            __nanosleep(20);
+            if (nap < 256) nap += nap >> 1;
         }
     } while (globaltimer_ns() - t0 < limit_ns);
     return false;

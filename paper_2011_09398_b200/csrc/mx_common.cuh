@@ -38,15 +38,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // Wait bounded by time, not by iterations; false when the limit was reached.  (try_wait with a
 // suspend-time hint was measured here: a suspended thread often slept out its whole hint, microseconds
 // after the barrier had flipped, so the plain form is polled, with a short sleep once the wait is long.)
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs)
+// The waiting itself is one copy of code shared by all call sites (inlined and unrolled, the loops below were
+// 4 KB per call site and two thirds of the kernel: four roles running side by side then miss the
+// instruction caches all the time).
+__device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, uint64_t limit_ns)
 {
+#pragma unroll 1
     for (int i = 0; i < 16; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     // a longer wait: sleep between polls, a little longer every time (polling warps take issue slots from
-    // the warps that work; ncu counted about as many poll instructions as useful ones without this)
+    // the warps that work)
     const uint64_t t0 = globaltimer_ns();
     uint32_t nap = 32;
     do {
+#pragma unroll 1
         for (int i = 0; i < 64; ++i) {
             __nanosleep(nap);
             if (mbar_try_wait(bar, parity)) return true;
@@ -54,6 +59,11 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity
         }
     } while (globaltimer_ns() - t0 < limit_ns);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs)
+{
+    if (mbar_try_wait(bar, parity)) return true;  // already there: the common case on the critical path
+    return mbar_wait_slow(bar, parity, limit_ns);
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
 {

@@ -22,23 +22,30 @@
 //     (ky % 2, kx % 2).  Positions that are no output (pad columns, pad rows) are computed and dropped.
 //   * shared memory holds, per phase, [channel word][position][16 bytes]: the B operand of a tap is
 //     the same buffer shifted by the tap's position offset (K-major, no swizzle, rows 16 bytes
-//     apart), so every staged position is expanded once for all taps.
+//     apart), so every staged position is expanded once for all taps.  T consecutive tiles share one
+//     buffer of T * Nt + halo rows, so the halo a tile reads beyond its own positions is staged once
+//     per T tiles; there are two such buffers.
 //   * the weights were expanded when the model was loaded (lce_bconv2d_pack_weights) into the exact
-//     operand image [channel block][tap][channel word][128 channels][16 bytes]; the bulk-copy engine
-//     brings one tap at a time into a ring of shared-memory stages (cp.async.bulk + mbarrier
-//     transaction count).  If the ring holds every tap they are fetched once per CTA, otherwise they
-//     stream past once per tile.
-//   * roles: 8 loader warps (prefetch packed words with cp.async, expand), one thread that issues
-//     the MMAs, one thread that feeds the weight ring, 8 finisher warps (tcgen05.ld, output
-//     transform, stores).  Two position buffers and two accumulator buffers: the expansion of tile
-//     t+1, the MMAs of tile t and the output transform of tile t-1 overlap.  The roles meet only
-//     through mbarriers; every wait is bounded by time, after which the kernel records a status,
-//     waits (bounded) for what it has in flight, frees its TMEM and returns.
+//     operand image [channel block][tap][channel word][128 channels][16 bytes] (for out_c <= 64 the
+//     channel block is repeated down the 128 rows, so that every TMEM lane quarter holds values a
+//     finisher warp can work on); the bulk-copy engine brings taps into a ring of shared-memory stages
+//     (cp.async.bulk + mbarrier transaction count).  If the ring holds every tap they are fetched once
+//     per CTA, all counted on one barrier; otherwise they stream past once per tile.
+//   * roles: 8 loader warps (prefetch the packed words of the next chunk with cp.async, expand the
+//     current one), one warp that issues the MMAs (all lanes run the same code, the elected lane
+//     issues), one thread that feeds the weight ring, 16 finisher warps (tcgen05.ld, output transform,
+//     stores).  Two accumulator buffers: the expansion of tile t+1, the MMAs of tile t and the output
+//     transform of tile t-1 overlap.  The roles meet only through mbarriers; every wait is bounded by
+//     time, after which the kernel records a status, waits (bounded) for what it has in flight, frees
+//     its TMEM and returns.
 //   * output transform (Section 3.2): a TMEM lane is a channel and a column a position.  Bit-packed
 //     output: the sign of (accumulator - threshold) of 32 positions per lane, then a 32 x 32 bit
 //     transpose across the warp gives each lane the finished word of one pixel.  Float / int32 output
 //     is written straight from the registers: per position a warp stores its 32 consecutive channels as
 //     one 128-byte line.
+//   * launched with programmatic stream serialization: set-up and the weight copies may overlap the
+//     tail of the previous kernel of the stream; activations, shortcut and outputs are touched only
+//     after griddepcontrol.wait.
 #include <atomic>
 #include <math.h>
 #include <mutex>

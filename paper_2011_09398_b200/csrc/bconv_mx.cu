@@ -182,7 +182,7 @@ struct MxParams {
     int32_t off_w, off_x;    // byte offsets in shared memory
     int32_t cp_words;        // words per cp.async: 4, 2 or 1
     int32_t pad_zero, out_type, activation, write_float;
-    int32_t dup;             // copies of the channel block in the 128 rows: 2 for out_c <= 64, 4 for out_c <= 32, else 1
+    int32_t dup_log2;        // log2 of the copies of the channel block in the 128 rows: 1 for out_c <= 64, 2 for out_c <= 32, else 0
 };
 
 // n / d for 0 <= n < 2^31 with (mul, sh) from the host: floor(n * mul / 2^sh), exact
@@ -469,54 +469,90 @@ __device__ __forceinline__ uint32_t warp_transpose32(uint32_t m, int lane)
     return m;
 }
 
-// Bit-packed output of one tile (Section 3.2: accumulator compared with the per-channel threshold).
-// Lane = channel ch0 + 32 * quarter + lane; this warp takes every fourth 32-column chunk (at most two).
-__device__ __forceinline__ void mx_epilogue_bits(const MxParams &p, uint32_t tmem_d, const int32_t *sPix, int ch0, const float *sThr,
-                                                 int fw, int lane, uint64_t *empty_d)
+// What a finisher warp needs for every tile, worked out once before its tile loop (divisions and
+// kernel-parameter reads per tile cost a third of the warp's instructions when they sat in the epilogue).
+// TMEM lane quarter of the warp = warp % 4; with few output channels the 128 rows hold `dup` copies of
+// the channel block, and the warps of copy `sub` take other columns than those of copy 0, so that no
+// finisher warp is idle.
+struct MxFin {
+    int Nt, n_chunks;        // tile width; 32-column chunks of a tile
+    int group, n_groups;     // this warp takes chunks group, group + n_groups, ...
+    int last_chunk;          // its last one (-1: none: nothing to read for this warp)
+    uint32_t lane_off;       // TMEM lane offset of its quarter
+    bool ch_ok;              // this lane's channel exists
+    float thr, mult, bias;   // this lane's channel: threshold (-inf if it does not exist), multiplier, bias
+    int64_t cout, cow;
+    uint32_t *out_words;     // bit-packed output, at this warp's channel word
+    float *outp;             // float / int32 output, at this lane's channel
+    const float *resp;       // shortcut tensor at this lane's channel, or null
+    uint32_t *packp;         // re-quantised copy at this warp's channel word, or null
+    bool relu, write_float;
+};
+
+__device__ __forceinline__ MxFin mx_fin_context(const MxParams &p, int fw, int lane, int ch0, const float *sThr, const float *sMult,
+                                                const float *sBias)
 {
-    // TMEM lane quarter of this warp; with few output channels the 128 rows hold `dup` copies of the channel
-    // block, and the warps of copy `sub` take other columns than those of copy 0: no finisher warp is idle
-    const int quarter = fw & 3, dup = p.dup, cq = quarter & (4 / dup - 1), sub = quarter / (4 / dup);
-    const int group = (fw >> 2) * dup + sub, n_groups = kColGroups * dup;
-    const int Nt = p.Nt;
-    const bool real = ch0 + cq * 32 < p.Cout;          // whole warp: any channel of its lanes exists
-    const float thr = sThr[cq * 32 + lane];            // -inf for channels that do not exist: bit 0
-    const uint32_t lane_addr = tmem_d + ((uint32_t)(quarter * 32) << 16);
-    uint32_t *out = static_cast<uint32_t *>(p.out) + (ch0 >> 5) + cq;
-    const int64_t cow = p.Cow;
-    uint32_t words[2] = {0u, 0u};
-    int pix[2] = {-1, -1};
-    if (real) {
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-            const int c0 = (group + k * n_groups) * 32;
-            if (c0 >= Nt) break;
-            float v[32];
-            const bool full = c0 + 32 <= Nt;
-            if (full) tmem_ld32(lane_addr + (uint32_t)c0, v);
-            else tmem_ld16(lane_addr + (uint32_t)c0, v);
-            // bit j = (acc_j < thr): the sign of acc - thr (both are small integers held exactly);
-            // four short chains instead of one long one
-            uint32_t m0 = 0u, m1 = 0u, m2 = 0u, m3 = 0u;
-#pragma unroll
-            for (int j = 7; j >= 0; --j) {
-                m0 = __funnelshift_l(__float_as_uint(v[j] - thr), m0, 1);
-                m1 = __funnelshift_l(__float_as_uint(v[8 + j] - thr), m1, 1);
-                m2 = __funnelshift_l(__float_as_uint(v[16 + j] - thr), m2, 1);
-                m3 = __funnelshift_l(__float_as_uint(v[24 + j] - thr), m3, 1);
-            }
-            uint32_t m = m0 | (m1 << 8);
-            if (full) m |= (m2 << 16) | (m3 << 24);
-            words[k] = warp_transpose32(m, lane);
-            pix[k] = (c0 + lane < Nt) ? sPix[c0 + lane] : -1;
+    MxFin f;
+    const int quarter = fw & 3, dl = p.dup_log2;                    // dup = 1 << dl copies of the channel block
+    const int cq = quarter & ((4 >> dl) - 1), sub = quarter >> (2 - dl);
+    const int channel = ch0 + cq * 32 + lane;
+    f.Nt = p.Nt;
+    f.n_chunks = (p.Nt + 31) >> 5;
+    f.group = ((fw >> 2) << dl) + sub;
+    f.n_groups = kColGroups << dl;                                   // 4, 8 or 16
+    const bool real = ch0 + cq * 32 < p.Cout && f.group < f.n_chunks;
+    f.last_chunk = real ? f.group + ((f.n_chunks - 1 - f.group) & ~(f.n_groups - 1)) : -1;
+    f.lane_off = (uint32_t)(quarter * 32) << 16;
+    f.ch_ok = channel < p.Cout;
+    f.thr = sThr[cq * 32 + lane];
+    f.mult = sMult[cq * 32 + lane];
+    f.bias = sBias[cq * 32 + lane];
+    f.cout = p.Cout;
+    f.cow = p.Cow;
+    f.out_words = static_cast<uint32_t *>(p.out) + (ch0 >> 5) + cq;
+    f.outp = static_cast<float *>(p.out) + channel;
+    f.resp = p.residual ? p.residual + channel : nullptr;
+    f.packp = p.out_packed ? p.out_packed + (ch0 >> 5) + cq : nullptr;
+    f.relu = p.activation == LCE_ACT_RELU;
+    f.write_float = p.write_float != 0;
+    return f;
+}
+
+// Bit-packed output of one tile (Section 3.2: accumulator compared with the per-channel threshold).
+// Lane = channel; per 32-column chunk the sign of (accumulator - threshold) of 32 positions, then a 32 x 32
+// bit transpose across the warp gives every lane the finished word of one pixel.
+__device__ __forceinline__ void mx_epilogue_bits(const MxFin &f, uint32_t tmem_d, const int32_t *sPix, int lane, uint64_t *empty_d)
+{
+    for (int ck = f.group; ck <= f.last_chunk; ck += f.n_groups) {
+        const int c0 = ck * 32;
+        float v[32];
+        const bool full = c0 + 32 <= f.Nt;
+        if (full) tmem_ld32(tmem_d + f.lane_off + (uint32_t)c0, v);
+        else tmem_ld16(tmem_d + f.lane_off + (uint32_t)c0, v);
+        if (ck == f.last_chunk) {  // last read of the accumulator by this warp: hand it back before the arithmetic
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            mbar_arrive(empty_d);
         }
-    }
-    // the accumulator buffer has been read: hand it back before the stores
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    mbar_arrive(empty_d);
+        // bit j = (acc_j < thr): the sign of acc - thr (both are small integers held exactly);
+        // four short chains instead of one long one
+        uint32_t m0 = 0u, m1 = 0u, m2 = 0u, m3 = 0u;
 #pragma unroll
-    for (int k = 0; k < 2; ++k)
-        if (pix[k] >= 0) out[pix[k] * cow] = words[k];
+        for (int j = 7; j >= 0; --j) {
+            m0 = __funnelshift_l(__float_as_uint(v[j] - f.thr), m0, 1);
+            m1 = __funnelshift_l(__float_as_uint(v[8 + j] - f.thr), m1, 1);
+            m2 = __funnelshift_l(__float_as_uint(v[16 + j] - f.thr), m2, 1);
+            m3 = __funnelshift_l(__float_as_uint(v[24 + j] - f.thr), m3, 1);
+        }
+        uint32_t m = m0 | (m1 << 8);
+        if (full) m |= (m2 << 16) | (m3 << 24);
+        const uint32_t word = warp_transpose32(m, lane);
+        const int pix = (c0 + lane < f.Nt) ? sPix[c0 + lane] : -1;
+        if (pix >= 0) f.out_words[pix * f.cow] = word;
+    }
+    if (f.last_chunk < 0) {  // nothing to read for this warp
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        mbar_arrive(empty_d);
+    }
 }
 
 // Float / int32 output of one tile (Section 3.2: int -> float, fused activation, one multiply-add;
@@ -583,39 +619,23 @@ __device__ __forceinline__ void mx_store_chunk(const float (&v)[32], int cols, c
 }
 
 template <int MODE>
-__device__ __forceinline__ void mx_epilogue_values(const MxParams &p, uint32_t tmem_d, const int32_t *sPix, int ch0, float mult, float bias,
-                                                   int fw, int lane, uint64_t *empty_d)
+__device__ __forceinline__ void mx_epilogue_values(const MxFin &f, uint32_t tmem_d, const int32_t *sPix, int lane, uint64_t *empty_d)
 {
-    const int quarter = fw & 3, dup = p.dup, cq = quarter & (4 / dup - 1), sub = quarter / (4 / dup);  // see mx_epilogue_bits
-    const int group = (fw >> 2) * dup + sub, n_groups = kColGroups * dup;
-    const int channel = ch0 + cq * 32 + lane;
-    const int Nt = p.Nt;
-    const int64_t cout = p.Cout, cow = p.Cow;
-    const bool real = ch0 + cq * 32 < p.Cout;          // whole warp: any channel of its lanes exists
-    const bool ch_ok = channel < p.Cout;
-    const bool relu = p.activation == LCE_ACT_RELU, write_float = p.write_float != 0;
-    float *outp = static_cast<float *>(p.out) + channel;
-    const float *resp = p.residual ? p.residual + channel : nullptr;
-    uint32_t *packp = p.out_packed ? p.out_packed + (ch0 >> 5) + cq : nullptr;
-    const uint32_t lane_addr = tmem_d + ((uint32_t)(quarter * 32) << 16);
-    const int n_chunks = (Nt + 31) >> 5;               // this warp takes chunk group, group + n_groups, ...
-    if (!real || group >= n_chunks) {  // nothing to read for this warp
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        mbar_arrive(empty_d);
-        return;
-    }
-    const int last_chunk = group + ((n_chunks - 1 - group) / n_groups) * n_groups;
-    for (int ck = group; ck < n_chunks; ck += n_groups) {
+    for (int ck = f.group; ck <= f.last_chunk; ck += f.n_groups) {
         const int c0 = ck * 32;
-        const int cols = min(32, Nt - c0);
+        const int cols = min(32, f.Nt - c0);
         float v[32];
-        if (cols == 32) tmem_ld32(lane_addr + (uint32_t)c0, v);
-        else tmem_ld16(lane_addr + (uint32_t)c0, v);
-        if (ck == last_chunk) {  // last read of the accumulator by this warp
+        if (cols == 32) tmem_ld32(tmem_d + f.lane_off + (uint32_t)c0, v);
+        else tmem_ld16(tmem_d + f.lane_off + (uint32_t)c0, v);
+        if (ck == f.last_chunk) {  // last read of the accumulator by this warp
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             mbar_arrive(empty_d);
         }
-        mx_store_chunk<MODE>(v, cols, sPix + c0, cout, outp, resp, packp, cow, ch_ok, relu, write_float, mult, bias, lane);
+        mx_store_chunk<MODE>(v, cols, sPix + c0, f.cout, f.outp, f.resp, f.packp, f.cow, f.ch_ok, f.relu, f.write_float, f.mult, f.bias, lane);
+    }
+    if (f.last_chunk < 0) {  // nothing to read for this warp
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        mbar_arrive(empty_d);
     }
 }
 
@@ -762,12 +782,12 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         // ======================= finishers ============================================================
         asm volatile("griddepcontrol.wait;" ::: "memory");  // outputs and the shortcut tensor: only after the previous kernel
         const int fw = warp - kLoaders / 32;  // 0..15: lane quarter fw & 3 (= warp & 3), column group fw >> 2
+        const MxFin fin = mx_fin_context(p, fw, lane, ch0, sThr, sMult, sBias);
+        const int T = p.T, n_tiles = p.n_tiles, n_super = p.n_super;
         uint32_t par_full_d[2] = {0, 0};
-        const int my_channel = ((fw & 3) & (4 / p.dup - 1)) * 32 + lane;
-        const float my_mult = sMult[my_channel], my_bias = sBias[my_channel];
         int it = 0;
-        for (int st = first_tile; st < p.n_super && ok; st += tile_step) {
-            for (int k = 0; k < p.T && st * p.T + k < p.n_tiles; ++k, ++it) {
+        for (int st = first_tile; st < n_super && ok; st += tile_step) {
+            for (int k = 0; k < T && st * T + k < n_tiles; ++k, ++it) {
                 const int buf = it & 1;
                 ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + buf], par_full_d[buf]);
                 par_full_d[buf] ^= 1u;
@@ -776,10 +796,8 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
                 const int32_t *pix = sPix + (it & (kPixSlots - 1)) * kMaxNt;
-                if (EPI == EPI_BITS)
-                    mx_epilogue_bits(p, tmem_d, pix, ch0, sThr, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
-                else
-                    mx_epilogue_values<EPI>(p, tmem_d, pix, ch0, my_mult, my_bias, fw, lane, &bars[BAR_EMPTY_D0 + buf]);
+                if (EPI == EPI_BITS) mx_epilogue_bits(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
+                else mx_epilogue_values<EPI>(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
             }
         }
     } else if (warp == kIssuerWarp) {
@@ -1157,7 +1175,7 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const void
     p.pad_zero = g.padding == LCE_PAD_SAME_ZERO;
     p.out_type = g.out_type; p.activation = g.activation;
     p.write_float = out != nullptr;
-    p.dup = mx_dup(g);
+    p.dup_log2 = mx_dup(g) == 4 ? 2 : mx_dup(g) == 2 ? 1 : 0;
     if (!aligned(w_image, 16)) return LCE_ERR_ALIGNMENT;
     const dim3 grid((unsigned)pl.ctas_x, (unsigned)pl.n_blocks);
     if (g.out_type == LCE_OUT_BITPACKED) return launch_mx<EPI_BITS>(p, grid, pl.smem, s);

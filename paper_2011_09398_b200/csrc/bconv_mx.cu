@@ -808,15 +808,20 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         // shared-memory descriptors (units of 16 bytes): low = start | K-chunk stride << 16; high = 8-row
         // group stride (128 bytes) | version 1 at bit 46; no swizzle
         const uint32_t desc_hi = 8u | (1u << 14);
+        // everything the loops use, read from the kernel parameters once
+        const int T = p.T, n_tiles = p.n_tiles, n_super = p.n_super, Nt = p.Nt, KH = p.KH, KW = p.KW, ksteps = p.ksteps, stages = p.stages;
+        const bool resident = p.resident != 0;
+        const bool by_table = use_table && (resident || (ksteps & 3) != 0);  // streamed taps: blocks of four by arithmetic waste nothing when 4 | K steps
         const uint32_t w_lo0 = ((uint32_t)p.off_w >> 4) + (smem_u32(smem) >> 4) + (128u << 16);
-        const uint32_t tap_units = (uint32_t)p.tap_bytes >> 4;
+        const uint32_t x_lo_buf0 = ((uint32_t)p.off_x >> 4) + (smem_u32(smem) >> 4) + ((uint32_t)p.P << 16);
+        const uint32_t x_units = (uint32_t)p.x_bytes >> 4, tap_units = (uint32_t)p.tap_bytes >> 4, b_kstep = 2u * (uint32_t)p.P;
         const uint32_t sfa = tmem_base + kSfaCol, sfb = tmem_base + kSfbCol;
         uint32_t par_full_x[2] = {0, 0}, par_empty_d[2] = {0, 0};
         int g = 0, stage_i = 0;
         uint32_t w_parity = 0;
         int it = 0;
-        for (int st = first_tile, is = 0; st < p.n_super && ok; st += tile_step, ++is)
-        for (int k = 0; k < p.T && st * p.T + k < p.n_tiles && ok; ++k, ++it) {
+        for (int st = first_tile, is = 0; st < n_super && ok; st += tile_step, ++is)
+        for (int k = 0; k < T && st * T + k < n_tiles && ok; ++k, ++it) {
             const int buf = it & 1, xbuf = is & 1;
             ok = mbar_wait_bounded(&bars[BAR_FULL_X0 + buf], par_full_x[buf]);
             par_full_x[buf] ^= 1u;
@@ -829,10 +834,9 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
             // B operand: the super-tile's position buffer from this tile's first row on
-            const uint32_t x_lo0 = ((uint32_t)p.off_x >> 4) + (smem_u32(smem) >> 4) + (uint32_t)xbuf * ((uint32_t)p.x_bytes >> 4) + (uint32_t)(k * p.Nt) +
-                                   ((uint32_t)p.P << 16);
+            const uint32_t x_lo0 = x_lo_buf0 + (uint32_t)xbuf * x_units + (uint32_t)(k * Nt);
             uint32_t accumulate = 0;
-            if (p.resident) {
+            if (resident) {
                 // every tap stays in shared memory: one wait for all of them (a single barrier counts the bytes
                 // of all the copies) before the CTA's first tile, then nothing between the MMAs of a tile
                 if (it == 0) {
@@ -841,31 +845,29 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                     if (lane == 0) fills[1] = 1;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 }
-                if (use_table) {
+                if (by_table) {
                     mx_issue_table(tmem_d, tbl, n_mma, w_lo0, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
                 } else {
                     uint32_t a_tap = w_lo0;
-                    for (int ky = 0; ky < p.KH; ++ky)
-                        for (int kx = 0; kx < p.KW; ++kx, a_tap += tap_units)
-                            mx_issue(tmem_d, a_tap, x_lo0 + tap_b_offset(p, ky, kx), 256u, 2u * (uint32_t)p.P, p.ksteps, desc_hi, idesc, sfa, sfb,
-                                     accumulate);
+                    for (int ky = 0; ky < KH; ++ky)
+                        for (int kx = 0; kx < KW; ++kx, a_tap += tap_units)
+                            mx_issue(tmem_d, a_tap, x_lo0 + tap_b_offset(p, ky, kx), 256u, b_kstep, ksteps, desc_hi, idesc, sfa, sfb, accumulate);
                 }
             } else {
                 // the taps stream through the ring: wait for each, issue its MMAs, hand its stage back
-                const bool by_table = use_table && (p.ksteps & 3) != 0;  // blocks of four by arithmetic waste nothing when 4 | K steps
                 int tap = 0;
-                for (int ky = 0; ky < p.KH && ok; ++ky) {
-                    for (int kx = 0; kx < p.KW; ++kx, ++tap) {
+                for (int ky = 0; ky < KH && ok; ++ky) {
+                    for (int kx = 0; kx < KW; ++kx, ++tap) {
                         ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_FULL_W0 + stage_i], w_parity));
                         if (!ok) break;
                         ++g;
                         if (lane == 0) fills[1] = g;
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         const uint32_t a_stage = w_lo0 + (uint32_t)stage_i * tap_units;
-                        if (by_table) mx_issue_table(tmem_d, tbl + tap * p.ksteps, p.ksteps, a_stage, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
-                        else mx_issue(tmem_d, a_stage, x_lo0 + tap_b_offset(p, ky, kx), 256u, 2u * (uint32_t)p.P, p.ksteps, desc_hi, idesc, sfa, sfb, accumulate);
+                        if (by_table) mx_issue_table(tmem_d, tbl + tap * ksteps, ksteps, a_stage, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
+                        else mx_issue(tmem_d, a_stage, x_lo0 + tap_b_offset(p, ky, kx), 256u, b_kstep, ksteps, desc_hi, idesc, sfa, sfb, accumulate);
                         if (elect_one()) mma_commit(&bars[BAR_EMPTY_W0 + stage_i]);
-                        if (++stage_i == p.stages) { stage_i = 0; w_parity ^= 1u; }
+                        if (++stage_i == stages) { stage_i = 0; w_parity ^= 1u; }
                     }
                 }
             }

@@ -457,14 +457,38 @@ __device__ __forceinline__ void mx_issue_table(uint32_t tmem_d, const uint2 *tbl
     }
 }
 
-// 32 x 32 bit transpose across the warp: in: lane = row, bit j = column j; out: lane j holds column j
-__device__ __forceinline__ uint32_t warp_transpose32(uint32_t m, int lane)
+// 32 x 32 bit transpose across the warp: in: lane = row, bit j = column j; out: lane j holds column j.
+// Five butterfly steps; in step k a lane keeps the bits under its mask and takes the others from its
+// partner's word rotated by k towards them (the bits that wrap around fall under the kept mask).  The
+// per-lane masks and rotation counts are worked out once per warp: a step is one shuffle, one funnel shift
+// and one three-input logic operation.
+struct Transpose32 {
+    uint32_t keep[5];   // bits this lane keeps in the steps k = 16, 8, 4, 2, 1
+    uint32_t rot[5];    // left-rotation of the partner's word
+};
+
+__device__ __forceinline__ Transpose32 transpose32_setup(int lane)
+{
+    Transpose32 t;
+#pragma unroll
+    for (int i = 0; i < 5; ++i) {
+        const int k = 16 >> i;
+        const uint32_t low = k == 16 ? 0x0000FFFFu : k == 8 ? 0x00FF00FFu : k == 4 ? 0x0F0F0F0Fu : k == 2 ? 0x33333333u : 0x55555555u;
+        // a lane without bit k keeps its low halves and takes the partner's low halves moved up by k;
+        // a lane with bit k keeps its high halves and takes the partner's high halves moved down by k
+        t.keep[i] = (lane & k) ? ~low : low;
+        t.rot[i] = (lane & k) ? 32u - (uint32_t)k : (uint32_t)k;
+    }
+    return t;
+}
+
+__device__ __forceinline__ uint32_t warp_transpose32(uint32_t m, const Transpose32 &t)
 {
 #pragma unroll
-    for (int k = 16; k >= 1; k >>= 1) {
-        const uint32_t keep = k == 16 ? 0x0000FFFFu : k == 8 ? 0x00FF00FFu : k == 4 ? 0x0F0F0F0Fu : k == 2 ? 0x33333333u : 0x55555555u;
-        const uint32_t y = __shfl_xor_sync(0xffffffffu, m, k);
-        m = (lane & k) ? (((y >> k) & keep) | (m & ~keep)) : ((m & keep) | ((y & keep) << k));
+    for (int i = 0; i < 5; ++i) {
+        const uint32_t y = __shfl_xor_sync(0xffffffffu, m, 16 >> i);
+        const uint32_t moved = __funnelshift_l(y, y, t.rot[i]);
+        m = (m & t.keep[i]) | (moved & ~t.keep[i]);
     }
     return m;
 }
@@ -487,6 +511,7 @@ struct MxFin {
     const float *resp;       // shortcut tensor at this lane's channel, or null
     uint32_t *packp;         // re-quantised copy at this warp's channel word, or null
     bool relu, write_float;
+    Transpose32 tr;          // bit-packed output: the transpose's per-lane constants
 };
 
 __device__ __forceinline__ MxFin mx_fin_context(const MxParams &p, int fw, int lane, int ch0, const float *sThr, const float *sMult,
@@ -515,6 +540,7 @@ __device__ __forceinline__ MxFin mx_fin_context(const MxParams &p, int fw, int l
     f.packp = p.out_packed ? p.out_packed + (ch0 >> 5) + cq : nullptr;
     f.relu = p.activation == LCE_ACT_RELU;
     f.write_float = p.write_float != 0;
+    f.tr = transpose32_setup(lane);
     return f;
 }
 
@@ -545,7 +571,7 @@ __device__ __forceinline__ void mx_epilogue_bits(const MxFin &f, uint32_t tmem_d
         }
         uint32_t m = m0 | (m1 << 8);
         if (full) m |= (m2 << 16) | (m3 << 24);
-        const uint32_t word = warp_transpose32(m, lane);
+        const uint32_t word = warp_transpose32(m, f.tr);
         const int pix = (c0 + lane < f.Nt) ? sPix[c0 + lane] : -1;
         if (pix >= 0) f.out_words[pix * f.cow] = word;
     }

@@ -259,6 +259,74 @@ __device__ __forceinline__ void mx_expand(const MxGeo &p, const MxChunk &c, cons
     }
 }
 
+// The common case (stride 1, no zero-padding, 2 / 4 / 8 / 16 channel words, aligned input) with everything
+// about the words known at compile time: one asynchronous copy of 8 bytes or CW / 4 of 16 bytes per position,
+// vector reads of the staged words, no loop or branch per word.
+template <int CW>
+__device__ __forceinline__ void mx_prefetch_fast(const MxGeo &p, const MxChunk &c, uint32_t *raw, int ltid)
+{
+    for (int j = ltid; j < c.count; j += kLoaders) {
+        int64_t off;
+        const bool ok = mx_locate(p, c.q0 + c.lo, 0, j, &off);
+        const uint32_t *src = p.in + off;
+        uint32_t *dst = raw + j * CW;
+        if (CW == 2) {
+            cp_async_zfill<8>(dst, src, ok);
+        } else {
+#pragma unroll
+            for (int w = 0; w < CW; w += 4) cp_async_zfill<16>(dst + w, src + w, ok);
+        }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+template <int CW>
+__device__ __forceinline__ void mx_expand_fast(const MxGeo &p, const MxChunk &c, const uint32_t *raw, uint8_t *X, int ltid)
+{
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    for (int j = ltid; j < c.count; j += kLoaders) {
+        uint32_t w[CW];
+        if (CW == 2) {
+            const uint2 q = *reinterpret_cast<const uint2 *>(raw + j * 2);
+            w[0] = q.x; w[1] = q.y;
+        } else {
+#pragma unroll
+            for (int k = 0; k < CW; k += 4) {
+                const uint4 q = *reinterpret_cast<const uint4 *>(raw + j * CW + k);
+                w[k] = q.x; w[k + 1] = q.y; w[k + 2] = q.z; w[k + 3] = q.w;
+            }
+        }
+        uint4 *dst = reinterpret_cast<uint4 *>(X) + c.lo + j;
+#pragma unroll
+        for (int k = 0; k < CW; ++k) dst[(size_t)k * p.P] = mx_expand_word(w[k]);
+    }
+}
+
+// which form the loaders use: CW of the fast form, or 0 for the general one
+__device__ __forceinline__ int mx_fast_words(const MxGeo &p)
+{
+    const bool fast = p.n_phase == 1 && !p.pad_zero && ((p.Cw == 2 && p.cp_words >= 2) || ((p.Cw == 4 || p.Cw == 8 || p.Cw == 16) && p.cp_words == 4));
+    return fast ? p.Cw : 0;
+}
+
+__device__ __forceinline__ void mx_prefetch_any(int fw, const MxGeo &p, const MxChunk &c, uint32_t *raw, int ltid)
+{
+    if (fw == 2) mx_prefetch_fast<2>(p, c, raw, ltid);
+    else if (fw == 4) mx_prefetch_fast<4>(p, c, raw, ltid);
+    else if (fw == 8) mx_prefetch_fast<8>(p, c, raw, ltid);
+    else if (fw == 16) mx_prefetch_fast<16>(p, c, raw, ltid);
+    else mx_prefetch(p, c, raw, ltid);
+}
+
+__device__ __forceinline__ void mx_expand_any(int fw, const MxGeo &p, const MxChunk &c, const uint32_t *raw, uint8_t *X, int ltid)
+{
+    if (fw == 2) mx_expand_fast<2>(p, c, raw, X, ltid);
+    else if (fw == 4) mx_expand_fast<4>(p, c, raw, X, ltid);
+    else if (fw == 8) mx_expand_fast<8>(p, c, raw, X, ltid);
+    else if (fw == 16) mx_expand_fast<16>(p, c, raw, X, ltid);
+    else mx_expand(p, c, raw, X, ltid);
+}
+
 // B operand of tap (ky, kx): its phase buffer (stride 2) shifted by the tap's position offset, in 16-byte units
 __device__ __forceinline__ uint32_t tap_b_offset(const MxParams &p, int ky, int kx)
 {
@@ -773,7 +841,8 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         };
         uint32_t par_full_d[2] = {0, 0};
         int it = 0;
-        if (first_tile < n_super) mx_prefetch(geo, chunk_of(first_tile * T * Nt, 0), raw0, tid);
+        const int fast_words = mx_fast_words(geo);
+        if (first_tile < n_super) mx_prefetch_any(fast_words, geo, chunk_of(first_tile * T * Nt, 0), raw0, tid);
         for (int st = first_tile, is = 0; st < n_super && ok; st += tile_step, ++is) {
             const int xbuf = is & 1, q0 = st * T * Nt;
             uint8_t *X = sX0 + xbuf * x_bytes;
@@ -787,7 +856,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                     par_full_d[it & 1] ^= 1u;
                     if (!ok) break;
                 }
-                mx_expand(geo, chunk_of(q0, k), raw0 + (it & 1) * raw_words, X, tid);
+                mx_expand_any(fast_words, geo, chunk_of(q0, k), raw0 + (it & 1) * raw_words, X, tid);
                 if (tid < Nt) {
                     const int f = q0 + k * Nt + tid;
                     const int r = fast_div(f, geo.Wg_mul, geo.Wg_sh), c = f - r * geo.Wg;
@@ -799,8 +868,9 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                 mbar_arrive(&bars[BAR_FULL_X0 + (it & 1)]);
                 // only now the words of the next chunk: the MMAs of this tile must not wait for loads they do not need
                 const bool more_here = k + 1 < T && st * T + k + 1 < n_tiles;
-                if (more_here) mx_prefetch(geo, chunk_of(q0, k + 1), raw0 + ((it + 1) & 1) * raw_words, tid);
-                else if (st + tile_step < n_super) mx_prefetch(geo, chunk_of((st + tile_step) * T * Nt, 0), raw0 + ((it + 1) & 1) * raw_words, tid);
+                if (more_here || st + tile_step < n_super)
+                    mx_prefetch_any(fast_words, geo, more_here ? chunk_of(q0, k + 1) : chunk_of((st + tile_step) * T * Nt, 0),
+                                    raw0 + ((it + 1) & 1) * raw_words, tid);
             }
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");

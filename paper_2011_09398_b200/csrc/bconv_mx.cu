@@ -74,15 +74,12 @@ constexpr int kPixSlots = 8;                                 // see the note at 
 // shared-memory map (bytes)
 constexpr int kOffBars = 0;          // full_x[2] full_d[2] empty_d[2] done full_w[32] empty_w[32]
 constexpr int kOffSlot = 1000;       // TMEM base address; 1004 fills issued, 1008 fills consumed
-constexpr int kOffThr = 1024;        // float[128]
-constexpr int kOffMult = 1536;       // float[128]
-constexpr int kOffBias = 2048;       // float[128]
 // int32[8][224]: output pixel of a column, or -1.  A ring of eight tiles: the finishers hand an
 // accumulator back before they have stored its values, so the loaders can be up to four tiles ahead
 // of a finisher that still reads its tile's slot (tile t + 5 cannot be staged before finisher t is done).
-constexpr int kOffPix = 2816;
-constexpr int kOffTbl = 9984;        // uint2[512]: operand offsets (A, B; 16-byte units) of the MMAs of a tile
-constexpr int kOffDyn = 14080;       // raw words, weight ring, position buffers
+constexpr int kOffPix = 1024;
+constexpr int kOffTbl = 8192;        // uint2[512]: operand offsets (A, B; 16-byte units) of the MMAs of a tile
+constexpr int kOffDyn = 12288;      // raw words, weight ring, position buffers
 constexpr int kMaxTblMmas = 512;
 
 enum { BAR_FULL_X0 = 0, BAR_FULL_X1, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_DONE, BAR_FULL_W0,
@@ -582,8 +579,7 @@ struct MxFin {
     Transpose32 tr;          // bit-packed output: the transpose's per-lane constants
 };
 
-__device__ __forceinline__ MxFin mx_fin_context(const MxParams &p, int fw, int lane, int ch0, const float *sThr, const float *sMult,
-                                                const float *sBias)
+__device__ __forceinline__ MxFin mx_fin_context(const MxParams &p, int fw, int lane, int ch0)
 {
     MxFin f;
     const int quarter = fw & 3, dl = p.dup_log2;                    // dup = 1 << dl copies of the channel block
@@ -597,9 +593,15 @@ __device__ __forceinline__ MxFin mx_fin_context(const MxParams &p, int fw, int l
     f.last_chunk = real ? f.group + ((f.n_chunks - 1 - f.group) & ~(f.n_groups - 1)) : -1;
     f.lane_off = (uint32_t)(quarter * 32) << 16;
     f.ch_ok = channel < p.Cout;
-    f.thr = sThr[cq * 32 + lane];
-    f.mult = sMult[cq * 32 + lane];
-    f.bias = sBias[cq * 32 + lane];
+    // this lane's constants straight from global memory (constants of the model, never the previous kernel's
+    // output): their latency passes while the first tile is being staged
+    f.thr = -INFINITY;
+    if (f.ch_ok && p.out_type == LCE_OUT_BITPACKED) {
+        // acc < thr is unchanged by clamping thr to [-K-1, K+1] (|acc| <= K), and then thr is exact in fp32
+        f.thr = (float)max(-p.K - 1, min(p.K + 1, __ldg(p.thr + channel)));
+    }
+    f.mult = (f.ch_ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.mult + channel) : 0.f;
+    f.bias = (f.ch_ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.bias + channel) : 0.f;
     f.cout = p.Cout;
     f.cow = p.Cow;
     f.out_words = static_cast<uint32_t *>(p.out) + (ch0 >> 5) + cq;
@@ -742,9 +744,6 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kOffBars);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kOffSlot);
     int32_t *fills = reinterpret_cast<int32_t *>(smem + kOffSlot + 4);  // [0] issued by the producer, [1] consumed by the issuer
-    float *sThr = reinterpret_cast<float *>(smem + kOffThr);
-    float *sMult = reinterpret_cast<float *>(smem + kOffMult);
-    float *sBias = reinterpret_cast<float *>(smem + kOffBias);
     int32_t *sPix = reinterpret_cast<int32_t *>(smem + kOffPix);
     uint2 *tbl = reinterpret_cast<uint2 *>(smem + kOffTbl);
     uint32_t *raw0 = reinterpret_cast<uint32_t *>(smem + kOffDyn);
@@ -755,64 +754,48 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
     const int ch0 = blockIdx.y * 128;
     const int first_tile = blockIdx.x, tile_step = gridDim.x;
 
-    // ---- set-up (all threads) -------------------------------------------------------------------------
-    for (int e = tid; e < 128; e += kMxThreads) {
-        const bool ok = ch0 + e < p.Cout;
-        float t = -INFINITY;
-        if (ok && p.out_type == LCE_OUT_BITPACKED) {
-            // acc < thr is unchanged by clamping thr to [-K-1, K+1] (|acc| <= K), and then thr is exact in fp32
-            const int32_t ti = __ldg(p.thr + ch0 + e);
-            t = (float)max(-p.K - 1, min(p.K + 1, ti));
-        }
-        sThr[e] = t;
-        sMult[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.mult + ch0 + e) : 0.f;
-        sBias[e] = (ok && p.out_type == LCE_OUT_FLOAT32) ? __ldg(p.bias + ch0 + e) : 0.f;
-    }
+    // ---- set-up, its parts side by side: warp 0 allocates TMEM, warp 1 initialises the barriers, the
+    // finisher warps fill the table of operand offsets ------------------------------------------------------
     const int n_mma = p.taps * p.ksteps;
     const bool use_table = n_mma <= kMaxTblMmas;
-    for (int e = tid; use_table && e < n_mma; e += kMxThreads) {
-        const int tap = e / p.ksteps, kk = e - tap * p.ksteps;
-        const int ky = tap / p.KW, kx = tap - ky * p.KW;
-        // A: K step (+ the tap's ring stage when all taps are resident: stage = tap); B: the tap's offset + K step
-        const uint32_t b_off = tap_b_offset(p, ky, kx);
-        tbl[e] = make_uint2((p.resident ? (uint32_t)tap * ((uint32_t)p.tap_bytes >> 4) : 0u) + 256u * kk, b_off + 2u * (uint32_t)p.P * kk);
-    }
-    if (tid == 0) {
-        mbar_init(&bars[BAR_FULL_X0], kLoaders);
-        mbar_init(&bars[BAR_FULL_X1], kLoaders);
-        mbar_init(&bars[BAR_FULL_D0], 1);
-        mbar_init(&bars[BAR_FULL_D1], 1);
-        mbar_init(&bars[BAR_EMPTY_D0], kFinishers);
-        mbar_init(&bars[BAR_EMPTY_D1], kFinishers);
-        mbar_init(&bars[BAR_DONE], 1);
-        for (int s = 0; s < p.stages; ++s) {
-            mbar_init(&bars[BAR_FULL_W0 + s], 1);
-            mbar_init(&bars[BAR_EMPTY_W0 + s], 1);
-        }
-        fills[0] = 0;
-        fills[1] = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else if (warp == 1) {
+        for (int b = lane; b < BAR_COUNT; b += 32) {
+            const uint32_t count = b <= BAR_FULL_X1 ? kLoaders : (b == BAR_EMPTY_D0 || b == BAR_EMPTY_D1) ? kFinishers : 1;
+            mbar_init(&bars[b], count);
+        }
+        if (lane == 0) {
+            fills[0] = 0;
+            fills[1] = 0;
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    } else if (tid >= kLoaders && use_table) {
+        for (int e = tid - kLoaders; e < n_mma; e += kMxThreads - kLoaders) {
+            const int tap = e / p.ksteps, kk = e - tap * p.ksteps;
+            const int ky = tap / p.KW, kx = tap - ky * p.KW;
+            // A: K step (+ the tap's ring stage when all taps are resident: stage = tap); B: the tap's offset + K step
+            const uint32_t b_off = tap_b_offset(p, ky, kx);
+            tbl[e] = make_uint2((p.resident ? (uint32_t)tap * ((uint32_t)p.tap_bytes >> 4) : 0u) + 256u * kk, b_off + 2u * (uint32_t)p.P * kk);
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
     if (warp < 4) {
-        // block scales: every byte 0x7F = 2^0 (ue8m0), for all 128 lanes of the 32 scale columns
+        // block scales: every byte 0x7F = 2^0 (ue8m0), for all 128 lanes of the 32 scale columns.  These are
+        // loader warps: their first arrival on full_x (after the fence below) orders the writes before the
+        // first MMA, so nobody else has to wait for them here.
         const uint32_t one = 0x7F7F7F7Fu;
         const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + kSfaCol;
 #pragma unroll
         for (int c = 0; c < 32; c += 8)
             asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1};" ::"r"(taddr + c), "r"(one) : "memory");
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
     // the next kernel of the stream may start setting itself up as soon as every CTA of this one has got here
     if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -876,9 +859,9 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     } else if (tid < kLoaders + kFinishers) {
         // ======================= finishers ============================================================
-        asm volatile("griddepcontrol.wait;" ::: "memory");  // outputs and the shortcut tensor: only after the previous kernel
         const int fw = warp - kLoaders / 32;  // 0..15: lane quarter fw & 3 (= warp & 3), column group fw >> 2
-        const MxFin fin = mx_fin_context(p, fw, lane, ch0, sThr, sMult, sBias);
+        const MxFin fin = mx_fin_context(p, fw, lane, ch0);
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // outputs and the shortcut tensor: only after the previous kernel
         const int T = p.T, n_tiles = p.n_tiles, n_super = p.n_super;
         uint32_t par_full_d[2] = {0, 0};
         int it = 0;

@@ -200,6 +200,25 @@ struct MxChunk {
     uint32_t mul, sh;
 };
 
+// What the loader threads keep in registers for the whole kernel (read from the kernel parameters once).
+struct MxLoad {
+    MxGeo geo;
+    int Nt, T, halo, n_tiles, n_super, OH, OW, raw_words, fast_words;
+    uint32_t c0_mul, c0_sh, c1_mul, c1_sh;
+};
+
+// the chunk of tile k of the super-tile that starts at position q0: the first tile brings the halo
+__device__ __forceinline__ MxChunk mx_chunk_of(const MxLoad &l, int q0, int k)
+{
+    MxChunk c;
+    c.q0 = q0;
+    c.lo = k ? k * l.Nt + l.halo : 0;
+    c.count = k ? l.Nt : l.Nt + l.halo;
+    c.mul = k ? l.c1_mul : l.c0_mul;
+    c.sh = k ? l.c1_sh : l.c0_sh;
+    return c;
+}
+
 // position j of the tile that starts at q0, phase ph -> inside the image? and the pixel's word offset
 __device__ __forceinline__ bool mx_locate(const MxGeo &p, int q0, int ph, int j, int64_t *word_offset)
 {
@@ -754,6 +773,9 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
     const int ch0 = blockIdx.y * 128;
     const int first_tile = blockIdx.x, tile_step = gridDim.x;
 
+    // the next kernel of the stream may start setting itself up as soon as every CTA of this one has got here
+    if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     // ---- set-up, its parts side by side: warp 0 allocates TMEM, warp 1 initialises the barriers, the
     // finisher warps fill the table of operand offsets ------------------------------------------------------
     const int n_mma = p.taps * p.ksteps;
@@ -780,6 +802,22 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             tbl[e] = make_uint2((p.resident ? (uint32_t)tap * ((uint32_t)p.tap_bytes >> 4) : 0u) + 256u * kk, b_off + 2u * (uint32_t)p.P * kk);
         }
     }
+    // The loaders' first prefetch goes out before the CTA-wide barrier of the set-up: it needs the previous
+    // kernel's output (hence the dependency wait) and plain shared memory, nothing that is set up above.
+    MxLoad ld;
+    if (tid < kLoaders) {
+        MxGeo &geo = ld.geo;
+        geo.N = p.N; geo.H = p.H; geo.W = p.W; geo.Cw = p.Cw; geo.Cw2 = p.Cw2; geo.Wg = p.Wg; geo.Hg = p.Hg; geo.P = p.P;
+        geo.n_phase = p.n_phase; geo.stride = p.stride; geo.pt = p.pt; geo.pl = p.pl; geo.pad_zero = p.pad_zero; geo.cp_words = p.cp_words;
+        geo.Wg_mul = p.Wg_mul; geo.Wg_sh = p.Wg_sh; geo.Hg_mul = p.Hg_mul; geo.Hg_sh = p.Hg_sh;
+        geo.in = p.in;
+        ld.Nt = p.Nt; ld.T = p.T; ld.halo = p.halo; ld.n_tiles = p.n_tiles; ld.n_super = p.n_super; ld.OH = p.OH; ld.OW = p.OW;
+        ld.raw_words = p.raw_words;
+        ld.c0_mul = p.c0_mul; ld.c0_sh = p.c0_sh; ld.c1_mul = p.c1_mul; ld.c1_sh = p.c1_sh;
+        ld.fast_words = mx_fast_words(geo);
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // the activations may come from the previous kernel
+        if (first_tile < ld.n_super) mx_prefetch_any(ld.fast_words, geo, mx_chunk_of(ld, first_tile * ld.T * ld.Nt, 0), raw0, tid);
+    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -797,35 +835,16 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
 
-    // the next kernel of the stream may start setting itself up as soon as every CTA of this one has got here
-    if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     bool ok = true;
     if (tid < kLoaders) {
         // ======================= loaders ==============================================================
-        asm volatile("griddepcontrol.wait;" ::: "memory");  // the activations may come from the previous kernel
-        MxGeo geo;
-        geo.N = p.N; geo.H = p.H; geo.W = p.W; geo.Cw = p.Cw; geo.Cw2 = p.Cw2; geo.Wg = p.Wg; geo.Hg = p.Hg; geo.P = p.P;
-        geo.n_phase = p.n_phase; geo.stride = p.stride; geo.pt = p.pt; geo.pl = p.pl; geo.pad_zero = p.pad_zero; geo.cp_words = p.cp_words;
-        geo.Wg_mul = p.Wg_mul; geo.Wg_sh = p.Wg_sh; geo.Hg_mul = p.Hg_mul; geo.Hg_sh = p.Hg_sh;
-        geo.in = p.in;
-        const int Nt = p.Nt, T = p.T, halo = p.halo, n_tiles = p.n_tiles, n_super = p.n_super, OH = p.OH, OW = p.OW, raw_words = p.raw_words;
-        const uint32_t c0_mul = p.c0_mul, c0_sh = p.c0_sh, c1_mul = p.c1_mul, c1_sh = p.c1_sh;
+        const MxGeo &geo = ld.geo;
+        const int Nt = ld.Nt, T = ld.T, n_tiles = ld.n_tiles, n_super = ld.n_super, OH = ld.OH, OW = ld.OW, raw_words = ld.raw_words;
         const size_t x_bytes = (size_t)p.x_bytes;
-        // the chunk of tile k of the super-tile that starts at position q0: the first tile brings the halo
-        auto chunk_of = [&](int q0, int k) {
-            MxChunk c;
-            c.q0 = q0;
-            c.lo = k ? k * Nt + halo : 0;
-            c.count = k ? Nt : Nt + halo;
-            c.mul = k ? c1_mul : c0_mul;
-            c.sh = k ? c1_sh : c0_sh;
-            return c;
-        };
+        auto chunk_of = [&](int q0, int k) { return mx_chunk_of(ld, q0, k); };
         uint32_t par_full_d[2] = {0, 0};
         int it = 0;
-        const int fast_words = mx_fast_words(geo);
-        if (first_tile < n_super) mx_prefetch_any(fast_words, geo, chunk_of(first_tile * T * Nt, 0), raw0, tid);
         for (int st = first_tile, is = 0; st < n_super && ok; st += tile_step, ++is) {
             const int xbuf = is & 1, q0 = st * T * Nt;
             uint8_t *X = sX0 + xbuf * x_bytes;
@@ -839,7 +858,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                     par_full_d[it & 1] ^= 1u;
                     if (!ok) break;
                 }
-                mx_expand_any(fast_words, geo, chunk_of(q0, k), raw0 + (it & 1) * raw_words, X, tid);
+                mx_expand_any(ld.fast_words, geo, chunk_of(q0, k), raw0 + (it & 1) * raw_words, X, tid);
                 if (tid < Nt) {
                     const int f = q0 + k * Nt + tid;
                     const int r = fast_div(f, geo.Wg_mul, geo.Wg_sh), c = f - r * geo.Wg;
@@ -852,7 +871,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                 // only now the words of the next chunk: the MMAs of this tile must not wait for loads they do not need
                 const bool more_here = k + 1 < T && st * T + k + 1 < n_tiles;
                 if (more_here || st + tile_step < n_super)
-                    mx_prefetch_any(fast_words, geo, more_here ? chunk_of(q0, k + 1) : chunk_of((st + tile_step) * T * Nt, 0),
+                    mx_prefetch_any(ld.fast_words, geo, more_here ? chunk_of(q0, k + 1) : chunk_of((st + tile_step) * T * Nt, 0),
                                     raw0 + ((it + 1) & 1) * raw_words, tid);
             }
         }

@@ -72,7 +72,7 @@ constexpr int kMaxStages = 32;
 constexpr int kPixSlots = 8;                                 // see the note at kOffPix
 
 // shared-memory map (bytes)
-constexpr int kOffBars = 0;          // full_x[2] full_d[2] empty_d[2] done full_w[32] empty_w[32]
+constexpr int kOffBars = 0;          // full_x[2] full_d[2] empty_d[2] done scales full_w[32] empty_w[32]
 constexpr int kOffSlot = 1000;       // TMEM base address; 1004 fills issued, 1008 fills consumed
 // int32[8][224]: output pixel of a column, or -1.  A ring of eight tiles: the finishers hand an
 // accumulator back before they have stored its values, so the loaders can be up to four tiles ahead
@@ -82,7 +82,7 @@ constexpr int kOffTbl = 8192;        // uint2[512]: operand offsets (A, B; 16-by
 constexpr int kOffDyn = 12288;      // raw words, weight ring, position buffers
 constexpr int kMaxTblMmas = 512;
 
-enum { BAR_FULL_X0 = 0, BAR_FULL_X1, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_DONE, BAR_FULL_W0,
+enum { BAR_FULL_X0 = 0, BAR_FULL_X1, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_DONE, BAR_SCALES, BAR_FULL_W0,
        BAR_EMPTY_W0 = BAR_FULL_W0 + kMaxStages, BAR_COUNT = BAR_EMPTY_W0 + kMaxStages };
 static_assert(BAR_COUNT * 8 <= kOffSlot, "barriers overlap the TMEM slot");
 
@@ -776,25 +776,50 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
     // the next kernel of the stream may start setting itself up as soon as every CTA of this one has got here
     if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-    // ---- set-up, its parts side by side: warp 0 allocates TMEM, warp 1 initialises the barriers, the
-    // finisher warps fill the table of operand offsets ------------------------------------------------------
+    // ---- set-up, its parts side by side: the issuer warp allocates TMEM, the producer warp initialises the
+    // barriers and starts the weight copies, the finisher warps fill the table of operand offsets, the
+    // loaders fetch the first chunk of activations ---------------------------------------------------------
     const int n_mma = p.taps * p.ksteps;
     const bool use_table = n_mma <= kMaxTblMmas;
-    if (warp == 0) {
+    // the weight producer's progress (one thread): fills issued, ring stage and tap of the next one
+    int prod_g = 0, prod_total = 0, prod_stage = 0, prod_tap = 0;
+    uint32_t prod_parity = 1;  // the first pass over the ring waits for nothing
+    if (warp == kIssuerWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    } else if (warp == 1) {
+    } else if (warp == kIssuerWarp + 1) {
         for (int b = lane; b < BAR_COUNT; b += 32) {
-            const uint32_t count = b <= BAR_FULL_X1 ? kLoaders : (b == BAR_EMPTY_D0 || b == BAR_EMPTY_D1) ? kFinishers : 1;
+            const uint32_t count = b <= BAR_FULL_X1 ? kLoaders : (b == BAR_EMPTY_D0 || b == BAR_EMPTY_D1) ? kFinishers : b == BAR_SCALES ? 4 : 1;
             mbar_init(&bars[b], count);
         }
-        if (lane == 0) {
-            fills[0] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        __syncwarp();
+        if (tid == kProducerTid) {
+            // The weights are constants of the model: their copies start at once, whatever the previous kernel
+            // of the stream is still doing.  Resident: all taps, every copy counted on the same barrier;
+            // streamed: the first pass over the ring.
+            const uint8_t *src = p.wimg + (size_t)blockIdx.y * p.taps * p.tap_bytes;
+            if (p.resident) {
+                mbar_expect_tx(&bars[BAR_FULL_W0], (uint32_t)(p.taps * p.tap_bytes));
+                for (int tap = 0; tap < p.taps; ++tap)
+                    bulk_copy_g2s(sW + (size_t)tap * p.tap_bytes, src + (size_t)tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0]);
+                prod_g = 1;
+            } else {
+                int my_tiles = 0;
+                for (int st = first_tile; st < p.n_super; st += tile_step) my_tiles += min(p.T, p.n_tiles - st * p.T);
+                prod_total = my_tiles * p.taps;
+                for (; prod_g < min(p.stages, prod_total); ++prod_g) {
+                    mbar_expect_tx(&bars[BAR_FULL_W0 + prod_stage], (uint32_t)p.tap_bytes);
+                    bulk_copy_g2s(sW + (size_t)prod_stage * p.tap_bytes, src + (size_t)prod_tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0 + prod_stage]);
+                    if (++prod_tap == p.taps) prod_tap = 0;
+                    if (++prod_stage == p.stages) { prod_stage = 0; prod_parity ^= 1u; }
+                }
+            }
+            fills[0] = prod_g;
             fills[1] = 0;
         }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     } else if (tid >= kLoaders && use_table) {
-        for (int e = tid - kLoaders; e < n_mma; e += kMxThreads - kLoaders) {
+        for (int e = tid - kLoaders; e < n_mma; e += kFinishers) {
             const int tap = e / p.ksteps, kk = e - tap * p.ksteps;
             const int ky = tap / p.KW, kx = tap - ky * p.KW;
             // A: K step (+ the tap's ring stage when all taps are resident: stage = tap); B: the tap's offset + K step
@@ -822,19 +847,20 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
-    if (warp < 4) {
-        // block scales: every byte 0x7F = 2^0 (ue8m0), for all 128 lanes of the 32 scale columns.  These are
-        // loader warps: their first arrival on full_x (after the fence below) orders the writes before the
-        // first MMA, so nobody else has to wait for them here.
+    if (warp >= kLoaders / 32 && warp < kLoaders / 32 + 4) {
+        // block scales: every byte 0x7F = 2^0 (ue8m0), for all 128 lanes of the 32 scale columns, written by the
+        // first four finisher warps (one per lane quarter; they have nothing else to do yet); the issuer
+        // waits for the four arrivals before its first MMA
         const uint32_t one = 0x7F7F7F7Fu;
-        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + kSfaCol;
+        const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kSfaCol;
 #pragma unroll
         for (int c = 0; c < 32; c += 8)
             asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1};" ::"r"(taddr + c), "r"(one) : "memory");
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars[BAR_SCALES]);
     }
-
 
     bool ok = true;
     if (tid < kLoaders) {
@@ -915,6 +941,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         const uint32_t x_units = (uint32_t)p.x_bytes >> 4, tap_units = (uint32_t)p.tap_bytes >> 4, b_kstep = 2u * (uint32_t)p.P;
         const uint32_t sfa = tmem_base + kSfaCol, sfb = tmem_base + kSfbCol;
         uint32_t par_full_x[2] = {0, 0}, par_empty_d[2] = {0, 0};
+        ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_SCALES], 0));  // the block scales are in TMEM
         int g = 0, stage_i = 0;
         uint32_t w_parity = 0;
         int it = 0;
@@ -973,50 +1000,40 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             if (elect_one()) mma_commit(&bars[BAR_FULL_D0 + buf]);
         }
     } else if (tid == kProducerTid) {
-        // ======================= weight producer: one thread ==========================================
+        // ======================= weight producer: one thread, the rest of the streamed taps ===========
         const uint8_t *src = p.wimg + (size_t)blockIdx.y * p.taps * p.tap_bytes;
-        if (p.resident) {
-            // all taps once, every copy counted on the same barrier
-            mbar_expect_tx(&bars[BAR_FULL_W0], (uint32_t)(p.taps * p.tap_bytes));
-            for (int tap = 0; tap < p.taps; ++tap)
-                bulk_copy_g2s(sW + (size_t)tap * p.tap_bytes, src + (size_t)tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0]);
-            fills[0] = 1;
-        } else {
-            int my_tiles = 0;
-            for (int st = first_tile; st < p.n_super; st += tile_step) my_tiles += min(p.T, p.n_tiles - st * p.T);
-            const int total = my_tiles * p.taps;
-            int stage_i = 0, tap = 0;
-            uint32_t e_parity = 1;  // the first pass over the ring waits for nothing
-            for (int g = 0; g < total; ++g) {
-                if (g >= p.stages) {
-                    ok = mbar_wait_bounded(&bars[BAR_EMPTY_W0 + stage_i], e_parity);
-                    if (!ok) break;
-                }
-                mbar_expect_tx(&bars[BAR_FULL_W0 + stage_i], (uint32_t)p.tap_bytes);
-                bulk_copy_g2s(sW + (size_t)stage_i * p.tap_bytes, src + (size_t)tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0 + stage_i]);
-                fills[0] = g + 1;
-                if (++tap == p.taps) tap = 0;
-                if (++stage_i == p.stages) { stage_i = 0; e_parity ^= 1u; }
-            }
+        for (; !p.resident && prod_g < prod_total; ++prod_g) {
+            ok = mbar_wait_bounded(&bars[BAR_EMPTY_W0 + prod_stage], prod_parity);
+            if (!ok) break;
+            mbar_expect_tx(&bars[BAR_FULL_W0 + prod_stage], (uint32_t)p.tap_bytes);
+            bulk_copy_g2s(sW + (size_t)prod_stage * p.tap_bytes, src + (size_t)prod_tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0 + prod_stage]);
+            fills[0] = prod_g + 1;
+            if (++prod_tap == p.taps) prod_tap = 0;
+            if (++prod_stage == p.stages) { prod_stage = 0; prod_parity ^= 1u; }
         }
     }
     if (!ok) mx_report_timeout(p.host_flag);
 
     // ---- tear-down: nothing of this CTA may still be in flight when its TMEM and shared memory go ----
+    // When no wait gave up, the finishers have waited for the MMAs of every tile and the issuer for every
+    // weight copy; otherwise the lane that issued the MMAs waits for what is still under way.
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    if (warp == kIssuerWarp && elect_one()) {              // the lane that issued the MMAs
-        mma_commit(&bars[BAR_DONE]);                       // arrives when every MMA issued above has finished
-        bool drained = mbar_wait_bounded(&bars[BAR_DONE], 0);
-        // weight copies that were started but never consumed (only after a wait gave up)
-        const int issued = fills[0], consumed = fills[1];
-        for (int g = consumed; g < issued && drained; ++g)
-            drained = mbar_wait_bounded(&bars[BAR_FULL_W0 + g % p.stages], (uint32_t)(g / p.stages) & 1u);
-        if (!drained) mx_report_timeout(p.host_flag);
+    const bool all_ok = __syncthreads_and(ok) != 0;
+    if (!all_ok || fills[0] != fills[1]) {
+        if (warp == kIssuerWarp && elect_one()) {
+            mma_commit(&bars[BAR_DONE]);                       // arrives when every MMA issued above has finished
+            bool drained = mbar_wait_bounded(&bars[BAR_DONE], 0);
+            // weight copies that were started but never consumed
+            const int issued = fills[0], consumed = fills[1];
+            for (int g = consumed; g < issued && drained; ++g)
+                drained = mbar_wait_bounded(&bars[BAR_FULL_W0 + g % p.stages], (uint32_t)(g / p.stages) & 1u);
+            if (!drained) mx_report_timeout(p.host_flag);
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (warp == kIssuerWarp) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
 }
 
 // ---- load-time weight image -----------------------------------------------------------------------------

@@ -794,27 +794,30 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         __syncwarp();
-        if (tid == kProducerTid) {
-            // The weights are constants of the model: their copies start at once, whatever the previous kernel
-            // of the stream is still doing.  Resident: all taps, every copy counted on the same barrier;
-            // streamed: the first pass over the ring.
-            const uint8_t *src = p.wimg + (size_t)blockIdx.y * p.taps * p.tap_bytes;
-            if (p.resident) {
-                mbar_expect_tx(&bars[BAR_FULL_W0], (uint32_t)(p.taps * p.tap_bytes));
-                for (int tap = 0; tap < p.taps; ++tap)
-                    bulk_copy_g2s(sW + (size_t)tap * p.tap_bytes, src + (size_t)tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0]);
-                prod_g = 1;
-            } else {
-                int my_tiles = 0;
-                for (int st = first_tile; st < p.n_super; st += tile_step) my_tiles += min(p.T, p.n_tiles - st * p.T);
-                prod_total = my_tiles * p.taps;
-                for (; prod_g < min(p.stages, prod_total); ++prod_g) {
-                    mbar_expect_tx(&bars[BAR_FULL_W0 + prod_stage], (uint32_t)p.tap_bytes);
-                    bulk_copy_g2s(sW + (size_t)prod_stage * p.tap_bytes, src + (size_t)prod_tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0 + prod_stage]);
-                    if (++prod_tap == p.taps) prod_tap = 0;
-                    if (++prod_stage == p.stages) { prod_stage = 0; prod_parity ^= 1u; }
-                }
+        // The weights are constants of the model: their copies start at once, whatever the previous kernel of
+        // the stream is still doing, one lane per copy.  Resident: all taps, every copy counted on the same
+        // barrier; streamed: the first pass over the ring (stage = fill number; at most 32 stages).
+        const uint8_t *src = p.wimg + (size_t)blockIdx.y * p.taps * p.tap_bytes;
+        if (p.resident) {
+            if (lane == 0) mbar_expect_tx(&bars[BAR_FULL_W0], (uint32_t)(p.taps * p.tap_bytes));
+            __syncwarp();
+            for (int tap = lane; tap < p.taps; tap += 32)
+                bulk_copy_g2s(sW + (size_t)tap * p.tap_bytes, src + (size_t)tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0]);
+            prod_g = 1;
+        } else {
+            int my_tiles = 0;
+            for (int st = first_tile; st < p.n_super; st += tile_step) my_tiles += min(p.T, p.n_tiles - st * p.T);
+            prod_total = my_tiles * p.taps;
+            prod_g = min(p.stages, prod_total);
+            if (lane < prod_g) {
+                mbar_expect_tx(&bars[BAR_FULL_W0 + lane], (uint32_t)p.tap_bytes);
+                bulk_copy_g2s(sW + (size_t)lane * p.tap_bytes, src + (size_t)(lane % p.taps) * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0 + lane]);
             }
+            prod_tap = prod_g % p.taps;
+            if (prod_g == p.stages) prod_parity ^= 1u; else prod_stage = prod_g;
+        }
+        __syncwarp();
+        if (lane == 0) {
             fills[0] = prod_g;
             fills[1] = 0;
         }

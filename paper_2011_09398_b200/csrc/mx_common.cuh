@@ -55,7 +55,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, uint
         for (int i = 0; i < 64; ++i) {
             __nanosleep(nap);
             if (mbar_try_wait(bar, parity)) return true;
-            if (nap < 256) nap += nap >> 1;
+            if (nap < 64) nap += nap >> 1;
         }
     } while (globaltimer_ns() - t0 < limit_ns);
     return false;

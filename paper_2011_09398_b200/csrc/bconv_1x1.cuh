@@ -104,6 +104,10 @@ bconv1x1_kernel(const TiledParams p)
     const int lane = tid & 31, warp = tid >> 5;
     const int ch0 = blockIdx.y * kChanPerCta;
 
+    // programmatic dependent launch, as in the KxK kernel: weights before the dependency wait, everything
+    // the previous kernel may have written after it
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     if (p.w_image != nullptr) {
         const uint32_t *src = p.w_image + blockIdx.y * image_block_words(groups);
         for (int e = tid * 4; e < w_words; e += kThreads * 4) cp_async16(smem + e, src + e);
@@ -134,6 +138,7 @@ bconv1x1_kernel(const TiledParams p)
     const uint32_t w_saddr0 = (uint32_t)__cvta_generic_to_shared(sW + cg * kWGroupStride);
 
     int tile = blockIdx.x;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (tile < p.n_tiles) stage_pixels(p, tile * p.tile_pixels, min((tile + 1) * p.tile_pixels, p.M), sA0, tid);
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 0;" ::: "memory");

@@ -153,6 +153,11 @@ bconv3x3_kernel(const TiledParams p)
     const int ch0 = block_y * kChanPerCta;
     const int plane_words = p.Cw * p.plane;  // one input buffer; two of them alternate between tiles
 
+    // Programmatic dependent launch: the next kernel of the stream may be scheduled from here on; this one
+    // fetches its weights (constants of the model) and waits for the previous kernel only before it touches
+    // the activations, the shortcut tensor or its outputs.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     // ---- weights ----------------------------------------------------------------------------
     if (p.w_image != nullptr) {
         // prepared image: a plain 16-byte asynchronous copy of this channel block
@@ -212,6 +217,7 @@ bconv3x3_kernel(const TiledParams p)
 
     // ---- loop over the tiles of this CTA's range; the next tile's input rows are copied into the
     // other buffer while the current tile is computed ---------------------------------------------
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (r_begin < r_end)
         stage_rows<KS, STRIDE, NW, F32>(p, r_begin, min(r_begin + p.tile_pixels, r_end), sA0, warp, lane);
     asm volatile("cp.async.commit_group;" ::: "memory");

@@ -35,14 +35,36 @@ namespace {
 
 // ---- host side: launchers, the tile / range chooser, weight packing, plan and launch ----------------
 
+// Launch with programmatic stream serialisation: the kernel's CTAs may be scheduled while the previous
+// kernel of the stream drains; the kernel itself waits (griddepcontrol.wait) before it reads or writes
+// anything but constants of the model.
+template <typename Kernel>
+lce_status launch_dependent(Kernel kernel, dim3 grid, int threads, size_t smem_bytes, cudaStream_t s, const TiledParams &p)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(threads, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, p) != cudaSuccess) {
+        cudaGetLastError();
+        return LCE_ERR_CUDA;
+    }
+    return launch_status();
+}
+
 template <int TP>
 lce_status launch1x1(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaStream_t s)
 {
     auto kernel = bconv1x1_kernel<TP>;
     static SmemOptIn opted;
     if (!opted.ensure(kernel, smem_bytes)) return LCE_ERR_CUDA;
-    kernel<<<grid, kThreads, smem_bytes, s>>>(p);
-    return launch_status();
+    return launch_dependent(kernel, grid, kThreads, smem_bytes, s, p);
 }
 
 template <int KS, int STRIDE, int TP, int NW, bool F32 = false>
@@ -51,8 +73,7 @@ lce_status launch_kxk(const TiledParams &p, size_t smem_bytes, dim3 grid, cudaSt
     auto kernel = bconv3x3_kernel<KS, STRIDE, TP, NW, F32>;
     static SmemOptIn opted;
     if (!opted.ensure(kernel, smem_bytes)) return LCE_ERR_CUDA;
-    kernel<<<grid, 32 * NW, smem_bytes, s>>>(p);
-    return launch_status();
+    return launch_dependent(kernel, grid, 32 * NW, smem_bytes, s, p);
 }
 
 // CTAs of 128 threads that the register file lets share an SM, per pixels-per-thread variant

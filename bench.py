@@ -207,6 +207,9 @@ def load_probe():
                                    ctypes.c_void_p]
     lib.lce_probe_pipe.restype = ctypes.c_int
 
+    lib.lce_probe_stage.argtypes = [ctypes.c_int32] * 7 + [ctypes.POINTER(ctypes.c_double)] * 2 + [ctypes.c_void_p]
+    lib.lce_probe_stage.restype = ctypes.c_int
+
     def probe(mix: int, iterations: int = 2000):
         import torch
         a, b = ctypes.c_double(), ctypes.c_double()
@@ -214,7 +217,27 @@ def load_probe():
         if st != 0:
             raise RuntimeError(f"lce_probe_pipe: status {st}")
         return a.value, b.value
+
+    def stage(mode: int, batch: int, h: int, w: int, words: int, rows: int, passes: int = 20):
+        import torch
+        a, b = ctypes.c_double(), ctypes.c_double()
+        st = lib.lce_probe_stage(mode, batch, h, w, words, rows, passes, ctypes.byref(a), ctypes.byref(b),
+                                 torch.cuda.current_stream().cuda_stream)
+        if st != 0:
+            raise RuntimeError(f"lce_probe_stage: status {st}")
+        return a.value, b.value
+    probe.stage = stage
     return probe
+
+
+def staging_probe(probe, batch: int) -> dict:
+    """The three ways of staging activation tiles (4-byte async copies into word planes, 16-byte async
+    copies, one tensor-map bulk copy per tile), timed with nothing behind them on the 28x28x128 layer."""
+    names = ("cp_async_4B_word_planes", "cp_async_16B", "tensor_map_bulk_copy")
+    res = [probe.stage(mode, batch, 28, 28, 4, 7) for mode in range(3)]
+    return {"workload": f"input of the 28x28x128 layer at batch {batch} (0.8 MB), tiles of 7 + 2 rows, 2 CTAs of 256 threads per SM",
+            "whole_tensor_us": {n: r[0] for n, r in zip(names, res)},
+            "first_tile_us": {n: r[1] for n, r in zip(names, res)}}
 
 
 def measured_peaks() -> dict:
@@ -454,6 +477,7 @@ def run_lce(args):
         "frac_bitpacked_launches": rate(us_int, bit) / (probe_ops * 32), "frac_float_launches": rate(us_int, flt) / (probe_ops * 32),
         "frac_of_derived_bitpacked_launches": rate(us_int, bit) / derived,
         "traffic": profiled_traffic("bconv3x3_kernel"),
+        "staging_probe": staging_probe(probe, BATCH),
     }
     per_layer = {
         l["spec"].name: {"kernel": "tensor" if l["kernel"] == lce.KERNEL_TENSOR else "integer", "us": us_auto[j],

@@ -33,10 +33,10 @@ def test_every_declared_symbol_is_exported(lib):
     # the measurement-only companion library has a header of its own
     probe = ctypes.CDLL(str(lce_build.PROBE_LIB))
     probe_names = declared_symbols("lce_probe.h")
-    assert probe_names == ["lce_probe_pipe"]
+    assert probe_names == ["lce_probe_pipe", "lce_probe_stage"]
     for name in probe_names:
         assert hasattr(probe, name), f"{name} declared in lce_probe.h but not exported"
-    assert not hasattr(lib, "lce_probe_pipe")
+    assert not hasattr(lib, "lce_probe_pipe") and not hasattr(lib, "lce_probe_stage")
     assert {h.name for h in (ROOT / "include").glob("*.h")} == {"lce.h", "lce_probe.h"}
 
 

@@ -72,7 +72,7 @@ constexpr int kMaxStages = 32;
 constexpr int kPixSlots = 8;                                 // see the note at kOffPix
 
 // shared-memory map (bytes)
-constexpr int kOffBars = 0;          // full_x[2] full_d[2] empty_d[2] done scales full_w[32] empty_w[32]
+constexpr int kOffBars = 0;          // full_x[4] tile_done[4] full_d[2] empty_d[2] done scales full_w[32] empty_w[32]
 constexpr int kOffSlot = 1000;       // TMEM base address; 1004 fills issued, 1008 fills consumed
 // int32[8][224]: output pixel of a column, or -1.  A ring of eight tiles: the finishers hand an
 // accumulator back before they have stored its values, so the loaders can be up to four tiles ahead
@@ -82,7 +82,8 @@ constexpr int kOffTbl = 8192;        // uint2[512]: operand offsets (A, B; 16-by
 constexpr int kOffDyn = 12288;      // raw words, weight ring, position buffers
 constexpr int kMaxTblMmas = 512;
 
-enum { BAR_FULL_X0 = 0, BAR_FULL_X1, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_DONE, BAR_SCALES, BAR_FULL_W0,
+enum { BAR_FULL_X0 = 0, BAR_FULL_X3 = 3, BAR_TILE_DONE0, BAR_TILE_DONE3 = BAR_TILE_DONE0 + 3, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_DONE,
+       BAR_SCALES, BAR_FULL_W0,
        BAR_EMPTY_W0 = BAR_FULL_W0 + kMaxStages, BAR_COUNT = BAR_EMPTY_W0 + kMaxStages };
 static_assert(BAR_COUNT * 8 <= kOffSlot, "barriers overlap the TMEM slot");
 
@@ -176,6 +177,7 @@ struct MxParams {
     int32_t n_tiles, n_super, total_q;
     int32_t taps, ksteps, stages, resident;
     int32_t tap_bytes, raw_words, x_bytes;
+    int32_t n_xbuf, ahead;   // position buffers (2..4); tiles the loaders may be ahead of the finished MMAs (2..4)
     int32_t off_w, off_x;    // byte offsets in shared memory
     int32_t cp_words;        // words per cp.async: 4, 2 or 1
     int32_t pad_zero, out_type, activation, write_float;
@@ -203,7 +205,7 @@ struct MxChunk {
 // What the loader threads keep in registers for the whole kernel (read from the kernel parameters once).
 struct MxLoad {
     MxGeo geo;
-    int Nt, T, halo, n_tiles, n_super, OH, OW, raw_words, fast_words;
+    int Nt, T, halo, n_tiles, n_super, OH, OW, raw_words, fast_words, n_xbuf, ahead;
     uint32_t c0_mul, c0_sh, c1_mul, c1_sh;
 };
 
@@ -789,7 +791,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     } else if (warp == kIssuerWarp + 1) {
         for (int b = lane; b < BAR_COUNT; b += 32) {
-            const uint32_t count = b <= BAR_FULL_X1 ? kLoaders : (b == BAR_EMPTY_D0 || b == BAR_EMPTY_D1) ? kFinishers : b == BAR_SCALES ? 4 : 1;
+            const uint32_t count = b <= BAR_FULL_X3 ? kLoaders : (b == BAR_EMPTY_D0 || b == BAR_EMPTY_D1) ? kFinishers : b == BAR_SCALES ? 4 : 1;
             mbar_init(&bars[b], count);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -840,7 +842,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         geo.Wg_mul = p.Wg_mul; geo.Wg_sh = p.Wg_sh; geo.Hg_mul = p.Hg_mul; geo.Hg_sh = p.Hg_sh;
         geo.in = p.in;
         ld.Nt = p.Nt; ld.T = p.T; ld.halo = p.halo; ld.n_tiles = p.n_tiles; ld.n_super = p.n_super; ld.OH = p.OH; ld.OW = p.OW;
-        ld.raw_words = p.raw_words;
+        ld.raw_words = p.raw_words; ld.n_xbuf = p.n_xbuf; ld.ahead = p.ahead;
         ld.c0_mul = p.c0_mul; ld.c0_sh = p.c0_sh; ld.c1_mul = p.c1_mul; ld.c1_sh = p.c1_sh;
         ld.fast_words = mx_fast_words(geo);
         asm volatile("griddepcontrol.wait;" ::: "memory");  // the activations may come from the previous kernel
@@ -872,19 +874,20 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         const int Nt = ld.Nt, T = ld.T, n_tiles = ld.n_tiles, n_super = ld.n_super, OH = ld.OH, OW = ld.OW, raw_words = ld.raw_words;
         const size_t x_bytes = (size_t)p.x_bytes;
         auto chunk_of = [&](int q0, int k) { return mx_chunk_of(ld, q0, k); };
-        uint32_t par_full_d[2] = {0, 0};
-        int it = 0;
-        for (int st = first_tile, is = 0; st < n_super && ok; st += tile_step, ++is) {
-            const int xbuf = is & 1, q0 = st * T * Nt;
+        const int n_xbuf = ld.n_xbuf, ahead = ld.ahead;
+        int it = 0, xbuf = 0;
+        for (int st = first_tile; st < n_super && ok; st += tile_step, xbuf = xbuf + 1 == n_xbuf ? 0 : xbuf + 1) {
+            const int q0 = st * T * Nt;
             uint8_t *X = sX0 + xbuf * x_bytes;
             for (int k = 0; k < T && st * T + k < n_tiles; ++k, ++it) {
-                if (it >= 2) {
-                    // At most two tiles ahead of the MMAs: the MMAs of tile it - 2 are done.  That keeps the
-                    // arrivals on full_x within one phase of what the issuer has seen, and (the MMAs finish
-                    // in order) it means super-tile is - 2, whose position buffer this chunk may overwrite,
-                    // has been read completely.
-                    ok = mbar_wait_bounded(&bars[BAR_FULL_D0 + (it & 1)], par_full_d[it & 1]);
-                    par_full_d[it & 1] ^= 1u;
+                if (it >= ahead) {
+                    // At most `ahead` tiles in front of the finished MMAs: those of tile it - ahead are done (a
+                    // ring of four barriers, one commit per tile).  That keeps the arrivals on the four full_x
+                    // barriers within one phase of what the issuer has seen, and (the MMAs finish in order; ahead
+                    // <= (n_xbuf - 1) * T + 1) it means that the super-tile whose position buffer this chunk
+                    // overwrites has been read completely.
+                    const int done = it - ahead;
+                    ok = mbar_wait_bounded(&bars[BAR_TILE_DONE0 + (done & 3)], (uint32_t)(done >> 2) & 1u);
                     if (!ok) break;
                 }
                 mx_expand_any(ld.fast_words, geo, chunk_of(q0, k), raw0 + (it & 1) * raw_words, X, tid);
@@ -896,7 +899,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                     sPix[(it & (kPixSlots - 1)) * kMaxNt + tid] = col_ok ? (n * OH + rr) * OW + c : -1;
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_arrive(&bars[BAR_FULL_X0 + (it & 1)]);
+                mbar_arrive(&bars[BAR_FULL_X0 + (it & 3)]);
                 // only now the words of the next chunk: the MMAs of this tile must not wait for loads they do not need
                 const bool more_here = k + 1 < T && st * T + k + 1 < n_tiles;
                 if (more_here || st + tile_step < n_super)
@@ -943,16 +946,17 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         const uint32_t x_lo_buf0 = ((uint32_t)p.off_x >> 4) + (smem_u32(smem) >> 4) + ((uint32_t)p.P << 16);
         const uint32_t x_units = (uint32_t)p.x_bytes >> 4, tap_units = (uint32_t)p.tap_bytes >> 4, b_kstep = 2u * (uint32_t)p.P;
         const uint32_t sfa = tmem_base + kSfaCol, sfb = tmem_base + kSfbCol;
-        uint32_t par_full_x[2] = {0, 0}, par_empty_d[2] = {0, 0};
+        uint32_t par_empty_d[2] = {0, 0};
+        const int n_xbuf = p.n_xbuf;
         ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_SCALES], 0));  // the block scales are in TMEM
         int g = 0, stage_i = 0;
         uint32_t w_parity = 0;
         int it = 0;
-        for (int st = first_tile, is = 0; st < n_super && ok; st += tile_step, ++is)
+        int xbuf = 0;
+        for (int st = first_tile; st < n_super && ok; st += tile_step, xbuf = xbuf + 1 == n_xbuf ? 0 : xbuf + 1)
         for (int k = 0; k < T && st * T + k < n_tiles && ok; ++k, ++it) {
-            const int buf = it & 1, xbuf = is & 1;
-            ok = mbar_wait_bounded(&bars[BAR_FULL_X0 + buf], par_full_x[buf]);
-            par_full_x[buf] ^= 1u;
+            const int buf = it & 1;
+            ok = mbar_wait_bounded(&bars[BAR_FULL_X0 + (it & 3)], (uint32_t)(it >> 2) & 1u);
             if (ok && it >= 2) {  // the accumulator buffer must have been read out
                 ok = mbar_wait_bounded(&bars[BAR_EMPTY_D0 + buf], par_empty_d[buf]);
                 par_empty_d[buf] ^= 1u;
@@ -1000,7 +1004,10 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                 }
             }
             if (!ok) break;
-            if (elect_one()) mma_commit(&bars[BAR_FULL_D0 + buf]);
+            if (elect_one()) {
+                mma_commit(&bars[BAR_FULL_D0 + buf]);         // to the finishers: the accumulator is complete
+                mma_commit(&bars[BAR_TILE_DONE0 + (it & 3)]);  // to the loaders: the tile's operands have been read
+            }
         }
     } else if (tid == kProducerTid) {
         // ======================= weight producer: one thread, the rest of the streamed taps ===========
@@ -1076,7 +1083,7 @@ __global__ void mx_pack_weights_kernel(const uint32_t *w, uint4 *image, int Cout
 }
 
 struct MxPlan {
-    int Nt, P, T, stages, resident, n_blocks, ctas_x, n_tiles, n_super, total_q, Wg, Hg, n_phase, Cw2, taps, halo;
+    int Nt, P, T, stages, resident, n_blocks, ctas_x, n_tiles, n_super, total_q, Wg, Hg, n_phase, Cw2, taps, halo, n_xbuf, ahead;
     size_t raw_words, x_bytes, tap_bytes, off_w, off_x, smem;
 };
 
@@ -1179,7 +1186,14 @@ bool mx_plan_uncached(const ConvGeom &g, int sms, MxPlan *pl)
                 pl->raw_words = raw_words; pl->x_bytes = x_bytes;
                 pl->off_w = off_w;
                 pl->off_x = (off_w + (size_t)stages * pl->tap_bytes + 127) / 128 * 128;
-                pl->smem = pl->off_x + 2 * x_bytes;
+                // More position buffers where shared memory is left over (thin layers): the loaders may then be
+                // up to four tiles ahead, ahead <= (n_xbuf - 1) * T + 1, and the hand-overs between the roles
+                // (a few hundred clocks each) drop out of the per-tile cycle.
+                int n_xbuf = 2;
+                while (n_xbuf < 4 && (n_xbuf - 1) * T + 1 < 4 && pl->off_x + (size_t)(n_xbuf + 1) * x_bytes <= kSmemLimit) ++n_xbuf;
+                pl->n_xbuf = n_xbuf;
+                pl->ahead = min(4, (n_xbuf - 1) * T + 1);
+                pl->smem = pl->off_x + (size_t)n_xbuf * x_bytes;
             }
         }
     }
@@ -1290,6 +1304,7 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const void
     p.Nt = pl.Nt; p.P = pl.P; p.T = pl.T; p.halo = pl.halo; p.n_tiles = pl.n_tiles; p.n_super = pl.n_super; p.total_q = pl.total_q;
     p.taps = pl.taps; p.ksteps = pl.Cw2 / 2; p.stages = pl.stages; p.resident = pl.resident;
     p.tap_bytes = (int32_t)pl.tap_bytes; p.raw_words = (int32_t)pl.raw_words; p.x_bytes = (int32_t)pl.x_bytes;
+    p.n_xbuf = pl.n_xbuf; p.ahead = pl.ahead;
     p.off_w = (int32_t)pl.off_w; p.off_x = (int32_t)pl.off_x;
     p.cp_words = (g.Cw % 4 == 0 && aligned(in, 16)) ? 4 : (g.Cw % 2 == 0 && aligned(in, 8)) ? 2 : 1;
     p.pad_zero = g.padding == LCE_PAD_SAME_ZERO;

@@ -72,7 +72,7 @@ constexpr int kMaxStages = 32;
 constexpr int kPixSlots = 8;                                 // see the note at kOffPix
 
 // shared-memory map (bytes)
-constexpr int kOffBars = 0;          // full_x[4] tile_done[4] full_d[2] empty_d[2] done scales full_w[32] empty_w[32]
+constexpr int kOffBars = 0;          // full_x[4] tile_done[4] full_d[2] empty_d[2] done[2] scales full_w[32] empty_w[32]
 constexpr int kOffSlot = 1000;       // TMEM base address; 1004 fills issued, 1008 fills consumed
 // int32[8][224]: output pixel of a column, or -1.  A ring of eight tiles: the finishers hand an
 // accumulator back before they have stored its values, so the loaders can be up to four tiles ahead
@@ -82,7 +82,7 @@ constexpr int kOffTbl = 8192;        // uint2[512]: operand offsets (A, B; 16-by
 constexpr int kOffDyn = 12288;      // raw words, weight ring, position buffers
 constexpr int kMaxTblMmas = 512;
 
-enum { BAR_FULL_X0 = 0, BAR_FULL_X3 = 3, BAR_TILE_DONE0, BAR_TILE_DONE3 = BAR_TILE_DONE0 + 3, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_DONE,
+enum { BAR_FULL_X0 = 0, BAR_FULL_X3 = 3, BAR_TILE_DONE0, BAR_TILE_DONE3 = BAR_TILE_DONE0 + 3, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_DONE, BAR_DONE_B,
        BAR_SCALES, BAR_FULL_W0,
        BAR_EMPTY_W0 = BAR_FULL_W0 + kMaxStages, BAR_COUNT = BAR_EMPTY_W0 + kMaxStages };
 static_assert(BAR_COUNT * 8 <= kOffSlot, "barriers overlap the TMEM slot");
@@ -930,8 +930,12 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                 else mx_epilogue_values<EPI>(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
             }
         }
-    } else if (warp == kIssuerWarp) {
-        // ======================= MMA issuer: one warp, every lane with the same values ================
+    } else if (warp == kIssuerWarp || (warp == kIssuerWarp + 1 && p.resident != 0)) {
+        // ======================= MMA issuer: a warp, every lane with the same values ==================
+        // With the weights resident the producer warp has nothing left to do and becomes a second issuer: the
+        // two take alternate tiles (one accumulator buffer each), so that one warp's per-tile bookkeeping and
+        // waits run while the other's MMAs are in the pipe.
+        const int my_parity = warp - kIssuerWarp;
         // instruction descriptor (block-scaled kinds): A, B = e2m1 (1), both K-major, N >> 3 at bit 17,
         // scales ue8m0 (bit 23), M >> 4 at bit 24, scale-factor ids 0
         const uint32_t idesc = (1u << 7) | (1u << 10) | ((uint32_t)(p.Nt >> 3) << 17) | (1u << 23) | ((uint32_t)(128 >> 4) << 24);
@@ -956,6 +960,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         for (int st = first_tile; st < n_super && ok; st += tile_step, xbuf = xbuf + 1 == n_xbuf ? 0 : xbuf + 1)
         for (int k = 0; k < T && st * T + k < n_tiles && ok; ++k, ++it) {
             const int buf = it & 1;
+            if (resident && buf != my_parity) continue;
             ok = mbar_wait_bounded(&bars[BAR_FULL_X0 + (it & 3)], (uint32_t)(it >> 2) & 1u);
             if (ok && it >= 2) {  // the accumulator buffer must have been read out
                 ok = mbar_wait_bounded(&bars[BAR_EMPTY_D0 + buf], par_empty_d[buf]);
@@ -971,7 +976,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             if (resident) {
                 // every tap stays in shared memory: one wait for all of them (a single barrier counts the bytes
                 // of all the copies) before the CTA's first tile, then nothing between the MMAs of a tile
-                if (it == 0) {
+                if (it < 2) {  // this warp's first tile
                     ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_FULL_W0], 0));
                     if (!ok) break;
                     if (lane == 0) fills[1] = 1;
@@ -1030,12 +1035,13 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     const bool all_ok = __syncthreads_and(ok) != 0;
     if (!all_ok || fills[0] != fills[1]) {
-        if (warp == kIssuerWarp && elect_one()) {
-            mma_commit(&bars[BAR_DONE]);                       // arrives when every MMA issued above has finished
-            bool drained = mbar_wait_bounded(&bars[BAR_DONE], 0);
+        if ((warp == kIssuerWarp || (warp == kIssuerWarp + 1 && p.resident != 0)) && elect_one()) {
+            uint64_t *done = &bars[warp == kIssuerWarp ? BAR_DONE : BAR_DONE_B];
+            mma_commit(done);                                  // arrives when every MMA this lane issued has finished
+            bool drained = mbar_wait_bounded(done, 0);
             // weight copies that were started but never consumed
             const int issued = fills[0], consumed = fills[1];
-            for (int g = consumed; g < issued && drained; ++g)
+            for (int g = consumed; warp == kIssuerWarp && g < issued && drained; ++g)
                 drained = mbar_wait_bounded(&bars[BAR_FULL_W0 + g % p.stages], (uint32_t)(g / p.stages) & 1u);
             if (!drained) mx_report_timeout(p.host_flag);
         }

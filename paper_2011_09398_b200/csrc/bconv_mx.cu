@@ -24,7 +24,8 @@
 //     the same buffer shifted by the tap's position offset (K-major, no swizzle, rows 16 bytes
 //     apart), so every staged position is expanded once for all taps.  T consecutive tiles share one
 //     buffer of T * Nt + halo rows, so the halo a tile reads beyond its own positions is staged once
-//     per T tiles; there are two such buffers.
+//     per T tiles; there are two to four such buffers (as many as shared memory has room for, up to what
+//     lets the loaders run four tiles ahead).
 //   * the weights were expanded when the model was loaded (lce_bconv2d_pack_weights) into the exact
 //     operand image [channel block][tap][channel word][128 channels][16 bytes] (for out_c <= 64 the
 //     channel block is repeated down the 128 rows, so that every TMEM lane quarter holds values a
@@ -33,19 +34,20 @@
 //     per CTA, all counted on one barrier; otherwise they stream past once per tile.
 //   * roles: 8 loader warps (prefetch the packed words of the next chunk with cp.async, expand the
 //     current one), one warp that issues the MMAs (all lanes run the same code, the elected lane
-//     issues), one thread that feeds the weight ring, 16 finisher warps (tcgen05.ld, output transform,
-//     stores).  Two accumulator buffers: the expansion of tile t+1, the MMAs of tile t and the output
-//     transform of tile t-1 overlap.  The roles meet only through mbarriers; every wait is bounded by
-//     time, after which the kernel records a status, waits (bounded) for what it has in flight, frees
-//     its TMEM and returns.
+//     issues), one warp that feeds the weight ring and, once the weights are resident, issues the MMAs
+//     of every other tile, 16 finisher warps (tcgen05.ld, output transform, stores).  Two accumulator
+//     buffers: the MMAs of tile t and the output transform of tile t-1 overlap, and the loaders run up
+//     to four tiles ahead of the finished MMAs (rings of four barriers).  The roles meet only through
+//     mbarriers; every wait is bounded by time, after which the kernel records a status, waits (bounded)
+//     for what it has in flight, frees its TMEM and returns.
 //   * output transform (Section 3.2): a TMEM lane is a channel and a column a position.  Bit-packed
 //     output: the sign of (accumulator - threshold) of 32 positions per lane, then a 32 x 32 bit
 //     transpose across the warp gives each lane the finished word of one pixel.  Float / int32 output
 //     is written straight from the registers: per position a warp stores its 32 consecutive channels as
 //     one 128-byte line.
-//   * launched with programmatic stream serialization: set-up and the weight copies may overlap the
-//     tail of the previous kernel of the stream; activations, shortcut and outputs are touched only
-//     after griddepcontrol.wait.
+//   * launched with programmatic stream serialization, dependents released at kernel entry: set-up and
+//     the weight copies may overlap the tail of the previous kernel of the stream; activations, shortcut
+//     and outputs are touched only after griddepcontrol.wait.
 #include <atomic>
 #include <math.h>
 #include <mutex>

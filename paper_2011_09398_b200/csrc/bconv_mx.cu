@@ -279,18 +279,39 @@ __device__ __forceinline__ void mx_expand(const MxGeo &p, const MxChunk &c, cons
     }
 }
 
-// The common case (stride 1, no zero-padding, 2 / 4 / 8 / 16 channel words, aligned input) with everything
-// about the words known at compile time: one asynchronous copy of 8 bytes or CW / 4 of 16 bytes per position,
-// vector reads of the staged words, no loop or branch per word.
-template <int CW>
+// The common cases (no zero-padding, aligned input; stride 1 with 2 / 4 / 8 / 16 channel words, stride 2 with
+// 1 / 2 / 4 / 8) with everything about the words and the phases known at compile time: one asynchronous copy of
+// 4 or 8 bytes or CW / 4 of 16 bytes per position, vector reads of the staged words, no loop or branch per
+// word, the phase of an item by comparison instead of division.
+template <int CW, int NPH>
+__device__ __forceinline__ void mx_fast_item(const MxChunk &c, int i, int *ph, int *j)
+{
+    if (NPH == 1) {
+        *ph = 0;
+        *j = i;
+    } else {
+        const int h = i >= 2 * c.count ? 2 : 0;
+        const int r = i - h * c.count;
+        const int q = r >= c.count ? 1 : 0;
+        *ph = h + q;
+        *j = r - q * c.count;
+    }
+}
+
+template <int CW, int NPH>
 __device__ __forceinline__ void mx_prefetch_fast(const MxGeo &p, const MxChunk &c, uint32_t *raw, int ltid)
 {
-    for (int j = ltid; j < c.count; j += kLoaders) {
+    const int items = NPH * c.count;
+    for (int i = ltid; i < items; i += kLoaders) {
+        int ph, j;
+        mx_fast_item<CW, NPH>(c, i, &ph, &j);
         int64_t off;
-        const bool ok = mx_locate(p, c.q0 + c.lo, 0, j, &off);
+        const bool ok = mx_locate(p, c.q0 + c.lo, ph, j, &off);
         const uint32_t *src = p.in + off;
-        uint32_t *dst = raw + j * CW;
-        if (CW == 2) {
+        uint32_t *dst = raw + i * CW;
+        if (CW == 1) {
+            cp_async_zfill<4>(dst, src, ok);
+        } else if (CW == 2) {
             cp_async_zfill<8>(dst, src, ok);
         } else {
 #pragma unroll
@@ -300,50 +321,65 @@ __device__ __forceinline__ void mx_prefetch_fast(const MxGeo &p, const MxChunk &
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
-template <int CW>
+template <int CW, int NPH>
 __device__ __forceinline__ void mx_expand_fast(const MxGeo &p, const MxChunk &c, const uint32_t *raw, uint8_t *X, int ltid)
 {
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    for (int j = ltid; j < c.count; j += kLoaders) {
+    const int items = NPH * c.count;
+    for (int i = ltid; i < items; i += kLoaders) {
+        int ph, j;
+        mx_fast_item<CW, NPH>(c, i, &ph, &j);
         uint32_t w[CW];
-        if (CW == 2) {
-            const uint2 q = *reinterpret_cast<const uint2 *>(raw + j * 2);
+        if (CW == 1) {
+            w[0] = raw[i];
+        } else if (CW == 2) {
+            const uint2 q = *reinterpret_cast<const uint2 *>(raw + i * 2);
             w[0] = q.x; w[1] = q.y;
         } else {
 #pragma unroll
             for (int k = 0; k < CW; k += 4) {
-                const uint4 q = *reinterpret_cast<const uint4 *>(raw + j * CW + k);
+                const uint4 q = *reinterpret_cast<const uint4 *>(raw + i * CW + k);
                 w[k] = q.x; w[k + 1] = q.y; w[k + 2] = q.z; w[k + 3] = q.w;
             }
         }
-        uint4 *dst = reinterpret_cast<uint4 *>(X) + c.lo + j;
+        uint4 *dst = reinterpret_cast<uint4 *>(X) + (size_t)ph * p.Cw2 * p.P + c.lo + j;
 #pragma unroll
         for (int k = 0; k < CW; ++k) dst[(size_t)k * p.P] = mx_expand_word(w[k]);
     }
 }
 
-// which form the loaders use: CW of the fast form, or 0 for the general one
+// which form the loaders use: 0 the general one, else channel words + 32 for the stride-2 form
 __device__ __forceinline__ int mx_fast_words(const MxGeo &p)
 {
-    const bool fast = p.n_phase == 1 && !p.pad_zero && ((p.Cw == 2 && p.cp_words >= 2) || ((p.Cw == 4 || p.Cw == 8 || p.Cw == 16) && p.cp_words == 4));
-    return fast ? p.Cw : 0;
+    const bool words_ok = (p.Cw == 1) || (p.Cw == 2 && p.cp_words >= 2) || ((p.Cw == 4 || p.Cw == 8 || p.Cw == 16) && p.cp_words == 4);
+    if (p.pad_zero || !words_ok) return 0;
+    if (p.n_phase == 1) return p.Cw >= 2 ? p.Cw : 0;
+    return p.Cw <= 8 ? 32 + p.Cw : 0;
 }
 
 __device__ __forceinline__ void mx_prefetch_any(int fw, const MxGeo &p, const MxChunk &c, uint32_t *raw, int ltid)
 {
-    if (fw == 2) mx_prefetch_fast<2>(p, c, raw, ltid);
-    else if (fw == 4) mx_prefetch_fast<4>(p, c, raw, ltid);
-    else if (fw == 8) mx_prefetch_fast<8>(p, c, raw, ltid);
-    else if (fw == 16) mx_prefetch_fast<16>(p, c, raw, ltid);
+    if (fw == 2) mx_prefetch_fast<2, 1>(p, c, raw, ltid);
+    else if (fw == 4) mx_prefetch_fast<4, 1>(p, c, raw, ltid);
+    else if (fw == 8) mx_prefetch_fast<8, 1>(p, c, raw, ltid);
+    else if (fw == 16) mx_prefetch_fast<16, 1>(p, c, raw, ltid);
+    else if (fw == 33) mx_prefetch_fast<1, 4>(p, c, raw, ltid);
+    else if (fw == 34) mx_prefetch_fast<2, 4>(p, c, raw, ltid);
+    else if (fw == 36) mx_prefetch_fast<4, 4>(p, c, raw, ltid);
+    else if (fw == 40) mx_prefetch_fast<8, 4>(p, c, raw, ltid);
     else mx_prefetch(p, c, raw, ltid);
 }
 
 __device__ __forceinline__ void mx_expand_any(int fw, const MxGeo &p, const MxChunk &c, const uint32_t *raw, uint8_t *X, int ltid)
 {
-    if (fw == 2) mx_expand_fast<2>(p, c, raw, X, ltid);
-    else if (fw == 4) mx_expand_fast<4>(p, c, raw, X, ltid);
-    else if (fw == 8) mx_expand_fast<8>(p, c, raw, X, ltid);
-    else if (fw == 16) mx_expand_fast<16>(p, c, raw, X, ltid);
+    if (fw == 2) mx_expand_fast<2, 1>(p, c, raw, X, ltid);
+    else if (fw == 4) mx_expand_fast<4, 1>(p, c, raw, X, ltid);
+    else if (fw == 8) mx_expand_fast<8, 1>(p, c, raw, X, ltid);
+    else if (fw == 16) mx_expand_fast<16, 1>(p, c, raw, X, ltid);
+    else if (fw == 33) mx_expand_fast<1, 4>(p, c, raw, X, ltid);
+    else if (fw == 34) mx_expand_fast<2, 4>(p, c, raw, X, ltid);
+    else if (fw == 36) mx_expand_fast<4, 4>(p, c, raw, X, ltid);
+    else if (fw == 40) mx_expand_fast<8, 4>(p, c, raw, X, ltid);
     else mx_expand(p, c, raw, X, ltid);
 }
 

@@ -59,8 +59,8 @@ bool tiled_accepts(const ConvGeom &g, const void *out, const void *residual)
 
 // AUTO takes the tensor-core kernel when the weights were packed at load time (its operand image exists)
 // and the layer is large enough to pay for that kernel's start-up, by what was measured on the paper's
-// layer sweep and the ImageNet-shaped bodies: from 2^29 binary MACs when all taps of a channel block
-// stay in shared memory, from 2^31 when they have to stream past once per tile; 3x3 and smaller filters
+// layer sweep (batch 1 and 64) and the ImageNet-shaped bodies: from 2^28 binary MACs when all taps of a channel
+// block stay in shared memory, from 2^29 when they have to stream past once per tile; 3x3 and smaller filters
 // on at most 32 input channels stay on the integer kernels (half of every 64-deep MMA would be padding).
 bool tensor_preferred(const ConvGeom &g)
 {
@@ -69,7 +69,7 @@ bool tensor_preferred(const ConvGeom &g)
     TensorPlanInfo t{};
     if (tensor_plan_info(g, &t) != LCE_OK) return false;
     const double macs = (double)g.M * g.Cout * g.KH * g.KW * g.Cin;
-    return macs >= (t.weights_resident ? 536870912.0 : 2147483648.0);
+    return macs >= (t.weights_resident ? 268435456.0 : 536870912.0);
 }
 
 enum KernelPick { PICK_NONE = 0, PICK_DIRECT, PICK_PATCH, PICK_TILED, PICK_TENSOR };

@@ -720,54 +720,24 @@ enum { EPI_FLOAT = 0, EPI_FLOAT_FUSED = 1, EPI_INT32 = 2, EPI_BITS = 3 };
 
 template <int MODE>
 __device__ __forceinline__ void mx_store_chunk(const float (&v)[32], int cols, const int32_t *sPixChunk, int64_t cout, float *outp,
-                                               const float *resp, uint32_t *packp, int64_t cow, bool ch_ok, bool relu, bool write_float,
-                                               float mult, float bias, int lane)
+                                               bool ch_ok, float mult, float bias)
 {
-    if (MODE != EPI_FLOAT_FUSED) {
-        // straight-line code: every store is predicated, nothing branches, so the 32 positions' address
-        // arithmetic, multiply-adds and stores overlap instead of running one position after the other
+    // straight-line code: every store is predicated, nothing branches, so the 32 positions' address
+    // arithmetic, multiply-adds and stores overlap instead of running one position after the other
 #pragma unroll
-        for (int j4 = 0; j4 < 32; j4 += 4) {
-            const int4 pix4 = *reinterpret_cast<const int4 *>(sPixChunk + j4);  // the same for every lane (slots past the tile: never stored)
-            const int pix[4] = {pix4.x, pix4.y, pix4.z, pix4.w};
+    for (int j4 = 0; j4 < 32; j4 += 4) {
+        const int4 pix4 = *reinterpret_cast<const int4 *>(sPixChunk + j4);  // the same for every lane (slots past the tile: never stored)
+        const int pix[4] = {pix4.x, pix4.y, pix4.z, pix4.w};
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const bool st = ch_ok && pix[u] >= 0 && j4 + u < cols;
-                const int64_t o = pix[u] * cout;
-                if (MODE == EPI_FLOAT) {
-                    const float y = __fmaf_rn(v[j4 + u], mult, bias);
-                    if (st) outp[o] = y;
-                } else {
-                    const int32_t y = __float2int_rn(v[j4 + u]);
-                    if (st) reinterpret_cast<int32_t *>(outp)[o] = y;
-                }
-            }
-        }
-        return;
-    }
-    // Eight positions at a time: first all their shortcut values are requested (eight independent 128-byte
-    // loads in flight; one position after the other would pay the memory latency 32 times per chunk), then
-    // the arithmetic, the stores and the ballots.
-    const float floor_v = relu ? 0.f : -INFINITY;
-#pragma unroll
-    for (int j8 = 0; j8 < 32; j8 += 8) {
-        const int4 pa = *reinterpret_cast<const int4 *>(sPixChunk + j8), pb = *reinterpret_cast<const int4 *>(sPixChunk + j8 + 4);  // the same for every lane
-        const int pix[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
-        float r[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            r[u] = 0.f;
-            if (resp != nullptr && ch_ok && pix[u] >= 0 && j8 + u < cols) r[u] = __ldg(resp + pix[u] * cout);
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const bool pos_ok = pix[u] >= 0 && j8 + u < cols;   // the same for every lane
-            float y = __fmaf_rn(fmaxf(v[j8 + u], floor_v), mult, bias);
-            if (resp != nullptr) y = __fadd_rn(y, r[u]);
-            if (write_float && ch_ok && pos_ok) outp[pix[u] * cout] = y;
-            if (packp != nullptr) {
-                const uint32_t word = __ballot_sync(0xffffffffu, ch_ok && y < 0.f);
-                if (lane == 0 && pos_ok) packp[pix[u] * cow] = word;
+        for (int u = 0; u < 4; ++u) {
+            const bool st = ch_ok && pix[u] >= 0 && j4 + u < cols;
+            const int64_t o = pix[u] * cout;
+            if (MODE != EPI_INT32) {
+                const float y = __fmaf_rn(v[j4 + u], mult, bias);
+                if (st) outp[o] = y;
+            } else {
+                const int32_t y = __float2int_rn(v[j4 + u]);
+                if (st) reinterpret_cast<int32_t *>(outp)[o] = y;
             }
         }
     }
@@ -786,7 +756,64 @@ __device__ __forceinline__ void mx_epilogue_values(const MxFin &f, uint32_t tmem
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             mbar_arrive(empty_d);
         }
-        mx_store_chunk<MODE>(v, cols, sPix + c0, f.cout, f.outp, f.resp, f.packp, f.cow, f.ch_ok, f.relu, f.write_float, f.mult, f.bias, lane);
+        mx_store_chunk<MODE>(v, cols, sPix + c0, f.cout, f.outp, f.ch_ok, f.mult, f.bias);
+    }
+    if (f.last_chunk < 0) {  // nothing to read for this warp
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        mbar_arrive(empty_d);
+    }
+}
+
+// Float output with the shortcut add and the re-quantised copy fused in (Section 5.3).  Per 32-column chunk
+// the warp first asks for the shortcut values of all 32 positions (they do not depend on the accumulator:
+// 32 independent 128-byte loads in flight per warp; with eight the memory latency set the pace), then reads
+// the accumulators 16 columns at a time, and per position does the multiply-add, the add, the 128-byte store
+// and the ballot whose result is the pixel's finished word.
+__device__ __forceinline__ void mx_epilogue_fused(const MxFin &f, uint32_t tmem_d, const int32_t *sPix, int lane, uint64_t *empty_d)
+{
+    const float floor_v = f.relu ? 0.f : -INFINITY;
+    for (int ck = f.group; ck <= f.last_chunk; ck += f.n_groups) {
+        const int c0 = ck * 32;
+        const int cols = min(32, f.Nt - c0);  // 32, or 16 in a tile's last chunk
+        const int32_t *pixc = sPix + c0;
+        float r[32];
+#pragma unroll
+        for (int j4 = 0; j4 < 32; j4 += 4) {
+            const int4 p4 = *reinterpret_cast<const int4 *>(pixc + j4);  // the same for every lane
+            const int pix[4] = {p4.x, p4.y, p4.z, p4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                r[j4 + u] = 0.f;
+                if (f.resp != nullptr && f.ch_ok && pix[u] >= 0 && j4 + u < cols) r[j4 + u] = __ldg(f.resp + pix[u] * f.cout);
+            }
+        }
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            if (half * 16 < cols) {
+                float v[16];
+                tmem_ld16x(tmem_d + f.lane_off + (uint32_t)(c0 + half * 16), v);
+                if (ck == f.last_chunk && (half + 1) * 16 >= cols) {  // last read of the accumulator by this warp
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    mbar_arrive(empty_d);
+                }
+#pragma unroll
+                for (int j4 = 0; j4 < 16; j4 += 4) {
+                    const int4 p4 = *reinterpret_cast<const int4 *>(pixc + half * 16 + j4);
+                    const int pix[4] = {p4.x, p4.y, p4.z, p4.w};
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const bool pos_ok = pix[u] >= 0 && half * 16 + j4 + u < cols;  // the same for every lane
+                        float y = __fmaf_rn(fmaxf(v[j4 + u], floor_v), f.mult, f.bias);
+                        if (f.resp != nullptr) y = __fadd_rn(y, r[half * 16 + j4 + u]);
+                        if (f.write_float && f.ch_ok && pos_ok) f.outp[pix[u] * f.cout] = y;
+                        if (f.packp != nullptr) {
+                            const uint32_t word = __ballot_sync(0xffffffffu, f.ch_ok && y < 0.f);
+                            if (lane == 0 && pos_ok) f.packp[pix[u] * f.cow] = word;
+                        }
+                    }
+                }
+            }
+        }
     }
     if (f.last_chunk < 0) {  // nothing to read for this warp
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -965,6 +992,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                 const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
                 const int32_t *pix = sPix + (it & (kPixSlots - 1)) * kMaxNt;
                 if (EPI == EPI_BITS) mx_epilogue_bits(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
+                else if (EPI == EPI_FLOAT_FUSED) mx_epilogue_fused(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
                 else mx_epilogue_values<EPI>(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
             }
         }

@@ -65,7 +65,7 @@ typedef enum { LCE_ACT_NONE = 0, LCE_ACT_RELU = 1 } lce_activation;
  *          padding mode and output type.  Needs weights packed by lce_bconv2d_pack_weights;
  *   DIRECT one thread per output, any shape (fallback, not tuned);
  *   AUTO   TENSOR when the weights are packed and the layer is large enough to pay for that kernel's
- *          start-up (at least 2^28 binary MACs, 2^29 when the filter does not fit in shared memory; not
+ *          start-up (at least 2^28 binary MACs, 2^29 when the filter does not fit in shared memory, 2^31
  *          for 3x3 or smaller filters on at most 32 input channels), otherwise TILED where it covers the
  *          shape, otherwise DIRECT.  lce_bconv2d_plan tells which.
  * Forcing a kernel on a shape (or on plain weights) it does not cover returns LCE_ERR_UNSUPPORTED. */

@@ -61,14 +61,15 @@ bool tiled_accepts(const ConvGeom &g, const void *out, const void *residual)
 // and the layer is large enough to pay for that kernel's start-up, by what was measured on the paper's
 // layer sweep (batch 1 and 64) and the ImageNet-shaped bodies: from 2^28 binary MACs when all taps of a channel
 // block stay in shared memory, from 2^29 when they have to stream past once per tile; 3x3 and smaller filters
-// on at most 32 input channels stay on the integer kernels (half of every 64-deep MMA would be padding).
+// on at most 32 input channels (half of every 64-deep MMA is padding) only from 2^31, where the two kernels
+// draw level (the 112x112x32 stride-2 layer of an ImageNet stem, 2^34 MACs, is twice as fast on the tensor cores).
 bool tensor_preferred(const ConvGeom &g)
 {
     if (patch_covers(g)) return false;
-    if (g.Cin <= 32 && g.KH * g.KW <= 9) return false;
     TensorPlanInfo t{};
     if (tensor_plan_info(g, &t) != LCE_OK) return false;
     const double macs = (double)g.M * g.Cout * g.KH * g.KW * g.Cin;
+    if (g.Cin <= 32 && g.KH * g.KW <= 9) return macs >= 2147483648.0;
     return macs >= (t.weights_resident ? 268435456.0 : 536870912.0);
 }
 

@@ -348,13 +348,67 @@ __device__ __forceinline__ void mx_expand_fast(const MxGeo &p, const MxChunk &c,
     }
 }
 
-// which form the loaders use: 0 the general one, else channel words + 32 for the stride-2 form
+// Stride 2 with an even image width and an even left pad: the pixels of the column phases 0 and 1 of a grid
+// position are neighbours in memory, so one item is a row phase and a position, one copy of 2 CW words brings
+// both column phases, and the address arithmetic is done once for the two.
+template <int CW>
+__device__ __forceinline__ void mx_prefetch_pair(const MxGeo &p, const MxChunk &c, uint32_t *raw, int ltid)
+{
+    const int items = 2 * c.count;
+    for (int i = ltid; i < items; i += kLoaders) {
+        const int py = i >= c.count ? 1 : 0, j = i - py * c.count;
+        int64_t off;
+        const bool ok = mx_locate(p, c.q0 + c.lo, 2 * py, j, &off);  // column phase 0; phase 1 is the next pixel, inside with it
+        const uint32_t *src = p.in + off;
+        uint32_t *dst = raw + i * 2 * CW;
+        if (CW == 1) {
+            cp_async_zfill<8>(dst, src, ok);
+        } else {
+#pragma unroll
+            for (int w = 0; w < 2 * CW; w += 4) cp_async_zfill<16>(dst + w, src + w, ok);
+        }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+template <int CW>
+__device__ __forceinline__ void mx_expand_pair(const MxGeo &p, const MxChunk &c, const uint32_t *raw, uint8_t *X, int ltid)
+{
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    const int items = 2 * c.count;
+    for (int i = ltid; i < items; i += kLoaders) {
+        const int py = i >= c.count ? 1 : 0, j = i - py * c.count;
+        uint32_t w[2 * CW];
+        if (CW == 1) {
+            const uint2 q = *reinterpret_cast<const uint2 *>(raw + i * 2);
+            w[0] = q.x; w[1] = q.y;
+        } else {
+#pragma unroll
+            for (int k = 0; k < 2 * CW; k += 4) {
+                const uint4 q = *reinterpret_cast<const uint4 *>(raw + i * 2 * CW + k);
+                w[k] = q.x; w[k + 1] = q.y; w[k + 2] = q.z; w[k + 3] = q.w;
+            }
+        }
+        uint4 *dst0 = reinterpret_cast<uint4 *>(X) + (size_t)(2 * py) * p.Cw2 * p.P + c.lo + j;  // column phase 0
+        uint4 *dst1 = dst0 + (size_t)p.Cw2 * p.P;                                                 // column phase 1
+#pragma unroll
+        for (int k = 0; k < CW; ++k) {
+            dst0[(size_t)k * p.P] = mx_expand_word(w[k]);
+            dst1[(size_t)k * p.P] = mx_expand_word(w[CW + k]);
+        }
+    }
+}
+
+// which form the loaders use: 0 the general one, else channel words (+ 32 for the stride-2 form, + 64 for the
+// stride-2 form that copies the two column phases together)
 __device__ __forceinline__ int mx_fast_words(const MxGeo &p)
 {
     const bool words_ok = (p.Cw == 1) || (p.Cw == 2 && p.cp_words >= 2) || ((p.Cw == 4 || p.Cw == 8 || p.Cw == 16) && p.cp_words == 4);
     if (p.pad_zero || !words_ok) return 0;
     if (p.n_phase == 1) return p.Cw >= 2 ? p.Cw : 0;
-    return p.Cw <= 8 ? 32 + p.Cw : 0;
+    if (p.Cw > 8) return 0;
+    const bool pairs = (p.W & 1) == 0 && (p.pl & 1) == 0 && (reinterpret_cast<uintptr_t>(p.in) & 15) == 0 && p.Cw <= 4;
+    return (pairs ? 64 : 32) + p.Cw;
 }
 
 __device__ __forceinline__ void mx_prefetch_any(int fw, const MxGeo &p, const MxChunk &c, uint32_t *raw, int ltid)
@@ -367,6 +421,9 @@ __device__ __forceinline__ void mx_prefetch_any(int fw, const MxGeo &p, const Mx
     else if (fw == 34) mx_prefetch_fast<2, 4>(p, c, raw, ltid);
     else if (fw == 36) mx_prefetch_fast<4, 4>(p, c, raw, ltid);
     else if (fw == 40) mx_prefetch_fast<8, 4>(p, c, raw, ltid);
+    else if (fw == 65) mx_prefetch_pair<1>(p, c, raw, ltid);
+    else if (fw == 66) mx_prefetch_pair<2>(p, c, raw, ltid);
+    else if (fw == 68) mx_prefetch_pair<4>(p, c, raw, ltid);
     else mx_prefetch(p, c, raw, ltid);
 }
 
@@ -380,6 +437,9 @@ __device__ __forceinline__ void mx_expand_any(int fw, const MxGeo &p, const MxCh
     else if (fw == 34) mx_expand_fast<2, 4>(p, c, raw, X, ltid);
     else if (fw == 36) mx_expand_fast<4, 4>(p, c, raw, X, ltid);
     else if (fw == 40) mx_expand_fast<8, 4>(p, c, raw, X, ltid);
+    else if (fw == 65) mx_expand_pair<1>(p, c, raw, X, ltid);
+    else if (fw == 66) mx_expand_pair<2>(p, c, raw, X, ltid);
+    else if (fw == 68) mx_expand_pair<4>(p, c, raw, X, ltid);
     else mx_expand(p, c, raw, X, ltid);
 }
 
@@ -1244,11 +1304,17 @@ bool mx_plan_uncached(const ConvGeom &g, int sms, MxPlan *pl)
             const int n_super = (n_tiles + T - 1) / T;
             const int ctas_x = min(ctas_max, n_super);
             const int per_cta = ((n_super + ctas_x - 1) / ctas_x) * T;
-            // clocks per MMA: 43 + N/2, at least 100 (measured); streamed weights cost about as much again from
-            // L2; the loaders need about 400 + 8 clocks per staged position and tile
-            const double mma = (double)taps * ksteps * fmax(100.0, 43.0 + nt / 2.0);
-            const double stream = resident ? 0.0 : (double)taps * pl->tap_bytes / 48.0;
-            const double load = 400.0 + 8.0 * pl->n_phase * (nt + (double)halo / T);
+            // clocks per MMA: 43 + N/2, at least 100 (measured); the loaders need about 400 + 8 clocks per staged
+            // position and tile
+            const double mma1 = fmax(100.0, 43.0 + nt / 2.0);
+            const double mma = (double)taps * ksteps * mma1;
+            // a streamed tap: its bytes from L2, or its share of a copy's latency, or what the single issuer needs
+            // per tap (wait for the stage, issue, hand the stage back: about 600 clocks on top of the MMAs;
+            // measured on a nine-tap, one-MMA-per-tap layer: 6000 clocks per tile whether 2 or 4 stages)
+            const double stream = resident ? 0.0 : (double)taps * fmax(fmax(pl->tap_bytes / 48.0, 1300.0 / stages), 600.0 + ksteps * mma1);
+            // stride 2: four phases per position, staged two at a time where the geometry allows (mx_prefetch_pair)
+            const double per_position = s == 1 ? 1.0 : ((g.W & 1) == 0 && (g.pl & 1) == 0 && g.Cw <= 4) ? 2.0 : 3.0;
+            const double load = 400.0 + 8.0 * per_position * (nt + (double)halo / T);
             const double cost = per_cta * (fmax(fmax(mma, stream), load) + 150.0);
             if (cost < best) {
                 best = cost;

@@ -173,7 +173,8 @@ def test_tensor_plan_fits_the_sm_and_auto_takes_it_for_large_packed_layers(lib, 
     auto, M = _plan(*shape, out_type=out_type, packed=1)
     macs = M * shape[4] * k * k * shape[3]
     few_channels = shape[3] <= 32 and k * k <= 9
-    assert (auto["kernel"] == lce.KERNEL_TENSOR) == (not few_channels and macs >= (2 ** 28 if forced["weights_resident"] else 2 ** 29))
+    threshold = 2 ** 31 if few_channels else 2 ** 28 if forced["weights_resident"] else 2 ** 29
+    assert (auto["kernel"] == lce.KERNEL_TENSOR) == (macs >= threshold)
     assert _plan(*shape, out_type=out_type)[0]["kernel"] != lce.KERNEL_TENSOR             # plain weights: integer kernels
 
 

@@ -178,6 +178,7 @@ struct MxParams {
     int32_t T, halo;         // tiles that share a position buffer; positions a tile reads beyond its own
     int32_t n_tiles, n_super, total_q;
     int32_t taps, ksteps, stages, resident;
+    int32_t group_taps, groups;  // streamed weights: taps per ring stage, stages' worth of taps per tile = ceil(taps / group_taps)
     int32_t tap_bytes, raw_words, x_bytes;
     int32_t n_xbuf, ahead;   // position buffers (2..4); tiles the loaders may be ahead of the finished MMAs (2..4)
     int32_t off_w, off_x;    // byte offsets in shared memory
@@ -908,7 +909,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
     // loaders fetch the first chunk of activations ---------------------------------------------------------
     const int n_mma = p.taps * p.ksteps;
     const bool use_table = n_mma <= kMaxTblMmas;
-    // the weight producer's progress (one thread): fills issued, ring stage and tap of the next one
+    // the weight producer's progress (one thread): fills issued, ring stage and (tile-local) tap group of the next one
     int prod_g = 0, prod_total = 0, prod_stage = 0, prod_tap = 0;
     uint32_t prod_parity = 1;  // the first pass over the ring waits for nothing
     if (warp == kIssuerWarp) {
@@ -934,13 +935,16 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         } else {
             int my_tiles = 0;
             for (int st = first_tile; st < p.n_super; st += tile_step) my_tiles += min(p.T, p.n_tiles - st * p.T);
-            prod_total = my_tiles * p.taps;
+            // a fill = one group of up to group_taps consecutive taps (one copy: they are contiguous in the image)
+            prod_total = my_tiles * p.groups;
             prod_g = min(p.stages, prod_total);
             if (lane < prod_g) {
-                mbar_expect_tx(&bars[BAR_FULL_W0 + lane], (uint32_t)p.tap_bytes);
-                bulk_copy_g2s(sW + (size_t)lane * p.tap_bytes, src + (size_t)(lane % p.taps) * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0 + lane]);
+                const int first = (lane % p.groups) * p.group_taps;
+                const uint32_t bytes = (uint32_t)(min(p.group_taps, p.taps - first) * p.tap_bytes);
+                mbar_expect_tx(&bars[BAR_FULL_W0 + lane], bytes);
+                bulk_copy_g2s(sW + (size_t)lane * p.group_taps * p.tap_bytes, src + (size_t)first * p.tap_bytes, bytes, &bars[BAR_FULL_W0 + lane]);
             }
-            prod_tap = prod_g % p.taps;
+            prod_tap = prod_g % p.groups;   // the next fill's group within its tile
             if (prod_g == p.stages) prod_parity ^= 1u; else prod_stage = prod_g;
         }
         __syncwarp();
@@ -1069,12 +1073,13 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         // group stride (128 bytes) | version 1 at bit 46; no swizzle
         const uint32_t desc_hi = 8u | (1u << 14);
         // everything the loops use, read from the kernel parameters once
-        const int T = p.T, n_tiles = p.n_tiles, n_super = p.n_super, Nt = p.Nt, KH = p.KH, KW = p.KW, ksteps = p.ksteps, stages = p.stages;
+        const int T = p.T, n_tiles = p.n_tiles, n_super = p.n_super, Nt = p.Nt, KH = p.KH, KW = p.KW, ksteps = p.ksteps, stages = p.stages, taps = p.taps, group_taps = p.group_taps;
         const bool resident = p.resident != 0;
         const bool by_table = use_table && (resident || (ksteps & 3) != 0);  // streamed taps: blocks of four by arithmetic waste nothing when 4 | K steps
         const uint32_t w_lo0 = ((uint32_t)p.off_w >> 4) + (smem_u32(smem) >> 4) + (128u << 16);
         const uint32_t x_lo_buf0 = ((uint32_t)p.off_x >> 4) + (smem_u32(smem) >> 4) + ((uint32_t)p.P << 16);
         const uint32_t x_units = (uint32_t)p.x_bytes >> 4, tap_units = (uint32_t)p.tap_bytes >> 4, b_kstep = 2u * (uint32_t)p.P;
+        const uint32_t group_units = tap_units * (uint32_t)p.group_taps;
         const uint32_t sfa = tmem_base + kSfaCol, sfb = tmem_base + kSfbCol;
         uint32_t par_empty_d[2] = {0, 0};
         const int n_xbuf = p.n_xbuf;
@@ -1117,21 +1122,25 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                             mx_issue(tmem_d, a_tap, x_lo0 + tap_b_offset(p, ky, kx), 256u, b_kstep, ksteps, desc_hi, idesc, sfa, sfb, accumulate);
                 }
             } else {
-                // the taps stream through the ring: wait for each, issue its MMAs, hand its stage back
-                int tap = 0;
-                for (int ky = 0; ky < KH && ok; ++ky) {
-                    for (int kx = 0; kx < KW; ++kx, ++tap) {
-                        ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_FULL_W0 + stage_i], w_parity));
-                        if (!ok) break;
-                        ++g;
-                        if (lane == 0) fills[1] = g;
-                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        const uint32_t a_stage = w_lo0 + (uint32_t)stage_i * tap_units;
-                        if (by_table) mx_issue_table(tmem_d, tbl + tap * ksteps, ksteps, a_stage, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
-                        else mx_issue(tmem_d, a_stage, x_lo0 + tap_b_offset(p, ky, kx), 256u, b_kstep, ksteps, desc_hi, idesc, sfa, sfb, accumulate);
-                        if (elect_one()) mma_commit(&bars[BAR_EMPTY_W0 + stage_i]);
-                        if (++stage_i == stages) { stage_i = 0; w_parity ^= 1u; }
+                // the taps stream through the ring a group at a time: wait for the group, issue its taps' MMAs,
+                // hand its stage back (the wait, the commit and the bookkeeping cost this warp about 600 clocks,
+                // as much as six MMAs: hence groups, not single taps)
+                int tap = 0, ky = 0, kx = 0;
+                while (tap < taps) {
+                    ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_FULL_W0 + stage_i], w_parity));
+                    if (!ok) break;
+                    ++g;
+                    if (lane == 0) fills[1] = g;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    uint32_t a_tap = w_lo0 + (uint32_t)stage_i * group_units;
+                    const int group_end = min(taps, tap + group_taps);
+                    for (; tap < group_end; ++tap, a_tap += tap_units) {
+                        if (by_table) mx_issue_table(tmem_d, tbl + tap * ksteps, ksteps, a_tap, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
+                        else mx_issue(tmem_d, a_tap, x_lo0 + tap_b_offset(p, ky, kx), 256u, b_kstep, ksteps, desc_hi, idesc, sfa, sfb, accumulate);
+                        if (++kx == KW) { kx = 0; ++ky; }
                     }
+                    if (elect_one()) mma_commit(&bars[BAR_EMPTY_W0 + stage_i]);
+                    if (++stage_i == stages) { stage_i = 0; w_parity ^= 1u; }
                 }
             }
             if (!ok) break;
@@ -1146,10 +1155,12 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         for (; !p.resident && prod_g < prod_total; ++prod_g) {
             ok = mbar_wait_bounded(&bars[BAR_EMPTY_W0 + prod_stage], prod_parity);
             if (!ok) break;
-            mbar_expect_tx(&bars[BAR_FULL_W0 + prod_stage], (uint32_t)p.tap_bytes);
-            bulk_copy_g2s(sW + (size_t)prod_stage * p.tap_bytes, src + (size_t)prod_tap * p.tap_bytes, (uint32_t)p.tap_bytes, &bars[BAR_FULL_W0 + prod_stage]);
+            const int first = prod_tap * p.group_taps;
+            const uint32_t bytes = (uint32_t)(min(p.group_taps, p.taps - first) * p.tap_bytes);
+            mbar_expect_tx(&bars[BAR_FULL_W0 + prod_stage], bytes);
+            bulk_copy_g2s(sW + (size_t)prod_stage * p.group_taps * p.tap_bytes, src + (size_t)first * p.tap_bytes, bytes, &bars[BAR_FULL_W0 + prod_stage]);
             fills[0] = prod_g + 1;
-            if (++prod_tap == p.taps) prod_tap = 0;
+            if (++prod_tap == p.groups) prod_tap = 0;
             if (++prod_stage == p.stages) { prod_stage = 0; prod_parity ^= 1u; }
         }
     }
@@ -1215,7 +1226,7 @@ __global__ void mx_pack_weights_kernel(const uint32_t *w, uint4 *image, int Cout
 }
 
 struct MxPlan {
-    int Nt, P, T, stages, resident, n_blocks, ctas_x, n_tiles, n_super, total_q, Wg, Hg, n_phase, Cw2, taps, halo, n_xbuf, ahead;
+    int Nt, P, T, stages, resident, group_taps, groups, n_blocks, ctas_x, n_tiles, n_super, total_q, Wg, Hg, n_phase, Cw2, taps, halo, n_xbuf, ahead;
     size_t raw_words, x_bytes, tap_bytes, off_w, off_x, smem;
 };
 
@@ -1297,10 +1308,20 @@ bool mx_plan_uncached(const ConvGeom &g, int sms, MxPlan *pl)
             const size_t off_w = (fixed + 127) / 128 * 128;
             const size_t rest = 2 * x_bytes + 256;
             if (off_w + rest + (taps > 1 ? 2 : 1) * pl->tap_bytes > kSmemLimit) break;
-            int stages = (int)((kSmemLimit - off_w - rest) / pl->tap_bytes);
-            if (stages > kMaxStages) stages = kMaxStages;
-            const bool resident = stages >= taps;
-            if (resident) stages = taps;
+            // taps that fit beside the position buffers: all of them -> resident (one stage per tap, one barrier);
+            // otherwise a ring of about three stages of several taps each (a group costs the issuer one wait and
+            // one commit, whatever its size)
+            const int slots = (int)((kSmemLimit - off_w - rest) / pl->tap_bytes);
+            const bool resident = slots >= taps;
+            int stages, group_taps, groups;
+            if (resident) {
+                stages = taps; group_taps = 1; groups = taps;
+            } else {
+                group_taps = slots >= 6 ? slots / 3 : 1;
+                groups = (taps + group_taps - 1) / group_taps;
+                group_taps = (taps + groups - 1) / groups;  // even groups
+                stages = min(kMaxStages, slots / group_taps);
+            }
             const int n_super = (n_tiles + T - 1) / T;
             const int ctas_x = min(ctas_max, n_super);
             const int per_cta = ((n_super + ctas_x - 1) / ctas_x) * T;
@@ -1311,7 +1332,7 @@ bool mx_plan_uncached(const ConvGeom &g, int sms, MxPlan *pl)
             // a streamed tap: its bytes from L2, or its share of a copy's latency, or what the single issuer needs
             // per tap (wait for the stage, issue, hand the stage back: about 600 clocks on top of the MMAs;
             // measured on a nine-tap, one-MMA-per-tap layer: 6000 clocks per tile whether 2 or 4 stages)
-            const double stream = resident ? 0.0 : (double)taps * fmax(fmax(pl->tap_bytes / 48.0, 1300.0 / stages), 600.0 + ksteps * mma1);
+            const double stream = resident ? 0.0 : (double)groups * fmax(fmax(group_taps * pl->tap_bytes / 48.0, 1300.0 / stages), 600.0 + group_taps * ksteps * mma1);
             // stride 2: four phases per position, staged two at a time where the geometry allows (mx_prefetch_pair)
             const double per_position = s == 1 ? 1.0 : ((g.W & 1) == 0 && (g.pl & 1) == 0 && g.Cw <= 4) ? 2.0 : 3.0;
             const double load = 400.0 + 8.0 * per_position * (nt + (double)halo / T);
@@ -1319,11 +1340,11 @@ bool mx_plan_uncached(const ConvGeom &g, int sms, MxPlan *pl)
             if (cost < best) {
                 best = cost;
                 found = true;
-                pl->Nt = nt; pl->P = P; pl->T = T; pl->stages = stages; pl->resident = resident ? 1 : 0;
+                pl->Nt = nt; pl->P = P; pl->T = T; pl->stages = stages; pl->resident = resident ? 1 : 0; pl->group_taps = group_taps; pl->groups = groups;
                 pl->n_tiles = n_tiles; pl->n_super = n_super; pl->ctas_x = ctas_x;
                 pl->raw_words = raw_words; pl->x_bytes = x_bytes;
                 pl->off_w = off_w;
-                pl->off_x = (off_w + (size_t)stages * pl->tap_bytes + 127) / 128 * 128;
+                pl->off_x = (off_w + (size_t)stages * group_taps * pl->tap_bytes + 127) / 128 * 128;
                 // More position buffers where shared memory is left over (thin layers): the loaders may then be
                 // up to four tiles ahead, ahead <= (n_xbuf - 1) * T + 1, and the hand-overs between the roles
                 // (a few hundred clocks each) drop out of the per-tile cycle.
@@ -1440,7 +1461,7 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const void
     fast_div_constants((uint32_t)(pl.Nt + pl.halo), &p.c0_mul, &p.c0_sh);
     fast_div_constants((uint32_t)pl.Nt, &p.c1_mul, &p.c1_sh);
     p.Nt = pl.Nt; p.P = pl.P; p.T = pl.T; p.halo = pl.halo; p.n_tiles = pl.n_tiles; p.n_super = pl.n_super; p.total_q = pl.total_q;
-    p.taps = pl.taps; p.ksteps = pl.Cw2 / 2; p.stages = pl.stages; p.resident = pl.resident;
+    p.taps = pl.taps; p.ksteps = pl.Cw2 / 2; p.stages = pl.stages; p.resident = pl.resident; p.group_taps = pl.group_taps; p.groups = pl.groups;
     p.tap_bytes = (int32_t)pl.tap_bytes; p.raw_words = (int32_t)pl.raw_words; p.x_bytes = (int32_t)pl.x_bytes;
     p.n_xbuf = pl.n_xbuf; p.ahead = pl.ahead;
     p.off_w = (int32_t)pl.off_w; p.off_x = (int32_t)pl.off_x;

@@ -777,7 +777,7 @@ __device__ __forceinline__ void mx_epilogue_bits(const MxFin &f, uint32_t tmem_d
 // costs one multiply-add and one store instruction and nothing is staged.  The re-quantised copy is a
 // warp ballot of the signs: the finished word of the pixel.  Everything the loops need sits in
 // registers before they start (kernel parameters read inside them cost more than the arithmetic).
-enum { EPI_FLOAT = 0, EPI_FLOAT_FUSED = 1, EPI_INT32 = 2, EPI_BITS = 3 };
+enum { EPI_FLOAT = 0, EPI_FLOAT_FUSED = 1, EPI_INT32 = 2, EPI_BITS = 3, EPI_PLAIN = 4 };
 
 template <int MODE>
 __device__ __forceinline__ void mx_store_chunk(const float (&v)[32], int cols, const int32_t *sPixChunk, int64_t cout, float *outp,
@@ -882,8 +882,12 @@ __device__ __forceinline__ void mx_epilogue_fused(const MxFin &f, uint32_t tmem_
     }
 }
 
-// EPI: the output transform this instantiation carries (one kernel per form keeps each one's code, and
-// with it the instruction-cache footprint of four roles running side by side, small)
+// EPI: EPI_PLAIN carries the three plain output transforms (bit-packed, float, int32; chosen per launch by the
+// output type), EPI_FLOAT_FUSED the float transform with the shortcut add, the activation and the re-quantised
+// copy.  One instantiation for the plain forms matters more than their few KB of code: a network alternates
+// bit-packed and float layers, and two kernels of 160 KB alternating evict each other from the SMs' instruction
+// caches at every launch (config 2 as one flushed step: 103 us with a kernel per form, 87 us with one for all
+// three); the fused form stays apart because its register needs spoil the float form's code when they share one.
 template <int EPI>
 __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_constant__ MxParams p)
 {
@@ -1042,7 +1046,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         const int fw = warp - kLoaders / 32;  // 0..15: lane quarter fw & 3 (= warp & 3), column group fw >> 2
         const MxFin fin = mx_fin_context(p, fw, lane, ch0);
         asm volatile("griddepcontrol.wait;" ::: "memory");  // outputs and the shortcut tensor: only after the previous kernel
-        const int T = p.T, n_tiles = p.n_tiles, n_super = p.n_super;
+        const int T = p.T, n_tiles = p.n_tiles, n_super = p.n_super, out_type = p.out_type;
         uint32_t par_full_d[2] = {0, 0};
         int it = 0;
         for (int st = first_tile; st < n_super && ok; st += tile_step) {
@@ -1055,9 +1059,10 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + (buf ? kD1Col : 0u);
                 const int32_t *pix = sPix + (it & (kPixSlots - 1)) * kMaxNt;
-                if (EPI == EPI_BITS) mx_epilogue_bits(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
-                else if (EPI == EPI_FLOAT_FUSED) mx_epilogue_fused(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
-                else mx_epilogue_values<EPI>(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
+                if (EPI == EPI_FLOAT_FUSED) mx_epilogue_fused(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
+                else if (out_type == LCE_OUT_BITPACKED) mx_epilogue_bits(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
+                else if (out_type == LCE_OUT_INT32) mx_epilogue_values<EPI_INT32>(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
+                else mx_epilogue_values<EPI_FLOAT>(fin, tmem_d, pix, lane, &bars[BAR_EMPTY_D0 + buf]);
             }
         }
     } else if (warp == kIssuerWarp || (warp == kIssuerWarp + 1 && p.resident != 0)) {
@@ -1472,10 +1477,9 @@ lce_status launch_bconv_tensor(const ConvGeom &g, const uint32_t *in, const void
     p.dup_log2 = mx_dup(g) == 4 ? 2 : mx_dup(g) == 2 ? 1 : 0;
     if (!aligned(w_image, 16)) return LCE_ERR_ALIGNMENT;
     const dim3 grid((unsigned)pl.ctas_x, (unsigned)pl.n_blocks);
-    if (g.out_type == LCE_OUT_BITPACKED) return launch_mx<EPI_BITS>(p, grid, pl.smem, s);
-    if (g.out_type == LCE_OUT_INT32) return launch_mx<EPI_INT32>(p, grid, pl.smem, s);
-    if (residual || out_packed || !out || g.activation != LCE_ACT_NONE) return launch_mx<EPI_FLOAT_FUSED>(p, grid, pl.smem, s);
-    return launch_mx<EPI_FLOAT>(p, grid, pl.smem, s);
+    if (g.out_type == LCE_OUT_FLOAT32 && (residual || out_packed || !out || g.activation != LCE_ACT_NONE))
+        return launch_mx<EPI_FLOAT_FUSED>(p, grid, pl.smem, s);
+    return launch_mx<EPI_PLAIN>(p, grid, pl.smem, s);
 }
 
 

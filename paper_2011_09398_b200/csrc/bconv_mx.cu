@@ -80,9 +80,9 @@ constexpr int kOffSlot = 1000;       // TMEM base address; 1004 fills issued, 10
 // accumulator back before they have stored its values, so the loaders can be up to four tiles ahead
 // of a finisher that still reads its tile's slot (tile t + 5 cannot be staged before finisher t is done).
 constexpr int kOffPix = 1024;
-constexpr int kOffTbl = 8192;        // uint2[512]: operand offsets (A, B; 16-byte units) of the MMAs of a tile
-constexpr int kOffDyn = 12288;      // raw words, weight ring, position buffers
-constexpr int kMaxTblMmas = 512;
+constexpr int kOffTbl = 8192;        // uint2[1024]: operand offsets (A, B; 16-byte units) of the MMAs of a tile
+constexpr int kOffDyn = 16384;      // raw words, weight ring, position buffers
+constexpr int kMaxTblMmas = kMaxTaps * 16;                   // 64 taps x 16 K steps (in_c <= 1024): every shape the kernel covers
 
 enum { BAR_FULL_X0 = 0, BAR_FULL_X3 = 3, BAR_TILE_DONE0, BAR_TILE_DONE3 = BAR_TILE_DONE0 + 3, BAR_FULL_D0, BAR_FULL_D1, BAR_EMPTY_D0, BAR_EMPTY_D1, BAR_DONE, BAR_DONE_B,
        BAR_SCALES, BAR_FULL_W0,
@@ -407,9 +407,8 @@ __device__ __forceinline__ int mx_fast_words(const MxGeo &p)
     const bool words_ok = (p.Cw == 1) || (p.Cw == 2 && p.cp_words >= 2) || ((p.Cw == 4 || p.Cw == 8 || p.Cw == 16) && p.cp_words == 4);
     if (p.pad_zero || !words_ok) return 0;
     if (p.n_phase == 1) return p.Cw >= 2 ? p.Cw : 0;
-    if (p.Cw > 8) return 0;
     const bool pairs = (p.W & 1) == 0 && (p.pl & 1) == 0 && (reinterpret_cast<uintptr_t>(p.in) & 15) == 0 && p.Cw <= 4;
-    return (pairs ? 64 : 32) + p.Cw;
+    return pairs ? 64 + p.Cw : p.Cw == 8 ? 40 : 0;
 }
 
 __device__ __forceinline__ void mx_prefetch_any(int fw, const MxGeo &p, const MxChunk &c, uint32_t *raw, int ltid)
@@ -418,9 +417,6 @@ __device__ __forceinline__ void mx_prefetch_any(int fw, const MxGeo &p, const Mx
     else if (fw == 4) mx_prefetch_fast<4, 1>(p, c, raw, ltid);
     else if (fw == 8) mx_prefetch_fast<8, 1>(p, c, raw, ltid);
     else if (fw == 16) mx_prefetch_fast<16, 1>(p, c, raw, ltid);
-    else if (fw == 33) mx_prefetch_fast<1, 4>(p, c, raw, ltid);
-    else if (fw == 34) mx_prefetch_fast<2, 4>(p, c, raw, ltid);
-    else if (fw == 36) mx_prefetch_fast<4, 4>(p, c, raw, ltid);
     else if (fw == 40) mx_prefetch_fast<8, 4>(p, c, raw, ltid);
     else if (fw == 65) mx_prefetch_pair<1>(p, c, raw, ltid);
     else if (fw == 66) mx_prefetch_pair<2>(p, c, raw, ltid);
@@ -434,9 +430,6 @@ __device__ __forceinline__ void mx_expand_any(int fw, const MxGeo &p, const MxCh
     else if (fw == 4) mx_expand_fast<4, 1>(p, c, raw, X, ltid);
     else if (fw == 8) mx_expand_fast<8, 1>(p, c, raw, X, ltid);
     else if (fw == 16) mx_expand_fast<16, 1>(p, c, raw, X, ltid);
-    else if (fw == 33) mx_expand_fast<1, 4>(p, c, raw, X, ltid);
-    else if (fw == 34) mx_expand_fast<2, 4>(p, c, raw, X, ltid);
-    else if (fw == 36) mx_expand_fast<4, 4>(p, c, raw, X, ltid);
     else if (fw == 40) mx_expand_fast<8, 4>(p, c, raw, X, ltid);
     else if (fw == 65) mx_expand_pair<1>(p, c, raw, X, ltid);
     else if (fw == 66) mx_expand_pair<2>(p, c, raw, X, ltid);
@@ -457,38 +450,6 @@ __device__ __forceinline__ bool elect_one()
     uint32_t pred;
     asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
     return pred != 0;
-}
-
-// `count` MMAs of one tap by descriptor arithmetic, up to four per block of code (filters with more MMAs
-// per tile than the offset table holds).  Descriptor low words advance by additions, the high word
-// never changes.
-__device__ __forceinline__ void mx_issue(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t a_step, uint32_t b_step, int count,
-                                         uint32_t desc_hi, uint32_t idesc, uint32_t sfa, uint32_t sfb, uint32_t &accumulate)
-{
-    for (int i0 = 0; i0 < count; i0 += 4) {
-        const int n = count - i0;
-        const uint32_t a0 = a_lo + (uint32_t)i0 * a_step, b0 = b_lo + (uint32_t)i0 * b_step;
-        if (elect_one()) {
-            asm volatile(
-                "{\n\t.reg .pred pa, pt, g;\n\t.reg .b64 da, db;\n\t"
-                "setp.ne.b32 pa, %13, 0;\n\t"
-                "setp.eq.b32 pt, 0, 0;\n\t"
-                "mov.b64 da, {%1, %9};\n\t mov.b64 db, {%5, %9};\n\t"
-                "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %10, [%11], [%12], pa;\n\t"
-                "setp.gt.s32 g, %14, 1;\n\t mov.b64 da, {%2, %9};\n\t mov.b64 db, {%6, %9};\n\t"
-                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %10, [%11], [%12], pt;\n\t"
-                "setp.gt.s32 g, %14, 2;\n\t mov.b64 da, {%3, %9};\n\t mov.b64 db, {%7, %9};\n\t"
-                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %10, [%11], [%12], pt;\n\t"
-                "setp.gt.s32 g, %14, 3;\n\t mov.b64 da, {%4, %9};\n\t mov.b64 db, {%8, %9};\n\t"
-                "@g tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], da, db, %10, [%11], [%12], pt;\n\t"
-                "}"
-                :
-                : "r"(tmem_d), "r"(a0), "r"(a0 + a_step), "r"(a0 + 2 * a_step), "r"(a0 + 3 * a_step), "r"(b0), "r"(b0 + b_step),
-                  "r"(b0 + 2 * b_step), "r"(b0 + 3 * b_step), "r"(desc_hi), "r"(idesc), "r"(sfa), "r"(sfb), "r"(accumulate), "r"(n)
-                : "memory");
-        }
-        accumulate = 1;
-    }
 }
 
 // N MMAs straight from a table of operand offsets, back to back in one block of code: the loads of the
@@ -912,7 +873,6 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
     // barriers and starts the weight copies, the finisher warps fill the table of operand offsets, the
     // loaders fetch the first chunk of activations ---------------------------------------------------------
     const int n_mma = p.taps * p.ksteps;
-    const bool use_table = n_mma <= kMaxTblMmas;
     // the weight producer's progress (one thread): fills issued, ring stage and (tile-local) tap group of the next one
     int prod_g = 0, prod_total = 0, prod_stage = 0, prod_tap = 0;
     uint32_t prod_parity = 1;  // the first pass over the ring waits for nothing
@@ -956,7 +916,7 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
             fills[0] = prod_g;
             fills[1] = 0;
         }
-    } else if (tid >= kLoaders && use_table) {
+    } else if (tid >= kLoaders) {
         for (int e = tid - kLoaders; e < n_mma; e += kFinishers) {
             const int tap = e / p.ksteps, kk = e - tap * p.ksteps;
             const int ky = tap / p.KW, kx = tap - ky * p.KW;
@@ -979,7 +939,13 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         ld.c0_mul = p.c0_mul; ld.c0_sh = p.c0_sh; ld.c1_mul = p.c1_mul; ld.c1_sh = p.c1_sh;
         ld.fast_words = mx_fast_words(geo);
         asm volatile("griddepcontrol.wait;" ::: "memory");  // the activations may come from the previous kernel
-        if (first_tile < ld.n_super) mx_prefetch_any(ld.fast_words, geo, mx_chunk_of(ld, first_tile * ld.T * ld.Nt, 0), raw0, tid);
+        if (first_tile < ld.n_super) {
+            // through the general form where its staging layout is the fast form's too (all but the paired stride-2
+            // form): one more inlined copy of every fast form costs more in code size than it saves here
+            const MxChunk c0 = mx_chunk_of(ld, first_tile * ld.T * ld.Nt, 0);
+            if (ld.fast_words >= 64) mx_prefetch_any(ld.fast_words, geo, c0, raw0, tid);
+            else mx_prefetch(geo, c0, raw0, tid);
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -1078,12 +1044,11 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
         // group stride (128 bytes) | version 1 at bit 46; no swizzle
         const uint32_t desc_hi = 8u | (1u << 14);
         // everything the loops use, read from the kernel parameters once
-        const int T = p.T, n_tiles = p.n_tiles, n_super = p.n_super, Nt = p.Nt, KH = p.KH, KW = p.KW, ksteps = p.ksteps, stages = p.stages, taps = p.taps, group_taps = p.group_taps;
+        const int T = p.T, n_tiles = p.n_tiles, n_super = p.n_super, Nt = p.Nt, ksteps = p.ksteps, stages = p.stages, taps = p.taps, group_taps = p.group_taps;
         const bool resident = p.resident != 0;
-        const bool by_table = use_table && (resident || (ksteps & 3) != 0);  // streamed taps: blocks of four by arithmetic waste nothing when 4 | K steps
         const uint32_t w_lo0 = ((uint32_t)p.off_w >> 4) + (smem_u32(smem) >> 4) + (128u << 16);
         const uint32_t x_lo_buf0 = ((uint32_t)p.off_x >> 4) + (smem_u32(smem) >> 4) + ((uint32_t)p.P << 16);
-        const uint32_t x_units = (uint32_t)p.x_bytes >> 4, tap_units = (uint32_t)p.tap_bytes >> 4, b_kstep = 2u * (uint32_t)p.P;
+        const uint32_t x_units = (uint32_t)p.x_bytes >> 4, tap_units = (uint32_t)p.tap_bytes >> 4;
         const uint32_t group_units = tap_units * (uint32_t)p.group_taps;
         const uint32_t sfa = tmem_base + kSfaCol, sfb = tmem_base + kSfbCol;
         uint32_t par_empty_d[2] = {0, 0};
@@ -1118,19 +1083,12 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                     if (lane == 0) fills[1] = 1;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 }
-                if (by_table) {
-                    mx_issue_table(tmem_d, tbl, n_mma, w_lo0, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
-                } else {
-                    uint32_t a_tap = w_lo0;
-                    for (int ky = 0; ky < KH; ++ky)
-                        for (int kx = 0; kx < KW; ++kx, a_tap += tap_units)
-                            mx_issue(tmem_d, a_tap, x_lo0 + tap_b_offset(p, ky, kx), 256u, b_kstep, ksteps, desc_hi, idesc, sfa, sfb, accumulate);
-                }
+                mx_issue_table(tmem_d, tbl, n_mma, w_lo0, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
             } else {
                 // the taps stream through the ring a group at a time: wait for the group, issue its taps' MMAs,
                 // hand its stage back (the wait, the commit and the bookkeeping cost this warp about 600 clocks,
                 // as much as six MMAs: hence groups, not single taps)
-                int tap = 0, ky = 0, kx = 0;
+                int tap = 0;
                 while (tap < taps) {
                     ok = __all_sync(0xffffffffu, mbar_wait_bounded(&bars[BAR_FULL_W0 + stage_i], w_parity));
                     if (!ok) break;
@@ -1139,11 +1097,8 @@ __global__ void __launch_bounds__(kMxThreads, 1) bconv_mx_kernel(const __grid_co
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     uint32_t a_tap = w_lo0 + (uint32_t)stage_i * group_units;
                     const int group_end = min(taps, tap + group_taps);
-                    for (; tap < group_end; ++tap, a_tap += tap_units) {
-                        if (by_table) mx_issue_table(tmem_d, tbl + tap * ksteps, ksteps, a_tap, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
-                        else mx_issue(tmem_d, a_tap, x_lo0 + tap_b_offset(p, ky, kx), 256u, b_kstep, ksteps, desc_hi, idesc, sfa, sfb, accumulate);
-                        if (++kx == KW) { kx = 0; ++ky; }
-                    }
+                    for (; tap < group_end; ++tap, a_tap += tap_units)
+                        mx_issue_table(tmem_d, tbl + tap * ksteps, ksteps, a_tap, x_lo0, desc_hi, idesc, sfa, sfb, accumulate);
                     if (elect_one()) mma_commit(&bars[BAR_EMPTY_W0 + stage_i]);
                     if (++stage_i == stages) { stage_i = 0; w_parity ^= 1u; }
                 }

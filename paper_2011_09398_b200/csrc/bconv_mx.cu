@@ -1269,15 +1269,15 @@ bool mx_plan_uncached(const ConvGeom &g, int sms, MxPlan *pl)
             const size_t rest = 2 * x_bytes + 256;
             if (off_w + rest + (taps > 1 ? 2 : 1) * pl->tap_bytes > kSmemLimit) break;
             // taps that fit beside the position buffers: all of them -> resident (one stage per tap, one barrier);
-            // otherwise a ring of about three stages of several taps each (a group costs the issuer one wait and
-            // one commit, whatever its size)
+            // otherwise a ring of two stages of half the fitting taps each (a group costs the issuer one wait and
+            // one commit, whatever its size: two large groups measured better than three or four smaller ones)
             const int slots = (int)((kSmemLimit - off_w - rest) / pl->tap_bytes);
             const bool resident = slots >= taps;
             int stages, group_taps, groups;
             if (resident) {
                 stages = taps; group_taps = 1; groups = taps;
             } else {
-                group_taps = slots >= 6 ? slots / 3 : 1;
+                group_taps = slots >= 4 ? slots / 2 : 1;
                 groups = (taps + group_taps - 1) / group_taps;
                 group_taps = (taps + groups - 1) / groups;  // even groups
                 stages = min(kMaxStages, slots / group_taps);

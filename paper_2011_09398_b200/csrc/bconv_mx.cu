@@ -30,8 +30,9 @@
 //     operand image [channel block][tap][channel word][128 channels][16 bytes] (for out_c <= 64 the
 //     channel block is repeated down the 128 rows, so that every TMEM lane quarter holds values a
 //     finisher warp can work on); the bulk-copy engine brings taps into a ring of shared-memory stages
-//     (cp.async.bulk + mbarrier transaction count).  If the ring holds every tap they are fetched once
-//     per CTA, all counted on one barrier; otherwise they stream past once per tile.
+//     (cp.async.bulk + mbarrier transaction count).  If every tap fits they are fetched once per CTA,
+//     all counted on one barrier; otherwise they stream past once per tile, in groups of taps that
+//     alternate between two stages (one copy, one wait and one commit per group).
 //   * roles: 8 loader warps (prefetch the packed words of the next chunk with cp.async, expand the
 //     current one), one warp that issues the MMAs (all lanes run the same code, the elected lane
 //     issues), one warp that feeds the weight ring and, once the weights are resident, issues the MMAs

@@ -117,8 +117,12 @@ lce_status lce_bconv2d_out_shape(const lce_bconv2d_desc *desc, int32_t *out_h, i
  * lce_bconv2d_pack_weights (the fast path: nothing is derived from the weights per call).
  * Pad bits of input and weights must be 0.  The float / int32 fast paths want `output` 16-byte
  * aligned (out_c a multiple of 4); a buffer that is only 4-byte aligned is served by the direct kernel
- * under AUTO.  The weights and per-channel arrays are constants of the model: they must not be written
- * by work that is still running on the stream when this call is made.  Errors: INVALID_ARG
+ * under AUTO.  The weights and per-channel arrays are constants of the model: the kernels read them
+ * before they wait for the stream's previous kernel where that kernel lets its dependents start early
+ * (programmatic dependent launch; this library's convolution kernels do), so they must not be the
+ * output of such a kernel that may still be running.  What lce_bconv2d_pack_weights, a copy or an
+ * ordinary kernel wrote earlier on the stream is complete before this call's kernel is scheduled.
+ * Errors: INVALID_ARG
  * (null/extent/enum/missing per-channel array), ALIGNMENT, UNSUPPORTED (a forced kernel does not cover
  * the shape), CUDA, DEVICE_TIMEOUT (see lce_device_status; nothing is launched). */
 lce_status lce_bconv2d(const lce_bconv2d_desc *desc, const uint32_t *input, const uint32_t *weights,

@@ -457,6 +457,9 @@ def run_lce(args):
         "frac_bitpacked_launches": rate(us_auto, bit) / tensor_peak, "frac_float_launches": rate(us_auto, flt) / tensor_peak,
         "traffic": profiled_traffic("bconv_mx_kernel"),
         "hbm_bound_us": hbm_bound_us,
+        # the float launches alone (their outputs are what moves): per launch, and as a fraction of their measured time
+        "hbm_bound_us_float_launches": [layers[j]["spec"].algorithmic_bytes / peak_hbm_bytes_per_s() * 1e6 for j in flt],
+        "hbm_frac_float_launches": sum(layers[j]["spec"].algorithmic_bytes for j in flt) / peak_hbm_bytes_per_s() * 1e6 / sum(us_auto[j] for j in flt),
     }
     # integer path (the pipe the benchmark spec names): ceiling = the best measured register-resident
     # instruction mix (probe run in this process), the derived figure beside it

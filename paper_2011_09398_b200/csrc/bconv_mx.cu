@@ -1290,10 +1290,11 @@ bool mx_plan_uncached(const ConvGeom &g, int sms, MxPlan *pl)
             // position and tile
             const double mma1 = fmax(100.0, 43.0 + nt / 2.0);
             const double mma = (double)taps * ksteps * mma1;
-            // a streamed tap: its bytes from L2, or its share of a copy's latency, or what the single issuer needs
+            // a streamed tap: its bytes from L2 (every SM streams at once: the L2 gives each about 19 bytes per clock,
+            // 5.5 TB/s in all), or its share of a copy's latency, or what the single issuer needs
             // per tap (wait for the stage, issue, hand the stage back: about 600 clocks on top of the MMAs;
             // measured on a nine-tap, one-MMA-per-tap layer: 6000 clocks per tile whether 2 or 4 stages)
-            const double stream = resident ? 0.0 : (double)groups * fmax(fmax(group_taps * pl->tap_bytes / 48.0, 1300.0 / stages), 600.0 + group_taps * ksteps * mma1);
+            const double stream = resident ? 0.0 : (double)groups * fmax(fmax(group_taps * pl->tap_bytes / 19.0, 1300.0 / stages), 600.0 + group_taps * ksteps * mma1);
             // stride 2: four phases per position, staged two at a time where the geometry allows (mx_prefetch_pair)
             const double per_position = s == 1 ? 1.0 : ((g.W & 1) == 0 && (g.pl & 1) == 0 && g.Cw <= 4) ? 2.0 : 3.0;
             const double load = 400.0 + 8.0 * per_position * (nt + (double)halo / T);

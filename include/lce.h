@@ -165,8 +165,9 @@ lce_status lce_bconv2d_f32(const lce_bconv2d_desc *desc, const float *input, con
  *   kernel              LCE_KERNEL_DIRECT, LCE_KERNEL_TILED or LCE_KERNEL_TENSOR (the one-word patch
  *                       kernel for very few input channels reports LCE_KERNEL_TILED with patch = 1).
  *                       For LCE_KERNEL_TENSOR: tile_pixels = grid positions per tile, ctas, shared_bytes,
- *                       weight_stages = taps the shared-memory weight ring holds, weights_resident = 1
- *                       when that is every tap (fetched once per CTA instead of once per tile)
+ *                       weights_resident = 1 when every tap of a channel block stays in shared memory
+ *                       (fetched once per CTA; weight_stages = taps), 0 when they stream past once per
+ *                       tile (weight_stages = stages of the ring, each a group of consecutive taps)
  *   pointwise           1 for the 1x1 tiled kernel
  *   warps_per_cta, pixels_per_thread, tile_pixels, shared_bytes      the variant of the tiled kernel
  *   ctas                CTAs of the launch; ctas_half_block of them work on the last, at most

@@ -792,33 +792,42 @@ __device__ __forceinline__ void mx_epilogue_values(const MxFin &f, uint32_t tmem
 // 32 independent 128-byte loads in flight per warp; with eight the memory latency set the pace), then reads
 // the accumulators 16 columns at a time, and per position does the multiply-add, the add, the 128-byte store
 // and the ballot whose result is the pixel's finished word.
-__device__ __forceinline__ void mx_epilogue_fused(const MxFin &f, uint32_t tmem_d, const int32_t *sPix, int lane, uint64_t *empty_d)
+template <bool RES, bool PACK, bool WRITE_FLOAT>
+__device__ __forceinline__ void mx_epilogue_fused_as(const MxFin &f, uint32_t tmem_d, const int32_t *sPix, int lane, uint64_t *empty_d)
 {
+    // which of the three parts (shortcut add, re-quantised copy, float output) a launch has is a template
+    // argument: a test of a pointer per position turns the unrolled block below into branchy code that
+    // runs at a third of the speed (measured on the plain float transform, and again here)
     const float floor_v = f.relu ? 0.f : -INFINITY;
     for (int ck = f.group; ck <= f.last_chunk; ck += f.n_groups) {
         const int c0 = ck * 32;
         const int cols = min(32, f.Nt - c0);  // 32, or 16 in a tile's last chunk
         const int32_t *pixc = sPix + c0;
-        float r[32];
-#pragma unroll
-        for (int j4 = 0; j4 < 32; j4 += 4) {
-            const int4 p4 = *reinterpret_cast<const int4 *>(pixc + j4);  // the same for every lane
-            const int pix[4] = {p4.x, p4.y, p4.z, p4.w};
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                r[j4 + u] = 0.f;
-                if (f.resp != nullptr && f.ch_ok && pix[u] >= 0 && j4 + u < cols) r[j4 + u] = __ldg(f.resp + pix[u] * f.cout);
-            }
-        }
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             if (half * 16 < cols) {
+                // the shortcut values of the half's 16 positions first (they do not depend on the accumulator: 16
+                // independent 128-byte loads in flight per warp), then the accumulators
+                float r[16];
+                if (RES) {
+#pragma unroll
+                    for (int j4 = 0; j4 < 16; j4 += 4) {
+                        const int4 p4 = *reinterpret_cast<const int4 *>(pixc + half * 16 + j4);  // the same for every lane
+                        const int pix[4] = {p4.x, p4.y, p4.z, p4.w};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const bool ld = f.ch_ok && pix[u] >= 0 && half * 16 + j4 + u < cols;
+                            r[j4 + u] = ld ? __ldg(f.resp + (ld ? pix[u] : 0) * f.cout) : 0.f;
+                        }
+                    }
+                }
                 float v[16];
                 tmem_ld16x(tmem_d + f.lane_off + (uint32_t)(c0 + half * 16), v);
                 if (ck == f.last_chunk && (half + 1) * 16 >= cols) {  // last read of the accumulator by this warp
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                     mbar_arrive(empty_d);
                 }
+                uint32_t my_word = 0u;  // lane u keeps the re-quantised word of the half's position u: one store for the 16
 #pragma unroll
                 for (int j4 = 0; j4 < 16; j4 += 4) {
                     const int4 p4 = *reinterpret_cast<const int4 *>(pixc + half * 16 + j4);
@@ -827,13 +836,20 @@ __device__ __forceinline__ void mx_epilogue_fused(const MxFin &f, uint32_t tmem_
                     for (int u = 0; u < 4; ++u) {
                         const bool pos_ok = pix[u] >= 0 && half * 16 + j4 + u < cols;  // the same for every lane
                         float y = __fmaf_rn(fmaxf(v[j4 + u], floor_v), f.mult, f.bias);
-                        if (f.resp != nullptr) y = __fadd_rn(y, r[half * 16 + j4 + u]);
-                        if (f.write_float && f.ch_ok && pos_ok) f.outp[pix[u] * f.cout] = y;
-                        if (f.packp != nullptr) {
+                        if (RES) y = __fadd_rn(y, r[j4 + u]);
+                        if (WRITE_FLOAT) {
+                            if (f.ch_ok && pos_ok) f.outp[pix[u] * f.cout] = y;
+                        }
+                        if (PACK) {
                             const uint32_t word = __ballot_sync(0xffffffffu, f.ch_ok && y < 0.f);
-                            if (lane == 0 && pos_ok) f.packp[pix[u] * f.cow] = word;
+                            if (lane == j4 + u) my_word = word;
                         }
                     }
+                }
+                if (PACK) {
+                    const int my_pos = half * 16 + (lane & 15);
+                    const int my_pix = pixc[my_pos];
+                    if (lane < 16 && my_pix >= 0 && my_pos < cols) f.packp[my_pix * f.cow] = my_word;
                 }
             }
         }
@@ -841,6 +857,20 @@ __device__ __forceinline__ void mx_epilogue_fused(const MxFin &f, uint32_t tmem_
     if (f.last_chunk < 0) {  // nothing to read for this warp
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         mbar_arrive(empty_d);
+    }
+}
+
+__device__ __forceinline__ void mx_epilogue_fused(const MxFin &f, uint32_t tmem_d, const int32_t *sPix, int lane, uint64_t *empty_d)
+{
+    const int form = (f.resp != nullptr ? 4 : 0) | (f.packp != nullptr ? 2 : 0) | (f.write_float ? 1 : 0);
+    switch (form) {
+        case 1: mx_epilogue_fused_as<false, false, true>(f, tmem_d, sPix, lane, empty_d); break;
+        case 2: mx_epilogue_fused_as<false, true, false>(f, tmem_d, sPix, lane, empty_d); break;
+        case 3: mx_epilogue_fused_as<false, true, true>(f, tmem_d, sPix, lane, empty_d); break;
+        case 5: mx_epilogue_fused_as<true, false, true>(f, tmem_d, sPix, lane, empty_d); break;
+        case 6: mx_epilogue_fused_as<true, true, false>(f, tmem_d, sPix, lane, empty_d); break;
+        case 7: mx_epilogue_fused_as<true, true, true>(f, tmem_d, sPix, lane, empty_d); break;
+        default: mx_epilogue_fused_as<false, false, false>(f, tmem_d, sPix, lane, empty_d); break;  // nothing to write: only hands the accumulator back
     }
 }
 
